@@ -1,0 +1,204 @@
+/*
+ * q4 -- 4-bit quantized GEMM and GEMM-based convolution for NVIDIA B200 (sm_100a).
+ *
+ * C ABI of the CUDA library.  The operations are those of the paper "Fast
+ * Implementation of 4-bit Convolutional Neural Networks for Mobile Devices"
+ * (arXiv 2009.06488): the widening product of two matrices of unsigned 4-bit
+ * values with per-tensor zero points (Section II-B, Eq. 2), kept as an integer
+ * result (Section III-A, Eq. 3) and handed to the next layer as 4-bit values
+ * again, and the convolution that reduces to it by unrolling the input
+ * (Section I; depth D = kh*kw*c, Section III-A).
+ *
+ * Naming.  C = A x B with A = activations (M x K, one row per output pixel) and
+ * B = weights (K x N, one column per output channel).  The paper writes R = W X
+ * with the weights on the left; C = R^T, za = z_x, zb = z_w, K = D,
+ * rowsum_a[m] = sum_k x^_{kj} (the second term's sum) and colsum_b[n] =
+ * sum_k w^_{ik} (the third term's sum, computed once per weight matrix).
+ *
+ * Data layout.  A uint4 array is a flat nibble array: element e lives in byte
+ * e >> 1, in the low nibble when e is even.  Both GEMM operands are
+ * K-contiguous: A is M rows of K nibbles with a row pitch of lda bytes, Bt
+ * (= B transposed) is N rows of K nibbles with a row pitch of ldb bytes.  Bytes of
+ * a row past ceil(K/2) are never read.  When K is odd the high nibble of a row's
+ * last byte must be 0 (q4_im2col and q4_pack_bt write it so).  int32 matrices are
+ * row-major with a pitch in elements; packed uint4 outputs are row-major along n
+ * with a pitch in bytes, and need an even N.
+ *
+ * Pointers.  Every data pointer is a DEVICE pointer owned by the caller; the
+ * library allocates nothing and keeps no buffers.  q4_requant and q4_conv_desc are
+ * small HOST structs read during the call.  `stream` is a cudaStream_t passed as
+ * void* (NULL = the legacy default stream).  Work is enqueued on that stream and
+ * the call returns without synchronizing.  The q4_*_host entry points are the
+ * exception: their data pointers are HOST pointers (see below).
+ *
+ * Errors.  Arguments are validated on the host before anything is launched; a
+ * q4_status is returned and nothing traps or aborts.  Device-side waits are
+ * bounded: a wait that expires sets a status word that q4_last_device_status
+ * reports.
+ *
+ * Fast path.  Base pointers aligned to 16 bytes and lda / ldb multiples of 16 bytes
+ * select the tensor-core kernels (TMA needs both); anything else runs a slower
+ * general kernel with the same results.
+ */
+#ifndef Q4_H
+#define Q4_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    Q4_OK = 0,
+    Q4_ERR_INVALID_ARG = 1,     /* NULL pointer, negative size, pitch smaller than a row   */
+    Q4_ERR_ALIGNMENT = 2,       /* a pointer / pitch breaks an alignment the call requires */
+    Q4_ERR_RANGE = 3,           /* zero point, multiplier, shift, clamp or K out of range  */
+    Q4_ERR_WORKSPACE = 4,       /* workspace missing or smaller than *_workspace_bytes     */
+    Q4_ERR_UNSUPPORTED = 5,     /* valid but not implemented (none at present)             */
+    Q4_ERR_CUDA = 6,            /* a CUDA runtime / driver call failed                     */
+    Q4_ERR_DEVICE_TIMEOUT = 7   /* a bounded device-side wait expired                      */
+} q4_status;
+
+/* Integer re-quantization of an int32 accumulator to the next layer's uint4 input.
+ * The paper re-quantizes each layer's integer result to 4 bits for the next layer
+ * (Section III-A/B) in floating point; here it is the fixed-point form
+ *     q = floor((acc * mult + 2^(30+shift)) / 2^(31+shift))        (one rounding,
+ *     y = min(max(q + zo, clamp_lo), clamp_hi)                      ties toward +inf)
+ * i.e. the real multiplier is mult / 2^(31+shift).  This is deliberately a single
+ * rounding, not a rounding high-multiply followed by a rounding shift.
+ * ReLU is clamp_lo = zo. */
+typedef struct {
+    int32_t mult;       /* [2^30, 2^31) */
+    int32_t shift;      /* 0..31        */
+    int32_t zo;         /* 0..15        */
+    int32_t clamp_lo;   /* 0 <= clamp_lo <= clamp_hi <= 15 */
+    int32_t clamp_hi;
+} q4_requant;
+
+/* Convolution geometry: NHWC input, OC filters of KH x KW x C, dilation 1, groups 1.
+ * Output extent per axis: floor((in + 2*pad - k) / stride) + 1.  Taps outside the
+ * image read the input zero point za, so they contribute exactly 0. */
+typedef struct {
+    int32_t N, H, W, C;
+    int32_t OC, KH, KW;
+    int32_t stride_h, stride_w;
+    int32_t pad_h, pad_w;
+} q4_conv_desc;
+
+/* Largest supported depth: every term of Eq. 2 (each at most 225*K) and their
+ * partial sums stay inside int32. */
+#define Q4_MAX_K (1 << 22)
+
+/*
+ * Quantized product, Eq. 2 / Eq. 3 without the float scales:
+ *   C[m][n] = sum_k (a(m,k) - za) * (b(k,n) - zb)
+ *           = sum_k a b  -  zb * rowsum_a[m]  -  za * colsum_b[n]  +  K * za * zb.
+ * A [M x K] pitch lda bytes; Bt [N x K] pitch ldb bytes; C [M x N] int32, pitch ldc
+ * elements (>= N).  za, zb in 0..15.  1 <= K <= Q4_MAX_K.  M or N = 0 is a no-op.
+ * rowsum_a [M] / colsum_b [N]: optional precomputed sums (e.g. from q4_im2col, or
+ * computed once for the weights); NULL = computed inside the kernel.
+ * ws / ws_bytes: workspace of at least q4_gemm_workspace_bytes(M, N, K) bytes
+ * (may be NULL when that is 0).
+ */
+q4_status q4_gemm(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                  int32_t* C, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                  int32_t za, int32_t zb,
+                  const int32_t* rowsum_a, const int32_t* colsum_b,
+                  void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Same product with the next layer's re-quantization fused into the epilogue
+ * (Section III-A: the integer result goes through the activation and is quantized
+ * to 4 bits again for the next layer):
+ *   Cq[m][n] = requant(C[m][n] + bias[n])       (see q4_requant)
+ * bias [N] int32 or NULL.  C[m][n] + bias[n] must fit in int32.  N must be even.
+ * Cq is packed along n, pitch ldcq bytes (>= N/2).  The int32 matrix is never
+ * written to memory.
+ */
+q4_status q4_gemm_requant(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                          int32_t M, int32_t N, int32_t K, int32_t za, int32_t zb,
+                          const int32_t* rowsum_a, const int32_t* colsum_b,
+                          const int32_t* bias, const q4_requant* rq,
+                          uint8_t* Cq, int64_t ldcq,
+                          void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Unrolling of a convolution input into the activation matrix of the GEMM
+ * (Section I; Section III-A):
+ *   A[(n,oh,ow)][(kh,kw,c)] = X[n, oh*stride_h - pad_h + kh, ow*stride_w - pad_w + kw, c]
+ * or za where that tap is outside the image.  X is the flat packed NHWC array (no
+ * pitches).  A has M = N*OH*OW rows of K = KH*KW*C nibbles, pitch lda bytes
+ * (>= ceil(K/2)); every nibble from K to the end of the pitch is written 0.
+ * rowsum_a [M] (optional): sum_k A[m][k], the second term's sums of Eq. 2, taken
+ * while unrolling as Section II-B suggests.  d->OC is ignored.
+ */
+q4_status q4_im2col(const uint8_t* X, const q4_conv_desc* d, int32_t za,
+                    uint8_t* A, int64_t lda, int32_t* rowsum_a, void* stream);
+
+/*
+ * One quantized convolution layer (Section III-A/B): unroll, multiply (Eq. 3), add
+ * bias, re-quantize.  Wt: filters [OC][KH][KW][C] packed along (kh,kw,c), pitch ldw
+ * bytes -- this is Bt of the GEMM.  colsum_w [OC]: optional precomputed
+ * sum_{kh,kw,c} w (the third term's sums), NULL = computed.  Y: packed NHWC output
+ * N x OH x OW x OC (flat, row pitch OC/2 bytes; OC even).
+ * ws: at least q4_conv2d_workspace_bytes(d) bytes, 256-byte aligned.
+ */
+q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
+                    const int32_t* colsum_w, const int32_t* bias,
+                    const q4_conv_desc* d, int32_t za, int32_t zb, const q4_requant* rq,
+                    uint8_t* Y, void* ws, size_t ws_bytes, void* stream);
+
+size_t q4_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
+size_t q4_conv2d_workspace_bytes(const q4_conv_desc* d);
+
+/*
+ * Weight preparation, done once per weight matrix (Section II-B): a K x N matrix
+ * packed along n (row k, pitch ldb_kn bytes) is rewritten as Bt, N x K packed along
+ * k (pitch ldb bytes, pad nibbles 0).
+ */
+q4_status q4_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int64_t ldb,
+                     int32_t K, int32_t N, void* stream);
+
+/* Sums over the depth of a packed matrix: sums[r] = sum_k P[r][k] (the sums of
+ * Eq. 2's second and third terms), for callers that want them precomputed. */
+q4_status q4_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
+                      int32_t* sums, void* stream);
+
+/*
+ * q4_gemm with HOST operands: copies A and Bt to the device, runs q4_gemm and
+ * copies C back, all on `stream`, then synchronizes it.  hA / hBt / hC are host
+ * pointers with the same pitches as above (pinned memory makes the copies
+ * asynchronous).  dev_staging is a DEVICE buffer owned by the caller of at least
+ * q4_gemm_host_staging_bytes(...) bytes, 256-byte aligned; it holds the device
+ * copies, so this entry point allocates nothing either.
+ */
+q4_status q4_gemm_host(const uint8_t* hA, int64_t lda, const uint8_t* hBt, int64_t ldb,
+                       int32_t* hC, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                       int32_t za, int32_t zb,
+                       void* dev_staging, size_t dev_staging_bytes, void* stream);
+size_t q4_gemm_host_staging_bytes(int32_t M, int32_t N, int32_t K,
+                                  int64_t lda, int64_t ldb, int64_t ldc);
+
+/* Synchronizes `stream`, then returns Q4_ERR_DEVICE_TIMEOUT if any kernel of this
+ * library gave up a bounded wait on the current device since the last call (the
+ * flag is cleared), Q4_ERR_CUDA if the stream reports an error, else Q4_OK. */
+q4_status q4_last_device_status(void* stream);
+
+/* Kernel selection for ablations and tests: 0 = automatic, 1 = general (SIMT)
+ * kernels only, 2 = tensor-core kernels wherever their alignment rules hold.
+ * Returns the previous value.  Process-wide; also read once from the environment
+ * variable Q4_FORCE_VARIANT ("simt" / "tc"). */
+int q4_set_variant(int variant);
+
+/* Number of kernels this library has launched in this process (all streams). */
+uint64_t q4_launch_count(void);
+
+const char* q4_status_string(q4_status s);
+int q4_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,306 @@
+// C ABI of the q4 library (declared in q4.h): argument validation, kernel selection,
+// launch.  No allocation, no synchronization except where the header says so.
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+
+#include "q4_common.cuh"
+
+namespace q4 {
+
+__device__ unsigned g_status_word = 0;
+
+static std::atomic<uint64_t> g_launches{0};
+static std::atomic<int> g_variant{-1};   // -1 = not read from the environment yet
+
+void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+static int variant()
+{
+    int v = g_variant.load(std::memory_order_relaxed);
+    if (v < 0) {
+        const char* e = std::getenv("Q4_FORCE_VARIANT");
+        v = 0;
+        if (e && !std::strcmp(e, "simt")) v = 1;
+        if (e && !std::strcmp(e, "tc")) v = 2;
+        g_variant.store(v, std::memory_order_relaxed);
+    }
+    return v;
+}
+
+static unsigned* status_ptr()
+{
+    // one address per device; looked up on first use with that device current
+    static unsigned* ptrs[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_status_word) != cudaSuccess) return nullptr;
+        ptrs[dev] = static_cast<unsigned*>(p);
+    }
+    return ptrs[dev];
+}
+
+static q4_status check_gemm(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                            int32_t M, int32_t N, int32_t K, int32_t za, int32_t zb)
+{
+    if (M < 0 || N < 0 || K < 1) return Q4_ERR_INVALID_ARG;
+    if (K > Q4_MAX_K) return Q4_ERR_RANGE;
+    if ((M > 0 && !A) || (N > 0 && !Bt)) return Q4_ERR_INVALID_ARG;
+    const int64_t kbytes = (K + 1) / 2;
+    if (lda < kbytes || ldb < kbytes) return Q4_ERR_INVALID_ARG;
+    if (za < 0 || za > 15 || zb < 0 || zb > 15) return Q4_ERR_RANGE;
+    return Q4_OK;
+}
+
+static q4_status check_requant(const q4_requant* rq)
+{
+    if (!rq) return Q4_ERR_INVALID_ARG;
+    if (rq->mult < (1 << 30)) return Q4_ERR_RANGE;
+    if (rq->shift < 0 || rq->shift > 31) return Q4_ERR_RANGE;
+    if (rq->zo < 0 || rq->zo > 15) return Q4_ERR_RANGE;
+    if (rq->clamp_lo < 0 || rq->clamp_hi > 15 || rq->clamp_lo > rq->clamp_hi) return Q4_ERR_RANGE;
+    return Q4_OK;
+}
+
+static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st)
+{
+    p.status = status_ptr();
+    if (!p.status) return Q4_ERR_CUDA;
+    const int v = variant();
+    if (v != 1 && gemm_tc_supported(p)) return launch_gemm_tc(p, rq, st);
+    if (v == 2) return Q4_ERR_ALIGNMENT;
+    return launch_gemm_simt(p, rq, st) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
+static q4_status check_conv(const q4_conv_desc* d, int32_t za)
+{
+    if (!d) return Q4_ERR_INVALID_ARG;
+    if (d->N < 0 || d->H < 1 || d->W < 1 || d->C < 1) return Q4_ERR_INVALID_ARG;
+    if (d->KH < 1 || d->KW < 1) return Q4_ERR_INVALID_ARG;
+    if (d->stride_h < 1 || d->stride_w < 1 || d->pad_h < 0 || d->pad_w < 0) return Q4_ERR_INVALID_ARG;
+    if (d->H + 2 * d->pad_h < d->KH || d->W + 2 * d->pad_w < d->KW) return Q4_ERR_INVALID_ARG;
+    const int64_t K = (int64_t)d->KH * d->KW * d->C;
+    if (K > Q4_MAX_K) return Q4_ERR_RANGE;
+    const int64_t OH = (d->H + 2 * d->pad_h - d->KH) / d->stride_h + 1;
+    const int64_t OW = (d->W + 2 * d->pad_w - d->KW) / d->stride_w + 1;
+    if ((int64_t)d->N * OH * OW > INT32_MAX) return Q4_ERR_RANGE;
+    if (za < 0 || za > 15) return Q4_ERR_RANGE;
+    return Q4_OK;
+}
+
+struct ConvShape { int64_t M; int32_t K; int64_t lda; size_t off_rowsum, bytes; };
+
+// Workspace of q4_conv2d: the unrolled matrix (pitch rounded up to 16 bytes so the
+// tensor-core path applies) followed by its row sums.
+static ConvShape conv_shape(const q4_conv_desc* d)
+{
+    ConvShape s;
+    const int64_t OH = (d->H + 2 * d->pad_h - d->KH) / d->stride_h + 1;
+    const int64_t OW = (d->W + 2 * d->pad_w - d->KW) / d->stride_w + 1;
+    s.M = (int64_t)d->N * OH * OW;
+    s.K = d->KH * d->KW * d->C;
+    s.lda = (((int64_t)s.K + 1) / 2 + 15) / 16 * 16;
+    s.off_rowsum = ((size_t)(s.M * s.lda) + 255) / 256 * 256;
+    s.bytes = s.off_rowsum + ((size_t)s.M * 4 + 255) / 256 * 256;
+    return s;
+}
+
+}  // namespace q4
+
+using namespace q4;
+
+extern "C" {
+
+q4_status q4_gemm(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                  int32_t* C, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                  int32_t za, int32_t zb, const int32_t* rowsum_a, const int32_t* colsum_b,
+                  void* ws, size_t ws_bytes, void* stream)
+{
+    (void)ws; (void)ws_bytes;
+    q4_status s = check_gemm(A, lda, Bt, ldb, M, N, K, za, zb);
+    if (s != Q4_OK) return s;
+    if (M == 0 || N == 0) return Q4_OK;
+    if (!C || ldc < N) return Q4_ERR_INVALID_ARG;
+    if ((uintptr_t)C % 4 != 0) return Q4_ERR_ALIGNMENT;
+    GemmParams p{};
+    p.A = A; p.Bt = Bt; p.lda = lda; p.ldb = ldb; p.M = M; p.N = N; p.K = K; p.za = za; p.zb = zb;
+    p.rowsum_a = rowsum_a; p.colsum_b = colsum_b; p.C = C; p.ldc = ldc;
+    return run_gemm(p, false, static_cast<cudaStream_t>(stream));
+}
+
+q4_status q4_gemm_requant(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                          int32_t M, int32_t N, int32_t K, int32_t za, int32_t zb,
+                          const int32_t* rowsum_a, const int32_t* colsum_b,
+                          const int32_t* bias, const q4_requant* rq,
+                          uint8_t* Cq, int64_t ldcq, void* ws, size_t ws_bytes, void* stream)
+{
+    (void)ws; (void)ws_bytes;
+    q4_status s = check_gemm(A, lda, Bt, ldb, M, N, K, za, zb);
+    if (s != Q4_OK) return s;
+    if ((s = check_requant(rq)) != Q4_OK) return s;
+    if (N & 1) return Q4_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return Q4_OK;
+    if (!Cq || ldcq < N / 2) return Q4_ERR_INVALID_ARG;
+    GemmParams p{};
+    p.A = A; p.Bt = Bt; p.lda = lda; p.ldb = ldb; p.M = M; p.N = N; p.K = K; p.za = za; p.zb = zb;
+    p.rowsum_a = rowsum_a; p.colsum_b = colsum_b; p.bias = bias; p.Cq = Cq; p.ldcq = ldcq;
+    p.rq = RequantParams{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
+    return run_gemm(p, true, static_cast<cudaStream_t>(stream));
+}
+
+q4_status q4_im2col(const uint8_t* X, const q4_conv_desc* d, int32_t za,
+                    uint8_t* A, int64_t lda, int32_t* rowsum_a, void* stream)
+{
+    q4_status s = check_conv(d, za);
+    if (s != Q4_OK) return s;
+    const ConvShape cs = conv_shape(d);
+    if (lda < ((int64_t)cs.K + 1) / 2) return Q4_ERR_INVALID_ARG;
+    if (cs.M == 0) return Q4_OK;
+    if (!X || !A) return Q4_ERR_INVALID_ARG;
+    if (rowsum_a && (uintptr_t)rowsum_a % 4 != 0) return Q4_ERR_ALIGNMENT;
+    return launch_im2col(X, *d, za, A, lda, rowsum_a, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
+size_t q4_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K)
+{
+    (void)M; (void)N; (void)K;
+    return 0;   // sums are taken inside the kernel; no split over the depth
+}
+
+size_t q4_conv2d_workspace_bytes(const q4_conv_desc* d)
+{
+    if (check_conv(d, 0) != Q4_OK) return 0;
+    return conv_shape(d).bytes;
+}
+
+q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
+                    const int32_t* colsum_w, const int32_t* bias,
+                    const q4_conv_desc* d, int32_t za, int32_t zb, const q4_requant* rq,
+                    uint8_t* Y, void* ws, size_t ws_bytes, void* stream)
+{
+    q4_status s = check_conv(d, za);
+    if (s != Q4_OK) return s;
+    if ((s = check_requant(rq)) != Q4_OK) return s;
+    if (zb < 0 || zb > 15) return Q4_ERR_RANGE;
+    if (d->OC < 0 || (d->OC & 1)) return Q4_ERR_INVALID_ARG;
+    const ConvShape cs = conv_shape(d);
+    if (ldw < ((int64_t)cs.K + 1) / 2) return Q4_ERR_INVALID_ARG;
+    if (cs.M == 0 || d->OC == 0) return Q4_OK;
+    if (!X || !Wt || !Y) return Q4_ERR_INVALID_ARG;
+    if (!ws || ws_bytes < cs.bytes) return Q4_ERR_WORKSPACE;
+    if ((uintptr_t)ws % 256 != 0) return Q4_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    uint8_t* A = static_cast<uint8_t*>(ws);
+    int32_t* rowsum = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + cs.off_rowsum);
+    if (launch_im2col(X, *d, za, A, cs.lda, rowsum, st) != cudaSuccess) return Q4_ERR_CUDA;
+
+    GemmParams p{};
+    p.A = A; p.Bt = Wt; p.lda = cs.lda; p.ldb = ldw; p.M = (int32_t)cs.M; p.N = d->OC; p.K = cs.K;
+    p.za = za; p.zb = zb; p.rowsum_a = rowsum; p.colsum_b = colsum_w; p.bias = bias;
+    p.Cq = Y; p.ldcq = d->OC / 2;
+    p.rq = RequantParams{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
+    return run_gemm(p, true, st);
+}
+
+q4_status q4_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int64_t ldb,
+                     int32_t K, int32_t N, void* stream)
+{
+    if (K < 1 || N < 0 || ldb_kn < (N + 1) / 2 || ldb < (K + 1) / 2) return Q4_ERR_INVALID_ARG;
+    if (N == 0) return Q4_OK;
+    if (!B_kn || !Bt) return Q4_ERR_INVALID_ARG;
+    return launch_pack_bt(B_kn, ldb_kn, Bt, ldb, K, N, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
+q4_status q4_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
+                      int32_t* sums, void* stream)
+{
+    if (rows < 0 || K < 1 || ld < (K + 1) / 2) return Q4_ERR_INVALID_ARG;
+    if (rows == 0) return Q4_OK;
+    if (!P || !sums) return Q4_ERR_INVALID_ARG;
+    return launch_row_sums(P, ld, rows, K, sums, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
+size_t q4_gemm_host_staging_bytes(int32_t M, int32_t N, int32_t K,
+                                  int64_t lda, int64_t ldb, int64_t ldc)
+{
+    (void)K;
+    if (M < 0 || N < 0 || lda < 0 || ldb < 0 || ldc < 0) return 0;
+    auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+    return up((size_t)M * (size_t)lda) + up((size_t)N * (size_t)ldb) + up((size_t)M * (size_t)ldc * 4);
+}
+
+q4_status q4_gemm_host(const uint8_t* hA, int64_t lda, const uint8_t* hBt, int64_t ldb,
+                       int32_t* hC, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                       int32_t za, int32_t zb, void* dev_staging, size_t dev_staging_bytes,
+                       void* stream)
+{
+    q4_status s = check_gemm(hA, lda, hBt, ldb, M, N, K, za, zb);
+    if (s != Q4_OK) return s;
+    if (M == 0 || N == 0) return Q4_OK;
+    if (!hC || ldc < N) return Q4_ERR_INVALID_ARG;
+    if (!dev_staging || dev_staging_bytes < q4_gemm_host_staging_bytes(M, N, K, lda, ldb, ldc))
+        return Q4_ERR_WORKSPACE;
+    if ((uintptr_t)dev_staging % 256 != 0) return Q4_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    auto up = [](size_t b) { return (b + 255) / 256 * 256; };
+    uint8_t* dA = static_cast<uint8_t*>(dev_staging);
+    uint8_t* dB = dA + up((size_t)M * lda);
+    int32_t* dC = reinterpret_cast<int32_t*>(dB + up((size_t)N * ldb));
+    if (cudaMemcpyAsync(dA, hA, (size_t)M * lda, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(dB, hBt, (size_t)N * ldb, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return Q4_ERR_CUDA;
+    s = q4_gemm(dA, lda, dB, ldb, dC, ldc, M, N, K, za, zb, nullptr, nullptr, nullptr, 0, stream);
+    if (s != Q4_OK) return s;
+    if (cudaMemcpyAsync(hC, dC, (size_t)M * ldc * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return Q4_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
+q4_status q4_last_device_status(void* stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaStreamSynchronize(st) != cudaSuccess) return Q4_ERR_CUDA;
+    unsigned* dptr = status_ptr();
+    if (!dptr) return Q4_ERR_CUDA;
+    unsigned word = 0;
+    if (cudaMemcpy(&word, dptr, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return Q4_ERR_CUDA;
+    if (word) {
+        if (cudaMemset(dptr, 0, sizeof(word)) != cudaSuccess) return Q4_ERR_CUDA;
+        return Q4_ERR_DEVICE_TIMEOUT;
+    }
+    return Q4_OK;
+}
+
+int q4_set_variant(int v)
+{
+    const int prev = variant();
+    g_variant.store((v == 1 || v == 2) ? v : 0, std::memory_order_relaxed);
+    return prev;
+}
+
+uint64_t q4_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* q4_status_string(q4_status s)
+{
+    switch (s) {
+        case Q4_OK: return "ok";
+        case Q4_ERR_INVALID_ARG: return "invalid argument";
+        case Q4_ERR_ALIGNMENT: return "misaligned pointer or pitch";
+        case Q4_ERR_RANGE: return "value out of range";
+        case Q4_ERR_WORKSPACE: return "workspace missing or too small";
+        case Q4_ERR_UNSUPPORTED: return "unsupported";
+        case Q4_ERR_CUDA: return "CUDA error";
+        case Q4_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+int q4_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,84 @@
+// Shared device-side pieces of the q4 library: the zero-point correction of Eq. 2,
+// the integer re-quantization, and the launch-parameter structs.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "q4.h"
+
+namespace q4 {
+
+// Bits of the device status word (reported by q4_last_device_status).
+constexpr unsigned kStatusTimeout = 1u;
+
+struct RequantParams {
+    int32_t mult, shift, zo, lo, hi;
+};
+
+struct GemmParams {
+    const uint8_t* A;      // [M, lda] packed
+    const uint8_t* Bt;     // [N, ldb] packed
+    int64_t lda, ldb;
+    int32_t M, N, K;
+    int32_t za, zb;
+    const int32_t* rowsum_a;   // optional
+    const int32_t* colsum_b;   // optional
+    const int32_t* bias;       // optional (requant only)
+    int32_t* C;                // int32 output (q4_gemm)
+    int64_t ldc;
+    uint8_t* Cq;               // packed output (q4_gemm_requant)
+    int64_t ldcq;
+    RequantParams rq;
+    unsigned* status;          // device status word
+};
+
+// Eq. 2, last line: raw product minus the two zero-point terms plus the constant.
+// Wrapping int32 arithmetic; the true value is bounded by 225*K <= 2^30.
+__device__ __forceinline__ int32_t correct(int32_t raw, int32_t rowsum, int32_t colsum,
+                                           int32_t za, int32_t zb, int32_t kzz)
+{
+    return (int32_t)((uint32_t)raw - (uint32_t)(zb * rowsum) - (uint32_t)(za * colsum)
+                     + (uint32_t)kzz);
+}
+
+// q = floor((acc*mult + 2^(30+shift)) / 2^(31+shift)); y = clamp(q + zo, lo, hi).
+// |acc| < 2^31 and mult < 2^31 keep the 64-bit sum below 2^63; >> on a signed
+// 64-bit value is an arithmetic (flooring) shift.
+__device__ __forceinline__ uint32_t requant(int32_t acc, const RequantParams& rq)
+{
+    const int t = 31 + rq.shift;
+    long long v = (long long)acc * (long long)rq.mult + (1ll << (t - 1));
+    int q = (int)(v >> t) + rq.zo;
+    q = max(q, rq.lo);
+    q = min(q, rq.hi);
+    return (uint32_t)q;
+}
+
+// Unsigned 4 x 8-bit dot product accumulated into a (wrapping) 32-bit value.
+__device__ __forceinline__ int dp4a_u8(uint32_t a, uint32_t b, int c)
+{
+    return (int)__dp4a(a, b, (uint32_t)c);
+}
+
+// Sum of the eight nibbles of a packed 32-bit word.
+__device__ __forceinline__ int nibble_sum(uint32_t w)
+{
+    uint32_t s = (w & 0x0F0F0F0Fu) + ((w >> 4) & 0x0F0F0F0Fu);   // bytes <= 30
+    return dp4a_u8(s, 0x01010101u, 0);
+}
+
+// ----- launchers implemented in the kernel translation units -----------------------
+cudaError_t launch_gemm_simt(const GemmParams& p, bool requant, cudaStream_t st);
+bool        gemm_tc_supported(const GemmParams& p);
+q4_status   launch_gemm_tc(const GemmParams& p, bool requant, cudaStream_t st);
+cudaError_t launch_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int64_t ldb,
+                           int32_t K, int32_t N, cudaStream_t st);
+cudaError_t launch_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
+                            int32_t* sums, cudaStream_t st);
+cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, uint8_t* A,
+                          int64_t lda, int32_t* rowsum_a, cudaStream_t st);
+
+void count_launch(int n = 1);
+
+}  // namespace q4

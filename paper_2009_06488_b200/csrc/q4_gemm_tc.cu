@@ -1,0 +1,532 @@
+// Tensor-core 4-bit quantized GEMM for sm_100a (Eq. 2 of the paper, all four terms).
+//
+// One persistent, warp-specialised kernel:
+//
+//   warp 0      TMA producer   packed-nibble tiles of A (128 rows) and Bt (BN rows),
+//                              64 bytes = 128 depth values per row per stage
+//   warps 2..   unpack         nibbles -> one byte per value, written in the K-major
+//                              128-byte-swizzled layout the MMA reads; the depth sums
+//                              of Eq. 2's second and third terms ride along (dp4a)
+//   warp 1      MMA issuer     tcgen05.mma kind::i8 (u8 x u8 -> s32), 128 x BN x 32
+//                              per instruction, accumulators in tensor memory
+//                              (two buffers, so the epilogue of tile t overlaps the
+//                              main loop of tile t+1)
+//   last 4 warps epilogue      tcgen05.ld, zero-point correction, then either the
+//                              int32 store or bias + re-quantization + nibble packing
+//
+// The sum over the depth commutes, so the unpack stores the even nibbles of each
+// 16-byte packed chunk as one 16-byte group and the odd nibbles as the next one
+// (three integer ops per eight values, no byte shuffles); A and Bt use the same
+// order, so the product is unchanged.
+//
+// Every mbarrier wait is bounded by a clock limit.  A wait that expires raises the
+// kernel's abort flag and the device status word; all roles then fall through their
+// loops with short waits and leave through the common exit (TMEM is freed).
+#include <cuda.h>
+
+#include <mutex>
+
+#include "q4_common.cuh"
+
+namespace q4 {
+
+constexpr int TM = 128;            // rows of A per tile (UMMA M)
+constexpr int PROW = 64;           // packed bytes per row per stage
+constexpr int UROW = 128;          // unpacked bytes per row per stage (one swizzle row)
+constexpr int SLAB = 128;          // depth values per stage
+constexpr int UW = 4;              // unpack warps
+constexpr int UT = UW * 32;        // unpack threads
+constexpr int NTHREADS = (2 + UW + 4) * 32;
+
+constexpr long long kWaitLong = 4000000000ll;   // ~2 s at 2 GHz
+constexpr long long kWaitShort = 2000000ll;     // ~1 ms, used once the kernel aborts
+
+template <int BN> struct Cfg {
+    static constexpr int ROWS = TM + BN;
+    static constexpr int PSTAGE = ROWS * PROW;
+    static constexpr int USTAGE = ROWS * UROW;
+    static constexpr int STAGES = (BN == 256) ? 3 : 4;
+    static constexpr int NT = (ROWS * 4 + UT - 1) / UT;        // unpack tasks per thread
+    static constexpr int TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
+    // layout: [U stages][P stages][sums 2*ROWS int32][colterm BN int32][barriers][misc]
+    static constexpr int OFF_U = 0;
+    static constexpr int OFF_P = OFF_U + STAGES * USTAGE;
+    static constexpr int OFF_SUMS = OFF_P + STAGES * PSTAGE;
+    static constexpr int OFF_COLTERM = OFF_SUMS + 2 * ROWS * 4;
+    static constexpr int OFF_BAR = OFF_COLTERM + BN * 4;
+    static constexpr int NBAR = 4 * STAGES + 6;
+    static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
+    static constexpr int SMEM = OFF_MISC + 16 + 1024;          // + slack to align the base
+};
+
+// ---- PTX wrappers -------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false (and raises the abort flag + status word) on expiry.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned* status)
+{
+    if (mbar_try(bar, parity)) return true;
+    const long long limit = *abort_flag ? kWaitShort : kWaitLong;
+    const long long t0 = clock64();
+    while (!mbar_try(bar, parity)) {
+        if (clock64() - t0 > limit) {
+            *abort_flag = 1;
+            atomicOr(status, kStatusTimeout);
+            return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
+                                            uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], u8 x u8 -> s32, shape 128 x N x 32.
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                          uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
+          "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
+          "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major, 128-byte swizzle shared-memory matrix descriptor: 8-row groups 1024 bytes
+// apart, descriptor version 1 (sm_100).
+__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t saddr)
+{
+    return (uint64_t)((saddr & 0x3FFFFu) >> 4)
+         | (1ull << 16)                 // leading byte offset (unused for swizzled K-major)
+         | ((uint64_t)(1024 >> 4) << 32)  // stride byte offset: next 8-row group
+         | (1ull << 46)                 // descriptor version
+         | (2ull << 61);                // SWIZZLE_128B
+}
+// Instruction descriptor: D = s32, A = B = unsigned 8-bit, both K-major, M = 128, N = BN.
+__host__ __device__ constexpr uint32_t make_idesc_u8(int n)
+{
+    return (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+}
+
+struct TcParams {
+    GemmParams g;
+    int32_t tiles_m, tiles_n, nslab;
+    int32_t c_vec;      // int32 rows may be stored with 16-byte vectors
+    int32_t cq_vec;     // packed rows may be stored with 16-byte vectors
+};
+
+template <int BN, bool REQUANT>
+__global__ void __launch_bounds__(NTHREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const TcParams p)
+{
+    using C = Cfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+
+    int32_t* sums_s = reinterpret_cast<int32_t*>(smem + C::OFF_SUMS);      // [2][ROWS]
+    int32_t* colterm_s = reinterpret_cast<int32_t*>(smem + C::OFF_COLTERM);
+    const uint32_t bar0 = sbase + C::OFF_BAR;
+    auto bar_full_p  = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto bar_empty_p = [&](int s) { return bar0 + 8u * (uint32_t)(C::STAGES + s); };
+    auto bar_full_u  = [&](int s) { return bar0 + 8u * (uint32_t)(2 * C::STAGES + s); };
+    auto bar_empty_u = [&](int s) { return bar0 + 8u * (uint32_t)(3 * C::STAGES + s); };
+    auto bar_tfull   = [&](int a) { return bar0 + 8u * (uint32_t)(4 * C::STAGES + a); };
+    auto bar_tempty  = [&](int a) { return bar0 + 8u * (uint32_t)(4 * C::STAGES + 2 + a); };
+    auto bar_sums    = [&](int a) { return bar0 + 8u * (uint32_t)(4 * C::STAGES + 4 + a); };
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + C::OFF_MISC);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const GemmParams& g = p.g;
+    const bool need_ra = (g.rowsum_a == nullptr);
+    const bool need_cb = (g.colsum_b == nullptr);
+    const bool need_sums = need_ra || need_cb;
+    const int ntiles = p.tiles_m * p.tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(bar_full_p(s), 1);
+            mbar_init(bar_empty_p(s), UT);
+            mbar_init(bar_full_u(s), UT);
+            mbar_init(bar_empty_u(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull(a), 1);
+            mbar_init(bar_tempty(a), 128);
+            mbar_init(bar_sums(a), UT);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32((const void*)tmem_slot)), "r"((uint32_t)C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+                const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+                for (int s = 0; s < p.nslab; ++s, ++it) {
+                    const int st = it % C::STAGES;
+                    const uint32_t ph = (it / C::STAGES) & 1u;
+                    mbar_wait(bar_empty_p(st), ph ^ 1u, abort_flag, g.status);
+                    mbar_expect_tx(bar_full_p(st), (uint32_t)C::PSTAGE);
+                    const uint32_t dst = sbase + C::OFF_P + st * C::PSTAGE;
+                    tma_load_2d(dst, &tmA, s * PROW, tm * TM, bar_full_p(st));
+                    tma_load_2d(dst + TM * PROW, &tmB, s * PROW, tn * BN, bar_full_p(st));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc_u8(BN);
+            uint32_t it = 0, lt = 0;
+            for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+                const int acc = lt & 1;
+                const uint32_t aph = (lt >> 1) & 1u;
+                mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int s = 0; s < p.nslab; ++s, ++it) {
+                    const int st = it % C::STAGES;
+                    const uint32_t ph = (it / C::STAGES) & 1u;
+                    mbar_wait(bar_full_u(st), ph, abort_flag, g.status);
+                    tc_fence_after();
+                    const uint32_t ua = sbase + C::OFF_U + st * C::USTAGE;
+                    const uint64_t adesc = make_kmajor_sw128_desc(ua);
+                    const uint64_t bdesc = make_kmajor_sw128_desc(ua + TM * UROW);
+                    const int rem = g.K - s * SLAB;
+                    const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
+                    for (int i = 0; i < ksteps; ++i)
+                        tc_mma_i8(d_tmem, adesc + (uint64_t)(2 * i), bdesc + (uint64_t)(2 * i), idesc,
+                                  (s > 0 || i > 0) ? 1u : 0u);
+                    tc_commit(bar_empty_u(st));
+                }
+                tc_commit(bar_tfull(acc));
+            }
+        }
+    } else if (warp < 2 + UW) {
+        // ------------------------------------------------------------ unpack warps
+        const int ut = threadIdx.x - 64;
+        uint32_t it = 0, lt = 0;
+        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+            int psum[C::NT];
+#pragma unroll
+            for (int j = 0; j < C::NT; ++j) psum[j] = 0;
+            for (int s = 0; s < p.nslab; ++s, ++it) {
+                const int st = it % C::STAGES;
+                const uint32_t ph = (it / C::STAGES) & 1u;
+                const int rem = g.K - s * SLAB;
+                const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
+                mbar_wait(bar_full_p(st), ph, abort_flag, g.status);
+                mbar_wait(bar_empty_u(st), ph ^ 1u, abort_flag, g.status);
+                tc_fence_after();
+                const uint8_t* ps = smem + C::OFF_P + st * C::PSTAGE;
+                uint8_t* us = smem + C::OFF_U + st * C::USTAGE;
+#pragma unroll
+                for (int j = 0; j < C::NT; ++j) {
+                    const int id = ut + j * UT;
+                    const int r = id >> 2, c = id & 3;
+                    if (id < C::ROWS * 4 && c < ksteps) {
+                        const uint4 w = *reinterpret_cast<const uint4*>(ps + r * PROW + c * 16);
+                        uint4 lo, hi;
+                        lo.x = w.x & 0x0F0F0F0Fu; hi.x = (w.x >> 4) & 0x0F0F0F0Fu;
+                        lo.y = w.y & 0x0F0F0F0Fu; hi.y = (w.y >> 4) & 0x0F0F0F0Fu;
+                        lo.z = w.z & 0x0F0F0F0Fu; hi.z = (w.z >> 4) & 0x0F0F0F0Fu;
+                        lo.w = w.w & 0x0F0F0F0Fu; hi.w = (w.w >> 4) & 0x0F0F0F0Fu;
+                        uint8_t* row = us + r * UROW;
+                        const int sw = r & 7;
+                        *reinterpret_cast<uint4*>(row + (((2 * c) ^ sw) << 4)) = lo;
+                        *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ sw) << 4)) = hi;
+                        if (need_sums) {
+                            int t = psum[j];
+                            t = dp4a_u8(lo.x + hi.x, 0x01010101u, t);
+                            t = dp4a_u8(lo.y + hi.y, 0x01010101u, t);
+                            t = dp4a_u8(lo.z + hi.z, 0x01010101u, t);
+                            t = dp4a_u8(lo.w + hi.w, 0x01010101u, t);
+                            psum[j] = t;
+                        }
+                    }
+                }
+                fence_async_smem();
+                mbar_arrive(bar_full_u(st));
+                mbar_arrive(bar_empty_p(st));
+            }
+            if (need_sums) {
+                const int acc = lt & 1;
+                const uint32_t aph = (lt >> 1) & 1u;
+                // the epilogue two tiles back must be done with this sums buffer
+                mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
+#pragma unroll
+                for (int j = 0; j < C::NT; ++j) {
+                    int t = psum[j];
+                    t += __shfl_xor_sync(0xFFFFFFFFu, t, 1);
+                    t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
+                    const int id = ut + j * UT;
+                    if (id < C::ROWS * 4 && (id & 3) == 0) sums_s[acc * C::ROWS + (id >> 2)] = t;
+                }
+                mbar_arrive(bar_sums(acc));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int lg = warp & 3;                 // TMEM lane group this warp may read
+        const int row = lg * 32 + lane;          // row of the tile held by this thread
+        const int et = threadIdx.x - (2 + UW) * 32;   // 0..127
+        const int kzz = g.K * g.za * g.zb;
+        uint32_t lt = 0;
+        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+            const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+            const int acc = lt & 1;
+            const uint32_t aph = (lt >> 1) & 1u;
+            const int m = tm * TM + row;
+            const int n0 = tn * BN;
+            if (need_sums) mbar_wait(bar_sums(acc), aph, abort_flag, g.status);
+            // per-column term of Eq. 2: -za * colsum + K za zb (+ bias)
+            for (int j = et; j < BN; j += 128) {
+                const int n = n0 + j;
+                int cb = 0, bias = 0;
+                if (n < g.N) {
+                    cb = need_cb ? sums_s[acc * C::ROWS + TM + j] : g.colsum_b[n];
+                    if (REQUANT && g.bias) bias = g.bias[n];
+                }
+                colterm_s[j] = (int)((uint32_t)kzz - (uint32_t)(g.za * cb) + (uint32_t)bias);
+            }
+            int ra = 0;
+            if (need_ra) ra = sums_s[acc * C::ROWS + row];
+            else if (m < g.M) ra = g.rowsum_a[m];
+            const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+
+            mbar_wait(bar_tfull(acc), aph, abort_flag, g.status);
+            tc_fence_after();
+            const uint32_t taddr0 = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+            for (int ch = 0; ch < BN / 32; ++ch) {
+                const int nc = n0 + ch * 32;
+                if (nc >= g.N) break;             // warp-uniform
+                uint32_t r[32];
+                tc_ld32(taddr0 + (uint32_t)(ch * 32), r);
+                tc_wait_ld();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = r[j] + rowterm + (uint32_t)colterm_s[ch * 32 + j];
+                if (m < g.M) {
+                    const bool full = (nc + 32 <= g.N);
+                    if (!REQUANT) {
+                        int32_t* dst = g.C + (int64_t)m * g.ldc + nc;
+                        if (full && p.c_vec) {
+#pragma unroll
+                            for (int q = 0; q < 8; ++q)
+                                *reinterpret_cast<uint4*>(dst + 4 * q) =
+                                    make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (nc + j < g.N) dst[j] = (int32_t)r[j];
+                        }
+                    } else {
+                        uint32_t o[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            uint32_t wv = 0;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                wv |= requant((int32_t)r[8 * q + e], g.rq) << (4 * e);
+                            o[q] = wv;
+                        }
+                        uint8_t* dst = g.Cq + (int64_t)m * g.ldcq + (nc >> 1);
+                        if (full && p.cq_vec) {
+                            *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                        } else {
+#pragma unroll
+                            for (int b = 0; b < 16; ++b)
+                                if (nc + 2 * b < g.N) dst[b] = (uint8_t)(o[b >> 2] >> (8 * (b & 3)));
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar_tempty(acc));
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // colterm_s is rewritten next tile
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) ==
+                cudaSuccess && qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    });
+    return fn;
+}
+
+// Packed matrix [rows x kbytes] with pitch ld, box = 64 bytes x box_rows; out-of-range
+// rows and bytes are filled with zeros (zero nibbles add nothing to any term of Eq. 2).
+static bool make_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows, int kbytes,
+                     int box_rows)
+{
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kbytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld};
+    cuuint32_t box[2] = {(cuuint32_t)PROW, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides,
+               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool gemm_tc_supported(const GemmParams& p)
+{
+    return ((uintptr_t)p.A % 16 == 0) && ((uintptr_t)p.Bt % 16 == 0) && (p.lda % 16 == 0) &&
+           (p.ldb % 16 == 0) && p.M > 0 && p.N > 0;
+}
+
+static int sm_count()
+{
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int BN>
+static q4_status launch_bn(const GemmParams& g, bool rq, cudaStream_t st)
+{
+    using C = Cfg<BN>;
+    TcParams p;
+    p.g = g;
+    p.tiles_m = (g.M + TM - 1) / TM;
+    p.tiles_n = (g.N + BN - 1) / BN;
+    const int kbytes = (g.K + 1) / 2;
+    p.nslab = (kbytes + PROW - 1) / PROW;
+    p.c_vec = (!rq && ((uintptr_t)g.C % 16 == 0) && (g.ldc % 4 == 0)) ? 1 : 0;
+    p.cq_vec = (rq && ((uintptr_t)g.Cq % 16 == 0) && (g.ldcq % 16 == 0)) ? 1 : 0;
+
+    CUtensorMap tmA, tmB;
+    if (!make_map(&tmA, g.A, g.lda, g.M, kbytes, TM)) return Q4_ERR_CUDA;
+    if (!make_map(&tmB, g.Bt, g.ldb, g.N, kbytes, BN)) return Q4_ERR_CUDA;
+
+    const long long tiles = (long long)p.tiles_m * p.tiles_n;
+    const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    cudaError_t e;
+    if (rq) {
+        static bool attr = false;
+        if (!attr) {
+            e = cudaFuncSetAttribute(gemm_tc_kernel<BN, true>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+            if (e != cudaSuccess) return Q4_ERR_CUDA;
+            attr = true;
+        }
+        gemm_tc_kernel<BN, true><<<grid, NTHREADS, C::SMEM, st>>>(tmA, tmB, p);
+    } else {
+        static bool attr = false;
+        if (!attr) {
+            e = cudaFuncSetAttribute(gemm_tc_kernel<BN, false>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+            if (e != cudaSuccess) return Q4_ERR_CUDA;
+            attr = true;
+        }
+        gemm_tc_kernel<BN, false><<<grid, NTHREADS, C::SMEM, st>>>(tmA, tmB, p);
+    }
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
+q4_status launch_gemm_tc(const GemmParams& g, bool rq, cudaStream_t st)
+{
+    if (g.N > 128) return launch_bn<256>(g, rq, st);
+    if (g.N > 64)  return launch_bn<128>(g, rq, st);
+    if (g.N > 32)  return launch_bn<64>(g, rq, st);
+    return launch_bn<32>(g, rq, st);
+}
+
+}  // namespace q4

@@ -1,0 +1,116 @@
+"""The C-ABI library loads without a GPU, exports every symbol the header declares,
+and validates arguments on the host before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2009_06488_b200 import build
+    return ctypes.CDLL(build.build())
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "q4.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(q4_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_four_calls():
+    syms = declared_symbols()
+    for name in ("q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d"):
+        assert name in syms
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in declared_symbols():
+        assert hasattr(lib, name), name
+
+
+def test_binding_lists_the_same_symbols():
+    from paper_2009_06488_b200 import binding
+    assert sorted(binding.EXPORTS) == declared_symbols()
+    for name in binding.EXPORTS:
+        assert hasattr(binding, name) or name in ("q4_gemm_workspace_bytes",)
+
+
+def test_status_strings_and_version(lib):
+    lib.q4_status_string.restype = ctypes.c_char_p
+    assert lib.q4_status_string(0) == b"ok"
+    assert len({lib.q4_status_string(i) for i in range(8)}) == 8
+    assert lib.q4_version() >= 100
+
+
+class RQ(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("mult", "shift", "zo", "lo", "hi")]
+
+
+class CD(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("N", "H", "W", "C", "OC", "KH", "KW", "sh", "sw", "ph", "pw")]
+
+
+def test_host_side_validation_needs_no_device(lib):
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    lib.q4_gemm.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+    fake = 0x1000   # never dereferenced: every call below is rejected before any launch
+    INVALID, ALIGN, RANGE, WORKSPACE = 1, 2, 3, 4
+    g = lambda **kw: lib.q4_gemm(kw.get("A", fake), kw.get("lda", 64), kw.get("B", fake),
+                                 kw.get("ldb", 64), kw.get("C", fake), kw.get("ldc", 8),
+                                 kw.get("M", 8), kw.get("N", 8), kw.get("K", 128),
+                                 kw.get("za", 0), kw.get("zb", 0), None, None, None, 0, None)
+    assert g(K=0) == INVALID
+    assert g(M=-1) == INVALID
+    assert g(A=None) == INVALID
+    assert g(C=None) == INVALID
+    assert g(lda=63) == INVALID            # pitch shorter than a row of 128 nibbles
+    assert g(ldc=7) == INVALID
+    assert g(za=16) == RANGE
+    assert g(zb=-1) == RANGE
+    assert g(K=(1 << 22) + 1, lda=1 << 22, ldb=1 << 22) == RANGE
+    assert g(C=fake + 2) == ALIGN
+    assert g(M=0) == 0 and g(N=0) == 0      # empty problems are no-ops
+
+    lib.q4_gemm_requant.argtypes = [vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp,
+                                    ctypes.POINTER(RQ), vp, i64, vp, sz, vp]
+    def r(rq, N=8, ldcq=4):
+        return lib.q4_gemm_requant(fake, 64, fake, 64, 8, N, 128, 0, 0, None, None, None,
+                                   ctypes.byref(rq) if rq else None, fake, ldcq, None, 0, None)
+    assert r(None) == INVALID
+    assert r(RQ(1 << 29, 8, 0, 0, 15)) == RANGE
+    assert r(RQ(1 << 30, 32, 0, 0, 15)) == RANGE
+    assert r(RQ(1 << 30, 8, 16, 0, 15)) == RANGE
+    assert r(RQ(1 << 30, 8, 0, 9, 8)) == RANGE
+    assert r(RQ(1 << 30, 8, 0, 0, 15), N=7) == INVALID
+    assert r(RQ(1 << 30, 8, 0, 0, 15), ldcq=3) == INVALID
+
+    lib.q4_conv2d.argtypes = [vp, vp, i64, vp, vp, ctypes.POINTER(CD), i32, i32,
+                              ctypes.POINTER(RQ), vp, vp, sz, vp]
+    lib.q4_conv2d_workspace_bytes.argtypes = [ctypes.POINTER(CD)]
+    lib.q4_conv2d_workspace_bytes.restype = sz
+    d = CD(2, 8, 8, 16, 32, 3, 3, 1, 1, 1, 1)
+    rq = RQ(1 << 30, 8, 0, 0, 15)
+    need = lib.q4_conv2d_workspace_bytes(ctypes.byref(d))
+    assert need >= 2 * 8 * 8 * (80 + 4)     # unrolled matrix at a 16-byte-multiple pitch + row sums
+    c = lambda d, ws, wsb: lib.q4_conv2d(fake, fake, 72, None, None, ctypes.byref(d), 0, 0,
+                                         ctypes.byref(rq), fake, ws, wsb, None)
+    assert c(d, None, 0) == WORKSPACE
+    assert c(d, 0x10000, need - 1) == WORKSPACE
+    assert c(d, 0x10010, need) == ALIGN
+    assert c(CD(2, 2, 2, 16, 32, 3, 3, 1, 1, 0, 0), 0x10000, 1 << 20) == INVALID   # kernel larger than image
+    assert c(CD(2, 8, 8, 16, 31, 3, 3, 1, 1, 1, 1), 0x10000, 1 << 20) == INVALID   # odd channel count out
+
+
+def test_compute_call_without_a_device_fails_loudly(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    lib.q4_gemm.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+    assert lib.q4_gemm(0x1000, 64, 0x1000, 64, 0x1000, 8, 8, 8, 128, 0, 0, None, None, None, 0,
+                       None) == 6   # Q4_ERR_CUDA: no silent CPU path

@@ -1,0 +1,230 @@
+"""GPU parity: q4_gemm / q4_gemm_requant through the C ABI against the CPU oracle,
+element by element, bit-exact (all work is integer)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2009_06488_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+SIMT, TC = 1, 2
+
+
+@pytest.fixture(scope="module")
+def q4():
+    from paper_2009_06488_b200 import binding
+    yield binding
+    binding.q4_set_variant(0)
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def run_gemm(q4, c, variant, ldc_pad=0, sums=False):
+    import torch
+    q4.q4_set_variant(variant)
+    A, Bt = dev(c.A), dev(c.Bt)
+    C = torch.full((c.M, c.N + ldc_pad), -1515870811, dtype=torch.int32, device="cuda")  # 0xA5A5A5A5
+    ra = cb = None
+    if sums:
+        ra = torch.empty(c.M, dtype=torch.int32, device="cuda")
+        cb = torch.empty(c.N, dtype=torch.int32, device="cuda")
+        q4.q4_row_sums(A, c.M, c.K, ra)
+        q4.q4_row_sums(Bt, c.N, c.K, cb)
+    q4.q4_gemm(A, Bt, C, c.M, c.N, c.K, c.za, c.zb, ra, cb)
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    out = C.cpu().numpy()
+    if ldc_pad:
+        assert (out[:, c.N:] == -1515870811).all()      # pitch padding untouched
+    return out[:, :c.N], ra, cb
+
+
+def run_requant(q4, c, variant, rq, bias=None, ld_pad=0):
+    import torch
+    q4.q4_set_variant(variant)
+    A, Bt = dev(c.A), dev(c.Bt)
+    Cq = torch.full((c.M, c.N // 2 + ld_pad), 0xA5, dtype=torch.uint8, device="cuda")
+    q4.q4_gemm_requant(A, Bt, Cq, c.M, c.N, c.K, c.za, c.zb,
+                       q4.Requant(rq.mult, rq.shift, rq.zo, rq.clamp_lo, rq.clamp_hi),
+                       None if bias is None else dev(bias))
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    out = Cq.cpu().numpy()
+    if ld_pad:
+        assert (out[:, c.N // 2:] == 0xA5).all()
+    return out[:, :c.N // 2]
+
+
+TABLE1 = [(h, w, d) for h in (8, 24) for w in (100, 400, 1600) for d in (10, 40, 100)]
+ODD = [(1, 1, 1), (3, 5, 7), (65, 33, 129), (130, 70, 255), (64, 64, 64)]
+
+
+@pytest.mark.parametrize("shape", TABLE1 + ODD)
+def test_simt_gemm_any_shape_any_pitch(q4, shape):
+    M, N, K = shape
+    kb = (K + 1) // 2
+    c = wl.gemm_case("t", M, N, K, seed=M * 7919 + N * 31 + K, lda=kb + 3, ldb=kb + 1)
+    got, _, _ = run_gemm(q4, c, SIMT, ldc_pad=3)
+    want = oracle.gemm(c.A, c.Bt, M, N, K, c.za, c.zb)
+    assert (got == want).all()
+
+
+# aligned problems for the tensor-core path: tails in M, N and K, small N, tiny K
+TC_SHAPES = [(64, 64, 256), (128, 256, 128), (128, 32, 32), (130, 260, 1000), (257, 40, 144),
+             (300, 16, 72), (1000, 8, 9), (129, 130, 131), (384, 512, 1024), (5, 3, 1),
+             (256, 96, 4096), (200, 200, 33)]
+
+
+def aligned_case(M, N, K, seed, **kw):
+    ld = ((K + 1) // 2 + 15) // 16 * 16
+    return wl.gemm_case("t", M, N, K, seed=seed, lda=ld, ldb=ld, **kw)
+
+
+@pytest.mark.parametrize("shape", TC_SHAPES)
+def test_tc_gemm_matches_oracle(q4, shape):
+    M, N, K = shape
+    c = aligned_case(M, N, K, seed=M * 7919 + N * 31 + K)
+    want = oracle.gemm(c.A, c.Bt, M, N, K, c.za, c.zb)
+    got, _, _ = run_gemm(q4, c, TC, ldc_pad=4)
+    assert (got == want).all()
+    got2, _, _ = run_gemm(q4, c, TC, ldc_pad=1)      # unaligned int32 pitch: scalar stores
+    assert (got2 == want).all()
+
+
+@pytest.mark.parametrize("variant", [SIMT, TC])
+def test_precomputed_sums_give_the_same_result(q4, variant):
+    c = aligned_case(200, 72, 300, seed=77)
+    want, ra_want, cb_want = oracle.gemm_fourterm(c.A, c.Bt, c.M, c.N, c.K, c.za, c.zb)
+    got, ra, cb = run_gemm(q4, c, variant, sums=True)
+    assert (ra.cpu().numpy() == ra_want).all() and (cb.cpu().numpy() == cb_want).all()
+    assert (got == want).all()
+
+
+@pytest.mark.parametrize("variant", [SIMT, TC])
+@pytest.mark.parametrize("zz", [(0, 0), (15, 15), (0, 15), (15, 0)])
+def test_extreme_zero_points(q4, variant, zz):
+    c = aligned_case(140, 48, 520, seed=5, za=zz[0], zb=zz[1])
+    got, _, _ = run_gemm(q4, c, variant)
+    assert (got == oracle.gemm(c.A, c.Bt, c.M, c.N, c.K, c.za, c.zb)).all()
+
+
+@pytest.mark.parametrize("variant", [SIMT, TC])
+def test_all_fifteen_inputs_reach_225K(q4, variant):
+    K = 4096
+    c = aligned_case(128, 32, K, seed=1, za=0, zb=0)
+    c.A[:, :K // 2] = 0xFF
+    c.Bt[:, :K // 2] = 0xFF
+    got, _, _ = run_gemm(q4, c, variant)
+    assert (got == 225 * K).all()
+
+
+def test_c1_single_gemm(q4):
+    c = wl.c1()
+    want = oracle.gemm(c.A, c.Bt, c.M, c.N, c.K, c.za, c.zb)
+    for v in (SIMT, TC):
+        got, _, _ = run_gemm(q4, c, v)
+        assert (got == want).all()
+
+
+@pytest.mark.parametrize("variant", [SIMT, TC])
+@pytest.mark.parametrize("shape", [(64, 64, 256), (130, 260, 1000), (257, 40, 144), (300, 16, 72),
+                                   (33, 2, 5), (128, 256, 512)])
+def test_gemm_requant_matches_oracle(q4, variant, shape):
+    M, N, K = shape
+    c = aligned_case(M, N, K, seed=M + N + K, with_bias=True)
+    for i, (shift, zo, lo, hi) in enumerate([(c.shift, 0, 0, 15), (4, 3, 3, 15), (0, 8, 0, 9)]):
+        rq = oracle.Requant(c.mult, shift, zo, lo, hi)
+        bias = c.bias if i else None
+        want = oracle.gemm_requant(c.A, c.Bt, M, N, K, c.za, c.zb, bias, rq)
+        got = run_requant(q4, c, variant, rq, bias, ld_pad=0 if i == 0 else 16)
+        assert (got == want).all()
+        if shift == 4:
+            assert len(np.unique(oracle.unpack_rows(got, N))) > 3   # not saturated everywhere
+
+
+@pytest.mark.parametrize("n", [512, 1024, 2048])
+def test_c2_square_sweep_full_compare(q4, n):
+    c = wl.c2(n)
+    want = oracle.gemm(c.A, c.Bt, n, n, n, c.za, c.zb)
+    got, _, _ = run_gemm(q4, c, TC)
+    assert (got == want).all()
+    rq = oracle.Requant(c.mult, c.shift, 0, 0, 15)
+    wantq = oracle.requant_matrix(want, None, rq)
+    gotq = run_requant(q4, c, TC, rq)
+    assert (gotq == wantq).all()
+
+
+def freivalds_check(c, C):
+    """Exact integer Freivalds: C r == A' (B' r) and l C == (l A') B' in int64, with
+    A' = A - za, B' = B - zb taken from the unpacked operands in row blocks."""
+    rng = np.random.default_rng(c.seed + 1)
+    r = rng.integers(1, 1 << 20, c.N).astype(np.int64)
+    l = rng.integers(1, 1 << 20, c.M).astype(np.int64)
+    blk = 512
+    y = np.zeros(c.K, np.int64)                     # B' r
+    for n0 in range(0, c.N, blk):
+        b = oracle.unpack_rows(c.Bt[n0:n0 + blk], c.K).astype(np.int64) - c.zb
+        y += b.T @ r[n0:n0 + blk]
+    lA = np.zeros(c.K, np.int64)                    # l A'
+    for m0 in range(0, c.M, blk):
+        a = oracle.unpack_rows(c.A[m0:m0 + blk], c.K).astype(np.int64) - c.za
+        assert (C[m0:m0 + blk].astype(np.int64) @ r == a @ y).all()
+        lA += l[m0:m0 + blk] @ a
+    lC = l @ C.astype(np.int64)
+    for n0 in range(0, c.N, blk):
+        b = oracle.unpack_rows(c.Bt[n0:n0 + blk], c.K).astype(np.int64) - c.zb
+        assert (lC[n0:n0 + blk] == b @ lA).all()
+
+
+def sampled_rows_check(c, C, rows):
+    sub = np.ascontiguousarray(c.A[rows])
+    want = oracle.gemm(sub, c.Bt, len(rows), c.N, c.K, c.za, c.zb)
+    assert (C[rows] == want).all()
+
+
+def test_c2_4096_sampled_rows_and_freivalds(q4):
+    c = wl.c2(4096)
+    got, _, _ = run_gemm(q4, c, TC)
+    rows = np.unique(np.concatenate([np.arange(0, 4096, 97), [0, 127, 128, 4095]]))
+    sampled_rows_check(c, got, rows)
+    freivalds_check(c, got)
+    # requantized output on the same sampled rows
+    rq = oracle.Requant(c.mult, c.shift, 0, 0, 15)
+    gotq = run_requant(q4, c, TC, rq)
+    wantq = oracle.requant_matrix(np.ascontiguousarray(got[rows]), None, rq)
+    assert (gotq[rows] == wantq).all()
+
+
+def test_empty_problem_is_a_no_op(q4):
+    import torch
+    A = torch.zeros((0, 64), dtype=torch.uint8, device="cuda")
+    Bt = torch.zeros((8, 64), dtype=torch.uint8, device="cuda")
+    C = torch.zeros((0, 8), dtype=torch.int32, device="cuda")
+    q4.q4_gemm(A, Bt, C, 0, 8, 128, 0, 0)
+    assert q4.q4_last_device_status() == q4.Q4_OK
+
+
+def test_pack_bt_matches_oracle(q4):
+    import torch
+    rng = np.random.default_rng(3)
+    for K, N in [(7, 5), (32, 64), (33, 18), (300, 130)]:
+        b_kn = oracle.pack_rows(rng.integers(0, 16, (K, N), dtype=np.uint8))
+        ldb = (K + 1) // 2 + 2
+        want = oracle.pack_bt(b_kn, K, N, ldb)
+        Bt = torch.full((N, ldb), 0xA5, dtype=torch.uint8, device="cuda")
+        q4.q4_pack_bt(dev(b_kn), Bt, K, N)
+        assert (Bt.cpu().numpy() == want).all()
+
+
+def test_host_entry_point(q4):
+    import torch
+    c = aligned_case(300, 200, 520, seed=12)
+    hA, hBt = torch.from_numpy(c.A).pin_memory(), torch.from_numpy(c.Bt).pin_memory()
+    hC = torch.zeros((c.M, c.N), dtype=torch.int32).pin_memory()
+    need = q4.q4_gemm_host_staging_bytes(c.M, c.N, c.K, c.lda, c.ldb, c.N)
+    staging = torch.empty(need, dtype=torch.uint8, device="cuda")
+    q4.q4_set_variant(0)
+    q4.q4_gemm_host(hA, hBt, hC, c.M, c.N, c.K, c.za, c.zb, staging)
+    assert (hC.numpy() == oracle.gemm(c.A, c.Bt, c.M, c.N, c.K, c.za, c.zb)).all()
