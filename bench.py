@@ -1,0 +1,356 @@
+#!/usr/bin/env python
+"""Benchmark of the 4-bit quantized GEMM / convolution path on B200.
+
+One "step" is one pass of the whole hot path over one batch of seeded synthetic input:
+  1. q4_gemm          M=N=K=8192, uint4 x uint4 -> int32 (zero-point corrected, Eq. 2)
+  2. q4_gemm_requant  same operands, re-quantized uint4 output (fused epilogue)
+  3. q4_conv2d        conv layer 256x32x32x16 -> 32 channels, 3x3, stride 1, pad 1
+                      (unroll + GEMM + re-quantize)
+The headline value is whole-job TOPS (2 ops per multiply-accumulate) with inputs
+resident in HBM; `e2e` is the same metric with host buffers and the copies inside the
+timed region.  The `roofline` object describes the dominant kernel (the 8192^3 GEMM
+with int32 output), timed live with CUDA events on the launching stream.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Under torchrun (N > 1) every rank runs the same independent problem on its own GPU
+(the path shards over independent problems; there is no data-path collective).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+GEMM_N = 8192
+DATASHEET_INT8_TOPS = 4500.0          # B200 dense INT8, public datasheet figure
+NOMINAL_INT8_OVER_BF16 = 2.0          # 4.5 / 2.25 PFLOP/s dense
+FALLBACK_BF16_TFLOPS = 1590.0
+FALLBACK_HBM_GBS = 6650.0
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel,
+# or None when no capture exists for the kernel as it stands (see profiles/).
+DOMINANT_KERNEL_TRAFFIC_BYTES = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16": float(d["bf16_tflops"]), "bf16_sustained": float(d["bf16_tflops_sustained"]),
+                "hbm": float(d["hbm_gbs"]), "source": "measured"}
+    return {"bf16": FALLBACK_BF16_TFLOPS, "bf16_sustained": 1400.0, "hbm": FALLBACK_HBM_GBS,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines: list[str] = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, smax, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2])); power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        # samples taken while the GPU was busy: the upper half by power draw
+        busy = sorted(zip(power, sm))[len(sm) // 2:] if sm else []
+        return {"sm_mhz": statistics.median(s for _, s in busy) if busy else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# --------------------------------------------------------------------------- CPU baseline
+
+def time_oracle_sample(case, target_s: float = 12.0):
+    """Times the oracle, as it stands, on a row slice of the GEMM sized for about
+    `target_s` seconds; returns (TOPS, seconds, rows, threads)."""
+    import oracle
+    probe = 16
+    t0 = time.perf_counter()
+    oracle.gemm(np.ascontiguousarray(case.A[:probe]), case.Bt, probe, case.N, case.K, case.za, case.zb)
+    dt = time.perf_counter() - t0
+    rows = int(max(probe, min(case.M, probe * target_s / max(dt, 1e-6))))
+    rows = min(rows, case.M)
+    t0 = time.perf_counter()
+    oracle.gemm(np.ascontiguousarray(case.A[:rows]), case.Bt, rows, case.N, case.K, case.za, case.zb)
+    dt = time.perf_counter() - t0
+    ops = 2.0 * rows * case.N * case.K
+    return ops / dt / 1e12, dt, rows, oracle.num_threads()
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on a bounded sample of the same workload."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return 0
+    from paper_2009_06488_b200 import workloads as wl
+    case = wl.c2(GEMM_N)
+    import oracle
+    # size one step for a few seconds so that steps + warmup end within minutes
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    per_step = max(0.5, min(10.0, budget))
+    tops0, dt0, rows, threads = time_oracle_sample(case, per_step)
+    sub = np.ascontiguousarray(case.A[:rows])
+    for _ in range(max(0, args.warmup - 1)):
+        oracle.gemm(sub, case.Bt, rows, case.N, case.K, case.za, case.zb)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.gemm(sub, case.Bt, rows, case.N, case.K, case.za, case.zb)
+    dt = (time.perf_counter() - t0) / args.steps
+    tops = 2.0 * rows * case.N * case.K / dt / 1e12
+    sample = f"{rows} of {case.M} rows of the {GEMM_N}^3 GEMM per step (int32 output)"
+    line = {"impl": "reference", "metric": "4-bit GEMM TOPS at M=N=K=8192", "value": tops,
+            "unit": "TOPS", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+            "config": {"workload": f"c2 4-bit GEMM M=N=K={GEMM_N}, CPU oracle on a row sample"},
+            "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": threads, "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------- GPU arm
+
+def run_ours(args):
+    import torch
+    rank, world, local = dist_env()
+    from paper_2009_06488_b200 import binding as q4
+    from paper_2009_06488_b200 import workloads as wl
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    peaks = measured_peaks()
+
+    # ---- inputs (host, pinned) -> device
+    g = wl.c2(GEMM_N)
+    net = wl.c3()
+    L = net.layers[0]
+    dq = q4.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
+    rq_g = q4.Requant(g.mult, g.shift, 0, 0, 15)
+    rq_c = q4.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    hA, hBt, hX, hW = pin(g.A), pin(g.Bt), pin(net.X), pin(L.Wt)
+    A, Bt, X, Wt = hA.cuda(), hBt.cuda(), hX.cuda(), hW.cuda()
+    C = torch.empty((g.M, g.N), dtype=torch.int32, device="cuda")
+    Cq = torch.empty((g.M, g.N // 2), dtype=torch.uint8, device="cuda")
+    Y = torch.empty((dq.M, L.OC // 2), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(q4.q4_conv2d_workspace_bytes(dq), dtype=torch.uint8, device="cuda")
+    hC = torch.empty((g.M, g.N), dtype=torch.int32).pin_memory()
+    hCq = torch.empty((g.M, g.N // 2), dtype=torch.uint8).pin_memory()
+    hY = torch.empty((dq.M, L.OC // 2), dtype=torch.uint8).pin_memory()
+    staging = torch.empty(q4.q4_gemm_host_staging_bytes(g.M, g.N, g.K, g.lda, g.ldb, g.N),
+                          dtype=torch.uint8, device="cuda")
+
+    gemm_ops = 2.0 * g.M * g.N * g.K
+    conv_ops = 2.0 * dq.M * dq.K * L.OC
+    step_ops = 2 * gemm_ops + conv_ops
+    lda_c = (dq.K // 2 + 15) // 16 * 16
+    conv_path_bytes = X.numel() + 2 * dq.M * lda_c + 2 * 4 * dq.M + Wt.numel() + Y.numel()
+    conv_compulsory_bytes = X.numel() + Wt.numel() + Y.numel()
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    marks = []
+
+    def step(record: bool):
+        e = [ev() for _ in range(4)] if record else None
+        if record: e[0].record()
+        q4.q4_gemm(A, Bt, C, g.M, g.N, g.K, g.za, g.zb)
+        if record: e[1].record()
+        q4.q4_gemm_requant(A, Bt, Cq, g.M, g.N, g.K, g.za, g.zb, rq_g)
+        if record: e[2].record()
+        q4.q4_conv2d(X, Wt, dq, L.za, L.zb, rq_c, Y, ws)
+        if record:
+            e[3].record()
+            marks.append(e)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        step(False)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    launches0 = q4.q4_launch_count()
+    t_begin, t_end = ev(), ev()
+    t_begin.record()
+    for _ in range(args.steps):
+        step(True)
+    t_end.record()
+    barrier()
+    launches = q4.q4_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    assert q4.q4_last_device_status() == q4.Q4_OK, "a device-side wait timed out"
+
+    total_ms = t_begin.elapsed_time(t_end)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * step_ops / (ms_per_step * 1e-3) / 1e12
+
+    gemm_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in marks)
+    gemm_rq_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in marks)
+    conv_ms = statistics.mean(e[2].elapsed_time(e[3]) for e in marks)
+    gemm_tops = gemm_ops / (gemm_ms * 1e-3) / 1e12
+    int8_peak = NOMINAL_INT8_OVER_BF16 * peaks["bf16"]
+
+    # ---- end to end: host buffers, copies inside the timed region
+    def e2e_step():
+        q4.q4_gemm_host(hA, hBt, hC, g.M, g.N, g.K, g.za, g.zb, staging)
+        A.copy_(hA, non_blocking=True); Bt.copy_(hBt, non_blocking=True)
+        q4.q4_gemm_requant(A, Bt, Cq, g.M, g.N, g.K, g.za, g.zb, rq_g)
+        hCq.copy_(Cq, non_blocking=True)
+        X.copy_(hX, non_blocking=True); Wt.copy_(hW, non_blocking=True)
+        q4.q4_conv2d(X, Wt, dq, L.za, L.zb, rq_c, Y, ws)
+        hY.copy_(Y, non_blocking=True)
+        torch.cuda.synchronize()
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = 2 * (hA.numel() + hBt.numel()) + hX.numel() + hW.numel()
+    d2h = hC.numel() * 4 + hCq.numel() + hY.numel()
+
+    if rank != 0:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+        return 0
+
+    # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
+    cpu_baseline = None
+    if world == 1 and not args.no_cpu_baseline:
+        tops, dt, rows, threads = time_oracle_sample(g, 12.0)
+        cpu_baseline = {"value": tops, "unit": "TOPS", "cores": threads, "kind": "oracle",
+                        "sample": f"first {rows} of {g.M} rows of the {GEMM_N}^3 GEMM, "
+                                  f"int32 output, {dt:.1f} s"}
+
+    line = {
+        "metric": "4-bit GEMM TOPS at M=N=K=8192", "value": value, "unit": "TOPS",
+        "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": f"c2 4-bit GEMM M=N=K={GEMM_N} (int32 output, then fused "
+                               "requantized uint4 output) + c3 conv layer 256x32x32x16->32 3x3 s1 p1",
+                   "l2": "each step writes 288 MB of GEMM output, larger than the 126 MB L2, "
+                         "so every timed iteration starts with its inputs evicted",
+                   "parallelism": f"{world} independent replicas" if world > 1 else "1 GPU"},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "e2e": {"value": world * step_ops / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS",
+                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
+                "ms_per_step": e2e_ms},
+        "roofline": {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
+                     "frac": gemm_tops / int8_peak, "traffic": DOMINANT_KERNEL_TRAFFIC_BYTES,
+                     "kernel": "gemm_tc_kernel<256,false> (q4_gemm 8192^3, int32 output)",
+                     "peak_source": f"2 x {peaks['source']} bf16 burst "
+                                    f"({peaks['bf16']} TFLOP/s), nominal int8:bf16 ratio",
+                     "frac_of_datasheet_int8_4500": gemm_tops / DATASHEET_INT8_TOPS,
+                     "frac_of_2x_bf16_sustained": gemm_tops / (2 * peaks["bf16_sustained"])},
+        "cpu_baseline": cpu_baseline,
+        "detail": {
+            "q4_gemm_8192_ms": gemm_ms, "q4_gemm_8192_tops": gemm_tops,
+            "q4_gemm_requant_8192_ms": gemm_rq_ms,
+            "q4_gemm_requant_8192_tops": gemm_ops / (gemm_rq_ms * 1e-3) / 1e12,
+            "q4_conv2d_c3_ms": conv_ms,
+            "q4_conv2d_c3_path_gbs": conv_path_bytes / (conv_ms * 1e-3) / 1e9,
+            "q4_conv2d_c3_compulsory_gbs": conv_compulsory_bytes / (conv_ms * 1e-3) / 1e9,
+            "q4_conv2d_c3_path_frac_of_hbm": conv_path_bytes / (conv_ms * 1e-3) / 1e9 / peaks["hbm"],
+            "hbm_peak_gbs": peaks["hbm"], "peaks": peaks["source"]},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -133,14 +133,14 @@ def test_c1_single_gemm(q4):
                                    (33, 2, 5), (128, 256, 512)])
 def test_gemm_requant_matches_oracle(q4, variant, shape):
     M, N, K = shape
-    c = aligned_case(M, N, K, seed=M + N + K, with_bias=True)
+    c = aligned_case(M, N, K, seed=M + N + K, with_bias=True, za=8, zb=7)   # centred: outputs spread
     for i, (shift, zo, lo, hi) in enumerate([(c.shift, 0, 0, 15), (4, 3, 3, 15), (0, 8, 0, 9)]):
         rq = oracle.Requant(c.mult, shift, zo, lo, hi)
         bias = c.bias if i else None
         want = oracle.gemm_requant(c.A, c.Bt, M, N, K, c.za, c.zb, bias, rq)
         got = run_requant(q4, c, variant, rq, bias, ld_pad=0 if i == 0 else 16)
         assert (got == want).all()
-        if shift == 4:
+        if shift == 4 and K >= 100:
             assert len(np.unique(oracle.unpack_rows(got, N))) > 3   # not saturated everywhere
 
 
