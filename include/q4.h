@@ -58,7 +58,8 @@ typedef enum {
     Q4_ERR_WORKSPACE = 4,       /* workspace missing or smaller than *_workspace_bytes     */
     Q4_ERR_UNSUPPORTED = 5,     /* valid but not implemented (none at present)             */
     Q4_ERR_CUDA = 6,            /* a CUDA runtime / driver call failed                     */
-    Q4_ERR_DEVICE_TIMEOUT = 7   /* a bounded device-side wait expired                      */
+    Q4_ERR_DEVICE_TIMEOUT = 7,  /* a bounded device-side wait expired                      */
+    Q4_ERR_STATIC_SCRATCH = 8   /* problem needs more scratch than q4_conv2d_static holds  */
 } q4_status;
 
 /* Integer re-quantization of an int32 accumulator to the next layer's uint4 input.
@@ -149,6 +150,41 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                     const int32_t* colsum_w, const int32_t* bias,
                     const q4_conv_desc* d, int32_t za, int32_t zb, const q4_requant* rq,
                     uint8_t* Y, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * q4_conv2d for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of q4_conv2d, same arithmetic, same
+ * kernels, same results.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a
+ * latency-critical loop whose owner forbids allocator calls, in a plugin that is
+ * handed device pointers by a host application but owns no allocator, or in a
+ * process whose memory pool is fixed at start-up.  Such a caller cannot provide the
+ * workspace q4_conv2d asks for, so this entry point brings its own: the unrolled
+ * activation matrix and its row sums live in a fixed array compiled into the
+ * library (static __device__ storage, Q4_STATIC_SCRATCH_BYTES bytes), which every
+ * GPU that loads the library holds from load until the process exits.  The caller
+ * still passes X, Wt, the optional sums / bias, and Y.  Nothing is allocated or
+ * freed here: no cudaMalloc, no cudaFree, no allocating library routine.
+ *
+ * Limit: q4_conv2d_workspace_bytes(d) must not exceed Q4_STATIC_SCRATCH_BYTES;
+ * a larger layer is rejected with Q4_ERR_STATIC_SCRATCH before anything is launched
+ * (split the batch, or use q4_conv2d with your own workspace).
+ *
+ * First call on a device: the array's device address is looked up once per device
+ * (with that device current) on the first call; make that first call outside any
+ * stream capture.
+ *
+ * Sharing: there is ONE array per device.  Every call overwrites it and finds the
+ * previous call's contents in it; the parts that must start from zero are cleared
+ * by the call itself.  Two calls that overlap on the GPU (different streams, or
+ * different host threads) race on the array -- serialize them.
+ */
+#define Q4_STATIC_SCRATCH_BYTES (8u << 20)
+q4_status q4_conv2d_static(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
+                           const int32_t* colsum_w, const int32_t* bias,
+                           const q4_conv_desc* d, int32_t za, int32_t zb, const q4_requant* rq,
+                           uint8_t* Y, void* stream);
 
 size_t q4_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
 size_t q4_conv2d_workspace_bytes(const q4_conv_desc* d);

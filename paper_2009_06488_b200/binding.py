@@ -27,9 +27,11 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 (Q4_OK, Q4_ERR_INVALID_ARG, Q4_ERR_ALIGNMENT, Q4_ERR_RANGE, Q4_ERR_WORKSPACE,
- Q4_ERR_UNSUPPORTED, Q4_ERR_CUDA, Q4_ERR_DEVICE_TIMEOUT) = range(8)
+ Q4_ERR_UNSUPPORTED, Q4_ERR_CUDA, Q4_ERR_DEVICE_TIMEOUT, Q4_ERR_STATIC_SCRATCH) = range(9)
+Q4_STATIC_SCRATCH_BYTES = 8 << 20
 
-EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_gemm_workspace_bytes",
+EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_static",
+           "q4_gemm_workspace_bytes",
            "q4_conv2d_workspace_bytes", "q4_pack_bt", "q4_row_sums", "q4_gemm_host",
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
            "q4_launch_count", "q4_status_string", "q4_version"]
@@ -105,6 +107,8 @@ _lib.q4_gemm_requant.argtypes = [_vp, _i64, _vp, _i64, _i32, _i32, _i32, _i32, _
 _lib.q4_im2col.argtypes = [_vp, ctypes.POINTER(_ConvDesc), _i32, _vp, _i64, _vp, _vp]
 _lib.q4_conv2d.argtypes = [_vp, _vp, _i64, _vp, _vp, ctypes.POINTER(_ConvDesc), _i32, _i32,
                            ctypes.POINTER(_Requant), _vp, _vp, _sz, _vp]
+_lib.q4_conv2d_static.argtypes = [_vp, _vp, _i64, _vp, _vp, ctypes.POINTER(_ConvDesc), _i32, _i32,
+                                  ctypes.POINTER(_Requant), _vp, _vp]
 _lib.q4_gemm_workspace_bytes.argtypes = [_i32, _i32, _i32]
 _lib.q4_gemm_workspace_bytes.restype = _sz
 _lib.q4_conv2d_workspace_bytes.argtypes = [ctypes.POINTER(_ConvDesc)]
@@ -221,6 +225,19 @@ def q4_conv2d(X, Wt, d: ConvDesc, za: int, zb: int, rq: Requant, Y, ws, bias=Non
                           ctypes.byref(c), za, zb, ctypes.byref(r), _ptr(Y), _ptr(ws),
                           0 if ws is None else ws.numel() * ws.element_size(), _stream()),
            "q4_conv2d")
+    return Y
+
+
+def q4_conv2d_static(X, Wt, d: ConvDesc, za: int, zb: int, rq: Requant, Y, bias=None, colsum_w=None):
+    """q4_conv2d for callers that cannot allocate: the workspace is the library's own
+    fixed device array (Q4_STATIC_SCRATCH_BYTES).  Layers that need more are rejected
+    with Q4_ERR_STATIC_SCRATCH.  One array per device: do not overlap calls."""
+    _dev(X, torch.uint8, "X"); _dev(Wt, torch.uint8, "Wt"); _dev(Y, torch.uint8, "Y")
+    _dev(bias, torch.int32, "bias"); _dev(colsum_w, torch.int32, "colsum_w")
+    c, r = d._c(), rq._c()
+    _check(_lib.q4_conv2d_static(_ptr(X), _ptr(Wt), _rows(Wt, "Wt"), _ptr(colsum_w), _ptr(bias),
+                                 ctypes.byref(c), za, zb, ctypes.byref(r), _ptr(Y), _stream()),
+           "q4_conv2d_static")
     return Y
 
 

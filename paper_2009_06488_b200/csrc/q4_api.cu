@@ -107,6 +107,26 @@ static ConvShape conv_shape(const q4_conv_desc* d)
     return s;
 }
 
+// Scratch of q4_conv2d_static: one fixed array per device, held from library load to
+// process exit.  In host code this name is only a handle for cudaGetSymbolAddress,
+// never a device address.
+static __device__ __align__(256) unsigned char g_static_scratch[Q4_STATIC_SCRATCH_BYTES];
+
+// Device address of the static scratch on the current device (looked up once per
+// device, with that device current); nullptr if the lookup fails.
+static void* static_scratch_ptr()
+{
+    static void* ptrs[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!ptrs[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess) return nullptr;
+        ptrs[dev] = p;
+    }
+    return ptrs[dev];
+}
+
 }  // namespace q4
 
 using namespace q4;
@@ -206,6 +226,23 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     return run_gemm(p, true, st);
 }
 
+q4_status q4_conv2d_static(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
+                           const int32_t* colsum_w, const int32_t* bias,
+                           const q4_conv_desc* d, int32_t za, int32_t zb, const q4_requant* rq,
+                           uint8_t* Y, void* stream)
+{
+    q4_status s = check_conv(d, za);
+    if (s != Q4_OK) return s;
+    // the layer must fit the built-in array; nothing is launched otherwise
+    if (conv_shape(d).bytes > (size_t)Q4_STATIC_SCRATCH_BYTES) return Q4_ERR_STATIC_SCRATCH;
+    void* scratch = static_scratch_ptr();
+    if (!scratch) return Q4_ERR_CUDA;
+    // q4_conv2d rewrites the whole unrolled matrix (pad nibbles included) and zeroes
+    // the row sums before accumulating them, so stale contents cannot leak through
+    return q4_conv2d(X, Wt, ldw, colsum_w, bias, d, za, zb, rq, Y, scratch,
+                     (size_t)Q4_STATIC_SCRATCH_BYTES, stream);
+}
+
 q4_status q4_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int64_t ldb,
                      int32_t K, int32_t N, void* stream)
 {
@@ -297,6 +334,8 @@ const char* q4_status_string(q4_status s)
         case Q4_ERR_UNSUPPORTED: return "unsupported";
         case Q4_ERR_CUDA: return "CUDA error";
         case Q4_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case Q4_ERR_STATIC_SCRATCH:
+            return "layer needs more scratch than the library's built-in static array holds";
     }
     return "unknown status";
 }
