@@ -339,6 +339,62 @@ def run_ours(args):
     return 0
 
 
+def run_case(args):
+    """--case: one call of the path in a loop, for profiling a single kernel on a
+    small problem.  Prints a short JSON line (not the benchmark contract line)."""
+    import torch
+    from paper_2009_06488_b200 import binding as q4
+    from paper_2009_06488_b200 import workloads as wl
+    torch.cuda.set_device(0)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    n = args.n
+    if args.case in ("gemm", "gemm_requant"):
+        g = wl.c2(n) if n in (512, 1024, 2048, 4096, 8192) else wl.gemm_case("case", n, n, n, seed=n)
+        A, Bt = dev(g.A), dev(g.Bt)
+        C = torch.empty((n, n), dtype=torch.int32, device="cuda")
+        Cq = torch.empty((n, n // 2), dtype=torch.uint8, device="cuda")
+        rq = q4.Requant(g.mult, g.shift, 0, 0, 15)
+        if args.case == "gemm":
+            call = lambda: q4.q4_gemm(A, Bt, C, n, n, n, g.za, g.zb)
+        else:
+            call = lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, g.za, g.zb, rq)
+        units, unit = 2.0 * n ** 3 / 1e12, "TOPS"
+    else:
+        net = wl.c3(batch=n)
+        L = net.layers[0]
+        dq = q4.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
+        X, Wt = dev(net.X), dev(L.Wt)
+        ws = torch.empty(q4.q4_conv2d_workspace_bytes(dq), dtype=torch.uint8, device="cuda")
+        Y = torch.empty((dq.M, L.OC // 2), dtype=torch.uint8, device="cuda")
+        lda = (dq.K // 2 + 15) // 16 * 16
+        Amat = torch.empty((dq.M, lda), dtype=torch.uint8, device="cuda")
+        ra = torch.empty(dq.M, dtype=torch.int32, device="cuda")
+        rq = q4.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi)
+        if args.case == "conv":
+            call = lambda: q4.q4_conv2d(X, Wt, dq, L.za, L.zb, rq, Y, ws)
+            units = (X.numel() + Wt.numel() + Y.numel()) / 1e9
+        else:
+            call = lambda: q4.q4_im2col(X, dq, L.za, Amat, ra)
+            units = (X.numel() + Amat.numel() + 4 * dq.M) / 1e9
+        unit = "GB/s"
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for _ in range(args.warmup):
+        call()
+    torch.cuda.synchronize()
+    times = []
+    for _ in range(args.steps):
+        flush.zero_()                      # evict L2 between timed calls
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(); call(); e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    ms = statistics.median(times)
+    print(json.dumps({"case": args.case, "n": n, "ms_median": ms, "ms_min": min(times),
+                      "value": units / (ms * 1e-3), "unit": unit, "steps": args.steps}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -346,7 +402,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "conv", "im2col"],
+                    help="profile one call in a loop instead of the benchmark step")
+    ap.add_argument("--n", type=int, default=4096, help="GEMM edge, or conv batch, for --case")
     args = ap.parse_args()
+    if args.case:
+        return run_case(args)
     if args.impl == "reference":
         return run_reference(args)
     return run_ours(args)

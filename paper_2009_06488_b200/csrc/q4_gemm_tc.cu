@@ -34,7 +34,7 @@ constexpr int TM = 128;            // rows of A per tile (UMMA M)
 constexpr int PROW = 64;           // packed bytes per row per stage
 constexpr int UROW = 128;          // unpacked bytes per row per stage (one swizzle row)
 constexpr int SLAB = 128;          // depth values per stage
-constexpr int UW = 4;              // unpack warps
+constexpr int UW = 8;              // unpack warps
 constexpr int UT = UW * 32;        // unpack threads
 constexpr int NTHREADS = (2 + UW + 4) * 32;
 
@@ -64,6 +64,30 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {
     return (uint32_t)__cvta_generic_to_shared(p);
 }
+// Explicit shared-space accesses (32-bit shared addresses): the generic-pointer forms
+// cost an address-space lookup per access.
+__device__ __forceinline__ uint4 lds128(uint32_t a)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t a, const uint4& v)
+{
+    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};"
+                 ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ int lds32(uint32_t a)
+{
+    int v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts32(uint32_t a, int v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
@@ -88,15 +112,15 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait.  Returns false (and raises the abort flag + status word) on expiry.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_flag,
                                           unsigned* status)
 {
     if (mbar_try(bar, parity)) return true;
-    const long long limit = *abort_flag ? kWaitShort : kWaitLong;
+    const long long limit = lds32(abort_flag) ? kWaitShort : kWaitLong;
     const long long t0 = clock64();
     while (!mbar_try(bar, parity)) {
         if (clock64() - t0 > limit) {
-            *abort_flag = 1;
+            sts32(abort_flag, 1);
             atomicOr(status, kStatusTimeout);
             return false;
         }
@@ -177,8 +201,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
 
-    int32_t* sums_s = reinterpret_cast<int32_t*>(smem + C::OFF_SUMS);      // [2][ROWS]
-    int32_t* colterm_s = reinterpret_cast<int32_t*>(smem + C::OFF_COLTERM);
+    const uint32_t sums_s = sbase + C::OFF_SUMS;          // int32 [2][ROWS]
+    const uint32_t colterm_s = sbase + C::OFF_COLTERM;    // int32 [BN]
     const uint32_t bar0 = sbase + C::OFF_BAR;
     auto bar_full_p  = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto bar_empty_p = [&](int s) { return bar0 + 8u * (uint32_t)(C::STAGES + s); };
@@ -188,7 +212,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     auto bar_tempty  = [&](int a) { return bar0 + 8u * (uint32_t)(4 * C::STAGES + 2 + a); };
     auto bar_sums    = [&](int a) { return bar0 + 8u * (uint32_t)(4 * C::STAGES + 4 + a); };
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem + C::OFF_MISC);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
+    const uint32_t abort_flag = sbase + C::OFF_MISC + 4;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const GemmParams& g = p.g;
@@ -209,7 +233,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             mbar_init(bar_tempty(a), 128);
             mbar_init(bar_sums(a), UT);
         }
-        *abort_flag = 0;
+        sts32(abort_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
@@ -285,23 +309,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 mbar_wait(bar_full_p(st), ph, abort_flag, g.status);
                 mbar_wait(bar_empty_u(st), ph ^ 1u, abort_flag, g.status);
                 tc_fence_after();
-                const uint8_t* ps = smem + C::OFF_P + st * C::PSTAGE;
-                uint8_t* us = smem + C::OFF_U + st * C::USTAGE;
+                const uint32_t ps = sbase + C::OFF_P + st * C::PSTAGE;
+                const uint32_t us = sbase + C::OFF_U + st * C::USTAGE;
 #pragma unroll
                 for (int j = 0; j < C::NT; ++j) {
                     const int id = ut + j * UT;
                     const int r = id >> 2, c = id & 3;
                     if (id < C::ROWS * 4 && c < ksteps) {
-                        const uint4 w = *reinterpret_cast<const uint4*>(ps + r * PROW + c * 16);
+                        const uint4 w = lds128(ps + r * PROW + c * 16);
                         uint4 lo, hi;
                         lo.x = w.x & 0x0F0F0F0Fu; hi.x = (w.x >> 4) & 0x0F0F0F0Fu;
                         lo.y = w.y & 0x0F0F0F0Fu; hi.y = (w.y >> 4) & 0x0F0F0F0Fu;
                         lo.z = w.z & 0x0F0F0F0Fu; hi.z = (w.z >> 4) & 0x0F0F0F0Fu;
                         lo.w = w.w & 0x0F0F0F0Fu; hi.w = (w.w >> 4) & 0x0F0F0F0Fu;
-                        uint8_t* row = us + r * UROW;
+                        const uint32_t row = us + r * UROW;
                         const int sw = r & 7;
-                        *reinterpret_cast<uint4*>(row + (((2 * c) ^ sw) << 4)) = lo;
-                        *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ sw) << 4)) = hi;
+                        sts128(row + (((2 * c) ^ sw) << 4), lo);
+                        sts128(row + (((2 * c + 1) ^ sw) << 4), hi);
                         if (need_sums) {
                             int t = psum[j];
                             t = dp4a_u8(lo.x + hi.x, 0x01010101u, t);
@@ -327,7 +351,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 1);
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
                     const int id = ut + j * UT;
-                    if (id < C::ROWS * 4 && (id & 3) == 0) sums_s[acc * C::ROWS + (id >> 2)] = t;
+                    if (id < C::ROWS * 4 && (id & 3) == 0)
+                        sts32(sums_s + 4 * (acc * C::ROWS + (id >> 2)), t);
                 }
                 mbar_arrive(bar_sums(acc));
             }
@@ -351,13 +376,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int n = n0 + j;
                 int cb = 0, bias = 0;
                 if (n < g.N) {
-                    cb = need_cb ? sums_s[acc * C::ROWS + TM + j] : g.colsum_b[n];
+                    cb = need_cb ? lds32(sums_s + 4 * (acc * C::ROWS + TM + j)) : g.colsum_b[n];
                     if (REQUANT && g.bias) bias = g.bias[n];
                 }
-                colterm_s[j] = (int)((uint32_t)kzz - (uint32_t)(g.za * cb) + (uint32_t)bias);
+                sts32(colterm_s + 4 * j, (int)((uint32_t)kzz - (uint32_t)(g.za * cb) + (uint32_t)bias));
             }
             int ra = 0;
-            if (need_ra) ra = sums_s[acc * C::ROWS + row];
+            if (need_ra) ra = lds32(sums_s + 4 * (acc * C::ROWS + row));
             else if (m < g.M) ra = g.rowsum_a[m];
             const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
             asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -373,7 +398,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 tc_ld32(taddr0 + (uint32_t)(ch * 32), r);
                 tc_wait_ld();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) r[j] = r[j] + rowterm + (uint32_t)colterm_s[ch * 32 + j];
+                for (int q = 0; q < 8; ++q) {
+                    const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * q));
+                    r[4 * q + 0] += rowterm + ct.x;
+                    r[4 * q + 1] += rowterm + ct.y;
+                    r[4 * q + 2] += rowterm + ct.z;
+                    r[4 * q + 3] += rowterm + ct.w;
+                }
                 if (m < g.M) {
                     const bool full = (nc + 32 <= g.N);
                     if (!REQUANT) {
