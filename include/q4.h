@@ -223,10 +223,26 @@ size_t q4_gemm_host_staging_bytes(int32_t M, int32_t N, int32_t K,
 q4_status q4_last_device_status(void* stream);
 
 /* Kernel selection for ablations and tests: 0 = automatic, 1 = general (SIMT)
- * kernels only, 2 = tensor-core kernels wherever their alignment rules hold.
- * Returns the previous value.  Process-wide; also read once from the environment
- * variable Q4_FORCE_VARIANT ("simt" / "tc"). */
+ * kernels only, 2 = tensor-core kernels or an error where their alignment rules do
+ * not hold, 3 = like 2 but never the CTA-pair kernel.  Returns the previous value.
+ * Process-wide; also read once from the environment variable Q4_FORCE_VARIANT
+ * ("simt" / "tc" / "tc1"). */
 int q4_set_variant(int variant);
+
+/*
+ * Measurement helper (no counterpart in the paper): the tensor pipe's issue peak on
+ * this device.  Launches num_ctas CTAs (one per SM is the intended use); each issues
+ * 4 * iters back-to-back tcgen05.mma instructions of shape 128 x n x (32 bytes of
+ * depth) on zero operands resident in shared memory and writes the elapsed SM clocks
+ * to cycles_dev[cta] (device pointer, num_ctas entries).  kind: 0 = kind::i8
+ * (u8 x u8 -> s32), 1 = kind::f16 (bf16 -> f32), 2 = kind::f8f6f4 (e4m3 -> f32),
+ * 3 = kind::i8 issued by CTA pairs (cta_group::2, 256 x n per instruction; num_ctas
+ * even, n a multiple of 32, one cycles_dev entry per pair, count 256 rows).
+ * n: multiple of 16 in 16..256.  Multiply-accumulates per clock per SM =
+ * 4 * iters * 128 * n * k / cycles, k = 32 for the 8-bit kinds and 16 for bf16.
+ */
+q4_status q4_measure_mma_peak(int kind, int n, int iters, unsigned long long* cycles_dev,
+                              int num_ctas, void* stream);
 
 /* Number of kernels this library has launched in this process (all streams). */
 uint64_t q4_launch_count(void);

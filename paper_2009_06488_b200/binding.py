@@ -34,7 +34,7 @@ EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_st
            "q4_gemm_workspace_bytes",
            "q4_conv2d_workspace_bytes", "q4_pack_bt", "q4_row_sums", "q4_gemm_host",
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
-           "q4_launch_count", "q4_status_string", "q4_version"]
+           "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak"]
 
 
 class Q4Error(RuntimeError):
@@ -119,6 +119,7 @@ _lib.q4_gemm_host.argtypes = [_vp, _i64, _vp, _i64, _vp, _i64, _i32, _i32, _i32,
                               _vp, _sz, _vp]
 _lib.q4_gemm_host_staging_bytes.argtypes = [_i32, _i32, _i32, _i64, _i64, _i64]
 _lib.q4_gemm_host_staging_bytes.restype = _sz
+_lib.q4_measure_mma_peak.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, _vp, ctypes.c_int, _vp]
 _lib.q4_last_device_status.argtypes = [_vp]
 _lib.q4_set_variant.argtypes = [ctypes.c_int]
 _lib.q4_launch_count.restype = ctypes.c_uint64
@@ -173,6 +174,22 @@ def q4_launch_count() -> int:
 
 def q4_last_device_status() -> int:
     return _lib.q4_last_device_status(_stream())
+
+
+def q4_measure_mma_peak(kind: int, n: int = 256, iters: int = 2048, num_ctas: int | None = None):
+    """Multiply-accumulates per clock per SM of back-to-back tcgen05.mma (median over
+    CTAs); kind 0 = i8, 1 = bf16, 2 = e4m3, 3 = i8 issued by CTA pairs.  Returns (mac_per_clk_per_sm, cycles_median)."""
+    if num_ctas is None:
+        num_ctas = torch.cuda.get_device_properties(torch.cuda.current_device()).multi_processor_count
+    if kind == 3:
+        num_ctas -= num_ctas % 2
+    cycles = torch.zeros(num_ctas // 2 if kind == 3 else num_ctas, dtype=torch.int64, device="cuda")
+    _check(_lib.q4_measure_mma_peak(kind, n, iters, _ptr(cycles), num_ctas, _stream()),
+           "q4_measure_mma_peak")
+    torch.cuda.synchronize()
+    med = float(cycles.double().median().item())
+    k = 16 if kind == 1 else 32
+    return 4.0 * iters * 128 * n * k / med, med      # per SM: a pair instruction is 128 rows per SM
 
 
 def q4_gemm_workspace_bytes(M: int, N: int, K: int) -> int:

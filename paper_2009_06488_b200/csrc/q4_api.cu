@@ -23,6 +23,7 @@ static int variant()
         v = 0;
         if (e && !std::strcmp(e, "simt")) v = 1;
         if (e && !std::strcmp(e, "tc")) v = 2;
+        if (e && !std::strcmp(e, "tc1")) v = 3;
         g_variant.store(v, std::memory_order_relaxed);
     }
     return v;
@@ -41,6 +42,8 @@ static unsigned* status_ptr()
     }
     return ptrs[dev];
 }
+
+unsigned* device_status_ptr() { return status_ptr(); }
 
 static q4_status check_gemm(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
                             int32_t M, int32_t N, int32_t K, int32_t za, int32_t zb)
@@ -69,8 +72,9 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st)
     p.status = status_ptr();
     if (!p.status) return Q4_ERR_CUDA;
     const int v = variant();
+    if (v != 1 && v != 3 && gemm_tc_pair_supported(p)) return launch_gemm_tc_pair(p, rq, st);
     if (v != 1 && gemm_tc_supported(p)) return launch_gemm_tc(p, rq, st);
-    if (v == 2) return Q4_ERR_ALIGNMENT;
+    if (v == 2 || v == 3) return Q4_ERR_ALIGNMENT;
     return launch_gemm_simt(p, rq, st) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
@@ -317,7 +321,7 @@ q4_status q4_last_device_status(void* stream)
 int q4_set_variant(int v)
 {
     const int prev = variant();
-    g_variant.store((v == 1 || v == 2) ? v : 0, std::memory_order_relaxed);
+    g_variant.store((v >= 1 && v <= 3) ? v : 0, std::memory_order_relaxed);
     return prev;
 }
 

@@ -27,6 +27,7 @@
 #include <mutex>
 
 #include "q4_common.cuh"
+#include "q4_tc_ptx.cuh"
 
 namespace q4 {
 
@@ -37,9 +38,6 @@ constexpr int SLAB = 128;          // depth values per stage
 constexpr int UW = 8;              // unpack warps
 constexpr int UT = UW * 32;        // unpack threads
 constexpr int NTHREADS = (2 + UW + 4) * 32;
-
-constexpr long long kWaitLong = 4000000000ll;   // ~2 s at 2 GHz
-constexpr long long kWaitShort = 2000000ll;     // ~1 ms, used once the kernel aborts
 
 template <int BN> struct Cfg {
     static constexpr int ROWS = TM + BN;
@@ -59,125 +57,6 @@ template <int BN> struct Cfg {
     static constexpr int SMEM = OFF_MISC + 16 + 1024;          // + slack to align the base
 };
 
-// ---- PTX wrappers -------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p)
-{
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-// Explicit shared-space accesses (32-bit shared addresses): the generic-pointer forms
-// cost an address-space lookup per access.
-__device__ __forceinline__ uint4 lds128(uint32_t a)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ void sts128(uint32_t a, const uint4& v)
-{
-    asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};"
-                 ::"r"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ int lds32(uint32_t a)
-{
-    int v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
-    return v;
-}
-__device__ __forceinline__ void sts32(uint32_t a, int v)
-{
-    asm volatile("st.shared.u32 [%0], %1;" ::"r"(a), "r"(v) : "memory");
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false (and raises the abort flag + status word) on expiry.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t abort_flag,
-                                          unsigned* status)
-{
-    if (mbar_try(bar, parity)) return true;
-    const long long limit = lds32(abort_flag) ? kWaitShort : kWaitLong;
-    const long long t0 = clock64();
-    while (!mbar_try(bar, parity)) {
-        if (clock64() - t0 > limit) {
-            sts32(abort_flag, 1);
-            atomicOr(status, kStatusTimeout);
-            return false;
-        }
-    }
-    return true;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
-                                            uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after()  { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                 ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem], u8 x u8 -> s32, shape 128 x N x 32.
-__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
-                                          uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
-          "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
-          "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]),
-          "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]),
-          "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// K-major, 128-byte swizzle shared-memory matrix descriptor: 8-row groups 1024 bytes
-// apart, descriptor version 1 (sm_100).
-__device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t saddr)
-{
-    return (uint64_t)((saddr & 0x3FFFFu) >> 4)
-         | (1ull << 16)                 // leading byte offset (unused for swizzled K-major)
-         | ((uint64_t)(1024 >> 4) << 32)  // stride byte offset: next 8-row group
-         | (1ull << 46)                 // descriptor version
-         | (2ull << 61);                // SWIZZLE_128B
-}
 // Instruction descriptor: D = s32, A = B = unsigned 8-bit, both K-major, M = 128, N = BN.
 __host__ __device__ constexpr uint32_t make_idesc_u8(int n)
 {
@@ -224,8 +103,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(bar_full_p(s), 1);
-            mbar_init(bar_empty_p(s), UT);
-            mbar_init(bar_full_u(s), UT);
+            mbar_init(bar_empty_p(s), UW);   // one arrive per unpack warp
+            mbar_init(bar_full_u(s), UW);
             mbar_init(bar_empty_u(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -336,9 +215,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     }
                 }
+                // every lane publishes its own writes to the async proxy; one lane per warp
+                // then arrives (256 arrives on one barrier word serialise badly)
                 fence_async_smem();
-                mbar_arrive(bar_full_u(st));
-                mbar_arrive(bar_empty_p(st));
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(bar_full_u(st));
+                    mbar_arrive(bar_empty_p(st));
+                }
             }
             if (need_sums) {
                 const int acc = lt & 1;
@@ -477,7 +361,7 @@ static EncodeTiledFn get_encode()
 
 // Packed matrix [rows x kbytes] with pitch ld, box = 64 bytes x box_rows; out-of-range
 // rows and bytes are filled with zeros (zero nibbles add nothing to any term of Eq. 2).
-static bool make_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows, int kbytes,
+bool make_packed_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows, int kbytes,
                      int box_rows)
 {
     EncodeTiledFn enc = get_encode();
@@ -523,8 +407,8 @@ static q4_status launch_bn(const GemmParams& g, bool rq, cudaStream_t st)
     p.cq_vec = (rq && ((uintptr_t)g.Cq % 16 == 0) && (g.ldcq % 16 == 0)) ? 1 : 0;
 
     CUtensorMap tmA, tmB;
-    if (!make_map(&tmA, g.A, g.lda, g.M, kbytes, TM)) return Q4_ERR_CUDA;
-    if (!make_map(&tmB, g.Bt, g.ldb, g.N, kbytes, BN)) return Q4_ERR_CUDA;
+    if (!make_packed_map(&tmA, g.A, g.lda, g.M, kbytes, TM)) return Q4_ERR_CUDA;
+    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, BN)) return Q4_ERR_CUDA;
 
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
     const int grid = (int)(tiles < sm_count() ? tiles : sm_count());

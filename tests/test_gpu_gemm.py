@@ -8,7 +8,7 @@ from paper_2009_06488_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
-SIMT, TC = 1, 2
+SIMT, TC, TC1 = 1, 2, 3      # general kernel / tensor-core (auto) / single-CTA tensor-core only
 
 
 @pytest.fixture(scope="module")
@@ -91,6 +91,27 @@ def test_tc_gemm_matches_oracle(q4, shape):
     assert (got == want).all()
     got2, _, _ = run_gemm(q4, c, TC, ldc_pad=1)      # unaligned int32 pitch: scalar stores
     assert (got2 == want).all()
+
+
+# shapes that reach the CTA-pair kernel (M, N >= 256): tails in M, N, K; short depths
+PAIR_SHAPES = [(256, 256, 128), (300, 260, 1000), (257, 514, 129), (1000, 300, 4096), (512, 768, 64),
+               (384, 512, 33), (2048, 256, 640)]
+
+
+@pytest.mark.parametrize("variant", [TC, TC1])
+@pytest.mark.parametrize("shape", PAIR_SHAPES)
+def test_pair_and_single_tensor_core_kernels_agree_with_oracle(q4, variant, shape):
+    M, N, K = shape
+    c = aligned_case(M, N, K, seed=M * 31 + N * 7 + K, with_bias=True)
+    want = oracle.gemm(c.A, c.Bt, M, N, K, c.za, c.zb)
+    got, _, _ = run_gemm(q4, c, variant, ldc_pad=4)
+    assert (got == want).all()
+    got, _, _ = run_gemm(q4, c, variant, sums=True)
+    assert (got == want).all()
+    rq = oracle.Requant(c.mult, 6, 4, 4, 15)
+    wantq = oracle.requant_matrix(want, c.bias, rq)
+    assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=16) == wantq).all()
+    assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=3) == wantq).all()   # byte stores
 
 
 @pytest.mark.parametrize("variant", [SIMT, TC])
