@@ -361,8 +361,10 @@ static EncodeTiledFn get_encode()
 
 // Packed matrix [rows x kbytes] with pitch ld, box = 64 bytes x box_rows; out-of-range
 // rows and bytes are filled with zeros (zero nibbles add nothing to any term of Eq. 2).
+// swizzle64: the 16-byte chunks of each 64-byte row are XOR-permuted by (row / 2) % 4 in
+// shared memory, which makes one-row-per-lane reads bank-conflict free.
 bool make_packed_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows, int kbytes,
-                     int box_rows)
+                     int box_rows, bool swizzle64)
 {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
@@ -371,7 +373,8 @@ bool make_packed_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows,
     cuuint32_t box[2] = {(cuuint32_t)PROW, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides,
-               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               swizzle64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_NONE,
                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -407,8 +410,8 @@ static q4_status launch_bn(const GemmParams& g, bool rq, cudaStream_t st)
     p.cq_vec = (rq && ((uintptr_t)g.Cq % 16 == 0) && (g.ldcq % 16 == 0)) ? 1 : 0;
 
     CUtensorMap tmA, tmB;
-    if (!make_packed_map(&tmA, g.A, g.lda, g.M, kbytes, TM)) return Q4_ERR_CUDA;
-    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, BN)) return Q4_ERR_CUDA;
+    if (!make_packed_map(&tmA, g.A, g.lda, g.M, kbytes, TM, false)) return Q4_ERR_CUDA;
+    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, BN, false)) return Q4_ERR_CUDA;
 
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
     const int grid = (int)(tiles < sm_count() ? tiles : sm_count());

@@ -1,24 +1,33 @@
-// Tensor-core 4-bit quantized GEMM for large problems: CTA pairs (thread-block clusters
-// of two) computing 256 x 256 output tiles with tcgen05.mma.cta_group::2 (Eq. 2 of the
-// paper, all four terms).
+// Tensor-core 4-bit quantized GEMM for large problems (Eq. 2 of the paper, all four
+// terms): CTA pairs computing 256 x 192 output tiles with tcgen05.mma.cta_group::2, the
+// A operand fed from tensor memory.
 //
-// Each CTA of a pair owns 128 rows of A and 128 of the tile's 256 rows of Bt; the pair
-// MMA reads A from both CTAs and shares the two halves of Bt between them, so every
-// CTA stages and unpacks only half of the Bt tile -- the step that bounds the
-// single-CTA kernel (the unpack is a shared-memory-bandwidth problem).  The
-// accumulator (256 x 256 int32) lives in the two CTAs' tensor memory, 128 rows each,
-// double-buffered, so each CTA's epilogue of tile t overlaps the main loop of t+1.
+// Why this shape.  The unpack (nibbles -> bytes) is bounded by the shared-memory
+// load/store pipe, 128 B/clk: every packed byte is read once and every unpacked byte
+// written once before the MMA can read it.  Two things cut that traffic:
+//   * a CTA pair shares the Bt tile, so each CTA stages and unpacks only half of it;
+//   * the unpacked A rows never touch shared memory: each unpack thread owns one row,
+//     expands its 64 packed bytes in registers and writes them to tensor memory
+//     (tcgen05.st), from where the MMA reads A directly.
+// Per 128-deep stage a CTA then moves 8 KB (A, loads only) + 6 KB + 12 KB (Bt, loads and
+// stores) through the load/store pipe -- about half of what the MMA's 384 clocks allow.
 //
-// Roles per CTA (14 warps): warp 0 TMA producer (its own rows of A and Bt, no
-// multicast); warps 2..9 unpack nibbles to bytes in the K-major 128-byte-swizzled
-// layout and take the depth sums; warp 1 of the leader CTA issues the pair MMAs and
-// commits to the barriers of both CTAs; warp 1 of the peer CTA relays "my operands are
-// ready" / "my accumulator is drained" to the leader with one remote arrive each;
-// warps 10..13 epilogue.  Column sums of the two Bt halves are exchanged through
-// distributed shared memory.
+// Tensor memory (512 columns): two accumulators of 192 columns (the epilogue of tile t
+// overlaps the main loop of t+1) and four A stages of 32 columns (128 depth bytes).
 //
-// Every mbarrier wait is bounded (see q4_tc_ptx.cuh); the only unbounded waits are the
-// two cluster barriers at entry and exit, which every thread reaches unconditionally.
+// Roles per CTA (14 warps): warp 0 TMA producer (its own 128 rows of A, 64-byte-swizzled
+// so that row-per-lane reads are conflict-free, and its own 96 rows of Bt; no
+// multicast); warps 2..9 unpack, as two groups of four that take alternate stages so
+// one group's waits and fences hide behind the other's work, and arrive -- from both
+// CTAs -- on the leader CTA's "operands ready" barrier; warp 1 of the leader CTA issues
+// the pair MMAs and commits to both CTAs' barriers; warp 1 of the peer CTA relays
+// "accumulator drained" once per tile; warps 10..13 epilogue.  Column sums of the two
+// Bt halves are exchanged through distributed shared memory.
+//
+// The depth order inside each 32-value group (even nibbles, then odd) is the same for A
+// and Bt, so the product is unchanged.  Every mbarrier wait is bounded; the only
+// unbounded waits are the cluster barriers at entry and exit, which every thread
+// reaches unconditionally.
 #include <cuda.h>
 
 #include "q4_common.cuh"
@@ -28,31 +37,37 @@ namespace q4 {
 namespace pair {
 
 constexpr int TMC = 128;             // rows of A per CTA
-constexpr int BNC = 256;             // columns of the pair tile
+constexpr int BNC = 192;             // columns of the pair tile
 constexpr int BH = BNC / 2;          // rows of Bt staged per CTA
-constexpr int ROWS = TMC + BH;       // rows unpacked per CTA per stage
 constexpr int PROW = 64, UROW = 128, SLAB = 128;
-constexpr int PSTAGE = ROWS * PROW;  // 16 KB
-constexpr int USTAGE = ROWS * UROW;  // 32 KB
-constexpr int STAGES = 4;
-constexpr int UW = 8, UT = UW * 32;
-constexpr int NT = ROWS * 4 / UT;    // unpack tasks per thread per stage
+constexpr int PS = 6;                // packed stages (A 8 KB + Bt 6 KB)
+constexpr int US = 4;                // operand stages (Bt bytes in smem, A bytes in TMEM)
+constexpr int PA = TMC * PROW;       // packed A bytes per stage
+constexpr int PSTAGE = PA + BH * PROW;
+constexpr int BSTAGE = BH * UROW;    // unpacked Bt bytes per stage
+constexpr int G = 2, WPG = 4, GT = WPG * 32;   // unpack groups, warps / threads per group
+constexpr int UW = G * WPG;
+constexpr int NTB = BH * 4 / GT;     // Bt tasks (16-byte packed chunks) per thread per stage
 constexpr int NTHREADS = (2 + UW + 4) * 32;
 constexpr int TMEM_COLS = 512;
-constexpr int SUMS_N = TMC + BNC;    // per buffer: 128 row sums, 256 column sums
+constexpr int ACOL0 = 2 * BNC;       // first TMEM column of the A stages
+constexpr int SUMS_N = TMC + BNC;    // per buffer and group: 128 row sums, BNC column sums
 
-constexpr int OFF_U = 0;
-constexpr int OFF_P = OFF_U + STAGES * USTAGE;
-constexpr int OFF_SUMS = OFF_P + STAGES * PSTAGE;
-constexpr int OFF_COLTERM = OFF_SUMS + 2 * SUMS_N * 4;
+constexpr int OFF_B = 0;
+constexpr int OFF_P = OFF_B + US * BSTAGE;
+constexpr int OFF_SUMS = OFF_P + PS * PSTAGE;
+constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
 constexpr int OFF_BAR = OFF_COLTERM + BNC * 4;
-constexpr int NBAR = 5 * STAGES + 10;
+constexpr int NBAR = 2 * PS + 2 * US + 10;
 constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
 constexpr int SMEM = OFF_MISC + 16 + 1024;
 
-static_assert(ROWS * 4 % UT == 0, "unpack tasks must divide evenly");
+static_assert(BH * 4 % GT == 0, "Bt tasks must divide evenly");
+static_assert(2 * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
+static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
+static_assert(US % G == 0, "a group always meets the same operand stages");
 
-// D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = 256.
+// D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC.
 constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)(BNC >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
 struct Params {
@@ -60,6 +75,20 @@ struct Params {
     int32_t tiles_m, tiles_n, nslab;
     int32_t c_vec, cq_vec;
 };
+
+__device__ __forceinline__ void unpack16(const uint4& w, uint4& lo, uint4& hi)
+{
+    lo.x = w.x & 0x0F0F0F0Fu; hi.x = (w.x >> 4) & 0x0F0F0F0Fu;
+    lo.y = w.y & 0x0F0F0F0Fu; hi.y = (w.y >> 4) & 0x0F0F0F0Fu;
+    lo.z = w.z & 0x0F0F0F0Fu; hi.z = (w.z >> 4) & 0x0F0F0F0Fu;
+    lo.w = w.w & 0x0F0F0F0Fu; hi.w = (w.w >> 4) & 0x0F0F0F0Fu;
+}
+// Sum of the 32 values of one unpacked chunk (bytes of the word sum stay <= 120).
+__device__ __forceinline__ int chunk_sum(const uint4& lo, const uint4& hi, int acc)
+{
+    const uint32_t t = (lo.x + hi.x) + (lo.y + hi.y) + (lo.z + hi.z) + (lo.w + hi.w);
+    return dp4a_u8(t, 0x01010101u, acc);
+}
 
 template <bool REQUANT>
 __global__ void __launch_bounds__(NTHREADS, 1)
@@ -70,19 +99,19 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // the same offset in both CTAs: dynamic shared memory starts at the same address
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
 
-    const uint32_t sums_s = sbase + OFF_SUMS;        // int32 [2][SUMS_N]
+    const uint32_t sums_s = sbase + OFF_SUMS;        // int32 [2 buffers][G][SUMS_N]
     const uint32_t colterm_s = sbase + OFF_COLTERM;  // int32 [BNC]
     const uint32_t bar0 = sbase + OFF_BAR;
     auto bar_full_p    = [&](int s) { return bar0 + 8u * (uint32_t)s; };
-    auto bar_empty_p   = [&](int s) { return bar0 + 8u * (uint32_t)(STAGES + s); };
-    auto bar_full_u    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * STAGES + s); };
-    auto bar_empty_u   = [&](int s) { return bar0 + 8u * (uint32_t)(3 * STAGES + s); };
-    auto bar_peer_full = [&](int s) { return bar0 + 8u * (uint32_t)(4 * STAGES + s); };
-    auto bar_tfull     = [&](int a) { return bar0 + 8u * (uint32_t)(5 * STAGES + a); };
-    auto bar_tempty    = [&](int a) { return bar0 + 8u * (uint32_t)(5 * STAGES + 2 + a); };
-    auto bar_peer_tempty = [&](int a) { return bar0 + 8u * (uint32_t)(5 * STAGES + 4 + a); };
-    auto bar_sums      = [&](int a) { return bar0 + 8u * (uint32_t)(5 * STAGES + 6 + a); };
-    auto bar_tstart    = [&](int a) { return bar0 + 8u * (uint32_t)(5 * STAGES + 8 + a); };
+    auto bar_empty_p   = [&](int s) { return bar0 + 8u * (uint32_t)(PS + s); };
+    auto bar_full_u    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + s); };
+    auto bar_empty_u   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + US + s); };
+    const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US);
+    auto bar_tfull       = [&](int a) { return barT + 8u * (uint32_t)a; };
+    auto bar_tempty      = [&](int a) { return barT + 8u * (uint32_t)(2 + a); };
+    auto bar_peer_tempty = [&](int a) { return barT + 8u * (uint32_t)(4 + a); };
+    auto bar_sums        = [&](int a) { return barT + 8u * (uint32_t)(6 + a); };
+    auto bar_tstart      = [&](int a) { return barT + 8u * (uint32_t)(8 + a); };
     const uint32_t tmem_slot = sbase + OFF_MISC;
     const uint32_t abort_flag = sbase + OFF_MISC + 4;
 
@@ -97,18 +126,19 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int ntiles = p.tiles_m * p.tiles_n;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
+        for (int s = 0; s < PS; ++s) {
             mbar_init(bar_full_p(s), 1);
-            mbar_init(bar_empty_p(s), UW);   // one arrive per unpack warp
-            mbar_init(bar_full_u(s), UW);
+            mbar_init(bar_empty_p(s), WPG);      // one arrive per warp of the group that took it
+        }
+        for (int s = 0; s < US; ++s) {
+            mbar_init(bar_full_u(s), 2 * WPG);   // used in the leader: a group's warps of both CTAs
             mbar_init(bar_empty_u(s), 1);
-            mbar_init(bar_peer_full(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull(a), 1);
             mbar_init(bar_tempty(a), 128);
             mbar_init(bar_peer_tempty(a), 1);
-            mbar_init(bar_sums(a), 2 * UW);       // one arrive per unpack warp of each CTA
+            mbar_init(bar_sums(a), 2 * UW);      // one arrive per unpack warp of each CTA
             mbar_init(bar_tstart(a), 1);
         }
         sts32(abort_flag, 0);
@@ -134,19 +164,23 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const int arow = tm * 256 + (int)rank * TMC;
                 const int brow = tn * BNC + (int)rank * BH;
                 for (int s = 0; s < p.nslab; ++s, ++it) {
-                    const int st = it % STAGES;
-                    const uint32_t ph = (it / STAGES) & 1u;
+                    const int st = it % PS;
+                    const uint32_t ph = (it / PS) & 1u;
                     mbar_wait_cl(bar_empty_p(st), ph ^ 1u, abort_flag, g.status);
                     mbar_expect_tx(bar_full_p(st), (uint32_t)PSTAGE);
                     const uint32_t dst = sbase + OFF_P + st * PSTAGE;
                     tma_load_2d(dst, &tmA, s * PROW, arow, bar_full_p(st));
-                    tma_load_2d(dst + TMC * PROW, &tmB, s * PROW, brow, bar_full_p(st));
+                    tma_load_2d(dst + PA, &tmB, s * PROW, brow, bar_full_p(st));
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
+        if (rank == 0) {
             // -------------------------------------------------------- pair MMA issuer
+            // The whole warp runs the loop (uniform control flow and addresses); one
+            // elected lane issues the MMAs and commits.
+            const uint32_t a_tmem0 = tmem_base + (uint32_t)ACOL0;
+            const uint64_t bdesc0 = make_kmajor_sw128_desc(sbase + OFF_B);
             uint32_t it = 0, lt = 0;
             for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
                 const int acc = lt & 1;
@@ -155,29 +189,40 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (lt >= 2) mbar_wait_cl(bar_peer_tempty(acc), aph ^ 1u, abort_flag, g.status);
                 tc_fence_after();
                 // both epilogues are done with buffer `acc`: tell the unpack warps of both CTAs
-                tc_commit_pair(bar_tstart(acc), 3);
+                if (elect_one()) tc_commit_pair(bar_tstart(acc), 3);
+                __syncwarp();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BNC);
                 for (int s = 0; s < p.nslab; ++s, ++it) {
-                    const int st = it % STAGES;
-                    const uint32_t ph = (it / STAGES) & 1u;
+                    const int st = it % US;
+                    const uint32_t ph = (it / US) & 1u;
                     mbar_wait_cl(bar_full_u(st), ph, abort_flag, g.status);
-                    mbar_wait_cl(bar_peer_full(st), ph, abort_flag, g.status);
                     tc_fence_after();
-                    const uint32_t ua = sbase + OFF_U + st * USTAGE;
-                    const uint64_t adesc = make_kmajor_sw128_desc(ua);
-                    const uint64_t bdesc = make_kmajor_sw128_desc(ua + TMC * UROW);
+                    const uint32_t a_tmem = a_tmem0 + (uint32_t)(st * 32);
+                    const uint64_t bdesc = bdesc0 + (uint64_t)(st * (BSTAGE >> 4));
                     const int rem = g.K - s * SLAB;
-                    const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
-                    for (int i = 0; i < ksteps; ++i)
-                        tc_mma_i8_pair(d_tmem, adesc + (uint64_t)(2 * i), bdesc + (uint64_t)(2 * i),
-                                       kIdesc, (s > 0 || i > 0) ? 1u : 0u);
-                    tc_commit_pair(bar_empty_u(st), 3);
+                    if (elect_one()) {
+                        if (rem >= SLAB) {
+                            tc_mma_i8_pair_ts(d_tmem, a_tmem, bdesc, kIdesc, s > 0 ? 1u : 0u);
+                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 8u, bdesc + 2u, kIdesc, 1u);
+                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 16u, bdesc + 4u, kIdesc, 1u);
+                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 24u, bdesc + 6u, kIdesc, 1u);
+                        } else {
+                            const int ksteps = (rem + 31) / 32;
+                            for (int i = 0; i < ksteps; ++i)
+                                tc_mma_i8_pair_ts(d_tmem, a_tmem + (uint32_t)(8 * i),
+                                                  bdesc + (uint64_t)(2 * i), kIdesc,
+                                                  (s > 0 || i > 0) ? 1u : 0u);
+                        }
+                        tc_commit_pair(bar_empty_u(st), 3);
+                    }
+                    __syncwarp();
                 }
-                tc_commit_pair(bar_tfull(acc), 3);
+                if (elect_one()) tc_commit_pair(bar_tfull(acc), 3);
+                __syncwarp();
             }
         } else if (lane == 0) {
-            // -------------------------------------------------------- peer relay
-            uint32_t it = 0, lt = 0;
+            // -------------------------------------------------------- peer relay (per tile)
+            uint32_t lt = 0;
             for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
                 const int acc = lt & 1;
                 const uint32_t aph = (lt >> 1) & 1u;
@@ -185,64 +230,89 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     mbar_wait_cl(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
                     mbar_arrive_cluster(map_to_cta(bar_peer_tempty(acc), 0));
                 }
-                for (int s = 0; s < p.nslab; ++s, ++it) {
-                    const int st = it % STAGES;
-                    const uint32_t ph = (it / STAGES) & 1u;
-                    mbar_wait_cl(bar_full_u(st), ph, abort_flag, g.status);
-                    mbar_arrive_cluster(map_to_cta(bar_peer_full(st), 0));
-                }
             }
         }
     } else if (warp < 2 + UW) {
         // ------------------------------------------------------------ unpack warps
-        const int ut = threadIdx.x - 64;
+        const int grp = (warp - 2) / WPG;               // takes the stages with it % G == grp
+        const int gt = threadIdx.x - 64 - grp * GT;     // 0..127 inside the group
+        const int q = warp & 3;                         // TMEM lane quarter of this warp
+        const int arow = q * 32 + lane;                 // row of A owned by this thread
+        const uint32_t a_sw = (uint32_t)((arow >> 1) & 3);            // 64-byte TMA swizzle
+        const uint32_t a_off = (uint32_t)(arow * PROW);
+        const uint32_t a_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ACOL0;
+        const uint32_t full_u_leader = map_to_cta(bar_full_u(0), 0);  // barrier in the leader CTA
         uint32_t it = 0, lt = 0;
         for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
-            int psum[NT];
+            int psum_a = 0;
+            int psum_b[NTB];
 #pragma unroll
-            for (int j = 0; j < NT; ++j) psum[j] = 0;
+            for (int j = 0; j < NTB; ++j) psum_b[j] = 0;
             for (int s = 0; s < p.nslab; ++s, ++it) {
-                const int st = it % STAGES;
-                const uint32_t ph = (it / STAGES) & 1u;
+                if ((int)(it % G) != grp) continue;
+                const int pst = it % PS, ust = it % US;
+                const uint32_t pph = (it / PS) & 1u, uph = (it / US) & 1u;
                 const int rem = g.K - s * SLAB;
                 const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
-                mbar_wait_cl(bar_full_p(st), ph, abort_flag, g.status);
-                mbar_wait_cl(bar_empty_u(st), ph ^ 1u, abort_flag, g.status);
-                tc_fence_after();
-                const uint32_t ps = sbase + OFF_P + st * PSTAGE;
-                const uint32_t us = sbase + OFF_U + st * USTAGE;
+                mbar_wait_cl(bar_full_p(pst), pph, abort_flag, g.status);
+                const uint32_t ps = sbase + OFF_P + pst * PSTAGE;
+                // all shared-memory loads first, so their latencies overlap
+                uint4 wa[4], wb[NTB];
 #pragma unroll
-                for (int j = 0; j < NT; ++j) {
-                    const int id = ut + j * UT;
-                    const int r = id >> 2, c = id & 3;
+                for (int c = 0; c < 4; ++c)
+                    if (c < ksteps) wa[c] = lds128(ps + a_off + (((uint32_t)c ^ a_sw) << 4));
+#pragma unroll
+                for (int j = 0; j < NTB; ++j) {
+                    const int id = gt + j * GT;
+                    if ((id & 3) < ksteps) wb[j] = lds128(ps + PA + (id >> 2) * PROW + (id & 3) * 16);
+                }
+                // expand in registers while the operand stage may still be in use
+                uint4 alo[4], ahi[4], blo[NTB], bhi[NTB];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
                     if (c < ksteps) {
-                        const uint4 w = lds128(ps + r * PROW + c * 16);
-                        uint4 lo, hi;
-                        lo.x = w.x & 0x0F0F0F0Fu; hi.x = (w.x >> 4) & 0x0F0F0F0Fu;
-                        lo.y = w.y & 0x0F0F0F0Fu; hi.y = (w.y >> 4) & 0x0F0F0F0Fu;
-                        lo.z = w.z & 0x0F0F0F0Fu; hi.z = (w.z >> 4) & 0x0F0F0F0Fu;
-                        lo.w = w.w & 0x0F0F0F0Fu; hi.w = (w.w >> 4) & 0x0F0F0F0Fu;
-                        const uint32_t row = us + r * UROW;
-                        const int sw = r & 7;
-                        sts128(row + (((2 * c) ^ sw) << 4), lo);
-                        sts128(row + (((2 * c + 1) ^ sw) << 4), hi);
-                        if (need_sums) {
-                            int t = psum[j];
-                            t = dp4a_u8(lo.x + hi.x, 0x01010101u, t);
-                            t = dp4a_u8(lo.y + hi.y, 0x01010101u, t);
-                            t = dp4a_u8(lo.z + hi.z, 0x01010101u, t);
-                            t = dp4a_u8(lo.w + hi.w, 0x01010101u, t);
-                            psum[j] = t;
-                        }
+                        unpack16(wa[c], alo[c], ahi[c]);
+                        if (need_ra) psum_a = chunk_sum(alo[c], ahi[c], psum_a);
                     }
                 }
-                // every lane publishes its own writes to the async proxy; one lane per warp
-                // then arrives (256 arrives on one barrier word serialise badly)
-                fence_async_smem();
+#pragma unroll
+                for (int j = 0; j < NTB; ++j) {
+                    if (((gt + j * GT) & 3) < ksteps) {
+                        unpack16(wb[j], blo[j], bhi[j]);
+                        if (need_cb) psum_b[j] = chunk_sum(blo[j], bhi[j], psum_b[j]);
+                    }
+                }
+                mbar_wait_cl(bar_empty_u(ust), uph ^ 1u, abort_flag, g.status);
+                tc_fence_after();
+                // A: 128 bytes of my row to tensor memory
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    if (c < ksteps) {
+                        const uint32_t r8[8] = {alo[c].x, alo[c].y, alo[c].z, alo[c].w,
+                                                ahi[c].x, ahi[c].y, ahi[c].z, ahi[c].w};
+                        tc_st8(a_taddr + (uint32_t)(ust * 32 + 8 * c), r8);
+                    }
+                }
+                // Bt: two 16-byte groups per packed chunk at the swizzled positions
+                const uint32_t us = sbase + OFF_B + ust * BSTAGE;
+#pragma unroll
+                for (int j = 0; j < NTB; ++j) {
+                    const int id = gt + j * GT;
+                    const int r = id >> 2, c = id & 3;
+                    if (c < ksteps) {
+                        const uint32_t row = us + r * UROW;
+                        const int sw = r & 7;
+                        sts128(row + (((2 * c) ^ sw) << 4), blo[j]);
+                        sts128(row + (((2 * c + 1) ^ sw) << 4), bhi[j]);
+                    }
+                }
+                tc_wait_st();                 // my tensor-memory stores are complete
+                fence_async_smem();           // my shared-memory stores are visible to the MMA
+                tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(bar_full_u(st));
-                    mbar_arrive(bar_empty_p(st));
+                    mbar_arrive_cluster(full_u_leader + 8u * (uint32_t)ust);
+                    mbar_arrive(bar_empty_p(pst));
                 }
             }
             if (need_sums) {
@@ -250,22 +320,19 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const uint32_t aph = (lt >> 1) & 1u;
                 // both CTAs' epilogues two tiles back are done with this sums buffer
                 mbar_wait_cl(bar_tstart(acc), aph, abort_flag, g.status);
+                const uint32_t mine = sums_s + 4 * ((acc * G + grp) * SUMS_N);
+                sts32(mine + 4 * arow, psum_a);
 #pragma unroll
-                for (int j = 0; j < NT; ++j) {
-                    int t = psum[j];
+                for (int j = 0; j < NTB; ++j) {
+                    int t = psum_b[j];
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 1);
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
-                    const int id = ut + j * UT;
+                    const int id = gt + j * GT;
                     if ((id & 3) == 0) {
-                        const int r = id >> 2;
-                        if (r < TMC) {
-                            sts32(sums_s + 4 * (acc * SUMS_N + r), t);         // row sum: local
-                        } else {
-                            // column sum of my half of Bt: both CTAs need it
-                            const uint32_t a = sums_s + 4 * (acc * SUMS_N + TMC + (int)rank * BH + (r - TMC));
-                            sts32(a, t);
-                            sts32_cluster(map_to_cta(a, peer), t);
-                        }
+                        // column sum of my half of Bt: both CTAs need it
+                        const uint32_t a = mine + 4 * (TMC + (int)rank * BH + (id >> 2));
+                        sts32(a, t);
+                        sts32_cluster(map_to_cta(a, peer), t);
                     }
                 }
                 __syncwarp();
@@ -289,17 +356,19 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int m = tm * 256 + (int)rank * TMC + row;
             const int n0 = tn * BNC;
             if (need_sums) mbar_wait_cl(bar_sums(acc), aph, abort_flag, g.status);
+            const uint32_t s0 = sums_s + 4 * (acc * G * SUMS_N);
             for (int j = et; j < BNC; j += 128) {
                 const int n = n0 + j;
                 int cb = 0, bias = 0;
                 if (n < g.N) {
-                    cb = need_cb ? lds32(sums_s + 4 * (acc * SUMS_N + TMC + j)) : g.colsum_b[n];
+                    cb = need_cb ? lds32(s0 + 4 * (TMC + j)) + lds32(s0 + 4 * (SUMS_N + TMC + j))
+                                 : g.colsum_b[n];
                     if (REQUANT && g.bias) bias = g.bias[n];
                 }
                 sts32(colterm_s + 4 * j, (int)((uint32_t)kzz - (uint32_t)(g.za * cb) + (uint32_t)bias));
             }
             int ra = 0;
-            if (need_ra) ra = lds32(sums_s + 4 * (acc * SUMS_N + row));
+            if (need_ra) ra = lds32(s0 + 4 * row) + lds32(s0 + 4 * (SUMS_N + row));
             else if (m < g.M) ra = g.rowsum_a[m];
             const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
             asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -315,12 +384,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 tc_ld32(taddr0 + (uint32_t)(ch * 32), r);
                 tc_wait_ld();
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * q));
-                    r[4 * q + 0] += rowterm + ct.x;
-                    r[4 * q + 1] += rowterm + ct.y;
-                    r[4 * q + 2] += rowterm + ct.z;
-                    r[4 * q + 3] += rowterm + ct.w;
+                for (int qd = 0; qd < 8; ++qd) {
+                    const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
+                    r[4 * qd + 0] += rowterm + ct.x;
+                    r[4 * qd + 1] += rowterm + ct.y;
+                    r[4 * qd + 2] += rowterm + ct.z;
+                    r[4 * qd + 3] += rowterm + ct.w;
                 }
                 if (m < g.M) {
                     const bool full = (nc + 32 <= g.N);
@@ -328,9 +397,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         int32_t* dst = g.C + (int64_t)m * g.ldc + nc;
                         if (full && p.c_vec) {
 #pragma unroll
-                            for (int q = 0; q < 8; ++q)
-                                *reinterpret_cast<uint4*>(dst + 4 * q) =
-                                    make_uint4(r[4 * q], r[4 * q + 1], r[4 * q + 2], r[4 * q + 3]);
+                            for (int qd = 0; qd < 8; ++qd)
+                                *reinterpret_cast<uint4*>(dst + 4 * qd) =
+                                    make_uint4(r[4 * qd], r[4 * qd + 1], r[4 * qd + 2], r[4 * qd + 3]);
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
@@ -339,12 +408,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     } else {
                         uint32_t o[4];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
+                        for (int qd = 0; qd < 4; ++qd) {
                             uint32_t wv = 0;
 #pragma unroll
                             for (int e = 0; e < 8; ++e)
-                                wv |= requant((int32_t)r[8 * q + e], g.rq) << (4 * e);
-                            o[q] = wv;
+                                wv |= requant((int32_t)r[8 * qd + e], g.rq) << (4 * e);
+                            o[qd] = wv;
                         }
                         uint8_t* dst = g.Cq + (int64_t)m * g.ldcq + (nc >> 1);
                         if (full && p.cq_vec) {
@@ -376,11 +445,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
 // ---- host side ------------------------------------------------------------------------
 bool make_packed_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows, int kbytes,
-                     int box_rows);
+                     int box_rows, bool swizzle64);
 
 bool gemm_tc_pair_supported(const GemmParams& p)
 {
-    return gemm_tc_supported(p) && p.M >= 256 && p.N >= 256;
+    return gemm_tc_supported(p) && p.M >= 256 && p.N >= pair::BNC;
 }
 
 template <bool RQ>
@@ -429,8 +498,8 @@ q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st)
     p.c_vec = (!rq && ((uintptr_t)g.C % 16 == 0) && (g.ldc % 4 == 0)) ? 1 : 0;
     p.cq_vec = (rq && ((uintptr_t)g.Cq % 16 == 0) && (g.ldcq % 16 == 0)) ? 1 : 0;
     CUtensorMap tmA, tmB;
-    if (!make_packed_map(&tmA, g.A, g.lda, g.M, kbytes, pair::TMC)) return Q4_ERR_CUDA;
-    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, pair::BH)) return Q4_ERR_CUDA;
+    if (!make_packed_map(&tmA, g.A, g.lda, g.M, kbytes, pair::TMC, true)) return Q4_ERR_CUDA;
+    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, pair::BH, false)) return Q4_ERR_CUDA;
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
     return rq ? launch_pair_t<true>(p, tmA, tmB, tiles, st) : launch_pair_t<false>(p, tmA, tmB, tiles, st);
 }

@@ -133,6 +133,29 @@ __device__ __forceinline__ uint64_t make_kmajor_sw128_desc(uint32_t saddr)
          | (2ull << 61);                // SWIZZLE_128B
 }
 
+// Tensor-memory store: 8 consecutive 32-bit columns of this thread's lane (lane =
+// 32 * (warp % 4) + lane id).
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&r)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]),
+                   "r"(r[6]), "r"(r[7]) : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// True in exactly one lane of a fully active warp.  Loops that issue tcgen05.mma run
+// warp-uniformly and predicate only the issue on this.
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xFFFFFFFF;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
+
 // ---- thread-block clusters (CTA pairs) ------------------------------------------------
 __device__ __forceinline__ uint32_t cluster_ctarank()
 {

@@ -95,7 +95,7 @@ def test_tc_gemm_matches_oracle(q4, shape):
 
 # shapes that reach the CTA-pair kernel (M, N >= 256): tails in M, N, K; short depths
 PAIR_SHAPES = [(256, 256, 128), (300, 260, 1000), (257, 514, 129), (1000, 300, 4096), (512, 768, 64),
-               (384, 512, 33), (2048, 256, 640)]
+               (384, 512, 33), (2048, 256, 640), (256, 192, 128), (700, 200, 257), (512, 400, 4096)]
 
 
 @pytest.mark.parametrize("variant", [TC, TC1])
