@@ -311,7 +311,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive_cluster(full_u_leader + 8u * (uint32_t)ust);
+                    mbar_arrive_cluster_relaxed(full_u_leader + 8u * (uint32_t)ust);
                     mbar_arrive(bar_empty_p(pst));
                 }
             }

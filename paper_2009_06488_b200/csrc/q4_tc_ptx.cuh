@@ -175,6 +175,15 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_bar)
     asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)
                  : "memory");
 }
+// Arrive without release semantics: only for a thread whose prior writes have already
+// been completed by explicit fences (tcgen05.wait::st, fence.proxy.async).  The
+// releasing form drains the thread's outstanding memory traffic and costs about a
+// thousand clocks when issued to another CTA once per pipeline stage.
+__device__ __forceinline__ void mbar_arrive_cluster_relaxed(uint32_t cluster_bar)
+{
+    asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_bar)
+                 : "memory");
+}
 __device__ __forceinline__ void sts32_cluster(uint32_t cluster_saddr, int v)
 {
     asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(cluster_saddr), "r"(v) : "memory");
