@@ -354,8 +354,14 @@ def run_case(args):
         C = torch.empty((n, n), dtype=torch.int32, device="cuda")
         Cq = torch.empty((n, n // 2), dtype=torch.uint8, device="cuda")
         rq = q4.Requant(g.mult, g.shift, 0, 0, 15)
+        ra = cb = None
+        if args.presums:
+            ra = torch.empty(n, dtype=torch.int32, device="cuda")
+            cb = torch.empty(n, dtype=torch.int32, device="cuda")
+            q4.q4_row_sums(A, n, n, ra)
+            q4.q4_row_sums(Bt, n, n, cb)
         if args.case == "gemm":
-            call = lambda: q4.q4_gemm(A, Bt, C, n, n, n, g.za, g.zb)
+            call = lambda: q4.q4_gemm(A, Bt, C, n, n, n, g.za, g.zb, ra, cb)
         else:
             call = lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, g.za, g.zb, rq)
         units, unit = 2.0 * n ** 3 / 1e12, "TOPS"
@@ -404,6 +410,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "conv", "im2col"],
                     help="profile one call in a loop instead of the benchmark step")
+    ap.add_argument("--presums", action="store_true", help="--case gemm: pass precomputed depth sums")
     ap.add_argument("--n", type=int, default=4096, help="GEMM edge, or conv batch, for --case")
     args = ap.parse_args()
     if args.case:

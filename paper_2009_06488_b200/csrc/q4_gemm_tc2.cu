@@ -15,13 +15,13 @@
 // Tensor memory (512 columns): two accumulators of 192 columns (the epilogue of tile t
 // overlaps the main loop of t+1) and four A stages of 32 columns (128 depth bytes).
 //
-// Roles per CTA (14 warps): warp 0 TMA producer (its own 128 rows of A, 64-byte-swizzled
+// Roles per CTA (18 warps): warp 0 TMA producer (its own 128 rows of A, 64-byte-swizzled
 // so that row-per-lane reads are conflict-free, and its own 96 rows of Bt; no
-// multicast); warps 2..9 unpack, as two groups of four that take alternate stages so
-// one group's waits and fences hide behind the other's work, and arrive -- from both
+// multicast); warps 2..13 unpack, as three groups of four that take stages in turn so
+// one group's waits and fences hide behind the others' work, and arrive -- from both
 // CTAs -- on the leader CTA's "operands ready" barrier; warp 1 of the leader CTA issues
 // the pair MMAs and commits to both CTAs' barriers; warp 1 of the peer CTA relays
-// "accumulator drained" once per tile; warps 10..13 epilogue.  Column sums of the two
+// "accumulator drained" once per tile; the last four warps are the epilogue.  Column sums of the two
 // Bt halves are exchanged through distributed shared memory.
 //
 // The depth order inside each 32-value group (even nibbles, then odd) is the same for A
@@ -45,7 +45,10 @@ constexpr int US = 4;                // operand stages (Bt bytes in smem, A byte
 constexpr int PA = TMC * PROW;       // packed A bytes per stage
 constexpr int PSTAGE = PA + BH * PROW;
 constexpr int BSTAGE = BH * UROW;    // unpacked Bt bytes per stage
-constexpr int G = 2, WPG = 4, GT = WPG * 32;   // unpack groups, warps / threads per group
+#ifndef Q4_PAIR_GROUPS
+#define Q4_PAIR_GROUPS 3
+#endif
+constexpr int G = Q4_PAIR_GROUPS, WPG = 4, GT = WPG * 32;   // unpack groups, warps / threads per group
 constexpr int UW = G * WPG;
 constexpr int NTB = BH * 4 / GT;     // Bt tasks (16-byte packed chunks) per thread per stage
 constexpr int NTHREADS = (2 + UW + 4) * 32;
@@ -65,7 +68,6 @@ constexpr int SMEM = OFF_MISC + 16 + 1024;
 static_assert(BH * 4 % GT == 0, "Bt tasks must divide evenly");
 static_assert(2 * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
 static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
-static_assert(US % G == 0, "a group always meets the same operand stages");
 
 // D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC.
 constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)(BNC >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
@@ -256,54 +258,54 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
                 mbar_wait_cl(bar_full_p(pst), pph, abort_flag, g.status);
                 const uint32_t ps = sbase + OFF_P + pst * PSTAGE;
-                // all shared-memory loads first, so their latencies overlap
-                uint4 wa[4], wb[NTB];
+                // phase A: my row of A.  Loads first (their latencies overlap), expand in
+                // registers, then wait for the operand stage and store to tensor memory.
+                {
+                    uint4 wa[4], alo[4], ahi[4];
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (c < ksteps) wa[c] = lds128(ps + a_off + (((uint32_t)c ^ a_sw) << 4));
+                    for (int c = 0; c < 4; ++c)
+                        if (c < ksteps) wa[c] = lds128(ps + a_off + (((uint32_t)c ^ a_sw) << 4));
 #pragma unroll
-                for (int j = 0; j < NTB; ++j) {
-                    const int id = gt + j * GT;
-                    if ((id & 3) < ksteps) wb[j] = lds128(ps + PA + (id >> 2) * PROW + (id & 3) * 16);
-                }
-                // expand in registers while the operand stage may still be in use
-                uint4 alo[4], ahi[4], blo[NTB], bhi[NTB];
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < ksteps) {
+                            unpack16(wa[c], alo[c], ahi[c]);
+                            if (need_ra) psum_a = chunk_sum(alo[c], ahi[c], psum_a);
+                        }
+                    }
+                    mbar_wait_cl(bar_empty_u(ust), uph ^ 1u, abort_flag, g.status);
+                    tc_fence_after();
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (c < ksteps) {
-                        unpack16(wa[c], alo[c], ahi[c]);
-                        if (need_ra) psum_a = chunk_sum(alo[c], ahi[c], psum_a);
+                    for (int c = 0; c < 4; ++c) {
+                        if (c < ksteps) {
+                            const uint32_t r8[8] = {alo[c].x, alo[c].y, alo[c].z, alo[c].w,
+                                                    ahi[c].x, ahi[c].y, ahi[c].z, ahi[c].w};
+                            tc_st8(a_taddr + (uint32_t)(ust * 32 + 8 * c), r8);
+                        }
                     }
                 }
+                // phase B: my share of Bt: two 16-byte groups per packed chunk at the
+                // swizzled positions
+                {
+                    uint4 wb[NTB];
 #pragma unroll
-                for (int j = 0; j < NTB; ++j) {
-                    if (((gt + j * GT) & 3) < ksteps) {
-                        unpack16(wb[j], blo[j], bhi[j]);
-                        if (need_cb) psum_b[j] = chunk_sum(blo[j], bhi[j], psum_b[j]);
+                    for (int j = 0; j < NTB; ++j) {
+                        const int id = gt + j * GT;
+                        if ((id & 3) < ksteps) wb[j] = lds128(ps + PA + (id >> 2) * PROW + (id & 3) * 16);
                     }
-                }
-                mbar_wait_cl(bar_empty_u(ust), uph ^ 1u, abort_flag, g.status);
-                tc_fence_after();
-                // A: 128 bytes of my row to tensor memory
+                    const uint32_t us = sbase + OFF_B + ust * BSTAGE;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (c < ksteps) {
-                        const uint32_t r8[8] = {alo[c].x, alo[c].y, alo[c].z, alo[c].w,
-                                                ahi[c].x, ahi[c].y, ahi[c].z, ahi[c].w};
-                        tc_st8(a_taddr + (uint32_t)(ust * 32 + 8 * c), r8);
-                    }
-                }
-                // Bt: two 16-byte groups per packed chunk at the swizzled positions
-                const uint32_t us = sbase + OFF_B + ust * BSTAGE;
-#pragma unroll
-                for (int j = 0; j < NTB; ++j) {
-                    const int id = gt + j * GT;
-                    const int r = id >> 2, c = id & 3;
-                    if (c < ksteps) {
-                        const uint32_t row = us + r * UROW;
-                        const int sw = r & 7;
-                        sts128(row + (((2 * c) ^ sw) << 4), blo[j]);
-                        sts128(row + (((2 * c + 1) ^ sw) << 4), bhi[j]);
+                    for (int j = 0; j < NTB; ++j) {
+                        const int id = gt + j * GT;
+                        const int r = id >> 2, c = id & 3;
+                        if (c < ksteps) {
+                            uint4 lo, hi;
+                            unpack16(wb[j], lo, hi);
+                            if (need_cb) psum_b[j] = chunk_sum(lo, hi, psum_b[j]);
+                            const uint32_t row = us + r * UROW;
+                            const int sw = r & 7;
+                            sts128(row + (((2 * c) ^ sw) << 4), lo);
+                            sts128(row + (((2 * c + 1) ^ sw) << 4), hi);
+                        }
                     }
                 }
                 tc_wait_st();                 // my tensor-memory stores are complete
@@ -361,15 +363,23 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const int n = n0 + j;
                 int cb = 0, bias = 0;
                 if (n < g.N) {
-                    cb = need_cb ? lds32(s0 + 4 * (TMC + j)) + lds32(s0 + 4 * (SUMS_N + TMC + j))
-                                 : g.colsum_b[n];
+                    if (need_cb) {
+#pragma unroll
+                        for (int gi = 0; gi < G; ++gi) cb += lds32(s0 + 4 * (gi * SUMS_N + TMC + j));
+                    } else {
+                        cb = g.colsum_b[n];
+                    }
                     if (REQUANT && g.bias) bias = g.bias[n];
                 }
                 sts32(colterm_s + 4 * j, (int)((uint32_t)kzz - (uint32_t)(g.za * cb) + (uint32_t)bias));
             }
             int ra = 0;
-            if (need_ra) ra = lds32(s0 + 4 * row) + lds32(s0 + 4 * (SUMS_N + row));
-            else if (m < g.M) ra = g.rowsum_a[m];
+            if (need_ra) {
+#pragma unroll
+                for (int gi = 0; gi < G; ++gi) ra += lds32(s0 + 4 * (gi * SUMS_N + row));
+            } else if (m < g.M) {
+                ra = g.rowsum_a[m];
+            }
             const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
             asm volatile("bar.sync 1, 128;" ::: "memory");
 
