@@ -244,14 +244,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t a_off = (uint32_t)(arow * PROW);
         const uint32_t a_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ACOL0;
         const uint32_t full_u_leader = map_to_cta(bar_full_u(0), 0);  // barrier in the leader CTA
-        uint32_t it = 0, lt = 0;
+        uint32_t lt = 0;
         for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
             int psum_a = 0;
             int psum_b[NTB];
 #pragma unroll
             for (int j = 0; j < NTB; ++j) psum_b[j] = 0;
-            for (int s = 0; s < p.nslab; ++s, ++it) {
-                if ((int)(it % G) != grp) continue;
+            // every tile has nslab stages, so stage s of my lt-th tile is number
+            // lt * nslab + s overall; this group takes the numbers congruent to grp mod G
+            const uint32_t it0 = lt * (uint32_t)p.nslab;
+            for (int s = (int)((grp + G - it0 % G) % G); s < p.nslab; s += G) {
+                const uint32_t it = it0 + (uint32_t)s;
                 const int pst = it % PS, ust = it % US;
                 const uint32_t pph = (it / PS) & 1u, uph = (it / US) & 1u;
                 const int rem = g.K - s * SLAB;
@@ -260,11 +263,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const uint32_t ps = sbase + OFF_P + pst * PSTAGE;
                 // phase A: my row of A.  Loads first (their latencies overlap), expand in
                 // registers, then wait for the operand stage and store to tensor memory.
+                uint4 wb[NTB];
                 {
                     uint4 wa[4], alo[4], ahi[4];
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
                         if (c < ksteps) wa[c] = lds128(ps + a_off + (((uint32_t)c ^ a_sw) << 4));
+#pragma unroll
+                    for (int j = 0; j < NTB; ++j) {
+                        const int id = gt + j * GT;
+                        if ((id & 3) < ksteps) wb[j] = lds128(ps + PA + (id >> 2) * PROW + (id & 3) * 16);
+                    }
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         if (c < ksteps) {
@@ -286,12 +295,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 // phase B: my share of Bt: two 16-byte groups per packed chunk at the
                 // swizzled positions
                 {
-                    uint4 wb[NTB];
-#pragma unroll
-                    for (int j = 0; j < NTB; ++j) {
-                        const int id = gt + j * GT;
-                        if ((id & 3) < ksteps) wb[j] = lds128(ps + PA + (id >> 2) * PROW + (id & 3) * 16);
-                    }
                     const uint32_t us = sbase + OFF_B + ust * BSTAGE;
 #pragma unroll
                     for (int j = 0; j < NTB; ++j) {
@@ -314,7 +317,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive_cluster_relaxed(full_u_leader + 8u * (uint32_t)ust);
-                    mbar_arrive(bar_empty_p(pst));
+                    mbar_arrive_relaxed(bar_empty_p(pst));
                 }
             }
             if (need_sums) {
