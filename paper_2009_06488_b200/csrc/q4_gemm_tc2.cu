@@ -14,6 +14,8 @@
 //
 // Tensor memory (512 columns): two accumulators of 192 columns (the epilogue of tile t
 // overlaps the main loop of t+1) and four A stages of 32 columns (128 depth bytes).
+// The unpacked Bt stages live in a deeper shared-memory ring (eight), so only the short
+// tensor-memory store of A sits between "stage free" and "operands ready".
 //
 // Roles per CTA (18 warps): warp 0 TMA producer (its own 128 rows of A, 64-byte-swizzled
 // so that row-per-lane reads are conflict-free, and its own 96 rows of Bt; no
@@ -41,7 +43,8 @@ constexpr int BNC = 192;             // columns of the pair tile
 constexpr int BH = BNC / 2;          // rows of Bt staged per CTA
 constexpr int PROW = 64, UROW = 128, SLAB = 128;
 constexpr int PS = 6;                // packed stages (A 8 KB + Bt 6 KB)
-constexpr int US = 4;                // operand stages (Bt bytes in smem, A bytes in TMEM)
+constexpr int US = 4;                // A operand stages in tensor memory (32 columns each)
+constexpr int BS = 8;                // Bt operand stages in shared memory (12 KB each)
 constexpr int PA = TMC * PROW;       // packed A bytes per stage
 constexpr int PSTAGE = PA + BH * PROW;
 constexpr int BSTAGE = BH * UROW;    // unpacked Bt bytes per stage
@@ -57,11 +60,11 @@ constexpr int ACOL0 = 2 * BNC;       // first TMEM column of the A stages
 constexpr int SUMS_N = TMC + BNC;    // per buffer and group: 128 row sums, BNC column sums
 
 constexpr int OFF_B = 0;
-constexpr int OFF_P = OFF_B + US * BSTAGE;
+constexpr int OFF_P = OFF_B + BS * BSTAGE;
 constexpr int OFF_SUMS = OFF_P + PS * PSTAGE;
 constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
 constexpr int OFF_BAR = OFF_COLTERM + BNC * 4;
-constexpr int NBAR = 2 * PS + 2 * US + 10;
+constexpr int NBAR = 2 * PS + 2 * US + BS + 10;
 constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
 constexpr int SMEM = OFF_MISC + 16 + 1024;
 
@@ -108,7 +111,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     auto bar_empty_p   = [&](int s) { return bar0 + 8u * (uint32_t)(PS + s); };
     auto bar_full_u    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + s); };
     auto bar_empty_u   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + US + s); };
-    const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US);
+    auto bar_empty_b   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + s); };
+    const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US + BS);
     auto bar_tfull       = [&](int a) { return barT + 8u * (uint32_t)a; };
     auto bar_tempty      = [&](int a) { return barT + 8u * (uint32_t)(2 + a); };
     auto bar_peer_tempty = [&](int a) { return barT + 8u * (uint32_t)(4 + a); };
@@ -136,6 +140,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(bar_full_u(s), 2 * WPG);   // used in the leader: a group's warps of both CTAs
             mbar_init(bar_empty_u(s), 1);
         }
+        for (int s = 0; s < BS; ++s) mbar_init(bar_empty_b(s), 1);
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull(a), 1);
             mbar_init(bar_tempty(a), 128);
@@ -200,7 +205,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     mbar_wait_cl(bar_full_u(st), ph, abort_flag, g.status);
                     tc_fence_after();
                     const uint32_t a_tmem = a_tmem0 + (uint32_t)(st * 32);
-                    const uint64_t bdesc = bdesc0 + (uint64_t)(st * (BSTAGE >> 4));
+                    const int bst = it % BS;
+                    const uint64_t bdesc = bdesc0 + (uint64_t)(bst * (BSTAGE >> 4));
                     const int rem = g.K - s * SLAB;
                     if (elect_one()) {
                         if (rem >= SLAB) {
@@ -216,6 +222,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                                   (s > 0 || i > 0) ? 1u : 0u);
                         }
                         tc_commit_pair(bar_empty_u(st), 3);
+                        tc_commit_pair(bar_empty_b(bst), 3);
                     }
                     __syncwarp();
                 }
@@ -263,17 +270,40 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const uint32_t ps = sbase + OFF_P + pst * PSTAGE;
                 // phase A: my row of A.  Loads first (their latencies overlap), expand in
                 // registers, then wait for the operand stage and store to tensor memory.
-                uint4 wb[NTB];
-                {
-                    uint4 wa[4], alo[4], ahi[4];
+                // all shared-memory loads first, so their latencies overlap
+                uint4 wa[4], wb[NTB];
 #pragma unroll
-                    for (int c = 0; c < 4; ++c)
-                        if (c < ksteps) wa[c] = lds128(ps + a_off + (((uint32_t)c ^ a_sw) << 4));
+                for (int c = 0; c < 4; ++c)
+                    if (c < ksteps) wa[c] = lds128(ps + a_off + (((uint32_t)c ^ a_sw) << 4));
+#pragma unroll
+                for (int j = 0; j < NTB; ++j) {
+                    const int id = gt + j * GT;
+                    if ((id & 3) < ksteps) wb[j] = lds128(ps + PA + (id >> 2) * PROW + (id & 3) * 16);
+                }
+                // Bt first: its shared-memory ring is twice as deep as the tensor-memory ring
+                // of A, so this wait is normally over and the work hides behind the MMAs
+                {
+                    const int bst = it % BS;
+                    mbar_wait_cl(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
+                    const uint32_t us = sbase + OFF_B + bst * BSTAGE;
 #pragma unroll
                     for (int j = 0; j < NTB; ++j) {
                         const int id = gt + j * GT;
-                        if ((id & 3) < ksteps) wb[j] = lds128(ps + PA + (id >> 2) * PROW + (id & 3) * 16);
+                        const int r = id >> 2, c = id & 3;
+                        if (c < ksteps) {
+                            uint4 lo, hi;
+                            unpack16(wb[j], lo, hi);
+                            if (need_cb) psum_b[j] = chunk_sum(lo, hi, psum_b[j]);
+                            const uint32_t row = us + r * UROW;
+                            const int sw = r & 7;
+                            sts128(row + (((2 * c) ^ sw) << 4), lo);
+                            sts128(row + (((2 * c + 1) ^ sw) << 4), hi);
+                        }
                     }
+                }
+                // A: expand my row in registers, then wait for its tensor-memory stage
+                {
+                    uint4 alo[4], ahi[4];
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         if (c < ksteps) {
@@ -289,25 +319,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                             const uint32_t r8[8] = {alo[c].x, alo[c].y, alo[c].z, alo[c].w,
                                                     ahi[c].x, ahi[c].y, ahi[c].z, ahi[c].w};
                             tc_st8(a_taddr + (uint32_t)(ust * 32 + 8 * c), r8);
-                        }
-                    }
-                }
-                // phase B: my share of Bt: two 16-byte groups per packed chunk at the
-                // swizzled positions
-                {
-                    const uint32_t us = sbase + OFF_B + ust * BSTAGE;
-#pragma unroll
-                    for (int j = 0; j < NTB; ++j) {
-                        const int id = gt + j * GT;
-                        const int r = id >> 2, c = id & 3;
-                        if (c < ksteps) {
-                            uint4 lo, hi;
-                            unpack16(wb[j], lo, hi);
-                            if (need_cb) psum_b[j] = chunk_sum(lo, hi, psum_b[j]);
-                            const uint32_t row = us + r * UROW;
-                            const int sw = r & 7;
-                            sts128(row + (((2 * c) ^ sw) << 4), lo);
-                            sts128(row + (((2 * c + 1) ^ sw) << 4), hi);
                         }
                     }
                 }
