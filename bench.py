@@ -197,6 +197,7 @@ def run_ours(args):
     Cq = torch.empty((g.M, g.N // 2), dtype=torch.uint8, device="cuda")
     Y = torch.empty((dq.M, L.OC // 2), dtype=torch.uint8, device="cuda")
     ws = torch.empty(q4.q4_conv2d_workspace_bytes(dq), dtype=torch.uint8, device="cuda")
+    wsg = torch.empty(q4.q4_gemm_workspace_bytes(g.M, g.N, g.K), dtype=torch.uint8, device="cuda")
     hC = torch.empty((g.M, g.N), dtype=torch.int32).pin_memory()
     hCq = torch.empty((g.M, g.N // 2), dtype=torch.uint8).pin_memory()
     hY = torch.empty((dq.M, L.OC // 2), dtype=torch.uint8).pin_memory()
@@ -216,9 +217,9 @@ def run_ours(args):
     def step(record: bool):
         e = [ev() for _ in range(4)] if record else None
         if record: e[0].record()
-        q4.q4_gemm(A, Bt, C, g.M, g.N, g.K, g.za, g.zb)
+        q4.q4_gemm(A, Bt, C, g.M, g.N, g.K, g.za, g.zb, ws=wsg)
         if record: e[1].record()
-        q4.q4_gemm_requant(A, Bt, Cq, g.M, g.N, g.K, g.za, g.zb, rq_g)
+        q4.q4_gemm_requant(A, Bt, Cq, g.M, g.N, g.K, g.za, g.zb, rq_g, ws=wsg)
         if record: e[2].record()
         q4.q4_conv2d(X, Wt, dq, L.za, L.zb, rq_c, Y, ws)
         if record:
@@ -267,7 +268,7 @@ def run_ours(args):
     def e2e_step():
         q4.q4_gemm_host(hA, hBt, hC, g.M, g.N, g.K, g.za, g.zb, staging)
         A.copy_(hA, non_blocking=True); Bt.copy_(hBt, non_blocking=True)
-        q4.q4_gemm_requant(A, Bt, Cq, g.M, g.N, g.K, g.za, g.zb, rq_g)
+        q4.q4_gemm_requant(A, Bt, Cq, g.M, g.N, g.K, g.za, g.zb, rq_g, ws=wsg)
         hCq.copy_(Cq, non_blocking=True)
         X.copy_(hX, non_blocking=True); Wt.copy_(hW, non_blocking=True)
         q4.q4_conv2d(X, Wt, dq, L.za, L.zb, rq_c, Y, ws)
@@ -360,10 +361,11 @@ def run_case(args):
             cb = torch.empty(n, dtype=torch.int32, device="cuda")
             q4.q4_row_sums(A, n, n, ra)
             q4.q4_row_sums(Bt, n, n, cb)
+        wsg = torch.empty(q4.q4_gemm_workspace_bytes(n, n, n), dtype=torch.uint8, device="cuda")
         if args.case == "gemm":
-            call = lambda: q4.q4_gemm(A, Bt, C, n, n, n, g.za, g.zb, ra, cb)
+            call = lambda: q4.q4_gemm(A, Bt, C, n, n, n, g.za, g.zb, ra, cb, ws=wsg)
         else:
-            call = lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, g.za, g.zb, rq)
+            call = lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, g.za, g.zb, rq, ws=wsg)
         units, unit = 2.0 * n ** 3 / 1e12, "TOPS"
     else:
         net = wl.c3(batch=n)

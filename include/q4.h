@@ -100,8 +100,10 @@ typedef struct {
  * elements (>= N).  za, zb in 0..15.  1 <= K <= Q4_MAX_K.  M or N = 0 is a no-op.
  * rowsum_a [M] / colsum_b [N]: optional precomputed sums (e.g. from q4_im2col, or
  * computed once for the weights); NULL = computed inside the kernel.
- * ws / ws_bytes: workspace of at least q4_gemm_workspace_bytes(M, N, K) bytes
- * (may be NULL when that is 0).
+ * ws / ws_bytes: optional workspace of at least q4_gemm_workspace_bytes(M, N, K) bytes,
+ * 16-byte aligned.  With it, large problems take the sums that were not supplied in
+ * one bandwidth-bound pass over the operands instead of inside the GEMM kernel, which
+ * is faster; without it (NULL) the result is the same.  Its contents are scratch.
  */
 q4_status q4_gemm(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
                   int32_t* C, int64_t ldc, int32_t M, int32_t N, int32_t K,

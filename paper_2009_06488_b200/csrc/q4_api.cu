@@ -67,12 +67,31 @@ static q4_status check_requant(const q4_requant* rq)
     return Q4_OK;
 }
 
-static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st)
+static size_t round256(size_t b) { return (b + 255) / 256 * 256; }
+
+static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nullptr,
+                          size_t ws_bytes = 0)
 {
     p.status = status_ptr();
     if (!p.status) return Q4_ERR_CUDA;
     const int v = variant();
-    if (v != 1 && v != 3 && gemm_tc_pair_supported(p)) return launch_gemm_tc_pair(p, rq, st);
+    if (v != 1 && v != 3 && gemm_tc_pair_supported(p)) {
+        // Large problems: the depth sums the caller did not supply are taken by one
+        // bandwidth-bound pass into the workspace (each operand element is then summed
+        // once instead of once per output tile that uses it).  Without a workspace the
+        // kernel takes them itself.
+        const size_t need = round256(4 * (size_t)p.M) + round256(4 * (size_t)p.N);
+        if ((!p.rowsum_a || !p.colsum_b) && ws && ws_bytes >= need && (uintptr_t)ws % 16 == 0) {
+            int32_t* wa = static_cast<int32_t*>(ws);
+            int32_t* wb = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + round256(4 * (size_t)p.M));
+            const bool do_a = !p.rowsum_a, do_b = !p.colsum_b;
+            if (launch_operand_sums(p.A, p.lda, do_a ? p.M : 0, wa, p.Bt, p.ldb, do_b ? p.N : 0, wb,
+                                    p.K, st) != cudaSuccess) return Q4_ERR_CUDA;
+            if (do_a) p.rowsum_a = wa;
+            if (do_b) p.colsum_b = wb;
+        }
+        return launch_gemm_tc_pair(p, rq, st);
+    }
     if (v != 1 && gemm_tc_supported(p)) return launch_gemm_tc(p, rq, st);
     if (v == 2 || v == 3) return Q4_ERR_ALIGNMENT;
     return launch_gemm_simt(p, rq, st) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
@@ -142,7 +161,6 @@ q4_status q4_gemm(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
                   int32_t za, int32_t zb, const int32_t* rowsum_a, const int32_t* colsum_b,
                   void* ws, size_t ws_bytes, void* stream)
 {
-    (void)ws; (void)ws_bytes;
     q4_status s = check_gemm(A, lda, Bt, ldb, M, N, K, za, zb);
     if (s != Q4_OK) return s;
     if (M == 0 || N == 0) return Q4_OK;
@@ -151,7 +169,7 @@ q4_status q4_gemm(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
     GemmParams p{};
     p.A = A; p.Bt = Bt; p.lda = lda; p.ldb = ldb; p.M = M; p.N = N; p.K = K; p.za = za; p.zb = zb;
     p.rowsum_a = rowsum_a; p.colsum_b = colsum_b; p.C = C; p.ldc = ldc;
-    return run_gemm(p, false, static_cast<cudaStream_t>(stream));
+    return run_gemm(p, false, static_cast<cudaStream_t>(stream), ws, ws_bytes);
 }
 
 q4_status q4_gemm_requant(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
@@ -160,7 +178,6 @@ q4_status q4_gemm_requant(const uint8_t* A, int64_t lda, const uint8_t* Bt, int6
                           const int32_t* bias, const q4_requant* rq,
                           uint8_t* Cq, int64_t ldcq, void* ws, size_t ws_bytes, void* stream)
 {
-    (void)ws; (void)ws_bytes;
     q4_status s = check_gemm(A, lda, Bt, ldb, M, N, K, za, zb);
     if (s != Q4_OK) return s;
     if ((s = check_requant(rq)) != Q4_OK) return s;
@@ -171,7 +188,7 @@ q4_status q4_gemm_requant(const uint8_t* A, int64_t lda, const uint8_t* Bt, int6
     p.A = A; p.Bt = Bt; p.lda = lda; p.ldb = ldb; p.M = M; p.N = N; p.K = K; p.za = za; p.zb = zb;
     p.rowsum_a = rowsum_a; p.colsum_b = colsum_b; p.bias = bias; p.Cq = Cq; p.ldcq = ldcq;
     p.rq = RequantParams{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
-    return run_gemm(p, true, static_cast<cudaStream_t>(stream));
+    return run_gemm(p, true, static_cast<cudaStream_t>(stream), ws, ws_bytes);
 }
 
 q4_status q4_im2col(const uint8_t* X, const q4_conv_desc* d, int32_t za,
@@ -190,8 +207,9 @@ q4_status q4_im2col(const uint8_t* X, const q4_conv_desc* d, int32_t za,
 
 size_t q4_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K)
 {
-    (void)M; (void)N; (void)K;
-    return 0;   // sums are taken inside the kernel; no split over the depth
+    (void)K;
+    if (M < 0 || N < 0) return 0;
+    return round256(4 * (size_t)M) + round256(4 * (size_t)N);   // depth sums of both operands
 }
 
 size_t q4_conv2d_workspace_bytes(const q4_conv_desc* d)

@@ -78,6 +78,9 @@ cudaError_t launch_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int
                            int32_t K, int32_t N, cudaStream_t st);
 cudaError_t launch_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
                             int32_t* sums, cudaStream_t st);
+cudaError_t launch_operand_sums(const uint8_t* A, int64_t lda, int32_t rows_a, int32_t* sums_a,
+                                const uint8_t* B, int64_t ldb, int32_t rows_b, int32_t* sums_b,
+                                int32_t K, cudaStream_t st);
 cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, uint8_t* A,
                           int64_t lda, int32_t* rowsum_a, cudaStream_t st);
 

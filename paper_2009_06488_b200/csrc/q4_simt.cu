@@ -182,6 +182,59 @@ __global__ void row_sums_kernel(const uint8_t* __restrict__ P, int64_t ld, int r
     }
 }
 
+// Depth sums of both GEMM operands in one launch (the sums of Eq. 2's second and third
+// terms), one warp per row, 128-bit loads when base and pitch allow.  HBM-bound: each
+// packed byte is read once.
+__global__ void __launch_bounds__(256) operand_sums_kernel(const uint8_t* __restrict__ A, int64_t lda,
+                                                           int rows_a, int32_t* __restrict__ sums_a,
+                                                           const uint8_t* __restrict__ B, int64_t ldb,
+                                                           int rows_b, int32_t* __restrict__ sums_b,
+                                                           int K, int vec)
+{
+    const int lane = threadIdx.x % 32;
+    const int kbytes = (K + 1) / 2;
+    const int total = rows_a + rows_b;
+    for (int r = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32; r < total;
+         r += gridDim.x * (blockDim.x / 32)) {
+        const bool is_a = r < rows_a;
+        const uint8_t* row = is_a ? A + (int64_t)r * lda : B + (int64_t)(r - rows_a) * ldb;
+        int s = 0;
+        int done = 0;
+        if (vec) {
+            const int nvec = kbytes / 16;
+            const uint4* v = reinterpret_cast<const uint4*>(row);
+            for (int i = lane; i < nvec; i += 32) {
+                const uint4 w = v[i];
+                s += nibble_sum(w.x) + nibble_sum(w.y) + nibble_sum(w.z) + nibble_sum(w.w);
+            }
+            done = nvec * 16;
+        }
+        for (int b = done + lane; b < kbytes; b += 32) {
+            const uint8_t byte = row[b];
+            s += (byte & 0x0F) + (byte >> 4);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        if (lane == 0) {
+            if (is_a) sums_a[r] = s; else sums_b[r - rows_a] = s;
+        }
+    }
+}
+
+cudaError_t launch_operand_sums(const uint8_t* A, int64_t lda, int32_t rows_a, int32_t* sums_a,
+                                const uint8_t* B, int64_t ldb, int32_t rows_b, int32_t* sums_b,
+                                int32_t K, cudaStream_t st)
+{
+    const int total = rows_a + rows_b;
+    if (total <= 0) return cudaSuccess;
+    const int vec = ((rows_a == 0 || ((uintptr_t)A % 16 == 0 && lda % 16 == 0)) &&
+                     (rows_b == 0 || ((uintptr_t)B % 16 == 0 && ldb % 16 == 0))) ? 1 : 0;
+    int blocks = (total + 7) / 8 < 148 * 8 ? (total + 7) / 8 : 148 * 8;
+    operand_sums_kernel<<<blocks, 256, 0, st>>>(A, lda, rows_a, sums_a, B, ldb, rows_b, sums_b, K, vec);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
                             int32_t* sums, cudaStream_t st)
 {

@@ -23,7 +23,7 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def run_gemm(q4, c, variant, ldc_pad=0, sums=False):
+def run_gemm(q4, c, variant, ldc_pad=0, sums=False, use_ws=False):
     import torch
     q4.q4_set_variant(variant)
     A, Bt = dev(c.A), dev(c.Bt)
@@ -34,7 +34,10 @@ def run_gemm(q4, c, variant, ldc_pad=0, sums=False):
         cb = torch.empty(c.N, dtype=torch.int32, device="cuda")
         q4.q4_row_sums(A, c.M, c.K, ra)
         q4.q4_row_sums(Bt, c.N, c.K, cb)
-    q4.q4_gemm(A, Bt, C, c.M, c.N, c.K, c.za, c.zb, ra, cb)
+    ws = None
+    if use_ws:     # scratch for the depth sums, poisoned
+        ws = torch.full((q4.q4_gemm_workspace_bytes(c.M, c.N, c.K),), 0xA5, dtype=torch.uint8, device="cuda")
+    q4.q4_gemm(A, Bt, C, c.M, c.N, c.K, c.za, c.zb, ra, cb, ws)
     assert q4.q4_last_device_status() == q4.Q4_OK
     out = C.cpu().numpy()
     if ldc_pad:
@@ -107,6 +110,8 @@ def test_pair_and_single_tensor_core_kernels_agree_with_oracle(q4, variant, shap
     got, _, _ = run_gemm(q4, c, variant, ldc_pad=4)
     assert (got == want).all()
     got, _, _ = run_gemm(q4, c, variant, sums=True)
+    assert (got == want).all()
+    got, _, _ = run_gemm(q4, c, variant, use_ws=True)     # sums taken by the pre-pass
     assert (got == want).all()
     rq = oracle.Requant(c.mult, 6, 4, 4, 15)
     wantq = oracle.requant_matrix(want, c.bias, rq)
