@@ -203,7 +203,15 @@ __global__ void __launch_bounds__(256) operand_sums_kernel(const uint8_t* __rest
         if (vec) {
             const int nvec = kbytes / 16;
             const uint4* v = reinterpret_cast<const uint4*>(row);
-            for (int i = lane; i < nvec; i += 32) {
+            int i = lane;
+            for (; i + 96 < nvec; i += 128) {          // four independent loads in flight
+                const uint4 w0 = v[i], w1 = v[i + 32], w2 = v[i + 64], w3 = v[i + 96];
+                s += nibble_sum(w0.x) + nibble_sum(w0.y) + nibble_sum(w0.z) + nibble_sum(w0.w);
+                s += nibble_sum(w1.x) + nibble_sum(w1.y) + nibble_sum(w1.z) + nibble_sum(w1.w);
+                s += nibble_sum(w2.x) + nibble_sum(w2.y) + nibble_sum(w2.z) + nibble_sum(w2.w);
+                s += nibble_sum(w3.x) + nibble_sum(w3.y) + nibble_sum(w3.z) + nibble_sum(w3.w);
+            }
+            for (; i < nvec; i += 32) {
                 const uint4 w = v[i];
                 s += nibble_sum(w.x) + nibble_sum(w.y) + nibble_sum(w.z) + nibble_sum(w.w);
             }
@@ -229,7 +237,7 @@ cudaError_t launch_operand_sums(const uint8_t* A, int64_t lda, int32_t rows_a, i
     if (total <= 0) return cudaSuccess;
     const int vec = ((rows_a == 0 || ((uintptr_t)A % 16 == 0 && lda % 16 == 0)) &&
                      (rows_b == 0 || ((uintptr_t)B % 16 == 0 && ldb % 16 == 0))) ? 1 : 0;
-    int blocks = (total + 7) / 8 < 148 * 8 ? (total + 7) / 8 : 148 * 8;
+    int blocks = (total + 7) / 8 < 148 * 16 ? (total + 7) / 8 : 148 * 16;
     operand_sums_kernel<<<blocks, 256, 0, st>>>(A, lda, rows_a, sums_a, B, ldb, rows_b, sums_b, K, vec);
     count_launch();
     return cudaGetLastError();

@@ -223,6 +223,34 @@ def test_c2_4096_sampled_rows_and_freivalds(q4):
     assert (gotq[rows] == wantq).all()
 
 
+def big_case_check(q4, c, nrows):
+    """Full-size problems in the launch configuration the benchmark times: rows sampled
+    across every row tile against the oracle, plus exact integer Freivalds on the whole
+    matrix (any wrong entry breaks one of the two products)."""
+    got, _, _ = run_gemm(q4, c, 0, use_ws=True)
+    rng = np.random.default_rng(c.seed)
+    rows = np.unique(np.concatenate([rng.integers(0, c.M, nrows), [0, 127, 128, 255, 256, c.M - 1]]))
+    sampled_rows_check(c, got, rows)
+    freivalds_check(c, got)
+    return got, rows
+
+
+def test_c2_8192_benchmark_shape(q4):
+    c = wl.c2(8192)
+    got, rows = big_case_check(q4, c, 40)
+    rq = oracle.Requant(c.mult, c.shift, 0, 0, 15)
+    gotq = run_requant(q4, c, 0, rq)
+    wantq = oracle.requant_matrix(np.ascontiguousarray(got[rows]), None, rq)
+    assert (gotq[rows] == wantq).all()
+
+
+def test_c5_deep_k_worst_case_zero_points(q4):
+    c = wl.c5()
+    assert (c.za, c.zb) == (0, 15)
+    got, _ = big_case_check(q4, c, 24)
+    assert got.max() <= 0 and got.min() >= -225 * c.K     # sum a (b - 15) is never positive
+
+
 def test_empty_problem_is_a_no_op(q4):
     import torch
     A = torch.zeros((0, 64), dtype=torch.uint8, device="cuda")
