@@ -236,6 +236,15 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     if ((uintptr_t)ws % 256 != 0) return Q4_ERR_ALIGNMENT;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
+    // Layers whose geometry allows it run as one fused kernel that never writes the
+    // unrolled matrix (variants 1 and 3 keep the explicit unroll + GEMM path testable).
+    const int v = variant();
+    if ((v == 0 || v == 2) && conv_fused_supported(*d, X, Wt, ldw, Y)) {
+        const RequantParams rqp{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
+        return launch_conv_fused(X, Wt, ldw, colsum_w, bias, *d, za, zb, rqp, Y, st) == cudaSuccess
+                   ? Q4_OK : Q4_ERR_CUDA;
+    }
+
     uint8_t* A = static_cast<uint8_t*>(ws);
     int32_t* rowsum = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + cs.off_rowsum);
     if (launch_im2col(X, *d, za, A, cs.lda, rowsum, st) != cudaSuccess) return Q4_ERR_CUDA;

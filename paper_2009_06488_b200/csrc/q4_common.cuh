@@ -81,6 +81,12 @@ cudaError_t launch_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t 
 cudaError_t launch_operand_sums(const uint8_t* A, int64_t lda, int32_t rows_a, int32_t* sums_a,
                                 const uint8_t* B, int64_t ldb, int32_t rows_b, int32_t* sums_b,
                                 int32_t K, cudaStream_t st);
+bool        conv_fused_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt,
+                                 int64_t ldw, const uint8_t* Y);
+cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
+                              const int32_t* colsum_w, const int32_t* bias, const q4_conv_desc& d,
+                              int32_t za, int32_t zb, const RequantParams& rq, uint8_t* Y,
+                              cudaStream_t st);
 cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, uint8_t* A,
                           int64_t lda, int32_t* rowsum_a, cudaStream_t st);
 
