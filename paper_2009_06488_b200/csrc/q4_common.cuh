@@ -45,11 +45,27 @@ __device__ __forceinline__ int32_t correct(int32_t raw, int32_t rowsum, int32_t 
 // q = floor((acc*mult + 2^(30+shift)) / 2^(31+shift)); y = clamp(q + zo, lo, hi).
 // |acc| < 2^31 and mult < 2^31 keep the 64-bit sum below 2^63; >> on a signed
 // 64-bit value is an arithmetic (flooring) shift.
-__device__ __forceinline__ uint32_t requant(int32_t acc, const RequantParams& rq)
+__device__ __forceinline__ uint32_t requant_wide(int32_t acc, const RequantParams& rq)
 {
     const int t = 31 + rq.shift;
     long long v = (long long)acc * (long long)rq.mult + (1ll << (t - 1));
     int q = (int)(v >> t) + rq.zo;
+    q = max(q, rq.lo);
+    q = min(q, rq.hi);
+    return (uint32_t)q;
+}
+
+// The same value from the high half of the product when shift >= 2.  With
+// P = acc*mult = hi*2^32 + lo (0 <= lo < 2^32) and s = shift - 1 >= 1:
+//   floor((P + 2^(31+shift-1)) / 2^(31+shift)) = floor((hi + 2^(s-1) + lo/2^32) / 2^s)
+//                                              = floor((hi + 2^(s-1)) / 2^s),
+// because hi + 2^(s-1) is an integer and lo/2^32 < 1 cannot carry it over a multiple
+// of 2^s.  |hi| < 2^30, so the 32-bit sum cannot overflow.
+__device__ __forceinline__ uint32_t requant(int32_t acc, const RequantParams& rq)
+{
+    if (rq.shift < 2) return requant_wide(acc, rq);       // uniform branch
+    const int s = rq.shift - 1;
+    int q = ((__mulhi(acc, rq.mult) + (1 << (s - 1))) >> s) + rq.zo;
     q = max(q, rq.lo);
     q = min(q, rq.hi);
     return (uint32_t)q;

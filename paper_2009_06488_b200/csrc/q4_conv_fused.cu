@@ -55,8 +55,11 @@ __device__ __forceinline__ void mma_u8(int (&c)[4], uint32_t a0, uint32_t a1, ui
 // NT = OC / 8 output-channel tiles.  Fragment column f of tile nt is output channel
 // 2 * (NT * (f / 2) + nt) + f % 2, so that the NT packed output bytes a thread ends up
 // with are contiguous in memory.
+#ifndef Q4_FUSED_MIN_CTAS
+#define Q4_FUSED_MIN_CTAS 2
+#endif
 template <int NT>
-__global__ void __launch_bounds__(WARPS * 32)
+__global__ void __launch_bounds__(WARPS * 32, Q4_FUSED_MIN_CTAS)
 conv_fused_kernel(const Params p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -119,16 +122,26 @@ conv_fused_kernel(const Params p)
         int ih0[4], iw0[4];
         const uint8_t* base[4];
         bool valid[4];
+        {
+            // one division for my first row; the others are 8 pixels further each
+            const int64_t mf = m0 + g;
+            const uint32_t mm = mf < p.M ? (uint32_t)mf : 0u;       // M < 2^31
+            int ow = (int)(mm % (uint32_t)p.OW);
+            const uint32_t q = mm / (uint32_t)p.OW;
+            int oh = (int)(q % (uint32_t)p.OH);
+            int64_t n = q / (uint32_t)p.OH;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int64_t m = m0 + g + 8 * i;
-            valid[i] = m < p.M;
-            const uint32_t mm = valid[i] ? (uint32_t)m : 0u;       // M < 2^31
-            const uint32_t ow = mm % (uint32_t)p.OW, q = mm / (uint32_t)p.OW;
-            const uint32_t oh = q % (uint32_t)p.OH, n = q / (uint32_t)p.OH;
-            ih0[i] = (int)oh * p.sh - p.ph;
-            iw0[i] = (int)ow * p.sw - p.pw;
-            base[i] = p.X + (((int64_t)n * p.H + ih0[i]) * p.W + iw0[i]) * tapb;
+            for (int i = 0; i < 4; ++i) {
+                valid[i] = mf + 8 * i < p.M;
+                ih0[i] = oh * p.sh - p.ph;
+                iw0[i] = ow * p.sw - p.pw;
+                base[i] = p.X + ((n * p.H + ih0[i]) * p.W + iw0[i]) * tapb;
+                ow += 8;
+                while (ow >= p.OW) {
+                    ow -= p.OW;
+                    if (++oh == p.OH) { oh = 0; ++n; }
+                }
+            }
         }
         int acc[2][NT][4];
 #pragma unroll
@@ -231,15 +244,27 @@ bool conv_fused_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t
 }
 
 template <int NT>
-static cudaError_t launch_nt(const fused::Params& p, size_t smem, int grid, cudaStream_t st)
+static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
     static bool attr = false;
+    static int sms = 148;
     if (!attr) {
         cudaError_t e = cudaFuncSetAttribute(fused::conv_fused_kernel<NT>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
         if (e != cudaSuccess) return e;
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         attr = true;
     }
+    // persistent CTAs: as many as are resident at once, so the per-CTA set-up (weights to
+    // fragments) is paid once per SM slot and there is no second wave
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused::conv_fused_kernel<NT>,
+                                                      fused::WARPS * 32, smem) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    const int64_t resident = (int64_t)sms * per_sm;
+    const int grid = (int)(tiles < resident ? tiles : resident);
     fused::conv_fused_kernel<NT><<<grid, fused::WARPS * 32, smem, st>>>(p);
     count_launch();
     return cudaGetLastError();
@@ -264,12 +289,11 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     const int NT = d.OC / 8;
     const size_t smem = (size_t)p.KS * NT * 32 * 8 + (size_t)p.KS * 4 * 8 + (size_t)d.OC * 4;
     const int64_t tiles = (p.M + fused::ROWS_PER_CTA - 1) / fused::ROWS_PER_CTA;
-    const int grid = (int)(tiles < 148 * 4 ? tiles : 148 * 4);
     switch (NT) {
-        case 1: return launch_nt<1>(p, smem, grid, st);
-        case 2: return launch_nt<2>(p, smem, grid, st);
-        case 4: return launch_nt<4>(p, smem, grid, st);
-        default: return launch_nt<8>(p, smem, grid, st);
+        case 1: return launch_nt<1>(p, smem, tiles, st);
+        case 2: return launch_nt<2>(p, smem, tiles, st);
+        case 4: return launch_nt<4>(p, smem, tiles, st);
+        default: return launch_nt<8>(p, smem, tiles, st);
     }
 }
 
