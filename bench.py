@@ -69,7 +69,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-i", str(self.gpu), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+                 "-i", str(self.gpu), "-lms", "20"], stdout=subprocess.PIPE, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
         except OSError:
@@ -121,11 +121,18 @@ def time_oracle_sample(case, target_s: float = 12.0):
     """Times the oracle, as it stands, on a row slice of the GEMM sized for about
     `target_s` seconds; returns (TOPS, seconds, rows, threads)."""
     import oracle
-    probe = 16
+    # two probes: the second one's extra rows give the marginal time per row (the first
+    # also pays for unpacking the whole weight matrix)
+    probe = 32
     t0 = time.perf_counter()
     oracle.gemm(np.ascontiguousarray(case.A[:probe]), case.Bt, probe, case.N, case.K, case.za, case.zb)
-    dt = time.perf_counter() - t0
-    rows = int(max(probe, min(case.M, probe * target_s / max(dt, 1e-6))))
+    dt1 = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    oracle.gemm(np.ascontiguousarray(case.A[:4 * probe]), case.Bt, 4 * probe, case.N, case.K, case.za, case.zb)
+    dt2 = time.perf_counter() - t0
+    per_row = max((dt2 - dt1) / (3 * probe), 1e-7)
+    fixed = max(dt1 - probe * per_row, 0.0)
+    rows = int(max(probe, min(case.M, (target_s - fixed) / per_row)))
     rows = min(rows, case.M)
     t0 = time.perf_counter()
     oracle.gemm(np.ascontiguousarray(case.A[:rows]), case.Bt, rows, case.N, case.K, case.za, case.zb)
@@ -320,7 +327,7 @@ def run_ours(args):
                 "ms_per_step": e2e_ms},
         "roofline": {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
                      "frac": gemm_tops / int8_peak, "traffic": DOMINANT_KERNEL_TRAFFIC_BYTES,
-                     "kernel": "gemm_tc_kernel<256,false> (q4_gemm 8192^3, int32 output)",
+                     "kernel": "gemm_tc_pair_kernel<false> (q4_gemm 8192^3, int32 output)",
                      "peak_source": f"2 x {peaks['source']} bf16 burst "
                                     f"({peaks['bf16']} TFLOP/s), nominal int8:bf16 ratio",
                      "frac_of_datasheet_int8_4500": gemm_tops / DATASHEET_INT8_TOPS,
@@ -331,9 +338,12 @@ def run_ours(args):
             "q4_gemm_requant_8192_ms": gemm_rq_ms,
             "q4_gemm_requant_8192_tops": gemm_ops / (gemm_rq_ms * 1e-3) / 1e12,
             "q4_conv2d_c3_ms": conv_ms,
-            "q4_conv2d_c3_path_gbs": conv_path_bytes / (conv_ms * 1e-3) / 1e9,
+            # the layer runs as one fused kernel: the bytes it must move are the compulsory
+            # ones; the explicit-unroll path's bytes are given only as the equivalent rate
             "q4_conv2d_c3_compulsory_gbs": conv_compulsory_bytes / (conv_ms * 1e-3) / 1e9,
-            "q4_conv2d_c3_path_frac_of_hbm": conv_path_bytes / (conv_ms * 1e-3) / 1e9 / peaks["hbm"],
+            "q4_conv2d_c3_compulsory_frac_of_hbm": conv_compulsory_bytes / (conv_ms * 1e-3) / 1e9 / peaks["hbm"],
+            "q4_conv2d_c3_unroll_path_equivalent_gbs": conv_path_bytes / (conv_ms * 1e-3) / 1e9,
+            "q4_conv2d_c3_gops": conv_ops / (conv_ms * 1e-3) / 1e9,
             "hbm_peak_gbs": peaks["hbm"], "peaks": peaks["source"]},
     }
     print(json.dumps(line))
@@ -406,7 +416,7 @@ def run_case(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
