@@ -42,7 +42,8 @@ constexpr int TMC = 128;             // rows of A per CTA
 constexpr int BNC = 192;             // columns of the pair tile
 constexpr int BH = BNC / 2;          // rows of Bt staged per CTA
 constexpr int PROW = 64, UROW = 128, SLAB = 128;
-constexpr int PS = 6;                // packed stages (A 8 KB + Bt 6 KB)
+constexpr int PS = 8;                // packed stages (A 8 KB + Bt 6 KB); powers of two keep the
+                                     // stage arithmetic to shifts and masks
 constexpr int US = 4;                // A operand stages in tensor memory (32 columns each)
 constexpr int BS = 8;                // Bt operand stages in shared memory (12 KB each)
 constexpr int PA = TMC * PROW;       // packed A bytes per stage
@@ -251,6 +252,19 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t a_off = (uint32_t)(arow * PROW);
         const uint32_t a_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ACOL0;
         const uint32_t full_u_leader = map_to_cta(bar_full_u(0), 0);  // barrier in the leader CTA
+        // per-thread, stage-independent offsets: my four packed chunks of A (swizzled), my
+        // packed chunks of Bt and where their two unpacked halves go
+        uint32_t a_ld[4], b_ld[NTB], b_lo[NTB], b_hi[NTB];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) a_ld[c] = a_off + (((uint32_t)c ^ a_sw) << 4);
+#pragma unroll
+        for (int j = 0; j < NTB; ++j) {
+            const int id = gt + j * GT;
+            const int r = id >> 2, c = id & 3, sw = r & 7;
+            b_ld[j] = (uint32_t)(PA + r * PROW + c * 16);
+            b_lo[j] = (uint32_t)(r * UROW + (((2 * c) ^ sw) << 4));
+            b_hi[j] = (uint32_t)(r * UROW + (((2 * c + 1) ^ sw) << 4));
+        }
         uint32_t lt = 0;
         for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
             int psum_a = 0;
@@ -274,12 +288,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 uint4 wa[4], wb[NTB];
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
-                    if (c < ksteps) wa[c] = lds128(ps + a_off + (((uint32_t)c ^ a_sw) << 4));
+                    if (c < ksteps) wa[c] = lds128(ps + a_ld[c]);
 #pragma unroll
-                for (int j = 0; j < NTB; ++j) {
-                    const int id = gt + j * GT;
-                    if ((id & 3) < ksteps) wb[j] = lds128(ps + PA + (id >> 2) * PROW + (id & 3) * 16);
-                }
+                for (int j = 0; j < NTB; ++j)
+                    if (((gt + j * GT) & 3) < ksteps) wb[j] = lds128(ps + b_ld[j]);
                 // Bt first: its shared-memory ring is twice as deep as the tensor-memory ring
                 // of A, so this wait is normally over and the work hides behind the MMAs
                 {
@@ -288,16 +300,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t us = sbase + OFF_B + bst * BSTAGE;
 #pragma unroll
                     for (int j = 0; j < NTB; ++j) {
-                        const int id = gt + j * GT;
-                        const int r = id >> 2, c = id & 3;
-                        if (c < ksteps) {
+                        if (((gt + j * GT) & 3) < ksteps) {
                             uint4 lo, hi;
                             unpack16(wb[j], lo, hi);
                             if (need_cb) psum_b[j] = chunk_sum(lo, hi, psum_b[j]);
-                            const uint32_t row = us + r * UROW;
-                            const int sw = r & 7;
-                            sts128(row + (((2 * c) ^ sw) << 4), lo);
-                            sts128(row + (((2 * c + 1) ^ sw) << 4), hi);
+                            sts128(us + b_lo[j], lo);
+                            sts128(us + b_hi[j], hi);
                         }
                     }
                 }
