@@ -76,14 +76,31 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
     if (!p.status) return Q4_ERR_CUDA;
     const int v = variant();
     if (v != 1 && v != 3 && gemm_tc_pair_supported(p)) {
-        // Large problems: the depth sums the caller did not supply are taken by one
-        // bandwidth-bound pass into the workspace (each operand element is then summed
-        // once instead of once per output tile that uses it).  Without a workspace the
-        // kernel takes them itself.
-        const size_t need = round256(4 * (size_t)p.M) + round256(4 * (size_t)p.N);
-        if ((!p.rowsum_a || !p.colsum_b) && ws && ws_bytes >= need && (uintptr_t)ws % 16 == 0) {
-            int32_t* wa = static_cast<int32_t*>(ws);
-            int32_t* wb = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + round256(4 * (size_t)p.M));
+        // Large problems use the workspace, if given, for work that is better done once per
+        // call than once per output tile: the depth sums, and -- with the full size -- the
+        // expansion of Bt to bytes.  A smaller workspace still takes the sums; without one
+        // the kernel does everything itself.  The results are identical.
+        // Layout of the workspace: [row sums of A][column sums of Bt][Bt expanded to bytes].
+        const size_t sums_bytes = round256(4 * (size_t)p.M) + round256(4 * (size_t)p.N);
+        const int64_t ld8 = ((int64_t)p.K + 127) / 128 * 128;
+        const size_t full_bytes = sums_bytes + (size_t)p.N * (size_t)ld8;
+        const bool ws_ok = ws && (uintptr_t)ws % 16 == 0;
+        int32_t* wa = static_cast<int32_t*>(ws);
+        int32_t* wb = ws ? reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + round256(4 * (size_t)p.M))
+                         : nullptr;
+        if (ws_ok && ws_bytes >= full_bytes) {
+            // weights prepared once per call: expanded Bt + its column sums; row sums of A
+            uint8_t* b8 = static_cast<uint8_t*>(ws) + sums_bytes;
+            if (launch_bt_expand(p.Bt, p.ldb, p.N, p.K, b8, ld8, wb, st) != cudaSuccess) return Q4_ERR_CUDA;
+            if (!p.colsum_b) p.colsum_b = wb;
+            if (!p.rowsum_a) {
+                if (launch_operand_sums(p.A, p.lda, p.M, wa, p.Bt, p.ldb, 0, wb, p.K, st) != cudaSuccess)
+                    return Q4_ERR_CUDA;
+                p.rowsum_a = wa;
+            }
+            return launch_gemm_tc_pair(p, rq, st, b8, ld8);
+        }
+        if ((!p.rowsum_a || !p.colsum_b) && ws_ok && ws_bytes >= sums_bytes) {
             const bool do_a = !p.rowsum_a, do_b = !p.colsum_b;
             if (launch_operand_sums(p.A, p.lda, do_a ? p.M : 0, wa, p.Bt, p.ldb, do_b ? p.N : 0, wb,
                                     p.K, st) != cudaSuccess) return Q4_ERR_CUDA;
@@ -207,9 +224,10 @@ q4_status q4_im2col(const uint8_t* X, const q4_conv_desc* d, int32_t za,
 
 size_t q4_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K)
 {
-    (void)K;
-    if (M < 0 || N < 0) return 0;
-    return round256(4 * (size_t)M) + round256(4 * (size_t)N);   // depth sums of both operands
+    if (M < 0 || N < 0 || K < 1) return 0;
+    // depth sums of both operands + Bt expanded to one byte per value
+    return round256(4 * (size_t)M) + round256(4 * (size_t)N) +
+           (size_t)N * (size_t)(((int64_t)K + 127) / 128 * 128);
 }
 
 size_t q4_conv2d_workspace_bytes(const q4_conv_desc* d)

@@ -65,7 +65,7 @@ constexpr int OFF_P = OFF_B + BS * BSTAGE;
 constexpr int OFF_SUMS = OFF_P + PS * PSTAGE;
 constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
 constexpr int OFF_BAR = OFF_COLTERM + BNC * 4;
-constexpr int NBAR = 2 * PS + 2 * US + BS + 10;
+constexpr int NBAR = 2 * PS + 2 * US + 2 * BS + 10;
 constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
 constexpr int SMEM = OFF_MISC + 16 + 1024;
 
@@ -96,7 +96,10 @@ __device__ __forceinline__ int chunk_sum(const uint4& lo, const uint4& hi, int a
     return dp4a_u8(t, 0x01010101u, acc);
 }
 
-template <bool REQUANT>
+// BPRE: Bt arrives already expanded to one byte per value (by bt_expand_kernel, once per
+// call, in the same depth order the unpack gives A) and is loaded by TMA straight into
+// the swizzled operand ring; the unpack warps then handle A only.
+template <bool REQUANT, bool BPRE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const Params p)
@@ -113,7 +116,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     auto bar_full_u    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + s); };
     auto bar_empty_u   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + US + s); };
     auto bar_empty_b   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + s); };
-    const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US + BS);
+    auto bar_full_b    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + BS + s); };
+    const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US + 2 * BS);
     auto bar_tfull       = [&](int a) { return barT + 8u * (uint32_t)a; };
     auto bar_tempty      = [&](int a) { return barT + 8u * (uint32_t)(2 + a); };
     auto bar_peer_tempty = [&](int a) { return barT + 8u * (uint32_t)(4 + a); };
@@ -141,7 +145,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(bar_full_u(s), 2 * WPG);   // used in the leader: a group's warps of both CTAs
             mbar_init(bar_empty_u(s), 1);
         }
-        for (int s = 0; s < BS; ++s) mbar_init(bar_empty_b(s), 1);
+        for (int s = 0; s < BS; ++s) {
+            mbar_init(bar_empty_b(s), 1);
+            mbar_init(bar_full_b(s), 1);         // BPRE: the TMA load of an expanded Bt stage
+        }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull(a), 1);
             mbar_init(bar_tempty(a), 128);
@@ -175,10 +182,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const int st = it % PS;
                     const uint32_t ph = (it / PS) & 1u;
                     mbar_wait_cl(bar_empty_p(st), ph ^ 1u, abort_flag, g.status);
-                    mbar_expect_tx(bar_full_p(st), (uint32_t)PSTAGE);
+                    mbar_expect_tx(bar_full_p(st), (uint32_t)(BPRE ? PA : PSTAGE));
                     const uint32_t dst = sbase + OFF_P + st * PSTAGE;
                     tma_load_2d(dst, &tmA, s * PROW, arow, bar_full_p(st));
-                    tma_load_2d(dst + PA, &tmB, s * PROW, brow, bar_full_p(st));
+                    if (!BPRE) {
+                        tma_load_2d(dst + PA, &tmB, s * PROW, brow, bar_full_p(st));
+                    } else {
+                        const int bst = it % BS;
+                        mbar_wait_cl(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
+                        mbar_expect_tx(bar_full_b(bst), (uint32_t)BSTAGE);
+                        tma_load_2d(sbase + OFF_B + bst * BSTAGE, &tmB, s * UROW, brow, bar_full_b(bst));
+                    }
                 }
             }
         }
@@ -291,10 +305,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (c < ksteps) wa[c] = lds128(ps + a_ld[c]);
 #pragma unroll
                 for (int j = 0; j < NTB; ++j)
-                    if (((gt + j * GT) & 3) < ksteps) wb[j] = lds128(ps + b_ld[j]);
+                    if (!BPRE && ((gt + j * GT) & 3) < ksteps) wb[j] = lds128(ps + b_ld[j]);
                 // Bt first: its shared-memory ring is twice as deep as the tensor-memory ring
                 // of A, so this wait is normally over and the work hides behind the MMAs
-                {
+                if (!BPRE) {
                     const int bst = it % BS;
                     mbar_wait_cl(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
                     const uint32_t us = sbase + OFF_B + bst * BSTAGE;
@@ -330,6 +344,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         }
                     }
                 }
+                // BPRE: my CTA's expanded Bt stage has landed (the leader learns it through my arrive)
+                if (BPRE) mbar_wait_cl(bar_full_b(it % BS), (it / BS) & 1u, abort_flag, g.status);
                 tc_wait_st();                 // my tensor-memory stores are complete
                 fence_async_smem();           // my shared-memory stores are visible to the MMA
                 tc_fence_before();
@@ -347,7 +363,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const uint32_t mine = sums_s + 4 * ((acc * G + grp) * SUMS_N);
                 sts32(mine + 4 * arow, psum_a);
 #pragma unroll
-                for (int j = 0; j < NTB; ++j) {
+                for (int j = 0; j < (BPRE ? 0 : NTB); ++j) {
                     int t = psum_b[j];
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 1);
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
@@ -484,12 +500,12 @@ bool gemm_tc_pair_supported(const GemmParams& p)
     return gemm_tc_supported(p) && p.M >= 256 && p.N >= pair::BNC;
 }
 
-template <bool RQ>
+template <bool RQ, bool BPRE>
 static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                long long tiles, cudaStream_t st)
 {
     static int max_clusters = 0;
-    auto kernel = pair::gemm_tc_pair_kernel<RQ>;
+    auto kernel = pair::gemm_tc_pair_kernel<RQ, BPRE>;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -519,7 +535,33 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     return e == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
-q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st)
+// Expanded Bt [N x K8 bytes], pitch ld8: box = 128 bytes x 96 rows, written with the
+// 128-byte swizzle, i.e. directly in the layout the MMA's K-major descriptor reads.
+static bool make_b8_map(CUtensorMap* tm, const uint8_t* base, int64_t ld8, int rows, int k8)
+{
+    typedef CUresult (*Fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                           const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                           CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                           CUtensorMapFloatOOBfill);
+    static Fn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) !=
+                cudaSuccess || qres != cudaDriverEntryPointSuccess) return false;
+        fn = reinterpret_cast<Fn>(sym);
+    }
+    cuuint64_t dims[2] = {(cuuint64_t)k8, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld8};
+    cuuint32_t box[2] = {(cuuint32_t)pair::UROW, (cuuint32_t)pair::BH};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box,
+              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8,
+                              int64_t ld8)
 {
     pair::Params p;
     p.g = g;
@@ -531,9 +573,17 @@ q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st)
     p.cq_vec = (rq && ((uintptr_t)g.Cq % 16 == 0) && (g.ldcq % 16 == 0)) ? 1 : 0;
     CUtensorMap tmA, tmB;
     if (!make_packed_map(&tmA, g.A, g.lda, g.M, kbytes, pair::TMC, true)) return Q4_ERR_CUDA;
-    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, pair::BH, false)) return Q4_ERR_CUDA;
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
-    return rq ? launch_pair_t<true>(p, tmA, tmB, tiles, st) : launch_pair_t<false>(p, tmA, tmB, tiles, st);
+    if (b8) {
+        // expanded Bt: the kernel cannot take the column sums itself
+        if (!g.colsum_b) return Q4_ERR_INVALID_ARG;
+        if (!make_b8_map(&tmB, b8, ld8, g.N, (g.K + 31) / 32 * 32)) return Q4_ERR_CUDA;
+        return rq ? launch_pair_t<true, true>(p, tmA, tmB, tiles, st)
+                  : launch_pair_t<false, true>(p, tmA, tmB, tiles, st);
+    }
+    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, pair::BH, false)) return Q4_ERR_CUDA;
+    return rq ? launch_pair_t<true, false>(p, tmA, tmB, tiles, st)
+              : launch_pair_t<false, false>(p, tmA, tmB, tiles, st);
 }
 
 }  // namespace q4

@@ -35,8 +35,11 @@ def run_gemm(q4, c, variant, ldc_pad=0, sums=False, use_ws=False):
         q4.q4_row_sums(A, c.M, c.K, ra)
         q4.q4_row_sums(Bt, c.N, c.K, cb)
     ws = None
-    if use_ws:     # scratch for the depth sums, poisoned
-        ws = torch.full((q4.q4_gemm_workspace_bytes(c.M, c.N, c.K),), 0xA5, dtype=torch.uint8, device="cuda")
+    if use_ws:     # scratch (poisoned): full size = depth sums + expanded Bt; "sums" = the sums only
+        nbytes = q4.q4_gemm_workspace_bytes(c.M, c.N, c.K)
+        if use_ws == "sums":
+            nbytes = (4 * c.M + 255) // 256 * 256 + (4 * c.N + 255) // 256 * 256
+        ws = torch.full((nbytes,), 0xA5, dtype=torch.uint8, device="cuda")
     q4.q4_gemm(A, Bt, C, c.M, c.N, c.K, c.za, c.zb, ra, cb, ws)
     assert q4.q4_last_device_status() == q4.Q4_OK
     out = C.cpu().numpy()
@@ -45,14 +48,17 @@ def run_gemm(q4, c, variant, ldc_pad=0, sums=False, use_ws=False):
     return out[:, :c.N], ra, cb
 
 
-def run_requant(q4, c, variant, rq, bias=None, ld_pad=0):
+def run_requant(q4, c, variant, rq, bias=None, ld_pad=0, use_ws=False):
     import torch
     q4.q4_set_variant(variant)
     A, Bt = dev(c.A), dev(c.Bt)
     Cq = torch.full((c.M, c.N // 2 + ld_pad), 0xA5, dtype=torch.uint8, device="cuda")
+    ws = None
+    if use_ws:
+        ws = torch.full((q4.q4_gemm_workspace_bytes(c.M, c.N, c.K),), 0xA5, dtype=torch.uint8, device="cuda")
     q4.q4_gemm_requant(A, Bt, Cq, c.M, c.N, c.K, c.za, c.zb,
                        q4.Requant(rq.mult, rq.shift, rq.zo, rq.clamp_lo, rq.clamp_hi),
-                       None if bias is None else dev(bias))
+                       None if bias is None else dev(bias), ws=ws)
     assert q4.q4_last_device_status() == q4.Q4_OK
     out = Cq.cpu().numpy()
     if ld_pad:
@@ -98,7 +104,7 @@ def test_tc_gemm_matches_oracle(q4, shape):
 
 # shapes that reach the CTA-pair kernel (M, N >= 256): tails in M, N, K; short depths
 PAIR_SHAPES = [(256, 256, 128), (300, 260, 1000), (257, 514, 129), (1000, 300, 4096), (512, 768, 64),
-               (384, 512, 33), (2048, 256, 640), (256, 192, 128), (700, 200, 257), (512, 400, 4096)]
+               (384, 512, 33), (2048, 256, 640), (256, 192, 128), (700, 200, 257), (512, 400, 4096), (300, 200, 1000), (256, 192, 100), (640, 384, 31)]
 
 
 @pytest.mark.parametrize("variant", [TC, TC1])
@@ -111,12 +117,17 @@ def test_pair_and_single_tensor_core_kernels_agree_with_oracle(q4, variant, shap
     assert (got == want).all()
     got, _, _ = run_gemm(q4, c, variant, sums=True)
     assert (got == want).all()
-    got, _, _ = run_gemm(q4, c, variant, use_ws=True)     # sums taken by the pre-pass
+    got, _, _ = run_gemm(q4, c, variant, use_ws=True)     # Bt expanded and sums taken once per call
+    assert (got == want).all()
+    got, _, _ = run_gemm(q4, c, variant, use_ws="sums")   # only the sums taken by the pre-pass
+    assert (got == want).all()
+    got, _, _ = run_gemm(q4, c, variant, sums=True, use_ws=True)
     assert (got == want).all()
     rq = oracle.Requant(c.mult, 6, 4, 4, 15)
     wantq = oracle.requant_matrix(want, c.bias, rq)
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=16) == wantq).all()
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=3) == wantq).all()   # byte stores
+    assert (run_requant(q4, c, variant, rq, c.bias, use_ws=True) == wantq).all()
 
 
 @pytest.mark.parametrize("variant", [SIMT, TC])
@@ -239,7 +250,7 @@ def test_c2_8192_benchmark_shape(q4):
     c = wl.c2(8192)
     got, rows = big_case_check(q4, c, 40)
     rq = oracle.Requant(c.mult, c.shift, 0, 0, 15)
-    gotq = run_requant(q4, c, 0, rq)
+    gotq = run_requant(q4, c, 0, rq, use_ws=True)
     wantq = oracle.requant_matrix(np.ascontiguousarray(got[rows]), None, rq)
     assert (gotq[rows] == wantq).all()
 
