@@ -114,7 +114,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     auto bar_full_p    = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto bar_empty_p   = [&](int s) { return bar0 + 8u * (uint32_t)(PS + s); };
     auto bar_full_u    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + s); };
-    auto bar_empty_u   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + US + s); };
     auto bar_empty_b   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + s); };
     auto bar_full_b    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + BS + s); };
     const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US + 2 * BS);
@@ -141,10 +140,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(bar_full_p(s), 1);
             mbar_init(bar_empty_p(s), WPG);      // one arrive per warp of the group that took it
         }
-        for (int s = 0; s < US; ++s) {
+        for (int s = 0; s < US; ++s)
             mbar_init(bar_full_u(s), 2 * WPG);   // used in the leader: a group's warps of both CTAs
-            mbar_init(bar_empty_u(s), 1);
-        }
         for (int s = 0; s < BS; ++s) {
             mbar_init(bar_empty_b(s), 1);
             mbar_init(bar_full_b(s), 1);         // BPRE: the TMA load of an expanded Bt stage
@@ -203,7 +200,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // elected lane issues the MMAs and commits.
             const uint32_t a_tmem0 = tmem_base + (uint32_t)ACOL0;
             const uint64_t bdesc0 = make_kmajor_sw128_desc(sbase + OFF_B);
-            uint32_t it = 0, lt = 0;
+            uint32_t lt = 0;
             for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
                 const int acc = lt & 1;
                 const uint32_t aph = (lt >> 1) & 1u;
@@ -214,32 +211,43 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (elect_one()) tc_commit_pair(bar_tstart(acc), 3);
                 __syncwarp();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BNC);
-                for (int s = 0; s < p.nslab; ++s, ++it) {
-                    const int st = it % US;
-                    const uint32_t ph = (it / US) & 1u;
-                    mbar_wait_cl(bar_full_u(st), ph, abort_flag, g.status);
-                    tc_fence_after();
-                    const uint32_t a_tmem = a_tmem0 + (uint32_t)(st * 32);
-                    const int bst = it % BS;
-                    const uint64_t bdesc = bdesc0 + (uint64_t)(bst * (BSTAGE >> 4));
-                    const int rem = g.K - s * SLAB;
-                    if (elect_one()) {
-                        if (rem >= SLAB) {
-                            tc_mma_i8_pair_ts(d_tmem, a_tmem, bdesc, kIdesc, s > 0 ? 1u : 0u);
-                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 8u, bdesc + 2u, kIdesc, 1u);
-                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 16u, bdesc + 4u, kIdesc, 1u);
-                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 24u, bdesc + 6u, kIdesc, 1u);
-                        } else {
-                            const int ksteps = (rem + 31) / 32;
-                            for (int i = 0; i < ksteps; ++i)
-                                tc_mma_i8_pair_ts(d_tmem, a_tmem + (uint32_t)(8 * i),
-                                                  bdesc + (uint64_t)(2 * i), kIdesc,
-                                                  (s > 0 || i > 0) ? 1u : 0u);
+                // Stages are numbered across tiles (stage s of my lt-th tile is lt*nslab + s).
+                // The loop walks them in aligned blocks of BS so that ring slots, tensor-memory
+                // columns, descriptors and barrier addresses are compile-time offsets.
+                const uint32_t it_begin = lt * (uint32_t)p.nslab, it_end = it_begin + (uint32_t)p.nslab;
+                for (uint32_t blk = it_begin & ~(uint32_t)(BS - 1); blk < it_end; blk += BS) {
+                    const uint32_t bph = (blk / BS) & 1u;
+#pragma unroll
+                    for (int j = 0; j < BS; ++j) {
+                        const uint32_t it = blk + (uint32_t)j;
+                        if (it < it_begin || it >= it_end) continue;        // warp-uniform
+                        // A ring slot j % US: its phase is (it / US) & 1 = (j / US) & 1, blk being
+                        // a multiple of 2 * US
+                        mbar_wait_cl(bar_full_u(j % US), (uint32_t)((j / US) & 1), abort_flag, g.status);
+                        tc_fence_after();
+                        const uint32_t a_tmem = a_tmem0 + (uint32_t)((j % US) * 32);
+                        const uint64_t bdesc = bdesc0 + (uint64_t)(j * (BSTAGE >> 4));
+                        const int rem = g.K - (int)(it - it_begin) * SLAB;
+                        if (elect_one()) {
+                            if (rem >= SLAB) {
+                                tc_mma_i8_pair_ts(d_tmem, a_tmem, bdesc, kIdesc, it > it_begin ? 1u : 0u);
+                                tc_mma_i8_pair_ts(d_tmem, a_tmem + 8u, bdesc + 2u, kIdesc, 1u);
+                                tc_mma_i8_pair_ts(d_tmem, a_tmem + 16u, bdesc + 4u, kIdesc, 1u);
+                                tc_mma_i8_pair_ts(d_tmem, a_tmem + 24u, bdesc + 6u, kIdesc, 1u);
+                            } else {
+                                const int ksteps = (rem + 31) / 32;
+                                for (int i = 0; i < ksteps; ++i)
+                                    tc_mma_i8_pair_ts(d_tmem, a_tmem + (uint32_t)(8 * i),
+                                                      bdesc + (uint64_t)(2 * i), kIdesc,
+                                                      (it > it_begin || i > 0) ? 1u : 0u);
+                            }
+                            // one commit frees this stage's Bt slot and, through the same
+                            // barrier, its A slot (see the unpack warps' wait)
+                            tc_commit_pair(bar_empty_b(j), 3);
                         }
-                        tc_commit_pair(bar_empty_u(st), 3);
-                        tc_commit_pair(bar_empty_b(bst), 3);
+                        __syncwarp();
                     }
-                    __syncwarp();
+                    (void)bph;
                 }
                 if (elect_one()) tc_commit_pair(bar_tfull(acc), 3);
                 __syncwarp();
@@ -291,7 +299,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int s = (int)((grp + G - it0 % G) % G); s < p.nslab; s += G) {
                 const uint32_t it = it0 + (uint32_t)s;
                 const int pst = it % PS, ust = it % US;
-                const uint32_t pph = (it / PS) & 1u, uph = (it / US) & 1u;
+                const uint32_t pph = (it / PS) & 1u;
                 const int rem = g.K - s * SLAB;
                 const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
                 mbar_wait_cl(bar_full_p(pst), pph, abort_flag, g.status);
@@ -333,7 +341,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                             if (need_ra) psum_a = chunk_sum(alo[c], ahi[c], psum_a);
                         }
                     }
-                    mbar_wait_cl(bar_empty_u(ust), uph ^ 1u, abort_flag, g.status);
+                    // my A slot was last used by stage it - US, whose MMAs' commit arrived on the
+                    // Bt ring's barrier of that stage
+                    if (it >= (uint32_t)US)
+                        mbar_wait_cl(bar_empty_b((it - US) % BS), ((it - US) / BS) & 1u, abort_flag, g.status);
                     tc_fence_after();
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
