@@ -35,10 +35,10 @@ def run_gemm(q4, c, variant, ldc_pad=0, sums=False, use_ws=False):
         q4.q4_row_sums(A, c.M, c.K, ra)
         q4.q4_row_sums(Bt, c.N, c.K, cb)
     ws = None
-    if use_ws:     # scratch (poisoned): full size = depth sums + expanded Bt; "sums" = the sums only
+    if use_ws:     # scratch (poisoned): the depth sums; "expanded" = sums + Bt expanded to bytes
         nbytes = q4.q4_gemm_workspace_bytes(c.M, c.N, c.K)
-        if use_ws == "sums":
-            nbytes = (4 * c.M + 255) // 256 * 256 + (4 * c.N + 255) // 256 * 256
+        if use_ws == "expanded":
+            nbytes = q4.q4_gemm_workspace_bytes_expanded(c.M, c.N, c.K)
         ws = torch.full((nbytes,), 0xA5, dtype=torch.uint8, device="cuda")
     q4.q4_gemm(A, Bt, C, c.M, c.N, c.K, c.za, c.zb, ra, cb, ws)
     assert q4.q4_last_device_status() == q4.Q4_OK
@@ -55,7 +55,8 @@ def run_requant(q4, c, variant, rq, bias=None, ld_pad=0, use_ws=False):
     Cq = torch.full((c.M, c.N // 2 + ld_pad), 0xA5, dtype=torch.uint8, device="cuda")
     ws = None
     if use_ws:
-        ws = torch.full((q4.q4_gemm_workspace_bytes(c.M, c.N, c.K),), 0xA5, dtype=torch.uint8, device="cuda")
+        ws = torch.full((q4.q4_gemm_workspace_bytes_expanded(c.M, c.N, c.K) if use_ws == "expanded" else
+                         q4.q4_gemm_workspace_bytes(c.M, c.N, c.K),), 0xA5, dtype=torch.uint8, device="cuda")
     q4.q4_gemm_requant(A, Bt, Cq, c.M, c.N, c.K, c.za, c.zb,
                        q4.Requant(rq.mult, rq.shift, rq.zo, rq.clamp_lo, rq.clamp_hi),
                        None if bias is None else dev(bias), ws=ws)
@@ -117,17 +118,18 @@ def test_pair_and_single_tensor_core_kernels_agree_with_oracle(q4, variant, shap
     assert (got == want).all()
     got, _, _ = run_gemm(q4, c, variant, sums=True)
     assert (got == want).all()
-    got, _, _ = run_gemm(q4, c, variant, use_ws=True)     # Bt expanded and sums taken once per call
+    got, _, _ = run_gemm(q4, c, variant, use_ws=True)     # sums taken by the pre-pass
     assert (got == want).all()
-    got, _, _ = run_gemm(q4, c, variant, use_ws="sums")   # only the sums taken by the pre-pass
+    got, _, _ = run_gemm(q4, c, variant, use_ws="expanded")   # Bt expanded once per call as well
     assert (got == want).all()
-    got, _, _ = run_gemm(q4, c, variant, sums=True, use_ws=True)
+    got, _, _ = run_gemm(q4, c, variant, sums=True, use_ws="expanded")
     assert (got == want).all()
     rq = oracle.Requant(c.mult, 6, 4, 4, 15)
     wantq = oracle.requant_matrix(want, c.bias, rq)
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=16) == wantq).all()
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=3) == wantq).all()   # byte stores
     assert (run_requant(q4, c, variant, rq, c.bias, use_ws=True) == wantq).all()
+    assert (run_requant(q4, c, variant, rq, c.bias, use_ws="expanded") == wantq).all()
 
 
 @pytest.mark.parametrize("variant", [SIMT, TC])
