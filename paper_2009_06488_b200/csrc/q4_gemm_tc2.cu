@@ -42,8 +42,7 @@ constexpr int TMC = 128;             // rows of A per CTA
 constexpr int BNC = 192;             // columns of the pair tile
 constexpr int BH = BNC / 2;          // rows of Bt staged per CTA
 constexpr int PROW = 64, UROW = 128, SLAB = 128;
-constexpr int PS = 8;                // packed stages (A 8 KB + Bt 6 KB); powers of two keep the
-                                     // stage arithmetic to shifts and masks
+constexpr int PS = 6;                // packed stages (A 8 KB + Bt 6 KB)
 constexpr int US = 4;                // A operand stages in tensor memory (32 columns each)
 constexpr int BS = 8;                // Bt operand stages in shared memory (12 KB each)
 constexpr int PA = TMC * PROW;       // packed A bytes per stage
@@ -62,7 +61,9 @@ constexpr int SUMS_N = TMC + BNC;    // per buffer and group: 128 row sums, BNC 
 
 constexpr int OFF_B = 0;
 constexpr int OFF_P = OFF_B + BS * BSTAGE;
-constexpr int OFF_SUMS = OFF_P + PS * PSTAGE;
+constexpr int OFF_STG = OFF_P + PS * PSTAGE;      // int32 epilogue staging: 4 warps x 32 rows x 128 B
+constexpr int STG_BYTES = 4 * 32 * 128;
+constexpr int OFF_SUMS = OFF_STG + STG_BYTES;
 constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
 constexpr int OFF_BAR = OFF_COLTERM + BNC * 4;
 constexpr int NBAR = 2 * PS + 2 * US + 2 * BS + 10;
@@ -72,6 +73,7 @@ constexpr int SMEM = OFF_MISC + 16 + 1024;
 static_assert(BH * 4 % GT == 0, "Bt tasks must divide evenly");
 static_assert(2 * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
 static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
+static_assert(OFF_STG % 1024 == 0, "staging tile alignment (128-byte swizzle atoms)");
 
 // D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC.
 constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)(BNC >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
@@ -80,6 +82,7 @@ struct Params {
     GemmParams g;
     int32_t tiles_m, tiles_n, nslab;
     int32_t c_vec, cq_vec;
+    int32_t c_tma;      // int32 output goes out through TMA stores (tmC is valid)
 };
 
 __device__ __forceinline__ void unpack16(const uint4& w, uint4& lo, uint4& hi)
@@ -102,7 +105,7 @@ __device__ __forceinline__ int chunk_sum(const uint4& lo, const uint4& hi, int a
 template <bool REQUANT, bool BPRE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const Params p)
+                    const __grid_constant__ CUtensorMap tmC, const Params p)
 {
     extern __shared__ uint8_t smem_raw[];
     // the same offset in both CTAs: dynamic shared memory starts at the same address
@@ -450,7 +453,24 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     r[4 * qd + 2] += rowterm + ct.z;
                     r[4 * qd + 3] += rowterm + ct.w;
                 }
-                if (m < g.M) {
+                if (!REQUANT && p.c_tma) {
+                    // int32 tile out through shared memory and one TMA store per warp: my
+                    // row's 128 bytes go to the swizzled staging slice of my warp; rows and
+                    // columns past M / N are clipped by the tensor map
+                    const uint32_t slice = sbase + OFF_STG + (uint32_t)(lg * 4096);
+                    if (lane == 0) bulk_wait_read();       // the previous store has read the slice
+                    __syncwarp();
+#pragma unroll
+                    for (int qd = 0; qd < 8; ++qd)
+                        sts128(slice + (uint32_t)(lane * 128 + ((qd ^ (lane & 7)) << 4)),
+                               make_uint4(r[4 * qd], r[4 * qd + 1], r[4 * qd + 2], r[4 * qd + 3]));
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmC, slice, nc, tm * 256 + (int)rank * TMC + lg * 32);
+                        bulk_commit();
+                    }
+                } else if (m < g.M) {
                     const bool full = (nc + 32 <= g.N);
                     if (!REQUANT) {
                         int32_t* dst = g.C + (int64_t)m * g.ldc + nc;
@@ -489,6 +509,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_arrive(bar_tempty(acc));
             asm volatile("bar.sync 1, 128;" ::: "memory");
         }
+        if (!REQUANT && p.c_tma && lane == 0) bulk_wait_all();   // my TMA stores are complete
     }
 
     tc_fence_before();
@@ -513,7 +534,7 @@ bool gemm_tc_pair_supported(const GemmParams& p)
 
 template <bool RQ, bool BPRE>
 static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
-                               long long tiles, cudaStream_t st)
+                               const CUtensorMap& tmC, long long tiles, cudaStream_t st)
 {
     static int max_clusters = 0;
     auto kernel = pair::gemm_tc_pair_kernel<RQ, BPRE>;
@@ -541,27 +562,49 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     }
     const long long clusters = tiles < max_clusters ? tiles : max_clusters;
     cfg.gridDim = dim3((unsigned)(2 * clusters));
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, p);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, tmA, tmB, tmC, p);
     count_launch();
     return e == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
 // Expanded Bt [N x K8 bytes], pitch ld8: box = 128 bytes x 96 rows, written with the
 // 128-byte swizzle, i.e. directly in the layout the MMA's K-major descriptor reads.
-static bool make_b8_map(CUtensorMap* tm, const uint8_t* base, int64_t ld8, int rows, int k8)
+typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                             CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                             CUtensorMapFloatOOBfill);
+static EncodeFn encode_fn()
 {
-    typedef CUresult (*Fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                           const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
-                           CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
-                           CUtensorMapFloatOOBfill);
-    static Fn fn = nullptr;
+    static EncodeFn fn = nullptr;
     if (!fn) {
         void* sym = nullptr;
         cudaDriverEntryPointQueryResult qres;
         if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) !=
-                cudaSuccess || qres != cudaDriverEntryPointSuccess) return false;
-        fn = reinterpret_cast<Fn>(sym);
+                cudaSuccess || qres != cudaDriverEntryPointSuccess) return nullptr;
+        fn = reinterpret_cast<EncodeFn>(sym);
     }
+    return fn;
+}
+
+// int32 C [M x N], pitch ldc elements: box = 32 columns (128 bytes) x 32 rows, read from a
+// 128-byte-swizzled shared-memory tile.
+static bool make_c_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, int cols)
+{
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+    cuuint32_t box[2] = {32, 32};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_INT32, 2, base, dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+              CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+static bool make_b8_map(CUtensorMap* tm, const uint8_t* base, int64_t ld8, int rows, int k8)
+{
+    EncodeFn fn = encode_fn();
+    if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)k8, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld8};
     cuuint32_t box[2] = {(cuuint32_t)pair::UROW, (cuuint32_t)pair::BH};
@@ -582,19 +625,25 @@ q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, con
     p.nslab = (kbytes + pair::PROW - 1) / pair::PROW;
     p.c_vec = (!rq && ((uintptr_t)g.C % 16 == 0) && (g.ldc % 4 == 0)) ? 1 : 0;
     p.cq_vec = (rq && ((uintptr_t)g.Cq % 16 == 0) && (g.ldcq % 16 == 0)) ? 1 : 0;
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB, tmC;
     if (!make_packed_map(&tmA, g.A, g.lda, g.M, kbytes, pair::TMC, true)) return Q4_ERR_CUDA;
+    p.c_tma = 0;
+    tmC = CUtensorMap{};
+    if (p.c_vec) {
+        if (!make_c_map(&tmC, g.C, g.ldc, g.M, g.N)) return Q4_ERR_CUDA;
+        p.c_tma = 1;
+    }
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
     if (b8) {
         // expanded Bt: the kernel cannot take the column sums itself
         if (!g.colsum_b) return Q4_ERR_INVALID_ARG;
         if (!make_b8_map(&tmB, b8, ld8, g.N, (g.K + 31) / 32 * 32)) return Q4_ERR_CUDA;
-        return rq ? launch_pair_t<true, true>(p, tmA, tmB, tiles, st)
-                  : launch_pair_t<false, true>(p, tmA, tmB, tiles, st);
+        return rq ? launch_pair_t<true, true>(p, tmA, tmB, tmC, tiles, st)
+                  : launch_pair_t<false, true>(p, tmA, tmB, tmC, tiles, st);
     }
     if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, pair::BH, false)) return Q4_ERR_CUDA;
-    return rq ? launch_pair_t<true, false>(p, tmA, tmB, tiles, st)
-              : launch_pair_t<false, false>(p, tmA, tmB, tiles, st);
+    return rq ? launch_pair_t<true, false>(p, tmA, tmB, tmC, tiles, st)
+              : launch_pair_t<false, false>(p, tmA, tmB, tmC, tiles, st);
 }
 
 }  // namespace q4
