@@ -270,11 +270,25 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                    ? Q4_OK : Q4_ERR_CUDA;
     }
 
+    GemmParams p{};
+    // A layer whose unrolled matrix is the input itself -- a filter as large as the
+    // unpadded image (a fully connected layer), or a 1x1 filter with stride 1 -- goes
+    // straight to the GEMM; the workspace then only holds the depth sums.
+    const bool whole_image = d->KH == d->H && d->KW == d->W;
+    const bool pointwise = d->KH == 1 && d->KW == 1 && d->stride_h == 1 && d->stride_w == 1;
+    if (v == 0 && d->pad_h == 0 && d->pad_w == 0 && (whole_image || pointwise) &&
+        cs.K % 2 == 0) {
+        p.A = X; p.Bt = Wt; p.lda = cs.K / 2; p.ldb = ldw; p.M = (int32_t)cs.M; p.N = d->OC; p.K = cs.K;
+        p.za = za; p.zb = zb; p.rowsum_a = nullptr; p.colsum_b = colsum_w; p.bias = bias;
+        p.Cq = Y; p.ldcq = d->OC / 2;
+        p.rq = RequantParams{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
+        return run_gemm(p, true, st, ws, ws_bytes);
+    }
+
     uint8_t* A = static_cast<uint8_t*>(ws);
     int32_t* rowsum = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + cs.off_rowsum);
     if (launch_im2col(X, *d, za, A, cs.lda, rowsum, st) != cudaSuccess) return Q4_ERR_CUDA;
 
-    GemmParams p{};
     p.A = A; p.Bt = Wt; p.lda = cs.lda; p.ldb = ldw; p.M = (int32_t)cs.M; p.N = d->OC; p.K = cs.K;
     p.za = za; p.zb = zb; p.rowsum_a = rowsum; p.colsum_b = colsum_w; p.bias = bias;
     p.Cq = Y; p.ldcq = d->OC / 2;

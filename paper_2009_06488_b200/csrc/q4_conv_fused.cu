@@ -1,32 +1,70 @@
 // Fused quantized convolution layer: the unrolled activation matrix of GEMM-based
 // convolution (Section I; depth D = kh*kw*c, Section III-A) is never written to
-// memory.  Each warp gathers its 32 output pixels' taps straight from the packed NHWC
-// input, expands the nibbles in registers into the A fragments of the warp-level
-// integer MMA (u8 x u8 -> s32, m16n8k32), multiplies against the layer's weights held
-// as B fragments in shared memory, and applies Eq. 3's zero-point terms, the bias, the
-// re-quantization and the nibble packing to the accumulators it holds.  The row sums of
-// Eq. 2's second term are taken from the same registers "while unrolling" (Section
-// II-B).
+// memory.  A CTA takes 224 consecutive output pixels.  It first copies the input rows
+// those pixels touch into shared memory -- with the padding materialised as the input
+// zero point, so the gather below needs no bounds checks -- while the previous tile is
+// still being multiplied (two buffers).  Each warp then gathers its 32 pixels' taps from
+// that copy into the A fragments of the warp-level integer MMA (u8 x s8 -> s32,
+// m16n8k32), multiplies against the layer's weights held as B fragments in shared
+// memory, and applies the remaining zero-point term of Eq. 3, the bias, the
+// re-quantization and the nibble packing to the accumulators it holds.
+//
+// Zero points.  The B fragments hold w - zb as signed bytes, so the accumulator is
+// sum a*(w - zb) = sum a*w - zb*sum a: Eq. 2's second term (the row sums taken "while
+// unrolling", Section II-B) is absorbed by the multiplication and never formed.  What
+// is left of Eq. 3 is one constant per output channel, K*za*zb - za*sum w.
+//
+// Two input modes:
+//  * packed   (C % 8 == 0, X 4-byte aligned): the copy in shared memory stays packed;
+//    a 32-bit word of a tap is split into its even and odd nibbles, which are exactly
+//    the two A registers of one thread, the same depth permutation being applied to
+//    the weights;
+//  * expanded (any C, e.g. the single-channel first layer): pixels are nibble-granular,
+//    so the copy in shared memory holds one byte per value; the depth is laid out as
+//    KH segments of KW*C contiguous bytes, each padded to a multiple of four with zero
+//    weights, and an A register is one (possibly unaligned) 32-bit word of a segment.
 //
 // Why not the tcgen05 path here: these layers have tiny depth and few output channels
-// (K = 72..288, N = 8..64), so the work per output tile is a few hundred clocks of
+// (K = 9..288, N = 8..64), so the work per output tile is a few hundred clocks of
 // tensor time -- far less than the hand-offs of a TMA / tensor-memory pipeline -- and
 // the traffic saved by not materialising the unrolled matrix (2 * M * K/2 bytes) is
-// what matters.  The register-fragment MMA needs no staging at all: a packed 32-bit
-// word of a row is exactly the two A registers of one thread (even nibbles, odd
-// nibbles), the same depth permutation being applied to the weights.
+// what matters.
 //
-// Requirements (else the caller falls back to unroll + GEMM): C % 8 == 0 (a 32-bit
-// packed word never straddles two taps), OC in {8, 16, 32, 64}, X and Y 16-byte
-// aligned.
+// Requirements (else the caller falls back to unroll + GEMM): OC a multiple of 8 up to
+// 64, Y 8-byte aligned, and the weights, tables and two input buffers fit in shared
+// memory.
+#include <type_traits>
+
 #include "q4_common.cuh"
 
 namespace q4 {
 namespace fused {
 
-constexpr int WARPS = 8;
+constexpr int WARPS = 7;                 // multiplying warps; one more warp produces
 constexpr int ROWS_PER_WARP = 32;
 constexpr int ROWS_PER_CTA = WARPS * ROWS_PER_WARP;
+constexpr int SMEM_LIMIT = 160 * 1024;
+
+// n / d for n < 2^31 as (umulhi(n, mul) + n) >> shift (round-up method: shift =
+// ceil(log2 d), mul = floor(2^32 * (2^shift - d) / d) + 1).
+struct FastDiv {
+    uint32_t mul, shift;
+};
+
+static FastDiv make_fastdiv(uint32_t d)
+{
+    FastDiv f;
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;
+    f.shift = l;
+    f.mul = (uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1);
+    return f;
+}
+
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
+{
+    return (__umulhi(n, f.mul) + n) >> f.shift;
+}
 
 struct Params {
     const uint8_t* X;
@@ -37,70 +75,296 @@ struct Params {
     uint8_t* Y;
     int64_t M;
     int32_t H, W, C, KH, KW, OH, OW, sh, sw, ph, pw;
-    int32_t K, KS;             // depth, number of 32-value depth steps
+    int32_t K, KS;             // depth, number of 32-byte MMA depth steps
     int32_t za, zb;
     RequantParams rq;
+    // staging geometry (host-derived)
+    int32_t unit;              // bytes per input pixel in shared memory (C/2 packed, C expanded)
+    int32_t rowbytes;          // W * unit: bytes of one image row in shared memory
+    int32_t lead;              // bytes before the left halo so that the image data start 16-aligned
+    int32_t pitch;             // bytes per staged row (multiple of 16)
+    int32_t bufbytes;          // one input buffer
+    int32_t segw;              // expanded: 32-bit words per kh segment
+    int32_t sfull;             // staged rows of an image all of whose output rows are in the tile
+    int32_t vec16;             // packed: image rows can be copied in 16-byte pieces
+    int32_t wt_words;          // weights can be read as aligned 32-bit words
+    int32_t cpr;               // packed: copy pieces (16 or 4 bytes) per image row
+    int32_t step8;             // staged-buffer offset of the pixel eight further in the same output row
+    int32_t rowwrap;           // ... added when that pixel is in the next output row
+    int32_t imgwrap;           // ... added on top when that row is the next image's first
+    FastDiv div_ow, div_oh, div_sfull, div_cpr;
 };
 
-__device__ __forceinline__ void mma_u8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                       uint32_t b0, uint32_t b1)
+__device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                         uint32_t b0, uint32_t b1)
 {
     asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
         "{%8, %9}, {%0, %1, %2, %3};"
         : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void cp_async16(void* dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+                 :: "r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* dst, const void* src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
+                 :: "r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.wait_all;" ::: "memory");
+}
+
+// Four nibbles in the low halves of four bytes, minus zb, as four signed bytes.  Setting
+// bit 7 of every byte first keeps the subtraction from borrowing across bytes
+// (128 + x - zb > 0); flipping it back leaves x - zb in two's complement.
+__device__ __forceinline__ uint32_t sub_zb(uint32_t x, uint32_t zb)
+{
+    return ((x | 0x80808080u) - zb * 0x01010101u) ^ 0x80808080u;
+}
+
+__device__ __forceinline__ uint32_t weight_nibble(const Params& p, int n, int k)
+{
+    const uint8_t byte = p.Wt[(int64_t)n * p.ldw + (k >> 1)];
+    return (k & 1) ? (uint32_t)(byte >> 4) : (uint32_t)(byte & 0x0F);
+}
+
+// Which input rows a tile's copy in shared memory holds.  The tile's output rows
+// (index q = n * OH + oh) run from q_first to q_last; the images they belong to are
+// "segments".  A segment's staged rows are the input rows from its first output row's
+// first tap row to its last output row's last tap row.
+struct Geo {
+    int32_t n_first, oh_first;   // image and output row of the tile's first pixel
+    int32_t s0;                  // staged rows of the first segment
+    int32_t nslots;              // staged rows in all
+};
+
+__device__ __forceinline__ Geo tile_geometry(const Params& p, int64_t tile)
+{
+    const int64_t mb = tile * ROWS_PER_CTA;
+    const int64_t me = (mb + ROWS_PER_CTA < p.M ? mb + ROWS_PER_CTA : p.M) - 1;
+    const uint32_t q_first = fdiv((uint32_t)mb, p.div_ow), q_last = fdiv((uint32_t)me, p.div_ow);
+    const uint32_t n_first = fdiv(q_first, p.div_oh), n_last = fdiv(q_last, p.div_oh);
+    const int oh_first = (int)(q_first - n_first * (uint32_t)p.OH);
+    const int oh_last = (int)(q_last - n_last * (uint32_t)p.OH);
+    Geo g;
+    g.n_first = (int)n_first;
+    g.oh_first = oh_first;
+    if (n_first == n_last) {
+        g.s0 = (oh_last - oh_first) * p.sh + p.KH;
+        g.nslots = g.s0;
+    } else {
+        g.s0 = (p.OH - 1 - oh_first) * p.sh + p.KH;
+        g.nslots = g.s0 + (int)(n_last - n_first - 1) * p.sfull + oh_last * p.sh + p.KH;
+    }
+    return g;
+}
+
+// Producer warp, packed mode: copies the image rows of a tile into `buf` with
+// asynchronous copies, one 16-byte (or 4-byte) piece per lane and step.  Only the
+// image columns are written: the lead and the halo columns hold the zero point from
+// the kernel's start.  Rows above or below the image are filled with the zero point.
+__device__ __forceinline__ void stage_packed(const Params& p, const Geo& g, uint8_t* buf, int lane)
+{
+    const int data0 = p.lead + p.pw * p.unit;          // multiple of 16
+    const int cb = p.vec16 ? 16 : 4;
+    const int total = g.nslots * p.cpr;
+    const int ih_first = g.oh_first * p.sh - p.ph;
+    const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
+    for (int idx = lane; idx < total; idx += 32) {
+        const int s = (int)fdiv((uint32_t)idx, p.div_cpr);
+        const int c = (idx - s * p.cpr) * cb;
+        int seg = 0, ih = ih_first + s;
+        if (s >= g.s0) {
+            const uint32_t r = (uint32_t)(s - g.s0);
+            const uint32_t sq = fdiv(r, p.div_sfull);
+            seg = 1 + (int)sq;
+            ih = (int)(r - sq * (uint32_t)p.sfull) - p.ph;
+        }
+        uint8_t* dst = buf + s * p.pitch + data0 + c;
+        if ((unsigned)ih < (unsigned)p.H) {
+            const uint8_t* src = p.X + ((int64_t)(g.n_first + seg) * p.H + ih) * p.rowbytes + c;
+            if (p.vec16) cp_async16(dst, src); else cp_async4(dst, src);
+        } else if (p.vec16) {
+            *reinterpret_cast<uint4*>(dst) = make_uint4(zfill, zfill, zfill, zfill);
+        } else {
+            *reinterpret_cast<uint32_t*>(dst) = zfill;
+        }
+    }
+}
+
+// Producer warp, expanded mode: one byte per value.  A lane takes one packed byte of
+// a row (two values); the loads of eight staged rows are issued before any of them is
+// used, so a tile costs one or two memory round trips.
+__device__ __forceinline__ void stage_expanded(const Params& p, const Geo& g, uint8_t* buf, int lane)
+{
+    constexpr int BATCH = 8;
+    const int data0 = p.lead + p.pw * p.unit;
+    const int wc = p.rowbytes;                         // values per image row
+    const int ih_first = g.oh_first * p.sh - p.ph;
+    for (int sb = 0; sb < g.nslots; sb += BATCH) {
+        for (int jb = 0; jb < (wc + 2) / 2; jb += 32) {
+            const int j = jb + lane;                   // my packed byte of each row
+            uint32_t raw[BATCH];
+            int v0[BATCH];                             // row position of my low nibble; INT_MIN/2 = no row
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                const int s = sb + u;
+                raw[u] = (uint32_t)p.za * 0x11u;
+                v0[u] = -(1 << 30);
+                if (s < g.nslots) {
+                    int seg = 0, ih = ih_first + s;
+                    if (s >= g.s0) {
+                        const uint32_t r = (uint32_t)(s - g.s0);
+                        const uint32_t sq = fdiv(r, p.div_sfull);
+                        seg = 1 + (int)sq;
+                        ih = (int)(r - sq * (uint32_t)p.sfull) - p.ph;
+                    }
+                    v0[u] = 2 * j;
+                    if ((unsigned)ih < (unsigned)p.H) {
+                        const int64_t e0 = ((int64_t)(g.n_first + seg) * p.H + ih) * wc;
+                        v0[u] = 2 * j - (int)(e0 & 1);
+                        if (v0[u] < wc) raw[u] = p.X[(e0 >> 1) + j];
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                uint8_t* dst = buf + (sb + u) * p.pitch + data0;
+                if (v0[u] >= 0 && v0[u] < wc) dst[v0[u]] = (uint8_t)(raw[u] & 0x0Fu);
+                if (v0[u] + 1 >= 0 && v0[u] + 1 < wc) dst[v0[u] + 1] = (uint8_t)(raw[u] >> 4);
+            }
+        }
+    }
+}
+
 // NT = OC / 8 output-channel tiles.  Fragment column f of tile nt is output channel
 // 2 * (NT * (f / 2) + nt) + f % 2, so that the NT packed output bytes a thread ends up
 // with are contiguous in memory.
-#ifndef Q4_FUSED_MIN_CTAS
-#define Q4_FUSED_MIN_CTAS 2
-#endif
-template <int NT>
-__global__ void __launch_bounds__(WARPS * 32, Q4_FUSED_MIN_CTAS)
+//
+// Warps 0..6 multiply; warp 7 is the producer: while the others work on tile k it
+// derives the geometry of tile k+1, copies its input rows into the other buffer and
+// leaves the geometry in shared memory.  One block-wide barrier per tile hands over
+// both the finished copy and the buffer that has just been read.
+constexpr int THREADS = (WARPS + 1) * 32;
+
+__device__ __forceinline__ void tile_barrier()
+{
+    asm volatile("bar.sync 1, %0;" :: "n"(THREADS) : "memory");
+}
+
+template <int NT, bool EXP>
+__global__ void __launch_bounds__(THREADS, NT <= 2 ? 3 : 2)
 conv_fused_kernel(const Params p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
-    uint2* bfrag = reinterpret_cast<uint2*>(smem);                       // [KS][NT][32]
-    int32_t* tab = reinterpret_cast<int32_t*>(smem + (size_t)p.KS * NT * 32 * 8);   // [KS][4] x 2
-    int32_t* colsum_s = tab + p.KS * 4 * 2;                               // [8 * NT]
+    constexpr int TW = EXP ? 8 : 4;                    // table entries per depth step
+    constexpr int N = 8 * NT;
+    uint2* bfrag = reinterpret_cast<uint2*>(smem);                                   // [KS][NT][32]
+    int32_t* tab = reinterpret_cast<int32_t*>(smem + (size_t)p.KS * NT * 32 * 8);    // [KS][TW]
+    int32_t* colsum_s = tab + p.KS * TW;                                             // [N]
+    int4* geo_s = reinterpret_cast<int4*>(colsum_s + N);                             // [2]
+    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + 2);                           // 16-byte aligned
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
-    const int tapb = p.C / 2;                  // bytes per tap
-    const int kbytes = p.K / 2;
-    constexpr int N = 8 * NT;
+    const int kbytes = p.K / 2;                        // packed mode: K is a multiple of 8
+    const int segbytes = p.KW * p.C;                   // expanded mode: bytes per kh segment
 
-    // ---- once per CTA: weights -> B fragments, tap table, weight sums
-    for (int i = tid; i < N; i += blockDim.x) colsum_s[i] = 0;
+    // ---- once per CTA: weights -> signed B fragments, depth table, weight sums, and
+    //      both input buffers filled with the zero point (this is what stays in the halo)
+    for (int i = tid; i < N; i += THREADS) colsum_s[i] = 0;
+    {
+        const uint32_t zfill = (uint32_t)p.za * (EXP ? 0x01010101u : 0x11111111u);
+        uint32_t* b = reinterpret_cast<uint32_t*>(buf0);
+        for (int i = tid; i < 2 * p.bufbytes / 4; i += THREADS) b[i] = zfill;
+    }
     __syncthreads();
-    for (int i = tid; i < p.KS * NT * 32; i += blockDim.x) {
+    for (int i = tid; i < p.KS * NT * 32; i += THREADS) {
         const int l = i & 31, nt = (i >> 5) % NT, j = (i >> 5) / NT;
         const int fg = l >> 2, ft = l & 3;
         const int n = 2 * (NT * (fg >> 1) + nt) + (fg & 1);
-        const int kb = 16 * j + 4 * ft;
-        uint32_t w = 0;
-        if (kb < kbytes) w = *reinterpret_cast<const uint32_t*>(p.Wt + (int64_t)n * p.ldw + kb);
-        bfrag[i] = make_uint2(w & 0x0F0F0F0Fu, (w >> 4) & 0x0F0F0F0Fu);
-        if (!p.colsum_w && w) atomicAdd(&colsum_s[n], nibble_sum(w));
-    }
-    for (int i = tid; i < p.KS * 4; i += blockDim.x) {
-        const int kb = 16 * (i >> 2) + 4 * (i & 3);
-        int delta = -1, khkw = 0;
-        if (kb < kbytes) {
-            const int tap = kb / tapb, off = kb % tapb;
-            const int kh = tap / p.KW, kw = tap % p.KW;
-            delta = (kh * p.W + kw) * tapb + off;
-            khkw = (kh << 16) | kw;
+        uint32_t b0 = 0, b1 = 0;
+        int raw = 0;
+        if (!EXP) {
+            const int kb = 16 * j + 4 * ft;
+            if (kb < kbytes) {
+                uint32_t w;
+                if (p.wt_words) {
+                    w = *reinterpret_cast<const uint32_t*>(p.Wt + (int64_t)n * p.ldw + kb);
+                } else {
+                    w = 0;
+                    for (int q = 0; q < 4; ++q) w |= (uint32_t)p.Wt[(int64_t)n * p.ldw + kb + q] << (8 * q);
+                }
+                raw = nibble_sum(w);
+                b0 = sub_zb(w & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                b1 = sub_zb((w >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
+            }
+        } else {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int wi = 8 * j + 4 * h + ft;
+                const int kh = wi / p.segw, ws = wi % p.segw;
+                uint32_t word = 0;
+                if (kh < p.KH) {
+                    for (int q = 0; q < 4; ++q) {
+                        const int bs = 4 * ws + q;
+                        if (bs < segbytes) {
+                            const uint32_t nib = weight_nibble(p, n, kh * segbytes + bs);
+                            raw += (int)nib;
+                            word |= ((nib - (uint32_t)p.zb) & 0xFFu) << (8 * q);
+                        }
+                    }
+                }
+                if (h == 0) b0 = word; else b1 = word;
+            }
         }
-        tab[2 * i] = delta;
-        tab[2 * i + 1] = khkw;
+        bfrag[i] = make_uint2(b0, b1);
+        if (!p.colsum_w && raw) atomicAdd(&colsum_s[n], raw);
+    }
+    for (int i = tid; i < p.KS * TW; i += THREADS) {
+        int delta = -1;
+        if (!EXP) {
+            const int kb = 16 * (i >> 2) + 4 * (i & 3);
+            if (kb < kbytes) {
+                const int kh = kb / (p.KW * p.unit);
+                delta = kh * p.pitch + (kb - kh * p.KW * p.unit);
+            }
+        } else {
+            const int kh = i / p.segw, ws = i % p.segw;      // i = 8 j + 4 h + t
+            if (kh < p.KH) delta = kh * p.pitch + 4 * ws;
+        }
+        tab[i] = delta;
     }
     __syncthreads();
 
-    // per-thread epilogue constants: the column term of Eq. 3 for my NT channel pairs
+    // Both roles go through the same number of barriers: one before the first tile and
+    // one after each of this CTA's `mytiles` tiles (the grid never exceeds the tile count).
+    const int64_t ntiles = (p.M + ROWS_PER_CTA - 1) / ROWS_PER_CTA;
+    const int mytiles = (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+
+    if (warp == WARPS) {
+        // ---------------- producer ----------------
+        for (int k = -1; k < mytiles; ++k) {
+            if (k + 1 < mytiles) {
+                const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)(k + 1) * gridDim.x);
+                uint8_t* buf = buf0 + ((k + 1) & 1) * p.bufbytes;
+                if (EXP) stage_expanded(p, gn, buf, lane); else stage_packed(p, gn, buf, lane);
+                if (lane == 0) geo_s[(k + 1) & 1] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
+                cp_async_wait_all();
+            }
+            tile_barrier();
+        }
+        return;
+    }
+
+    // ---------------- consumers ----------------
+    // per-thread epilogue constants: what is left of Eq. 3 for my NT channel pairs
     int colterm[NT][2];
     const int kzz = p.K * p.za * p.zb;
 #pragma unroll
@@ -112,145 +376,224 @@ conv_fused_kernel(const Params p)
             colterm[nt][e] = (int)((uint32_t)kzz - (uint32_t)(p.za * cs) +
                                    (uint32_t)(p.bias ? p.bias[n] : 0));
         }
-    const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
+    const int pix0 = p.lead;                           // offset of input column -pw in a staged row
+    const int yoff = (warp * ROWS_PER_WARP + g) * (N / 2) + NT * t;    // my first row within a tile
 
-    const int64_t ntiles = (p.M + ROWS_PER_CTA - 1) / ROWS_PER_CTA;
-    for (int64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const int64_t m0 = tile * ROWS_PER_CTA + warp * ROWS_PER_WARP;
-        if (m0 >= p.M) continue;                       // warp-uniform
-        // my four rows: g, g+8 (first 16-row tile), 16+g, 24+g (second)
-        int ih0[4], iw0[4];
-        const uint8_t* base[4];
-        bool valid[4];
-        {
-            // one division for my first row; the others are 8 pixels further each
-            const int64_t mf = m0 + g;
-            const uint32_t mm = mf < p.M ? (uint32_t)mf : 0u;       // M < 2^31
-            int ow = (int)(mm % (uint32_t)p.OW);
-            const uint32_t q = mm / (uint32_t)p.OW;
-            int oh = (int)(q % (uint32_t)p.OH);
-            int64_t n = q / (uint32_t)p.OH;
+    tile_barrier();
+    for (int k = 0; k < mytiles; ++k) {
+        const int64_t tile = blockIdx.x + (int64_t)k * gridDim.x;
+        const uint8_t* buf = buf0 + (k & 1) * p.bufbytes;
+        const int4 gv = geo_s[k & 1];                  // n_first, oh_first, s0
+        const int64_t mbase = tile * ROWS_PER_CTA;
+        const int64_t left = p.M - mbase;              // > 0
+        const int myrows = (int)(left < ROWS_PER_CTA ? left : ROWS_PER_CTA) - warp * ROWS_PER_WARP;
+        if (myrows > 0) {                              // warp-uniform
+            // my four rows: g, g+8 (first 16-row tile), 16+g, 24+g (second)
+            int base[4], shf[4];
+            {
+                const uint32_t mm = (uint32_t)mbase + (uint32_t)(warp * ROWS_PER_WARP) +
+                                    (uint32_t)(g < myrows ? g : 0);                  // M < 2^31
+                const uint32_t q = fdiv(mm, p.div_ow);
+                int ow = (int)(mm - q * (uint32_t)p.OW);
+                const uint32_t n0 = fdiv(q, p.div_oh);
+                int oh = (int)(q - n0 * (uint32_t)p.OH);
+                int seg = (int)n0 - gv.x;
+                const int slot0 = seg == 0 ? (oh - gv.y) * p.sh : gv.z + (seg - 1) * p.sfull + oh * p.sh;
+                int b = slot0 * p.pitch + pix0 + ow * p.sw * p.unit;
+                const int first = b;
+                if (p.OW >= 8) {
+                    // eight pixels on: at most one step into the next output row (+sh staged
+                    // rows), which may be the next image's first (+KH instead)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                valid[i] = mf + 8 * i < p.M;
-                ih0[i] = oh * p.sh - p.ph;
-                iw0[i] = ow * p.sw - p.pw;
-                base[i] = p.X + ((n * p.H + ih0[i]) * p.W + iw0[i]) * tapb;
-                ow += 8;
-                while (ow >= p.OW) {
-                    ow -= p.OW;
-                    if (++oh == p.OH) { oh = 0; ++n; }
+                    for (int i = 0; i < 4; ++i) {
+                        const int bi = g + 8 * i < myrows ? b : first;   // rows past the end read a valid place
+                        shf[i] = (bi & 3) * 8;
+                        base[i] = EXP ? (bi & ~3) : bi;
+                        ow += 8;
+                        b += p.step8;
+                        if (ow >= p.OW) {
+                            ow -= p.OW;
+                            b += p.rowwrap;
+                            if (++oh == p.OH) { oh = 0; b += p.imgwrap; }
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int s0i = seg == 0 ? (oh - gv.y) * p.sh : gv.z + (seg - 1) * p.sfull + oh * p.sh;
+                        const int bb = s0i * p.pitch + pix0 + ow * p.sw * p.unit;
+                        const int bi = g + 8 * i < myrows ? bb : first;
+                        shf[i] = (bi & 3) * 8;
+                        base[i] = EXP ? (bi & ~3) : bi;
+                        ow += 8;
+                        while (ow >= p.OW) {
+                            ow -= p.OW;
+                            if (++oh == p.OH) { oh = 0; ++seg; }
+                        }
+                    }
                 }
             }
-        }
-        int acc[2][NT][4];
+            int acc[2][NT][4];
 #pragma unroll
-        for (int mt = 0; mt < 2; ++mt)
+            for (int mt = 0; mt < 2; ++mt)
 #pragma unroll
-            for (int nt = 0; nt < NT; ++nt)
+                for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0;
-        int rsum[4] = {0, 0, 0, 0};
+                    for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0;
 
-        // gather of one depth step: my packed word of each of my four rows (the zero
-        // point outside the image, zero past the depth)
-        auto gather = [&](int j, uint32_t (&w)[4]) {
-            const int delta = tab[2 * (4 * j + t)];
-            const int khkw = tab[2 * (4 * j + t) + 1];
-            const int kh = khkw >> 16, kw = khkw & 0xFFFF;
+            for (int j = 0; j < p.KS; ++j) {
+                uint32_t a[2][4];
+                if (!EXP) {
+                    // one packed word per row: even nibbles feed depth 4t.., odd ones 16+4t..
+                    const int delta = tab[4 * j + t];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                w[i] = 0;
-                if (delta >= 0) {
-                    const int ih = ih0[i] + kh, iw = iw0[i] + kw;
-                    w[i] = zfill;
-                    if (valid[i] && (unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W)
-                        w[i] = __ldg(reinterpret_cast<const uint32_t*>(base[i] + delta));
+                    for (int i = 0; i < 4; ++i) {
+                        uint32_t w = 0;
+                        if (delta >= 0) w = *reinterpret_cast<const uint32_t*>(buf + base[i] + delta);
+                        a[0][i] = w & 0x0F0F0F0Fu;
+                        a[1][i] = (w >> 4) & 0x0F0F0F0Fu;
+                    }
+                } else {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int delta = tab[8 * j + 4 * h + t];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint32_t w = 0;
+                            if (delta >= 0) {
+                                const uint32_t* src = reinterpret_cast<const uint32_t*>(buf + base[i] + delta);
+                                w = __funnelshift_r(src[0], src[1], shf[i]);
+                            }
+                            a[h][i] = w;
+                        }
+                    }
+                }
+                const uint2* bj = bfrag + (size_t)j * NT * 32 + lane;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const uint2 b = bj[nt * 32];
+                    mma_u8s8(acc[0][nt], a[0][0], a[0][1], a[1][0], a[1][1], b.x, b.y);
+                    mma_u8s8(acc[1][nt], a[0][2], a[0][3], a[1][2], a[1][3], b.x, b.y);
                 }
             }
-        };
-        uint32_t wcur[4], wnext[4];
-        gather(0, wcur);
-        for (int j = 0; j < p.KS; ++j) {
-            if (j + 1 < p.KS) gather(j + 1, wnext);      // in flight while this step multiplies
-            uint32_t lo[4], hi[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                lo[i] = wcur[i] & 0x0F0F0F0Fu;
-                hi[i] = (wcur[i] >> 4) & 0x0F0F0F0Fu;
-                rsum[i] = dp4a_u8(lo[i] + hi[i], 0x01010101u, rsum[i]);
-            }
-            const uint2* bj = bfrag + (size_t)j * NT * 32 + lane;
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const uint2 b = bj[nt * 32];
-                mma_u8(acc[0][nt], lo[0], lo[1], hi[0], hi[1], b.x, b.y);
-                mma_u8(acc[1][nt], lo[2], lo[3], hi[2], hi[3], b.x, b.y);
-            }
-#pragma unroll
-            for (int i = 0; i < 4; ++i) wcur[i] = wnext[i];
-        }
 
-        // row sums: add the four depth slices held by the lanes of a row
+            // epilogue: accumulator (mt, nt) holds rows g + 16 mt (c0, c1) and g + 8 + 16 mt
+            // (c2, c3), fragment columns 2t, 2t+1
+            uint8_t* ytile = p.Y + mbase * (N / 2) + yoff;
+            auto epilogue = [&](auto fast_tag) {
+                constexpr bool FAST = decltype(fast_tag)::value;
+                const int s = p.rq.shift - 1, rnd = FAST ? 1 << (s - 1) : 0;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            rsum[i] += __shfl_xor_sync(0xFFFFFFFFu, rsum[i], 1);
-            rsum[i] += __shfl_xor_sync(0xFFFFFFFFu, rsum[i], 2);
+                for (int i = 0; i < 4; ++i) {
+                    const int mt = i >> 1, hrow = i & 1;
+                    if (g + 8 * i >= myrows) continue;
+                    uint32_t bytes[NT];
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        uint32_t qv[2];
+#pragma unroll
+                        for (int e = 0; e < 2; ++e) {
+                            const int v = (int)((uint32_t)acc[mt][nt][2 * hrow + e] + (uint32_t)colterm[nt][e]);
+                            if (FAST) {
+                                int q = ((__mulhi(v, p.rq.mult) + rnd) >> s) + p.rq.zo;
+                                q = max(q, p.rq.lo);
+                                qv[e] = (uint32_t)min(q, p.rq.hi);
+                            } else {
+                                qv[e] = requant_wide(v, p.rq);
+                            }
+                        }
+                        bytes[nt] = qv[0] | (qv[1] << 4);
+                    }
+                    uint8_t* dst = ytile + i * (8 * (N / 2));
+                    if (NT % 4 == 0) {
+#pragma unroll
+                        for (int q = 0; q < NT / 4; ++q)
+                            reinterpret_cast<uint32_t*>(dst)[q] =
+                                bytes[(4 * q) % NT] | (bytes[(4 * q + 1) % NT] << 8) |
+                                (bytes[(4 * q + 2) % NT] << 16) | (bytes[(4 * q + 3) % NT] << 24);
+                    } else if (NT % 2 == 0) {
+#pragma unroll
+                        for (int q = 0; q < NT / 2; ++q)
+                            reinterpret_cast<uint16_t*>(dst)[q] =
+                                (uint16_t)(bytes[(2 * q) % NT] | (bytes[(2 * q + 1) % NT] << 8));
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < NT; ++q) dst[q] = (uint8_t)bytes[q];
+                    }
+                }
+            };
+            // the 32-bit form of the rounding shift needs shift >= 2 (see requant())
+            if (p.rq.shift >= 2) epilogue(std::true_type{}); else epilogue(std::false_type{});
         }
-        // epilogue: accumulator (mt, nt) holds rows g + 16 mt (c0, c1) and g + 8 + 16 mt
-        // (c2, c3), fragment columns 2t, 2t+1
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int mt = i >> 1, hrow = i & 1;
-            const int64_t m = m0 + g + 8 * i;
-            if (m >= p.M) continue;
-            const uint32_t rowterm = (uint32_t)0 - (uint32_t)(p.zb * rsum[i]);
-            uint32_t bytes[NT];
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-                const int v0 = (int)((uint32_t)acc[mt][nt][2 * hrow] + rowterm + (uint32_t)colterm[nt][0]);
-                const int v1 = (int)((uint32_t)acc[mt][nt][2 * hrow + 1] + rowterm + (uint32_t)colterm[nt][1]);
-                bytes[nt] = requant(v0, p.rq) | (requant(v1, p.rq) << 4);
-            }
-            uint8_t* dst = p.Y + m * (N / 2) + NT * t;
-            if (NT == 8) {
-                const uint32_t w0 = bytes[0] | (bytes[1] << 8) | (bytes[2] << 16) | (bytes[3] << 24);
-                const uint32_t w1 = bytes[4 % NT] | (bytes[5 % NT] << 8) | (bytes[6 % NT] << 16) | (bytes[7 % NT] << 24);
-                *reinterpret_cast<uint2*>(dst) = make_uint2(w0, w1);
-            } else if (NT == 4) {
-                *reinterpret_cast<uint32_t*>(dst) =
-                    bytes[0] | (bytes[1 % NT] << 8) | (bytes[2 % NT] << 16) | (bytes[3 % NT] << 24);
-            } else if (NT == 2) {
-                *reinterpret_cast<uint16_t*>(dst) = (uint16_t)(bytes[0] | (bytes[1 % NT] << 8));
-            } else {
-                *dst = (uint8_t)bytes[0];
-            }
-        }
+        tile_barrier();
     }
 }
 
 }  // namespace fused
 
+// Fills the host-derived fields of the launch parameters; returns the dynamic shared
+// memory the kernel needs (0 = the layer does not fit this kernel).
+static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt,
+                         int64_t ldw, bool& expanded)
+{
+    if (d.OC % 8 != 0 || d.OC < 8 || d.OC > 64) return 0;
+    if (d.KH > 64 || d.KW > 64 || d.stride_h > 64 || d.stride_w > 64) return 0;
+    p.H = d.H; p.W = d.W; p.C = d.C; p.KH = d.KH; p.KW = d.KW;
+    p.sh = d.stride_h; p.sw = d.stride_w; p.ph = d.pad_h; p.pw = d.pad_w;
+    p.OH = (d.H + 2 * d.pad_h - d.KH) / d.stride_h + 1;
+    p.OW = (d.W + 2 * d.pad_w - d.KW) / d.stride_w + 1;
+    p.M = (int64_t)d.N * p.OH * p.OW;
+    p.K = d.KH * d.KW * d.C;
+    expanded = !(d.C % 8 == 0 && (uintptr_t)X % 4 == 0);
+    const int64_t unit = expanded ? d.C : d.C / 2;
+    const int64_t rowbytes = (int64_t)d.W * unit;
+    const int64_t lead = (16 - (d.pad_w * unit) % 16) % 16;
+    const int64_t pitch = (lead + ((int64_t)d.W + 2 * d.pad_w) * unit + 15) / 16 * 16;
+    // a tile's consecutive pixels touch at most `rows` output rows in `nseg` images
+    const int64_t rows = (fused::ROWS_PER_CTA - 1 + p.OW - 1) / p.OW + 1;
+    const int64_t nseg = (rows - 1 + p.OH - 1) / p.OH + 1;
+    const int64_t slots = rows * d.stride_h + nseg * (d.KH > d.stride_h ? d.KH - d.stride_h : 0);
+    const int64_t bufbytes = slots * pitch + 16;       // the slack takes the expanded mode's over-read
+    const int64_t segw = expanded ? ((int64_t)d.KW * d.C + 3) / 4 : 1;
+    const int64_t KS = expanded ? ((int64_t)d.KH * segw + 7) / 8 : ((int64_t)p.K + 31) / 32;
+    const int64_t smem = KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 4 + 32 + 2 * bufbytes;
+    if (smem > fused::SMEM_LIMIT) return 0;
+    p.unit = (int32_t)unit; p.rowbytes = (int32_t)rowbytes; p.lead = (int32_t)lead;
+    p.pitch = (int32_t)pitch; p.bufbytes = (int32_t)bufbytes; p.segw = (int32_t)segw;
+    p.KS = (int32_t)KS;
+    p.sfull = (p.OH - 1) * d.stride_h + d.KH;
+    p.vec16 = !expanded && rowbytes % 16 == 0 && (uintptr_t)X % 16 == 0;
+    p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
+    p.div_ow = fused::make_fastdiv((uint32_t)p.OW);
+    p.div_oh = fused::make_fastdiv((uint32_t)p.OH);
+    p.div_sfull = fused::make_fastdiv((uint32_t)p.sfull);
+    p.cpr = (int32_t)(rowbytes / (p.vec16 ? 16 : 4));
+    if (p.cpr < 1) p.cpr = 1;                          // expanded mode does not use it
+    p.div_cpr = fused::make_fastdiv((uint32_t)p.cpr);
+    p.step8 = (int32_t)(8 * d.stride_w * unit);
+    p.rowwrap = (int32_t)(d.stride_h * pitch - (int64_t)p.OW * d.stride_w * unit);
+    p.imgwrap = (int32_t)((d.KH - d.stride_h) * pitch);
+    return (size_t)smem;
+}
+
 bool conv_fused_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                           const uint8_t* Y)
 {
-    if (d.C % 8 != 0) return false;
-    if (d.OC != 8 && d.OC != 16 && d.OC != 32 && d.OC != 64) return false;
-    if ((uintptr_t)X % 16 || (uintptr_t)Y % 16 || (uintptr_t)Wt % 4 || ldw % 4) return false;
-    const int K = d.KH * d.KW * d.C;
-    const int KS = (K + 31) / 32;
-    const size_t smem = (size_t)KS * (d.OC / 8) * 32 * 8 + (size_t)KS * 4 * 8 + (size_t)d.OC * 4;
-    return smem <= 96 * 1024 && d.KH < 256 && d.KW < 256;
+    if ((uintptr_t)Y % 8) return false;
+    fused::Params p;
+    bool expanded;
+    return plan_fused(p, d, X, Wt, ldw, expanded) != 0;
 }
 
-template <int NT>
+template <int NT, bool EXP>
 static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
     static bool attr = false;
     static int sms = 148;
     if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(fused::conv_fused_kernel<NT>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, 96 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(fused::conv_fused_kernel<NT, EXP>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             fused::SMEM_LIMIT);
         if (e != cudaSuccess) return e;
         int dev = 0;
         cudaGetDevice(&dev);
@@ -260,14 +603,29 @@ static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles,
     // persistent CTAs: as many as are resident at once, so the per-CTA set-up (weights to
     // fragments) is paid once per SM slot and there is no second wave
     int per_sm = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused::conv_fused_kernel<NT>,
-                                                      fused::WARPS * 32, smem) != cudaSuccess || per_sm < 1)
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused::conv_fused_kernel<NT, EXP>,
+                                                      fused::THREADS, smem) != cudaSuccess || per_sm < 1)
         per_sm = 1;
     const int64_t resident = (int64_t)sms * per_sm;
     const int grid = (int)(tiles < resident ? tiles : resident);
-    fused::conv_fused_kernel<NT><<<grid, fused::WARPS * 32, smem, st>>>(p);
+    fused::conv_fused_kernel<NT, EXP><<<grid, fused::THREADS, smem, st>>>(p);
     count_launch();
     return cudaGetLastError();
+}
+
+template <bool EXP>
+static cudaError_t launch_mode(int NT, const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
+{
+    switch (NT) {
+        case 1: return launch_nt<1, EXP>(p, smem, tiles, st);
+        case 2: return launch_nt<2, EXP>(p, smem, tiles, st);
+        case 3: return launch_nt<3, EXP>(p, smem, tiles, st);
+        case 4: return launch_nt<4, EXP>(p, smem, tiles, st);
+        case 5: return launch_nt<5, EXP>(p, smem, tiles, st);
+        case 6: return launch_nt<6, EXP>(p, smem, tiles, st);
+        case 7: return launch_nt<7, EXP>(p, smem, tiles, st);
+        default: return launch_nt<8, EXP>(p, smem, tiles, st);
+    }
 }
 
 cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
@@ -276,25 +634,15 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                               cudaStream_t st)
 {
     fused::Params p;
+    bool expanded = false;
+    const size_t smem = plan_fused(p, d, X, Wt, ldw, expanded);
+    if (smem == 0) return cudaErrorInvalidValue;
     p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;
-    p.H = d.H; p.W = d.W; p.C = d.C; p.KH = d.KH; p.KW = d.KW;
-    p.sh = d.stride_h; p.sw = d.stride_w; p.ph = d.pad_h; p.pw = d.pad_w;
-    p.OH = (d.H + 2 * d.pad_h - d.KH) / d.stride_h + 1;
-    p.OW = (d.W + 2 * d.pad_w - d.KW) / d.stride_w + 1;
-    p.M = (int64_t)d.N * p.OH * p.OW;
-    p.K = d.KH * d.KW * d.C;
-    p.KS = (p.K + 31) / 32;
     p.za = za; p.zb = zb; p.rq = rq;
     if (p.M == 0) return cudaSuccess;
-    const int NT = d.OC / 8;
-    const size_t smem = (size_t)p.KS * NT * 32 * 8 + (size_t)p.KS * 4 * 8 + (size_t)d.OC * 4;
     const int64_t tiles = (p.M + fused::ROWS_PER_CTA - 1) / fused::ROWS_PER_CTA;
-    switch (NT) {
-        case 1: return launch_nt<1>(p, smem, tiles, st);
-        case 2: return launch_nt<2>(p, smem, tiles, st);
-        case 4: return launch_nt<4>(p, smem, tiles, st);
-        default: return launch_nt<8>(p, smem, tiles, st);
-    }
+    return expanded ? launch_mode<true>(d.OC / 8, p, smem, tiles, st)
+                    : launch_mode<false>(d.OC / 8, p, smem, tiles, st);
 }
 
 }  // namespace q4
