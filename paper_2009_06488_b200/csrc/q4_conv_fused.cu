@@ -81,7 +81,9 @@ struct Params {
     // staging geometry (host-derived)
     int32_t unit;              // bytes per input pixel in shared memory (C/2 packed, C expanded)
     int32_t rowbytes;          // W * unit: bytes of one image row in shared memory
-    int32_t lead;              // bytes before the left halo so that the image data start 16-aligned
+    int32_t data0;             // byte offset of input column 0 in a staged row (multiple of 16)
+    int32_t pix0;              // offset of input column -pw in a staged row, in bytes (nibbles in
+                               // the per-lane kernel's packed mode)
     int32_t pitch;             // bytes per staged row (multiple of 16)
     int32_t bufbytes;          // one input buffer
     int32_t segw;              // expanded: 32-bit words per kh segment
@@ -171,7 +173,7 @@ __device__ __forceinline__ Geo tile_geometry(const Params& p, int64_t tile)
 // the kernel's start.  Rows above or below the image are filled with the zero point.
 __device__ __forceinline__ void stage_packed(const Params& p, const Geo& g, uint8_t* buf, int lane)
 {
-    const int data0 = p.lead + p.pw * p.unit;          // multiple of 16
+    const int data0 = p.data0;
     const int cb = p.vec16 ? 16 : 4;
     const int total = g.nslots * p.cpr;
     const int ih_first = g.oh_first * p.sh - p.ph;
@@ -204,7 +206,7 @@ __device__ __forceinline__ void stage_packed(const Params& p, const Geo& g, uint
 __device__ __forceinline__ void stage_expanded(const Params& p, const Geo& g, uint8_t* buf, int lane)
 {
     constexpr int BATCH = 8;
-    const int data0 = p.lead + p.pw * p.unit;
+    const int data0 = p.data0;
     const int wc = p.rowbytes;                         // values per image row
     const int ih_first = g.oh_first * p.sh - p.ph;
     for (int sb = 0; sb < g.nslots; sb += BATCH) {
@@ -376,7 +378,7 @@ conv_fused_kernel(const Params p)
             colterm[nt][e] = (int)((uint32_t)kzz - (uint32_t)(p.za * cs) +
                                    (uint32_t)(p.bias ? p.bias[n] : 0));
         }
-    const int pix0 = p.lead;                           // offset of input column -pw in a staged row
+    const int pix0 = p.pix0;
     const int yoff = (warp * ROWS_PER_WARP + g) * (N / 2) + NT * t;    // my first row within a tile
 
     tile_barrier();
@@ -529,12 +531,186 @@ conv_fused_kernel(const Params p)
     }
 }
 
+
+// ---------------------------------------------------------------------------------
+// One output pixel per lane.  For the thinnest layers (a single-channel first layer:
+// depth 9 or 25, eight outputs) an MMA tile is almost empty and the fragment layout --
+// four pixels per thread, two columns each -- costs more index arithmetic than the layer
+// has multiplications.  Here a lane owns one pixel and all its output channels: it reads
+// its taps from the same expanded copy in shared memory, one 32-bit word of a kh segment
+// at a time, and multiplies with 4-way byte dot products (u8 x s8) against weight words
+// that every lane reads from the same shared-memory address.  The packed output of a
+// pixel is one 4- or 8-byte store, a warp's is contiguous.
+// ---------------------------------------------------------------------------------
+__device__ __forceinline__ int dp4a_u8s8(uint32_t a, uint32_t b, int c)
+{
+    int d;
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+__device__ __forceinline__ int mulhi_add(int a, int b, int c)
+{
+    int d;
+    asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+template <int OC, bool NIB>
+__global__ void __launch_bounds__(THREADS, 3)
+conv_lane_kernel(const Params p)
+{
+    extern __shared__ __align__(16) uint8_t smem[];
+    const int nw = p.KH * p.segw;                      // 32-bit depth words per pixel
+    uint32_t* wsm = reinterpret_cast<uint32_t*>(smem);                               // [nw][OC]
+    int32_t* colterm_s = reinterpret_cast<int32_t*>(wsm + nw * OC);                  // [OC]
+    int4* geo_s = reinterpret_cast<int4*>(colterm_s + OC);                           // [2]
+    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + 2);                           // 16-byte aligned
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int segbytes = p.KW * p.C;
+
+    // ---- once per CTA: signed weight words, the constant left of Eq. 3, zero-point fill
+    for (int i = tid; i < OC; i += THREADS) colterm_s[i] = 0;
+    {
+        uint32_t* b = reinterpret_cast<uint32_t*>(buf0);
+        const uint32_t zfill = (uint32_t)p.za * (NIB ? 0x11111111u : 0x01010101u);
+        for (int i = tid; i < 2 * p.bufbytes / 4; i += THREADS) b[i] = zfill;
+    }
+    __syncthreads();
+    for (int i = tid; i < nw * OC; i += THREADS) {
+        const int n = i % OC, wi = i / OC;
+        const int kh = wi / p.segw, ws = wi % p.segw;
+        uint32_t word = 0;
+        int raw = 0;
+        for (int q = 0; q < 4; ++q) {
+            const int bs = 4 * ws + q;
+            if (bs < segbytes) {
+                const uint32_t nib = weight_nibble(p, n, kh * segbytes + bs);
+                raw += (int)nib;
+                word |= ((nib - (uint32_t)p.zb) & 0xFFu) << (8 * q);
+            }
+        }
+        wsm[i] = word;
+        if (!p.colsum_w && raw) atomicAdd(&colterm_s[n], raw);
+    }
+    __syncthreads();
+    if (tid < OC) {
+        const int cs = p.colsum_w ? p.colsum_w[tid] : colterm_s[tid];
+        colterm_s[tid] = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
+                               (uint32_t)(p.bias ? p.bias[tid] : 0));
+    }
+    __syncthreads();
+
+    const int64_t ntiles = (p.M + ROWS_PER_CTA - 1) / ROWS_PER_CTA;
+    const int mytiles = (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+
+    if (warp == WARPS) {
+        // ---------------- producer (same protocol as conv_fused_kernel) ----------------
+        for (int k = -1; k < mytiles; ++k) {
+            if (k + 1 < mytiles) {
+                const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)(k + 1) * gridDim.x);
+                uint8_t* buf = buf0 + ((k + 1) & 1) * p.bufbytes;
+                if (NIB) stage_packed(p, gn, buf, lane); else stage_expanded(p, gn, buf, lane);
+                if (lane == 0) geo_s[(k + 1) & 1] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
+                if (NIB) cp_async_wait_all();
+            }
+            tile_barrier();
+        }
+        return;
+    }
+
+    // ---------------- consumers ----------------
+    const int pix0 = p.pix0;
+    const int r = warp * ROWS_PER_WARP + lane;         // my pixel within a tile
+    tile_barrier();
+    for (int k = 0; k < mytiles; ++k) {
+        const int64_t tile = blockIdx.x + (int64_t)k * gridDim.x;
+        const uint8_t* buf = buf0 + (k & 1) * p.bufbytes;
+        const int4 gv = geo_s[k & 1];                  // n_first, oh_first, s0
+        const int64_t mbase = tile * ROWS_PER_CTA;
+        const int64_t left = p.M - mbase;              // > 0
+        const int rows = (int)(left < ROWS_PER_CTA ? left : ROWS_PER_CTA);
+        if (warp * ROWS_PER_WARP < rows) {             // warp-uniform
+            const bool valid = r < rows;
+            const uint32_t mm = (uint32_t)mbase + (uint32_t)(valid ? r : 0);       // M < 2^31
+            const uint32_t q = fdiv(mm, p.div_ow);
+            const int ow = (int)(mm - q * (uint32_t)p.OW);
+            const uint32_t n0 = fdiv(q, p.div_oh);
+            const int oh = (int)(q - n0 * (uint32_t)p.OH);
+            const int seg = (int)n0 - gv.x;
+            const int slot0 = seg == 0 ? (oh - gv.y) * p.sh : gv.z + (seg - 1) * p.sfull + oh * p.sh;
+            // where my pixel's first tap starts: a byte offset (expanded copy), or a nibble
+            // offset (packed copy); `shf` is its bit offset within the aligned word at `src`
+            const int b = slot0 * p.pitch * (NIB ? 2 : 1) + pix0 + ow * p.sw * p.unit;
+            const int shf = NIB ? (b & 7) * 4 : (b & 3) * 8;
+            const uint8_t* src = buf + (NIB ? (b >> 3) << 2 : b & ~3);
+
+            int acc[OC];
+#pragma unroll
+            for (int n = 0; n < OC; n += 4) {
+                const int4 c = *reinterpret_cast<const int4*>(colterm_s + n);
+                acc[n] = c.x; acc[n + 1] = c.y; acc[n + 2] = c.z; acc[n + 3] = c.w;
+            }
+            const uint32_t* wrow = wsm;
+            for (int kh = 0; kh < p.KH; ++kh) {
+                const uint32_t* arow = reinterpret_cast<const uint32_t*>(src + kh * p.pitch);
+                for (int ws = 0; ws < p.segw; ++ws) {
+                    uint32_t a;
+                    if (NIB) {
+                        // four nibbles -> four bytes
+                        const int bo = shf + 16 * ws;
+                        uint32_t x = __funnelshift_r(arow[bo >> 5], arow[(bo >> 5) + 1], bo & 31) & 0xFFFFu;
+                        x = (x | (x << 8)) & 0x00FF00FFu;
+                        a = (x | (x << 4)) & 0x0F0F0F0Fu;
+                    } else {
+                        a = __funnelshift_r(arow[ws], arow[ws + 1], shf);
+                    }
+#pragma unroll
+                    for (int n = 0; n < OC; n += 4) {
+                        const uint4 w = *reinterpret_cast<const uint4*>(wrow + n);
+                        acc[n] = dp4a_u8s8(a, w.x, acc[n]);
+                        acc[n + 1] = dp4a_u8s8(a, w.y, acc[n + 1]);
+                        acc[n + 2] = dp4a_u8s8(a, w.z, acc[n + 2]);
+                        acc[n + 3] = dp4a_u8s8(a, w.w, acc[n + 3]);
+                    }
+                    wrow += OC;
+                }
+            }
+
+            uint32_t out[OC / 8];
+            if (p.rq.shift >= 2) {
+                // the 32-bit form of the rounding shift (see requant())
+                const int s = p.rq.shift - 1, rnd = 1 << (s - 1);
+#pragma unroll
+                for (int n = 0; n < OC; ++n) {
+                    int qv = (mulhi_add(acc[n], p.rq.mult, rnd) >> s) + p.rq.zo;
+                    qv = min(max(qv, p.rq.lo), p.rq.hi);
+                    if (n % 8 == 0) out[n / 8] = (uint32_t)qv; else out[n / 8] |= (uint32_t)qv << (4 * (n % 8));
+                }
+            } else {
+#pragma unroll
+                for (int n = 0; n < OC; ++n) {
+                    const uint32_t qv = requant_wide(acc[n], p.rq);
+                    if (n % 8 == 0) out[n / 8] = qv; else out[n / 8] |= qv << (4 * (n % 8));
+                }
+            }
+            if (valid) {
+                uint8_t* dst = p.Y + (mbase + r) * (OC / 2);
+                if (OC == 8) *reinterpret_cast<uint32_t*>(dst) = out[0];
+                else *reinterpret_cast<uint2*>(dst) = make_uint2(out[0], out[(OC / 8 - 1)]);
+            }
+        }
+        tile_barrier();
+    }
+}
+
 }  // namespace fused
 
 // Fills the host-derived fields of the launch parameters; returns the dynamic shared
 // memory the kernel needs (0 = the layer does not fit this kernel).
 static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt,
-                         int64_t ldw, bool& expanded)
+                         int64_t ldw, bool& expanded, bool& per_lane, bool& nibbles)
 {
     if (d.OC % 8 != 0 || d.OC < 8 || d.OC > 64) return 0;
     if (d.KH > 64 || d.KW > 64 || d.stride_h > 64 || d.stride_w > 64) return 0;
@@ -545,24 +721,41 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     p.M = (int64_t)d.N * p.OH * p.OW;
     p.K = d.KH * d.KW * d.C;
     expanded = !(d.C % 8 == 0 && (uintptr_t)X % 4 == 0);
-    const int64_t unit = expanded ? d.C : d.C / 2;
-    const int64_t rowbytes = (int64_t)d.W * unit;
-    const int64_t lead = (16 - (d.pad_w * unit) % 16) % 16;
-    const int64_t pitch = (lead + ((int64_t)d.W + 2 * d.pad_w) * unit + 15) / 16 * 16;
+    const int64_t segw = expanded ? ((int64_t)d.KW * d.C + 3) / 4 : 1;
+    // thinnest layers: one pixel per lane, byte dot products (at most 128 per pixel); their
+    // copy in shared memory stays packed when image rows are whole 32-bit words
+    per_lane = expanded && (d.OC == 8 || d.OC == 16) && (int64_t)d.KH * segw * d.OC <= 128;
+    nibbles = per_lane && ((int64_t)d.W * d.C) % 8 == 0 && (uintptr_t)X % 4 == 0;
+    int64_t unit, rowbytes, data0, pix0, pitch;
+    if (nibbles) {
+        const int64_t halo = ((int64_t)d.pad_w * d.C + 1) / 2;     // bytes that hold a side's halo
+        unit = d.C;                                                // nibbles per pixel
+        rowbytes = (int64_t)d.W * d.C / 2;
+        data0 = (halo + 15) / 16 * 16;
+        pix0 = 2 * data0 - (int64_t)d.pad_w * d.C;
+        pitch = (data0 + rowbytes + halo + 15) / 16 * 16;
+    } else {
+        unit = expanded ? d.C : d.C / 2;
+        rowbytes = (int64_t)d.W * unit;
+        data0 = (d.pad_w * unit + 15) / 16 * 16;
+        pix0 = data0 - d.pad_w * unit;
+        pitch = (data0 + rowbytes + d.pad_w * unit + 15) / 16 * 16;
+    }
     // a tile's consecutive pixels touch at most `rows` output rows in `nseg` images
     const int64_t rows = (fused::ROWS_PER_CTA - 1 + p.OW - 1) / p.OW + 1;
     const int64_t nseg = (rows - 1 + p.OH - 1) / p.OH + 1;
     const int64_t slots = rows * d.stride_h + nseg * (d.KH > d.stride_h ? d.KH - d.stride_h : 0);
-    const int64_t bufbytes = slots * pitch + 16;       // the slack takes the expanded mode's over-read
-    const int64_t segw = expanded ? ((int64_t)d.KW * d.C + 3) / 4 : 1;
+    const int64_t bufbytes = slots * pitch + 16;       // the slack takes the unaligned words' over-read
     const int64_t KS = expanded ? ((int64_t)d.KH * segw + 7) / 8 : ((int64_t)p.K + 31) / 32;
-    const int64_t smem = KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 4 + 32 + 2 * bufbytes;
+    const int64_t smem = per_lane
+        ? (int64_t)d.KH * segw * d.OC * 4 + (int64_t)d.OC * 4 + 32 + 2 * bufbytes
+        : KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 4 + 32 + 2 * bufbytes;
     if (smem > fused::SMEM_LIMIT) return 0;
-    p.unit = (int32_t)unit; p.rowbytes = (int32_t)rowbytes; p.lead = (int32_t)lead;
+    p.unit = (int32_t)unit; p.rowbytes = (int32_t)rowbytes; p.data0 = (int32_t)data0; p.pix0 = (int32_t)pix0;
     p.pitch = (int32_t)pitch; p.bufbytes = (int32_t)bufbytes; p.segw = (int32_t)segw;
     p.KS = (int32_t)KS;
     p.sfull = (p.OH - 1) * d.stride_h + d.KH;
-    p.vec16 = !expanded && rowbytes % 16 == 0 && (uintptr_t)X % 16 == 0;
+    p.vec16 = (!expanded || nibbles) && rowbytes % 16 == 0 && (uintptr_t)X % 16 == 0;
     p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
     p.div_ow = fused::make_fastdiv((uint32_t)p.OW);
     p.div_oh = fused::make_fastdiv((uint32_t)p.OH);
@@ -581,36 +774,40 @@ bool conv_fused_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t
 {
     if ((uintptr_t)Y % 8) return false;
     fused::Params p;
-    bool expanded;
-    return plan_fused(p, d, X, Wt, ldw, expanded) != 0;
+    bool expanded, per_lane, nibbles;
+    return plan_fused(p, d, X, Wt, ldw, expanded, per_lane, nibbles) != 0;
+}
+
+// Launches one of the kernels above as persistent CTAs: as many as are resident at
+// once, so the per-CTA set-up (weights to fragments) is paid once per SM slot and there
+// is no second wave.
+using FusedKernel = void (*)(const fused::Params);
+
+static cudaError_t launch_kernel(FusedKernel kernel, const fused::Params& p, size_t smem, int64_t tiles,
+                                 cudaStream_t st)
+{
+    // the attribute is per kernel (and per device: set on every call, it is cheap)
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         fused::SMEM_LIMIT);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 148, per_sm = 1;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        sms = 148;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, fused::THREADS, smem) != cudaSuccess ||
+        per_sm < 1)
+        per_sm = 1;
+    const int64_t resident = (int64_t)sms * per_sm;
+    const int grid = (int)(tiles < resident ? tiles : resident);
+    kernel<<<grid, fused::THREADS, smem, st>>>(p);
+    count_launch();
+    return cudaGetLastError();
 }
 
 template <int NT, bool EXP>
 static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
-    static bool attr = false;
-    static int sms = 148;
-    if (!attr) {
-        cudaError_t e = cudaFuncSetAttribute(fused::conv_fused_kernel<NT, EXP>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             fused::SMEM_LIMIT);
-        if (e != cudaSuccess) return e;
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        attr = true;
-    }
-    // persistent CTAs: as many as are resident at once, so the per-CTA set-up (weights to
-    // fragments) is paid once per SM slot and there is no second wave
-    int per_sm = 1;
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fused::conv_fused_kernel<NT, EXP>,
-                                                      fused::THREADS, smem) != cudaSuccess || per_sm < 1)
-        per_sm = 1;
-    const int64_t resident = (int64_t)sms * per_sm;
-    const int grid = (int)(tiles < resident ? tiles : resident);
-    fused::conv_fused_kernel<NT, EXP><<<grid, fused::THREADS, smem, st>>>(p);
-    count_launch();
-    return cudaGetLastError();
+    return launch_kernel(fused::conv_fused_kernel<NT, EXP>, p, smem, tiles, st);
 }
 
 template <bool EXP>
@@ -634,13 +831,20 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                               cudaStream_t st)
 {
     fused::Params p;
-    bool expanded = false;
-    const size_t smem = plan_fused(p, d, X, Wt, ldw, expanded);
+    bool expanded = false, per_lane = false, nibbles = false;
+    const size_t smem = plan_fused(p, d, X, Wt, ldw, expanded, per_lane, nibbles);
     if (smem == 0) return cudaErrorInvalidValue;
     p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;
     p.za = za; p.zb = zb; p.rq = rq;
     if (p.M == 0) return cudaSuccess;
     const int64_t tiles = (p.M + fused::ROWS_PER_CTA - 1) / fused::ROWS_PER_CTA;
+    if (per_lane) {
+        if (nibbles)
+            return d.OC == 8 ? launch_kernel(fused::conv_lane_kernel<8, true>, p, smem, tiles, st)
+                             : launch_kernel(fused::conv_lane_kernel<16, true>, p, smem, tiles, st);
+        return d.OC == 8 ? launch_kernel(fused::conv_lane_kernel<8, false>, p, smem, tiles, st)
+                         : launch_kernel(fused::conv_lane_kernel<16, false>, p, smem, tiles, st);
+    }
     return expanded ? launch_mode<true>(d.OC / 8, p, smem, tiles, st)
                     : launch_mode<false>(d.OC / 8, p, smem, tiles, st);
 }

@@ -142,3 +142,54 @@ def test_c4_chain_full_batch(q4):
 
 def test_paper_table2_topology_with_random_weights(q4):
     run_chain(q4, wl.paper_table2_net(batch=3))
+
+
+FUSED = [  # N, H, W, C, OC, KH, KW, sh, sw, ph, pw, byte offset of X, shift
+    (3, 16, 16, 1, 8, 3, 3, 1, 1, 1, 1, 0, 5),      # pixel per lane, packed copy (rows are whole words)
+    (5, 9, 8, 2, 16, 3, 3, 2, 2, 1, 1, 0, 5),       # pixel per lane, packed copy, two channels
+    (2, 8, 24, 1, 8, 5, 5, 1, 1, 2, 2, 0, 1),       # ... 5x5, 64-bit rounding path (shift < 2)
+    (3, 33, 25, 1, 8, 5, 5, 1, 1, 0, 0, 0, 6),      # pixel per lane, expanded copy (odd row length)
+    (2, 7, 7, 3, 8, 2, 2, 1, 1, 0, 0, 0, 4),        # ... three channels, odd nibble offsets per row
+    (4, 16, 16, 1, 8, 3, 3, 1, 1, 1, 1, 1, 5),      # ... forced by a misaligned input pointer
+    (2, 11, 9, 3, 24, 3, 3, 1, 1, 1, 1, 0, 5),      # MMA, expanded copy, 24 outputs
+    (2, 10, 12, 5, 32, 3, 2, 2, 1, 1, 0, 0, 5),     # MMA, expanded copy, rectangular filter and strides
+    (3, 12, 12, 8, 16, 3, 3, 1, 1, 1, 1, 2, 5),     # MMA, expanded copy forced by a misaligned pointer
+    (2, 9, 10, 8, 40, 3, 3, 1, 1, 1, 1, 0, 5),      # MMA, packed copy in 4-byte pieces, 40 outputs
+    (2, 9, 12, 8, 56, 3, 3, 3, 3, 0, 2, 0, 0),      # MMA, packed copy in 16-byte pieces, stride 3, shift 0
+    (300, 3, 3, 8, 8, 3, 3, 1, 1, 1, 1, 0, 5),      # tiles spanning dozens of images, OW < 8
+    (90, 5, 6, 16, 48, 2, 3, 2, 1, 1, 1, 0, 5),     # OW < 8, rows of several images per thread
+    (700, 1, 1, 8, 8, 1, 1, 1, 1, 0, 0, 0, 5),      # one pixel per image
+    (2, 20, 40, 32, 64, 3, 3, 1, 1, 1, 1, 0, 7),    # widest tile the MMA kernel has
+    (1, 30, 300, 8, 8, 1, 7, 1, 2, 0, 3, 0, 5),     # long rows: a tile inside one output row
+]
+
+
+@pytest.mark.parametrize("g", FUSED)
+@pytest.mark.parametrize("given_sums", [False, True])
+def test_conv2d_fused_modes(q4, g, given_sums):
+    """Every staging mode and both kernels of the fused layer against the oracle."""
+    import torch
+    N, H, W, C, OC, KH, KW, sh, sw, ph, pw, xoff, shift = g
+    seed = 7000 + sum(g)
+    args = (N, H, W, C, OC, KH, KW, sh, sw, ph, pw)
+    dq, do = q4.ConvDesc(*args), oracle.ConvDesc(*args)
+    K = KH * KW * C
+    X = wl.rand_flat_nibbles(seed, 1, N * H * W * C)
+    Wt = wl.rand_packed(seed, 2, OC, K)
+    bias = wl.rand_ints(seed, 3, -300, 300, OC).astype(np.int32)
+    za, zb = (int(v) for v in wl.rand_ints(seed, 4, 0, 15, 2))
+    rq = ((1 << 30) + 987654321 % (1 << 30), shift, 3, 1, 14)
+    want = oracle.conv2d(X, Wt, bias, do, za, zb, oracle.Requant(*rq))
+    Xbuf = torch.zeros(xoff + (X.size + 31) // 16 * 16, dtype=torch.uint8, device="cuda")
+    Xd = Xbuf[xoff:xoff + X.size]
+    Xd.copy_(dev(X))
+    ws = torch.empty(q4.q4_conv2d_workspace_bytes(dq), dtype=torch.uint8, device="cuda")
+    Y = torch.full((dq.M, OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
+    colsum = None
+    if given_sums:
+        colsum = dev(oracle.unpack_rows(Wt, K).astype(np.int64).sum(axis=1).astype(np.int32))
+    n0 = q4.q4_launch_count()
+    q4.q4_conv2d(Xd, dev(Wt), dq, za, zb, q4.Requant(*rq), Y, ws, dev(bias), colsum)
+    assert q4.q4_launch_count() - n0 == 1            # the fused path: one kernel, no unrolled matrix
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    assert (Y.cpu().numpy() == want).all()
