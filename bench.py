@@ -176,6 +176,45 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------- GPU arm
 
+def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20):
+    """Device time of every layer of the c4 chain, each layer launched `reps` times back to
+    back behind a busy GPU so that launch latency is not what is measured."""
+    import torch
+    net = wl.c4(batch=batch, seed=4000, centred=True)
+    X = torch.from_numpy(net.X).cuda()
+    layers, total_ms, total_bytes = {}, 0.0, 0
+    for L in net.layers:
+        d = q4.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
+        ws = torch.empty(q4.q4_conv2d_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+        Y = torch.empty((d.M, L.OC // 2), dtype=torch.uint8, device="cuda")
+        Wt, b = torch.from_numpy(L.Wt).cuda(), torch.from_numpy(L.bias).cuda()
+        rq = q4.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi)
+        Xf = X.reshape(-1)
+        call = lambda: q4.q4_conv2d(Xf, Wt, d, L.za, L.zb, rq, Y, ws, b)
+        for _ in range(3):
+            call()
+        ts = []
+        for _ in range(5):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda._sleep(2_000_000)           # about 1 ms of GPU work for the launches to queue behind
+            e0.record()
+            for _ in range(reps):
+                call()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / reps)
+        ms = statistics.median(ts)
+        nbytes = X.numel() + Wt.numel() + 4 * b.numel() + Y.numel()
+        layers[L.name] = {"ms": ms, "compulsory_gbs": nbytes / (ms * 1e-3) / 1e9,
+                          "gops": 2.0 * d.M * d.K * L.OC / (ms * 1e-3) / 1e9}
+        total_ms += ms
+        total_bytes += nbytes
+        X = Y
+    return {"ms": total_ms, "compulsory_bytes": total_bytes,
+            "compulsory_gbs": total_bytes / (total_ms * 1e-3) / 1e9, "layers": layers,
+            "timing": f"median of 5 x {reps} back-to-back launches per layer"}
+
+
 def run_ours(args):
     import torch
     rank, world, local = dist_env()
@@ -302,6 +341,9 @@ def run_ours(args):
             torch.distributed.destroy_process_group()
         return 0
 
+    # ---- the c4 layer chain (batch 4096), outside the timed region: per-layer device times
+    c4_detail = time_c4_chain(q4, wl) if world == 1 else None
+
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
     cpu_baseline = None
     if world == 1 and not args.no_cpu_baseline:
@@ -344,6 +386,7 @@ def run_ours(args):
             "q4_conv2d_c3_compulsory_frac_of_hbm": conv_compulsory_bytes / (conv_ms * 1e-3) / 1e9 / peaks["hbm"],
             "q4_conv2d_c3_unroll_path_equivalent_gbs": conv_path_bytes / (conv_ms * 1e-3) / 1e9,
             "q4_conv2d_c3_gops": conv_ops / (conv_ms * 1e-3) / 1e9,
+            "c4_chain_batch4096": c4_detail,
             "hbm_peak_gbs": peaks["hbm"], "peaks": peaks["source"]},
     }
     print(json.dumps(line))

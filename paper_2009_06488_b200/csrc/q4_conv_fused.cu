@@ -3,7 +3,7 @@
 // memory.  A CTA takes 224 consecutive output pixels.  It first copies the input rows
 // those pixels touch into shared memory -- with the padding materialised as the input
 // zero point, so the gather below needs no bounds checks -- while the previous tile is
-// still being multiplied (two buffers).  Each warp then gathers its 32 pixels' taps from
+// still being multiplied (a ring of buffers).  Each warp then gathers its 32 pixels' taps from
 // that copy into the A fragments of the warp-level integer MMA (u8 x s8 -> s32,
 // m16n8k32), multiplies against the layer's weights held as B fragments in shared
 // memory, and applies the remaining zero-point term of Eq. 3, the bias, the
@@ -44,6 +44,8 @@ constexpr int WARPS = 7;                 // multiplying warps; one more warp pro
 constexpr int ROWS_PER_WARP = 32;
 constexpr int ROWS_PER_CTA = WARPS * ROWS_PER_WARP;
 constexpr int SMEM_LIMIT = 160 * 1024;
+constexpr int NBUF_MMA = 3;              // input buffers: the producer runs NBUF - 1 tiles ahead
+constexpr int NBUF_LANE = 4;
 
 // n / d for n < 2^31 as (umulhi(n, mul) + n) >> shift (round-up method: shift =
 // ceil(log2 d), mul = floor(2^32 * (2^shift - d) / d) + 1).
@@ -117,9 +119,15 @@ __device__ __forceinline__ void cp_async4(void* dst, const void* src)
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
                  :: "r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
 }
-__device__ __forceinline__ void cp_async_wait_all()
+__device__ __forceinline__ void cp_async_commit()
 {
-    asm volatile("cp.async.wait_all;" ::: "memory");
+    asm volatile("cp.async.commit_group;" ::: "memory");
+}
+// Waits until at most PENDING of this thread's most recent copy groups are still in flight.
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait_group()
+{
+    asm volatile("cp.async.wait_group %0;" :: "n"(PENDING) : "memory");
 }
 
 // Four nibbles in the low halves of four bytes, minus zb, as four signed bytes.  Setting
@@ -128,6 +136,20 @@ __device__ __forceinline__ void cp_async_wait_all()
 __device__ __forceinline__ uint32_t sub_zb(uint32_t x, uint32_t zb)
 {
     return ((x | 0x80808080u) - zb * 0x01010101u) ^ 0x80808080u;
+}
+
+__device__ __forceinline__ int dp4a_u8s8(uint32_t a, uint32_t b, int c)
+{
+    int d;
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+__device__ __forceinline__ int mulhi_add(int a, int b, int c)
+{
+    int d;
+    asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
 }
 
 __device__ __forceinline__ uint32_t weight_nibble(const Params& p, int n, int k)
@@ -270,8 +292,9 @@ conv_fused_kernel(const Params p)
     uint2* bfrag = reinterpret_cast<uint2*>(smem);                                   // [KS][NT][32]
     int32_t* tab = reinterpret_cast<int32_t*>(smem + (size_t)p.KS * NT * 32 * 8);    // [KS][TW]
     int32_t* colsum_s = tab + p.KS * TW;                                             // [N]
-    int4* geo_s = reinterpret_cast<int4*>(colsum_s + N);                             // [2]
-    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + 2);                           // 16-byte aligned
+    constexpr int NB = NBUF_MMA;
+    int4* geo_s = reinterpret_cast<int4*>(colsum_s + N);                             // [NB]
+    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB);                          // 16-byte aligned
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
@@ -279,12 +302,12 @@ conv_fused_kernel(const Params p)
     const int segbytes = p.KW * p.C;                   // expanded mode: bytes per kh segment
 
     // ---- once per CTA: weights -> signed B fragments, depth table, weight sums, and
-    //      both input buffers filled with the zero point (this is what stays in the halo)
+    //      the input buffers filled with the zero point (this is what stays in the halo)
     for (int i = tid; i < N; i += THREADS) colsum_s[i] = 0;
     {
         const uint32_t zfill = (uint32_t)p.za * (EXP ? 0x01010101u : 0x11111111u);
         uint32_t* b = reinterpret_cast<uint32_t*>(buf0);
-        for (int i = tid; i < 2 * p.bufbytes / 4; i += THREADS) b[i] = zfill;
+        for (int i = tid; i < NB * p.bufbytes / 4; i += THREADS) b[i] = zfill;
     }
     __syncthreads();
     for (int i = tid; i < p.KS * NT * 32; i += THREADS) {
@@ -352,14 +375,22 @@ conv_fused_kernel(const Params p)
 
     if (warp == WARPS) {
         // ---------------- producer ----------------
-        for (int k = -1; k < mytiles; ++k) {
-            if (k + 1 < mytiles) {
-                const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)(k + 1) * gridDim.x);
-                uint8_t* buf = buf0 + ((k + 1) & 1) * p.bufbytes;
+        // Tile j lives in buffer j % NB.  Before barrier k+1 the copy of tile k+1 must have
+        // landed; the copies of the NB - 2 tiles after it may still be in flight.  The
+        // buffer of tile k + NB - 1 is the one tile k - 1 was read from, free since barrier k.
+        auto produce = [&](int j) {
+            if (j < mytiles) {
+                const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
+                uint8_t* buf = buf0 + (j % NB) * p.bufbytes;
                 if (EXP) stage_expanded(p, gn, buf, lane); else stage_packed(p, gn, buf, lane);
-                if (lane == 0) geo_s[(k + 1) & 1] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
-                cp_async_wait_all();
+                if (lane == 0) geo_s[j % NB] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
             }
+            cp_async_commit();                         // one group per tile, empty past the end
+        };
+        for (int j = 0; j < NB - 1; ++j) produce(j);
+        for (int k = -1; k < mytiles; ++k) {
+            if (k >= 0) produce(k + NB - 1);
+            cp_async_wait_group<NB - 2>();
             tile_barrier();
         }
         return;
@@ -381,20 +412,23 @@ conv_fused_kernel(const Params p)
     const int pix0 = p.pix0;
     const int yoff = (warp * ROWS_PER_WARP + g) * (N / 2) + NT * t;    // my first row within a tile
 
+    // pixel indices fit 32 bits (M < 2^31, and a tile starts below M)
+    const uint32_t M32 = (uint32_t)p.M, mstep = gridDim.x * (uint32_t)ROWS_PER_CTA;
+    uint32_t mbase = blockIdx.x * (uint32_t)ROWS_PER_CTA;
+    int kb = 0;                                        // k % NB
     tile_barrier();
-    for (int k = 0; k < mytiles; ++k) {
-        const int64_t tile = blockIdx.x + (int64_t)k * gridDim.x;
-        const uint8_t* buf = buf0 + (k & 1) * p.bufbytes;
-        const int4 gv = geo_s[k & 1];                  // n_first, oh_first, s0
-        const int64_t mbase = tile * ROWS_PER_CTA;
-        const int64_t left = p.M - mbase;              // > 0
-        const int myrows = (int)(left < ROWS_PER_CTA ? left : ROWS_PER_CTA) - warp * ROWS_PER_WARP;
+    for (int k = 0; k < mytiles; ++k, mbase += mstep, kb = kb + 1 == NB ? 0 : kb + 1) {
+        const uint8_t* buf = buf0 + kb * p.bufbytes;
+        const int4 gv = geo_s[kb];                     // n_first, oh_first, s0
+        const uint32_t left = M32 - mbase;             // > 0
+        const int myrows = (int)(left < (uint32_t)ROWS_PER_CTA ? left : (uint32_t)ROWS_PER_CTA) -
+                           warp * ROWS_PER_WARP;
         if (myrows > 0) {                              // warp-uniform
             // my four rows: g, g+8 (first 16-row tile), 16+g, 24+g (second)
             int base[4], shf[4];
             {
-                const uint32_t mm = (uint32_t)mbase + (uint32_t)(warp * ROWS_PER_WARP) +
-                                    (uint32_t)(g < myrows ? g : 0);                  // M < 2^31
+                const uint32_t mm = mbase + (uint32_t)(warp * ROWS_PER_WARP) +
+                                    (uint32_t)(g < myrows ? g : 0);
                 const uint32_t q = fdiv(mm, p.div_ow);
                 int ow = (int)(mm - q * (uint32_t)p.OW);
                 const uint32_t n0 = fdiv(q, p.div_oh);
@@ -441,7 +475,7 @@ conv_fused_kernel(const Params p)
 #pragma unroll
                 for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0;
+                    for (int e = 0; e < 4; ++e) acc[mt][nt][e] = colterm[nt][e & 1];   // columns 2t + e % 2
 
             for (int j = 0; j < p.KS; ++j) {
                 uint32_t a[2][4];
@@ -481,7 +515,7 @@ conv_fused_kernel(const Params p)
 
             // epilogue: accumulator (mt, nt) holds rows g + 16 mt (c0, c1) and g + 8 + 16 mt
             // (c2, c3), fragment columns 2t, 2t+1
-            uint8_t* ytile = p.Y + mbase * (N / 2) + yoff;
+            uint8_t* ytile = p.Y + (uint64_t)mbase * (N / 2) + yoff;
             auto epilogue = [&](auto fast_tag) {
                 constexpr bool FAST = decltype(fast_tag)::value;
                 const int s = p.rq.shift - 1, rnd = FAST ? 1 << (s - 1) : 0;
@@ -495,9 +529,9 @@ conv_fused_kernel(const Params p)
                         uint32_t qv[2];
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
-                            const int v = (int)((uint32_t)acc[mt][nt][2 * hrow + e] + (uint32_t)colterm[nt][e]);
+                            const int v = acc[mt][nt][2 * hrow + e];       // started from the column's constant
                             if (FAST) {
-                                int q = ((__mulhi(v, p.rq.mult) + rnd) >> s) + p.rq.zo;
+                                int q = (mulhi_add(v, p.rq.mult, rnd) >> s) + p.rq.zo;
                                 q = max(q, p.rq.lo);
                                 qv[e] = (uint32_t)min(q, p.rq.hi);
                             } else {
@@ -542,20 +576,6 @@ conv_fused_kernel(const Params p)
 // that every lane reads from the same shared-memory address.  The packed output of a
 // pixel is one 4- or 8-byte store, a warp's is contiguous.
 // ---------------------------------------------------------------------------------
-__device__ __forceinline__ int dp4a_u8s8(uint32_t a, uint32_t b, int c)
-{
-    int d;
-    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-
-__device__ __forceinline__ int mulhi_add(int a, int b, int c)
-{
-    int d;
-    asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-
 template <int OC, bool NIB>
 __global__ void __launch_bounds__(THREADS, 3)
 conv_lane_kernel(const Params p)
@@ -564,8 +584,9 @@ conv_lane_kernel(const Params p)
     const int nw = p.KH * p.segw;                      // 32-bit depth words per pixel
     uint32_t* wsm = reinterpret_cast<uint32_t*>(smem);                               // [nw][OC]
     int32_t* colterm_s = reinterpret_cast<int32_t*>(wsm + nw * OC);                  // [OC]
-    int4* geo_s = reinterpret_cast<int4*>(colterm_s + OC);                           // [2]
-    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + 2);                           // 16-byte aligned
+    constexpr int NB = NBUF_LANE;
+    int4* geo_s = reinterpret_cast<int4*>(colterm_s + OC);                           // [NB]
+    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB);                          // 16-byte aligned
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int segbytes = p.KW * p.C;
@@ -575,7 +596,7 @@ conv_lane_kernel(const Params p)
     {
         uint32_t* b = reinterpret_cast<uint32_t*>(buf0);
         const uint32_t zfill = (uint32_t)p.za * (NIB ? 0x11111111u : 0x01010101u);
-        for (int i = tid; i < 2 * p.bufbytes / 4; i += THREADS) b[i] = zfill;
+        for (int i = tid; i < NB * p.bufbytes / 4; i += THREADS) b[i] = zfill;
     }
     __syncthreads();
     for (int i = tid; i < nw * OC; i += THREADS) {
@@ -607,14 +628,19 @@ conv_lane_kernel(const Params p)
 
     if (warp == WARPS) {
         // ---------------- producer (same protocol as conv_fused_kernel) ----------------
-        for (int k = -1; k < mytiles; ++k) {
-            if (k + 1 < mytiles) {
-                const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)(k + 1) * gridDim.x);
-                uint8_t* buf = buf0 + ((k + 1) & 1) * p.bufbytes;
+        auto produce = [&](int j) {
+            if (j < mytiles) {
+                const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
+                uint8_t* buf = buf0 + (j % NB) * p.bufbytes;
                 if (NIB) stage_packed(p, gn, buf, lane); else stage_expanded(p, gn, buf, lane);
-                if (lane == 0) geo_s[(k + 1) & 1] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
-                if (NIB) cp_async_wait_all();
+                if (lane == 0) geo_s[j % NB] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
             }
+            cp_async_commit();
+        };
+        for (int j = 0; j < NB - 1; ++j) produce(j);
+        for (int k = -1; k < mytiles; ++k) {
+            if (k >= 0) produce(k + NB - 1);
+            cp_async_wait_group<NB - 2>();
             tile_barrier();
         }
         return;
@@ -623,17 +649,19 @@ conv_lane_kernel(const Params p)
     // ---------------- consumers ----------------
     const int pix0 = p.pix0;
     const int r = warp * ROWS_PER_WARP + lane;         // my pixel within a tile
+    // pixel indices fit 32 bits (M < 2^31, and a tile starts below M)
+    const uint32_t M32 = (uint32_t)p.M, mstep = gridDim.x * (uint32_t)ROWS_PER_CTA;
+    uint32_t mbase = blockIdx.x * (uint32_t)ROWS_PER_CTA;
+    int kb = 0;                                        // k % NB
     tile_barrier();
-    for (int k = 0; k < mytiles; ++k) {
-        const int64_t tile = blockIdx.x + (int64_t)k * gridDim.x;
-        const uint8_t* buf = buf0 + (k & 1) * p.bufbytes;
-        const int4 gv = geo_s[k & 1];                  // n_first, oh_first, s0
-        const int64_t mbase = tile * ROWS_PER_CTA;
-        const int64_t left = p.M - mbase;              // > 0
-        const int rows = (int)(left < ROWS_PER_CTA ? left : ROWS_PER_CTA);
+    for (int k = 0; k < mytiles; ++k, mbase += mstep, kb = kb + 1 == NB ? 0 : kb + 1) {
+        const uint8_t* buf = buf0 + kb * p.bufbytes;
+        const int4 gv = geo_s[kb];                     // n_first, oh_first, s0
+        const uint32_t left = M32 - mbase;             // > 0
+        const int rows = (int)(left < (uint32_t)ROWS_PER_CTA ? left : (uint32_t)ROWS_PER_CTA);
         if (warp * ROWS_PER_WARP < rows) {             // warp-uniform
             const bool valid = r < rows;
-            const uint32_t mm = (uint32_t)mbase + (uint32_t)(valid ? r : 0);       // M < 2^31
+            const uint32_t mm = mbase + (uint32_t)(valid ? r : 0);
             const uint32_t q = fdiv(mm, p.div_ow);
             const int ow = (int)(mm - q * (uint32_t)p.OW);
             const uint32_t n0 = fdiv(q, p.div_oh);
@@ -696,7 +724,7 @@ conv_lane_kernel(const Params p)
                 }
             }
             if (valid) {
-                uint8_t* dst = p.Y + (mbase + r) * (OC / 2);
+                uint8_t* dst = p.Y + (uint64_t)(mbase + (uint32_t)r) * (OC / 2);
                 if (OC == 8) *reinterpret_cast<uint32_t*>(dst) = out[0];
                 else *reinterpret_cast<uint2*>(dst) = make_uint2(out[0], out[(OC / 8 - 1)]);
             }
@@ -748,8 +776,10 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     const int64_t bufbytes = slots * pitch + 16;       // the slack takes the unaligned words' over-read
     const int64_t KS = expanded ? ((int64_t)d.KH * segw + 7) / 8 : ((int64_t)p.K + 31) / 32;
     const int64_t smem = per_lane
-        ? (int64_t)d.KH * segw * d.OC * 4 + (int64_t)d.OC * 4 + 32 + 2 * bufbytes
-        : KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 4 + 32 + 2 * bufbytes;
+        ? (int64_t)d.KH * segw * d.OC * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_LANE +
+              fused::NBUF_LANE * bufbytes
+        : KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_MMA +
+              fused::NBUF_MMA * bufbytes;
     if (smem > fused::SMEM_LIMIT) return 0;
     p.unit = (int32_t)unit; p.rowbytes = (int32_t)rowbytes; p.data0 = (int32_t)data0; p.pix0 = (int32_t)pix0;
     p.pitch = (int32_t)pitch; p.bufbytes = (int32_t)bufbytes; p.segw = (int32_t)segw;
