@@ -36,8 +36,12 @@
 #include <type_traits>
 
 #include "q4_common.cuh"
+#include "q4_tc_ptx.cuh"
 
 namespace q4 {
+
+unsigned* device_status_ptr();     // the device status word (q4_api.cu)
+
 namespace fused {
 
 constexpr int WARPS = 7;                 // multiplying warps; one more warp produces
@@ -46,6 +50,7 @@ constexpr int ROWS_PER_CTA = WARPS * ROWS_PER_WARP;
 constexpr int SMEM_LIMIT = 160 * 1024;
 constexpr int NBUF_MMA = 3;              // input buffers: the producer runs NBUF - 1 tiles ahead
 constexpr int NBUF_LANE = 4;
+constexpr int SYNC_BYTES = 64;             // the buffers' mbarriers and the abort flag
 
 // n / d for n < 2^31 as (umulhi(n, mul) + n) >> shift (round-up method: shift =
 // ceil(log2 d), mul = floor(2^32 * (2^shift - d) / d) + 1).
@@ -90,7 +95,9 @@ struct Params {
     int32_t bufbytes;          // one input buffer
     int32_t segw;              // expanded: 32-bit words per kh segment
     int32_t sfull;             // staged rows of an image all of whose output rows are in the tile
-    int32_t vec16;             // packed: image rows can be copied in 16-byte pieces
+    int32_t vec16;             // packed: image rows are whole 16-byte pieces, 16-byte aligned: each
+                               // is copied by one bulk copy that reports to the buffer's mbarrier
+    unsigned* status;          // device status word (a wait that ran out is recorded there)
     int32_t wt_words;          // weights can be read as aligned 32-bit words
     int32_t cpr;               // packed: copy pieces (16 or 4 bytes) per image row
     int32_t step8;             // staged-buffer offset of the pixel eight further in the same output row
@@ -109,11 +116,6 @@ __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, 
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ void cp_async16(void* dst, const void* src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
-                 :: "r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
-}
 __device__ __forceinline__ void cp_async4(void* dst, const void* src)
 {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;"
@@ -189,36 +191,69 @@ __device__ __forceinline__ Geo tile_geometry(const Params& p, int64_t tile)
     return g;
 }
 
-// Producer warp, packed mode: copies the image rows of a tile into `buf` with
-// asynchronous copies, one 16-byte (or 4-byte) piece per lane and step.  Only the
-// image columns are written: the lead and the halo columns hold the zero point from
-// the kernel's start.  Rows above or below the image are filled with the zero point.
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+
+// Which image row staged row `s` of a tile holds: returns the row index n * H + ih, or
+// -1 for a row above or below the image.
+__device__ __forceinline__ int64_t staged_row(const Params& p, const Geo& g, int s)
+{
+    int seg = 0, ih = g.oh_first * p.sh - p.ph + s;
+    if (s >= g.s0) {
+        const uint32_t r = (uint32_t)(s - g.s0);
+        const uint32_t sq = fdiv(r, p.div_sfull);
+        seg = 1 + (int)sq;
+        ih = (int)(r - sq * (uint32_t)p.sfull) - p.ph;
+    }
+    if ((unsigned)ih >= (unsigned)p.H) return -1;
+    return (int64_t)(g.n_first + seg) * p.H + ih;
+}
+
+// Producer warp, packed mode, rows of whole 16-byte pieces: one bulk copy per staged
+// row, a lane per row; the copies report their bytes to `bar`, which lane 0 has armed
+// with the tile's total.  Only the image columns are written: the halo columns hold the
+// zero point from the kernel's start.  Rows above or below the image are filled with
+// the zero point by ordinary stores.
+__device__ __forceinline__ void stage_packed_bulk(const Params& p, const Geo& g, uint8_t* buf, uint32_t bar,
+                                                  int lane)
+{
+    // ordinary stores to this buffer (the initial fill, earlier border rows) come before
+    // the copy engine's writes
+    fence_async_smem();
+    int inside = 0;
+    for (int s = lane; s < g.nslots; s += 32) inside += staged_row(p, g, s) >= 0;
+    inside = __reduce_add_sync(0xFFFFFFFFu, inside);
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)inside * (uint32_t)p.rowbytes);
+    __syncwarp();
+    const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
+    for (int s = lane; s < g.nslots; s += 32) {
+        const int64_t row = staged_row(p, g, s);
+        uint8_t* dst = buf + s * p.pitch + p.data0;
+        if (row >= 0) {
+            bulk_load_row(smem_u32(dst), p.X + row * p.rowbytes, (uint32_t)p.rowbytes, bar);
+        } else {
+            for (int c = 0; c < p.rowbytes; c += 16)
+                *reinterpret_cast<uint4*>(dst + c) = make_uint4(zfill, zfill, zfill, zfill);
+        }
+    }
+}
+
+// Producer warp, packed mode, any 4-byte-aligned rows: asynchronous 4-byte copies, one
+// piece per lane and step.
 __device__ __forceinline__ void stage_packed(const Params& p, const Geo& g, uint8_t* buf, int lane)
 {
-    const int data0 = p.data0;
-    const int cb = p.vec16 ? 16 : 4;
     const int total = g.nslots * p.cpr;
-    const int ih_first = g.oh_first * p.sh - p.ph;
     const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
     for (int idx = lane; idx < total; idx += 32) {
         const int s = (int)fdiv((uint32_t)idx, p.div_cpr);
-        const int c = (idx - s * p.cpr) * cb;
-        int seg = 0, ih = ih_first + s;
-        if (s >= g.s0) {
-            const uint32_t r = (uint32_t)(s - g.s0);
-            const uint32_t sq = fdiv(r, p.div_sfull);
-            seg = 1 + (int)sq;
-            ih = (int)(r - sq * (uint32_t)p.sfull) - p.ph;
-        }
-        uint8_t* dst = buf + s * p.pitch + data0 + c;
-        if ((unsigned)ih < (unsigned)p.H) {
-            const uint8_t* src = p.X + ((int64_t)(g.n_first + seg) * p.H + ih) * p.rowbytes + c;
-            if (p.vec16) cp_async16(dst, src); else cp_async4(dst, src);
-        } else if (p.vec16) {
-            *reinterpret_cast<uint4*>(dst) = make_uint4(zfill, zfill, zfill, zfill);
-        } else {
-            *reinterpret_cast<uint32_t*>(dst) = zfill;
-        }
+        const int c = (idx - s * p.cpr) * 4;
+        const int64_t row = staged_row(p, g, s);
+        uint8_t* dst = buf + s * p.pitch + p.data0 + c;
+        if (row >= 0) cp_async4(dst, p.X + row * p.rowbytes + c);
+        else *reinterpret_cast<uint32_t*>(dst) = zfill;
     }
 }
 
@@ -294,7 +329,9 @@ conv_fused_kernel(const Params p)
     int32_t* colsum_s = tab + p.KS * TW;                                             // [N]
     constexpr int NB = NBUF_MMA;
     int4* geo_s = reinterpret_cast<int4*>(colsum_s + N);                             // [NB]
-    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB);                          // 16-byte aligned
+    uint64_t* full_s = reinterpret_cast<uint64_t*>(geo_s + NB);                      // [NB] "tile landed"
+    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB) + SYNC_BYTES;             // 16-byte aligned
+    const uint32_t full0 = smem_u32(full_s), abort_flag = full0 + 8 * NB;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
@@ -308,6 +345,12 @@ conv_fused_kernel(const Params p)
         const uint32_t zfill = (uint32_t)p.za * (EXP ? 0x01010101u : 0x11111111u);
         uint32_t* b = reinterpret_cast<uint32_t*>(buf0);
         for (int i = tid; i < NB * p.bufbytes / 4; i += THREADS) b[i] = zfill;
+        fence_async_smem();                            // before the copy engine writes the same bytes
+    }
+    if (tid == 0) {
+        for (int i = 0; i < NB; ++i) mbar_init(full0 + 8 * i, 1);
+        sts32(abort_flag, 0);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     for (int i = tid; i < p.KS * NT * 32; i += THREADS) {
@@ -378,11 +421,16 @@ conv_fused_kernel(const Params p)
         // Tile j lives in buffer j % NB.  Before barrier k+1 the copy of tile k+1 must have
         // landed; the copies of the NB - 2 tiles after it may still be in flight.  The
         // buffer of tile k + NB - 1 is the one tile k - 1 was read from, free since barrier k.
+        // Either way the consumers also wait on the buffer's mbarrier: bulk copies report
+        // to it themselves; otherwise lane 0 arrives once this warp's copies have landed.
+        const bool bulk = !EXP && p.vec16;
         auto produce = [&](int j) {
             if (j < mytiles) {
                 const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
                 uint8_t* buf = buf0 + (j % NB) * p.bufbytes;
-                if (EXP) stage_expanded(p, gn, buf, lane); else stage_packed(p, gn, buf, lane);
+                if (EXP) stage_expanded(p, gn, buf, lane);
+                else if (bulk) stage_packed_bulk(p, gn, buf, full0 + 8 * (j % NB), lane);
+                else stage_packed(p, gn, buf, lane);
                 if (lane == 0) geo_s[j % NB] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
             }
             cp_async_commit();                         // one group per tile, empty past the end
@@ -390,7 +438,11 @@ conv_fused_kernel(const Params p)
         for (int j = 0; j < NB - 1; ++j) produce(j);
         for (int k = -1; k < mytiles; ++k) {
             if (k >= 0) produce(k + NB - 1);
-            cp_async_wait_group<NB - 2>();
+            if (!bulk) {
+                cp_async_wait_group<NB - 2>();
+                __syncwarp();
+                if (lane == 0 && k + 1 < mytiles) mbar_arrive(full0 + 8 * ((k + 1) % NB));
+            }
             tile_barrier();
         }
         return;
@@ -416,10 +468,13 @@ conv_fused_kernel(const Params p)
     const uint32_t M32 = (uint32_t)p.M, mstep = gridDim.x * (uint32_t)ROWS_PER_CTA;
     uint32_t mbase = blockIdx.x * (uint32_t)ROWS_PER_CTA;
     int kb = 0;                                        // k % NB
+    uint32_t phase = 0;                                // (k / NB) % 2
     tile_barrier();
-    for (int k = 0; k < mytiles; ++k, mbase += mstep, kb = kb + 1 == NB ? 0 : kb + 1) {
+    for (int k = 0; k < mytiles; ++k, mbase += mstep) {
         const uint8_t* buf = buf0 + kb * p.bufbytes;
         const int4 gv = geo_s[kb];                     // n_first, oh_first, s0
+        mbar_wait(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
+        if (++kb == NB) { kb = 0; phase ^= 1; }
         const uint32_t left = M32 - mbase;             // > 0
         const int myrows = (int)(left < (uint32_t)ROWS_PER_CTA ? left : (uint32_t)ROWS_PER_CTA) -
                            warp * ROWS_PER_WARP;
@@ -576,17 +631,22 @@ conv_fused_kernel(const Params p)
 // that every lane reads from the same shared-memory address.  The packed output of a
 // pixel is one 4- or 8-byte store, a warp's is contiguous.
 // ---------------------------------------------------------------------------------
-template <int OC, bool NIB>
+// KH_T, SEGW_T: the filter height and the words per kh segment when known at compile time
+// (the loops over the depth unroll), 0 = taken from the parameters.
+template <int OC, bool NIB, int KH_T, int SEGW_T>
 __global__ void __launch_bounds__(THREADS, 3)
 conv_lane_kernel(const Params p)
 {
+    const int KH = KH_T ? KH_T : p.KH, SEGW = SEGW_T ? SEGW_T : p.segw;
     extern __shared__ __align__(16) uint8_t smem[];
     const int nw = p.KH * p.segw;                      // 32-bit depth words per pixel
     uint32_t* wsm = reinterpret_cast<uint32_t*>(smem);                               // [nw][OC]
     int32_t* colterm_s = reinterpret_cast<int32_t*>(wsm + nw * OC);                  // [OC]
     constexpr int NB = NBUF_LANE;
     int4* geo_s = reinterpret_cast<int4*>(colterm_s + OC);                           // [NB]
-    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB);                          // 16-byte aligned
+    uint64_t* full_s = reinterpret_cast<uint64_t*>(geo_s + NB);                      // [NB] "tile landed"
+    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB) + SYNC_BYTES;             // 16-byte aligned
+    const uint32_t full0 = smem_u32(full_s), abort_flag = full0 + 8 * NB;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int segbytes = p.KW * p.C;
@@ -597,6 +657,12 @@ conv_lane_kernel(const Params p)
         uint32_t* b = reinterpret_cast<uint32_t*>(buf0);
         const uint32_t zfill = (uint32_t)p.za * (NIB ? 0x11111111u : 0x01010101u);
         for (int i = tid; i < NB * p.bufbytes / 4; i += THREADS) b[i] = zfill;
+        fence_async_smem();                            // before the copy engine writes the same bytes
+    }
+    if (tid == 0) {
+        for (int i = 0; i < NB; ++i) mbar_init(full0 + 8 * i, 1);
+        sts32(abort_flag, 0);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
     for (int i = tid; i < nw * OC; i += THREADS) {
@@ -628,11 +694,14 @@ conv_lane_kernel(const Params p)
 
     if (warp == WARPS) {
         // ---------------- producer (same protocol as conv_fused_kernel) ----------------
+        const bool bulk = NIB && p.vec16;
         auto produce = [&](int j) {
             if (j < mytiles) {
                 const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
                 uint8_t* buf = buf0 + (j % NB) * p.bufbytes;
-                if (NIB) stage_packed(p, gn, buf, lane); else stage_expanded(p, gn, buf, lane);
+                if (!NIB) stage_expanded(p, gn, buf, lane);
+                else if (bulk) stage_packed_bulk(p, gn, buf, full0 + 8 * (j % NB), lane);
+                else stage_packed(p, gn, buf, lane);
                 if (lane == 0) geo_s[j % NB] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
             }
             cp_async_commit();
@@ -640,7 +709,11 @@ conv_lane_kernel(const Params p)
         for (int j = 0; j < NB - 1; ++j) produce(j);
         for (int k = -1; k < mytiles; ++k) {
             if (k >= 0) produce(k + NB - 1);
-            cp_async_wait_group<NB - 2>();
+            if (!bulk) {
+                cp_async_wait_group<NB - 2>();
+                __syncwarp();
+                if (lane == 0 && k + 1 < mytiles) mbar_arrive(full0 + 8 * ((k + 1) % NB));
+            }
             tile_barrier();
         }
         return;
@@ -653,10 +726,13 @@ conv_lane_kernel(const Params p)
     const uint32_t M32 = (uint32_t)p.M, mstep = gridDim.x * (uint32_t)ROWS_PER_CTA;
     uint32_t mbase = blockIdx.x * (uint32_t)ROWS_PER_CTA;
     int kb = 0;                                        // k % NB
+    uint32_t phase = 0;                                // (k / NB) % 2
     tile_barrier();
-    for (int k = 0; k < mytiles; ++k, mbase += mstep, kb = kb + 1 == NB ? 0 : kb + 1) {
+    for (int k = 0; k < mytiles; ++k, mbase += mstep) {
         const uint8_t* buf = buf0 + kb * p.bufbytes;
         const int4 gv = geo_s[kb];                     // n_first, oh_first, s0
+        mbar_wait(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
+        if (++kb == NB) { kb = 0; phase ^= 1; }
         const uint32_t left = M32 - mbase;             // > 0
         const int rows = (int)(left < (uint32_t)ROWS_PER_CTA ? left : (uint32_t)ROWS_PER_CTA);
         if (warp * ROWS_PER_WARP < rows) {             // warp-uniform
@@ -681,9 +757,11 @@ conv_lane_kernel(const Params p)
                 acc[n] = c.x; acc[n + 1] = c.y; acc[n + 2] = c.z; acc[n + 3] = c.w;
             }
             const uint32_t* wrow = wsm;
-            for (int kh = 0; kh < p.KH; ++kh) {
+#pragma unroll
+            for (int kh = 0; kh < KH; ++kh) {
                 const uint32_t* arow = reinterpret_cast<const uint32_t*>(src + kh * p.pitch);
-                for (int ws = 0; ws < p.segw; ++ws) {
+#pragma unroll
+                for (int ws = 0; ws < SEGW; ++ws) {
                     uint32_t a;
                     if (NIB) {
                         // four nibbles -> four bytes
@@ -776,9 +854,9 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     const int64_t bufbytes = slots * pitch + 16;       // the slack takes the unaligned words' over-read
     const int64_t KS = expanded ? ((int64_t)d.KH * segw + 7) / 8 : ((int64_t)p.K + 31) / 32;
     const int64_t smem = per_lane
-        ? (int64_t)d.KH * segw * d.OC * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_LANE +
+        ? (int64_t)d.KH * segw * d.OC * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_LANE + fused::SYNC_BYTES +
               fused::NBUF_LANE * bufbytes
-        : KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_MMA +
+        : KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_MMA + fused::SYNC_BYTES +
               fused::NBUF_MMA * bufbytes;
     if (smem > fused::SMEM_LIMIT) return 0;
     p.unit = (int32_t)unit; p.rowbytes = (int32_t)rowbytes; p.data0 = (int32_t)data0; p.pix0 = (int32_t)pix0;
@@ -790,7 +868,7 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     p.div_ow = fused::make_fastdiv((uint32_t)p.OW);
     p.div_oh = fused::make_fastdiv((uint32_t)p.OH);
     p.div_sfull = fused::make_fastdiv((uint32_t)p.sfull);
-    p.cpr = (int32_t)(rowbytes / (p.vec16 ? 16 : 4));
+    p.cpr = (int32_t)(rowbytes / 4);
     if (p.cpr < 1) p.cpr = 1;                          // expanded mode does not use it
     p.div_cpr = fused::make_fastdiv((uint32_t)p.cpr);
     p.step8 = (int32_t)(8 * d.stride_w * unit);
@@ -866,14 +944,19 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     if (smem == 0) return cudaErrorInvalidValue;
     p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;
     p.za = za; p.zb = zb; p.rq = rq;
+    p.status = device_status_ptr();
+    if (!p.status) return cudaErrorUnknown;
     if (p.M == 0) return cudaSuccess;
     const int64_t tiles = (p.M + fused::ROWS_PER_CTA - 1) / fused::ROWS_PER_CTA;
     if (per_lane) {
+        // the 3x3 single-channel first layer gets its own fully unrolled instance
+        if (nibbles && d.OC == 8 && d.KH == 3 && p.segw == 1)
+            return launch_kernel(fused::conv_lane_kernel<8, true, 3, 1>, p, smem, tiles, st);
         if (nibbles)
-            return d.OC == 8 ? launch_kernel(fused::conv_lane_kernel<8, true>, p, smem, tiles, st)
-                             : launch_kernel(fused::conv_lane_kernel<16, true>, p, smem, tiles, st);
-        return d.OC == 8 ? launch_kernel(fused::conv_lane_kernel<8, false>, p, smem, tiles, st)
-                         : launch_kernel(fused::conv_lane_kernel<16, false>, p, smem, tiles, st);
+            return d.OC == 8 ? launch_kernel(fused::conv_lane_kernel<8, true, 0, 0>, p, smem, tiles, st)
+                             : launch_kernel(fused::conv_lane_kernel<16, true, 0, 0>, p, smem, tiles, st);
+        return d.OC == 8 ? launch_kernel(fused::conv_lane_kernel<8, false, 0, 0>, p, smem, tiles, st)
+                         : launch_kernel(fused::conv_lane_kernel<16, false, 0, 0>, p, smem, tiles, st);
     }
     return expanded ? launch_mode<true>(d.OC / 8, p, smem, tiles, st)
                     : launch_mode<false>(d.OC / 8, p, smem, tiles, st);
