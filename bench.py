@@ -115,6 +115,22 @@ def dist_env():
     return rank, world, local
 
 
+def max_over_ranks(value: float, world: int, device="cuda") -> float:
+    """The slowest rank's figure (the path has no exchange step: every rank runs an
+    independent replica of the same work, so the job takes as long as its slowest rank)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world: int, ops_per_rank_step: float, ms_per_step: float) -> float:
+    """Whole-job TOPS: every rank does `ops_per_rank_step` per step (weak scaling)."""
+    return world * ops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
 # --------------------------------------------------------------------------- CPU baseline
 
 def time_oracle_sample(case, target_s: float = 12.0):
@@ -152,6 +168,8 @@ def run_reference(args):
     # size one step for a few seconds so that steps + warmup end within minutes
     budget = 120.0 / max(1, args.steps + args.warmup)
     per_step = max(0.5, min(10.0, budget))
+    if args.ref_seconds is not None:
+        per_step = args.ref_seconds
     tops0, dt0, rows, threads = time_oracle_sample(case, per_step)
     sub = np.ascontiguousarray(case.A[:rows])
     for _ in range(max(0, args.warmup - 1)):
@@ -296,13 +314,9 @@ def run_ours(args):
     clocks = sampler.stop() if rank == 0 else None
     assert q4.q4_last_device_status() == q4.Q4_OK, "a device-side wait timed out"
 
-    total_ms = t_begin.elapsed_time(t_end)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(t_begin.elapsed_time(t_end), world)
     ms_per_step = total_ms / args.steps
-    value = world * step_ops / (ms_per_step * 1e-3) / 1e12
+    value = job_throughput(world, step_ops, ms_per_step)
 
     gemm_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in marks)
     gemm_rq_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in marks)
@@ -329,10 +343,7 @@ def run_ours(args):
         e2e_step()
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3 / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], dtype=torch.float64, device="cuda")
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world)
     h2d = 2 * (hA.numel() + hBt.numel()) + hX.numel() + hW.numel()
     d2h = hC.numel() * 4 + hCq.numel() + hY.numel()
 
@@ -364,7 +375,7 @@ def run_ours(args):
                    "parallelism": f"{world} independent replicas" if world > 1 else "1 GPU"},
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "e2e": {"value": world * step_ops / (e2e_ms * 1e-3) / 1e12, "unit": "TOPS",
+        "e2e": {"value": job_throughput(world, step_ops, e2e_ms), "unit": "TOPS",
                 "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h),
                 "ms_per_step": e2e_ms},
         "roofline": {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
@@ -463,6 +474,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ref-seconds", type=float, default=None,
+                    help="--impl reference: CPU seconds of oracle work per step (default: sized from --steps)")
     ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "conv", "im2col"],
                     help="profile one call in a loop instead of the benchmark step")
     ap.add_argument("--presums", action="store_true", help="--case gemm: pass precomputed depth sums")
