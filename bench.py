@@ -353,7 +353,7 @@ def run_ours(args):
         return 0
 
     # ---- the c4 layer chain (batch 4096), outside the timed region: per-layer device times
-    c4_detail = time_c4_chain(q4, wl) if world == 1 else None
+    c4_detail = time_c4_chain(q4, wl) if world == 1 and not args.no_c4_chain else None
 
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
     cpu_baseline = None
@@ -432,18 +432,24 @@ def run_case(args):
             call = lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, g.za, g.zb, rq, ws=wsg)
         units, unit = 2.0 * n ** 3 / 1e12, "TOPS"
     else:
-        net = wl.c3(batch=n)
-        L = net.layers[0]
+        if args.case == "c4layer":
+            # layer `--layer` of the c4 chain on random input of its shape
+            L = wl.c4(batch=n, seed=4000, centred=True).layers[args.layer]
+            net_X = wl.rand_flat_nibbles(77, 1, L.N * L.H * L.W * L.C)
+        else:
+            net = wl.c3(batch=n)
+            L, net_X = net.layers[0], net.X
         dq = q4.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
-        X, Wt = dev(net.X), dev(L.Wt)
+        X, Wt = dev(net_X), dev(L.Wt)
+        bias = None if L.bias is None else dev(L.bias)
         ws = torch.empty(q4.q4_conv2d_workspace_bytes(dq), dtype=torch.uint8, device="cuda")
         Y = torch.empty((dq.M, L.OC // 2), dtype=torch.uint8, device="cuda")
         lda = (dq.K // 2 + 15) // 16 * 16
         Amat = torch.empty((dq.M, lda), dtype=torch.uint8, device="cuda")
         ra = torch.empty(dq.M, dtype=torch.int32, device="cuda")
         rq = q4.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi)
-        if args.case == "conv":
-            call = lambda: q4.q4_conv2d(X, Wt, dq, L.za, L.zb, rq, Y, ws)
+        if args.case in ("conv", "c4layer"):
+            call = lambda: q4.q4_conv2d(X, Wt, dq, L.za, L.zb, rq, Y, ws, bias)
             units = (X.numel() + Wt.numel() + Y.numel()) / 1e9
         else:
             call = lambda: q4.q4_im2col(X, dq, L.za, Amat, ra)
@@ -474,10 +480,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-c4-chain", action="store_true",
+                    help="skip the per-layer timing of the c4 chain that follows the timed steps")
     ap.add_argument("--ref-seconds", type=float, default=None,
                     help="--impl reference: CPU seconds of oracle work per step (default: sized from --steps)")
-    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "conv", "im2col"],
+    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "conv", "im2col", "c4layer"],
                     help="profile one call in a loop instead of the benchmark step")
+    ap.add_argument("--layer", type=int, default=0, help="--case c4layer: 0..4 = L1..L4, FC")
     ap.add_argument("--presums", action="store_true", help="--case gemm: pass precomputed depth sums")
     ap.add_argument("--n", type=int, default=4096, help="GEMM edge, or conv batch, for --case")
     args = ap.parse_args()

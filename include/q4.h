@@ -150,7 +150,10 @@ q4_status q4_im2col(const uint8_t* X, const q4_conv_desc* d, int32_t za,
  * bytes -- this is Bt of the GEMM.  colsum_w [OC]: optional precomputed
  * sum_{kh,kw,c} w (the third term's sums), NULL = computed.  Y: packed NHWC output
  * N x OH x OW x OC (flat, row pitch OC/2 bytes; OC even).
- * ws: at least q4_conv2d_workspace_bytes(d) bytes, 256-byte aligned.
+ * ws: at least q4_conv2d_workspace_bytes(d) bytes, 256-byte aligned.  It is required
+ * for every layer, but a layer with OC a multiple of 8 (at most 64) and Y 8-byte
+ * aligned normally runs as one kernel that reads its taps straight from X and leaves
+ * ws untouched; other layers unroll into ws first.  The results are identical.
  */
 q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                     const int32_t* colsum_w, const int32_t* bias,
