@@ -38,13 +38,23 @@
 namespace q4 {
 namespace pair {
 
+#ifndef Q4_PAIR_BNC
+#define Q4_PAIR_BNC 192
+#endif
 constexpr int TMC = 128;             // rows of A per CTA
-constexpr int BNC = 192;             // columns of the pair tile
+constexpr int BNC = Q4_PAIR_BNC;     // columns of the pair tile (192 or 256)
 constexpr int BH = BNC / 2;          // rows of Bt staged per CTA
 constexpr int PROW = 64, UROW = 128, SLAB = 128;
-constexpr int PS = 6;                // packed stages (A 8 KB + Bt 6 KB)
-constexpr int US = 4;                // A operand stages in tensor memory (32 columns each)
-constexpr int BS = 8;                // Bt operand stages in shared memory (12 KB each)
+// Tensor memory holds NACC accumulators of BNC columns and US A stages of 32 columns.
+// 192 columns: two accumulators (the epilogue of a tile overlaps the next tile's main
+// loop) and four A stages.  256 columns (-DQ4_PAIR_BNC=256; bit-exact, measured 2 %
+// slower at 8192^3): one accumulator, six A stages, a third more work per MMA
+// instruction, but also a third more unpack work per CTA and stage, which is what
+// binds.
+constexpr int NACC = BNC == 256 ? 1 : 2;
+constexpr int PS = 6;                // packed stages (A 8 KB + Bt BH * 64 B)
+constexpr int US = BNC == 256 ? 6 : 4;   // A operand stages in tensor memory
+constexpr int BS = BNC == 256 ? 6 : 8;   // Bt operand stages in shared memory (BH * 128 B each)
 constexpr int PA = TMC * PROW;       // packed A bytes per stage
 constexpr int PSTAGE = PA + BH * PROW;
 constexpr int BSTAGE = BH * UROW;    // unpacked Bt bytes per stage
@@ -56,7 +66,7 @@ constexpr int UW = G * WPG;
 constexpr int NTB = BH * 4 / GT;     // Bt tasks (16-byte packed chunks) per thread per stage
 constexpr int NTHREADS = (2 + UW + 4) * 32;
 constexpr int TMEM_COLS = 512;
-constexpr int ACOL0 = 2 * BNC;       // first TMEM column of the A stages
+constexpr int ACOL0 = NACC * BNC;    // first TMEM column of the A stages
 constexpr int SUMS_N = TMC + BNC;    // per buffer and group: 128 row sums, BNC column sums
 
 constexpr int OFF_B = 0;
@@ -71,7 +81,8 @@ constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
 constexpr int SMEM = OFF_MISC + 16 + 1024;
 
 static_assert(BH * 4 % GT == 0, "Bt tasks must divide evenly");
-static_assert(2 * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
+static_assert(NACC * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
+static_assert(BS % US == 0, "the MMA loop walks blocks of BS stages and derives the A slot from the position in the block");
 static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
 static_assert(OFF_STG % 1024 == 0, "staging tile alignment (128-byte swizzle atoms)");
 
@@ -205,10 +216,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint64_t bdesc0 = make_kmajor_sw128_desc(sbase + OFF_B);
             uint32_t lt = 0;
             for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
-                const int acc = lt & 1;
-                const uint32_t aph = (lt >> 1) & 1u;
+                const int acc = (int)(lt % NACC);
+                const uint32_t aph = (lt / NACC) & 1u;
                 mbar_wait_cl(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
-                if (lt >= 2) mbar_wait_cl(bar_peer_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                if (lt >= (uint32_t)NACC) mbar_wait_cl(bar_peer_tempty(acc), aph ^ 1u, abort_flag, g.status);
                 tc_fence_after();
                 // both epilogues are done with buffer `acc`: tell the unpack warps of both CTAs
                 if (elect_one()) tc_commit_pair(bar_tstart(acc), 3);
@@ -218,15 +229,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 // The loop walks them in aligned blocks of BS so that ring slots, tensor-memory
                 // columns, descriptors and barrier addresses are compile-time offsets.
                 const uint32_t it_begin = lt * (uint32_t)p.nslab, it_end = it_begin + (uint32_t)p.nslab;
-                for (uint32_t blk = it_begin & ~(uint32_t)(BS - 1); blk < it_end; blk += BS) {
-                    const uint32_t bph = (blk / BS) & 1u;
+                for (uint32_t blk = it_begin - it_begin % BS; blk < it_end; blk += BS) {
+                    const uint32_t bph = (blk / US) & 1u;     // phase of A slot 0 in this block
 #pragma unroll
                     for (int j = 0; j < BS; ++j) {
                         const uint32_t it = blk + (uint32_t)j;
                         if (it < it_begin || it >= it_end) continue;        // warp-uniform
-                        // A ring slot j % US: its phase is (it / US) & 1 = (j / US) & 1, blk being
-                        // a multiple of 2 * US
-                        mbar_wait_cl(bar_full_u(j % US), (uint32_t)((j / US) & 1), abort_flag, g.status);
+                        // A ring slot j % US: its phase is (it / US) & 1, blk being a multiple of US
+                        mbar_wait_cl(bar_full_u(j % US), (bph + (uint32_t)(j / US)) & 1u, abort_flag, g.status);
                         tc_fence_after();
                         const uint32_t a_tmem = a_tmem0 + (uint32_t)((j % US) * 32);
                         const uint64_t bdesc = bdesc0 + (uint64_t)(j * (BSTAGE >> 4));
@@ -259,9 +269,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // -------------------------------------------------------- peer relay (per tile)
             uint32_t lt = 0;
             for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
-                const int acc = lt & 1;
-                const uint32_t aph = (lt >> 1) & 1u;
-                if (lt >= 2) {
+                const int acc = (int)(lt % NACC);
+                const uint32_t aph = (lt / NACC) & 1u;
+                if (lt >= (uint32_t)NACC) {
                     mbar_wait_cl(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
                     mbar_arrive_cluster(map_to_cta(bar_peer_tempty(acc), 0));
                 }
@@ -370,9 +380,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
             }
             if (need_sums) {
-                const int acc = lt & 1;
-                const uint32_t aph = (lt >> 1) & 1u;
-                // both CTAs' epilogues two tiles back are done with this sums buffer
+                const int acc = (int)(lt % NACC);
+                const uint32_t aph = (lt / NACC) & 1u;
+                // both CTAs' epilogues NACC tiles back are done with this sums buffer
                 mbar_wait_cl(bar_tstart(acc), aph, abort_flag, g.status);
                 const uint32_t mine = sums_s + 4 * ((acc * G + grp) * SUMS_N);
                 sts32(mine + 4 * arow, psum_a);
@@ -405,8 +415,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         uint32_t lt = 0;
         for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
             const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
-            const int acc = lt & 1;
-            const uint32_t aph = (lt >> 1) & 1u;
+            const int acc = (int)(lt % NACC);
+            const uint32_t aph = (lt / NACC) & 1u;
             const int m = tm * 256 + (int)rank * TMC + row;
             const int n0 = tn * BNC;
             if (need_sums) mbar_wait_cl(bar_sums(acc), aph, abort_flag, g.status);
