@@ -233,6 +233,37 @@ def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20):
             "timing": f"median of 5 x {reps} back-to-back launches per layer"}
 
 
+def time_im2col(q4, wl, hbm_peak: float, batch: int = 4096, reps: int = 10):
+    """Device time of q4_im2col (the explicit unrolling, with row sums) on the c3 layer shape at a
+    batch whose matrix (about 0.34 GB at 4096) exceeds L2, so the stores go to HBM.  Algorithmic
+    bytes: |X| + M * lda + 4 * M."""
+    import torch
+    L = wl.c3(batch=1).layers[0]
+    d = q4.ConvDesc(batch, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
+    X = torch.from_numpy(wl.rand_flat_nibbles(78, 1, batch * L.H * L.W * L.C)).cuda()
+    lda = (d.K // 2 + 15) // 16 * 16
+    A = torch.empty((d.M, lda), dtype=torch.uint8, device="cuda")
+    ra = torch.empty(d.M, dtype=torch.int32, device="cuda")
+    for _ in range(3):
+        q4.q4_im2col(X, d, L.za, A, ra)
+    ts = []
+    for _ in range(5):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda._sleep(2_000_000)
+        e0.record()
+        for _ in range(reps):
+            q4.q4_im2col(X, d, L.za, A, ra)
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1) / reps)
+    ms = statistics.median(ts)
+    nbytes = X.numel() + A.numel() + 4 * d.M
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"shape": f"c3 layer geometry, batch {batch}: M={d.M}, K={d.K}, pitch {lda} B", "ms": ms,
+            "algorithmic_bytes": nbytes, "gbs": gbs, "frac_of_hbm": gbs / hbm_peak,
+            "timing": f"median of 5 x {reps} back-to-back launches"}
+
+
 def run_ours(args):
     import torch
     rank, world, local = dist_env()
@@ -354,6 +385,7 @@ def run_ours(args):
 
     # ---- the c4 layer chain (batch 4096), outside the timed region: per-layer device times
     c4_detail = time_c4_chain(q4, wl) if world == 1 and not args.no_c4_chain else None
+    im2col_detail = time_im2col(q4, wl, peaks["hbm"]) if world == 1 and not args.no_c4_chain else None
 
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
     cpu_baseline = None
@@ -398,6 +430,7 @@ def run_ours(args):
             "q4_conv2d_c3_unroll_path_equivalent_gbs": conv_path_bytes / (conv_ms * 1e-3) / 1e9,
             "q4_conv2d_c3_gops": conv_ops / (conv_ms * 1e-3) / 1e9,
             "c4_chain_batch4096": c4_detail,
+            "q4_im2col": im2col_detail,
             "hbm_peak_gbs": peaks["hbm"], "peaks": peaks["source"]},
     }
     print(json.dumps(line))

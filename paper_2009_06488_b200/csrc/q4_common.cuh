@@ -84,6 +84,27 @@ __device__ __forceinline__ int nibble_sum(uint32_t w)
     return dp4a_u8(s, 0x01010101u, 0);
 }
 
+// n / d for n < 2^31 as (umulhi(n, mul) + n) >> shift (round-up method: shift =
+// ceil(log2 d), mul = floor(2^32 * (2^shift - d) / d) + 1).
+struct FastDiv {
+    uint32_t mul, shift;
+};
+
+inline FastDiv make_fastdiv(uint32_t d)
+{
+    FastDiv f;
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;
+    f.shift = l;
+    f.mul = (uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1);
+    return f;
+}
+
+__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
+{
+    return (__umulhi(n, f.mul) + n) >> f.shift;
+}
+
 // ----- launchers implemented in the kernel translation units -----------------------
 cudaError_t launch_gemm_simt(const GemmParams& p, bool requant, cudaStream_t st);
 bool        gemm_tc_supported(const GemmParams& p);

@@ -52,27 +52,6 @@ constexpr int NBUF_MMA = 3;              // input buffers: the producer runs NBU
 constexpr int NBUF_LANE = 4;
 constexpr int SYNC_BYTES = 64;             // the buffers' mbarriers and the abort flag
 
-// n / d for n < 2^31 as (umulhi(n, mul) + n) >> shift (round-up method: shift =
-// ceil(log2 d), mul = floor(2^32 * (2^shift - d) / d) + 1).
-struct FastDiv {
-    uint32_t mul, shift;
-};
-
-static FastDiv make_fastdiv(uint32_t d)
-{
-    FastDiv f;
-    uint32_t l = 0;
-    while ((1ull << l) < d) ++l;
-    f.shift = l;
-    f.mul = (uint32_t)(((1ull << 32) * ((1ull << l) - d)) / d + 1);
-    return f;
-}
-
-__device__ __forceinline__ uint32_t fdiv(uint32_t n, const FastDiv& f)
-{
-    return (__umulhi(n, f.mul) + n) >> f.shift;
-}
-
 struct Params {
     const uint8_t* X;
     const uint8_t* Wt;
@@ -865,12 +844,12 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     p.sfull = (p.OH - 1) * d.stride_h + d.KH;
     p.vec16 = (!expanded || nibbles) && rowbytes % 16 == 0 && (uintptr_t)X % 16 == 0;
     p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
-    p.div_ow = fused::make_fastdiv((uint32_t)p.OW);
-    p.div_oh = fused::make_fastdiv((uint32_t)p.OH);
-    p.div_sfull = fused::make_fastdiv((uint32_t)p.sfull);
+    p.div_ow = make_fastdiv((uint32_t)p.OW);
+    p.div_oh = make_fastdiv((uint32_t)p.OH);
+    p.div_sfull = make_fastdiv((uint32_t)p.sfull);
     p.cpr = (int32_t)(rowbytes / 4);
     if (p.cpr < 1) p.cpr = 1;                          // expanded mode does not use it
-    p.div_cpr = fused::make_fastdiv((uint32_t)p.cpr);
+    p.div_cpr = make_fastdiv((uint32_t)p.cpr);
     p.step8 = (int32_t)(8 * d.stride_w * unit);
     p.rowwrap = (int32_t)(d.stride_h * pitch - (int64_t)p.OW * d.stride_w * unit);
     p.imgwrap = (int32_t)((d.KH - d.stride_h) * pitch);

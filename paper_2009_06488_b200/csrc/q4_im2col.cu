@@ -2,7 +2,14 @@
 // (GEMM-based convolution, Section I; depth D = kh*kw*c, Section III-A), with the
 // per-row sums of Eq. 2's second term taken on the way (Section II-B).
 //
-// Two kernels:
+// Three kernels:
+//  * im2col_tile_kernel -- same geometry as the next one, output pitch up to 256 bytes:
+//    a warp takes 32 consecutive output rows, one row per lane.  A lane decodes its
+//    pixel once, walks its row's taps (the lanes' loads of one tap are consecutive
+//    pixels of the input: coalesced), sums its row's values in a register and writes
+//    the row into a shared-memory tile; the warp then copies the tile, which is one
+//    contiguous piece of the matrix, to memory with full-line 128-bit stores.  No
+//    atomics, no 64-bit divisions.
 //  * im2col_vec_kernel  -- channels give byte-aligned taps of 4, 8 or a multiple of 16
 //    bytes and the output pitch is a multiple of 16: one thread per 16-byte output
 //    chunk, consecutive lanes write consecutive chunks (fully coalesced 128-bit
@@ -125,6 +132,98 @@ __global__ void __launch_bounds__(256) im2col_vec_kernel(const Im2colParams p, i
     }
 }
 
+// One output row per lane, 32 rows per warp and step; see the head of the file.
+constexpr int TILE_WARPS = 8;
+constexpr int TILE_MAX_LDA = 256;
+
+template <int TAPB>
+__global__ void __launch_bounds__(TILE_WARPS * 32)
+im2col_tile_kernel(const Im2colParams p, int tapb, FastDiv div_ow, FastDiv div_oh)
+{
+    extern __shared__ __align__(16) uint8_t tile_smem[];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int lda = (int)p.lda, cpr = lda >> 4;
+    uint8_t* tile = tile_smem + warp * 32 * lda;
+    uint8_t* myrow = tile + lane * lda;
+    const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
+    const uint32_t M = (uint32_t)p.M;
+    const int64_t groups = ((int64_t)M + 31) / 32;
+    const int64_t imgbytes = (int64_t)p.H * p.W * tapb;
+
+    for (int64_t gi = (int64_t)blockIdx.x * TILE_WARPS + warp; gi < groups;
+         gi += (int64_t)gridDim.x * TILE_WARPS) {
+        const uint32_t m0 = (uint32_t)(gi * 32);
+        const bool valid = m0 + lane < M;
+        const uint32_t m = valid ? m0 + lane : m0;      // lanes past the end redo row m0 (not stored)
+        const uint32_t q = fdiv(m, div_ow);
+        const int ow = (int)(m - q * (uint32_t)p.OW);
+        const uint32_t n = fdiv(q, div_oh);
+        const int oh = (int)(q - n * (uint32_t)p.OH);
+        const int ih0 = oh * p.sh - p.ph, iw0 = ow * p.sw - p.pw;
+        const uint8_t* img = p.X + (int64_t)n * imgbytes;
+
+        // row sum = (sum of low nibbles) + (sum of bytes - sum of low nibbles) / 16
+        int sum_bytes = 0, sum_low = 0, kh = 0, kw = 0, off = 0;
+#pragma unroll 4
+        for (int j = 0; j < cpr; ++j) {
+            uint32_t w[4] = {0, 0, 0, 0};
+            if (TAPB < 16) {
+                constexpr int TPC = 16 / TAPB;          // taps per chunk
+                constexpr int WPT = TAPB / 4;           // words per tap
+#pragma unroll
+                for (int i = 0; i < TPC; ++i) {
+                    if (kh < p.KH) {
+                        const int ih = ih0 + kh, iw = iw0 + kw;
+                        if ((unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W) {
+                            const uint8_t* src = img + (ih * p.W + iw) * TAPB;
+                            if (WPT == 1) {
+                                w[i] = *reinterpret_cast<const uint32_t*>(src);
+                            } else {
+                                const uint2 v = *reinterpret_cast<const uint2*>(src);
+                                w[2 * i] = v.x; w[2 * i + 1] = v.y;
+                            }
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < WPT; ++e) w[i * WPT + e] = zfill;
+                        }
+                        if (++kw == p.KW) { kw = 0; ++kh; }
+                    }
+                }
+            } else {
+                if (kh < p.KH) {
+                    const int ih = ih0 + kh, iw = iw0 + kw;
+                    if ((unsigned)ih < (unsigned)p.H && (unsigned)iw < (unsigned)p.W) {
+                        const uint4 v = *reinterpret_cast<const uint4*>(
+                            img + (int64_t)(ih * p.W + iw) * tapb + off);
+                        w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+                    } else {
+                        w[0] = w[1] = w[2] = w[3] = zfill;
+                    }
+                    off += 16;
+                    if (off == tapb) {
+                        off = 0;
+                        if (++kw == p.KW) { kw = 0; ++kh; }
+                    }
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                sum_bytes = dp4a_u8(w[e], 0x01010101u, sum_bytes);
+                sum_low = dp4a_u8(w[e] & 0x0F0F0F0Fu, 0x01010101u, sum_low);
+            }
+            *reinterpret_cast<uint4*>(myrow + 16 * j) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        __syncwarp();
+        const uint32_t left = M - m0;
+        const int nchunks = (int)(left < 32u ? left : 32u) * cpr;
+        uint8_t* out = p.A + (int64_t)m0 * lda;
+        for (int c = lane; c < nchunks; c += 32)
+            __stcs(reinterpret_cast<uint4*>(out + 16 * c), *reinterpret_cast<const uint4*>(tile + 16 * c));
+        if (p.rowsum && valid) p.rowsum[m] = sum_low + ((sum_bytes - sum_low) >> 4);
+        __syncwarp();                                  // the tile is rewritten in the next step
+    }
+}
+
 __device__ __forceinline__ uint32_t fetch_nibble(const Im2colParams& p, int n, int ih0, int iw0, int k)
 {
     if (k >= p.K) return 0;
@@ -174,14 +273,34 @@ cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, u
     p.za = za;
     if (p.M == 0) return cudaSuccess;
 
+    const int tapb = d.C / 2;
+    const bool aligned = ((uintptr_t)X % 16 == 0) && ((uintptr_t)A % 16 == 0) && (lda % 16 == 0);
+    const bool vec = aligned && (d.C % 2 == 0) && (tapb == 4 || tapb == 8 || tapb % 16 == 0);
+
+    if (vec && lda <= TILE_MAX_LDA && p.M < (1ll << 31)) {
+        const size_t smem = (size_t)TILE_WARPS * 32 * (size_t)lda;
+        const FastDiv dow = make_fastdiv((uint32_t)p.OW), doh = make_fastdiv((uint32_t)p.OH);
+        auto kernel = tapb == 4 ? im2col_tile_kernel<4> : tapb == 8 ? im2col_tile_kernel<8>
+                                                                   : im2col_tile_kernel<16>;
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             TILE_WARPS * 32 * TILE_MAX_LDA);
+        if (e != cudaSuccess) return e;
+        int per_sm = 1;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, TILE_WARPS * 32, smem) !=
+                cudaSuccess || per_sm < 1)
+            per_sm = 1;
+        const int64_t groups = (p.M + 31) / 32;
+        int64_t blocks = (groups + TILE_WARPS - 1) / TILE_WARPS;
+        if (blocks > 148ll * per_sm) blocks = 148ll * per_sm;
+        kernel<<<(int)blocks, TILE_WARPS * 32, smem, st>>>(p, tapb, dow, doh);
+        count_launch();
+        return cudaGetLastError();
+    }
+
     if (rowsum_a) {
         cudaError_t e = cudaMemsetAsync(rowsum_a, 0, sizeof(int32_t) * (size_t)p.M, st);
         if (e != cudaSuccess) return e;
     }
-
-    const int tapb = d.C / 2;
-    const bool aligned = ((uintptr_t)X % 16 == 0) && ((uintptr_t)A % 16 == 0) && (lda % 16 == 0);
-    const bool vec = aligned && (d.C % 2 == 0) && (tapb == 4 || tapb == 8 || tapb % 16 == 0);
     const int64_t work = vec ? p.M * (lda / 16) : p.M * lda;
     int64_t blocks = (work + 255) / 256;
     const int64_t cap = 148 * 32;

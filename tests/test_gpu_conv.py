@@ -39,6 +39,9 @@ IM2COL = [  # N, H, W, C, KH, KW, stride_h, stride_w, pad_h, pad_w
     (3, 4, 4, 96, 1, 1, 1, 1, 0, 0),       # 48-byte taps, pointwise
     (1, 6, 6, 4, 3, 3, 1, 1, 2, 2),        # 2-byte taps -> byte kernel
     (2, 8, 8, 12, 5, 5, 1, 1, 2, 2),       # 6-byte taps -> byte kernel
+    (5, 19, 17, 16, 3, 3, 1, 1, 1, 1),     # 1615 rows: many 32-row tiles and a ragged last one
+    (7, 21, 13, 8, 3, 3, 2, 2, 1, 1),      # 4-byte taps, stride 2, 539 rows
+    (3, 9, 11, 32, 3, 3, 1, 1, 1, 1),      # 16-byte taps, pitch 144
 ]
 
 
