@@ -50,7 +50,7 @@ constexpr int ROWS_PER_CTA = WARPS * ROWS_PER_WARP;
 constexpr int SMEM_LIMIT = 160 * 1024;
 constexpr int NBUF_MMA = 3;              // input buffers: the producer runs NBUF - 1 tiles ahead
 constexpr int NBUF_LANE = 4;
-constexpr int SYNC_BYTES = 64;             // the buffers' mbarriers and the abort flag
+constexpr int SYNC_BYTES = 96;             // the buffers' "landed" and "read" mbarriers and the abort flag
 
 struct Params {
     const uint8_t* X;
@@ -79,6 +79,7 @@ struct Params {
     unsigned* status;          // device status word (a wait that ran out is recorded there)
     int32_t wt_words;          // weights can be read as aligned 32-bit words
     int32_t cpr;               // packed: copy pieces (16 or 4 bytes) per image row
+    int32_t tile;              // output pixels per CTA tile
     int32_t step8;             // staged-buffer offset of the pixel eight further in the same output row
     int32_t rowwrap;           // ... added when that pixel is in the next output row
     int32_t imgwrap;           // ... added on top when that row is the next image's first
@@ -151,8 +152,8 @@ struct Geo {
 
 __device__ __forceinline__ Geo tile_geometry(const Params& p, int64_t tile)
 {
-    const int64_t mb = tile * ROWS_PER_CTA;
-    const int64_t me = (mb + ROWS_PER_CTA < p.M ? mb + ROWS_PER_CTA : p.M) - 1;
+    const int64_t mb = tile * p.tile;
+    const int64_t me = (mb + p.tile < p.M ? mb + p.tile : p.M) - 1;
     const uint32_t q_first = fdiv((uint32_t)mb, p.div_ow), q_last = fdiv((uint32_t)me, p.div_ow);
     const uint32_t n_first = fdiv(q_first, p.div_oh), n_last = fdiv(q_last, p.div_oh);
     const int oh_first = (int)(q_first - n_first * (uint32_t)p.OH);
@@ -202,21 +203,25 @@ __device__ __forceinline__ void stage_packed_bulk(const Params& p, const Geo& g,
     // ordinary stores to this buffer (the initial fill, earlier border rows) come before
     // the copy engine's writes
     fence_async_smem();
-    int inside = 0;
-    for (int s = lane; s < g.nslots; s += 32) inside += staged_row(p, g, s) >= 0;
-    inside = __reduce_add_sync(0xFFFFFFFFu, inside);
-    if (lane == 0) mbar_expect_tx(bar, (uint32_t)inside * (uint32_t)p.rowbytes);
-    __syncwarp();
     const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
+    int inside = 0;
     for (int s = lane; s < g.nslots; s += 32) {
-        const int64_t row = staged_row(p, g, s);
-        uint8_t* dst = buf + s * p.pitch + p.data0;
-        if (row >= 0) {
-            bulk_load_row(smem_u32(dst), p.X + row * p.rowbytes, (uint32_t)p.rowbytes, bar);
+        if (staged_row(p, g, s) >= 0) {
+            ++inside;
         } else {
+            uint8_t* dst = buf + s * p.pitch + p.data0;
             for (int c = 0; c < p.rowbytes; c += 16)
                 *reinterpret_cast<uint4*>(dst + c) = make_uint4(zfill, zfill, zfill, zfill);
         }
+    }
+    inside = __reduce_add_sync(0xFFFFFFFFu, inside);   // also orders the fills before lane 0's arrive
+    if (lane == 0) mbar_expect_tx(bar, (uint32_t)inside * (uint32_t)p.rowbytes);
+    __syncwarp();
+    for (int s = lane; s < g.nslots; s += 32) {
+        const int64_t row = staged_row(p, g, s);
+        if (row >= 0)
+            bulk_load_row(smem_u32(buf + s * p.pitch + p.data0), p.X + row * p.rowbytes,
+                          (uint32_t)p.rowbytes, bar);
     }
 }
 
@@ -281,23 +286,61 @@ __device__ __forceinline__ void stage_expanded(const Params& p, const Geo& g, ui
     }
 }
 
+// The producer warp's loop.  Tile j lives in buffer j % NB.  A buffer is refilled once every
+// multiplying warp has reported (on its "read" mbarrier) that it is done with the tile that
+// was there; a tile is announced on the buffer's "landed" mbarrier -- by the bulk copies
+// themselves, or by lane 0 once this warp's copies of that tile have landed, which is
+// checked NB - 2 tiles later so that copies stay in flight.  The tile's geometry is
+// written before the arrive that publishes it.
+template <int NB, bool EXPANDED>
+__device__ __forceinline__ void producer_loop(const Params& p, int mytiles, uint8_t* buf0, int4* geo_s,
+                                              uint32_t full0, uint32_t empty0, uint32_t abort_flag, int lane)
+{
+    constexpr int LOOK = NB - 2;
+    const bool bulk = !EXPANDED && p.vec16;
+    int b = 0;                                         // j % NB
+    uint32_t round = 0;                                // j / NB
+    for (int j = 0; j < mytiles + LOOK; ++j) {
+        if (j < mytiles) {
+            if (round > 0) mbar_wait(empty0 + 8 * b, (round - 1) & 1, abort_flag, p.status);
+            const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
+            if (lane == 0) geo_s[b] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
+            uint8_t* buf = buf0 + b * p.bufbytes;
+            if (EXPANDED) stage_expanded(p, gn, buf, lane);
+            else if (bulk) stage_packed_bulk(p, gn, buf, full0 + 8 * b, lane);
+            else stage_packed(p, gn, buf, lane);
+            if (++b == NB) { b = 0; ++round; }
+        }
+        cp_async_commit();                             // one group per tile, empty past the end
+        if (!bulk) {
+            cp_async_wait_group<LOOK>();
+            __syncwarp();
+            const int d = j - LOOK;                    // this tile's copies have landed
+            if (lane == 0 && d >= 0) mbar_arrive(full0 + 8 * (d % NB));
+        }
+    }
+}
+
+// A multiplying warp is done reading a buffer.
+__device__ __forceinline__ void release_buffer(uint32_t empty_bar, int lane)
+{
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty_bar);
+}
+
 // NT = OC / 8 output-channel tiles.  Fragment column f of tile nt is output channel
 // 2 * (NT * (f / 2) + nt) + f % 2, so that the NT packed output bytes a thread ends up
 // with are contiguous in memory.
 //
-// Warps 0..6 multiply; warp 7 is the producer: while the others work on tile k it
-// derives the geometry of tile k+1, copies its input rows into the other buffer and
-// leaves the geometry in shared memory.  One block-wide barrier per tile hands over
-// both the finished copy and the buffer that has just been read.
+// Warps 0..6 multiply; warp 7 is the producer: it runs up to NB tiles ahead, deriving a
+// tile's geometry and copying its input rows into the next buffer of the ring.  Buffers
+// change hands through two mbarriers each ("landed", "read"), so no warp waits for
+// another multiplying warp.
 constexpr int THREADS = (WARPS + 1) * 32;
 
-__device__ __forceinline__ void tile_barrier()
-{
-    asm volatile("bar.sync 1, %0;" :: "n"(THREADS) : "memory");
-}
 
 template <int NT, bool EXP>
-__global__ void __launch_bounds__(THREADS, NT <= 2 ? 3 : 2)
+__global__ void __launch_bounds__(THREADS, NT <= 2 ? 4 : NT <= 4 ? 3 : 2)
 conv_fused_kernel(const Params p)
 {
     extern __shared__ __align__(16) uint8_t smem[];
@@ -310,7 +353,7 @@ conv_fused_kernel(const Params p)
     int4* geo_s = reinterpret_cast<int4*>(colsum_s + N);                             // [NB]
     uint64_t* full_s = reinterpret_cast<uint64_t*>(geo_s + NB);                      // [NB] "tile landed"
     uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB) + SYNC_BYTES;             // 16-byte aligned
-    const uint32_t full0 = smem_u32(full_s), abort_flag = full0 + 8 * NB;
+    const uint32_t full0 = smem_u32(full_s), empty0 = full0 + 8 * NB, abort_flag = full0 + 16 * NB;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;
@@ -327,7 +370,10 @@ conv_fused_kernel(const Params p)
         fence_async_smem();                            // before the copy engine writes the same bytes
     }
     if (tid == 0) {
-        for (int i = 0; i < NB; ++i) mbar_init(full0 + 8 * i, 1);
+        for (int i = 0; i < NB; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, WARPS);
+        }
         sts32(abort_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -397,33 +443,7 @@ conv_fused_kernel(const Params p)
 
     if (warp == WARPS) {
         // ---------------- producer ----------------
-        // Tile j lives in buffer j % NB.  Before barrier k+1 the copy of tile k+1 must have
-        // landed; the copies of the NB - 2 tiles after it may still be in flight.  The
-        // buffer of tile k + NB - 1 is the one tile k - 1 was read from, free since barrier k.
-        // Either way the consumers also wait on the buffer's mbarrier: bulk copies report
-        // to it themselves; otherwise lane 0 arrives once this warp's copies have landed.
-        const bool bulk = !EXP && p.vec16;
-        auto produce = [&](int j) {
-            if (j < mytiles) {
-                const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
-                uint8_t* buf = buf0 + (j % NB) * p.bufbytes;
-                if (EXP) stage_expanded(p, gn, buf, lane);
-                else if (bulk) stage_packed_bulk(p, gn, buf, full0 + 8 * (j % NB), lane);
-                else stage_packed(p, gn, buf, lane);
-                if (lane == 0) geo_s[j % NB] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
-            }
-            cp_async_commit();                         // one group per tile, empty past the end
-        };
-        for (int j = 0; j < NB - 1; ++j) produce(j);
-        for (int k = -1; k < mytiles; ++k) {
-            if (k >= 0) produce(k + NB - 1);
-            if (!bulk) {
-                cp_async_wait_group<NB - 2>();
-                __syncwarp();
-                if (lane == 0 && k + 1 < mytiles) mbar_arrive(full0 + 8 * ((k + 1) % NB));
-            }
-            tile_barrier();
-        }
+        producer_loop<NB, EXP>(p, mytiles, buf0, geo_s, full0, empty0, abort_flag, lane);
         return;
     }
 
@@ -448,11 +468,11 @@ conv_fused_kernel(const Params p)
     uint32_t mbase = blockIdx.x * (uint32_t)ROWS_PER_CTA;
     int kb = 0;                                        // k % NB
     uint32_t phase = 0;                                // (k / NB) % 2
-    tile_barrier();
     for (int k = 0; k < mytiles; ++k, mbase += mstep) {
         const uint8_t* buf = buf0 + kb * p.bufbytes;
-        const int4 gv = geo_s[kb];                     // n_first, oh_first, s0
         mbar_wait(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
+        const int4 gv = geo_s[kb];                     // n_first, oh_first, s0 (published with the tile)
+        const uint32_t done_bar = empty0 + 8 * kb;
         if (++kb == NB) { kb = 0; phase ^= 1; }
         const uint32_t left = M32 - mbase;             // > 0
         const int myrows = (int)(left < (uint32_t)ROWS_PER_CTA ? left : (uint32_t)ROWS_PER_CTA) -
@@ -595,7 +615,7 @@ conv_fused_kernel(const Params p)
             // the 32-bit form of the rounding shift needs shift >= 2 (see requant())
             if (p.rq.shift >= 2) epilogue(std::true_type{}); else epilogue(std::false_type{});
         }
-        tile_barrier();
+        release_buffer(done_bar, lane);
     }
 }
 
@@ -625,7 +645,7 @@ conv_lane_kernel(const Params p)
     int4* geo_s = reinterpret_cast<int4*>(colterm_s + OC);                           // [NB]
     uint64_t* full_s = reinterpret_cast<uint64_t*>(geo_s + NB);                      // [NB] "tile landed"
     uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB) + SYNC_BYTES;             // 16-byte aligned
-    const uint32_t full0 = smem_u32(full_s), abort_flag = full0 + 8 * NB;
+    const uint32_t full0 = smem_u32(full_s), empty0 = full0 + 8 * NB, abort_flag = full0 + 16 * NB;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int segbytes = p.KW * p.C;
@@ -639,7 +659,10 @@ conv_lane_kernel(const Params p)
         fence_async_smem();                            // before the copy engine writes the same bytes
     }
     if (tid == 0) {
-        for (int i = 0; i < NB; ++i) mbar_init(full0 + 8 * i, 1);
+        for (int i = 0; i < NB; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, WARPS);
+        }
         sts32(abort_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -672,29 +695,8 @@ conv_lane_kernel(const Params p)
     const int mytiles = (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
 
     if (warp == WARPS) {
-        // ---------------- producer (same protocol as conv_fused_kernel) ----------------
-        const bool bulk = NIB && p.vec16;
-        auto produce = [&](int j) {
-            if (j < mytiles) {
-                const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
-                uint8_t* buf = buf0 + (j % NB) * p.bufbytes;
-                if (!NIB) stage_expanded(p, gn, buf, lane);
-                else if (bulk) stage_packed_bulk(p, gn, buf, full0 + 8 * (j % NB), lane);
-                else stage_packed(p, gn, buf, lane);
-                if (lane == 0) geo_s[j % NB] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
-            }
-            cp_async_commit();
-        };
-        for (int j = 0; j < NB - 1; ++j) produce(j);
-        for (int k = -1; k < mytiles; ++k) {
-            if (k >= 0) produce(k + NB - 1);
-            if (!bulk) {
-                cp_async_wait_group<NB - 2>();
-                __syncwarp();
-                if (lane == 0 && k + 1 < mytiles) mbar_arrive(full0 + 8 * ((k + 1) % NB));
-            }
-            tile_barrier();
-        }
+        // ---------------- producer ----------------
+        producer_loop<NB, !NIB>(p, mytiles, buf0, geo_s, full0, empty0, abort_flag, lane);
         return;
     }
 
@@ -706,11 +708,11 @@ conv_lane_kernel(const Params p)
     uint32_t mbase = blockIdx.x * (uint32_t)ROWS_PER_CTA;
     int kb = 0;                                        // k % NB
     uint32_t phase = 0;                                // (k / NB) % 2
-    tile_barrier();
     for (int k = 0; k < mytiles; ++k, mbase += mstep) {
         const uint8_t* buf = buf0 + kb * p.bufbytes;
-        const int4 gv = geo_s[kb];                     // n_first, oh_first, s0
         mbar_wait(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
+        const int4 gv = geo_s[kb];                     // n_first, oh_first, s0 (published with the tile)
+        const uint32_t done_bar = empty0 + 8 * kb;
         if (++kb == NB) { kb = 0; phase ^= 1; }
         const uint32_t left = M32 - mbase;             // > 0
         const int rows = (int)(left < (uint32_t)ROWS_PER_CTA ? left : (uint32_t)ROWS_PER_CTA);
@@ -786,7 +788,176 @@ conv_lane_kernel(const Params p)
                 else *reinterpret_cast<uint2*>(dst) = make_uint2(out[0], out[(OC / 8 - 1)]);
             }
         }
-        tile_barrier();
+        release_buffer(done_bar, lane);
+    }
+}
+
+// ---------------------------------------------------------------------------------
+// Four horizontally adjacent output pixels per lane, for 3x3 stride-1 layers on a
+// single-channel input with eight output channels (a gray-image first layer) whose
+// output rows are whole groups of four.  The four pixels' taps of one filter row are
+// six consecutive nibbles of the packed copy in shared memory: one unaligned 32-bit
+// window per filter row is split into its even and odd nibbles (as bytes), from which
+// each pixel's three taps are picked by one byte permutation.  Pixel decode, window
+// loads and weight loads are paid once per four pixels, and a lane's 16 packed output
+// bytes leave in one store (a warp's stores are 512 contiguous bytes).  A CTA tile is
+// 4 * 224 pixels; staging protocol and weight set-up are those of conv_lane_kernel.
+// ---------------------------------------------------------------------------------
+constexpr int QUAD = 4;
+constexpr int QUAD_TILE = QUAD * ROWS_PER_CTA;
+
+__global__ void __launch_bounds__(THREADS, 4)
+conv_quad_kernel(const Params p)
+{
+    constexpr int OC = 8, KH = 3;
+    extern __shared__ __align__(16) uint8_t smem[];
+    uint32_t* wsm = reinterpret_cast<uint32_t*>(smem);                               // [KH][OC]
+    int32_t* colterm_s = reinterpret_cast<int32_t*>(wsm + KH * OC);                  // [OC]
+    constexpr int NB = NBUF_LANE;
+    int4* geo_s = reinterpret_cast<int4*>(colterm_s + OC);                           // [NB]
+    uint64_t* full_s = reinterpret_cast<uint64_t*>(geo_s + NB);                      // [NB] "tile landed"
+    uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB) + SYNC_BYTES;             // 16-byte aligned
+    const uint32_t full0 = smem_u32(full_s), empty0 = full0 + 8 * NB, abort_flag = full0 + 16 * NB;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+    // ---- once per CTA: signed weight words, the constant left of Eq. 3, zero-point fill
+    for (int i = tid; i < OC; i += THREADS) colterm_s[i] = 0;
+    {
+        uint32_t* b = reinterpret_cast<uint32_t*>(buf0);
+        const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
+        for (int i = tid; i < NB * p.bufbytes / 4; i += THREADS) b[i] = zfill;
+        fence_async_smem();                            // before the copy engine writes the same bytes
+    }
+    if (tid == 0) {
+        for (int i = 0; i < NB; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, WARPS);
+        }
+        sts32(abort_flag, 0);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    for (int i = tid; i < KH * OC; i += THREADS) {
+        const int n = i % OC, kh = i / OC;
+        uint32_t word = 0;
+        int raw = 0;
+        for (int q = 0; q < 3; ++q) {
+            const uint32_t nib = weight_nibble(p, n, kh * 3 + q);
+            raw += (int)nib;
+            word |= ((nib - (uint32_t)p.zb) & 0xFFu) << (8 * q);
+        }
+        wsm[i] = word;                                 // fourth byte 0: the window's next nibble counts for nothing
+        if (!p.colsum_w && raw) atomicAdd(&colterm_s[n], raw);
+    }
+    __syncthreads();
+    if (tid < OC) {
+        const int cs = p.colsum_w ? p.colsum_w[tid] : colterm_s[tid];
+        colterm_s[tid] = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
+                               (uint32_t)(p.bias ? p.bias[tid] : 0));
+    }
+    __syncthreads();
+
+    const int64_t ntiles = (p.M + QUAD_TILE - 1) / QUAD_TILE;
+    const int mytiles = (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+
+    if (warp == WARPS) {
+        // ---------------- producer ----------------
+        producer_loop<NB, false>(p, mytiles, buf0, geo_s, full0, empty0, abort_flag, lane);
+        return;
+    }
+
+    // ---------------- consumers ----------------
+    const int r = warp * ROWS_PER_WARP + lane;         // my group of four within a tile
+    const uint32_t M32 = (uint32_t)p.M, mstep = gridDim.x * (uint32_t)QUAD_TILE;
+    uint32_t mbase = blockIdx.x * (uint32_t)QUAD_TILE;
+    const int s = p.rq.shift - 1, rnd = s > 0 ? 1 << (s - 1) : 0;
+    int kb = 0;                                        // k % NB
+    uint32_t phase = 0;                                // (k / NB) % 2
+    for (int k = 0; k < mytiles; ++k, mbase += mstep) {
+        const uint8_t* buf = buf0 + kb * p.bufbytes;
+        mbar_wait(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
+        const int4 gv = geo_s[kb];                     // n_first, oh_first, s0 (published with the tile)
+        const uint32_t done_bar = empty0 + 8 * kb;
+        if (++kb == NB) { kb = 0; phase ^= 1; }
+        const uint32_t left = M32 - mbase;             // > 0, a multiple of four
+        const int groups = (int)(left < (uint32_t)QUAD_TILE ? left : (uint32_t)QUAD_TILE) / QUAD;
+        if (warp * ROWS_PER_WARP < groups) {           // warp-uniform
+            const bool valid = r < groups;
+            const uint32_t mm = mbase + (uint32_t)(valid ? QUAD * r : 0);
+            const uint32_t q = fdiv(mm, p.div_ow);
+            const int ow = (int)(mm - q * (uint32_t)p.OW);
+            const uint32_t n0 = fdiv(q, p.div_oh);
+            const int oh = (int)(q - n0 * (uint32_t)p.OH);
+            const int seg = (int)n0 - gv.x;
+            const int slot0 = seg == 0 ? oh - gv.y : gv.z + (seg - 1) * p.sfull + oh;
+            const int b = slot0 * p.pitch * 2 + p.pix0 + ow;       // nibble offset of my first tap
+            const int shf = (b & 7) * 4;
+            const uint8_t* src = buf + ((b >> 3) << 2);
+
+            int acc[QUAD][OC];
+            {
+                const int4 c0 = *reinterpret_cast<const int4*>(colterm_s);
+                const int4 c1 = *reinterpret_cast<const int4*>(colterm_s + 4);
+#pragma unroll
+                for (int px = 0; px < QUAD; ++px) {
+                    acc[px][0] = c0.x; acc[px][1] = c0.y; acc[px][2] = c0.z; acc[px][3] = c0.w;
+                    acc[px][4] = c1.x; acc[px][5] = c1.y; acc[px][6] = c1.z; acc[px][7] = c1.w;
+                }
+            }
+#pragma unroll
+            for (int kh = 0; kh < KH; ++kh) {
+                const uint32_t* arow = reinterpret_cast<const uint32_t*>(src + kh * p.pitch);
+                const uint32_t win = __funnelshift_r(arow[0], arow[1], shf);   // nibble i = column ow - pw + i
+                const uint32_t ev = win & 0x0F0F0F0Fu, od = (win >> 4) & 0x0F0F0F0Fu;
+                uint32_t a[QUAD];
+                a[0] = __byte_perm(ev, od, 0x0140);    // nibbles 0 1 2
+                a[1] = __byte_perm(ev, od, 0x0514);    //         1 2 3
+                a[2] = __byte_perm(ev, od, 0x0251);    //         2 3 4
+                a[3] = __byte_perm(ev, od, 0x0625);    //         3 4 5
+                const uint4 w0 = *reinterpret_cast<const uint4*>(wsm + kh * OC);
+                const uint4 w1 = *reinterpret_cast<const uint4*>(wsm + kh * OC + 4);
+#pragma unroll
+                for (int px = 0; px < QUAD; ++px) {
+                    acc[px][0] = dp4a_u8s8(a[px], w0.x, acc[px][0]);
+                    acc[px][1] = dp4a_u8s8(a[px], w0.y, acc[px][1]);
+                    acc[px][2] = dp4a_u8s8(a[px], w0.z, acc[px][2]);
+                    acc[px][3] = dp4a_u8s8(a[px], w0.w, acc[px][3]);
+                    acc[px][4] = dp4a_u8s8(a[px], w1.x, acc[px][4]);
+                    acc[px][5] = dp4a_u8s8(a[px], w1.y, acc[px][5]);
+                    acc[px][6] = dp4a_u8s8(a[px], w1.z, acc[px][6]);
+                    acc[px][7] = dp4a_u8s8(a[px], w1.w, acc[px][7]);
+                }
+            }
+
+            uint32_t out[QUAD];
+            if (p.rq.shift >= 2) {
+                // the 32-bit form of the rounding shift (see requant())
+#pragma unroll
+                for (int px = 0; px < QUAD; ++px) {
+                    uint32_t o = 0;
+#pragma unroll
+                    for (int n = 0; n < OC; ++n) {
+                        int qv = (mulhi_add(acc[px][n], p.rq.mult, rnd) >> s) + p.rq.zo;
+                        qv = min(max(qv, p.rq.lo), p.rq.hi);
+                        o |= (uint32_t)qv << (4 * n);
+                    }
+                    out[px] = o;
+                }
+            } else {
+#pragma unroll
+                for (int px = 0; px < QUAD; ++px) {
+                    uint32_t o = 0;
+#pragma unroll
+                    for (int n = 0; n < OC; ++n) o |= requant_wide(acc[px][n], p.rq) << (4 * n);
+                    out[px] = o;
+                }
+            }
+            if (valid)
+                *reinterpret_cast<uint4*>(p.Y + (uint64_t)(mbase + (uint32_t)(QUAD * r)) * (OC / 2)) =
+                    make_uint4(out[0], out[1], out[2], out[3]);
+        }
+        release_buffer(done_bar, lane);
     }
 }
 
@@ -795,7 +966,8 @@ conv_lane_kernel(const Params p)
 // Fills the host-derived fields of the launch parameters; returns the dynamic shared
 // memory the kernel needs (0 = the layer does not fit this kernel).
 static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt,
-                         int64_t ldw, bool& expanded, bool& per_lane, bool& nibbles)
+                         int64_t ldw, const uint8_t* Y, bool& expanded, bool& per_lane, bool& nibbles,
+                         bool& quad)
 {
     if (d.OC % 8 != 0 || d.OC < 8 || d.OC > 64) return 0;
     if (d.KH > 64 || d.KW > 64 || d.stride_h > 64 || d.stride_w > 64) return 0;
@@ -811,6 +983,10 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     // copy in shared memory stays packed when image rows are whole 32-bit words
     per_lane = expanded && (d.OC == 8 || d.OC == 16) && (int64_t)d.KH * segw * d.OC <= 128;
     nibbles = per_lane && ((int64_t)d.W * d.C) % 8 == 0 && (uintptr_t)X % 4 == 0;
+    // a gray-image first layer: four pixels per lane, four times the tile
+    quad = nibbles && d.C == 1 && d.OC == 8 && d.KH == 3 && d.KW == 3 && d.stride_h == 1 &&
+           d.stride_w == 1 && p.OW % 4 == 0 && (uintptr_t)Y % 16 == 0;
+    p.tile = quad ? fused::QUAD_TILE : fused::ROWS_PER_CTA;
     int64_t unit, rowbytes, data0, pix0, pitch;
     if (nibbles) {
         const int64_t halo = ((int64_t)d.pad_w * d.C + 1) / 2;     // bytes that hold a side's halo
@@ -827,7 +1003,7 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
         pitch = (data0 + rowbytes + d.pad_w * unit + 15) / 16 * 16;
     }
     // a tile's consecutive pixels touch at most `rows` output rows in `nseg` images
-    const int64_t rows = (fused::ROWS_PER_CTA - 1 + p.OW - 1) / p.OW + 1;
+    const int64_t rows = (p.tile - 1 + p.OW - 1) / p.OW + 1;
     const int64_t nseg = (rows - 1 + p.OH - 1) / p.OH + 1;
     const int64_t slots = rows * d.stride_h + nseg * (d.KH > d.stride_h ? d.KH - d.stride_h : 0);
     const int64_t bufbytes = slots * pitch + 16;       // the slack takes the unaligned words' over-read
@@ -861,8 +1037,8 @@ bool conv_fused_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t
 {
     if ((uintptr_t)Y % 8) return false;
     fused::Params p;
-    bool expanded, per_lane, nibbles;
-    return plan_fused(p, d, X, Wt, ldw, expanded, per_lane, nibbles) != 0;
+    bool expanded, per_lane, nibbles, quad;
+    return plan_fused(p, d, X, Wt, ldw, Y, expanded, per_lane, nibbles, quad) != 0;
 }
 
 // Launches one of the kernels above as persistent CTAs: as many as are resident at
@@ -884,6 +1060,9 @@ static cudaError_t launch_kernel(FusedKernel kernel, const fused::Params& p, siz
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, fused::THREADS, smem) != cudaSuccess ||
         per_sm < 1)
         per_sm = 1;
+    // every CTA converts the weights once: with fewer than three tiles per resident CTA,
+    // launch one CTA per SM fewer (where that still leaves two)
+    if (per_sm >= 3 && tiles < 3ll * sms * per_sm) --per_sm;
     const int64_t resident = (int64_t)sms * per_sm;
     const int grid = (int)(tiles < resident ? tiles : resident);
     kernel<<<grid, fused::THREADS, smem, st>>>(p);
@@ -918,15 +1097,16 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                               cudaStream_t st)
 {
     fused::Params p;
-    bool expanded = false, per_lane = false, nibbles = false;
-    const size_t smem = plan_fused(p, d, X, Wt, ldw, expanded, per_lane, nibbles);
+    bool expanded = false, per_lane = false, nibbles = false, quad = false;
+    const size_t smem = plan_fused(p, d, X, Wt, ldw, Y, expanded, per_lane, nibbles, quad);
     if (smem == 0) return cudaErrorInvalidValue;
     p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;
     p.za = za; p.zb = zb; p.rq = rq;
     p.status = device_status_ptr();
     if (!p.status) return cudaErrorUnknown;
     if (p.M == 0) return cudaSuccess;
-    const int64_t tiles = (p.M + fused::ROWS_PER_CTA - 1) / fused::ROWS_PER_CTA;
+    const int64_t tiles = (p.M + p.tile - 1) / p.tile;
+    if (quad) return launch_kernel(fused::conv_quad_kernel, p, smem, tiles, st);
     if (per_lane) {
         // the 3x3 single-channel first layer gets its own fully unrolled instance
         if (nibbles && d.OC == 8 && d.KH == 3 && p.segw == 1)
