@@ -290,3 +290,7 @@ def pack_bt(B_kn, K: int, N: int, ldb: int | None = None) -> np.ndarray:
     Bt = np.full((N, ldb), 0xA5, np.uint8)
     _check(lib().q4ref_pack_bt(_p(B_kn), B_kn.shape[1], _p(Bt), ldb, K, N), "pack_bt")
     return Bt
+
+
+# The float boundary of a quantized layer (Eq. 1 quantizer, Eq. 4 scale-back), numpy float32.
+from .qfloat import dequantize, quant_params, quantize  # noqa: E402,F401
