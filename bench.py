@@ -264,6 +264,38 @@ def time_im2col(q4, wl, hbm_peak: float, batch: int = 4096, reps: int = 10):
             "timing": f"median of 5 x {reps} back-to-back launches"}
 
 
+def time_float_boundary(q4, wl, hbm_peak: float, n: int = 1 << 26, reps: int = 10):
+    """Device times of the float boundary on n = 64 Mi values (256 MB of floats, larger than
+    L2): Eq. 1's range pass (reads 4n bytes), its quantizing pass (reads 4n, writes n/2), and
+    Eq. 4's scale-back of an int32 matrix of the same size (reads 4n, writes 4n)."""
+    import torch
+    X = torch.from_numpy(wl.rand_floats(79, 1 << 20)).cuda().repeat(n >> 20)
+    qp = torch.zeros(2, dtype=torch.int32, device="cuda")
+    Q = torch.empty(n // 2, dtype=torch.uint8, device="cuda")
+    C = torch.randint(-(1 << 20), 1 << 20, (n,), dtype=torch.int32, device="cuda")
+    R = torch.empty(n, dtype=torch.float32, device="cuda")
+    calls = {"q4_quant_params": (lambda: q4.q4_quant_params(X, qp), 4 * n),
+             "q4_quantize": (lambda: q4.q4_quantize(X, qp, Q), 4 * n + n // 2),
+             "q4_dequantize": (lambda: q4.q4_dequantize(C, 1e-3, R), 8 * n)}
+    out = {"values": n}
+    for name, (call, nbytes) in calls.items():
+        for _ in range(3):
+            call()
+        ts = []
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                call()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / reps)
+        ms = statistics.median(ts)
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out[name] = {"ms": ms, "algorithmic_bytes": nbytes, "gbs": gbs, "frac_of_hbm": gbs / hbm_peak}
+    return out
+
+
 def run_ours(args):
     import torch
     rank, world, local = dist_env()
@@ -386,6 +418,7 @@ def run_ours(args):
     # ---- the c4 layer chain (batch 4096), outside the timed region: per-layer device times
     c4_detail = time_c4_chain(q4, wl) if world == 1 and not args.no_c4_chain else None
     im2col_detail = time_im2col(q4, wl, peaks["hbm"]) if world == 1 and not args.no_c4_chain else None
+    float_detail = time_float_boundary(q4, wl, peaks["hbm"]) if world == 1 and not args.no_c4_chain else None
 
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
     cpu_baseline = None
@@ -431,6 +464,7 @@ def run_ours(args):
             "q4_conv2d_c3_gops": conv_ops / (conv_ms * 1e-3) / 1e9,
             "c4_chain_batch4096": c4_detail,
             "q4_im2col": im2col_detail,
+            "float_boundary": float_detail,
             "hbm_peak_gbs": peaks["hbm"], "peaks": peaks["source"]},
     }
     print(json.dumps(line))

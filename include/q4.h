@@ -213,6 +213,40 @@ q4_status q4_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
                       int32_t* sums, void* stream);
 
 /*
+ * Float boundary of a quantized layer (Section II-A, Eq. 1; Section III-B, the F -> Q and
+ * Q -> F cases; Eq. 4).  All floating-point steps are IEEE binary32, correctly rounded.
+ *
+ * Reading of Eq. 1 (its zero point is printed in real units while Eq. 2 uses it in steps of
+ * the scale): scale = (max(max x, 0) - min(min x, 0)) / 15 (1 for an all-zero tensor);
+ * zero = -floor(min(min x, 0) / scale) clamped to 0..15; code = clamp(floor(x / scale) +
+ * zero, 0, 15); x ~= scale * (code - zero).  Inputs must be finite.
+ */
+typedef struct {
+    float scale;     /* s of Eq. 1 */
+    int32_t zero;    /* integer zero point, 0..15: the za / zb of q4_gemm */
+} q4_qparams;
+
+/* Derives *qp (DEVICE memory, 8 bytes, 4-byte aligned, owned by the caller) from the
+ * rows x cols float matrix X (device, row pitch ldx ELEMENTS >= cols).  Asynchronous on
+ * `stream`; the host reads *qp back (after synchronizing) to pass `zero` to q4_gemm. */
+q4_status q4_quant_params(const float* X, int64_t ldx, int32_t rows, int32_t cols,
+                          q4_qparams* qp, void* stream);
+
+/* Quantizes X with the parameters at qp (DEVICE pointer, e.g. from q4_quant_params or
+ * uploaded by the caller for a calibrated layer) into packed codes Q: row pitch ldq BYTES
+ * >= ceil(cols / 2), low nibble = even column, an odd row's last high nibble 0; bytes
+ * between ceil(cols / 2) and ldq are left untouched. */
+q4_status q4_quantize(const float* X, int64_t ldx, int32_t rows, int32_t cols,
+                      const q4_qparams* qp, uint8_t* Q, int64_t ldq, void* stream);
+
+/* Eq. 4: R[r][c] = scale * C[r][c] (int32 -> float32 round-to-nearest-even, one
+ * multiplication).  C: int32 results with zero point 0 (q4_gemm output), pitch ldc
+ * elements; R: float, pitch ldr elements; scale = s_w * s_x, or the running product of
+ * Section III-B, a host value. */
+q4_status q4_dequantize(const int32_t* C, int64_t ldc, int32_t rows, int32_t cols, float scale,
+                        float* R, int64_t ldr, void* stream);
+
+/*
  * q4_gemm with HOST operands: copies A and Bt to the device, runs q4_gemm and
  * copies C back, all on `stream`, then synchronizes it.  hA / hBt / hC are host
  * pointers with the same pitches as above (pinned memory makes the copies

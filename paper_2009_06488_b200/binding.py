@@ -34,7 +34,8 @@ EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_st
            "q4_gemm_workspace_bytes", "q4_gemm_workspace_bytes_expanded",
            "q4_conv2d_workspace_bytes", "q4_pack_bt", "q4_row_sums", "q4_gemm_host",
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
-           "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak"]
+           "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak",
+           "q4_quant_params", "q4_quantize", "q4_dequantize"]
 
 
 class Q4Error(RuntimeError):
@@ -122,6 +123,9 @@ _lib.q4_gemm_host.argtypes = [_vp, _i64, _vp, _i64, _vp, _i64, _i32, _i32, _i32,
 _lib.q4_gemm_host_staging_bytes.argtypes = [_i32, _i32, _i32, _i64, _i64, _i64]
 _lib.q4_gemm_host_staging_bytes.restype = _sz
 _lib.q4_measure_mma_peak.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, _vp, ctypes.c_int, _vp]
+_lib.q4_quant_params.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp]
+_lib.q4_quantize.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp, _i64, _vp]
+_lib.q4_dequantize.argtypes = [_vp, _i64, _i32, _i32, ctypes.c_float, _vp, _i64, _vp]
 _lib.q4_last_device_status.argtypes = [_vp]
 _lib.q4_set_variant.argtypes = [ctypes.c_int]
 _lib.q4_launch_count.restype = ctypes.c_uint64
@@ -269,6 +273,40 @@ def q4_pack_bt(B_kn, Bt, K: int, N: int):
     _check(_lib.q4_pack_bt(_ptr(B_kn), _rows(B_kn, "B_kn"), _ptr(Bt), _rows(Bt, "Bt"), K, N,
                            _stream()), "q4_pack_bt")
     return Bt
+
+
+def _pitch_elems(t, name: str) -> int:
+    if t.dim() == 1:
+        return t.numel()
+    if t.dim() != 2 or t.stride(1) != 1:
+        raise ValueError(f"{name}: expected a 2-D tensor with contiguous rows")
+    return t.stride(0)
+
+
+def q4_quant_params(X, qp):
+    """Eq. 1's scale and zero point of the float matrix X into ``qp``: a CUDA tensor of two
+    32-bit words (``torch.int32``, shape [2]; word 0 holds the scale's float bits)."""
+    _dev(X, torch.float32, "X"); _dev(qp, torch.int32, "qp")
+    rows, cols = (1, X.numel()) if X.dim() == 1 else X.shape
+    _check(_lib.q4_quant_params(_ptr(X), _pitch_elems(X, "X"), rows, cols, _ptr(qp), _stream()),
+           "q4_quant_params")
+    return qp
+
+
+def q4_quantize(X, qp, Q):
+    _dev(X, torch.float32, "X"); _dev(qp, torch.int32, "qp"); _dev(Q, torch.uint8, "Q")
+    rows, cols = (1, X.numel()) if X.dim() == 1 else X.shape
+    _check(_lib.q4_quantize(_ptr(X), _pitch_elems(X, "X"), rows, cols, _ptr(qp), _ptr(Q),
+                            _rows(Q, "Q") if Q.dim() == 2 else Q.numel(), _stream()), "q4_quantize")
+    return Q
+
+
+def q4_dequantize(C, scale: float, R):
+    _dev(C, torch.int32, "C"); _dev(R, torch.float32, "R")
+    rows, cols = (1, C.numel()) if C.dim() == 1 else C.shape
+    _check(_lib.q4_dequantize(_ptr(C), _pitch_elems(C, "C"), rows, cols, float(scale), _ptr(R),
+                              _pitch_elems(R, "R"), _stream()), "q4_dequantize")
+    return R
 
 
 def q4_row_sums(P, rows: int, K: int, sums):

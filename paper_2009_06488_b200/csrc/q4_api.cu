@@ -313,6 +313,38 @@ q4_status q4_conv2d_static(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                      (size_t)Q4_STATIC_SCRATCH_BYTES, stream);
 }
 
+q4_status q4_quant_params(const float* X, int64_t ldx, int32_t rows, int32_t cols,
+                          q4_qparams* qp, void* stream)
+{
+    if (rows < 0 || cols < 0 || ldx < cols || !qp) return Q4_ERR_INVALID_ARG;
+    if ((int64_t)rows * cols > 0 && !X) return Q4_ERR_INVALID_ARG;
+    if ((uintptr_t)X % 4 || (uintptr_t)qp % 4) return Q4_ERR_ALIGNMENT;
+    return launch_quant_params(X, ldx, rows, cols, qp, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
+q4_status q4_quantize(const float* X, int64_t ldx, int32_t rows, int32_t cols,
+                      const q4_qparams* qp, uint8_t* Q, int64_t ldq, void* stream)
+{
+    if (rows < 0 || cols < 0 || ldx < cols || ldq < (cols + 1) / 2 || !qp) return Q4_ERR_INVALID_ARG;
+    if ((int64_t)rows * cols == 0) return Q4_OK;
+    if (!X || !Q) return Q4_ERR_INVALID_ARG;
+    if ((uintptr_t)X % 4 || (uintptr_t)qp % 4) return Q4_ERR_ALIGNMENT;
+    return launch_quantize(X, ldx, rows, cols, qp, Q, ldq, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
+q4_status q4_dequantize(const int32_t* C, int64_t ldc, int32_t rows, int32_t cols, float scale,
+                        float* R, int64_t ldr, void* stream)
+{
+    if (rows < 0 || cols < 0 || ldc < cols || ldr < cols) return Q4_ERR_INVALID_ARG;
+    if ((int64_t)rows * cols == 0) return Q4_OK;
+    if (!C || !R) return Q4_ERR_INVALID_ARG;
+    if ((uintptr_t)C % 4 || (uintptr_t)R % 4) return Q4_ERR_ALIGNMENT;
+    return launch_dequantize(C, ldc, rows, cols, scale, R, ldr, static_cast<cudaStream_t>(stream)) ==
+                   cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
 q4_status q4_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int64_t ldb,
                      int32_t K, int32_t N, void* stream)
 {

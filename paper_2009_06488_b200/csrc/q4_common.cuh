@@ -130,6 +130,13 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
 cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, uint8_t* A,
                           int64_t lda, int32_t* rowsum_a, cudaStream_t st);
 
+cudaError_t launch_quant_params(const float* X, int64_t ldx, int32_t rows, int32_t cols,
+                                q4_qparams* qp, cudaStream_t st);
+cudaError_t launch_quantize(const float* X, int64_t ldx, int32_t rows, int32_t cols,
+                            const q4_qparams* qp, uint8_t* Q, int64_t ldq, cudaStream_t st);
+cudaError_t launch_dequantize(const int32_t* C, int64_t ldc, int32_t rows, int32_t cols, float scale,
+                              float* R, int64_t ldr, cudaStream_t st);
+
 void count_launch(int n = 1);
 
 }  // namespace q4

@@ -1,0 +1,126 @@
+"""GPU parity: q4_quant_params / q4_quantize / q4_dequantize against the float-boundary
+oracle.  Codes, zero points and packed bytes are compared bit for bit; the scale and the
+scaled-back floats too, because both sides use the same correctly rounded binary32
+operations in the same order (tolerance 0, stated here on purpose)."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2009_06488_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q4():
+    from paper_2009_06488_b200 import binding
+    return binding
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def params_on_gpu(q4, Xd):
+    import torch
+    qp = torch.full((2,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    q4.q4_quant_params(Xd, qp)
+    h = qp.cpu().numpy()
+    return qp, h[:1].view(np.float32)[0], int(h[1])
+
+
+SHAPES = [(1, 8), (3, 40), (7, 33), (64, 256), (5, 1001), (300, 264), (1, 1 << 20), (1025, 72)]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("kind", ["signed", "nonneg", "neg", "zeros"])
+def test_quantizer_matches_oracle(q4, shape, kind):
+    import torch
+    rows, cols = shape
+    X = wl.rand_floats(17 + rows + cols, rows * cols).reshape(rows, cols)
+    if kind == "nonneg":
+        X = np.abs(X)
+    elif kind == "neg":
+        X = -np.abs(X) - np.float32(0.125)
+    elif kind == "zeros":
+        X = np.zeros_like(X)
+    s, z = oracle.quant_params(X)
+    Xd = dev(X)
+    qp, gs, gz = params_on_gpu(q4, Xd)
+    assert gs == s and gz == z
+    kb = (cols + 1) // 2
+    for ldq in (kb, (kb + 15) // 16 * 16 + 16):
+        Q = torch.full((rows, ldq), 0xA5, dtype=torch.uint8, device="cuda")
+        q4.q4_quantize(Xd, qp, Q[:, :ldq] if ldq == kb else Q)
+        got = Q.cpu().numpy()
+        want = oracle.quantize(X, s, z, ldq)
+        assert (got[:, :kb] == want[:, :kb]).all()
+        assert (got[:, kb:] == 0xA5).all()             # bytes past the row are not touched
+
+
+def test_quantizer_on_a_strided_view(q4):
+    import torch
+    X = wl.rand_floats(5, 37 * 80).reshape(37, 80)
+    Xd = dev(X)[:, 8:72]                                # pitch 80, 64 columns, 32-byte offset
+    Xv = X[:, 8:72]
+    s, z = oracle.quant_params(Xv)
+    qp, gs, gz = params_on_gpu(q4, Xd)
+    assert (gs, gz) == (s, z)
+    Q = torch.zeros((37, 48), dtype=torch.uint8, device="cuda")
+    q4.q4_quantize(Xd, qp, Q)
+    assert (Q.cpu().numpy() == oracle.quantize(Xv, s, z, 48)).all()
+
+
+def test_caller_supplied_parameters(q4):
+    """A calibrated layer uploads its own scale and zero point; out-of-range values clamp."""
+    import torch
+    X = (wl.rand_floats(9, 4096).reshape(16, 256) * np.float32(40)).astype(np.float32)
+    s, z = np.float32(0.37), 6
+    words = np.array([np.float32(s).view(np.int32), z], dtype=np.int32)
+    Q = torch.zeros((16, 128), dtype=torch.uint8, device="cuda")
+    q4.q4_quantize(dev(X), dev(words), Q)
+    assert (Q.cpu().numpy() == oracle.quantize(X, s, z)).all()
+
+
+@pytest.mark.parametrize("shape", [(1, 4), (3, 7), (64, 64), (300, 264), (1000, 1000)])
+def test_scale_back_matches_oracle(q4, shape):
+    import torch
+    rows, cols = shape
+    rng = np.random.default_rng(rows * 131 + cols)
+    C = rng.integers(-(1 << 26), 1 << 26, size=shape).astype(np.int32)
+    C[0, 0] = (1 << 24) + 1                             # not a float32: must round, not truncate
+    scale = np.float32(3.1e-4)
+    R = torch.full((rows, cols + 4), 7.0, dtype=torch.float32, device="cuda")
+    q4.q4_dequantize(dev(C), float(scale), R[:, :cols])
+    got = R.cpu().numpy()
+    assert (got[:, :cols] == oracle.dequantize(C, scale)).all()
+    assert (got[:, cols:] == 7.0).all()
+
+
+def test_float_in_float_out_layer(q4):
+    """F -> Q -> F: quantize activations and weights, multiply with q4_gemm, scale back
+    (Section III-B), every stage equal to the oracle's."""
+    import torch
+    M, N, K = 160, 72, 200
+    Xf = wl.rand_floats(21, M * K).reshape(M, K)
+    Wf = wl.rand_floats(22, N * K).reshape(N, K) * np.float32(0.1)
+    sx, zx = oracle.quant_params(Xf)
+    sw, zw = oracle.quant_params(Wf)
+    A, Bt = oracle.quantize(Xf, sx, zx), oracle.quantize(Wf, sw, zw)
+    want = oracle.dequantize(oracle.gemm(A, Bt, M, N, K, zx, zw), np.float32(sx * sw))
+
+    Xd, Wd = dev(Xf), dev(Wf)
+    qpx, gsx, gzx = params_on_gpu(q4, Xd)
+    qpw, gsw, gzw = params_on_gpu(q4, Wd)
+    Ad = torch.empty((M, K // 2), dtype=torch.uint8, device="cuda")
+    Bd = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+    q4.q4_quantize(Xd, qpx, Ad); q4.q4_quantize(Wd, qpw, Bd)
+    C = torch.empty((M, N), dtype=torch.int32, device="cuda")
+    q4.q4_gemm(Ad, Bd, C, M, N, K, gzx, gzw)
+    R = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    q4.q4_dequantize(C, float(np.float32(gsx * gsw)), R)
+    assert (R.cpu().numpy() == want).all()
+    # and the quantized product approximates the float one (Eq. 2's "~="): loose sanity bound
+    exact = Xf.astype(np.float64) @ Wf.astype(np.float64).T
+    assert np.abs(want - exact).max() <= K * float(sx) * float(sw) * 15 * 2
