@@ -294,3 +294,6 @@ def pack_bt(B_kn, K: int, N: int, ldb: int | None = None) -> np.ndarray:
 
 # The float boundary of a quantized layer (Eq. 1 quantizer, Eq. 4 scale-back), numpy float32.
 from .qfloat import dequantize, quant_params, quantize  # noqa: E402,F401
+
+# The 8-bit product of the paper's comparison (Eq. 2 with 8-bit values), numpy int64.
+from .q8 import gemm_u8, gemm_u8_fourterm  # noqa: E402,F401
