@@ -296,6 +296,47 @@ def time_float_boundary(q4, wl, hbm_peak: float, n: int = 1 << 26, reps: int = 1
     return out
 
 
+def time_u8_comparison(q4, wl, n: int, reps: int = 10):
+    """The paper's experiment on this GPU: the 8-bit product (q4_gemm_u8, one byte per value, no
+    unpack stage) at the benchmark shape, beside it -- as context only -- the library's int8
+    GEMM (torch._int_mm, cuBLASLt) on operands of the same shape."""
+    import torch
+    ld = (n + 15) // 16 * 16
+    A = torch.from_numpy(wl.rand_bytes(n, 1, n * ld).reshape(n, ld)).cuda()
+    Bt = torch.from_numpy(wl.rand_bytes(n, 2, n * ld).reshape(n, ld)).cuda()
+    C = torch.empty((n, n), dtype=torch.int32, device="cuda")
+    ws = torch.empty(q4.q4_gemm_u8_workspace_bytes(n, n), dtype=torch.uint8, device="cuda")
+
+    def timed(call):
+        for _ in range(3):
+            call()
+        ts = []
+        for _ in range(3):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                call()
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(e0.elapsed_time(e1) / reps)
+        return statistics.median(ts)
+
+    ms = timed(lambda: q4.q4_gemm_u8(A, Bt, C, n, n, n, 3, 200, ws=ws))
+    out = {"q4_gemm_u8_ms": ms, "q4_gemm_u8_tops": 2.0 * n ** 3 / (ms * 1e-3) / 1e12,
+           "note": "zero-point sums taken by the pre-pass inside the call, as for q4_gemm"}
+    try:
+        a8 = A.view(torch.int8)[:, :n].contiguous()
+        b8 = Bt.view(torch.int8)[:, :n].t()            # column-major right operand
+        lib_ms = timed(lambda: torch._int_mm(a8, b8))
+        out["library_int8_gemm_ms"] = lib_ms
+        out["library_int8_gemm_tops"] = 2.0 * n ** 3 / (lib_ms * 1e-3) / 1e12
+        out["library_note"] = "torch._int_mm (s8 x s8 -> s32, no zero-point terms): context, not part of the path"
+    except Exception as e:                             # the library routine is optional context
+        out["library_int8_gemm_ms"] = None
+        out["library_note"] = f"torch._int_mm unavailable: {type(e).__name__}"
+    return out
+
+
 def run_ours(args):
     import torch
     rank, world, local = dist_env()
@@ -418,6 +459,7 @@ def run_ours(args):
     # ---- the c4 layer chain (batch 4096), outside the timed region: per-layer device times
     c4_detail = time_c4_chain(q4, wl) if world == 1 and not args.no_c4_chain else None
     im2col_detail = time_im2col(q4, wl, peaks["hbm"]) if world == 1 and not args.no_c4_chain else None
+    u8_detail = time_u8_comparison(q4, wl, GEMM_N) if world == 1 and not args.no_c4_chain else None
     float_detail = time_float_boundary(q4, wl, peaks["hbm"]) if world == 1 and not args.no_c4_chain else None
 
     # ---- CPU baseline: the oracle on a bounded sample (rank 0, N = 1 only)
@@ -465,6 +507,7 @@ def run_ours(args):
             "c4_chain_batch4096": c4_detail,
             "q4_im2col": im2col_detail,
             "float_boundary": float_detail,
+            "eight_bit_comparison": u8_detail,
             "hbm_peak_gbs": peaks["hbm"], "peaks": peaks["source"]},
     }
     print(json.dumps(line))
@@ -480,7 +523,20 @@ def run_case(args):
     torch.cuda.set_device(0)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     n = args.n
-    if args.case in ("gemm", "gemm_requant"):
+    if args.case == "gemm_u8":
+        ld = (n + 15) // 16 * 16
+        A = dev(wl.rand_bytes(n, 1, n * ld).reshape(n, ld))
+        Bt = dev(wl.rand_bytes(n, 2, n * ld).reshape(n, ld))
+        C = torch.empty((n, n), dtype=torch.int32, device="cuda")
+        ra = torch.empty(n, dtype=torch.int32, device="cuda")
+        cb = torch.empty(n, dtype=torch.int32, device="cuda")
+        wsg = torch.empty(q4.q4_gemm_u8_workspace_bytes(n, n), dtype=torch.uint8, device="cuda")
+        if args.presums:
+            call = lambda: q4.q4_gemm_u8(A, Bt, C, n, n, n, 3, 200, ra, cb)
+        else:
+            call = lambda: q4.q4_gemm_u8(A, Bt, C, n, n, n, 3, 200, ws=wsg)
+        units, unit = 2.0 * n ** 3 / 1e12, "TOPS"
+    elif args.case in ("gemm", "gemm_requant"):
         g = wl.c2(n) if n in (512, 1024, 2048, 4096, 8192) else wl.gemm_case("case", n, n, n, seed=n)
         A, Bt = dev(g.A), dev(g.Bt)
         C = torch.empty((n, n), dtype=torch.int32, device="cuda")
@@ -551,7 +607,7 @@ def main():
                     help="skip the per-layer timing of the c4 chain that follows the timed steps")
     ap.add_argument("--ref-seconds", type=float, default=None,
                     help="--impl reference: CPU seconds of oracle work per step (default: sized from --steps)")
-    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "conv", "im2col", "c4layer"],
+    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "gemm_u8", "conv", "im2col", "c4layer"],
                     help="profile one call in a loop instead of the benchmark step")
     ap.add_argument("--layer", type=int, default=0, help="--case c4layer: 0..4 = L1..L4, FC")
     ap.add_argument("--presums", action="store_true", help="--case gemm: pass precomputed depth sums")

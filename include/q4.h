@@ -213,6 +213,24 @@ q4_status q4_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
                       int32_t* sums, void* stream);
 
 /*
+ * The 8-bit product of the paper's comparison (Section II-B: values in 0..255 with 32-bit
+ * accumulators; the experiments of Section IV measure the 4-bit product against it):
+ *   C[m][n] = sum_k (A[m][k] - za) * (Bt[n][k] - zb),  za, zb in 0..255,
+ * evaluated as Eq. 2's four terms like q4_gemm.  A [M][lda] and Bt [N][ldb] hold one byte
+ * per value, depth-contiguous; pitches in bytes.  Tensor-core path only: A, Bt 16-byte
+ * aligned and lda, ldb multiples of 16 (Q4_ERR_ALIGNMENT otherwise); 1 <= K <= 33024 so that
+ * 255 * 255 * K fits the 32-bit accumulator (Q4_ERR_RANGE).  rowsum_a / colsum_b as in
+ * q4_gemm; when either is NULL the workspace must hold q4_gemm_u8_workspace_bytes(M, N)
+ * bytes (Q4_ERR_WORKSPACE) and the sums are taken by a pre-pass.
+ */
+q4_status q4_gemm_u8(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                     int32_t* C, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                     int32_t za, int32_t zb,
+                     const int32_t* rowsum_a, const int32_t* colsum_b,
+                     void* workspace, size_t workspace_bytes, void* stream);
+size_t q4_gemm_u8_workspace_bytes(int32_t M, int32_t N);
+
+/*
  * Float boundary of a quantized layer (Section II-A, Eq. 1; Section III-B, the F -> Q and
  * Q -> F cases; Eq. 4).  All floating-point steps are IEEE binary32, correctly rounded.
  *

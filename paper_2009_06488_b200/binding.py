@@ -35,7 +35,8 @@ EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_st
            "q4_conv2d_workspace_bytes", "q4_pack_bt", "q4_row_sums", "q4_gemm_host",
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
            "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak",
-           "q4_quant_params", "q4_quantize", "q4_dequantize"]
+           "q4_quant_params", "q4_quantize", "q4_dequantize", "q4_gemm_u8",
+           "q4_gemm_u8_workspace_bytes"]
 
 
 class Q4Error(RuntimeError):
@@ -123,6 +124,10 @@ _lib.q4_gemm_host.argtypes = [_vp, _i64, _vp, _i64, _vp, _i64, _i32, _i32, _i32,
 _lib.q4_gemm_host_staging_bytes.argtypes = [_i32, _i32, _i32, _i64, _i64, _i64]
 _lib.q4_gemm_host_staging_bytes.restype = _sz
 _lib.q4_measure_mma_peak.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_int, _vp, ctypes.c_int, _vp]
+_lib.q4_gemm_u8.argtypes = [_vp, _i64, _vp, _i64, _vp, _i64, _i32, _i32, _i32, _i32, _i32,
+                            _vp, _vp, _vp, _sz, _vp]
+_lib.q4_gemm_u8_workspace_bytes.argtypes = [_i32, _i32]
+_lib.q4_gemm_u8_workspace_bytes.restype = _sz
 _lib.q4_quant_params.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp]
 _lib.q4_quantize.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp, _i64, _vp]
 _lib.q4_dequantize.argtypes = [_vp, _i64, _i32, _i32, ctypes.c_float, _vp, _i64, _vp]
@@ -273,6 +278,25 @@ def q4_pack_bt(B_kn, Bt, K: int, N: int):
     _check(_lib.q4_pack_bt(_ptr(B_kn), _rows(B_kn, "B_kn"), _ptr(Bt), _rows(Bt, "Bt"), K, N,
                            _stream()), "q4_pack_bt")
     return Bt
+
+
+def q4_gemm_u8_workspace_bytes(M: int, N: int) -> int:
+    return int(_lib.q4_gemm_u8_workspace_bytes(M, N))
+
+
+def q4_gemm_u8(A, Bt, C, M: int, N: int, K: int, za: int, zb: int, rowsum_a=None, colsum_b=None,
+               ws=None):
+    """8-bit product (one byte per value); see include/q4.h."""
+    _dev(A, torch.uint8, "A"); _dev(Bt, torch.uint8, "Bt"); _dev(C, torch.int32, "C")
+    for t, n in ((rowsum_a, "rowsum_a"), (colsum_b, "colsum_b")):
+        if t is not None:
+            _dev(t, torch.int32, n)
+    if ws is not None:
+        _dev(ws, torch.uint8, "ws")
+    _check(_lib.q4_gemm_u8(_ptr(A), _rows(A, "A"), _ptr(Bt), _rows(Bt, "Bt"), _ptr(C), _rows(C, "C"),
+                           M, N, K, za, zb, _ptr(rowsum_a), _ptr(colsum_b), _ptr(ws),
+                           0 if ws is None else ws.numel(), _stream()), "q4_gemm_u8")
+    return C
 
 
 def _pitch_elems(t, name: str) -> int:

@@ -313,6 +313,47 @@ q4_status q4_conv2d_static(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                      (size_t)Q4_STATIC_SCRATCH_BYTES, stream);
 }
 
+size_t q4_gemm_u8_workspace_bytes(int32_t M, int32_t N)
+{
+    if (M < 0 || N < 0) return 0;
+    return round256(4 * (size_t)M) + round256(4 * (size_t)N);   // depth sums of both operands
+}
+
+q4_status q4_gemm_u8(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                     int32_t* C, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                     int32_t za, int32_t zb, const int32_t* rowsum_a, const int32_t* colsum_b,
+                     void* ws, size_t ws_bytes, void* stream)
+{
+    if (M < 0 || N < 0 || K < 1 || lda < K || ldb < K) return Q4_ERR_INVALID_ARG;
+    if (za < 0 || za > 255 || zb < 0 || zb > 255 || K > 33024) return Q4_ERR_RANGE;
+    if (M == 0 || N == 0) return Q4_OK;
+    if (!A || !Bt || !C || ldc < N) return Q4_ERR_INVALID_ARG;
+    if ((uintptr_t)A % 16 || (uintptr_t)Bt % 16 || lda % 16 || ldb % 16 || (uintptr_t)C % 4)
+        return Q4_ERR_ALIGNMENT;
+    if ((rowsum_a && (uintptr_t)rowsum_a % 4) || (colsum_b && (uintptr_t)colsum_b % 4))
+        return Q4_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    GemmParams p{};
+    p.A = A; p.Bt = Bt; p.lda = lda; p.ldb = ldb; p.M = M; p.N = N; p.K = K; p.za = za; p.zb = zb;
+    p.rowsum_a = rowsum_a; p.colsum_b = colsum_b; p.C = C; p.ldc = ldc;
+    p.status = device_status_ptr();
+    if (!p.status) return Q4_ERR_CUDA;
+    if (!rowsum_a || !colsum_b) {
+        if (!ws || (uintptr_t)ws % 4 || ws_bytes < q4_gemm_u8_workspace_bytes(M, N)) return Q4_ERR_WORKSPACE;
+        int32_t* sa = static_cast<int32_t*>(ws);
+        int32_t* sb = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + round256(4 * (size_t)M));
+        if (!rowsum_a) {
+            if (launch_byte_sums(A, lda, M, K, sa, st) != cudaSuccess) return Q4_ERR_CUDA;
+            p.rowsum_a = sa;
+        }
+        if (!colsum_b) {
+            if (launch_byte_sums(Bt, ldb, N, K, sb, st) != cudaSuccess) return Q4_ERR_CUDA;
+            p.colsum_b = sb;
+        }
+    }
+    return launch_gemm_u8(p, st);
+}
+
 q4_status q4_quant_params(const float* X, int64_t ldx, int32_t rows, int32_t cols,
                           q4_qparams* qp, void* stream)
 {

@@ -137,6 +137,10 @@ cudaError_t launch_quantize(const float* X, int64_t ldx, int32_t rows, int32_t c
 cudaError_t launch_dequantize(const int32_t* C, int64_t ldc, int32_t rows, int32_t cols, float scale,
                               float* R, int64_t ldr, cudaStream_t st);
 
+q4_status   launch_gemm_u8(const GemmParams& p, cudaStream_t st);
+cudaError_t launch_byte_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K, int32_t* sums,
+                             cudaStream_t st);
+
 void count_launch(int n = 1);
 
 }  // namespace q4

@@ -378,6 +378,22 @@ bool make_packed_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows,
                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// One-byte-per-value matrix [rows x kbytes] with pitch ld, box = 128 bytes x box_rows with
+// the 128-byte swizzle: the tile lands in the K-major layout the MMA descriptors describe.
+// Out-of-range rows and bytes are filled with zeros.
+bool make_byte_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows, int kbytes, int box_rows)
+{
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)kbytes, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld};
+    cuuint32_t box[2] = {128u, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides,
+               box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 bool gemm_tc_supported(const GemmParams& p)
 {
     return ((uintptr_t)p.A % 16 == 0) && ((uintptr_t)p.Bt % 16 == 0) && (p.lda % 16 == 0) &&
