@@ -523,7 +523,17 @@ def run_case(args):
     torch.cuda.set_device(0)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     n = args.n
-    if args.case == "gemm_u8":
+    if args.case == "quantize":
+        # Eq. 1 on an n x 4096 float matrix: range pass + quantizing pass per call
+        X = dev(wl.rand_floats(80, 1 << 20)).repeat(n * 4096 >> 20).reshape(n, 4096)
+        qp = torch.zeros(2, dtype=torch.int32, device="cuda")
+        Q = torch.empty((n, 2048), dtype=torch.uint8, device="cuda")
+
+        def call():
+            q4.q4_quant_params(X, qp)
+            q4.q4_quantize(X, qp, Q)
+        units, unit = (8 * X.numel() + Q.numel()) / 1e9, "GB/s"
+    elif args.case == "gemm_u8":
         ld = (n + 15) // 16 * 16
         A = dev(wl.rand_bytes(n, 1, n * ld).reshape(n, ld))
         Bt = dev(wl.rand_bytes(n, 2, n * ld).reshape(n, ld))
@@ -607,7 +617,7 @@ def main():
                     help="skip the per-layer timing of the c4 chain that follows the timed steps")
     ap.add_argument("--ref-seconds", type=float, default=None,
                     help="--impl reference: CPU seconds of oracle work per step (default: sized from --steps)")
-    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "gemm_u8", "conv", "im2col", "c4layer"],
+    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "gemm_u8", "quantize", "conv", "im2col", "c4layer"],
                     help="profile one call in a loop instead of the benchmark step")
     ap.add_argument("--layer", type=int, default=0, help="--case c4layer: 0..4 = L1..L4, FC")
     ap.add_argument("--presums", action="store_true", help="--case gemm: pass precomputed depth sums")
