@@ -339,10 +339,14 @@ __device__ __forceinline__ void release_buffer(uint32_t empty_bar, int lane)
 constexpr int THREADS = (WARPS + 1) * 32;
 
 
-template <int NT, bool EXP>
+// KS_T: the number of depth steps when known at compile time (packed mode only): the loop
+// over the depth unrolls and each thread keeps its tap offsets in registers; 0 = taken
+// from the parameters.
+template <int NT, bool EXP, int KS_T = 0>
 __global__ void __launch_bounds__(THREADS, NT <= 2 ? 4 : NT <= 4 ? 3 : 2)
 conv_fused_kernel(const Params p)
 {
+    static_assert(!(EXP && KS_T), "the unrolled depth loop is for the packed mode");
     extern __shared__ __align__(16) uint8_t smem[];
     constexpr int TW = EXP ? 8 : 4;                    // table entries per depth step
     constexpr int N = 8 * NT;
@@ -462,6 +466,14 @@ conv_fused_kernel(const Params p)
         }
     const int pix0 = p.pix0;
     const int yoff = (warp * ROWS_PER_WARP + g) * (N / 2) + NT * t;    // my first row within a tile
+    // my tap offset of every depth step; steps past the depth read offset 0 (any valid place:
+    // their weights are zero)
+    int dl[KS_T ? KS_T : 1];
+#pragma unroll
+    for (int j = 0; j < KS_T; ++j) {
+        const int d = tab[4 * j + t];
+        dl[j] = d < 0 ? 0 : d;
+    }
 
     // pixel indices fit 32 bits (M < 2^31, and a tile starts below M)
     const uint32_t M32 = (uint32_t)p.M, mstep = gridDim.x * (uint32_t)ROWS_PER_CTA;
@@ -531,15 +543,16 @@ conv_fused_kernel(const Params p)
 #pragma unroll
                     for (int e = 0; e < 4; ++e) acc[mt][nt][e] = colterm[nt][e & 1];   // columns 2t + e % 2
 
-            for (int j = 0; j < p.KS; ++j) {
+#pragma unroll
+            for (int j = 0; j < (KS_T ? KS_T : p.KS); ++j) {
                 uint32_t a[2][4];
                 if (!EXP) {
                     // one packed word per row: even nibbles feed depth 4t.., odd ones 16+4t..
-                    const int delta = tab[4 * j + t];
+                    const int delta = KS_T ? dl[KS_T ? j : 0] : tab[4 * j + t];
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         uint32_t w = 0;
-                        if (delta >= 0) w = *reinterpret_cast<const uint32_t*>(buf + base[i] + delta);
+                        if (KS_T || delta >= 0) w = *reinterpret_cast<const uint32_t*>(buf + base[i] + delta);
                         a[0][i] = w & 0x0F0F0F0Fu;
                         a[1][i] = (w >> 4) & 0x0F0F0F0Fu;
                     }
@@ -1073,6 +1086,16 @@ static cudaError_t launch_kernel(FusedKernel kernel, const fused::Params& p, siz
 template <int NT, bool EXP>
 static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
+    // 3x3 layers with 8, 16 or 32 input channels and twice as many outputs (and the c3 layer)
+    if constexpr (!EXP && NT == 2) {
+        if (p.KS == 3) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 3>, p, smem, tiles, st);
+    }
+    if constexpr (!EXP && NT == 4) {
+        if (p.KS == 5) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 5>, p, smem, tiles, st);
+    }
+    if constexpr (!EXP && NT == 8) {
+        if (p.KS == 9) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 9>, p, smem, tiles, st);
+    }
     return launch_kernel(fused::conv_fused_kernel<NT, EXP>, p, smem, tiles, st);
 }
 
