@@ -336,10 +336,12 @@ q4_status q4_gemm_u8(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t l
     GemmParams p{};
     p.A = A; p.Bt = Bt; p.lda = lda; p.ldb = ldb; p.M = M; p.N = N; p.K = K; p.za = za; p.zb = zb;
     p.rowsum_a = rowsum_a; p.colsum_b = colsum_b; p.C = C; p.ldc = ldc;
+    if ((!rowsum_a || !colsum_b) &&
+        (!ws || (uintptr_t)ws % 4 || ws_bytes < q4_gemm_u8_workspace_bytes(M, N)))
+        return Q4_ERR_WORKSPACE;
     p.status = device_status_ptr();
     if (!p.status) return Q4_ERR_CUDA;
     if (!rowsum_a || !colsum_b) {
-        if (!ws || (uintptr_t)ws % 4 || ws_bytes < q4_gemm_u8_workspace_bytes(M, N)) return Q4_ERR_WORKSPACE;
         int32_t* sa = static_cast<int32_t*>(ws);
         int32_t* sb = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + round256(4 * (size_t)M));
         if (!rowsum_a) {

@@ -114,3 +114,39 @@ def test_compute_call_without_a_device_fails_loudly(lib):
     lib.q4_gemm.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
     assert lib.q4_gemm(0x1000, 64, 0x1000, 64, 0x1000, 8, 8, 8, 128, 0, 0, None, None, None, 0,
                        None) == 6   # Q4_ERR_CUDA: no silent CPU path
+
+
+def test_validation_of_the_float_boundary_and_the_8bit_product(lib):
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    fake = 0x1000
+    INVALID, ALIGN, RANGE, WORKSPACE = 1, 2, 3, 4
+    lib.q4_gemm_u8.argtypes = [vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, i32, vp, vp, vp, sz, vp]
+    lib.q4_gemm_u8_workspace_bytes.argtypes = [i32, i32]
+    lib.q4_gemm_u8_workspace_bytes.restype = sz
+    u = lambda **kw: lib.q4_gemm_u8(kw.get("A", fake), kw.get("lda", 128), fake, 128, kw.get("C", fake), 8,
+                                    kw.get("M", 8), 8, kw.get("K", 128), kw.get("za", 0), kw.get("zb", 0),
+                                    kw.get("ra", fake), kw.get("cb", fake), kw.get("ws"), kw.get("wsb", 0), None)
+    assert u(K=0) == INVALID and u(M=-1) == INVALID and u(A=None) == INVALID
+    assert u(lda=127) == INVALID                     # pitch shorter than a row
+    assert u(za=256) == RANGE and u(zb=-1) == RANGE
+    assert u(K=33025, lda=33040) == INVALID          # ldb (128) is shorter than the row
+    assert lib.q4_gemm_u8(fake, 33040, fake, 33040, fake, 8, 8, 8, 33025, 0, 0, fake, fake, None, 0, None) == RANGE
+    assert u(A=fake + 8) == ALIGN and u(lda=136) == ALIGN and u(C=fake + 2) == ALIGN
+    assert u(ra=None) == WORKSPACE                   # sums wanted, no workspace given
+    assert u(ra=None, ws=0x2000, wsb=lib.q4_gemm_u8_workspace_bytes(8, 8) - 1) == WORKSPACE
+    assert u(M=0) == 0
+    assert lib.q4_gemm_u8_workspace_bytes(1000, 10) >= 4 * 1010
+
+    lib.q4_quant_params.argtypes = [vp, i64, i32, i32, vp, vp]
+    lib.q4_quantize.argtypes = [vp, i64, i32, i32, vp, vp, i64, vp]
+    lib.q4_dequantize.argtypes = [vp, i64, i32, i32, ctypes.c_float, vp, i64, vp]
+    assert lib.q4_quant_params(fake, 7, 4, 8, fake, None) == INVALID       # pitch shorter than a row
+    assert lib.q4_quant_params(fake, 8, 4, 8, None, None) == INVALID
+    assert lib.q4_quant_params(fake + 2, 8, 4, 8, fake, None) == ALIGN
+    assert lib.q4_quantize(fake, 8, 4, 8, fake, fake, 3, None) == INVALID  # 8 codes need 4 bytes
+    assert lib.q4_quantize(fake, 8, 4, 9, fake, fake, 4, None) == INVALID  # 9 codes need 5 bytes
+    assert lib.q4_quantize(fake, 8, 0, 8, fake, fake, 4, None) == 0        # empty: no-op
+    assert lib.q4_quantize(None, 8, 4, 8, fake, fake, 4, None) == INVALID
+    assert lib.q4_dequantize(fake, 7, 4, 8, 1.0, fake, 8, None) == INVALID
+    assert lib.q4_dequantize(fake, 8, 4, 8, 1.0, fake + 1, 8, None) == ALIGN
+    assert lib.q4_dequantize(fake, 8, 4, 0, 1.0, fake, 8, None) == 0
