@@ -124,3 +124,58 @@ def test_float_in_float_out_layer(q4):
     # and the quantized product approximates the float one (Eq. 2's "~="): loose sanity bound
     exact = Xf.astype(np.float64) @ Wf.astype(np.float64).T
     assert np.abs(want - exact).max() <= K * float(sx) * float(sw) * 15 * 2
+
+
+def test_float_image_through_the_table2_layers_and_back_to_float(q4):
+    """The layer model of Section III-B on the Table II topology with random weights: a float
+    image is quantized (F -> Q), five layers hand 4-bit activations to the next (Q -> Q, with
+    the fused integer re-quantization), and the last convolution's integer result is scaled
+    back to float (Q -> F).  Every stage equals the oracle's."""
+    import dataclasses
+    import torch
+    net = wl.paper_table2_net(batch=5)
+    L0 = net.layers[0]
+    img = np.abs(wl.rand_floats(31, L0.N * L0.H * L0.W)).reshape(L0.N * L0.H, L0.W)
+    s_x, z_x = oracle.quant_params(img)
+    assert z_x == 0                                      # non-negative image
+    layers = [dataclasses.replace(L0, za=z_x)] + net.layers[1:]
+    s_total = np.float32(s_x * np.float32(0.01))         # stand-in for the product of the layers' scales
+
+    # ---- oracle
+    Xo = oracle.quantize(img.reshape(1, -1), s_x, z_x).reshape(-1)
+    for L in layers[:-1]:
+        Xo = oracle_layer(L, Xo).reshape(-1)
+    LL = layers[-1]
+    do = oracle.ConvDesc(LL.N, LL.H, LL.W, LL.C, LL.OC, LL.KH, LL.KW, LL.stride, LL.stride, LL.pad, LL.pad)
+    lda = (LL.K // 2 + 15) // 16 * 16
+    Ao, _ = oracle.im2col(Xo, do, LL.za, lda)
+    want = oracle.dequantize(oracle.gemm(Ao, LL.Wt, LL.M, LL.OC, LL.K, LL.za, LL.zb), s_total)
+
+    # ---- GPU
+    imgd = dev(img)
+    qp, gs, gz = params_on_gpu(q4, imgd)
+    assert (gs, gz) == (s_x, z_x)
+    Xd = torch.zeros((img.size + 1) // 2 + 16, dtype=torch.uint8, device="cuda")
+    q4.q4_quantize(imgd.reshape(-1), qp, Xd)
+    for L in layers[:-1]:
+        d = q4.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
+        ws = torch.empty(q4.q4_conv2d_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+        Y = torch.zeros((d.M, L.OC // 2), dtype=torch.uint8, device="cuda")
+        q4.q4_conv2d(Xd, dev(L.Wt), d, L.za, L.zb,
+                     q4.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi), Y, ws)
+        Xd = Y.reshape(-1)
+    d = q4.ConvDesc(LL.N, LL.H, LL.W, LL.C, LL.OC, LL.KH, LL.KW, LL.stride, LL.stride, LL.pad, LL.pad)
+    A = torch.zeros((d.M, lda), dtype=torch.uint8, device="cuda")
+    q4.q4_im2col(Xd, d, LL.za, A, None)
+    C = torch.empty((d.M, LL.OC), dtype=torch.int32, device="cuda")
+    q4.q4_gemm(A, dev(LL.Wt), C, d.M, LL.OC, d.K, LL.za, LL.zb)
+    R = torch.empty((d.M, LL.OC), dtype=torch.float32, device="cuda")
+    q4.q4_dequantize(C, float(s_total), R)
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    assert (R.cpu().numpy() == want).all()
+
+
+def oracle_layer(L, X):
+    do = oracle.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
+    return oracle.conv2d(X, L.Wt, L.bias, do, L.za, L.zb,
+                         oracle.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi))
