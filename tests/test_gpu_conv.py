@@ -164,6 +164,11 @@ FUSED = [  # N, H, W, C, OC, KH, KW, sh, sw, ph, pw, byte offset of X, shift
     (700, 1, 1, 8, 8, 1, 1, 1, 1, 0, 0, 0, 5),      # one pixel per image
     (2, 20, 40, 32, 64, 3, 3, 1, 1, 1, 1, 0, 7),    # widest tile the MMA kernel has
     (1, 30, 300, 8, 8, 1, 7, 1, 2, 0, 3, 0, 5),     # long rows: a tile inside one output row
+    (9, 48, 48, 1, 8, 3, 3, 1, 1, 1, 1, 0, 1),      # four pixels per lane: tiles over two images, shift < 2
+    (4, 20, 32, 1, 8, 3, 3, 1, 1, 1, 1, 0, 5),      # ... rows copied by bulk copies (16-byte rows)
+    (6, 10, 24, 1, 8, 3, 3, 1, 1, 0, 1, 0, 9),      # ... no vertical padding
+    (3, 16, 40, 1, 8, 3, 3, 1, 1, 1, 3, 0, 5),      # ... horizontal padding of three
+    (5, 12, 20, 1, 8, 3, 3, 1, 1, 0, 0, 0, 5),      # output rows not groups of four: pixel per lane
 ]
 
 
