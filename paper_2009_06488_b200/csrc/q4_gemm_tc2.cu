@@ -624,6 +624,12 @@ static bool make_b8_map(CUtensorMap* tm, const uint8_t* base, int64_t ld8, int r
               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same map for other translation units.
+bool make_c32_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, int cols)
+{
+    return make_c_map(tm, base, ldc, rows, cols);
+}
+
 q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8,
                               int64_t ld8)
 {

@@ -266,4 +266,26 @@ __device__ __forceinline__ void tc_mma_i8_pair_ts(uint32_t d_tmem, uint32_t a_tm
         ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// ---- loads of a CTA pair that report to the leader CTA --------------------------------
+// TMA load into this CTA's shared memory whose byte count is reported to an mbarrier given
+// by its cluster address -- with cta_group::2 that barrier may live in the peer CTA of the
+// pair.  No multicast: each CTA loads its own tile.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, int x, int y,
+                                                 uint32_t cluster_bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(cluster_bar) : "memory");
+}
+// One arrival plus `bytes` expected bytes on a barrier given by its cluster address.
+// Relaxed: the announcing thread has written nothing that the waiter reads (the bytes come
+// from the copy engine), and the releasing form would first wait for the thread's earlier
+// loads in flight -- one round trip to memory per stage.
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.relaxed.cluster.shared::cluster.b64 _, [%0], %1;"
+                 ::"r"(cluster_bar), "r"(bytes) : "memory");
+}
+
 }  // namespace q4

@@ -247,6 +247,221 @@ byte_sums_kernel(const uint8_t* __restrict__ P, int64_t ld, int32_t rows, int32_
 
 }  // namespace u8
 
+// ---------------------------------------------------------------------------------------
+// CTA pairs (clusters of two, tcgen05.mma.cta_group::2): 256 x 256 output tiles, each CTA
+// staging its own 128 rows of A and its own 128 rows of Bt, so a byte of an operand tile is
+// brought from L2 once per pair instead of once per CTA.  Both CTAs' TMA loads report to
+// the LEADER's "stage landed" barrier (cta_group::2 loads, no multicast; each CTA also
+// announces its byte count there), so the leader's MMA thread waits on one local barrier
+// and no relay is needed; its commits arrive on both CTAs' "stage free" and "accumulator
+// full" barriers.  The peer's epilogue warps report "accumulator drained" directly to the
+// leader.  int32 tiles leave through a swizzled staging tile and TMA stores.
+// ---------------------------------------------------------------------------------------
+namespace u8p {
+
+constexpr int TMC = 128;             // rows of A per CTA
+constexpr int BNC = 256;             // columns of the pair tile
+constexpr int BH = BNC / 2;          // rows of Bt staged per CTA
+constexpr int ROWB = 128;            // bytes (= depth values) per row per stage
+constexpr int STAGES = 6;
+constexpr int STAGE = (TMC + BH) * ROWB;          // 32 KB per CTA
+constexpr int NTHREADS = 6 * 32;
+constexpr int TMEM_COLS = 512;       // two accumulators of 256 columns
+constexpr int OFF_STG = STAGES * STAGE;           // int32 epilogue staging: 4 warps x 32 rows x 128 B
+constexpr int STG_BYTES = 4 * 32 * 128;
+constexpr int OFF_COLTERM = OFF_STG + STG_BYTES;
+constexpr int OFF_BAR = OFF_COLTERM + BNC * 4;
+constexpr int NBAR = 2 * STAGES + 4;
+constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
+constexpr int SMEM = OFF_MISC + 16 + 1024;
+static_assert(STAGE % 1024 == 0 && OFF_STG % 1024 == 0, "stage and staging alignment");
+
+// D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC.
+constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)(BNC >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+
+struct Params {
+    GemmParams g;
+    int32_t tiles_m, tiles_n, nslab;
+    int32_t c_tma;                   // int32 output goes out through TMA stores (tmC is valid)
+};
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+gemm_u8_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmC, const Params p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    // the same offset in both CTAs: dynamic shared memory starts at the same address
+    const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t colterm_s = sbase + OFF_COLTERM;  // int32 [BNC]
+    const uint32_t bar0 = sbase + OFF_BAR;
+    auto bar_full   = [&](int s) { return bar0 + 8u * (uint32_t)s; };                  // used in the leader
+    auto bar_empty  = [&](int s) { return bar0 + 8u * (uint32_t)(STAGES + s); };
+    auto bar_tfull  = [&](int a) { return bar0 + 8u * (uint32_t)(2 * STAGES + a); };
+    auto bar_tempty = [&](int a) { return bar0 + 8u * (uint32_t)(2 * STAGES + 2 + a); };  // used in the leader
+    const uint32_t tmem_slot = sbase + OFF_MISC;
+    const uint32_t abort_flag = sbase + OFF_MISC + 4;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int cluster_id = blockIdx.x >> 1, nclusters = gridDim.x >> 1;
+    const GemmParams& g = p.g;
+    const int ntiles = p.tiles_m * p.tiles_n;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full(s), 2);       // one announcement per CTA's producer
+            mbar_init(bar_empty(s), 1);      // the leader's commit
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull(a), 1);
+            mbar_init(bar_tempty(a), 8);     // four epilogue warps of each CTA
+        }
+        sts32(abort_flag, 0);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(tmem_slot), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    cluster_sync_all();              // barriers of both CTAs are initialised past this point
+    tc_fence_after();
+    const uint32_t tmem_base = (uint32_t)lds32(tmem_slot);
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            const uint32_t full_leader = map_to_cta(bar_full(0), 0);
+            uint32_t it = 0;
+            for (int tile = cluster_id; tile < ntiles; tile += nclusters) {
+                const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+                const int arow = tm * 256 + (int)rank * TMC;
+                const int brow = tn * BNC + (int)rank * BH;
+                for (int s = 0; s < p.nslab; ++s, ++it) {
+                    const int st = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    mbar_wait_cl(bar_empty(st), ph ^ 1u, abort_flag, g.status);
+                    const uint32_t full = full_leader + 8u * (uint32_t)st;
+                    mbar_expect_tx_cluster(full, (uint32_t)STAGE);
+                    const uint32_t dst = sbase + st * STAGE;
+                    tma_load_2d_pair(dst, &tmA, s * ROWB, arow, full);
+                    tma_load_2d_pair(dst + TMC * ROWB, &tmB, s * ROWB, brow, full);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ pair MMA issuer (leader)
+        if (rank == 0 && lane == 0) {
+            uint32_t it = 0, lt = 0;
+            for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
+                const int acc = lt & 1;
+                const uint32_t aph = (lt >> 1) & 1u;
+                mbar_wait_cl(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BNC);
+                for (int s = 0; s < p.nslab; ++s, ++it) {
+                    const int st = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    mbar_wait_cl(bar_full(st), ph, abort_flag, g.status);
+                    tc_fence_after();
+                    const uint32_t ua = sbase + st * STAGE;
+                    const uint64_t adesc = make_kmajor_sw128_desc(ua);
+                    const uint64_t bdesc = make_kmajor_sw128_desc(ua + TMC * ROWB);
+                    const int rem = g.K - s * ROWB;
+                    const int ksteps = rem >= ROWB ? 4 : (rem + 31) / 32;
+                    for (int i = 0; i < ksteps; ++i)
+                        tc_mma_i8_pair(d_tmem, adesc + (uint64_t)(2 * i), bdesc + (uint64_t)(2 * i), kIdesc,
+                                       (s > 0 || i > 0) ? 1u : 0u);
+                    tc_commit_pair(bar_empty(st), 3);
+                }
+                tc_commit_pair(bar_tfull(acc), 3);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int lg = warp & 3;
+        const int row = lg * 32 + lane;
+        const int et = threadIdx.x - 64;
+        const int kzz = g.K * g.za * g.zb;
+        const uint32_t tempty_leader = map_to_cta(bar_tempty(0), 0);
+        uint32_t lt = 0;
+        for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
+            const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+            const int acc = lt & 1;
+            const uint32_t aph = (lt >> 1) & 1u;
+            const int m = tm * 256 + (int)rank * TMC + row;
+            const int n0 = tn * BNC;
+            for (int j = et; j < BNC; j += 128) {
+                const int n = n0 + j;
+                const int cb = n < g.N ? g.colsum_b[n] : 0;
+                sts32(colterm_s + 4 * j, (int)((uint32_t)kzz - (uint32_t)(g.za * cb)));
+            }
+            const int ra = m < g.M ? g.rowsum_a[m] : 0;
+            const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+
+            mbar_wait_cl(bar_tfull(acc), aph, abort_flag, g.status);
+            tc_fence_after();
+            const uint32_t taddr0 = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(acc * BNC);
+#pragma unroll 1
+            for (int ch = 0; ch < BNC / 32; ++ch) {
+                const int nc = n0 + ch * 32;
+                if (nc >= g.N) break;             // warp-uniform
+                uint32_t r[32];
+                tc_ld32(taddr0 + (uint32_t)(ch * 32), r);
+                tc_wait_ld();
+#pragma unroll
+                for (int qd = 0; qd < 8; ++qd) {
+                    const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
+                    r[4 * qd + 0] += rowterm + ct.x;
+                    r[4 * qd + 1] += rowterm + ct.y;
+                    r[4 * qd + 2] += rowterm + ct.z;
+                    r[4 * qd + 3] += rowterm + ct.w;
+                }
+                if (p.c_tma) {
+                    // my row's 128 bytes go to the swizzled staging slice of my warp; rows and
+                    // columns past M / N are clipped by the tensor map
+                    const uint32_t slice = sbase + OFF_STG + (uint32_t)(lg * 4096);
+                    if (lane == 0) bulk_wait_read();       // the previous store has read the slice
+                    __syncwarp();
+#pragma unroll
+                    for (int qd = 0; qd < 8; ++qd)
+                        sts128(slice + (uint32_t)(lane * 128 + ((qd ^ (lane & 7)) << 4)),
+                               make_uint4(r[4 * qd], r[4 * qd + 1], r[4 * qd + 2], r[4 * qd + 3]));
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_2d(&tmC, slice, nc, tm * 256 + (int)rank * TMC + lg * 32);
+                        bulk_commit();
+                    }
+                } else if (m < g.M) {
+                    int32_t* dst = g.C + (int64_t)m * g.ldc + nc;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (nc + j < g.N) dst[j] = (int32_t)r[j];
+                }
+            }
+            tc_fence_before();
+            __syncwarp();                          // every lane's tensor-memory loads are done
+            if (lane == 0) mbar_arrive_cluster(tempty_leader + 8u * (uint32_t)acc);
+            asm volatile("bar.sync 1, 128;" ::: "memory");   // colterm_s is rewritten next tile
+        }
+        if (p.c_tma && lane == 0) bulk_wait_all();   // my TMA stores are complete
+    }
+
+    tc_fence_before();
+    cluster_sync_all();          // no CTA leaves (or frees TMEM) while its peer may still use it
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace u8p
+
 static int sm_count_u8()
 {
     int dev = 0, n = 0;
@@ -293,8 +508,52 @@ static q4_status launch_u8_bn(const GemmParams& g, cudaStream_t st)
     return cudaGetLastError() == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
+bool make_c32_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, int cols);
+
+static q4_status launch_u8_pair(const GemmParams& g, cudaStream_t st)
+{
+    u8p::Params p;
+    p.g = g;
+    p.tiles_m = (g.M + 255) / 256;
+    p.tiles_n = (g.N + u8p::BNC - 1) / u8p::BNC;
+    p.nslab = (g.K + u8p::ROWB - 1) / u8p::ROWB;
+    CUtensorMap tmA, tmB, tmC{};
+    if (!make_byte_map(&tmA, g.A, g.lda, g.M, g.K, u8p::TMC)) return Q4_ERR_CUDA;
+    if (!make_byte_map(&tmB, g.Bt, g.ldb, g.N, g.K, u8p::BH)) return Q4_ERR_CUDA;
+    p.c_tma = 0;
+    if ((uintptr_t)g.C % 16 == 0 && g.ldc % 4 == 0) {
+        if (!make_c32_map(&tmC, g.C, g.ldc, g.M, g.N)) return Q4_ERR_CUDA;
+        p.c_tma = 1;
+    }
+    if (cudaFuncSetAttribute(u8p::gemm_u8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             u8p::SMEM) != cudaSuccess)
+        return Q4_ERR_CUDA;
+    const long long tiles = (long long)p.tiles_m * p.tiles_n;
+    const int max_clusters = sm_count_u8() / 2;
+    const long long clusters = tiles < max_clusters ? tiles : max_clusters;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)(2 * clusters));
+    cfg.blockDim = dim3(u8p::NTHREADS);
+    cfg.dynamicSmemBytes = u8p::SMEM;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, u8p::gemm_u8_pair_kernel, tmA, tmB, tmC, p);
+    count_launch();
+    return e == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
 q4_status launch_gemm_u8(const GemmParams& g, cudaStream_t st)
 {
+    // large problems: CTA pairs on 256 x 256 tiles (at least one tile per pair of SMs)
+    if (g.M >= 256 && g.N >= 256 &&
+        (long long)((g.M + 255) / 256) * ((g.N + 255) / 256) >= sm_count_u8() / 2)
+        return launch_u8_pair(g, st);
     if (g.N > 128) return launch_u8_bn<256>(g, st);
     if (g.N > 64)  return launch_u8_bn<128>(g, st);
     return launch_u8_bn<64>(g, st);

@@ -51,7 +51,9 @@ def run(q4, A, Bt, M, N, K, za, zb, sums=False, ldc_pad=0):
 
 
 SHAPES = [(1, 1, 1), (64, 64, 256), (130, 70, 100), (128, 256, 128), (300, 264, 1000), (257, 129, 33),
-          (1000, 520, 777), (384, 1024, 4096), (5, 300, 33024)]
+          (1000, 520, 777), (384, 1024, 4096), (5, 300, 33024),
+          # at least 74 tiles of 256 x 256: the CTA-pair kernel, ragged in every dimension
+          (2321, 2344, 200), (2560, 2304, 640), (4100, 1290, 96)]
 
 
 @pytest.mark.parametrize("shape", SHAPES)
