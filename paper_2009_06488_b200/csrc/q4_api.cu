@@ -75,7 +75,11 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
     p.status = status_ptr();
     if (!p.status) return Q4_ERR_CUDA;
     const int v = variant();
-    if (v != 1 && v != 3 && gemm_tc_pair_supported(p)) {
+    // The CTA-pair kernel pays off from about two waves of its 256 x 192 tiles (74 pairs);
+    // below that the single-CTA kernel, with narrower tiles and its sums taken in the
+    // kernel, finishes sooner.  Variant 2 always takes the pair kernel where it applies.
+    const long long pair_tiles = ((long long)p.M + 255) / 256 * (((long long)p.N + 191) / 192);
+    if (v != 1 && v != 3 && gemm_tc_pair_supported(p) && (v == 2 || pair_tiles >= 148)) {
         // Large problems use the workspace, if given, for work that is better done once per
         // call than once per output tile: the depth sums, and -- with the full size -- the
         // expansion of Bt to bytes.  A smaller workspace still takes the sums; without one

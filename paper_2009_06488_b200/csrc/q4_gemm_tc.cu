@@ -457,9 +457,13 @@ static q4_status launch_bn(const GemmParams& g, bool rq, cudaStream_t st)
 
 q4_status launch_gemm_tc(const GemmParams& g, bool rq, cudaStream_t st)
 {
-    if (g.N > 128) return launch_bn<256>(g, rq, st);
-    if (g.N > 64)  return launch_bn<128>(g, rq, st);
-    if (g.N > 32)  return launch_bn<64>(g, rq, st);
+    int bn = g.N > 128 ? 256 : g.N > 64 ? 128 : g.N > 32 ? 64 : 32;
+    // a grid that would leave more than a quarter of the SMs idle: narrower tiles, more CTAs
+    const long long rows = (g.M + TM - 1) / TM;
+    while (bn > 32 && rows * ((g.N + bn - 1) / bn) * 4 < 3LL * sm_count()) bn >>= 1;
+    if (bn == 256) return launch_bn<256>(g, rq, st);
+    if (bn == 128) return launch_bn<128>(g, rq, st);
+    if (bn == 64)  return launch_bn<64>(g, rq, st);
     return launch_bn<32>(g, rq, st);
 }
 
