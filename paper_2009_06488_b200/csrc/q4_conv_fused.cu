@@ -342,11 +342,17 @@ constexpr int THREADS = (WARPS + 1) * 32;
 // KS_T: the number of depth steps when known at compile time (packed mode only): the loop
 // over the depth unrolls and each thread keeps its tap offsets in registers; 0 = taken
 // from the parameters.
-template <int NT, bool EXP, int KS_T = 0>
+// CONSEC (with KS_T; output rows are whole groups of four pixels): the four MMA rows a thread
+// feeds and reads back (g, g + 8, g + 16, g + 24 of its warp's two 16-row tiles) are assigned
+// to four CONSECUTIVE pixels 4g .. 4g + 3 instead of pixels eight apart -- which pixel an MMA
+// row stands for is free --, so a thread decodes one pixel per tile and the other three are
+// a constant step away.
+template <int NT, bool EXP, int KS_T = 0, bool CONSEC = false>
 __global__ void __launch_bounds__(THREADS, NT <= 2 ? 4 : NT <= 4 ? 3 : 2)
 conv_fused_kernel(const Params p)
 {
     static_assert(!(EXP && KS_T), "the unrolled depth loop is for the packed mode");
+    static_assert(!CONSEC || KS_T, "consecutive pixels per thread come with the unrolled depth loop");
     extern __shared__ __align__(16) uint8_t smem[];
     constexpr int TW = EXP ? 8 : 4;                    // table entries per depth step
     constexpr int N = 8 * NT;
@@ -465,7 +471,7 @@ conv_fused_kernel(const Params p)
                                    (uint32_t)(p.bias ? p.bias[n] : 0));
         }
     const int pix0 = p.pix0;
-    const int yoff = (warp * ROWS_PER_WARP + g) * (N / 2) + NT * t;    // my first row within a tile
+    const int yoff = (warp * ROWS_PER_WARP + (CONSEC ? 4 * g : g)) * (N / 2) + NT * t;    // my first row within a tile
     // my tap offset of every depth step; steps past the depth read offset 0 (any valid place:
     // their weights are zero)
     int dl[KS_T ? KS_T : 1];
@@ -492,7 +498,25 @@ conv_fused_kernel(const Params p)
         if (myrows > 0) {                              // warp-uniform
             // my four rows: g, g+8 (first 16-row tile), 16+g, 24+g (second)
             int base[4], shf[4];
-            {
+            if (CONSEC) {
+                // pixels 4g .. 4g + 3 of my warp: same output row (rows are whole groups of four,
+                // so the tile's pixel count, a multiple of four, is reached group-wise)
+                const uint32_t mm = mbase + (uint32_t)(warp * ROWS_PER_WARP) +
+                                    (uint32_t)(4 * g < myrows ? 4 * g : 0);
+                const uint32_t q = fdiv(mm, p.div_ow);
+                const int ow = (int)(mm - q * (uint32_t)p.OW);
+                const uint32_t n0 = fdiv(q, p.div_oh);
+                const int oh = (int)(q - n0 * (uint32_t)p.OH);
+                const int seg = (int)n0 - gv.x;
+                const int slot0 = seg == 0 ? (oh - gv.y) * p.sh : gv.z + (seg - 1) * p.sfull + oh * p.sh;
+                const int b = slot0 * p.pitch + pix0 + ow * p.sw * p.unit;
+                const int step = p.step8 >> 3;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    shf[i] = 0;
+                    base[i] = b + i * step;
+                }
+            } else {
                 const uint32_t mm = mbase + (uint32_t)(warp * ROWS_PER_WARP) +
                                     (uint32_t)(g < myrows ? g : 0);
                 const uint32_t q = fdiv(mm, p.div_ow);
@@ -589,7 +613,7 @@ conv_fused_kernel(const Params p)
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int mt = i >> 1, hrow = i & 1;
-                    if (g + 8 * i >= myrows) continue;
+                    if ((CONSEC ? 4 * g + i : g + 8 * i) >= myrows) continue;
                     uint32_t bytes[NT];
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
@@ -607,7 +631,7 @@ conv_fused_kernel(const Params p)
                         }
                         bytes[nt] = qv[0] | (qv[1] << 4);
                     }
-                    uint8_t* dst = ytile + i * (8 * (N / 2));
+                    uint8_t* dst = ytile + (CONSEC ? i : 8 * i) * (N / 2);
                     if (NT % 4 == 0) {
 #pragma unroll
                         for (int q = 0; q < NT / 4; ++q)
@@ -1087,14 +1111,13 @@ template <int NT, bool EXP>
 static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
     // 3x3 layers with 8, 16 or 32 input channels and twice as many outputs (and the c3 layer)
-    if constexpr (!EXP && NT == 2) {
-        if (p.KS == 3) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 3>, p, smem, tiles, st);
-    }
-    if constexpr (!EXP && NT == 4) {
-        if (p.KS == 5) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 5>, p, smem, tiles, st);
-    }
-    if constexpr (!EXP && NT == 8) {
-        if (p.KS == 9) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 9>, p, smem, tiles, st);
+    constexpr int KS_OF_NT = NT == 2 ? 3 : NT == 4 ? 5 : NT == 8 ? 9 : 0;
+    if constexpr (!EXP && KS_OF_NT != 0) {
+        if (p.KS == KS_OF_NT) {
+            if (p.OW % 4 == 0)
+                return launch_kernel(fused::conv_fused_kernel<NT, EXP, KS_OF_NT, true>, p, smem, tiles, st);
+            return launch_kernel(fused::conv_fused_kernel<NT, EXP, KS_OF_NT, false>, p, smem, tiles, st);
+        }
     }
     return launch_kernel(fused::conv_fused_kernel<NT, EXP>, p, smem, tiles, st);
 }
