@@ -134,6 +134,14 @@ __device__ __forceinline__ int mulhi_add(int a, int b, int c)
     return d;
 }
 
+// a * b + c in one instruction (the compiler otherwise splits a shift-and-or into two).
+__device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 __device__ __forceinline__ uint32_t weight_nibble(const Params& p, int n, int k)
 {
     const uint8_t byte = p.Wt[(int64_t)n * p.ldw + (k >> 1)];
@@ -302,7 +310,7 @@ __device__ __forceinline__ void producer_loop(const Params& p, int mytiles, uint
     uint32_t round = 0;                                // j / NB
     for (int j = 0; j < mytiles + LOOK; ++j) {
         if (j < mytiles) {
-            if (round > 0) mbar_wait(empty0 + 8 * b, (round - 1) & 1, abort_flag, p.status);
+            if (round > 0) mbar_wait_suspend(empty0 + 8 * b, (round - 1) & 1, abort_flag, p.status);
             const Geo gn = tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
             if (lane == 0) geo_s[b] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
             uint8_t* buf = buf0 + b * p.bufbytes;
@@ -488,7 +496,7 @@ conv_fused_kernel(const Params p)
     uint32_t phase = 0;                                // (k / NB) % 2
     for (int k = 0; k < mytiles; ++k, mbase += mstep) {
         const uint8_t* buf = buf0 + kb * p.bufbytes;
-        mbar_wait(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
+        mbar_wait_suspend(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
         const int4 gv = geo_s[kb];                     // n_first, oh_first, s0 (published with the tile)
         const uint32_t done_bar = empty0 + 8 * kb;
         if (++kb == NB) { kb = 0; phase ^= 1; }
@@ -747,7 +755,7 @@ conv_lane_kernel(const Params p)
     uint32_t phase = 0;                                // (k / NB) % 2
     for (int k = 0; k < mytiles; ++k, mbase += mstep) {
         const uint8_t* buf = buf0 + kb * p.bufbytes;
-        mbar_wait(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
+        mbar_wait_suspend(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
         const int4 gv = geo_s[kb];                     // n_first, oh_first, s0 (published with the tile)
         const uint32_t done_bar = empty0 + 8 * kb;
         if (++kb == NB) { kb = 0; phase ^= 1; }
@@ -913,7 +921,7 @@ conv_quad_kernel(const Params p)
     uint32_t phase = 0;                                // (k / NB) % 2
     for (int k = 0; k < mytiles; ++k, mbase += mstep) {
         const uint8_t* buf = buf0 + kb * p.bufbytes;
-        mbar_wait(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
+        mbar_wait_suspend(full0 + 8 * kb, phase, abort_flag, p.status);    // the tile's rows have landed
         const int4 gv = geo_s[kb];                     // n_first, oh_first, s0 (published with the tile)
         const uint32_t done_bar = empty0 + 8 * kb;
         if (++kb == NB) { kb = 0; phase ^= 1; }
@@ -977,7 +985,7 @@ conv_quad_kernel(const Params p)
                     for (int n = 0; n < OC; ++n) {
                         int qv = (mulhi_add(acc[px][n], p.rq.mult, rnd) >> s) + p.rq.zo;
                         qv = min(max(qv, p.rq.lo), p.rq.hi);
-                        o |= (uint32_t)qv << (4 * n);
+                        o = n == 0 ? (uint32_t)qv : mad_u32((uint32_t)qv, 1u << (4 * n), o);   // nibble fields do not overlap
                     }
                     out[px] = o;
                 }

@@ -87,6 +87,37 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_
     }
     return true;
 }
+// The same bounded wait for warps that share their scheduler with working warps: each try
+// may keep the thread suspended for up to `kSuspendNs` before it reports failure, so a
+// waiting warp issues a handful of instructions instead of spinning through try / clock /
+// compare / branch (about a seventh of all instructions the convolution kernels issued
+// were such spins).
+constexpr uint32_t kSuspendNs = 20000;
+__device__ __forceinline__ bool mbar_try_suspend(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendNs) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_suspend(uint32_t bar, uint32_t parity, uint32_t abort_flag,
+                                                  unsigned* status)
+{
+    if (mbar_try(bar, parity)) return true;
+    const long long limit = lds32(abort_flag) ? kWaitShort : kWaitLong;
+    const long long t0 = clock64();
+    while (!mbar_try_suspend(bar, parity)) {
+        if (clock64() - t0 > limit) {
+            sts32(abort_flag, 1);
+            atomicOr(status, kStatusTimeout);
+            return false;
+        }
+    }
+    return true;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
                                             uint32_t bar)
 {
