@@ -284,6 +284,15 @@ size_t q4_gemm_host_staging_bytes(int32_t M, int32_t N, int32_t K,
  * flag is cleared), Q4_ERR_CUDA if the stream reports an error, else Q4_OK. */
 q4_status q4_last_device_status(void* stream);
 
+/*
+ * Diagnostic (no counterpart in the paper): launches one small kernel that waits, with the
+ * short limit of this library's bounded waits (about a millisecond), on a barrier nothing
+ * arrives on.  The wait gives up, the kernel ends normally, and the next
+ * q4_last_device_status on the device returns Q4_ERR_DEVICE_TIMEOUT once.  outcome_dev
+ * (device int, may be NULL) receives 2 when the wait ran out and 1 if it completed.
+ */
+q4_status q4_selftest_wait_timeout(int* outcome_dev, void* stream);
+
 /* Kernel selection for ablations and tests: 0 = automatic, 1 = general (SIMT)
  * kernels only, 2 = tensor-core kernels or an error where their alignment rules do
  * not hold, 3 = like 2 but never the CTA-pair kernel.  Returns the previous value.

@@ -36,7 +36,7 @@ EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_st
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
            "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak",
            "q4_quant_params", "q4_quantize", "q4_dequantize", "q4_gemm_u8",
-           "q4_gemm_u8_workspace_bytes"]
+           "q4_gemm_u8_workspace_bytes", "q4_selftest_wait_timeout"]
 
 
 class Q4Error(RuntimeError):
@@ -131,6 +131,7 @@ _lib.q4_gemm_u8_workspace_bytes.restype = _sz
 _lib.q4_quant_params.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp]
 _lib.q4_quantize.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp, _i64, _vp]
 _lib.q4_dequantize.argtypes = [_vp, _i64, _i32, _i32, ctypes.c_float, _vp, _i64, _vp]
+_lib.q4_selftest_wait_timeout.argtypes = [_vp, _vp]
 _lib.q4_last_device_status.argtypes = [_vp]
 _lib.q4_set_variant.argtypes = [ctypes.c_int]
 _lib.q4_launch_count.restype = ctypes.c_uint64
@@ -331,6 +332,13 @@ def q4_dequantize(C, scale: float, R):
     _check(_lib.q4_dequantize(_ptr(C), _pitch_elems(C, "C"), rows, cols, float(scale), _ptr(R),
                               _pitch_elems(R, "R"), _stream()), "q4_dequantize")
     return R
+
+
+def q4_selftest_wait_timeout(outcome=None):
+    """Launches the diagnostic kernel whose bounded wait runs out (see include/q4.h);
+    ``outcome`` is an optional CUDA int32 tensor of one element."""
+    _dev(outcome, torch.int32, "outcome")
+    _check(_lib.q4_selftest_wait_timeout(_ptr(outcome), _stream()), "q4_selftest_wait_timeout")
 
 
 def q4_row_sums(P, rows: int, K: int, sums):

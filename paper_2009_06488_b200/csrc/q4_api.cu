@@ -392,6 +392,13 @@ q4_status q4_dequantize(const int32_t* C, int64_t ldc, int32_t rows, int32_t col
                    cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
+q4_status q4_selftest_wait_timeout(int* outcome_dev, void* stream)
+{
+    if (outcome_dev && (uintptr_t)outcome_dev % 4) return Q4_ERR_ALIGNMENT;
+    return launch_wait_selftest(outcome_dev, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? Q4_OK : Q4_ERR_CUDA;
+}
+
 q4_status q4_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int64_t ldb,
                      int32_t K, int32_t N, void* stream)
 {

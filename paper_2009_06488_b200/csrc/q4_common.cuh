@@ -141,6 +141,8 @@ q4_status   launch_gemm_u8(const GemmParams& p, cudaStream_t st);
 cudaError_t launch_byte_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K, int32_t* sums,
                              cudaStream_t st);
 
+cudaError_t launch_wait_selftest(int* outcome_dev, cudaStream_t st);
+
 void count_launch(int n = 1);
 
 }  // namespace q4
