@@ -194,18 +194,21 @@ def run_reference(args):
 
 # --------------------------------------------------------------------------- GPU arm
 
-def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20):
-    """Device time of every layer of the c4 chain, each layer launched `reps` times back to
-    back behind a busy GPU so that launch latency is not what is measured."""
+def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20, net=None):
+    """Device time of every layer of a layer chain (default: the c4 chain), each layer
+    launched `reps` times back to back behind a busy GPU so that launch latency is not what
+    is measured."""
     import torch
-    net = wl.c4(batch=batch, seed=4000, centred=True)
+    if net is None:
+        net = wl.c4(batch=batch, seed=4000, centred=True)
     X = torch.from_numpy(net.X).cuda()
     layers, total_ms, total_bytes = {}, 0.0, 0
     for L in net.layers:
         d = q4.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
         ws = torch.empty(q4.q4_conv2d_workspace_bytes(d), dtype=torch.uint8, device="cuda")
         Y = torch.empty((d.M, L.OC // 2), dtype=torch.uint8, device="cuda")
-        Wt, b = torch.from_numpy(L.Wt).cuda(), torch.from_numpy(L.bias).cuda()
+        Wt = torch.from_numpy(L.Wt).cuda()
+        b = None if L.bias is None else torch.from_numpy(L.bias).cuda()
         # the weights' depth sums are part of the prepared weights: taken once (Section II-B)
         cw = q4.q4_row_sums(Wt, L.OC, d.K, torch.empty(L.OC, dtype=torch.int32, device="cuda"))
         rq = q4.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi)
@@ -224,7 +227,7 @@ def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20):
             torch.cuda.synchronize()
             ts.append(e0.elapsed_time(e1) / reps)
         ms = statistics.median(ts)
-        nbytes = X.numel() + Wt.numel() + 4 * b.numel() + Y.numel()
+        nbytes = X.numel() + Wt.numel() + (0 if b is None else 4 * b.numel()) + Y.numel()
         layers[L.name] = {"ms": ms, "compulsory_gbs": nbytes / (ms * 1e-3) / 1e9,
                           "gops": 2.0 * d.M * d.K * L.OC / (ms * 1e-3) / 1e9}
         total_ms += ms
@@ -460,6 +463,14 @@ def run_ours(args):
 
     # ---- the c4 layer chain (batch 4096), outside the timed region: per-layer device times
     c4_detail = time_c4_chain(q4, wl) if world == 1 and not args.no_c4_chain else None
+    t2_detail = None
+    if world == 1 and not args.no_c4_chain:
+        # the layer list of the paper's Table II (six convolutions on 25 x 33 gray images) with
+        # random weights, batch 4096; the paper's Table III gives 0.45 ms of convolution time
+        # per image for its 4-bit network on one ARM Cortex-A73 core
+        t2_detail = time_c4_chain(q4, wl, net=wl.paper_table2_net(batch=4096))
+        t2_detail["us_per_image"] = t2_detail["ms"] * 1e3 / 4096
+        t2_detail["paper_table3_qnn4_conv_ms_per_image"] = 0.45
     im2col_detail = time_im2col(q4, wl, peaks["hbm"]) if world == 1 and not args.no_c4_chain else None
     u8_detail = time_u8_comparison(q4, wl, GEMM_N) if world == 1 and not args.no_c4_chain else None
     float_detail = time_float_boundary(q4, wl, peaks["hbm"]) if world == 1 and not args.no_c4_chain else None
@@ -507,6 +518,7 @@ def run_ours(args):
             "q4_conv2d_c3_unroll_path_equivalent_gbs": conv_path_bytes / (conv_ms * 1e-3) / 1e9,
             "q4_conv2d_c3_gops": conv_ops / (conv_ms * 1e-3) / 1e9,
             "c4_chain_batch4096": c4_detail,
+            "paper_table2_layers_batch4096": t2_detail,
             "q4_im2col": im2col_detail,
             "float_boundary": float_detail,
             "eight_bit_comparison": u8_detail,
