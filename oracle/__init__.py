@@ -297,3 +297,6 @@ from .qfloat import dequantize, quant_params, quantize  # noqa: E402,F401
 
 # The 8-bit product of the paper's comparison (Eq. 2 with 8-bit values), numpy int64.
 from .q8 import gemm_u8, gemm_u8_fourterm  # noqa: E402,F401
+
+# Per-output-channel weight zero points and re-quantization multipliers, numpy int64.
+from .perchannel import gemm_channels, requant_channels  # noqa: E402,F401
