@@ -271,15 +271,27 @@ def time_im2col(q4, wl, hbm_peak: float, batch: int = 4096, reps: int = 10):
 
 def time_float_boundary(q4, wl, hbm_peak: float, n: int = 1 << 26, reps: int = 10):
     """Device times of the float boundary on n = 64 Mi values (256 MB of floats, larger than
-    L2): Eq. 1's range pass (reads 4n bytes), its quantizing pass (reads 4n, writes n/2), and
-    Eq. 4's scale-back of an int32 matrix of the same size (reads 4n, writes 4n)."""
+    L2): Eq. 1's range pass (reads 4n bytes), its quantizing pass (reads 4n, writes n/2),
+    Eq. 4's scale-back of an int32 matrix of the same size (reads 4n, writes 4n), and the
+    per-channel finishing pass q4_requant_channels on an 8192 x 8192 int32 matrix (reads 4n,
+    writes n/2)."""
     import torch
     X = torch.from_numpy(wl.rand_floats(79, 1 << 20)).cuda().repeat(n >> 20)
     qp = torch.zeros(2, dtype=torch.int32, device="cuda")
     Q = torch.empty(n // 2, dtype=torch.uint8, device="cuda")
     C = torch.randint(-(1 << 20), 1 << 20, (n,), dtype=torch.int32, device="cuda")
     R = torch.empty(n, dtype=torch.float32, device="cuda")
+    side = 1 << 13
+    rows_c = n // side
+    ra = torch.randint(0, 15 * 64, (rows_c,), dtype=torch.int32, device="cuda")
+    chan = lambda lo, hi: torch.randint(lo, hi, (side,), dtype=torch.int32, device="cuda")
+    zb_c, bias_c, mult_c, shift_c = chan(0, 16), chan(-512, 513), chan(1 << 30, (1 << 31) - 1), chan(2, 15)
+    Cq2 = torch.empty((rows_c, side // 2), dtype=torch.uint8, device="cuda")
+    C2 = C.reshape(rows_c, side)
     calls = {"q4_quant_params": (lambda: q4.q4_quant_params(X, qp), 4 * n),
+             "q4_requant_channels": (lambda: q4.q4_requant_channels(C2, rows_c, side, 64, 7, ra, zb_c, bias_c,
+                                                                    mult_c, shift_c, 0, 0, 15, Cq2),
+                                     4 * n + n // 2),
              "q4_quantize": (lambda: q4.q4_quantize(X, qp, Q), 4 * n + n // 2),
              "q4_dequantize": (lambda: q4.q4_dequantize(C, 1e-3, R), 8 * n)}
     out = {"values": n}

@@ -213,6 +213,26 @@ q4_status q4_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
                       int32_t* sums, void* stream);
 
 /*
+ * Per-output-channel weight quantization: an extension of the paper's scheme, which has one
+ * scale and one zero point per weight matrix (Section II-A, III-B).  Eq. 2 holds column by
+ * column, and a column's zero point enters only through a rank-one term, so the product is
+ * taken once with zb = 0 and finished here:
+ *   C0 = q4_gemm(A, Bt, za, zb = 0)            (int32, M x N, pitch ldc elements)
+ *   acc[m][n] = C0[m][n] - zb[n] * (rowsum_a[m] - K * za) + bias[n]
+ *   y[m][n]   = clamp(floor((acc * mult[n] + 2^(30 + shift[n])) / 2^(31 + shift[n])) + zo, lo, hi)
+ * written packed two per byte to Cq (pitch ldcq bytes >= N / 2; N even).  rowsum_a[m] =
+ * sum_k A[m][k] (q4_row_sums, or q4_im2col's side output).  zb (values 0..15) and bias may be
+ * NULL (= 0); mult[n] in [2^30, 2^31) and shift[n] in 0..31 are required; all are DEVICE
+ * arrays of N int32 and are not range-checked.  zo, clamp_lo, clamp_hi as in q4_requant.
+ */
+q4_status q4_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                              int32_t za, const int32_t* rowsum_a,
+                              const int32_t* zb, const int32_t* bias,
+                              const int32_t* mult, const int32_t* shift,
+                              int32_t zo, int32_t clamp_lo, int32_t clamp_hi,
+                              uint8_t* Cq, int64_t ldcq, void* stream);
+
+/*
  * The 8-bit product of the paper's comparison (Section II-B: values in 0..255 with 32-bit
  * accumulators; the experiments of Section IV measure the 4-bit product against it):
  *   C[m][n] = sum_k (A[m][k] - za) * (Bt[n][k] - zb),  za, zb in 0..255,

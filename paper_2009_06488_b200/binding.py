@@ -36,7 +36,7 @@ EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_st
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
            "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak",
            "q4_quant_params", "q4_quantize", "q4_dequantize", "q4_gemm_u8",
-           "q4_gemm_u8_workspace_bytes", "q4_selftest_wait_timeout"]
+           "q4_gemm_u8_workspace_bytes", "q4_selftest_wait_timeout", "q4_requant_channels"]
 
 
 class Q4Error(RuntimeError):
@@ -132,6 +132,8 @@ _lib.q4_quant_params.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp]
 _lib.q4_quantize.argtypes = [_vp, _i64, _i32, _i32, _vp, _vp, _i64, _vp]
 _lib.q4_dequantize.argtypes = [_vp, _i64, _i32, _i32, ctypes.c_float, _vp, _i64, _vp]
 _lib.q4_selftest_wait_timeout.argtypes = [_vp, _vp]
+_lib.q4_requant_channels.argtypes = [_vp, _i64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
+                                     _i32, _i32, _i32, _vp, _i64, _vp]
 _lib.q4_last_device_status.argtypes = [_vp]
 _lib.q4_set_variant.argtypes = [ctypes.c_int]
 _lib.q4_launch_count.restype = ctypes.c_uint64
@@ -339,6 +341,19 @@ def q4_selftest_wait_timeout(outcome=None):
     ``outcome`` is an optional CUDA int32 tensor of one element."""
     _dev(outcome, torch.int32, "outcome")
     _check(_lib.q4_selftest_wait_timeout(_ptr(outcome), _stream()), "q4_selftest_wait_timeout")
+
+
+def q4_requant_channels(C0, M: int, N: int, K: int, za: int, rowsum_a, zb, bias, mult, shift,
+                        zo: int, clamp_lo: int, clamp_hi: int, Cq):
+    """Finishes a product taken with zb = 0 for per-channel weight zero points and
+    multipliers; see include/q4.h."""
+    _dev(C0, torch.int32, "C0"); _dev(Cq, torch.uint8, "Cq")
+    for t, n in ((rowsum_a, "rowsum_a"), (zb, "zb"), (bias, "bias"), (mult, "mult"), (shift, "shift")):
+        _dev(t, torch.int32, n)
+    _check(_lib.q4_requant_channels(_ptr(C0), _rows(C0, "C0"), M, N, K, za, _ptr(rowsum_a), _ptr(zb),
+                                    _ptr(bias), _ptr(mult), _ptr(shift), zo, clamp_lo, clamp_hi,
+                                    _ptr(Cq), _rows(Cq, "Cq"), _stream()), "q4_requant_channels")
+    return Cq
 
 
 def q4_row_sums(P, rows: int, K: int, sums):

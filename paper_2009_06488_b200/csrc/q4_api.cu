@@ -399,6 +399,27 @@ q4_status q4_selftest_wait_timeout(int* outcome_dev, void* stream)
                ? Q4_OK : Q4_ERR_CUDA;
 }
 
+q4_status q4_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                              int32_t za, const int32_t* rowsum_a,
+                              const int32_t* zb, const int32_t* bias,
+                              const int32_t* mult, const int32_t* shift,
+                              int32_t zo, int32_t clamp_lo, int32_t clamp_hi,
+                              uint8_t* Cq, int64_t ldcq, void* stream)
+{
+    if (M < 0 || N < 0 || (N & 1) || K < 1 || ldc < N || ldcq < N / 2) return Q4_ERR_INVALID_ARG;
+    if (K > Q4_MAX_K || za < 0 || za > 15 || zo < 0 || zo > 15 || clamp_lo < 0 || clamp_hi > 15 ||
+        clamp_lo > clamp_hi)
+        return Q4_ERR_RANGE;
+    if (M == 0 || N == 0) return Q4_OK;
+    if (!C0 || !rowsum_a || !mult || !shift || !Cq) return Q4_ERR_INVALID_ARG;
+    const void* words[] = {C0, rowsum_a, zb, bias, mult, shift};
+    for (const void* w : words)
+        if ((uintptr_t)w % 4) return Q4_ERR_ALIGNMENT;
+    return launch_requant_channels(C0, ldc, M, N, K, za, rowsum_a, zb, bias, mult, shift, zo, clamp_lo,
+                                   clamp_hi, Cq, ldcq, static_cast<cudaStream_t>(stream)) == cudaSuccess
+               ? Q4_OK : Q4_ERR_CUDA;
+}
+
 q4_status q4_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int64_t ldb,
                      int32_t K, int32_t N, void* stream)
 {

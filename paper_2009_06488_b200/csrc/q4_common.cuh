@@ -143,6 +143,12 @@ cudaError_t launch_byte_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t
 
 cudaError_t launch_wait_selftest(int* outcome_dev, cudaStream_t st);
 
+cudaError_t launch_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                                    int32_t za, const int32_t* rowsum_a, const int32_t* zb,
+                                    const int32_t* bias, const int32_t* mult, const int32_t* shift,
+                                    int32_t zo, int32_t lo, int32_t hi, uint8_t* Cq, int64_t ldcq,
+                                    cudaStream_t st);
+
 void count_launch(int n = 1);
 
 }  // namespace q4

@@ -1,0 +1,133 @@
+// Per-output-channel weight quantization (an extension of the paper's per-matrix scheme of
+// Section II-A / III-B: every output channel n has its own weight zero point zb[n] and its
+// own re-quantization multiplier).  Eq. 2 holds column by column, and the zero point of a
+// column enters only through a rank-one term:
+//   sum_k (a - za)(b - zb[n]) = [sum_k (a - za) b]  -  zb[n] * (sum_k a - K za),
+// so the product is taken once with zb = 0 by q4_gemm and this kernel finishes it:
+//   acc = C0[m][n] - zb[n] * (rowsum_a[m] - K za) + bias[n]
+//   y   = clamp(floor((acc * mult[n] + 2^(30 + shift[n])) / 2^(31 + shift[n])) + zo, lo, hi)
+// packed two per byte.  One pass over the int32 matrix: bound by HBM (4 bytes read and half
+// a byte written per value).
+#include "q4_common.cuh"
+
+namespace q4 {
+
+struct ChannelParams {
+    const int32_t* C0;
+    int64_t ldc;
+    int32_t M, N, K, za;
+    const int32_t* rowsum_a;
+    const int32_t* zb;       // optional
+    const int32_t* bias;     // optional
+    const int32_t* mult;
+    const int32_t* shift;
+    int32_t zo, lo, hi;
+    uint8_t* Cq;
+    int64_t ldcq;
+};
+
+__device__ __forceinline__ uint32_t requant_one(int32_t acc, int32_t mult, int32_t shift, int zo, int lo, int hi)
+{
+    const int t = 31 + shift;
+    const long long v = (long long)acc * (long long)mult + (1ll << (t - 1));
+    int q = (int)(v >> t) + zo;
+    return (uint32_t)min(max(q, lo), hi);
+}
+
+// Eight consecutive channels (one 32-bit word of output) per thread; a thread keeps its
+// channels' parameters in registers and walks rows blockIdx.y, blockIdx.y + gridDim.y, ...
+__global__ void __launch_bounds__(256)
+requant_channels_vec_kernel(const ChannelParams p)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;      // output word within a row
+    if (j >= p.N / 8) return;
+    int zb[8], bias[8], mult[8], sh[8];
+    bool fast = true;                                         // the 32-bit rounding shift needs shift >= 2
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const int n = 8 * j + e;
+        zb[e] = p.zb ? p.zb[n] : 0;
+        bias[e] = p.bias ? p.bias[n] : 0;
+        mult[e] = p.mult[n];
+        sh[e] = p.shift[n];
+        fast = fast && sh[e] >= 2;
+    }
+    const int kza = p.K * p.za;
+    for (int r = blockIdx.y; r < p.M; r += gridDim.y) {
+        const int rowfac = p.rowsum_a[r] - kza;               // sum_k (a - za)
+        const int4* src = reinterpret_cast<const int4*>(p.C0 + (int64_t)r * p.ldc + 8 * j);
+        const int4 c0 = __ldcs(src), c1 = __ldcs(src + 1);
+        const int c[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+        uint32_t word = 0;
+        if (fast) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac) + (uint32_t)bias[e]);
+                const int s = sh[e] - 1;                      // see requant() in q4_common.cuh
+                int q = ((__mulhi(acc, mult[e]) + (1 << (s - 1))) >> s) + p.zo;
+                q = min(max(q, p.lo), p.hi);
+                word |= (uint32_t)q << (4 * e);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac) + (uint32_t)bias[e]);
+                word |= requant_one(acc, mult[e], sh[e], p.zo, p.lo, p.hi) << (4 * e);
+            }
+        }
+        *reinterpret_cast<uint32_t*>(p.Cq + (int64_t)r * p.ldcq + 4 * j) = word;
+    }
+}
+
+// Any shape and alignment: one output byte (two channels) per thread.
+__global__ void __launch_bounds__(256)
+requant_channels_byte_kernel(const ChannelParams p)
+{
+    const int nb = p.N / 2;
+    const int64_t total = (int64_t)p.M * nb;
+    const int kza = p.K * p.za;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / nb;
+        const int j = (int)(i - r * nb);
+        const int rowfac = p.rowsum_a[r] - kza;
+        uint32_t byte = 0;
+#pragma unroll
+        for (int e = 0; e < 2; ++e) {
+            const int n = 2 * j + e;
+            const int zb = p.zb ? p.zb[n] : 0, bias = p.bias ? p.bias[n] : 0;
+            const int acc = (int)((uint32_t)p.C0[r * p.ldc + n] - (uint32_t)(zb * rowfac) + (uint32_t)bias);
+            byte |= requant_one(acc, p.mult[n], p.shift[n], p.zo, p.lo, p.hi) << (4 * e);
+        }
+        p.Cq[r * p.ldcq + j] = (uint8_t)byte;
+    }
+}
+
+cudaError_t launch_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, int32_t N, int32_t K,
+                                    int32_t za, const int32_t* rowsum_a, const int32_t* zb,
+                                    const int32_t* bias, const int32_t* mult, const int32_t* shift,
+                                    int32_t zo, int32_t lo, int32_t hi, uint8_t* Cq, int64_t ldcq,
+                                    cudaStream_t st)
+{
+    ChannelParams p{C0, ldc, M, N, K, za, rowsum_a, zb, bias, mult, shift, zo, lo, hi, Cq, ldcq};
+    const bool vec = N % 8 == 0 && ldc % 4 == 0 && (uintptr_t)C0 % 16 == 0 && ldcq % 4 == 0 &&
+                     (uintptr_t)Cq % 4 == 0;
+    if (vec) {
+        const int words = N / 8;
+        const int bx = words < 256 ? (words + 31) / 32 * 32 : 256;
+        const unsigned gx = (unsigned)((words + bx - 1) / bx);
+        int64_t gy = (int64_t)148 * 16 / gx;
+        if (gy < 1) gy = 1;
+        if (gy > M) gy = M;
+        if (gy > 65535) gy = 65535;
+        requant_channels_vec_kernel<<<dim3(gx, (unsigned)gy), bx, 0, st>>>(p);
+    } else {
+        int64_t blocks = ((int64_t)M * (N / 2) + 255) / 256;
+        if (blocks > 148 * 16) blocks = 148 * 16;
+        requant_channels_byte_kernel<<<(int)blocks, 256, 0, st>>>(p);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace q4

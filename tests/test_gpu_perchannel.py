@@ -1,0 +1,119 @@
+"""GPU parity: per-output-channel weight zero points and multipliers (q4_gemm with zb = 0, then
+q4_requant_channels) against the per-channel oracle, byte for byte."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2009_06488_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q4():
+    from paper_2009_06488_b200 import binding
+    return binding
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def channel_params(seed, N, min_shift=0):
+    zb = wl.rand_ints(seed, 4, 0, 15, N).astype(np.int32)
+    bias = wl.rand_ints(seed, 3, -512, 512, N).astype(np.int32)
+    mult = wl.rand_ints(seed, 5, 1 << 30, (1 << 31) - 1, N).astype(np.int32)
+    shift = wl.rand_ints(seed, 6, min_shift, 14, N).astype(np.int32)
+    return zb, bias, mult, shift
+
+
+def run(q4, A, Bt, M, N, K, za, zb, bias, mult, shift, zo, lo, hi, ldc_pad=0, ldq_pad=0):
+    import torch
+    Ad, Bd = dev(A), dev(Bt)
+    C0 = torch.empty((M, N + ldc_pad), dtype=torch.int32, device="cuda")
+    q4.q4_gemm(Ad, Bd, C0[:, :N] if ldc_pad else C0, M, N, K, za, 0)
+    ra = torch.empty(M, dtype=torch.int32, device="cuda")
+    q4.q4_row_sums(Ad, M, K, ra)
+    Cq = torch.full((M, N // 2 + ldq_pad), 0xA5, dtype=torch.uint8, device="cuda")
+    opt = lambda a: None if a is None else dev(a)
+    q4.q4_requant_channels(C0[:, :N] if ldc_pad else C0, M, N, K, za, ra, opt(zb), opt(bias), dev(mult),
+                           dev(shift), zo, lo, hi, Cq[:, :N // 2] if ldq_pad else Cq)
+    out = Cq.cpu().numpy()
+    assert (out[:, N // 2:] == 0xA5).all()
+    return out[:, :N // 2]
+
+
+SHAPES = [(1, 2, 1), (64, 64, 256), (130, 70, 100), (300, 264, 1000), (257, 136, 33), (1000, 520, 777),
+          (2048, 1024, 512)]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("min_shift", [0, 2])
+def test_gemm_with_per_channel_parameters(q4, shape, min_shift):
+    M, N, K = shape
+    seed = 9000 + sum(shape)
+    c = wl.gemm_case("pc", M, N, K, seed=seed)
+    zb, bias, mult, shift = channel_params(seed, N, min_shift)
+    want = oracle.requant_channels(oracle.gemm_channels(c.A, c.Bt, M, N, K, c.za, zb, bias), mult, shift, 3, 1, 14)
+    pad = 4 if M % 2 else 0
+    got = run(q4, c.A, c.Bt, M, N, K, c.za, zb, bias, mult, shift, 3, 1, 14, ldc_pad=pad, ldq_pad=pad)
+    assert (got == want).all()
+
+
+def test_optional_arrays_and_uniform_channels_match_the_fused_path(q4):
+    """No zero points and no bias: the plain product; one zero point for every channel: the
+    same bytes as q4_gemm_requant's fused epilogue."""
+    import torch
+    M, N, K = 200, 136, 520
+    c = wl.gemm_case("pc", M, N, K, seed=12, lda=272, ldb=272)
+    _, _, mult, shift = channel_params(12, N, 2)
+    want = oracle.requant_channels(oracle.gemm_channels(c.A, c.Bt, M, N, K, c.za, [0] * N), mult, shift, 0, 0, 15)
+    assert (run(q4, c.A, c.Bt, M, N, K, c.za, None, None, mult, shift, 0, 0, 15) == want).all()
+    zb1 = np.full(N, c.zb, np.int32)
+    m1, s1 = np.full(N, c.mult, np.int32), np.full(N, 7, np.int32)
+    Cq = torch.empty((M, N // 2), dtype=torch.uint8, device="cuda")
+    q4.q4_gemm_requant(dev(c.A), dev(c.Bt), Cq, M, N, K, c.za, c.zb, q4.Requant(c.mult, 7, 2, 0, 15))
+    assert (run(q4, c.A, c.Bt, M, N, K, c.za, zb1, None, m1, s1, 2, 0, 15) == Cq.cpu().numpy()).all()
+
+
+def test_conv_layer_with_per_channel_weights(q4):
+    """Explicit path of a layer: q4_im2col (matrix and row sums), q4_gemm with zb = 0,
+    q4_requant_channels."""
+    import torch
+    g = (3, 12, 14, 16, 24, 3, 3, 1, 1, 1, 1)
+    N_, H, W, C, OC, KH, KW, sh, sw, ph, pw = g
+    dq = q4.ConvDesc(*g)
+    do = oracle.ConvDesc(*g)
+    K = KH * KW * C
+    X = wl.rand_flat_nibbles(31, 1, N_ * H * W * C)
+    Wt = wl.rand_packed(31, 2, OC, K)
+    zb, bias, mult, shift = channel_params(31, OC, 0)
+    za = 6
+    lda = (K // 2 + 15) // 16 * 16
+    Ao, _ = oracle.im2col(X, do, za, lda)
+    want = oracle.requant_channels(oracle.gemm_channels(Ao, Wt, dq.M, OC, K, za, zb, bias), mult, shift, 0, 0, 15)
+    A = torch.zeros((dq.M, lda), dtype=torch.uint8, device="cuda")
+    ra = torch.empty(dq.M, dtype=torch.int32, device="cuda")
+    q4.q4_im2col(dev(X), dq, za, A, ra)
+    C0 = torch.empty((dq.M, OC), dtype=torch.int32, device="cuda")
+    q4.q4_gemm(A, dev(Wt), C0, dq.M, OC, K, za, 0, ra)
+    Y = torch.empty((dq.M, OC // 2), dtype=torch.uint8, device="cuda")
+    q4.q4_requant_channels(C0, dq.M, OC, K, za, ra, dev(zb), dev(bias), dev(mult), dev(shift), 0, 0, 15, Y)
+    assert (Y.cpu().numpy() == want).all()
+
+
+def test_argument_checks(q4):
+    import torch
+    C0 = torch.zeros((4, 8), dtype=torch.int32, device="cuda")
+    v = torch.zeros(8, dtype=torch.int32, device="cuda")
+    Cq = torch.zeros((4, 4), dtype=torch.uint8, device="cuda")
+    with pytest.raises(q4.Q4Error) as e:
+        q4.q4_requant_channels(C0, 4, 7, 16, 0, v, None, None, v, v, 0, 0, 15, Cq)       # odd N
+    assert e.value.status == q4.Q4_ERR_INVALID_ARG
+    with pytest.raises(q4.Q4Error) as e:
+        q4.q4_requant_channels(C0, 4, 8, 16, 16, v, None, None, v, v, 0, 0, 15, Cq)      # za out of range
+    assert e.value.status == q4.Q4_ERR_RANGE
+    with pytest.raises(q4.Q4Error) as e:
+        q4.q4_requant_channels(C0, 4, 8, 16, 0, v, None, None, None, v, 0, 0, 15, Cq)    # multipliers missing
+    assert e.value.status == q4.Q4_ERR_INVALID_ARG
