@@ -41,8 +41,11 @@ requant_channels_vec_kernel(const ChannelParams p)
 {
     const int j = blockIdx.x * blockDim.x + threadIdx.x;      // output word within a row
     if (j >= p.N / 8) return;
-    int zb[8], bias[8], mult[8], sh[8];
-    bool fast = true;                                         // the 32-bit rounding shift needs shift >= 2
+    int zb[8], bias[8], mult[8], sh[8], rnd[8];
+    // 32-bit form of the rounding shift (see requant() in q4_common.cuh) with the output zero
+    // point folded into the rounding constant: ((hi + 2^(s-1) + zo * 2^s) >> s), s = shift - 1;
+    // it needs 2 <= shift <= 27 so that the sum stays inside 32 bits
+    bool fast = true;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         const int n = 8 * j + e;
@@ -50,7 +53,9 @@ requant_channels_vec_kernel(const ChannelParams p)
         bias[e] = p.bias ? p.bias[n] : 0;
         mult[e] = p.mult[n];
         sh[e] = p.shift[n];
-        fast = fast && sh[e] >= 2;
+        fast = fast && sh[e] >= 2 && sh[e] <= 27;
+        const int s = fast ? sh[e] - 1 : 1;
+        rnd[e] = (1 << (s - 1)) + (p.zo << s);
     }
     const int kza = p.K * p.za;
     for (int r = blockIdx.y; r < p.M; r += gridDim.y) {
@@ -63,8 +68,7 @@ requant_channels_vec_kernel(const ChannelParams p)
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac) + (uint32_t)bias[e]);
-                const int s = sh[e] - 1;                      // see requant() in q4_common.cuh
-                int q = ((__mulhi(acc, mult[e]) + (1 << (s - 1))) >> s) + p.zo;
+                int q = (__mulhi(acc, mult[e]) + rnd[e]) >> (sh[e] - 1);
                 q = min(max(q, p.lo), p.hi);
                 word |= (uint32_t)q << (4 * e);
             }

@@ -20,11 +20,11 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-def channel_params(seed, N, min_shift=0):
+def channel_params(seed, N, min_shift=0, max_shift=14):
     zb = wl.rand_ints(seed, 4, 0, 15, N).astype(np.int32)
     bias = wl.rand_ints(seed, 3, -512, 512, N).astype(np.int32)
     mult = wl.rand_ints(seed, 5, 1 << 30, (1 << 31) - 1, N).astype(np.int32)
-    shift = wl.rand_ints(seed, 6, min_shift, 14, N).astype(np.int32)
+    shift = wl.rand_ints(seed, 6, min_shift, max_shift, N).astype(np.int32)
     return zb, bias, mult, shift
 
 
@@ -49,12 +49,12 @@ SHAPES = [(1, 2, 1), (64, 64, 256), (130, 70, 100), (300, 264, 1000), (257, 136,
 
 
 @pytest.mark.parametrize("shape", SHAPES)
-@pytest.mark.parametrize("min_shift", [0, 2])
-def test_gemm_with_per_channel_parameters(q4, shape, min_shift):
+@pytest.mark.parametrize("shifts", [(0, 14), (2, 14), (20, 31)])
+def test_gemm_with_per_channel_parameters(q4, shape, shifts):
     M, N, K = shape
     seed = 9000 + sum(shape)
     c = wl.gemm_case("pc", M, N, K, seed=seed)
-    zb, bias, mult, shift = channel_params(seed, N, min_shift)
+    zb, bias, mult, shift = channel_params(seed, N, *shifts)
     want = oracle.requant_channels(oracle.gemm_channels(c.A, c.Bt, M, N, K, c.za, zb, bias), mult, shift, 3, 1, 14)
     pad = 4 if M % 2 else 0
     got = run(q4, c.A, c.Bt, M, N, K, c.za, zb, bias, mult, shift, 3, 1, 14, ldc_pad=pad, ldq_pad=pad)
