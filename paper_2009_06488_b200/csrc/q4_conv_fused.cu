@@ -1115,17 +1115,23 @@ static cudaError_t launch_kernel(FusedKernel kernel, const fused::Params& p, siz
     return cudaGetLastError();
 }
 
+template <int NT, int KS>
+static cudaError_t launch_ks(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
+{
+    if (p.OW % 4 == 0)
+        return launch_kernel(fused::conv_fused_kernel<NT, false, KS, true>, p, smem, tiles, st);
+    return launch_kernel(fused::conv_fused_kernel<NT, false, KS, false>, p, smem, tiles, st);
+}
+
 template <int NT, bool EXP>
 static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
-    // 3x3 layers with 8, 16 or 32 input channels and twice as many outputs (and the c3 layer)
-    constexpr int KS_OF_NT = NT == 2 ? 3 : NT == 4 ? 5 : NT == 8 ? 9 : 0;
-    if constexpr (!EXP && KS_OF_NT != 0) {
-        if (p.KS == KS_OF_NT) {
-            if (p.OW % 4 == 0)
-                return launch_kernel(fused::conv_fused_kernel<NT, EXP, KS_OF_NT, true>, p, smem, tiles, st);
-            return launch_kernel(fused::conv_fused_kernel<NT, EXP, KS_OF_NT, false>, p, smem, tiles, st);
-        }
+    // 3x3 layers with 8, 16 or 32 input channels (3, 5, 9 depth steps) get instances with the
+    // depth loop unrolled, for the channel counts the workloads pair them with
+    if constexpr (!EXP) {
+        if (p.KS == 3 && NT <= 2) return launch_ks<NT, 3>(p, smem, tiles, st);
+        if (p.KS == 5 && NT >= 2 && NT <= 4) return launch_ks<NT, 5>(p, smem, tiles, st);
+        if (p.KS == 9 && NT == 8) return launch_ks<NT, 9>(p, smem, tiles, st);
     }
     return launch_kernel(fused::conv_fused_kernel<NT, EXP>, p, smem, tiles, st);
 }
@@ -1168,6 +1174,9 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
         if (nibbles)
             return d.OC == 8 ? launch_kernel(fused::conv_lane_kernel<8, true, 0, 0>, p, smem, tiles, st)
                              : launch_kernel(fused::conv_lane_kernel<16, true, 0, 0>, p, smem, tiles, st);
+        // a 5x5 single-channel first layer whose rows are not whole words (25-pixel rows)
+        if (d.OC == 8 && d.KH == 5 && p.segw == 2)
+            return launch_kernel(fused::conv_lane_kernel<8, false, 5, 2>, p, smem, tiles, st);
         return d.OC == 8 ? launch_kernel(fused::conv_lane_kernel<8, false, 0, 0>, p, smem, tiles, st)
                          : launch_kernel(fused::conv_lane_kernel<16, false, 0, 0>, p, smem, tiles, st);
     }
