@@ -311,8 +311,9 @@ q4_status q4_conv2d_static(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     if (conv_shape(d).bytes > (size_t)Q4_STATIC_SCRATCH_BYTES) return Q4_ERR_STATIC_SCRATCH;
     void* scratch = static_scratch_ptr();
     if (!scratch) return Q4_ERR_CUDA;
-    // q4_conv2d rewrites the whole unrolled matrix (pad nibbles included) and zeroes
-    // the row sums before accumulating them, so stale contents cannot leak through
+    // q4_conv2d rewrites the whole unrolled matrix (pad nibbles included) and every row
+    // sum (written directly, or zeroed before accumulation), so stale contents cannot leak
+    // through
     return q4_conv2d(X, Wt, ldw, colsum_w, bias, d, za, zb, rq, Y, scratch,
                      (size_t)Q4_STATIC_SCRATCH_BYTES, stream);
 }

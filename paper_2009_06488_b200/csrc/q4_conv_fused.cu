@@ -31,8 +31,8 @@
 // what matters.
 //
 // Requirements (else the caller falls back to unroll + GEMM): OC a multiple of 8 up to
-// 64, Y 8-byte aligned, and the weights, tables and two input buffers fit in shared
-// memory.
+// 64, Y 8-byte aligned, and the weights, tables and the ring of input buffers fit in
+// shared memory.
 #include <type_traits>
 
 #include "q4_common.cuh"
@@ -454,8 +454,8 @@ conv_fused_kernel(const Params p)
     }
     __syncthreads();
 
-    // Both roles go through the same number of barriers: one before the first tile and
-    // one after each of this CTA's `mytiles` tiles (the grid never exceeds the tile count).
+    // This CTA's tiles: blockIdx.x, blockIdx.x + gridDim.x, ... (the grid never exceeds the
+    // tile count).
     const int64_t ntiles = (p.M + ROWS_PER_CTA - 1) / ROWS_PER_CTA;
     const int mytiles = (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
 

@@ -17,8 +17,9 @@
 //    is re-read kh*kw times, the input itself is read from HBM once).
 //  * im2col_byte_kernel -- any geometry (odd channel counts make pixels
 //    nibble-granular): one thread per output byte.
-// Row sums: lanes of one row are contiguous in a warp, so a segmented warp reduction
-// leaves one atomicAdd per row per warp (rowsum is zeroed first).
+// Row sums of the last two kernels: lanes of one row are contiguous in a warp, so a segmented
+// warp reduction leaves one atomicAdd per row per warp (rowsum is zeroed first); the tile
+// kernel writes each row's sum directly.
 #include "q4_common.cuh"
 
 namespace q4 {
