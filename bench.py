@@ -549,7 +549,17 @@ def run_case(args):
     torch.cuda.set_device(0)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     n = args.n
-    if args.case == "quantize":
+    if args.case == "requant_channels":
+        # per-channel finishing pass on an n x 8192 int32 matrix
+        side = 8192
+        C0 = torch.randint(-(1 << 16), 1 << 16, (n, side), dtype=torch.int32, device="cuda")
+        ra = torch.randint(0, 15 * 64, (n,), dtype=torch.int32, device="cuda")
+        chan = lambda lo, hi: torch.randint(lo, hi, (side,), dtype=torch.int32, device="cuda")
+        zb_c, bias_c, mult_c, shift_c = chan(0, 16), chan(-512, 513), chan(1 << 30, (1 << 31) - 1), chan(2, 15)
+        Cq = torch.empty((n, side // 2), dtype=torch.uint8, device="cuda")
+        call = lambda: q4.q4_requant_channels(C0, n, side, 64, 7, ra, zb_c, bias_c, mult_c, shift_c, 0, 0, 15, Cq)
+        units, unit = (C0.numel() * 4 + Cq.numel()) / 1e9, "GB/s"
+    elif args.case == "quantize":
         # Eq. 1 on an n x 4096 float matrix: range pass + quantizing pass per call
         X = dev(wl.rand_floats(80, 1 << 20)).repeat(n * 4096 >> 20).reshape(n, 4096)
         qp = torch.zeros(2, dtype=torch.int32, device="cuda")
@@ -643,7 +653,7 @@ def main():
                     help="skip the per-layer timing of the c4 chain that follows the timed steps")
     ap.add_argument("--ref-seconds", type=float, default=None,
                     help="--impl reference: CPU seconds of oracle work per step (default: sized from --steps)")
-    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "gemm_u8", "quantize", "conv", "im2col", "c4layer"],
+    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "gemm_u8", "quantize", "requant_channels", "conv", "im2col", "c4layer"],
                     help="profile one call in a loop instead of the benchmark step")
     ap.add_argument("--layer", type=int, default=0, help="--case c4layer: 0..4 = L1..L4, FC")
     ap.add_argument("--presums", action="store_true", help="--case gemm: pass precomputed depth sums")
