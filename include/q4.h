@@ -233,6 +233,21 @@ q4_status q4_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, int32_t
                               uint8_t* Cq, int64_t ldcq, void* stream);
 
 /*
+ * A convolution layer with per-output-channel weight quantization, as ONE fused kernel (the
+ * unrolled matrix is never written; no workspace): like q4_conv2d, but output channel n has
+ * its own weight zero point zb[n] (0..15), multiplier mult[n] in [2^30, 2^31) and shift[n] in
+ * 0..31 (DEVICE arrays of OC int32, not range-checked); colsum_w and bias may be NULL.
+ * Layers the fused kernel does not take (OC not a multiple of 8 or above 64, Y not 8-byte
+ * aligned, too large for shared memory) return Q4_ERR_UNSUPPORTED: run those as q4_im2col,
+ * q4_gemm with zb = 0 and q4_requant_channels.  Extension of the paper's per-matrix scheme
+ * (Section II-A), see q4_requant_channels.
+ */
+q4_status q4_conv2d_channels(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
+                             const int32_t* colsum_w, const int32_t* bias, const q4_conv_desc* d,
+                             int32_t za, const int32_t* zb, const int32_t* mult, const int32_t* shift,
+                             int32_t zo, int32_t clamp_lo, int32_t clamp_hi, uint8_t* Y, void* stream);
+
+/*
  * The 8-bit product of the paper's comparison (Section II-B: values in 0..255 with 32-bit
  * accumulators; the experiments of Section IV measure the 4-bit product against it):
  *   C[m][n] = sum_k (A[m][k] - za) * (Bt[n][k] - zb),  za, zb in 0..255,

@@ -36,7 +36,7 @@ EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_st
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
            "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak",
            "q4_quant_params", "q4_quantize", "q4_dequantize", "q4_gemm_u8",
-           "q4_gemm_u8_workspace_bytes", "q4_selftest_wait_timeout", "q4_requant_channels"]
+           "q4_gemm_u8_workspace_bytes", "q4_selftest_wait_timeout", "q4_requant_channels", "q4_conv2d_channels"]
 
 
 class Q4Error(RuntimeError):
@@ -134,6 +134,8 @@ _lib.q4_dequantize.argtypes = [_vp, _i64, _i32, _i32, ctypes.c_float, _vp, _i64,
 _lib.q4_selftest_wait_timeout.argtypes = [_vp, _vp]
 _lib.q4_requant_channels.argtypes = [_vp, _i64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                                      _i32, _i32, _i32, _vp, _i64, _vp]
+_lib.q4_conv2d_channels.argtypes = [_vp, _vp, _i64, _vp, _vp, ctypes.POINTER(_ConvDesc), _i32, _vp, _vp, _vp,
+                                    _i32, _i32, _i32, _vp, _vp]
 _lib.q4_last_device_status.argtypes = [_vp]
 _lib.q4_set_variant.argtypes = [ctypes.c_int]
 _lib.q4_launch_count.restype = ctypes.c_uint64
@@ -354,6 +356,20 @@ def q4_requant_channels(C0, M: int, N: int, K: int, za: int, rowsum_a, zb, bias,
                                     _ptr(bias), _ptr(mult), _ptr(shift), zo, clamp_lo, clamp_hi,
                                     _ptr(Cq), _rows(Cq, "Cq"), _stream()), "q4_requant_channels")
     return Cq
+
+
+def q4_conv2d_channels(X, Wt, d: ConvDesc, za: int, zb, mult, shift, zo: int, clamp_lo: int,
+                       clamp_hi: int, Y, bias=None, colsum_w=None):
+    """Fused convolution layer with per-output-channel weight zero points, multipliers and
+    shifts (CUDA int32 tensors of OC elements); see include/q4.h."""
+    _dev(X, torch.uint8, "X"); _dev(Wt, torch.uint8, "Wt"); _dev(Y, torch.uint8, "Y")
+    for t, n in ((zb, "zb"), (mult, "mult"), (shift, "shift"), (bias, "bias"), (colsum_w, "colsum_w")):
+        _dev(t, torch.int32, n)
+    c = d._c()
+    _check(_lib.q4_conv2d_channels(_ptr(X), _ptr(Wt), _rows(Wt, "Wt"), _ptr(colsum_w), _ptr(bias),
+                                   ctypes.byref(c), za, _ptr(zb), _ptr(mult), _ptr(shift), zo, clamp_lo,
+                                   clamp_hi, _ptr(Y), _stream()), "q4_conv2d_channels")
+    return Y
 
 
 def q4_row_sums(P, rows: int, K: int, sums):

@@ -400,6 +400,28 @@ q4_status q4_selftest_wait_timeout(int* outcome_dev, void* stream)
                ? Q4_OK : Q4_ERR_CUDA;
 }
 
+q4_status q4_conv2d_channels(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
+                             const int32_t* colsum_w, const int32_t* bias, const q4_conv_desc* d,
+                             int32_t za, const int32_t* zb, const int32_t* mult, const int32_t* shift,
+                             int32_t zo, int32_t clamp_lo, int32_t clamp_hi, uint8_t* Y, void* stream)
+{
+    q4_status s = check_conv(d, za);
+    if (s != Q4_OK) return s;
+    if (zo < 0 || zo > 15 || clamp_lo < 0 || clamp_hi > 15 || clamp_lo > clamp_hi) return Q4_ERR_RANGE;
+    if (d->OC < 0 || (d->OC & 1)) return Q4_ERR_INVALID_ARG;
+    const ConvShape cs = conv_shape(d);
+    if (ldw < ((int64_t)cs.K + 1) / 2) return Q4_ERR_INVALID_ARG;
+    if (cs.M == 0 || d->OC == 0) return Q4_OK;
+    if (!X || !Wt || !Y || !zb || !mult || !shift) return Q4_ERR_INVALID_ARG;
+    const void* words[] = {colsum_w, bias, zb, mult, shift};
+    for (const void* w : words)
+        if ((uintptr_t)w % 4) return Q4_ERR_ALIGNMENT;
+    if (!conv_fused_supported(*d, X, Wt, ldw, Y, true)) return Q4_ERR_UNSUPPORTED;
+    const RequantParams rqp{1 << 30, 2, zo, clamp_lo, clamp_hi};     // multiplier and shift come per channel
+    return launch_conv_fused(X, Wt, ldw, colsum_w, bias, *d, za, 0, rqp, Y, static_cast<cudaStream_t>(stream),
+                             zb, mult, shift) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+}
+
 q4_status q4_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, int32_t N, int32_t K,
                               int32_t za, const int32_t* rowsum_a,
                               const int32_t* zb, const int32_t* bias,

@@ -122,11 +122,14 @@ cudaError_t launch_operand_sums(const uint8_t* A, int64_t lda, int32_t rows_a, i
                                 const uint8_t* B, int64_t ldb, int32_t rows_b, int32_t* sums_b,
                                 int32_t K, cudaStream_t st);
 bool        conv_fused_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt,
-                                 int64_t ldw, const uint8_t* Y);
+                                 int64_t ldw, const uint8_t* Y, bool per_channel = false);
+// zb_ch / mult_ch / shift_ch: all three (per-output-channel weight zero points, multipliers
+// and shifts; zb and rq.mult / rq.shift are then unused) or none.
 cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                               const int32_t* colsum_w, const int32_t* bias, const q4_conv_desc& d,
                               int32_t za, int32_t zb, const RequantParams& rq, uint8_t* Y,
-                              cudaStream_t st);
+                              cudaStream_t st, const int32_t* zb_ch = nullptr,
+                              const int32_t* mult_ch = nullptr, const int32_t* shift_ch = nullptr);
 cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, uint8_t* A,
                           int64_t lda, int32_t* rowsum_a, cudaStream_t st);
 

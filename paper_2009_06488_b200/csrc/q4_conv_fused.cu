@@ -58,6 +58,10 @@ struct Params {
     int64_t ldw;
     const int32_t* colsum_w;   // optional
     const int32_t* bias;       // optional
+    // per output channel (all three or none): weight zero points, multipliers, shifts
+    const int32_t* zb_ch;
+    const int32_t* mult_ch;
+    const int32_t* shift_ch;
     uint8_t* Y;
     int64_t M;
     int32_t H, W, C, KH, KW, OH, OW, sh, sw, ph, pw;
@@ -355,7 +359,9 @@ constexpr int THREADS = (WARPS + 1) * 32;
 // to four CONSECUTIVE pixels 4g .. 4g + 3 instead of pixels eight apart -- which pixel an MMA
 // row stands for is free --, so a thread decodes one pixel per tile and the other three are
 // a constant step away.
-template <int NT, bool EXP, int KS_T = 0, bool CONSEC = false>
+// PC: every output channel has its own weight zero point and re-quantization multiplier
+// and shift (device arrays in the parameters) instead of the layer-wide ones.
+template <int NT, bool EXP, int KS_T = 0, bool CONSEC = false, bool PC = false>
 __global__ void __launch_bounds__(THREADS, NT <= 2 ? 4 : NT <= 4 ? 3 : 2)
 conv_fused_kernel(const Params p)
 {
@@ -368,7 +374,8 @@ conv_fused_kernel(const Params p)
     int32_t* tab = reinterpret_cast<int32_t*>(smem + (size_t)p.KS * NT * 32 * 8);    // [KS][TW]
     int32_t* colsum_s = tab + p.KS * TW;                                             // [N]
     constexpr int NB = NBUF_MMA;
-    int4* geo_s = reinterpret_cast<int4*>(colsum_s + N);                             // [NB]
+    int32_t* pc_s = colsum_s + N;                                                    // [2][N] multipliers, shifts (PC)
+    int4* geo_s = reinterpret_cast<int4*>(pc_s + 2 * N);                             // [NB]
     uint64_t* full_s = reinterpret_cast<uint64_t*>(geo_s + NB);                      // [NB] "tile landed"
     uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB) + SYNC_BYTES;             // 16-byte aligned
     const uint32_t full0 = smem_u32(full_s), empty0 = full0 + 8 * NB, abort_flag = full0 + 16 * NB;
@@ -381,6 +388,16 @@ conv_fused_kernel(const Params p)
     // ---- once per CTA: weights -> signed B fragments, depth table, weight sums, and
     //      the input buffers filled with the zero point (this is what stays in the halo)
     for (int i = tid; i < N; i += THREADS) colsum_s[i] = 0;
+    int pc_fast = 1;                                   // every channel's shift allows the 32-bit rounding
+    if (PC) {
+        int ok = 1;
+        for (int i = tid; i < N; i += THREADS) {
+            pc_s[i] = p.mult_ch[i];
+            pc_s[N + i] = p.shift_ch[i];
+            ok = ok && p.shift_ch[i] >= 2;
+        }
+        pc_fast = __syncthreads_and(ok);
+    }
     {
         const uint32_t zfill = (uint32_t)p.za * (EXP ? 0x01010101u : 0x11111111u);
         uint32_t* b = reinterpret_cast<uint32_t*>(buf0);
@@ -400,6 +417,7 @@ conv_fused_kernel(const Params p)
         const int l = i & 31, nt = (i >> 5) % NT, j = (i >> 5) / NT;
         const int fg = l >> 2, ft = l & 3;
         const int n = 2 * (NT * (fg >> 1) + nt) + (fg & 1);
+        const uint32_t zbn = PC ? (uint32_t)p.zb_ch[n] : (uint32_t)p.zb;
         uint32_t b0 = 0, b1 = 0;
         int raw = 0;
         if (!EXP) {
@@ -413,8 +431,8 @@ conv_fused_kernel(const Params p)
                     for (int q = 0; q < 4; ++q) w |= (uint32_t)p.Wt[(int64_t)n * p.ldw + kb + q] << (8 * q);
                 }
                 raw = nibble_sum(w);
-                b0 = sub_zb(w & 0x0F0F0F0Fu, (uint32_t)p.zb);
-                b1 = sub_zb((w >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                b0 = sub_zb(w & 0x0F0F0F0Fu, zbn);
+                b1 = sub_zb((w >> 4) & 0x0F0F0F0Fu, zbn);
             }
         } else {
 #pragma unroll
@@ -428,7 +446,7 @@ conv_fused_kernel(const Params p)
                         if (bs < segbytes) {
                             const uint32_t nib = weight_nibble(p, n, kh * segbytes + bs);
                             raw += (int)nib;
-                            word |= ((nib - (uint32_t)p.zb) & 0xFFu) << (8 * q);
+                            word |= ((nib - zbn) & 0xFFu) << (8 * q);
                         }
                     }
                 }
@@ -468,13 +486,13 @@ conv_fused_kernel(const Params p)
     // ---------------- consumers ----------------
     // per-thread epilogue constants: what is left of Eq. 3 for my NT channel pairs
     int colterm[NT][2];
-    const int kzz = p.K * p.za * p.zb;
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
             const int n = 2 * (NT * t + nt) + e;
             const int cs = p.colsum_w ? p.colsum_w[n] : colsum_s[n];
+            const int kzz = p.K * p.za * (PC ? p.zb_ch[n] : p.zb);
             colterm[nt][e] = (int)((uint32_t)kzz - (uint32_t)(p.za * cs) +
                                    (uint32_t)(p.bias ? p.bias[n] : 0));
         }
@@ -629,7 +647,18 @@ conv_fused_kernel(const Params p)
 #pragma unroll
                         for (int e = 0; e < 2; ++e) {
                             const int v = acc[mt][nt][2 * hrow + e];       // started from the column's constant
-                            if (FAST) {
+                            if (PC) {
+                                const int n = 2 * (NT * t + nt) + e;
+                                const int mlt = pc_s[n], sh = pc_s[N + n];
+                                if (FAST) {
+                                    int q = (mulhi_add(v, mlt, 1 << (sh - 2)) >> (sh - 1)) + p.rq.zo;
+                                    q = max(q, p.rq.lo);
+                                    qv[e] = (uint32_t)min(q, p.rq.hi);
+                                } else {
+                                    const RequantParams rqn{mlt, sh, p.rq.zo, p.rq.lo, p.rq.hi};
+                                    qv[e] = requant_wide(v, rqn);
+                                }
+                            } else if (FAST) {
                                 int q = (mulhi_add(v, p.rq.mult, rnd) >> s) + p.rq.zo;
                                 q = max(q, p.rq.lo);
                                 qv[e] = (uint32_t)min(q, p.rq.hi);
@@ -658,7 +687,7 @@ conv_fused_kernel(const Params p)
                 }
             };
             // the 32-bit form of the rounding shift needs shift >= 2 (see requant())
-            if (p.rq.shift >= 2) epilogue(std::true_type{}); else epilogue(std::false_type{});
+            if (PC ? pc_fast != 0 : p.rq.shift >= 2) epilogue(std::true_type{}); else epilogue(std::false_type{});
         }
         release_buffer(done_bar, lane);
     }
@@ -1012,7 +1041,7 @@ conv_quad_kernel(const Params p)
 // memory the kernel needs (0 = the layer does not fit this kernel).
 static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt,
                          int64_t ldw, const uint8_t* Y, bool& expanded, bool& per_lane, bool& nibbles,
-                         bool& quad)
+                         bool& quad, bool allow_lane = true)
 {
     if (d.OC % 8 != 0 || d.OC < 8 || d.OC > 64) return 0;
     if (d.KH > 64 || d.KW > 64 || d.stride_h > 64 || d.stride_w > 64) return 0;
@@ -1026,7 +1055,7 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     const int64_t segw = expanded ? ((int64_t)d.KW * d.C + 3) / 4 : 1;
     // thinnest layers: one pixel per lane, byte dot products (at most 128 per pixel); their
     // copy in shared memory stays packed when image rows are whole 32-bit words
-    per_lane = expanded && (d.OC == 8 || d.OC == 16) && (int64_t)d.KH * segw * d.OC <= 128;
+    per_lane = allow_lane && expanded && (d.OC == 8 || d.OC == 16) && (int64_t)d.KH * segw * d.OC <= 128;
     nibbles = per_lane && ((int64_t)d.W * d.C) % 8 == 0 && (uintptr_t)X % 4 == 0;
     // a gray-image first layer: four pixels per lane, four times the tile
     quad = nibbles && d.C == 1 && d.OC == 8 && d.KH == 3 && d.KW == 3 && d.stride_h == 1 &&
@@ -1056,7 +1085,7 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     const int64_t smem = per_lane
         ? (int64_t)d.KH * segw * d.OC * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_LANE + fused::SYNC_BYTES +
               fused::NBUF_LANE * bufbytes
-        : KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_MMA + fused::SYNC_BYTES +
+        : KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 12 + 16 * fused::NBUF_MMA + fused::SYNC_BYTES +
               fused::NBUF_MMA * bufbytes;
     if (smem > fused::SMEM_LIMIT) return 0;
     p.unit = (int32_t)unit; p.rowbytes = (int32_t)rowbytes; p.data0 = (int32_t)data0; p.pix0 = (int32_t)pix0;
@@ -1078,12 +1107,12 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
 }
 
 bool conv_fused_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt, int64_t ldw,
-                          const uint8_t* Y)
+                          const uint8_t* Y, bool per_channel)
 {
     if ((uintptr_t)Y % 8) return false;
     fused::Params p;
     bool expanded, per_lane, nibbles, quad;
-    return plan_fused(p, d, X, Wt, ldw, Y, expanded, per_lane, nibbles, quad) != 0;
+    return plan_fused(p, d, X, Wt, ldw, Y, expanded, per_lane, nibbles, quad, !per_channel) != 0;
 }
 
 // Launches one of the kernels above as persistent CTAs: as many as are resident at
@@ -1126,12 +1155,18 @@ static cudaError_t launch_ks(const fused::Params& p, size_t smem, int64_t tiles,
 template <int NT, bool EXP>
 static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
+    // per-channel parameters: the general instance
+    if (p.mult_ch) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 0, false, true>, p, smem, tiles, st);
     // 3x3 layers with 8, 16 or 32 input channels (3, 5, 9 depth steps) get instances with the
     // depth loop unrolled, for the channel counts the workloads pair them with
-    if constexpr (!EXP) {
-        if (p.KS == 3 && NT <= 2) return launch_ks<NT, 3>(p, smem, tiles, st);
-        if (p.KS == 5 && NT >= 2 && NT <= 4) return launch_ks<NT, 5>(p, smem, tiles, st);
-        if (p.KS == 9 && NT == 8) return launch_ks<NT, 9>(p, smem, tiles, st);
+    if constexpr (!EXP && NT <= 2) {
+        if (p.KS == 3) return launch_ks<NT, 3>(p, smem, tiles, st);
+    }
+    if constexpr (!EXP && NT >= 2 && NT <= 4) {
+        if (p.KS == 5) return launch_ks<NT, 5>(p, smem, tiles, st);
+    }
+    if constexpr (!EXP && NT == 8) {
+        if (p.KS == 9) return launch_ks<NT, 9>(p, smem, tiles, st);
     }
     return launch_kernel(fused::conv_fused_kernel<NT, EXP>, p, smem, tiles, st);
 }
@@ -1154,11 +1189,14 @@ static cudaError_t launch_mode(int NT, const fused::Params& p, size_t smem, int6
 cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                               const int32_t* colsum_w, const int32_t* bias, const q4_conv_desc& d,
                               int32_t za, int32_t zb, const RequantParams& rq, uint8_t* Y,
-                              cudaStream_t st)
+                              cudaStream_t st, const int32_t* zb_ch, const int32_t* mult_ch,
+                              const int32_t* shift_ch)
 {
     fused::Params p;
     bool expanded = false, per_lane = false, nibbles = false, quad = false;
-    const size_t smem = plan_fused(p, d, X, Wt, ldw, Y, expanded, per_lane, nibbles, quad);
+    // layers with per-channel parameters always take the MMA kernel
+    const size_t smem = plan_fused(p, d, X, Wt, ldw, Y, expanded, per_lane, nibbles, quad, mult_ch == nullptr);
+    p.zb_ch = zb_ch; p.mult_ch = mult_ch; p.shift_ch = shift_ch;
     if (smem == 0) return cudaErrorInvalidValue;
     p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;
     p.za = za; p.zb = zb; p.rq = rq;

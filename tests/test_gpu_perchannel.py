@@ -117,3 +117,51 @@ def test_argument_checks(q4):
     with pytest.raises(q4.Q4Error) as e:
         q4.q4_requant_channels(C0, 4, 8, 16, 0, v, None, None, None, v, 0, 0, 15, Cq)    # multipliers missing
     assert e.value.status == q4.Q4_ERR_INVALID_ARG
+
+
+CONV_PC = [  # N, H, W, C, OC, KH, KW, sh, sw, ph, pw
+    (3, 12, 14, 16, 24, 3, 3, 1, 1, 1, 1),      # packed copy
+    (4, 16, 16, 8, 16, 3, 3, 2, 2, 1, 1),       # packed copy, stride 2
+    (2, 20, 40, 32, 64, 3, 3, 1, 1, 1, 1),      # widest tile
+    (5, 16, 16, 1, 8, 3, 3, 1, 1, 1, 1),        # one input channel: expanded copy in the MMA kernel
+    (2, 11, 9, 3, 24, 3, 3, 1, 1, 1, 1),        # odd channel count
+    (40, 9, 10, 8, 40, 3, 3, 1, 1, 1, 1),       # many tiles
+]
+
+
+@pytest.mark.parametrize("g", CONV_PC)
+@pytest.mark.parametrize("shifts", [(0, 12), (2, 12)])
+def test_fused_conv_layer_with_per_channel_weights(q4, g, shifts):
+    import torch
+    N_, H, W, C, OC, KH, KW, sh, sw, ph, pw = g
+    dq, do = q4.ConvDesc(*g), oracle.ConvDesc(*g)
+    K = KH * KW * C
+    seed = 500 + sum(g)
+    X = wl.rand_flat_nibbles(seed, 1, N_ * H * W * C)
+    Wt = wl.rand_packed(seed, 2, OC, K)
+    zb, bias, mult, shift = channel_params(seed, OC, *shifts)
+    za = 9
+    lda = (K + 1) // 2
+    Ao, _ = oracle.im2col(X, do, za, lda)
+    want = oracle.requant_channels(oracle.gemm_channels(Ao, Wt, dq.M, OC, K, za, zb, bias), mult, shift, 2, 1, 14)
+    Xd = torch.zeros((X.size + 31) // 16 * 16, dtype=torch.uint8, device="cuda")
+    Xd[:X.size] = dev(X)
+    Y = torch.full((dq.M, OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
+    n0 = q4.q4_launch_count()
+    q4.q4_conv2d_channels(Xd, dev(Wt), dq, za, dev(zb), dev(mult), dev(shift), 2, 1, 14, Y, dev(bias))
+    assert q4.q4_launch_count() - n0 == 1
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    assert (Y.cpu().numpy() == want).all()
+
+
+def test_fused_per_channel_layer_rejects_what_the_kernel_does_not_take(q4):
+    import torch
+    g = (1, 8, 8, 16, 72, 3, 3, 1, 1, 1, 1)              # 72 output channels
+    dq = q4.ConvDesc(*g)
+    v = torch.zeros(72, dtype=torch.int32, device="cuda")
+    X = torch.zeros(1 * 8 * 8 * 8, dtype=torch.uint8, device="cuda")
+    Wt = torch.zeros((72, 72), dtype=torch.uint8, device="cuda")
+    Y = torch.zeros((dq.M, 36), dtype=torch.uint8, device="cuda")
+    with pytest.raises(q4.Q4Error) as e:
+        q4.q4_conv2d_channels(X, Wt, dq, 0, v, v, v, 0, 0, 15, Y)
+    assert e.value.status == q4.Q4_ERR_UNSUPPORTED
