@@ -150,3 +150,31 @@ def test_validation_of_the_float_boundary_and_the_8bit_product(lib):
     assert lib.q4_dequantize(fake, 7, 4, 8, 1.0, fake, 8, None) == INVALID
     assert lib.q4_dequantize(fake, 8, 4, 8, 1.0, fake + 1, 8, None) == ALIGN
     assert lib.q4_dequantize(fake, 8, 4, 0, 1.0, fake, 8, None) == 0
+
+
+def test_validation_of_the_per_channel_entry_points(lib):
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    fake = 0x1000
+    INVALID, ALIGN, RANGE = 1, 2, 3
+    lib.q4_requant_channels.argtypes = [vp, i64, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, i32, vp, i64, vp]
+    r = lambda **kw: lib.q4_requant_channels(kw.get("C0", fake), kw.get("ldc", 8), kw.get("M", 4), kw.get("N", 8),
+                                             kw.get("K", 16), kw.get("za", 0), kw.get("ra", fake), None, None,
+                                             kw.get("mult", fake), fake, kw.get("zo", 0), kw.get("lo", 0),
+                                             kw.get("hi", 15), fake, kw.get("ldcq", 4), None)
+    assert r(N=7) == INVALID and r(ldc=7) == INVALID and r(ldcq=3) == INVALID and r(K=0) == INVALID
+    assert r(za=16) == RANGE and r(zo=-1) == RANGE and r(lo=9, hi=8) == RANGE
+    assert r(mult=None) == INVALID and r(ra=None) == INVALID
+    assert r(C0=fake + 2) == ALIGN
+    assert r(M=0) == 0
+
+    lib.q4_conv2d_channels.argtypes = [vp, vp, i64, vp, vp, ctypes.POINTER(CD), i32, vp, vp, vp, i32, i32, i32, vp, vp]
+    c = lambda d, **kw: lib.q4_conv2d_channels(fake, fake, kw.get("ldw", 72), None, None, ctypes.byref(d),
+                                               kw.get("za", 0), kw.get("zb", fake), fake, fake, 0, 0,
+                                               kw.get("hi", 15), kw.get("Y", fake), None)
+    d = CD(2, 8, 8, 16, 32, 3, 3, 1, 1, 1, 1)
+    assert c(d, ldw=71) == INVALID and c(d, zb=None) == INVALID
+    assert c(d, za=16) == RANGE and c(d, hi=16) == RANGE
+    assert c(d, zb=fake + 2) == ALIGN
+    assert c(CD(2, 8, 8, 16, 72, 3, 3, 1, 1, 1, 1), ldw=72) == 5            # unsupported: 72 output channels
+    assert c(d, Y=fake + 4) == 5                                            # unsupported: Y not 8-byte aligned
+    assert c(CD(0, 8, 8, 16, 32, 3, 3, 1, 1, 1, 1)) == 0
