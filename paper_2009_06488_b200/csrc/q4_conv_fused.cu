@@ -666,20 +666,21 @@ conv_fused_kernel(const Params p)
                                 qv[e] = requant_wide(v, p.rq);
                             }
                         }
-                        bytes[nt] = qv[0] | (qv[1] << 4);
+                        bytes[nt] = mad_u32(qv[1], 16u, qv[0]);     // fields do not overlap: add = or
                     }
                     uint8_t* dst = ytile + (CONSEC ? i : 8 * i) * (N / 2);
                     if (NT % 4 == 0) {
 #pragma unroll
                         for (int q = 0; q < NT / 4; ++q)
                             reinterpret_cast<uint32_t*>(dst)[q] =
-                                bytes[(4 * q) % NT] | (bytes[(4 * q + 1) % NT] << 8) |
-                                (bytes[(4 * q + 2) % NT] << 16) | (bytes[(4 * q + 3) % NT] << 24);
+                                mad_u32(bytes[(4 * q + 3) % NT], 1u << 24,
+                                        mad_u32(bytes[(4 * q + 2) % NT], 1u << 16,
+                                                mad_u32(bytes[(4 * q + 1) % NT], 1u << 8, bytes[(4 * q) % NT])));
                     } else if (NT % 2 == 0) {
 #pragma unroll
                         for (int q = 0; q < NT / 2; ++q)
                             reinterpret_cast<uint16_t*>(dst)[q] =
-                                (uint16_t)(bytes[(2 * q) % NT] | (bytes[(2 * q + 1) % NT] << 8));
+                                (uint16_t)mad_u32(bytes[(2 * q + 1) % NT], 1u << 8, bytes[(2 * q) % NT]);
                     } else {
 #pragma unroll
                         for (int q = 0; q < NT; ++q) dst[q] = (uint8_t)bytes[q];
