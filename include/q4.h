@@ -334,6 +334,8 @@ q4_status q4_selftest_wait_timeout(int* outcome_dev, void* stream);
  * Process-wide; also read once from the environment variable Q4_FORCE_VARIANT
  * ("simt" / "tc" / "tc1"). */
 int q4_set_variant(int variant);
+/* With Q4_LOG=1 in the environment every GEMM / convolution call prints one line to stderr
+ * naming the kernel it was given. */
 
 /*
  * Measurement helper (no counterpart in the paper): the tensor pipe's issue peak on

@@ -1,6 +1,7 @@
 // C ABI of the q4 library (declared in q4.h): argument validation, kernel selection,
 // launch.  No allocation, no synchronization except where the header says so.
 #include <atomic>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 
@@ -14,6 +15,17 @@ static std::atomic<uint64_t> g_launches{0};
 static std::atomic<int> g_variant{-1};   // -1 = not read from the environment yet
 
 void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// Q4_LOG=1 in the environment: one line on stderr per call saying which kernel it was given.
+void log_choice(const char* call, const char* kernel)
+{
+    static int on = -1;
+    if (on < 0) {
+        const char* e = std::getenv("Q4_LOG");
+        on = (e && e[0] == '1') ? 1 : 0;
+    }
+    if (on) std::fprintf(stderr, "[q4] %s -> %s\n", call, kernel);
+}
 
 static int variant()
 {
@@ -102,6 +114,7 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
                     return Q4_ERR_CUDA;
                 p.rowsum_a = wa;
             }
+            log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "CTA-pair tcgen05 kernel, Bt expanded once per call");
             return launch_gemm_tc_pair(p, rq, st, b8, ld8);
         }
         if ((!p.rowsum_a || !p.colsum_b) && ws_ok && ws_bytes >= sums_bytes) {
@@ -111,10 +124,15 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
             if (do_a) p.rowsum_a = wa;
             if (do_b) p.colsum_b = wb;
         }
+        log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "CTA-pair tcgen05 kernel");
         return launch_gemm_tc_pair(p, rq, st);
     }
-    if (v != 1 && gemm_tc_supported(p)) return launch_gemm_tc(p, rq, st);
+    if (v != 1 && gemm_tc_supported(p)) {
+        log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "single-CTA tcgen05 kernel");
+        return launch_gemm_tc(p, rq, st);
+    }
     if (v == 2 || v == 3) return Q4_ERR_ALIGNMENT;
+    log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "general kernel (operands not aligned for TMA)");
     return launch_gemm_simt(p, rq, st) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
@@ -289,6 +307,7 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
         return run_gemm(p, true, st, ws, ws_bytes);
     }
 
+    log_choice("q4_conv2d", "explicit path: unroll into the workspace, then GEMM");
     uint8_t* A = static_cast<uint8_t*>(ws);
     int32_t* rowsum = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + cs.off_rowsum);
     if (launch_im2col(X, *d, za, A, cs.lda, rowsum, st) != cudaSuccess) return Q4_ERR_CUDA;

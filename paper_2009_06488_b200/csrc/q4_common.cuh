@@ -153,5 +153,6 @@ cudaError_t launch_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, i
                                     cudaStream_t st);
 
 void count_launch(int n = 1);
+void log_choice(const char* call, const char* kernel);   // Q4_LOG=1: which kernel a call was given
 
 }  // namespace q4

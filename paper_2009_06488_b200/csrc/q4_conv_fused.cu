@@ -1205,6 +1205,9 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     if (!p.status) return cudaErrorUnknown;
     if (p.M == 0) return cudaSuccess;
     const int64_t tiles = (p.M + p.tile - 1) / p.tile;
+    log_choice(mult_ch ? "q4_conv2d_channels" : "q4_conv2d",
+               quad ? "fused, four pixels per lane" : per_lane ? "fused, one pixel per lane"
+                    : expanded ? "fused implicit GEMM (MMA), expanded copy" : "fused implicit GEMM (MMA), packed copy");
     if (quad) return launch_kernel(fused::conv_quad_kernel, p, smem, tiles, st);
     if (per_lane) {
         // the 3x3 single-channel first layer gets its own fully unrolled instance

@@ -552,8 +552,11 @@ q4_status launch_gemm_u8(const GemmParams& g, cudaStream_t st)
 {
     // large problems: CTA pairs on 256 x 256 tiles (at least one tile per pair of SMs)
     if (g.M >= 256 && g.N >= 256 &&
-        (long long)((g.M + 255) / 256) * ((g.N + 255) / 256) >= sm_count_u8() / 2)
+        (long long)((g.M + 255) / 256) * ((g.N + 255) / 256) >= sm_count_u8() / 2) {
+        log_choice("q4_gemm_u8", "CTA-pair tcgen05 kernel");
         return launch_u8_pair(g, st);
+    }
+    log_choice("q4_gemm_u8", "single-CTA tcgen05 kernel");
     if (g.N > 128) return launch_u8_bn<256>(g, st);
     if (g.N > 64)  return launch_u8_bn<128>(g, st);
     return launch_u8_bn<64>(g, st);
