@@ -56,7 +56,7 @@ typedef enum {
     Q4_ERR_ALIGNMENT = 2,       /* a pointer / pitch breaks an alignment the call requires */
     Q4_ERR_RANGE = 3,           /* zero point, multiplier, shift, clamp or K out of range  */
     Q4_ERR_WORKSPACE = 4,       /* workspace missing or smaller than *_workspace_bytes     */
-    Q4_ERR_UNSUPPORTED = 5,     /* valid but not implemented (none at present)             */
+    Q4_ERR_UNSUPPORTED = 5,     /* valid, but this entry point has no kernel for it         */
     Q4_ERR_CUDA = 6,            /* a CUDA runtime / driver call failed                     */
     Q4_ERR_DEVICE_TIMEOUT = 7,  /* a bounded device-side wait expired                      */
     Q4_ERR_STATIC_SCRATCH = 8   /* problem needs more scratch than q4_conv2d_static holds  */
