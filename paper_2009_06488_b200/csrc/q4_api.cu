@@ -368,14 +368,10 @@ q4_status q4_gemm_u8(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t l
     if (!rowsum_a || !colsum_b) {
         int32_t* sa = static_cast<int32_t*>(ws);
         int32_t* sb = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + round256(4 * (size_t)M));
-        if (!rowsum_a) {
-            if (launch_byte_sums(A, lda, M, K, sa, st) != cudaSuccess) return Q4_ERR_CUDA;
-            p.rowsum_a = sa;
-        }
-        if (!colsum_b) {
-            if (launch_byte_sums(Bt, ldb, N, K, sb, st) != cudaSuccess) return Q4_ERR_CUDA;
-            p.colsum_b = sb;
-        }
+        if (launch_byte_sums(A, lda, rowsum_a ? 0 : M, sa, Bt, ldb, colsum_b ? 0 : N, sb, K, st) != cudaSuccess)
+            return Q4_ERR_CUDA;
+        if (!rowsum_a) p.rowsum_a = sa;
+        if (!colsum_b) p.colsum_b = sb;
     }
     return launch_gemm_u8(p, st);
 }

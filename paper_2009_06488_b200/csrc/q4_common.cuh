@@ -141,7 +141,10 @@ cudaError_t launch_dequantize(const int32_t* C, int64_t ldc, int32_t rows, int32
                               float* R, int64_t ldr, cudaStream_t st);
 
 q4_status   launch_gemm_u8(const GemmParams& p, cudaStream_t st);
-cudaError_t launch_byte_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K, int32_t* sums,
+// depth sums of the rows of A and of Bt (one byte per value) in one launch; rows_a or rows_b
+// may be 0
+cudaError_t launch_byte_sums(const uint8_t* A, int64_t lda, int32_t rows_a, int32_t* sums_a,
+                             const uint8_t* B, int64_t ldb, int32_t rows_b, int32_t* sums_b, int32_t K,
                              cudaStream_t st);
 
 cudaError_t launch_wait_selftest(int* outcome_dev, cudaStream_t st);

@@ -211,37 +211,52 @@ gemm_u8_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
-// sums[r] = sum of the K bytes of row r: a warp per row, 16-byte loads, bytes past K masked.
+// sums[r] = sum of the K bytes of row r, for the rows of A and then those of Bt in one launch:
+// a warp per row, 16-byte loads, four of them in flight per lane, bytes past K masked.
+__device__ __forceinline__ int masked_chunk_sum(uint4 v, int valid, int s)
+{
+    if (valid < 16) {
+        uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int vb = valid - 4 * e;              // valid bytes of word e
+            if (vb <= 0) w[e] = 0;
+            else if (vb < 4) w[e] &= (1u << (8 * vb)) - 1u;
+        }
+        v = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    s = dp4a_u8(v.x, 0x01010101u, s);
+    s = dp4a_u8(v.y, 0x01010101u, s);
+    s = dp4a_u8(v.z, 0x01010101u, s);
+    return dp4a_u8(v.w, 0x01010101u, s);
+}
+
 __global__ void __launch_bounds__(256)
-byte_sums_kernel(const uint8_t* __restrict__ P, int64_t ld, int32_t rows, int32_t K, int32_t* __restrict__ sums)
+byte_sums_kernel(const uint8_t* __restrict__ A, int64_t lda, int32_t rows_a, int32_t* __restrict__ sums_a,
+                 const uint8_t* __restrict__ B, int64_t ldb, int32_t rows_b, int32_t* __restrict__ sums_b,
+                 int32_t K)
 {
     const int lane = threadIdx.x & 31;
     const int chunks = (K + 15) / 16;
-    for (int64_t r = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); r < rows;
+    const int64_t total = (int64_t)rows_a + rows_b;
+    for (int64_t r = blockIdx.x * (int64_t)(blockDim.x >> 5) + (threadIdx.x >> 5); r < total;
          r += (int64_t)gridDim.x * (blockDim.x >> 5)) {
-        const uint4* row = reinterpret_cast<const uint4*>(P + r * ld);
+        const bool second = r >= rows_a;
+        const int64_t rr = second ? r - rows_a : r;
+        const uint4* row = reinterpret_cast<const uint4*>(second ? B + rr * ldb : A + rr * lda);
         int s = 0;
-        for (int c = lane; c < chunks; c += 32) {
-            uint4 v = row[c];
-            const int valid = K - 16 * c;              // bytes of this chunk inside the row
-            if (valid < 16) {
-                uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const int vb = valid - 4 * e;      // valid bytes of word e
-                    if (vb <= 0) w[e] = 0;
-                    else if (vb < 4) w[e] &= (1u << (8 * vb)) - 1u;
-                }
-                v = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            s = dp4a_u8(v.x, 0x01010101u, s);
-            s = dp4a_u8(v.y, 0x01010101u, s);
-            s = dp4a_u8(v.z, 0x01010101u, s);
-            s = dp4a_u8(v.w, 0x01010101u, s);
+        int c = lane;
+        for (; c + 96 < chunks; c += 128) {            // four loads in flight
+            const uint4 v0 = row[c], v1 = row[c + 32], v2 = row[c + 64], v3 = row[c + 96];
+            s = masked_chunk_sum(v0, K - 16 * c, s);
+            s = masked_chunk_sum(v1, K - 16 * (c + 32), s);
+            s = masked_chunk_sum(v2, K - 16 * (c + 64), s);
+            s = masked_chunk_sum(v3, K - 16 * (c + 96), s);
         }
+        for (; c < chunks; c += 32) s = masked_chunk_sum(row[c], K - 16 * c, s);
 #pragma unroll
         for (int off = 16; off; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
-        if (lane == 0) sums[r] = s;
+        if (lane == 0) (second ? sums_b : sums_a)[rr] = s;
     }
 }
 
@@ -471,13 +486,15 @@ static int sm_count_u8()
     return n;
 }
 
-cudaError_t launch_byte_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K, int32_t* sums,
+cudaError_t launch_byte_sums(const uint8_t* A, int64_t lda, int32_t rows_a, int32_t* sums_a,
+                             const uint8_t* B, int64_t ldb, int32_t rows_b, int32_t* sums_b, int32_t K,
                              cudaStream_t st)
 {
+    const int64_t rows = (int64_t)rows_a + rows_b;
     if (rows == 0) return cudaSuccess;
-    int blocks = (rows + 7) / 8;
+    int64_t blocks = (rows + 7) / 8;
     if (blocks > 148 * 8) blocks = 148 * 8;
-    u8::byte_sums_kernel<<<blocks, 256, 0, st>>>(P, ld, rows, K, sums);
+    u8::byte_sums_kernel<<<(int)blocks, 256, 0, st>>>(A, lda, rows_a, sums_a, B, ldb, rows_b, sums_b, K);
     count_launch();
     return cudaGetLastError();
 }
