@@ -86,6 +86,25 @@ __global__ void finalize_kernel(int* range)
     range[1] = z;
 }
 
+// floor(fl(w / s)) -- the floor of the CORRECTLY ROUNDED binary32 quotient, which is what Eq. 1's
+// code is defined by here -- without a division for almost every value.  With r = fl(1 / s)
+// and x = fl(w * r): |x - fl(w / s)| <= (2^-23 + 2^-24) |w / s| (two roundings on one side, one
+// on the other), so floor(x) is the wanted floor unless x lies within that distance of an
+// integer; only then (and for a zero product, whose sign may have been lost to underflow) is
+// the division carried out.  The test distance is 1e-6 |x|, five times the bound.  `fast` is
+// false for scales so small or large that r would overflow or be subnormal.
+__device__ __forceinline__ int floor_quotient(float w, float s, float r, bool fast)
+{
+    if (fast) {
+        const float x = __fmul_rn(w, r);
+        const float fx = floorf(x);
+        const float d = __fsub_rn(x, fx);                      // exact, in [0, 1)
+        const float thr = 1e-6f * fmaxf(fabsf(x), 1.0f);
+        if (!(d < thr) && !(d > 1.0f - thr)) return __float2int_rd(fx);
+    }
+    return __float2int_rd(__fdiv_rn(w, s));
+}
+
 // Rows are walked by blockIdx.y, the 32-bit words of a row by blockIdx.x and the thread
 // index: no divisions.  A dense matrix is passed as one row.
 __global__ void __launch_bounds__(256)
@@ -94,6 +113,8 @@ quantize_vec_kernel(const float* __restrict__ X, int64_t ldx, int32_t rows, int6
 {
     const float s = qp->scale;
     const int z = qp->zero;
+    const bool fast = s > 1e-30f && s < 1e30f;
+    const float rs = __frcp_rn(s);
     for (int64_t r = blockIdx.y; r < rows; r += gridDim.y) {
         const float* xr = X + r * ldx;
         uint8_t* qr = Q + r * ldq;
@@ -105,7 +126,7 @@ quantize_vec_kernel(const float* __restrict__ X, int64_t ldx, int32_t rows, int6
             uint32_t word = 0;
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                int q = __float2int_rd(__fdiv_rn(v[e], s));
+                int q = floor_quotient(v[e], s, rs, fast);
                 q = min(max(q, -z), 15 - z) + z;       // clamp before adding: no overflow
                 word |= (uint32_t)q << (4 * e);
             }
@@ -120,6 +141,8 @@ quantize_byte_kernel(const float* __restrict__ X, int64_t ldx, int32_t rows, int
 {
     const float s = qp->scale;
     const int z = qp->zero;
+    const bool fast = s > 1e-30f && s < 1e30f;
+    const float rs = __frcp_rn(s);
     const int kb = (cols + 1) / 2;
     const int64_t total = (int64_t)rows * kb;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
@@ -131,7 +154,7 @@ quantize_byte_kernel(const float* __restrict__ X, int64_t ldx, int32_t rows, int
         for (int e = 0; e < 2; ++e) {
             const int c = 2 * j + e;
             if (c < cols) {
-                int q = __float2int_rd(__fdiv_rn(X[r * ldx + c], s));
+                int q = floor_quotient(X[r * ldx + c], s, rs, fast);
                 q = min(max(q, -z), 15 - z) + z;
                 byte |= (uint32_t)q << (4 * e);
             }

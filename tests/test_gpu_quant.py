@@ -179,3 +179,34 @@ def oracle_layer(L, X):
     do = oracle.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
     return oracle.conv2d(X, L.Wt, L.bias, do, L.za, L.zb,
                          oracle.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi))
+
+
+@pytest.mark.parametrize("scale", [0.37, 1.0 / 3.0, 7.3e-5, 1234.567, 0.25, 3.0e-39, 2.5e38, 1.1754944e-38])
+def test_codes_at_the_integer_boundaries_of_the_quotient(q4, scale):
+    """Inputs that sit on, and a few units in the last place around, every multiple of the
+    scale: where the floor of the rounded quotient is decided by the last bit (the kernel's
+    division-free path must hand exactly these to the exact division)."""
+    import torch
+    s = np.float32(scale)
+    k = np.arange(-24, 25, dtype=np.float32)
+    with np.errstate(over="ignore"):
+        base = (k * s).astype(np.float32)               # infinities (largest scale) are replaced below
+    vals = [base]
+    for _ in range(4):
+        vals.append(np.nextafter(vals[-1], np.float32(np.inf)).astype(np.float32))
+    lo = base
+    for _ in range(4):
+        lo = np.nextafter(lo, np.float32(-np.inf)).astype(np.float32)
+        vals.append(lo)
+    X = np.concatenate(vals + [np.array([0.0, -0.0, 1e-45, -1e-45], np.float32)])
+    X = np.resize(X, (X.size + 7) // 8 * 8).reshape(1, -1)
+    z = 7
+    words = np.array([s.view(np.int32), z], dtype=np.int32)
+    with np.errstate(over="ignore", invalid="ignore"):
+        want = oracle.quantize(np.where(np.isfinite(X), X, 0).astype(np.float32), s, z)
+    Xf = np.where(np.isfinite(X), X, 0).astype(np.float32)
+    for cols in (Xf.shape[1], Xf.shape[1] - 3):              # word path and byte path
+        Q = torch.zeros((1, (cols + 1) // 2), dtype=torch.uint8, device="cuda")
+        q4.q4_quantize(dev(Xf[:, :cols]), dev(words), Q)
+        with np.errstate(over="ignore", invalid="ignore"):
+            assert (Q.cpu().numpy() == oracle.quantize(Xf[:, :cols], s, z)).all()
