@@ -43,7 +43,16 @@ range_kernel(const float* __restrict__ X, int64_t ldx, int32_t rows, int32_t col
         // dense, 16-byte aligned: the matrix is one array of rows * cols floats
         const int64_t n4 = (int64_t)rows * cols / 4;
         const float4* X4 = reinterpret_cast<const float4*>(X);
-        for (int64_t i = tid; i < n4; i += nthreads) {
+        int64_t i = tid;
+        for (; i + 3 * nthreads < n4; i += 4 * nthreads) {     // four loads in flight
+            const float4 a = __ldcs(X4 + i), b = __ldcs(X4 + i + nthreads), c = __ldcs(X4 + i + 2 * nthreads),
+                         d = __ldcs(X4 + i + 3 * nthreads);
+            lo = fminf(lo, fminf(fminf(fminf(a.x, a.y), fminf(a.z, a.w)), fminf(fminf(b.x, b.y), fminf(b.z, b.w))));
+            lo = fminf(lo, fminf(fminf(fminf(c.x, c.y), fminf(c.z, c.w)), fminf(fminf(d.x, d.y), fminf(d.z, d.w))));
+            hi = fmaxf(hi, fmaxf(fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)), fmaxf(fmaxf(b.x, b.y), fmaxf(b.z, b.w))));
+            hi = fmaxf(hi, fmaxf(fmaxf(fmaxf(c.x, c.y), fmaxf(c.z, c.w)), fmaxf(fmaxf(d.x, d.y), fmaxf(d.z, d.w))));
+        }
+        for (; i < n4; i += nthreads) {
             const float4 v = X4[i];
             lo = fminf(fminf(lo, v.x), fminf(v.y, fminf(v.z, v.w)));
             hi = fmaxf(fmaxf(hi, v.x), fmaxf(v.y, fmaxf(v.z, v.w)));
