@@ -881,6 +881,7 @@ conv_lane_kernel(const Params p)
 constexpr int QUAD = 4;
 constexpr int QUAD_TILE = QUAD * ROWS_PER_CTA;
 
+template <bool PC>
 __global__ void __launch_bounds__(THREADS, 4)
 conv_quad_kernel(const Params p)
 {
@@ -889,7 +890,8 @@ conv_quad_kernel(const Params p)
     uint32_t* wsm = reinterpret_cast<uint32_t*>(smem);                               // [KH][OC]
     int32_t* colterm_s = reinterpret_cast<int32_t*>(wsm + KH * OC);                  // [OC]
     constexpr int NB = NBUF_LANE;
-    int4* geo_s = reinterpret_cast<int4*>(colterm_s + OC);                           // [NB]
+    int32_t* pc_s = colterm_s + OC;                                                  // [2][OC] multipliers, shifts (PC)
+    int4* geo_s = reinterpret_cast<int4*>(pc_s + 2 * OC);                            // [NB]
     uint64_t* full_s = reinterpret_cast<uint64_t*>(geo_s + NB);                      // [NB] "tile landed"
     uint8_t* buf0 = reinterpret_cast<uint8_t*>(geo_s + NB) + SYNC_BYTES;             // 16-byte aligned
     const uint32_t full0 = smem_u32(full_s), empty0 = full0 + 8 * NB, abort_flag = full0 + 16 * NB;
@@ -920,7 +922,7 @@ conv_quad_kernel(const Params p)
         for (int q = 0; q < 3; ++q) {
             const uint32_t nib = weight_nibble(p, n, kh * 3 + q);
             raw += (int)nib;
-            word |= ((nib - (uint32_t)p.zb) & 0xFFu) << (8 * q);
+            word |= ((nib - (PC ? (uint32_t)p.zb_ch[n] : (uint32_t)p.zb)) & 0xFFu) << (8 * q);
         }
         wsm[i] = word;                                 // fourth byte 0: the window's next nibble counts for nothing
         if (!p.colsum_w && raw) atomicAdd(&colterm_s[n], raw);
@@ -928,9 +930,14 @@ conv_quad_kernel(const Params p)
     __syncthreads();
     if (tid < OC) {
         const int cs = p.colsum_w ? p.colsum_w[tid] : colterm_s[tid];
-        colterm_s[tid] = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
+        colterm_s[tid] = (int)((uint32_t)(p.K * p.za * (PC ? p.zb_ch[tid] : p.zb)) - (uint32_t)(p.za * cs) +
                                (uint32_t)(p.bias ? p.bias[tid] : 0));
+        if (PC) {
+            pc_s[tid] = p.mult_ch[tid];
+            pc_s[OC + tid] = p.shift_ch[tid];
+        }
     }
+    const int pc_fast = PC ? __syncthreads_and(tid >= OC || p.shift_ch[tid] >= 2) : 1;
     __syncthreads();
 
     const int64_t ntiles = (p.M + QUAD_TILE - 1) / QUAD_TILE;
@@ -1006,7 +1013,34 @@ conv_quad_kernel(const Params p)
             }
 
             uint32_t out[QUAD];
-            if (p.rq.shift >= 2) {
+            if (PC) {
+                int mlt[OC], shf_n[OC];
+                {
+                    const int4 m0 = *reinterpret_cast<const int4*>(pc_s), m1 = *reinterpret_cast<const int4*>(pc_s + 4);
+                    const int4 s0 = *reinterpret_cast<const int4*>(pc_s + 8), s1 = *reinterpret_cast<const int4*>(pc_s + 12);
+                    mlt[0] = m0.x; mlt[1] = m0.y; mlt[2] = m0.z; mlt[3] = m0.w;
+                    mlt[4] = m1.x; mlt[5] = m1.y; mlt[6] = m1.z; mlt[7] = m1.w;
+                    shf_n[0] = s0.x; shf_n[1] = s0.y; shf_n[2] = s0.z; shf_n[3] = s0.w;
+                    shf_n[4] = s1.x; shf_n[5] = s1.y; shf_n[6] = s1.z; shf_n[7] = s1.w;
+                }
+#pragma unroll
+                for (int px = 0; px < QUAD; ++px) {
+                    uint32_t o = 0;
+#pragma unroll
+                    for (int n = 0; n < OC; ++n) {
+                        uint32_t qv;
+                        if (pc_fast) {
+                            int q = (mulhi_add(acc[px][n], mlt[n], 1 << (shf_n[n] - 2)) >> (shf_n[n] - 1)) + p.rq.zo;
+                            qv = (uint32_t)min(max(q, p.rq.lo), p.rq.hi);
+                        } else {
+                            const RequantParams rqn{mlt[n], shf_n[n], p.rq.zo, p.rq.lo, p.rq.hi};
+                            qv = requant_wide(acc[px][n], rqn);
+                        }
+                        o = n == 0 ? qv : mad_u32(qv, 1u << (4 * n), o);
+                    }
+                    out[px] = o;
+                }
+            } else if (p.rq.shift >= 2) {
                 // the 32-bit form of the rounding shift (see requant())
 #pragma unroll
                 for (int px = 0; px < QUAD; ++px) {
@@ -1056,11 +1090,14 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     const int64_t segw = expanded ? ((int64_t)d.KW * d.C + 3) / 4 : 1;
     // thinnest layers: one pixel per lane, byte dot products (at most 128 per pixel); their
     // copy in shared memory stays packed when image rows are whole 32-bit words
-    per_lane = allow_lane && expanded && (d.OC == 8 || d.OC == 16) && (int64_t)d.KH * segw * d.OC <= 128;
+    per_lane = expanded && (d.OC == 8 || d.OC == 16) && (int64_t)d.KH * segw * d.OC <= 128;
     nibbles = per_lane && ((int64_t)d.W * d.C) % 8 == 0 && (uintptr_t)X % 4 == 0;
     // a gray-image first layer: four pixels per lane, four times the tile
     quad = nibbles && d.C == 1 && d.OC == 8 && d.KH == 3 && d.KW == 3 && d.stride_h == 1 &&
            d.stride_w == 1 && p.OW % 4 == 0 && (uintptr_t)Y % 16 == 0;
+    // per-channel parameters: the four-pixel kernel and the MMA kernel have instances for them,
+    // the pixel-per-lane kernel has not
+    if (!allow_lane && !quad) per_lane = nibbles = false;
     p.tile = quad ? fused::QUAD_TILE : fused::ROWS_PER_CTA;
     int64_t unit, rowbytes, data0, pix0, pitch;
     if (nibbles) {
@@ -1084,7 +1121,7 @@ static size_t plan_fused(fused::Params& p, const q4_conv_desc& d, const uint8_t*
     const int64_t bufbytes = slots * pitch + 16;       // the slack takes the unaligned words' over-read
     const int64_t KS = expanded ? ((int64_t)d.KH * segw + 7) / 8 : ((int64_t)p.K + 31) / 32;
     const int64_t smem = per_lane
-        ? (int64_t)d.KH * segw * d.OC * 4 + (int64_t)d.OC * 4 + 16 * fused::NBUF_LANE + fused::SYNC_BYTES +
+        ? (int64_t)d.KH * segw * d.OC * 4 + (int64_t)d.OC * 12 + 16 * fused::NBUF_LANE + fused::SYNC_BYTES +
               fused::NBUF_LANE * bufbytes
         : KS * (d.OC / 8) * 256 + KS * (expanded ? 8 : 4) * 4 + (int64_t)d.OC * 12 + 16 * fused::NBUF_MMA + fused::SYNC_BYTES +
               fused::NBUF_MMA * bufbytes;
@@ -1148,6 +1185,11 @@ static cudaError_t launch_kernel(FusedKernel kernel, const fused::Params& p, siz
 template <int NT, int KS>
 static cudaError_t launch_ks(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
+    if (p.mult_ch) {
+        if (p.OW % 4 == 0)
+            return launch_kernel(fused::conv_fused_kernel<NT, false, KS, true, true>, p, smem, tiles, st);
+        return launch_kernel(fused::conv_fused_kernel<NT, false, KS, false, true>, p, smem, tiles, st);
+    }
     if (p.OW % 4 == 0)
         return launch_kernel(fused::conv_fused_kernel<NT, false, KS, true>, p, smem, tiles, st);
     return launch_kernel(fused::conv_fused_kernel<NT, false, KS, false>, p, smem, tiles, st);
@@ -1156,8 +1198,6 @@ static cudaError_t launch_ks(const fused::Params& p, size_t smem, int64_t tiles,
 template <int NT, bool EXP>
 static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles, cudaStream_t st)
 {
-    // per-channel parameters: the general instance
-    if (p.mult_ch) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 0, false, true>, p, smem, tiles, st);
     // 3x3 layers with 8, 16 or 32 input channels (3, 5, 9 depth steps) get instances with the
     // depth loop unrolled, for the channel counts the workloads pair them with
     if constexpr (!EXP && NT <= 2) {
@@ -1169,6 +1209,7 @@ static cudaError_t launch_nt(const fused::Params& p, size_t smem, int64_t tiles,
     if constexpr (!EXP && NT == 8) {
         if (p.KS == 9) return launch_ks<NT, 9>(p, smem, tiles, st);
     }
+    if (p.mult_ch) return launch_kernel(fused::conv_fused_kernel<NT, EXP, 0, false, true>, p, smem, tiles, st);
     return launch_kernel(fused::conv_fused_kernel<NT, EXP>, p, smem, tiles, st);
 }
 
@@ -1208,7 +1249,9 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     log_choice(mult_ch ? "q4_conv2d_channels" : "q4_conv2d",
                quad ? "fused, four pixels per lane" : per_lane ? "fused, one pixel per lane"
                     : expanded ? "fused implicit GEMM (MMA), expanded copy" : "fused implicit GEMM (MMA), packed copy");
-    if (quad) return launch_kernel(fused::conv_quad_kernel, p, smem, tiles, st);
+    if (quad)
+        return mult_ch ? launch_kernel(fused::conv_quad_kernel<true>, p, smem, tiles, st)
+                       : launch_kernel(fused::conv_quad_kernel<false>, p, smem, tiles, st);
     if (per_lane) {
         // the 3x3 single-channel first layer gets its own fully unrolled instance
         if (nibbles && d.OC == 8 && d.KH == 3 && p.segw == 1)
