@@ -138,6 +138,14 @@ __device__ __forceinline__ int mulhi_add(int a, int b, int c)
     return d;
 }
 
+// clamp(q + zo, lo, hi) - lo = max(min(q + (zo - lo), hi - lo), 0): one instruction (add, min
+// and the lower clamp at zero fused).  The kernels keep this value per nibble and add lo to
+// all nibbles of a packed word at once (no carries: value + lo <= hi <= 15).
+__device__ __forceinline__ uint32_t clamp_above_lo(int q, int zo_minus_lo, int hi_minus_lo)
+{
+    return (uint32_t)__viaddmin_s32_relu(q, zo_minus_lo, hi_minus_lo);
+}
+
 // a * b + c in one instruction (the compiler otherwise splits a shift-and-or into two).
 __device__ __forceinline__ uint32_t mad_u32(uint32_t a, uint32_t b, uint32_t c)
 {
@@ -636,6 +644,8 @@ conv_fused_kernel(const Params p)
             auto epilogue = [&](auto fast_tag) {
                 constexpr bool FAST = decltype(fast_tag)::value;
                 const int s = p.rq.shift - 1, rnd = FAST ? 1 << (s - 1) : 0;
+                const int zml = p.rq.zo - p.rq.lo, hml = p.rq.hi - p.rq.lo;
+                const uint32_t lofill = (uint32_t)p.rq.lo * 0x11111111u;     // lo in every nibble
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
                     const int mt = i >> 1, hrow = i & 1;
@@ -651,19 +661,15 @@ conv_fused_kernel(const Params p)
                                 const int n = 2 * (NT * t + nt) + e;
                                 const int mlt = pc_s[n], sh = pc_s[N + n];
                                 if (FAST) {
-                                    int q = (mulhi_add(v, mlt, 1 << (sh - 2)) >> (sh - 1)) + p.rq.zo;
-                                    q = max(q, p.rq.lo);
-                                    qv[e] = (uint32_t)min(q, p.rq.hi);
+                                    qv[e] = clamp_above_lo(mulhi_add(v, mlt, 1 << (sh - 2)) >> (sh - 1), zml, hml);
                                 } else {
                                     const RequantParams rqn{mlt, sh, p.rq.zo, p.rq.lo, p.rq.hi};
-                                    qv[e] = requant_wide(v, rqn);
+                                    qv[e] = requant_wide(v, rqn) - (uint32_t)p.rq.lo;
                                 }
                             } else if (FAST) {
-                                int q = (mulhi_add(v, p.rq.mult, rnd) >> s) + p.rq.zo;
-                                q = max(q, p.rq.lo);
-                                qv[e] = (uint32_t)min(q, p.rq.hi);
+                                qv[e] = clamp_above_lo(mulhi_add(v, p.rq.mult, rnd) >> s, zml, hml);
                             } else {
-                                qv[e] = requant_wide(v, p.rq);
+                                qv[e] = requant_wide(v, p.rq) - (uint32_t)p.rq.lo;
                             }
                         }
                         bytes[nt] = mad_u32(qv[1], 16u, qv[0]);     // fields do not overlap: add = or
@@ -675,15 +681,16 @@ conv_fused_kernel(const Params p)
                             reinterpret_cast<uint32_t*>(dst)[q] =
                                 mad_u32(bytes[(4 * q + 3) % NT], 1u << 24,
                                         mad_u32(bytes[(4 * q + 2) % NT], 1u << 16,
-                                                mad_u32(bytes[(4 * q + 1) % NT], 1u << 8, bytes[(4 * q) % NT])));
+                                                mad_u32(bytes[(4 * q + 1) % NT], 1u << 8,
+                                                        bytes[(4 * q) % NT] + lofill)));
                     } else if (NT % 2 == 0) {
 #pragma unroll
                         for (int q = 0; q < NT / 2; ++q)
                             reinterpret_cast<uint16_t*>(dst)[q] =
-                                (uint16_t)mad_u32(bytes[(2 * q + 1) % NT], 1u << 8, bytes[(2 * q) % NT]);
+                                (uint16_t)mad_u32(bytes[(2 * q + 1) % NT], 1u << 8, bytes[(2 * q) % NT] + lofill);
                     } else {
 #pragma unroll
-                        for (int q = 0; q < NT; ++q) dst[q] = (uint8_t)bytes[q];
+                        for (int q = 0; q < NT; ++q) dst[q] = (uint8_t)(bytes[q] + lofill);
                     }
                 }
             };
@@ -954,6 +961,8 @@ conv_quad_kernel(const Params p)
     const uint32_t M32 = (uint32_t)p.M, mstep = gridDim.x * (uint32_t)QUAD_TILE;
     uint32_t mbase = blockIdx.x * (uint32_t)QUAD_TILE;
     const int s = p.rq.shift - 1, rnd = s > 0 ? 1 << (s - 1) : 0;
+    const int zml = p.rq.zo - p.rq.lo, hml = p.rq.hi - p.rq.lo;
+    const uint32_t lofill = (uint32_t)p.rq.lo * 0x11111111u;         // lo in every nibble
     int kb = 0;                                        // k % NB
     uint32_t phase = 0;                                // (k / NB) % 2
     for (int k = 0; k < mytiles; ++k, mbase += mstep) {
@@ -1030,15 +1039,15 @@ conv_quad_kernel(const Params p)
                     for (int n = 0; n < OC; ++n) {
                         uint32_t qv;
                         if (pc_fast) {
-                            int q = (mulhi_add(acc[px][n], mlt[n], 1 << (shf_n[n] - 2)) >> (shf_n[n] - 1)) + p.rq.zo;
-                            qv = (uint32_t)min(max(q, p.rq.lo), p.rq.hi);
+                            qv = clamp_above_lo(mulhi_add(acc[px][n], mlt[n], 1 << (shf_n[n] - 2)) >> (shf_n[n] - 1),
+                                                zml, hml);
                         } else {
                             const RequantParams rqn{mlt[n], shf_n[n], p.rq.zo, p.rq.lo, p.rq.hi};
-                            qv = requant_wide(acc[px][n], rqn);
+                            qv = requant_wide(acc[px][n], rqn) - (uint32_t)p.rq.lo;
                         }
                         o = n == 0 ? qv : mad_u32(qv, 1u << (4 * n), o);
                     }
-                    out[px] = o;
+                    out[px] = o + lofill;
                 }
             } else if (p.rq.shift >= 2) {
                 // the 32-bit form of the rounding shift (see requant())
@@ -1047,11 +1056,10 @@ conv_quad_kernel(const Params p)
                     uint32_t o = 0;
 #pragma unroll
                     for (int n = 0; n < OC; ++n) {
-                        int qv = (mulhi_add(acc[px][n], p.rq.mult, rnd) >> s) + p.rq.zo;
-                        qv = min(max(qv, p.rq.lo), p.rq.hi);
-                        o = n == 0 ? (uint32_t)qv : mad_u32((uint32_t)qv, 1u << (4 * n), o);   // nibble fields do not overlap
+                        const uint32_t qv = clamp_above_lo(mulhi_add(acc[px][n], p.rq.mult, rnd) >> s, zml, hml);
+                        o = n == 0 ? qv : mad_u32(qv, 1u << (4 * n), o);   // nibble fields do not overlap
                     }
-                    out[px] = o;
+                    out[px] = o + lofill;
                 }
             } else {
 #pragma unroll
