@@ -3,7 +3,7 @@
 // per-row sums of Eq. 2's second term taken on the way (Section II-B).
 //
 // Three kernels:
-//  * im2col_tile_kernel -- same geometry as the next one, output pitch up to 256 bytes:
+//  * im2col_tile_kernel -- same geometry as the next one, output pitch up to 1024 bytes:
 //    a warp takes 32 consecutive output rows, one row per lane.  A lane decodes its
 //    pixel once, walks its row's taps (the lanes' loads of one tap are consecutive
 //    pixels of the input: coalesced), sums its row's values in a register and writes
@@ -134,8 +134,9 @@ __global__ void __launch_bounds__(256) im2col_vec_kernel(const Im2colParams p, i
 }
 
 // One output row per lane, 32 rows per warp and step; see the head of the file.
-constexpr int TILE_WARPS = 8;
-constexpr int TILE_MAX_LDA = 256;
+constexpr int TILE_WARPS = 8;             // warps per block at pitches up to 256 bytes; fewer above
+constexpr int TILE_SMEM = TILE_WARPS * 32 * 256;   // 64 KB of tiles per block
+constexpr int TILE_MAX_LDA = 1024;        // two warps per block at least; longer rows: next kernel
 
 template <int TAPB>
 __global__ void __launch_bounds__(TILE_WARPS * 32)
@@ -151,8 +152,8 @@ im2col_tile_kernel(const Im2colParams p, int tapb, FastDiv div_ow, FastDiv div_o
     const int64_t groups = ((int64_t)M + 31) / 32;
     const int64_t imgbytes = (int64_t)p.H * p.W * tapb;
 
-    for (int64_t gi = (int64_t)blockIdx.x * TILE_WARPS + warp; gi < groups;
-         gi += (int64_t)gridDim.x * TILE_WARPS) {
+    const int wpb = blockDim.x >> 5;                     // warps per block
+    for (int64_t gi = (int64_t)blockIdx.x * wpb + warp; gi < groups; gi += (int64_t)gridDim.x * wpb) {
         const uint32_t m0 = (uint32_t)(gi * 32);
         const bool valid = m0 + lane < M;
         const uint32_t m = valid ? m0 + lane : m0;      // lanes past the end redo row m0 (not stored)
@@ -279,21 +280,23 @@ cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, u
     const bool vec = aligned && (d.C % 2 == 0) && (tapb == 4 || tapb == 8 || tapb % 16 == 0);
 
     if (vec && lda <= TILE_MAX_LDA && p.M < (1ll << 31)) {
-        const size_t smem = (size_t)TILE_WARPS * 32 * (size_t)lda;
+        // as many warps per block (up to eight) as fit 64 KB of row tiles
+        int wpb = (int)(TILE_SMEM / (32 * lda));
+        wpb = wpb < 1 ? 1 : wpb > TILE_WARPS ? TILE_WARPS : wpb;
+        const size_t smem = (size_t)wpb * 32 * (size_t)lda;
         const FastDiv dow = make_fastdiv((uint32_t)p.OW), doh = make_fastdiv((uint32_t)p.OH);
         auto kernel = tapb == 4 ? im2col_tile_kernel<4> : tapb == 8 ? im2col_tile_kernel<8>
                                                                    : im2col_tile_kernel<16>;
-        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             TILE_WARPS * 32 * TILE_MAX_LDA);
+        cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, TILE_SMEM);
         if (e != cudaSuccess) return e;
         int per_sm = 1;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, TILE_WARPS * 32, smem) !=
-                cudaSuccess || per_sm < 1)
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, wpb * 32, smem) != cudaSuccess ||
+            per_sm < 1)
             per_sm = 1;
         const int64_t groups = (p.M + 31) / 32;
-        int64_t blocks = (groups + TILE_WARPS - 1) / TILE_WARPS;
+        int64_t blocks = (groups + wpb - 1) / wpb;
         if (blocks > 148ll * per_sm) blocks = 148ll * per_sm;
-        kernel<<<(int)blocks, TILE_WARPS * 32, smem, st>>>(p, tapb, dow, doh);
+        kernel<<<(int)blocks, wpb * 32, smem, st>>>(p, tapb, dow, doh);
         count_launch();
         return cudaGetLastError();
     }

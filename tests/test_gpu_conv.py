@@ -42,6 +42,8 @@ IM2COL = [  # N, H, W, C, KH, KW, stride_h, stride_w, pad_h, pad_w
     (5, 19, 17, 16, 3, 3, 1, 1, 1, 1),     # 1615 rows: many 32-row tiles and a ragged last one
     (7, 21, 13, 8, 3, 3, 2, 2, 1, 1),      # 4-byte taps, stride 2, 539 rows
     (3, 9, 11, 32, 3, 3, 1, 1, 1, 1),      # 16-byte taps, pitch 144
+    (2, 9, 9, 128, 3, 3, 1, 1, 1, 1),      # pitch 576: tile kernel with three warps per block
+    (1, 4, 4, 256, 3, 3, 1, 1, 1, 1),      # pitch 1152: beyond the tile kernel, chunk-per-thread kernel
 ]
 
 
