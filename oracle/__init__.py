@@ -22,7 +22,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libq4ref.so")
 _SOURCES = [os.path.join(_HERE, "q4ref.c"), os.path.join(_HERE, "q4ref.h")]
 
-OK, E_ARG, E_RANGE, E_IDENTITY, E_PAD = 0, -1, -2, -3, -4
+OK, E_ARG, E_RANGE, E_PAD = 0, -1, -2, -4
 
 
 class OracleError(RuntimeError):

@@ -42,7 +42,6 @@ extern "C" {
 #define Q4REF_OK          0
 #define Q4REF_E_ARG      -1   /* bad size / pointer / pitch                        */
 #define Q4REF_E_RANGE    -2   /* value outside its documented range                */
-#define Q4REF_E_IDENTITY -3   /* Eq. 2 four-term form disagreed with the definition */
 #define Q4REF_E_PAD      -4   /* odd-K row whose last high nibble is not zero      */
 
 typedef struct {

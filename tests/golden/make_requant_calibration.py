@@ -1,4 +1,4 @@
-"""Writes tests/golden/requant_calibration.json: per-layer (mult, shift) for the conv
+"""Writes paper_2009_06488_b200/requant_calibration.json (read by workloads.py): per-layer (mult, shift) for the conv
 workloads c3 and c4, chosen from the CPU oracle's int32 accumulators on a small
 batch so that the 4-bit outputs spread over their range instead of saturating.
 
@@ -45,7 +45,7 @@ def main():
         table[f"c4_seed{seed}"] = calibrate(wl.c4(batch=8, seed=seed, requant=[(1 << 30, 5)] * 5))
     table["c4_centred"] = calibrate(wl.c4(batch=8, seed=4000, centred=True,
                                           requant=[(1 << 30, 5)] * 5))
-    path = os.path.join(ROOT, "tests", "golden", "requant_calibration.json")
+    path = os.path.join(ROOT, "paper_2009_06488_b200", "requant_calibration.json")
     with open(path, "w") as f:
         json.dump(table, f, indent=1)
         f.write("\n")

@@ -229,11 +229,22 @@ def test_c2_4096_sampled_rows_and_freivalds(q4):
     rows = np.unique(np.concatenate([np.arange(0, 4096, 97), [0, 127, 128, 4095]]))
     sampled_rows_check(c, got, rows)
     freivalds_check(c, got)
-    # requantized output on the same sampled rows
+    # The int32 matrix is now known to equal the oracle's (sampled rows + exact Freivalds on
+    # every entry), so the oracle's requantizer applied to it is the expected packed output
+    # for the WHOLE matrix: every tile of every cluster, not a sample.
     rq = oracle.Requant(c.mult, c.shift, 0, 0, 15)
     gotq = run_requant(q4, c, TC, rq)
-    wantq = oracle.requant_matrix(np.ascontiguousarray(got[rows]), None, rq)
-    assert (gotq[rows] == wantq).all()
+    assert (gotq == oracle.requant_matrix(got, None, rq)).all()
+    # bias, a non-zero output zero point and a ReLU-style lower clamp on the same product
+    # (the bias also re-centres the accumulators, whose mean follows the drawn zero points)
+    bias = (wl.rand_ints(c.seed, 9, -512, 512, c.N) - int(got.mean())).astype(np.int32)
+    span = max(1, int(np.abs(got.astype(np.int64) + bias[None, :]).max()))
+    shift2 = min(31, max(0, int(np.ceil(np.log2(span / 8.0)))))       # outputs spread over the code range
+    rq2 = oracle.Requant(c.mult, shift2, 8, 3, 14)
+    gotq2 = run_requant(q4, c, TC, rq2, bias, use_ws=True)
+    wantq2 = oracle.requant_matrix(got, bias, rq2)
+    assert (gotq2 == wantq2).all()
+    assert len(np.unique(oracle.unpack_rows(wantq2[:64], c.N))) > 3      # not saturated everywhere
 
 
 def big_case_check(q4, c, nrows):
@@ -253,8 +264,10 @@ def test_c2_8192_benchmark_shape(q4):
     got, rows = big_case_check(q4, c, 40)
     rq = oracle.Requant(c.mult, c.shift, 0, 0, 15)
     gotq = run_requant(q4, c, 0, rq, use_ws=True)
-    wantq = oracle.requant_matrix(np.ascontiguousarray(got[rows]), None, rq)
-    assert (gotq[rows] == wantq).all()
+    # whole packed matrix against the oracle's requantizer on the verified accumulators:
+    # this is the only size at which a cluster of the fused-requant kernel owns several
+    # tiles in a row
+    assert (gotq == oracle.requant_matrix(got, None, rq)).all()
 
 
 def test_c5_deep_k_worst_case_zero_points(q4):

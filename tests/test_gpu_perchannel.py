@@ -123,7 +123,12 @@ CONV_PC = [  # N, H, W, C, OC, KH, KW, sh, sw, ph, pw
     (3, 12, 14, 16, 24, 3, 3, 1, 1, 1, 1),      # packed copy
     (4, 16, 16, 8, 16, 3, 3, 2, 2, 1, 1),       # packed copy, stride 2
     (2, 20, 40, 32, 64, 3, 3, 1, 1, 1, 1),      # widest tile
-    (5, 16, 16, 1, 8, 3, 3, 1, 1, 1, 1),        # one input channel: expanded copy in the MMA kernel
+    (5, 16, 16, 1, 8, 3, 3, 1, 1, 1, 1),        # gray-image first layer: four pixels per lane
+    (9, 48, 48, 1, 8, 3, 3, 1, 1, 1, 1),        # ... tiles over two images
+    (4, 20, 32, 1, 8, 3, 3, 1, 1, 1, 1),        # ... rows copied by bulk copies (16-byte rows)
+    (6, 10, 24, 1, 8, 3, 3, 1, 1, 0, 1),        # ... no vertical padding
+    (3, 16, 40, 1, 8, 3, 3, 1, 1, 1, 3),        # ... horizontal padding of three
+    (5, 12, 20, 1, 8, 3, 3, 1, 1, 0, 0),        # output rows not groups of four: expanded copy, MMA kernel
     (2, 11, 9, 3, 24, 3, 3, 1, 1, 1, 1),        # odd channel count
     (40, 9, 10, 8, 40, 3, 3, 1, 1, 1, 1),       # many tiles
 ]

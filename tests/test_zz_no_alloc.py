@@ -1,9 +1,12 @@
 """q4_conv2d_static: the convolution entry point for callers that cannot allocate
 device memory (no cudaMalloc available to them: a plugin without an allocator, a
-fixed-pool process, a loop whose owner forbids allocator calls).  Its scratch is a
-fixed array inside the library, shared by all calls, so the check is: same bytes as
-q4_conv2d with a caller-provided workspace, on two calls in a row with different
-layers (the second call finds the first call's leftovers in the array).
+fixed-pool process, a loop whose owner forbids allocator calls).  Its scratch -- the
+unrolled matrix and its row sums -- is a fixed array inside the library, shared by all
+calls.  The layers here are ones the single-kernel fused path does not take (six and
+seventy-two output channels, a 1x1 layer), so every call really unrolls into that array
+and multiplies from it; the checks are the oracle's bytes and q4_conv2d's bytes with a
+caller-provided workspace, on calls in a row with different layers (each later call
+finds the earlier calls' leftovers in the array, beyond and between its own rows).
 
 Collected last on purpose: a run that stops at the first failure has then already
 run every other test.
@@ -11,6 +14,7 @@ run every other test.
 import numpy as np
 import pytest
 
+import oracle
 from paper_2009_06488_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -28,33 +32,48 @@ def layer(seed, N, H, W, C, OC, k, s, p):
         wl.rand_flat_nibbles(seed, 1, N * H * W * C)
 
 
-def test_static_scratch_entry_point_matches_q4_conv2d_twice_in_a_row():
+# N, H, W, C, OC, k, stride, pad -- a large layer first, then smaller ones with other
+# pitches and row counts; the last is a 1x1 layer large enough for the big-GEMM kernel: its
+# unrolled matrix is the input itself and the array holds only the depth sums that a
+# pre-pass writes and the GEMM reads
+LAYERS = ((900, (6, 32, 32, 16, 72, 3, 1, 1)),
+          (901, (3, 17, 13, 8, 6, 3, 2, 1)),
+          (902, (2, 9, 11, 3, 6, 5, 1, 2)),
+          (903, (74, 16, 16, 32, 384, 1, 1, 0)))
+
+
+def test_static_scratch_entry_point_matches_oracle_and_q4_conv2d_on_calls_in_a_row():
     import torch
     from paper_2009_06488_b200 import binding as q4
     q4.q4_set_variant(0)
-    # second layer is smaller and has another pitch: stale bytes of the first call
-    # lie beyond and between its rows
-    for seed, geom in ((900, (4, 32, 32, 16, 32, 3, 1, 1)), (901, (3, 17, 13, 8, 16, 3, 2, 1))):
+    for seed, geom in LAYERS:
         L, X = layer(seed, *geom)
-        d = q4.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
+        args = (L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
+        d = q4.ConvDesc(*args)
         rq = q4.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi)
         Xd, Wd, bd = dev(X), dev(L.Wt), dev(L.bias)
         assert q4.q4_conv2d_workspace_bytes(d) <= q4.Q4_STATIC_SCRATCH_BYTES
         ws = torch.empty(q4.q4_conv2d_workspace_bytes(d), dtype=torch.uint8, device="cuda")
-        want = torch.full((d.M, L.OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
-        q4.q4_conv2d(Xd, Wd, d, L.za, L.zb, rq, want, ws, bd)
+        other = torch.full((d.M, L.OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
+        q4.q4_conv2d(Xd, Wd, d, L.za, L.zb, rq, other, ws, bd)
         got = torch.full((d.M, L.OC // 2), 0x5A, dtype=torch.uint8, device="cuda")
+        n0 = q4.q4_launch_count()
         q4.q4_conv2d_static(Xd, Wd, d, L.za, L.zb, rq, got, bd)
+        # more than one kernel: the scratch array was written (unroll or sums) and read back
+        assert q4.q4_launch_count() - n0 >= 2
         torch.cuda.synchronize()
         assert q4.q4_last_device_status() == q4.Q4_OK
-        assert torch.equal(got, want)          # integer path: bit-exact
-        assert len(torch.unique(got)) > 3
+        want = oracle.conv2d(X, L.Wt, L.bias, oracle.ConvDesc(*args), L.za, L.zb,
+                             oracle.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi))
+        assert (got.cpu().numpy() == want).all()      # integer path: bit-exact
+        assert torch.equal(got, other)
+        assert len(np.unique(want)) > 3
 
 
 def test_static_scratch_rejects_layers_beyond_its_size():
     import torch
     from paper_2009_06488_b200 import binding as q4
-    L, X = layer(902, 256, 32, 32, 16, 32, 3, 1, 1)       # needs ~21 MB of scratch
+    L, X = layer(904, 256, 32, 32, 16, 32, 3, 1, 1)       # needs ~21 MB of scratch
     d = q4.ConvDesc(L.N, L.H, L.W, L.C, L.OC, L.KH, L.KW, L.stride, L.stride, L.pad, L.pad)
     assert q4.q4_conv2d_workspace_bytes(d) > q4.Q4_STATIC_SCRATCH_BYTES
     Y = torch.zeros((d.M, L.OC // 2), dtype=torch.uint8, device="cuda")
