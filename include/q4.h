@@ -330,9 +330,10 @@ q4_status q4_selftest_wait_timeout(int* outcome_dev, void* stream);
 
 /* Kernel selection for ablations and tests: 0 = automatic, 1 = general (SIMT)
  * kernels only, 2 = tensor-core kernels or an error where their alignment rules do
- * not hold, 3 = like 2 but never the CTA-pair kernel.  Returns the previous value.
- * Process-wide; also read once from the environment variable Q4_FORCE_VARIANT
- * ("simt" / "tc" / "tc1"). */
+ * not hold, 3 = like 2 but never the CTA-pair kernel, 4 = automatic except that
+ * convolution layers skip the tensor-memory (tcgen05) fused kernel and take the warp-level
+ * fused kernels.  Returns the previous value.  Process-wide; also read once from the
+ * environment variable Q4_FORCE_VARIANT ("simt" / "tc" / "tc1" / "fused1"). */
 int q4_set_variant(int variant);
 /* With Q4_LOG=1 in the environment every GEMM / convolution call prints one line to stderr
  * naming the kernel it was given. */

@@ -16,7 +16,8 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libq4.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]
+              "-Xcompiler", "-fPIC", "-cudart", "static"]
+OBJ_DIR = os.path.join(HERE, "_build")
 
 
 def sources() -> list[str]:
@@ -28,17 +29,35 @@ def _deps() -> list[str]:
     return sources() + hdrs + [os.path.join(INCLUDE, "q4.h")]
 
 
+def _headers() -> list[str]:
+    return [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cuh", ".h"))] + \
+           [os.path.join(INCLUDE, "q4.h")]
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    stale = force or not os.path.exists(LIB) or any(
-        os.path.getmtime(s) > os.path.getmtime(LIB) for s in _deps())
-    if stale:
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    """One object per source file (compiled in parallel, rebuilt when the source or any
+    header is newer), then one link step."""
+    from concurrent.futures import ThreadPoolExecutor
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(OBJ_DIR, exist_ok=True)
+    hdr_time = max(os.path.getmtime(h) for h in _headers())
+    jobs, objs = [], []
+    for src in sources():
+        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        objs.append(obj)
+        if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time):
+            cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-c", "-o", obj, src]
+            if verbose:
+                cmd[1:1] = ["-Xptxas", "-v"]
+            jobs.append(cmd)
+    if jobs:
+        with ThreadPoolExecutor(max_workers=min(8, len(jobs))) as pool:
+            for rc in pool.map(subprocess.call, jobs):
+                if rc != 0:
+                    raise subprocess.CalledProcessError(rc, "nvcc")
+    if jobs or not os.path.exists(LIB):
         tmp = LIB + f".tmp{os.getpid()}"
-        cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-o", tmp, *sources()]
-        if verbose:
-            cmd.insert(1, "-Xptxas")
-            cmd.insert(2, "-v")
-        subprocess.check_call(cmd)
+        subprocess.check_call([nvcc, *NVCC_FLAGS, "-shared", "-o", tmp, *objs])
         os.replace(tmp, LIB)
     return LIB
 

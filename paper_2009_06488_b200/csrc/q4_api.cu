@@ -36,6 +36,7 @@ static int variant()
         if (e && !std::strcmp(e, "simt")) v = 1;
         if (e && !std::strcmp(e, "tc")) v = 2;
         if (e && !std::strcmp(e, "tc1")) v = 3;
+        if (e && !std::strcmp(e, "fused1")) v = 4;
         g_variant.store(v, std::memory_order_relaxed);
     }
     return v;
@@ -284,9 +285,16 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     // Layers whose geometry allows it run as one fused kernel that never writes the
-    // unrolled matrix (variants 1 and 3 keep the explicit unroll + GEMM path testable).
+    // unrolled matrix (variants 1 and 3 keep the explicit unroll + GEMM path testable):
+    // on the tensor-memory path where it has an instance for the layer (variant 4 skips
+    // it), else on the warp-level kernels.
     const int v = variant();
-    if ((v == 0 || v == 2) && conv_fused_supported(*d, X, Wt, ldw, Y)) {
+    if ((v == 0 || v == 2) && conv_tc_supported(*d, X, Wt, ldw, Y)) {
+        const RequantParams rqp{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
+        return launch_conv_tc(X, Wt, ldw, colsum_w, bias, *d, za, zb, rqp, Y, st) == cudaSuccess
+                   ? Q4_OK : Q4_ERR_CUDA;
+    }
+    if ((v == 0 || v == 2 || v == 4) && conv_fused_supported(*d, X, Wt, ldw, Y)) {
         const RequantParams rqp{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
         return launch_conv_fused(X, Wt, ldw, colsum_w, bias, *d, za, zb, rqp, Y, st) == cudaSuccess
                    ? Q4_OK : Q4_ERR_CUDA;
@@ -298,7 +306,7 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     // straight to the GEMM; the workspace then only holds the depth sums.
     const bool whole_image = d->KH == d->H && d->KW == d->W;
     const bool pointwise = d->KH == 1 && d->KW == 1 && d->stride_h == 1 && d->stride_w == 1;
-    if (v == 0 && d->pad_h == 0 && d->pad_w == 0 && (whole_image || pointwise) &&
+    if ((v == 0 || v == 4) && d->pad_h == 0 && d->pad_w == 0 && (whole_image || pointwise) &&
         cs.K % 2 == 0) {
         p.A = X; p.Bt = Wt; p.lda = cs.K / 2; p.ldb = ldw; p.M = (int32_t)cs.M; p.N = d->OC; p.K = cs.K;
         p.za = za; p.zb = zb; p.rowsum_a = nullptr; p.colsum_b = colsum_w; p.bias = bias;
@@ -532,7 +540,7 @@ q4_status q4_last_device_status(void* stream)
 int q4_set_variant(int v)
 {
     const int prev = variant();
-    g_variant.store((v >= 1 && v <= 3) ? v : 0, std::memory_order_relaxed);
+    g_variant.store((v >= 1 && v <= 4) ? v : 0, std::memory_order_relaxed);
     return prev;
 }
 

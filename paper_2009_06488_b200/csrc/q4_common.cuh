@@ -130,6 +130,13 @@ cudaError_t launch_conv_fused(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                               int32_t za, int32_t zb, const RequantParams& rq, uint8_t* Y,
                               cudaStream_t st, const int32_t* zb_ch = nullptr,
                               const int32_t* mult_ch = nullptr, const int32_t* shift_ch = nullptr);
+// The same layer on the tensor-memory path (tcgen05 implicit GEMM), for the layer classes
+// it has instances for.
+bool        conv_tc_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt, int64_t ldw,
+                              const uint8_t* Y);
+cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, const int32_t* colsum_w,
+                           const int32_t* bias, const q4_conv_desc& d, int32_t za, int32_t zb,
+                           const RequantParams& rq, uint8_t* Y, cudaStream_t st);
 cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, uint8_t* A,
                           int64_t lda, int32_t* rowsum_a, cudaStream_t st);
 

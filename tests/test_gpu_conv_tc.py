@@ -1,0 +1,113 @@
+"""GPU parity of the tensor-memory (tcgen05) fused convolution kernel against the CPU
+oracle, byte for byte: every layer class it has an instance for, with tiles that end in the
+middle of a row / an image / the batch, several images per tile, one image over many tiles,
+vertical paddings and strides it takes at run time, given and derived weight sums, the
+32-bit and the 64-bit rounding path, and saturating clamps."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2009_06488_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def q4():
+    from paper_2009_06488_b200 import binding
+    binding.q4_set_variant(0)
+    return binding
+
+
+def dev(a):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+TC_LAYERS = [  # N, H, W, C, OC, stride, pad_h, shift
+    (2, 8, 8, 1, 8, 1, 1, 5),          # gray first layer, less than one tile
+    (5, 48, 48, 1, 8, 1, 1, 5),        # ... tiles that end inside an image
+    (70, 12, 16, 1, 8, 1, 1, 1),       # ... many images per tile, 64-bit rounding path
+    (3, 20, 32, 1, 8, 1, 0, 6),        # ... no vertical padding
+    (3, 48, 48, 8, 16, 2, 1, 5),       # 8 -> 16, stride 2 (c4 L2 geometry)
+    (37, 10, 16, 8, 16, 2, 1, 0),      # ... several images per tile, shift 0
+    (2, 9, 40, 8, 16, 2, 0, 5),        # ... odd height, no vertical padding
+    (5, 24, 24, 16, 32, 2, 1, 5),      # 16 -> 32, stride 2 (c4 L3)
+    (40, 6, 8, 16, 32, 2, 1, 4),       # ... tiny images
+    (9, 12, 12, 32, 64, 2, 1, 6),      # 32 -> 64, stride 2 (c4 L4)
+    (2, 30, 20, 32, 64, 2, 1, 1),
+    (3, 32, 32, 16, 32, 1, 1, 5),      # 16 -> 32, stride 1 (c3)
+    (1, 7, 12, 16, 32, 1, 1, 5),       # ... less than one tile
+    (21, 5, 8, 16, 32, 1, 0, 3),       # ... several images per tile, no vertical padding
+    (1, 200, 64, 16, 32, 1, 1, 5),     # ... one image over many tiles
+]
+
+
+@pytest.mark.parametrize("g", TC_LAYERS)
+@pytest.mark.parametrize("given_sums", [False, True])
+def test_tensor_memory_conv_kernel_matches_oracle(q4, g, given_sums):
+    import torch
+    N, H, W, C, OC, s, ph, shift = g
+    seed = 9000 + sum(g)
+    args = (N, H, W, C, OC, 3, 3, s, s, ph, 1)
+    dq, do = q4.ConvDesc(*args), oracle.ConvDesc(*args)
+    K = 9 * C
+    X = wl.rand_flat_nibbles(seed, 1, N * H * W * C)
+    Wt = wl.rand_packed(seed, 2, OC, K)
+    bias = wl.rand_ints(seed, 3, -300, 300, OC).astype(np.int32) if given_sums else None
+    za, zb = (int(v) for v in wl.rand_ints(seed, 4, 0, 15, 2))
+    rq = ((1 << 30) + 987654321 % (1 << 30), shift, 3, 1, 14)
+    want = oracle.conv2d(X, Wt, bias, do, za, zb, oracle.Requant(*rq))
+    Xd = torch.zeros((X.size + 31) // 16 * 16, dtype=torch.uint8, device="cuda")
+    Xd[:X.size] = dev(X)
+    ws = torch.empty(q4.q4_conv2d_workspace_bytes(dq), dtype=torch.uint8, device="cuda")
+    Y = torch.full((dq.M + 64, OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
+    colsum = None
+    if given_sums:
+        colsum = dev(oracle.unpack_rows(Wt, K).astype(np.int64).sum(axis=1).astype(np.int32))
+    n0 = q4.q4_launch_count()
+    q4.q4_conv2d(Xd[:X.size], dev(Wt), dq, za, zb, q4.Requant(*rq), Y[:dq.M], ws,
+                 None if bias is None else dev(bias), colsum)
+    assert q4.q4_launch_count() - n0 == 1            # one fused kernel, no unrolled matrix
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    out = Y.cpu().numpy()
+    assert (out[:dq.M] == want).all()
+    assert (out[dq.M:] == 0xA5).all()                # nothing written past the last pixel
+    # the warp-level fused kernels (variant 4) give the same bytes
+    q4.q4_set_variant(4)
+    try:
+        Y2 = torch.full((dq.M, OC // 2), 0x5A, dtype=torch.uint8, device="cuda")
+        q4.q4_conv2d(Xd[:X.size], dev(Wt), dq, za, zb, q4.Requant(*rq), Y2, ws,
+                     None if bias is None else dev(bias), colsum)
+        assert (Y2.cpu().numpy() == want).all()
+    finally:
+        q4.q4_set_variant(0)
+
+
+def test_which_layers_take_the_tensor_memory_kernel(q4, capfd):
+    """The kernel's instances are chosen by layer class; everything else keeps its path."""
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import torch\n"
+        "from paper_2009_06488_b200 import binding as q4\n"
+        "def run(*a):\n"
+        "    d = q4.ConvDesc(*a)\n"
+        "    X = torch.zeros(d.N*d.H*d.W*d.C//2 + 16, dtype=torch.uint8, device='cuda')\n"
+        "    Wt = torch.zeros((d.OC, (d.K + 1)//2), dtype=torch.uint8, device='cuda')\n"
+        "    Y = torch.zeros((d.M, d.OC//2), dtype=torch.uint8, device='cuda')\n"
+        "    ws = torch.empty(q4.q4_conv2d_workspace_bytes(d), dtype=torch.uint8, device='cuda')\n"
+        "    q4.q4_conv2d(X, Wt, d, 1, 2, q4.Requant(1 << 30, 4, 0, 0, 15), Y, ws)\n"
+        "run(2, 32, 32, 16, 32, 3, 3, 1, 1, 1, 1)\n"     # c3 class
+        "run(2, 32, 31, 16, 32, 3, 3, 1, 1, 1, 1)\n"     # output rows not whole groups of pixels
+        "run(2, 32, 32, 16, 24, 3, 3, 1, 1, 1, 1)\n"     # another channel count
+        "torch.cuda.synchronize()\n")
+    env = dict(os.environ, Q4_LOG="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, env=env, cwd=root)
+    assert r.returncode == 0, r.stderr
+    lines = [l for l in r.stderr.splitlines() if l.startswith("[q4] q4_conv2d")]
+    assert len(lines) == 3
+    assert "tcgen05" in lines[0]
+    assert "tcgen05" not in lines[1] and "tcgen05" not in lines[2]
