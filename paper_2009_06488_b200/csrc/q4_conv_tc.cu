@@ -269,20 +269,45 @@ __device__ __forceinline__ void producer(const Params& p, int mytiles, int nb, i
     }
 }
 
-// Eight accumulators -> eight re-quantized nibbles of one 32-bit word (value - lo per
-// nibble; the caller adds lo to all nibbles at once).
+// Saturating pack of two 32-bit integers into the signed 16-bit halves of one register.
+__device__ __forceinline__ uint32_t pack_sat16(int hi, int lo)
+{
+    uint32_t d;
+    asm("cvt.pack.sat.s16.s32 %0, %1, %2;" : "=r"(d) : "r"(hi), "r"(lo));
+    return d;
+}
+
+// Position c of a group of eight accumulator columns holds output channel ch8(c) of the
+// group: a register pair (columns 2i, 2i+1) then holds channels i and i+4, which lets the
+// epilogue clamp two values per instruction in 16-bit halves and gather the four pairs
+// into one word of eight nibbles with three multiply-adds.
+__host__ __device__ constexpr int ch8(int c) { return (c >> 1) + 4 * (c & 1); }
+
+// Eight accumulators (columns in the ch8 order) -> the eight re-quantized nibbles of one
+// 32-bit word, channel k in nibble k.  Fast form (shift >= 2, see requant(); and shift <= 27
+// so that the output zero point can ride in the rounding constant): the caller passes
+// rnd = 2^(s-1) + ((zo - lo) << s), so (mulhi + rnd) >> s is already q + zo - lo; two such
+// values are packed with saturation into 16-bit halves and clamped to [0, hi - lo] by one
+// instruction.  The result holds value - lo per nibble; the caller adds lo to all nibbles.
 template <bool FAST>
 __device__ __forceinline__ uint32_t requant8(const uint32_t* r, const RequantParams& rq, int s, int rnd,
-                                             int zml, int hml)
+                                             uint32_t hml2)
 {
+    if (FAST) {
+        uint32_t c[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int q0 = fused::mulhi_add((int)r[2 * i], rq.mult, rnd) >> s;
+            const int q1 = fused::mulhi_add((int)r[2 * i + 1], rq.mult, rnd) >> s;
+            c[i] = __vimin_s16x2_relu(pack_sat16(q1, q0), hml2);
+        }
+        // c[i] = channel i | channel (i + 4) << 16, each 0..15
+        return fused::mad_u32(c[3], 1u << 12, fused::mad_u32(c[2], 1u << 8, fused::mad_u32(c[1], 1u << 4, c[0])));
+    }
     uint32_t o = 0;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        uint32_t qv;
-        if (FAST) qv = fused::clamp_above_lo(fused::mulhi_add((int)r[e], rq.mult, rnd) >> s, zml, hml);
-        else qv = requant_wide((int)r[e], rq) - (uint32_t)rq.lo;
-        o = e == 0 ? qv : fused::mad_u32(qv, 1u << (4 * e), o);      // nibble fields do not overlap
-    }
+    for (int e = 0; e < 8; ++e)
+        o |= (requant_wide((int)r[e], rq) - (uint32_t)rq.lo) << (4 * ch8(e));
     return o;
 }
 
@@ -332,6 +357,13 @@ conv_tc_kernel(const Params p)
     tc_fence_before();
     __syncthreads();                       // barriers initialised, tensor memory allocated
     tc_fence_after();
+    // The kernel is launched with programmatic stream serialization: everything above may
+    // run while the previous kernel of the stream is still finishing.  Nothing below -- no
+    // read of the operands, no write of the output -- happens before that kernel has
+    // completed and its writes are visible; the kernel after this one may begin its own
+    // prologue from here on.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t ntiles = (p.M + S::TILE - 1) / S::TILE;
     const int mytiles = (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
     const uint32_t M32 = (uint32_t)p.M;
@@ -356,7 +388,8 @@ conv_tc_kernel(const Params p)
             const int idx = wt + it * NT;
             if (idx >= TASKS) break;
             const int n = idx / (KS * 4), wd = idx - n * (KS * 4);
-            const int px = n / OC, oc = n - px * OC;
+            const int px = n / OC, ocp = n - px * OC;
+            const int oc = (ocp & ~7) + ch8(ocp & 7);  // the channel this column stands for
             uint32_t lo = 0, hi = 0;
             int raw = 0;
             if (wd < S::NW) {
@@ -402,11 +435,17 @@ conv_tc_kernel(const Params p)
         fence_async_smem();                // B, before the async proxy (the MMA) reads it
         sync_workers();
         // per-column constant: what is left of Eq. 3 (column n = px*OC + oc)
+        int cterm = 0;
         if (wt < OC) {
             const int cs = p.colsum_w ? p.colsum_w[wt] : colterm[wt];
-            const int v = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
-                                (uint32_t)(p.bias ? p.bias[wt] : 0));
-            for (int px = 0; px < P; ++px) colterm[px * OC + wt] = v;
+            cterm = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
+                          (uint32_t)(p.bias ? p.bias[wt] : 0));
+        }
+        sync_workers();                    // every weight sum has been read
+        if (wt < OC) {
+            // column position of channel wt within its group of eight: the inverse of ch8
+            const int pos = (wt & ~7) + 2 * (wt & 3) + ((wt >> 2) & 1);
+            for (int px = 0; px < P; ++px) colterm[px * OC + pos] = cterm;
         }
         tc_fence_before();
         sync_workers();
@@ -452,9 +491,12 @@ conv_tc_kernel(const Params p)
         const uint32_t acc_taddr = lane_taddr + (uint32_t)(g * S::ACCW);
         const uint32_t a_taddr = lane_taddr + (uint32_t)(G * S::ACCW + g * S::ACOLS);
         const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
-        const bool fast = p.rq.shift >= 2;             // the 32-bit form of the rounding shift (see requant())
-        const int sh1 = p.rq.shift - 1, rnd = fast ? 1 << (sh1 - 1) : 0;
-        const int zml = p.rq.zo - p.rq.lo, hml = p.rq.hi - p.rq.lo;
+        // the 32-bit form of the rounding shift with the output zero point folded into the
+        // rounding constant (see requant8())
+        const bool fast = p.rq.shift >= 2 && p.rq.shift <= 27;
+        const int sh1 = p.rq.shift - 1;
+        const int rnd = fast ? (1 << (sh1 - 1)) + (p.rq.zo - p.rq.lo) * (1 << sh1) : 0;
+        const uint32_t hml2 = (uint32_t)(p.rq.hi - p.rq.lo) * 0x00010001u;
         const uint32_t lofill = (uint32_t)p.rq.lo * 0x11111111u;
         const uint32_t mstep = gridDim.x * (uint32_t)(S::TILE * G);
         uint32_t mbase = (blockIdx.x + (uint32_t)g * gridDim.x) * (uint32_t)S::TILE;
@@ -570,8 +612,8 @@ conv_tc_kernel(const Params p)
                     uint32_t o[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        o[j] = (fast ? requant8<true>(r[c] + 8 * j, p.rq, sh1, rnd, zml, hml)
-                                     : requant8<false>(r[c] + 8 * j, p.rq, sh1, rnd, zml, hml)) + lofill;
+                        o[j] = (fast ? requant8<true>(r[c] + 8 * j, p.rq, sh1, rnd, hml2)
+                                     : requant8<false>(r[c] + 8 * j, p.rq, sh1, rnd, hml2)) + lofill;
                     if (mrow < M32)
                         *reinterpret_cast<uint4*>(dst + (cb + c) * 16) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
@@ -709,9 +751,22 @@ cudaError_t launch_instance(const fused::Params& p, cudaStream_t st)
         sms = 148;
     const int64_t tiles = (p.M + S::TILE - 1) / S::TILE;
     const int grid = (int)(tiles < sms ? tiles : sms);
-    kernel<<<grid, (convtc::PWN + 1 + 4 * G) * 32, smem, st>>>(p);
+    // Programmatic stream serialization: the grid may be scheduled while the previous
+    // kernel of the stream drains; the kernel itself waits (griddepcontrol.wait) before it
+    // touches memory.
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((convtc::PWN + 1 + 4 * G) * 32);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kernel, p);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 // Input buffers of the ring: enough bytes in flight to cover the memory latency (about
