@@ -445,6 +445,21 @@ def time_gemm_sweep(q4, wl, reps: int = 20):
                                                            colsum_b=cb, ws=ws)], r)
             out[name].update({"q4_gemm_requant_ms": ms, "q4_gemm_requant_tops": ops / (ms * 1e-3) / 1e12})
         del A, Bt, C
+    # per-channel parameters in the epilogue against the per-tensor fused call, 8192^3
+    c = wl.c2(GEMM_N)
+    n = GEMM_N
+    A, Bt = torch.from_numpy(c.A).cuda(), torch.from_numpy(c.Bt).cuda()
+    Cq = torch.empty((n, n // 2), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(q4.q4_gemm_workspace_bytes(n, n, n), dtype=torch.uint8, device="cuda")
+    cb = q4.q4_row_sums(Bt, n, n, torch.empty(n, dtype=torch.int32, device="cuda"))
+    chan = lambda lo, hi: torch.randint(lo, hi, (n,), dtype=torch.int32, device="cuda")
+    zb_c, bias_c, mult_c, shift_c = chan(0, 16), chan(-512, 513), chan(1 << 30, (1 << 31) - 1), chan(8, 17)
+    rq = q4.Requant(c.mult, c.shift, 0, 0, 15)
+    t_pt = graph_time_ms([lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, c.za, c.zb, rq, colsum_b=cb, ws=ws)], 5)
+    t_pc = graph_time_ms([lambda: q4.q4_gemm_requant_channels(A, Bt, Cq, n, n, n, c.za, zb_c, mult_c, shift_c,
+                                                              0, 0, 15, bias_c, None, cb, ws)], 5)
+    out["per_channel_epilogue_8192"] = {"q4_gemm_requant_ms": t_pt, "q4_gemm_requant_channels_ms": t_pc,
+                                        "ratio": t_pc / t_pt}
     return out
 
 

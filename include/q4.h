@@ -233,6 +233,26 @@ q4_status q4_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, int32_t
                               uint8_t* Cq, int64_t ldcq, void* stream);
 
 /*
+ * The product with per-output-channel weight quantization finished in the GEMM's own
+ * epilogue (no int32 matrix in memory): same result as q4_gemm with zb = 0 followed by
+ * q4_requant_channels,
+ *   acc[m][n] = sum_k (A[m][k] - za)(B[k][n] - zb[n]) + bias[n]
+ *   y[m][n]   = clamp(floor((acc * mult[n] + 2^(30 + shift[n])) / 2^(31 + shift[n])) + zo, lo, hi)
+ * packed two per byte to Cq.  Extension of the paper's per-matrix scheme (Section II-A; Eq. 2
+ * applied column by column).  A, Bt, rowsum_a, colsum_b, ws as in q4_gemm_requant; zb (values
+ * 0..15, NULL = all 0), bias (NULL = none), mult in [2^30, 2^31) and shift in 0..31 are DEVICE
+ * arrays of N int32, not range-checked.  The per-channel epilogue exists in the tensor-core
+ * kernels only: operands that break their alignment rules (16-byte aligned A, Bt, lda, ldb)
+ * return Q4_ERR_ALIGNMENT -- use q4_gemm with zb = 0 and q4_requant_channels for those.
+ */
+q4_status q4_gemm_requant_channels(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                                   int32_t M, int32_t N, int32_t K, int32_t za, const int32_t* zb,
+                                   const int32_t* rowsum_a, const int32_t* colsum_b,
+                                   const int32_t* bias, const int32_t* mult, const int32_t* shift,
+                                   int32_t zo, int32_t clamp_lo, int32_t clamp_hi,
+                                   uint8_t* Cq, int64_t ldcq, void* ws, size_t ws_bytes, void* stream);
+
+/*
  * A convolution layer with per-output-channel weight quantization, as ONE fused kernel (the
  * unrolled matrix is never written; no workspace): like q4_conv2d, but output channel n has
  * its own weight zero point zb[n] (0..15), multiplier mult[n] in [2^30, 2^31) and shift[n] in

@@ -36,7 +36,8 @@ EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_st
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
            "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak",
            "q4_quant_params", "q4_quantize", "q4_dequantize", "q4_gemm_u8",
-           "q4_gemm_u8_workspace_bytes", "q4_selftest_wait_timeout", "q4_requant_channels", "q4_conv2d_channels"]
+           "q4_gemm_u8_workspace_bytes", "q4_selftest_wait_timeout", "q4_requant_channels", "q4_conv2d_channels",
+           "q4_gemm_requant_channels"]
 
 
 class Q4Error(RuntimeError):
@@ -134,6 +135,8 @@ _lib.q4_dequantize.argtypes = [_vp, _i64, _i32, _i32, ctypes.c_float, _vp, _i64,
 _lib.q4_selftest_wait_timeout.argtypes = [_vp, _vp]
 _lib.q4_requant_channels.argtypes = [_vp, _i64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp,
                                      _i32, _i32, _i32, _vp, _i64, _vp]
+_lib.q4_gemm_requant_channels.argtypes = [_vp, _i64, _vp, _i64, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp,
+                                          _i32, _i32, _i32, _vp, _i64, _vp, _sz, _vp]
 _lib.q4_conv2d_channels.argtypes = [_vp, _vp, _i64, _vp, _vp, ctypes.POINTER(_ConvDesc), _i32, _vp, _vp, _vp,
                                     _i32, _i32, _i32, _vp, _vp]
 _lib.q4_last_device_status.argtypes = [_vp]
@@ -355,6 +358,22 @@ def q4_requant_channels(C0, M: int, N: int, K: int, za: int, rowsum_a, zb, bias,
     _check(_lib.q4_requant_channels(_ptr(C0), _rows(C0, "C0"), M, N, K, za, _ptr(rowsum_a), _ptr(zb),
                                     _ptr(bias), _ptr(mult), _ptr(shift), zo, clamp_lo, clamp_hi,
                                     _ptr(Cq), _rows(Cq, "Cq"), _stream()), "q4_requant_channels")
+    return Cq
+
+
+def q4_gemm_requant_channels(A, Bt, Cq, M: int, N: int, K: int, za: int, zb, mult, shift, zo: int,
+                             clamp_lo: int, clamp_hi: int, bias=None, rowsum_a=None, colsum_b=None, ws=None):
+    """4-bit product with per-output-channel weight zero points, multipliers and shifts
+    (CUDA int32 tensors of N elements) finished in the GEMM's epilogue; see include/q4.h."""
+    _dev(A, torch.uint8, "A"); _dev(Bt, torch.uint8, "Bt"); _dev(Cq, torch.uint8, "Cq")
+    for t, n in ((zb, "zb"), (mult, "mult"), (shift, "shift"), (bias, "bias"), (rowsum_a, "rowsum_a"),
+                 (colsum_b, "colsum_b")):
+        _dev(t, torch.int32, n)
+    _check(_lib.q4_gemm_requant_channels(_ptr(A), _rows(A, "A"), _ptr(Bt), _rows(Bt, "Bt"), M, N, K, za,
+                                         _ptr(zb), _ptr(rowsum_a), _ptr(colsum_b), _ptr(bias), _ptr(mult),
+                                         _ptr(shift), zo, clamp_lo, clamp_hi, _ptr(Cq), _rows(Cq, "Cq"),
+                                         _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size(),
+                                         _stream()), "q4_gemm_requant_channels")
     return Cq
 
 

@@ -231,6 +231,33 @@ q4_status q4_gemm_requant(const uint8_t* A, int64_t lda, const uint8_t* Bt, int6
     return run_gemm(p, true, static_cast<cudaStream_t>(stream), ws, ws_bytes);
 }
 
+q4_status q4_gemm_requant_channels(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
+                                   int32_t M, int32_t N, int32_t K, int32_t za, const int32_t* zb,
+                                   const int32_t* rowsum_a, const int32_t* colsum_b,
+                                   const int32_t* bias, const int32_t* mult, const int32_t* shift,
+                                   int32_t zo, int32_t clamp_lo, int32_t clamp_hi,
+                                   uint8_t* Cq, int64_t ldcq, void* ws, size_t ws_bytes, void* stream)
+{
+    q4_status s = check_gemm(A, lda, Bt, ldb, M, N, K, za, 0);
+    if (s != Q4_OK) return s;
+    if (zo < 0 || zo > 15 || clamp_lo < 0 || clamp_hi > 15 || clamp_lo > clamp_hi) return Q4_ERR_RANGE;
+    if (N & 1) return Q4_ERR_INVALID_ARG;
+    if (M == 0 || N == 0) return Q4_OK;
+    if (!Cq || ldcq < N / 2 || !mult || !shift) return Q4_ERR_INVALID_ARG;
+    const void* words[] = {zb, rowsum_a, colsum_b, bias, mult, shift};
+    for (const void* w : words)
+        if ((uintptr_t)w % 4) return Q4_ERR_ALIGNMENT;
+    GemmParams p{};
+    p.A = A; p.Bt = Bt; p.lda = lda; p.ldb = ldb; p.M = M; p.N = N; p.K = K; p.za = za; p.zb = 0;
+    p.rowsum_a = rowsum_a; p.colsum_b = colsum_b; p.bias = bias; p.Cq = Cq; p.ldcq = ldcq;
+    p.rq = RequantParams{1 << 30, 2, zo, clamp_lo, clamp_hi};      // multiplier and shift come per channel
+    p.zb_ch = zb; p.mult_ch = mult; p.shift_ch = shift;
+    // the per-channel epilogue lives in the tensor-core kernels
+    if (variant() == 1) return Q4_ERR_UNSUPPORTED;
+    if (!gemm_tc_supported(p)) return Q4_ERR_ALIGNMENT;
+    return run_gemm(p, true, static_cast<cudaStream_t>(stream), ws, ws_bytes);
+}
+
 q4_status q4_im2col(const uint8_t* X, const q4_conv_desc* d, int32_t za,
                     uint8_t* A, int64_t lda, int32_t* rowsum_a, void* stream)
 {

@@ -30,6 +30,12 @@ struct GemmParams {
     uint8_t* Cq;               // packed output (q4_gemm_requant)
     int64_t ldcq;
     RequantParams rq;
+    // per output channel (q4_gemm_requant_channels; mult_ch and shift_ch both or neither):
+    // weight zero points (NULL = 0), multipliers, shifts.  zb, rq.mult and rq.shift are
+    // then unused.
+    const int32_t* zb_ch;
+    const int32_t* mult_ch;
+    const int32_t* shift_ch;
     unsigned* status;          // device status word
 };
 
@@ -69,6 +75,23 @@ __device__ __forceinline__ uint32_t requant(int32_t acc, const RequantParams& rq
     q = max(q, rq.lo);
     q = min(q, rq.hi);
     return (uint32_t)q;
+}
+
+// Per-channel form of requant(): the column's multiplier, and for the fast form (every
+// shift of the call in 2..27) the rounding constant 2^(s-1) + zo * 2^s with s = shift - 1,
+// so that (mulhi + rnd) >> s is already q + zo; otherwise `s` holds the shift itself and the
+// 64-bit form is used.
+__device__ __forceinline__ uint32_t requant_channel(int32_t acc, int32_t mult, int32_t rnd, int32_t s,
+                                                    bool fast, const RequantParams& rq)
+{
+    if (fast) {
+        int q = (__mulhi(acc, mult) + rnd) >> s;
+        q = max(q, rq.lo);
+        q = min(q, rq.hi);
+        return (uint32_t)q;
+    }
+    const RequantParams one{mult, s, rq.zo, rq.lo, rq.hi};
+    return requant_wide(acc, one);
 }
 
 // Unsigned 4 x 8-bit dot product accumulated into a (wrapping) 32-bit value.

@@ -51,7 +51,8 @@ template <int BN> struct Cfg {
     static constexpr int OFF_P = OFF_U + STAGES * USTAGE;
     static constexpr int OFF_SUMS = OFF_P + STAGES * PSTAGE;
     static constexpr int OFF_COLTERM = OFF_SUMS + 2 * ROWS * 4;
-    static constexpr int OFF_BAR = OFF_COLTERM + BN * 4;
+    static constexpr int OFF_PC = OFF_COLTERM + BN * 4;        // per-channel: int32 [4][BN]
+    static constexpr int OFF_BAR = OFF_PC + 4 * BN * 4;
     static constexpr int NBAR = 4 * STAGES + 6;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM = OFF_MISC + 16 + 1024;          // + slack to align the base
@@ -82,6 +83,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
     const uint32_t sums_s = sbase + C::OFF_SUMS;          // int32 [2][ROWS]
     const uint32_t colterm_s = sbase + C::OFF_COLTERM;    // int32 [BN]
+    const uint32_t pc_s = sbase + C::OFF_PC;              // int32 [4][BN]: zero point, multiplier, rounding, shift
     const uint32_t bar0 = sbase + C::OFF_BAR;
     auto bar_full_p  = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto bar_empty_p = [&](int s) { return bar0 + 8u * (uint32_t)(C::STAGES + s); };
@@ -99,6 +101,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool need_cb = (g.colsum_b == nullptr);
     const bool need_sums = need_ra || need_cb;
     const int ntiles = p.tiles_m * p.tiles_n;
+    // per-channel re-quantization: the 32-bit rounding form needs every shift in 2..27
+    const bool pc = REQUANT && g.mult_ch != nullptr;
+    int pc_fast = 1;
+    if (pc) {
+        int ok = 1;
+        for (int n = threadIdx.x; n < g.N; n += NTHREADS) {
+            const int sh = g.shift_ch[n];
+            ok = ok && sh >= 2 && sh <= 27;
+        }
+        pc_fast = __syncthreads_and(ok);
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
@@ -246,7 +259,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int lg = warp & 3;                 // TMEM lane group this warp may read
         const int row = lg * 32 + lane;          // row of the tile held by this thread
         const int et = threadIdx.x - (2 + UW) * 32;   // 0..127
-        const int kzz = g.K * g.za * g.zb;
         uint32_t lt = 0;
         for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
             const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
@@ -258,12 +270,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // per-column term of Eq. 2: -za * colsum + K za zb (+ bias)
             for (int j = et; j < BN; j += 128) {
                 const int n = n0 + j;
-                int cb = 0, bias = 0;
+                int cb = 0, bias = 0, zbn = pc ? 0 : g.zb;
                 if (n < g.N) {
                     cb = need_cb ? lds32(sums_s + 4 * (acc * C::ROWS + TM + j)) : g.colsum_b[n];
                     if (REQUANT && g.bias) bias = g.bias[n];
+                    if (pc && g.zb_ch) zbn = g.zb_ch[n];
                 }
-                sts32(colterm_s + 4 * j, (int)((uint32_t)kzz - (uint32_t)(g.za * cb) + (uint32_t)bias));
+                sts32(colterm_s + 4 * j,
+                      (int)((uint32_t)(g.K * g.za * zbn) - (uint32_t)(g.za * cb) + (uint32_t)bias));
+                if (pc) {
+                    const int mult = n < g.N ? g.mult_ch[n] : (1 << 30);
+                    const int sh = n < g.N ? g.shift_ch[n] : 2;
+                    const int s = pc_fast ? sh - 1 : sh;
+                    sts32(pc_s + 4 * j, zbn);
+                    sts32(pc_s + 4 * (BN + j), mult);
+                    sts32(pc_s + 4 * (2 * BN + j), pc_fast ? (1 << (s - 1)) + g.rq.zo * (1 << s) : 0);
+                    sts32(pc_s + 4 * (3 * BN + j), s);
+                }
             }
             int ra = 0;
             if (need_ra) ra = lds32(sums_s + 4 * (acc * C::ROWS + row));
@@ -281,13 +304,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 uint32_t r[32];
                 tc_ld32(taddr0 + (uint32_t)(ch * 32), r);
                 tc_wait_ld();
+                if (pc) {
+                    // the column's own zero point in Eq. 2's row-sum term
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * q));
-                    r[4 * q + 0] += rowterm + ct.x;
-                    r[4 * q + 1] += rowterm + ct.y;
-                    r[4 * q + 2] += rowterm + ct.z;
-                    r[4 * q + 3] += rowterm + ct.w;
+                    for (int q = 0; q < 8; ++q) {
+                        const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * q));
+                        const uint4 zz = lds128(pc_s + 4 * (ch * 32 + 4 * q));
+                        r[4 * q + 0] += ct.x - (uint32_t)ra * zz.x;
+                        r[4 * q + 1] += ct.y - (uint32_t)ra * zz.y;
+                        r[4 * q + 2] += ct.z - (uint32_t)ra * zz.z;
+                        r[4 * q + 3] += ct.w - (uint32_t)ra * zz.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * q));
+                        r[4 * q + 0] += rowterm + ct.x;
+                        r[4 * q + 1] += rowterm + ct.y;
+                        r[4 * q + 2] += rowterm + ct.z;
+                        r[4 * q + 3] += rowterm + ct.w;
+                    }
                 }
                 if (m < g.M) {
                     const bool full = (nc + 32 <= g.N);
@@ -305,13 +341,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                         }
                     } else {
                         uint32_t o[4];
+                        if (pc) {
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            uint32_t wv = 0;
+                            for (int q = 0; q < 8; ++q) {
+                                const uint4 mu = lds128(pc_s + 4 * (BN + ch * 32 + 4 * q));
+                                const uint4 rn = lds128(pc_s + 4 * (2 * BN + ch * 32 + 4 * q));
+                                const uint4 sf = lds128(pc_s + 4 * (3 * BN + ch * 32 + 4 * q));
+                                const uint32_t h =
+                                    requant_channel((int32_t)r[4 * q + 0], (int)mu.x, (int)rn.x, (int)sf.x, pc_fast, g.rq) |
+                                    requant_channel((int32_t)r[4 * q + 1], (int)mu.y, (int)rn.y, (int)sf.y, pc_fast, g.rq) << 4 |
+                                    requant_channel((int32_t)r[4 * q + 2], (int)mu.z, (int)rn.z, (int)sf.z, pc_fast, g.rq) << 8 |
+                                    requant_channel((int32_t)r[4 * q + 3], (int)mu.w, (int)rn.w, (int)sf.w, pc_fast, g.rq) << 12;
+                                if (q & 1) o[q >> 1] |= h << 16; else o[q >> 1] = h;
+                            }
+                        } else {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                wv |= requant((int32_t)r[8 * q + e], g.rq) << (4 * e);
-                            o[q] = wv;
+                            for (int q = 0; q < 4; ++q) {
+                                uint32_t wv = 0;
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    wv |= requant((int32_t)r[8 * q + e], g.rq) << (4 * e);
+                                o[q] = wv;
+                            }
                         }
                         uint8_t* dst = g.Cq + (int64_t)m * g.ldcq + (nc >> 1);
                         if (full && p.cq_vec) {
@@ -402,10 +453,11 @@ bool gemm_tc_supported(const GemmParams& p)
 
 static int sm_count()
 {
-    static int n = 0;
+    static int per_dev[64] = {};           // SM count of each device, looked up with it current
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    int& n = per_dev[dev];
     if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
         if (n <= 0) n = 148;
     }
@@ -432,23 +484,16 @@ static q4_status launch_bn(const GemmParams& g, bool rq, cudaStream_t st)
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
     const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     cudaError_t e;
+    // the attribute is per kernel and per device: set on every call, it is cheap
     if (rq) {
-        static bool attr = false;
-        if (!attr) {
-            e = cudaFuncSetAttribute(gemm_tc_kernel<BN, true>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
-            if (e != cudaSuccess) return Q4_ERR_CUDA;
-            attr = true;
-        }
+        e = cudaFuncSetAttribute(gemm_tc_kernel<BN, true>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+        if (e != cudaSuccess) return Q4_ERR_CUDA;
         gemm_tc_kernel<BN, true><<<grid, NTHREADS, C::SMEM, st>>>(tmA, tmB, p);
     } else {
-        static bool attr = false;
-        if (!attr) {
-            e = cudaFuncSetAttribute(gemm_tc_kernel<BN, false>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
-            if (e != cudaSuccess) return Q4_ERR_CUDA;
-            attr = true;
-        }
+        e = cudaFuncSetAttribute(gemm_tc_kernel<BN, false>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
+        if (e != cudaSuccess) return Q4_ERR_CUDA;
         gemm_tc_kernel<BN, false><<<grid, NTHREADS, C::SMEM, st>>>(tmA, tmB, p);
     }
     count_launch();

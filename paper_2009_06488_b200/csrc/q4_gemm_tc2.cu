@@ -75,7 +75,8 @@ constexpr int OFF_STG = OFF_P + PS * PSTAGE;      // int32 epilogue staging: 4 w
 constexpr int STG_BYTES = 4 * 32 * 128;
 constexpr int OFF_SUMS = OFF_STG + STG_BYTES;
 constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
-constexpr int OFF_BAR = OFF_COLTERM + BNC * 4;
+constexpr int OFF_PC = OFF_COLTERM + BNC * 4;       // per-channel: int32 [4][BNC] zero point, multiplier, rounding, shift
+constexpr int OFF_BAR = OFF_PC + 4 * BNC * 4;
 constexpr int NBAR = 2 * PS + 2 * US + 2 * BS + 10;
 constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
 constexpr int SMEM = OFF_MISC + 16 + 1024;
@@ -124,6 +125,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
     const uint32_t sums_s = sbase + OFF_SUMS;        // int32 [2 buffers][G][SUMS_N]
     const uint32_t colterm_s = sbase + OFF_COLTERM;  // int32 [BNC]
+    const uint32_t pc_s = sbase + OFF_PC;            // int32 [4][BNC]
     const uint32_t bar0 = sbase + OFF_BAR;
     auto bar_full_p    = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto bar_empty_p   = [&](int s) { return bar0 + 8u * (uint32_t)(PS + s); };
@@ -148,6 +150,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const bool need_cb = (g.colsum_b == nullptr);
     const bool need_sums = need_ra || need_cb;
     const int ntiles = p.tiles_m * p.tiles_n;
+    // per-channel re-quantization: the 32-bit rounding form needs every shift in 2..27
+    const bool pc = REQUANT && g.mult_ch != nullptr;
+    int pc_fast = 1;
+    if (pc) {
+        int ok = 1;
+        for (int n = threadIdx.x; n < g.N; n += NTHREADS) {
+            const int sh = g.shift_ch[n];
+            ok = ok && sh >= 2 && sh <= 27;
+        }
+        pc_fast = __syncthreads_and(ok);
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < PS; ++s) {
@@ -411,7 +424,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int lg = warp & 3;
         const int row = lg * 32 + lane;
         const int et = threadIdx.x - (2 + UW) * 32;
-        const int kzz = g.K * g.za * g.zb;
         uint32_t lt = 0;
         for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
             const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
@@ -423,7 +435,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t s0 = sums_s + 4 * (acc * G * SUMS_N);
             for (int j = et; j < BNC; j += 128) {
                 const int n = n0 + j;
-                int cb = 0, bias = 0;
+                int cb = 0, bias = 0, zbn = pc ? 0 : g.zb;
                 if (n < g.N) {
                     if (need_cb) {
 #pragma unroll
@@ -432,8 +444,19 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         cb = g.colsum_b[n];
                     }
                     if (REQUANT && g.bias) bias = g.bias[n];
+                    if (pc && g.zb_ch) zbn = g.zb_ch[n];
                 }
-                sts32(colterm_s + 4 * j, (int)((uint32_t)kzz - (uint32_t)(g.za * cb) + (uint32_t)bias));
+                sts32(colterm_s + 4 * j,
+                      (int)((uint32_t)(g.K * g.za * zbn) - (uint32_t)(g.za * cb) + (uint32_t)bias));
+                if (pc) {
+                    const int mult = n < g.N ? g.mult_ch[n] : (1 << 30);
+                    const int sh = n < g.N ? g.shift_ch[n] : 2;
+                    const int s = pc_fast ? sh - 1 : sh;
+                    sts32(pc_s + 4 * j, zbn);
+                    sts32(pc_s + 4 * (BNC + j), mult);
+                    sts32(pc_s + 4 * (2 * BNC + j), pc_fast ? (1 << (s - 1)) + g.rq.zo * (1 << s) : 0);
+                    sts32(pc_s + 4 * (3 * BNC + j), s);
+                }
             }
             int ra = 0;
             if (need_ra) {
@@ -455,13 +478,26 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 uint32_t r[32];
                 tc_ld32(taddr0 + (uint32_t)(ch * 32), r);
                 tc_wait_ld();
+                if (pc) {
+                    // the column's own zero point in Eq. 2's row-sum term
 #pragma unroll
-                for (int qd = 0; qd < 8; ++qd) {
-                    const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
-                    r[4 * qd + 0] += rowterm + ct.x;
-                    r[4 * qd + 1] += rowterm + ct.y;
-                    r[4 * qd + 2] += rowterm + ct.z;
-                    r[4 * qd + 3] += rowterm + ct.w;
+                    for (int qd = 0; qd < 8; ++qd) {
+                        const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
+                        const uint4 zz = lds128(pc_s + 4 * (ch * 32 + 4 * qd));
+                        r[4 * qd + 0] += ct.x - (uint32_t)ra * zz.x;
+                        r[4 * qd + 1] += ct.y - (uint32_t)ra * zz.y;
+                        r[4 * qd + 2] += ct.z - (uint32_t)ra * zz.z;
+                        r[4 * qd + 3] += ct.w - (uint32_t)ra * zz.w;
+                    }
+                } else {
+#pragma unroll
+                    for (int qd = 0; qd < 8; ++qd) {
+                        const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
+                        r[4 * qd + 0] += rowterm + ct.x;
+                        r[4 * qd + 1] += rowterm + ct.y;
+                        r[4 * qd + 2] += rowterm + ct.z;
+                        r[4 * qd + 3] += rowterm + ct.w;
+                    }
                 }
                 if (!REQUANT && p.c_tma) {
                     // int32 tile out through shared memory and one TMA store per warp: my
@@ -496,13 +532,28 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         }
                     } else {
                         uint32_t o[4];
+                        if (pc) {
 #pragma unroll
-                        for (int qd = 0; qd < 4; ++qd) {
-                            uint32_t wv = 0;
+                            for (int qd = 0; qd < 8; ++qd) {
+                                const uint4 mu = lds128(pc_s + 4 * (BNC + ch * 32 + 4 * qd));
+                                const uint4 rn = lds128(pc_s + 4 * (2 * BNC + ch * 32 + 4 * qd));
+                                const uint4 sf = lds128(pc_s + 4 * (3 * BNC + ch * 32 + 4 * qd));
+                                const uint32_t h =
+                                    requant_channel((int32_t)r[4 * qd + 0], (int)mu.x, (int)rn.x, (int)sf.x, pc_fast, g.rq) |
+                                    requant_channel((int32_t)r[4 * qd + 1], (int)mu.y, (int)rn.y, (int)sf.y, pc_fast, g.rq) << 4 |
+                                    requant_channel((int32_t)r[4 * qd + 2], (int)mu.z, (int)rn.z, (int)sf.z, pc_fast, g.rq) << 8 |
+                                    requant_channel((int32_t)r[4 * qd + 3], (int)mu.w, (int)rn.w, (int)sf.w, pc_fast, g.rq) << 12;
+                                if (qd & 1) o[qd >> 1] |= h << 16; else o[qd >> 1] = h;
+                            }
+                        } else {
 #pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                wv |= requant((int32_t)r[8 * qd + e], g.rq) << (4 * e);
-                            o[qd] = wv;
+                            for (int qd = 0; qd < 4; ++qd) {
+                                uint32_t wv = 0;
+#pragma unroll
+                                for (int e = 0; e < 8; ++e)
+                                    wv |= requant((int32_t)r[8 * qd + e], g.rq) << (4 * e);
+                                o[qd] = wv;
+                            }
                         }
                         uint8_t* dst = g.Cq + (int64_t)m * g.ldcq + (nc >> 1);
                         if (full && p.cq_vec) {
@@ -546,7 +597,10 @@ template <bool RQ, bool BPRE>
 static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                const CUtensorMap& tmC, long long tiles, cudaStream_t st)
 {
-    static int max_clusters = 0;
+    static int max_clusters_dev[64] = {};     // per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return Q4_ERR_CUDA;
+    int& max_clusters = max_clusters_dev[dev];
     auto kernel = pair::gemm_tc_pair_kernel<RQ, BPRE>;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -560,8 +614,7 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     if (!max_clusters) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM) !=
             cudaSuccess) return Q4_ERR_CUDA;
-        int dev = 0, sms = 148, n = 0;
-        cudaGetDevice(&dev);
+        int sms = 148, n = 0;
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         cfg.gridDim = dim3((unsigned)(sms / 2 * 2));
         if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {

@@ -58,28 +58,44 @@ requant_channels_vec_kernel(const ChannelParams p)
         rnd[e] = (1 << (s - 1)) + (p.zo << s);
     }
     const int kza = p.K * p.za;
-    for (int r = blockIdx.y; r < p.M; r += gridDim.y) {
-        const int rowfac = p.rowsum_a[r] - kza;               // sum_k (a - za)
-        const int4* src = reinterpret_cast<const int4*>(p.C0 + (int64_t)r * p.ldc + 8 * j);
-        const int4 c0 = __ldcs(src), c1 = __ldcs(src + 1);
-        const int c[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-        uint32_t word = 0;
-        if (fast) {
+    // four rows per step: their eight 16-byte loads are issued before any is used
+    constexpr int RB = 4;
+    for (int r0 = blockIdx.y; r0 < p.M; r0 += RB * gridDim.y) {
+        int4 c0[RB], c1[RB];
+        int rowfac[RB];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac) + (uint32_t)bias[e]);
-                int q = (__mulhi(acc, mult[e]) + rnd[e]) >> (sh[e] - 1);
-                q = min(max(q, p.lo), p.hi);
-                word |= (uint32_t)q << (4 * e);
-            }
-        } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac) + (uint32_t)bias[e]);
-                word |= requant_one(acc, mult[e], sh[e], p.zo, p.lo, p.hi) << (4 * e);
+        for (int u = 0; u < RB; ++u) {
+            const int r = r0 + u * gridDim.y;
+            if (r < p.M) {
+                const int4* src = reinterpret_cast<const int4*>(p.C0 + (int64_t)r * p.ldc + 8 * j);
+                c0[u] = __ldcs(src);
+                c1[u] = __ldcs(src + 1);
+                rowfac[u] = p.rowsum_a[r] - kza;              // sum_k (a - za)
             }
         }
-        *reinterpret_cast<uint32_t*>(p.Cq + (int64_t)r * p.ldcq + 4 * j) = word;
+#pragma unroll
+        for (int u = 0; u < RB; ++u) {
+            const int r = r0 + u * gridDim.y;
+            if (r >= p.M) break;
+            const int c[8] = {c0[u].x, c0[u].y, c0[u].z, c0[u].w, c1[u].x, c1[u].y, c1[u].z, c1[u].w};
+            uint32_t word = 0;
+            if (fast) {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac[u]) + (uint32_t)bias[e]);
+                    int q = (__mulhi(acc, mult[e]) + rnd[e]) >> (sh[e] - 1);
+                    q = min(max(q, p.lo), p.hi);
+                    word |= (uint32_t)q << (4 * e);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac[u]) + (uint32_t)bias[e]);
+                    word |= requant_one(acc, mult[e], sh[e], p.zo, p.lo, p.hi) << (4 * e);
+                }
+            }
+            *reinterpret_cast<uint32_t*>(p.Cq + (int64_t)r * p.ldcq + 4 * j) = word;
+        }
     }
 }
 

@@ -61,6 +61,78 @@ def test_gemm_with_per_channel_parameters(q4, shape, shifts):
     assert (got == want).all()
 
 
+FUSED_SHAPES = [(64, 64, 256), (130, 72, 100), (300, 264, 1000), (257, 136, 33), (1000, 520, 777),
+                (256, 192, 128), (700, 200, 257), (512, 768, 64), (2048, 1024, 512)]
+
+
+@pytest.mark.parametrize("variant", [3, 2])          # single-CTA / CTA-pair tensor-core kernel
+@pytest.mark.parametrize("shape", FUSED_SHAPES)
+@pytest.mark.parametrize("shifts", [(0, 14), (2, 14), (20, 31)])
+def test_per_channel_parameters_in_the_gemm_epilogue(q4, variant, shape, shifts):
+    """q4_gemm_requant_channels: the per-channel finish inside the GEMM kernel, against the
+    per-channel oracle, with and without a workspace and given sums."""
+    import torch
+    M, N, K = shape
+    seed = 9100 + sum(shape)
+    ld = ((K + 1) // 2 + 15) // 16 * 16
+    c = wl.gemm_case("pc", M, N, K, seed=seed, lda=ld, ldb=ld)
+    zb, bias, mult, shift = channel_params(seed, N, *shifts)
+    want = oracle.requant_channels(oracle.gemm_channels(c.A, c.Bt, M, N, K, c.za, zb, bias), mult, shift, 3, 1, 14)
+    Ad, Bd = dev(c.A), dev(c.Bt)
+    q4.q4_set_variant(variant)
+    try:
+        for use_ws, sums in ((False, False), (True, False), (False, True)):
+            Cq = torch.full((M, N // 2 + 16), 0xA5, dtype=torch.uint8, device="cuda")
+            ws = torch.full((q4.q4_gemm_workspace_bytes(M, N, K),), 0xA5, dtype=torch.uint8, device="cuda") \
+                if use_ws else None
+            ra = cb = None
+            if sums:
+                ra = q4.q4_row_sums(Ad, M, K, torch.empty(M, dtype=torch.int32, device="cuda"))
+                cb = q4.q4_row_sums(Bd, N, K, torch.empty(N, dtype=torch.int32, device="cuda"))
+            q4.q4_gemm_requant_channels(Ad, Bd, Cq[:, :N // 2], M, N, K, c.za, dev(zb), dev(mult), dev(shift),
+                                        3, 1, 14, dev(bias), ra, cb, ws)
+            assert q4.q4_last_device_status() == q4.Q4_OK
+            out = Cq.cpu().numpy()
+            assert (out[:, :N // 2] == want).all()
+            assert (out[:, N // 2:] == 0xA5).all()
+    finally:
+        q4.q4_set_variant(0)
+
+
+def test_per_channel_gemm_epilogue_at_the_benchmark_shape(q4):
+    """8192^3 through the CTA-pair kernel: the whole packed matrix against the per-channel
+    oracle's finishing pass applied to an int32 product (zb = 0) that exact Freivalds checks
+    and sampled oracle rows have verified."""
+    import torch
+    c = wl.c2(8192)
+    n = 8192
+    zb, bias, mult, shift = channel_params(77, n, 8, 16)
+    A, Bt = dev(c.A), dev(c.Bt)
+    C0 = torch.empty((n, n), dtype=torch.int32, device="cuda")
+    ws = torch.empty(q4.q4_gemm_workspace_bytes(n, n, n), dtype=torch.uint8, device="cuda")
+    q4.q4_gemm(A, Bt, C0, n, n, n, c.za, 0, ws=ws)
+    got0 = C0.cpu().numpy()
+    del C0
+    rows = np.unique(np.concatenate([np.random.default_rng(5).integers(0, n, 24), [0, 255, 256, n - 1]]))
+    assert (got0[rows] == oracle.gemm(np.ascontiguousarray(c.A[rows]), c.Bt, len(rows), n, n, c.za, 0)).all()
+    r = np.random.default_rng(6).integers(1, 1 << 20, n).astype(np.int64)
+    y = np.zeros(n, np.int64)
+    for n0 in range(0, n, 1024):
+        y += oracle.unpack_rows(c.Bt[n0:n0 + 1024], n).astype(np.int64).T @ r[n0:n0 + 1024]
+    for m0 in range(0, n, 1024):
+        a = oracle.unpack_rows(c.A[m0:m0 + 1024], n).astype(np.int64) - c.za
+        assert (got0[m0:m0 + 1024].astype(np.int64) @ r == a @ y).all()
+    ra = oracle.unpack_rows(c.A, n).astype(np.int64).sum(axis=1)
+    # the oracle's finishing pass: acc = C0 - zb[n] (rowsum - K za) + bias[n], then per-channel requant
+    acc = got0.astype(np.int64) - zb.astype(np.int64)[None, :] * (ra - n * c.za)[:, None] + bias[None, :]
+    want = oracle.requant_channels(acc.astype(np.int32), mult, shift, 0, 0, 15)
+    Cq = torch.empty((n, n // 2), dtype=torch.uint8, device="cuda")
+    q4.q4_gemm_requant_channels(A, Bt, Cq, n, n, n, c.za, dev(zb), dev(mult), dev(shift), 0, 0, 15,
+                                dev(bias), ws=ws)
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    assert (Cq.cpu().numpy() == want).all()
+
+
 def test_optional_arrays_and_uniform_channels_match_the_fused_path(q4):
     """No zero points and no bias: the plain product; one zero point for every channel: the
     same bytes as q4_gemm_requant's fused epilogue."""
