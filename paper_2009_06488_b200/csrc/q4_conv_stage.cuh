@@ -45,6 +45,9 @@ struct Params {
                                // kernel: bytes per asynchronous copy, 8 or 4)
     int32_t tile;              // output pixels per CTA tile
     int32_t nbuf;              // input buffers of the ring where the kernel takes it at run time
+    // the tensor-memory kernel for wide layers: output channels per CTA, CTAs that share the
+    // channels of one pixel tile, all output channels
+    int32_t tcN, tcSplit, OCtot;
     int32_t step8;             // staged-buffer offset of the pixel eight further in the same output row
     int32_t rowwrap;           // ... added when that pixel is in the next output row
     int32_t imgwrap;           // ... added on top when that row is the next image's first

@@ -57,6 +57,7 @@ constexpr int NBMAX = 8;           // staged input buffers: at most this many, a
 constexpr int PWN = 4;             // producer warps
 constexpr int ROWS = 128;          // GEMM rows per tile (UMMA M)
 constexpr int SMEM_LIMIT = 200 * 1024;
+constexpr int SMEM_LIMIT_WIDE = 224 * 1024;
 
 __host__ __device__ constexpr int pow2_at_least(int v) { int r = 32; while (r < v) r *= 2; return r; }
 
@@ -196,18 +197,18 @@ __device__ __forceinline__ Segment tile_segment(const Params& p, const fused::Ge
 // is written before the arrive that publishes it.
 __device__ __forceinline__ void producer(const Params& p, int mytiles, int nb, int pwi, uint8_t* buf0,
                                          int4* geo_s, uint32_t full0, uint32_t empty0, uint32_t abort_flag,
-                                         int lane)
+                                         int lane, int64_t tile0, int64_t tstride, int npw = PWN)
 {
     const bool bulk = p.vec16;
     const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
     const int rowwords = p.rowbytes >> 2;
-    int b = pwi, prev_b = -1;                          // j % nb (nb > PWN), buffer of my previous tile
+    int b = pwi, prev_b = -1;                          // j % nb (nb > npw), buffer of my previous tile
     uint32_t round = 0;                                // j / nb
-    for (int j = pwi; j < mytiles; j += PWN) {
+    for (int j = pwi; j < mytiles; j += npw) {
         TR(0, j, 0);
         if (round > 0 && !wait_idle(empty0 + 8 * b, (round - 1) & 1, abort_flag, p.status)) return;
         TR(0, j, 1);
-        const fused::Geo gn = fused::tile_geometry(p, blockIdx.x + (int64_t)j * gridDim.x);
+        const fused::Geo gn = fused::tile_geometry(p, tile0 + (int64_t)j * tstride);      // my j-th tile
         if (lane == 0) geo_s[b] = make_int4(gn.n_first, gn.oh_first, gn.s0, gn.nslots);
         const int nseg = gn.nslots <= gn.s0
             ? 1 : 1 + (int)fdiv((uint32_t)(gn.nslots - gn.s0 + p.sfull - 1), p.div_sfull);
@@ -259,7 +260,7 @@ __device__ __forceinline__ void producer(const Params& p, int mytiles, int nb, i
             prev_b = b;
         }
         TR(0, j, 2);
-        b += PWN;
+        b += npw;
         if (b >= nb) { b -= nb; ++round; }
     }
     if (!bulk) {
@@ -455,7 +456,7 @@ conv_tc_kernel(const Params p)
 
     if (warp < PWN) {
         // ---------------------------------------------------------------- producers
-        producer(p, mytiles, NB, warp, buf0, geo_s, full0, empty0, abort_flag, lane);
+        producer(p, mytiles, NB, warp, buf0, geo_s, full0, empty0, abort_flag, lane, blockIdx.x, gridDim.x);
     } else if (warp == PWN) {
         // ---------------------------------------------------------------- MMA issuer
         // D = s32, A = unsigned bytes (tensor memory), B = signed bytes, K-major, M = 128
@@ -629,6 +630,423 @@ conv_tc_kernel(const Params p)
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                      ::"r"(tmem_base), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+
+// ---------------------------------------------------------------------------------------
+// Layers whose input pixels are whole 16-byte pieces (C a multiple of 32): any filter size,
+// strides and paddings, 32 .. 128 output channels per CTA (more are split over CTAs, each
+// with its own share of the weights), geometry taken at run time.  These are the layers with
+// enough depth to keep the tensor pipe busy, so the tile is pipelined in depth as a GEMM is:
+//   warps 0..1      producers, as above (a tile is one bulk copy per image: two keep up)
+//   warp 2          MMA issuer
+//   8 build warps   two sets of four (one warp per lane quarter) that take the depth
+//                   chunks of a tile in turn: a GEMM row is one pixel, a 32-byte depth step is
+//                   32 channels of one tap -- one 16-byte load from the staged copy, one
+//                   tcgen05.st --, so the depth needs no padding and the steps are
+//                   consecutive 16-byte pieces of a weight row; a chunk of CK steps goes
+//                   into one slot of a ring in tensor memory
+//   8 epilogue warps  two per lane quarter, sharing the 32-column chunks of the accumulator
+// with two accumulators, so that the MMAs of a tile overlap the epilogue of the tile before
+// and the build of the chunks after.
+// ---------------------------------------------------------------------------------------
+constexpr int WCK = 8;              // depth steps per chunk (64 columns of tensor memory)
+constexpr int WNCH = 4;             // chunks in the ring
+#ifndef Q4_CTC_WSB
+#define Q4_CTC_WSB 2
+#endif
+#ifndef Q4_CTC_WSE
+#define Q4_CTC_WSE 2
+#endif
+constexpr int WSB = Q4_CTC_WSB, WSE = Q4_CTC_WSE;     // build / epilogue warps per lane quarter
+constexpr int WPW = 2;              // producer warps (a tile is one bulk copy per image; two keep up)
+constexpr int WNBAR = 2 * NBMAX + 2 * WNCH + 4;
+
+struct WideLayout {
+    int off_tab, off_ct, off_geo, off_bar, off_misc, off_buf;     // after B (at 0)
+};
+__host__ __device__ inline WideLayout wide_layout(int N, int KS)
+{
+    WideLayout l;
+    l.off_tab = ((KS + 1 + 3) / 4) * N * 128;          // B holds KS + 1 steps; then int2 [KS]: offset of the
+                                                       // step's 16 bytes, its window column
+    l.off_ct = l.off_tab + (KS * 8 + 15) / 16 * 16;
+    l.off_geo = l.off_ct + N * 4;
+    l.off_bar = l.off_geo + NBMAX * 16;
+    l.off_misc = l.off_bar + WNBAR * 8;
+    l.off_buf = l.off_misc + 16;
+    return l;
+}
+
+constexpr int WIDE_THREADS = (WPW + 1 + 4 * WSB + 4 * WSE) * 32;
+
+__global__ void __launch_bounds__(WIDE_THREADS, 1)
+conv_tc_wide_kernel(const Params p)
+{
+    const int N = p.tcN, KS = p.KS, CW4 = p.C / 32;   // columns of my tile, depth steps, steps per tap
+    // One more depth step carries the per-channel constants of Eq. 3 into the product: its A
+    // bytes are the same for every row, 1 then thirty-one times 255, and its B bytes are the
+    // constant's digits d0 + 255 * (d1 + ... + d31), each a signed byte.  The accumulators
+    // then need no preloading and can be handed back as soon as they have been read.  A
+    // constant beyond the digits' range (about a million) switches the whole CTA to
+    // preloaded accumulators, the step's B bytes being zero then.
+    const int KSX = KS + 1;
+    const int nchunks = (KSX + WCK - 1) / WCK;
+    const WideLayout L = wide_layout(N, KS);
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const uint32_t sbase = smem_u32(smem);
+    int2* tab = reinterpret_cast<int2*>(smem + L.off_tab);
+    int32_t* colterm = reinterpret_cast<int32_t*>(smem + L.off_ct);
+    const uint32_t colterm_s = sbase + L.off_ct, tab_s = sbase + L.off_tab;
+    int4* geo_s = reinterpret_cast<int4*>(smem + L.off_geo);
+    const uint32_t bar0 = sbase + L.off_bar;
+    const uint32_t full0 = bar0, empty0 = bar0 + 8 * NBMAX;
+    auto bar_a_ready   = [&](int c) { return bar0 + 8u * (uint32_t)(2 * NBMAX + c); };
+    auto bar_a_free    = [&](int c) { return bar0 + 8u * (uint32_t)(2 * NBMAX + WNCH + c); };
+    auto bar_acc_full  = [&](int a) { return bar0 + 8u * (uint32_t)(2 * NBMAX + 2 * WNCH + a); };
+    auto bar_acc_empty = [&](int a) { return bar0 + 8u * (uint32_t)(2 * NBMAX + 2 * WNCH + 2 + a); };
+    const int NB = p.nbuf;
+    const uint32_t tmem_slot = sbase + L.off_misc, abort_flag = sbase + L.off_misc + 4;
+    const uint32_t preload_flag = sbase + L.off_misc + 8;
+    uint8_t* buf0 = smem + L.off_buf;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // my share of the output channels, and my pixel tiles
+    const int nsplit = p.tcSplit;
+    const int oc0 = (int)(blockIdx.x % nsplit) * N;
+    const int64_t tile0 = blockIdx.x / nsplit, tstride = gridDim.x / nsplit;
+    constexpr int ACC0 = 0, ARING0 = 256;              // tensor-memory columns: two accumulators, then the ring
+
+    if (tid == 0) {
+        for (int i = 0; i < NB; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, 4 * WSB);
+        }
+        for (int c = 0; c < WNCH; ++c) {
+            mbar_init(bar_a_ready(c), 4);
+            mbar_init(bar_a_free(c), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_acc_full(a), 1);
+            mbar_init(bar_acc_empty(a), 4 * WSE);
+        }
+        sts32(abort_flag, 0);
+        sts32(preload_flag, 0);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == WPW) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(tmem_slot), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    asm volatile("griddepcontrol.wait;" ::: "memory");             // see conv_tc_kernel
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int64_t ntiles = (p.M + ROWS - 1) / ROWS;
+    const int mytiles = (int)((ntiles - tile0 + tstride - 1) / tstride);
+    const uint32_t M32 = (uint32_t)p.M;
+
+    uint32_t tmem_base = 0;
+    bool use_preload = false;
+    if (warp >= WPW) {
+        constexpr int NT = WIDE_THREADS - WPW * 32;
+        const int wt = tid - WPW * 32;
+        auto sync_workers = [] { asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory"); };
+        for (int i = wt; i < N; i += NT) colterm[i] = 0;
+        // depth step ks = (kh, kw, c4): where its 16 bytes sit relative to a pixel's window
+        // start, and which window column it belongs to
+        for (int ks = wt; ks < KS; ks += NT) {
+            const int tap = ks / CW4, c4 = ks - tap * CW4;
+            const int kh = tap / p.KW, kw = tap - kh * p.KW;
+            tab[ks] = make_int2(kh * p.rowbytes + kw * p.unit + 16 * c4, kw);
+        }
+        sync_workers();
+        // B: row n is output channel oc0 + (n with the ch8 order inside each group of eight);
+        // depth step ks is bytes 16 ks .. 16 ks + 15 of the weight row
+        const int tasks = N * KS;
+#pragma unroll 4
+        for (int idx = wt; idx < tasks; idx += NT) {
+            const int n = idx / KS, ks = idx - n * KS;
+            const int oc = oc0 + (n & ~7) + ch8(n & 7);
+            const uint8_t* src = p.Wt + (int64_t)oc * p.ldw + 16 * ks;
+            uint32_t wv[4];
+            if (p.wt_words) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) wv[j] = reinterpret_cast<const uint32_t*>(src)[j];
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    wv[j] = 0;
+                    for (int q = 0; q < 4; ++q) wv[j] |= (uint32_t)src[4 * j + q] << (8 * q);
+                }
+            }
+            uint32_t o[8];
+            int raw = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                raw += nibble_sum(wv[j]);
+                o[2 * j] = fused::sub_zb(wv[j] & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                o[2 * j + 1] = fused::sub_zb((wv[j] >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
+            }
+            uint8_t* row = smem + (ks >> 2) * (N * 128) + n * 128;
+            const int c = 2 * (ks & 3);
+            *reinterpret_cast<uint4*>(row + ((c ^ (n & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(row + (((c + 1) ^ (n & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+            if (!p.colsum_w && raw) atomicAdd(&colterm[n], raw);          // by column position
+        }
+        sync_workers();
+        int cterm = 0;
+        if (wt < N) {
+            const int oc = oc0 + (wt & ~7) + ch8(wt & 7);
+            const int cs = p.colsum_w ? p.colsum_w[oc] : colterm[wt];
+            cterm = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
+                          (uint32_t)(p.bias ? p.bias[oc] : 0));
+            // digits: cterm = d0 + 255 * q, d0 in -127..127, q spread over thirty-one bytes
+            int d0 = cterm % 255;
+            if (d0 > 127) d0 -= 255;
+            if (d0 < -127) d0 += 255;
+            const int qd = (cterm - d0) / 255;
+            if (qd > 31 * 127 || qd < -31 * 127) sts32(preload_flag, 1);
+        }
+        sync_workers();
+        use_preload = lds32(preload_flag) != 0;
+        if (wt < N) {
+            colterm[wt] = cterm;
+            int d0 = cterm % 255;
+            if (d0 > 127) d0 -= 255;
+            if (d0 < -127) d0 += 255;
+            int qd = use_preload ? 0 : (cterm - d0) / 255;
+            if (use_preload) d0 = 0;
+            uint32_t o[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    int dgt;
+                    if (i == 0 && b == 0) {
+                        dgt = d0;
+                    } else {
+                        dgt = qd > 127 ? 127 : qd < -127 ? -127 : qd;
+                        qd -= dgt;
+                    }
+                    word |= ((uint32_t)dgt & 0xFFu) << (8 * b);
+                }
+                o[i] = word;
+            }
+            uint8_t* row = smem + (KS >> 2) * (N * 128) + wt * 128;
+            const int c = 2 * (KS & 3);
+            *reinterpret_cast<uint4*>(row + ((c ^ (wt & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+            *reinterpret_cast<uint4*>(row + (((c + 1) ^ (wt & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+        }
+        fence_async_smem();                // B, before the async proxy (the MMA) reads it
+        tc_fence_before();
+        sync_workers();
+        tc_fence_after();
+        tmem_base = (uint32_t)lds32(tmem_slot);
+    }
+
+    if (warp < WPW) {
+        // ---------------------------------------------------------------- producers
+        producer(p, mytiles, NB, warp, buf0, geo_s, full0, empty0, abort_flag, lane, tile0, tstride, WPW);
+    } else if (warp == WPW) {
+        // ---------------------------------------------------------------- MMA issuer
+        const uint32_t idesc = (2u << 4) | (1u << 10) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(ROWS >> 4) << 24);
+        const uint64_t bdesc0 = make_kmajor_sw128_desc(sbase);
+        const uint32_t blk = (uint32_t)(N * 128) >> 4;          // descriptor units per 128-byte depth block of B
+        uint32_t cg = 0;                               // chunks issued so far
+        bool ok = true;
+        for (int k = 0; k < mytiles && ok; ++k) {
+            const int acc = k & 1;
+            TR(1, k, 0);
+            // the accumulator has been read back (and, where the constants do not ride in
+            // the product, preloaded with them)
+            if (!wait_idle(bar_acc_empty(acc), ((uint32_t)k >> 1) & 1u, abort_flag, p.status)) break;
+            TR(1, k, 1);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(ACC0 + acc * 128);
+            for (int c = 0; c < nchunks; ++c, ++cg) {
+                const int slot = (int)(cg % WNCH);
+                if (!wait_idle(bar_a_ready(slot), (cg / WNCH) & 1u, abort_flag, p.status)) { ok = false; break; }
+                TR(1, k, 2 + c);
+                tc_fence_after();
+                if (elect_one()) {
+                    // the chunk's steps with compile-time offsets: issuing must not cost more
+                    // than the 64 clocks an MMA takes
+                    const uint32_t a_tmem = tmem_base + (uint32_t)(ARING0 + slot * (8 * WCK));
+                    const uint64_t bd = bdesc0 + (uint64_t)((uint32_t)(c * (WCK / 4)) * blk);
+                    const int nst = KSX - c * WCK;     // steps of this chunk (WCK unless it is the last)
+#pragma unroll
+                    for (int j = 0; j < WCK; ++j)
+                        if (j < nst)
+                            tc_mma_i8_ts(d_tmem, a_tmem + (uint32_t)(8 * j),
+                                         bd + (uint64_t)((uint32_t)(j >> 2) * blk + 2u * (uint32_t)(j & 3)), idesc,
+                                         (c > 0 || j > 0 || use_preload) ? 1u : 0u);
+                    tc_commit(bar_a_free(slot));
+                    if (c == nchunks - 1) tc_commit(bar_acc_full(acc));
+                }
+                __syncwarp();
+            }
+        }
+    } else if (warp < WPW + 1 + 4 * WSB) {
+        // ---------------------------------------------------------------- build warps
+        const int sb = (warp - (WPW + 1)) >> 2;        // my set: the tile's chunks sb, sb + WSB, ...
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t a_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ARING0;
+        const uint32_t zfill = (uint32_t)p.za * 0x11111111u;
+        const uint32_t mstep = (uint32_t)tstride * (uint32_t)ROWS;
+        uint32_t mbase = (uint32_t)tile0 * (uint32_t)ROWS;
+        int kb = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int k = 0; k < mytiles && ok; ++k, mbase += mstep) {
+            if (warp == WPW + 1) TR(2, k, 0);
+            if (!wait_idle(full0 + 8 * kb, phase, abort_flag, p.status)) break;
+            if (warp == WPW + 1) TR(2, k, 1);
+            const int4 gv = geo_s[kb];
+            const uint32_t bufaddr = smem_u32(buf0 + kb * p.bufbytes);
+            const uint32_t done_bar = empty0 + 8 * kb;
+            if (++kb == NB) { kb = 0; phase ^= 1; }
+            const uint32_t mrow = mbase + (uint32_t)row;
+            const uint32_t mm = mrow < M32 ? mrow : mbase;
+            const uint32_t qq = fdiv(mm, p.div_ow);
+            const int ow = (int)(mm - qq * (uint32_t)p.OW);
+            const uint32_t n0 = fdiv(qq, p.div_oh);
+            const int oh = (int)(qq - n0 * (uint32_t)p.OH);
+            const int seg = (int)n0 - gv.x;
+            const int slot0 = seg == 0 ? (oh - gv.y) * p.sh : gv.z + (seg - 1) * p.sfull + oh * p.sh;
+            const int col0 = ow * p.sw - p.pw;         // input column of my window's first column
+            const uint32_t src = bufaddr + (uint32_t)(16 + slot0 * p.rowbytes + col0 * p.unit);
+            const uint32_t cg0 = (uint32_t)k * (uint32_t)nchunks;
+            for (int c = sb; c < nchunks; c += WSB) {
+                const uint32_t cg = cg0 + (uint32_t)c;
+                const int slot = (int)(cg % WNCH);
+                // the MMAs that read this slot WNCH chunks ago are complete
+                if (warp == WPW + 1) TR(2, k, 2 + c);
+                if (!wait_idle(bar_a_free(slot), ((cg / WNCH) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
+                tc_fence_after();
+                const int ks0 = c * WCK;
+                // a depth step is 16 bytes of one tap; taps left or right of the image read as
+                // the zero point.  All table entries, then all loads, then the unpacking: the
+                // loads' latencies overlap.
+                uint2 te[WCK];
+                uint4 v[WCK];
+#pragma unroll
+                for (int j = 0; j < WCK; ++j)
+                    if (ks0 + j < KS) te[j] = lds64(tab_s + 8 * (ks0 + j));
+#pragma unroll
+                for (int j = 0; j < WCK; ++j) {
+                    v[j] = make_uint4(zfill, zfill, zfill, zfill);
+                    if (ks0 + j < KS && (unsigned)(col0 + (int)te[j].y) < (unsigned)p.W) v[j] = lds128(src + te[j].x);
+                }
+#pragma unroll
+                for (int j = 0; j < WCK; ++j) {
+                    const int ks = ks0 + j;
+                    if (ks < KS) {
+                        const uint32_t r8[8] = {v[j].x & 0x0F0F0F0Fu, (v[j].x >> 4) & 0x0F0F0F0Fu,
+                                                v[j].y & 0x0F0F0F0Fu, (v[j].y >> 4) & 0x0F0F0F0Fu,
+                                                v[j].z & 0x0F0F0F0Fu, (v[j].z >> 4) & 0x0F0F0F0Fu,
+                                                v[j].w & 0x0F0F0F0Fu, (v[j].w >> 4) & 0x0F0F0F0Fu};
+                        tc_st8(a_taddr + (uint32_t)(slot * (8 * WCK) + 8 * j), r8);
+                    } else if (ks == KS) {
+                        // the step of the constants: 1, then thirty-one times 255
+                        const uint32_t r8[8] = {0xFFFFFF01u, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu,
+                                                0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+                        tc_st8(a_taddr + (uint32_t)(slot * (8 * WCK) + 8 * j), r8);
+                    }
+                }
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_a_ready(slot));
+            }
+            __syncwarp();
+            if (warp == WPW + 1) TR(2, k, 7);
+            if (lane == 0) mbar_arrive(done_bar);      // the staged copy has been read
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps
+        const int se = (warp - (WPW + 1 + 4 * WSB)) >> 2;      // my share of the 32-column chunks
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const uint32_t acc_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ACC0;
+        const bool fast = p.rq.shift >= 2 && p.rq.shift <= 27;
+        const int sh1 = p.rq.shift - 1;
+        const int rnd = fast ? (1 << (sh1 - 1)) + (p.rq.zo - p.rq.lo) * (1 << sh1) : 0;
+        const uint32_t hml2 = (uint32_t)(p.rq.hi - p.rq.lo) * 0x00010001u;
+        const uint32_t lofill = (uint32_t)p.rq.lo * 0x11111111u;
+        auto preload = [&](int acc) {                  // my chunks start from the channels' constants
+            for (int ch = se; ch < N / 32; ch += WSE) {
+#pragma unroll
+                for (int j = 4 * ch; j < 4 * ch + 4; ++j) {
+                    const uint4 x = lds128(colterm_s + 4 * (8 * j)), y = lds128(colterm_s + 4 * (8 * j + 4));
+                    const uint32_t r8[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
+                    tc_st8(acc_taddr + (uint32_t)(acc * 128 + 8 * j), r8);
+                }
+            }
+        };
+        if (use_preload) {
+            preload(0);
+            preload(1);
+            tc_wait_st();
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+            mbar_arrive(bar_acc_empty(0));
+            mbar_arrive(bar_acc_empty(1));
+        }
+        const uint32_t mstep = (uint32_t)tstride * (uint32_t)ROWS;
+        uint32_t mbase = (uint32_t)tile0 * (uint32_t)ROWS;
+        const int nch = N / 32;
+        for (int k = 0; k < mytiles; ++k, mbase += mstep) {
+            const int acc = k & 1;
+            if (warp == WPW + 1 + 4 * WSB) TR(3, k, 0);
+            if (!wait_idle(bar_acc_full(acc), ((uint32_t)k >> 1) & 1u, abort_flag, p.status)) break;
+            if (warp == WPW + 1 + 4 * WSB) TR(3, k, 1);
+            tc_fence_after();
+            const uint32_t mrow = mbase + (uint32_t)row;
+            uint8_t* dst = p.Y + (uint64_t)mrow * (p.OCtot / 2) + (oc0 >> 1);
+            for (int ch = se; ch < nch; ch += WSE) {
+                uint32_t r[32];
+                tc_ld32(acc_taddr + (uint32_t)(acc * 128 + ch * 32), r);
+                tc_wait_ld();
+                if (!use_preload && ch + WSE >= nch) {
+                    // my last chunk is in registers: the accumulator can take the next tile
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_acc_empty(acc));
+                }
+                uint32_t o[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    o[j] = (fast ? requant8<true>(r + 8 * j, p.rq, sh1, rnd, hml2)
+                                 : requant8<false>(r + 8 * j, p.rq, sh1, rnd, hml2)) + lofill;
+                if (mrow < M32) *reinterpret_cast<uint4*>(dst + ch * 16) = make_uint4(o[0], o[1], o[2], o[3]);
+            }
+            if (warp == WPW + 1 + 4 * WSB) TR(3, k, 2);
+            if (use_preload || se >= nch) {
+                // (a warp without a chunk of its own still reports)
+                if (use_preload) {
+                    preload(acc);
+                    tc_wait_st();
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_acc_empty(acc));
+            }
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == WPW) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem_base), "r"(512u) : "memory");
     }
 }
 
@@ -807,12 +1225,72 @@ static int ring_for(int id, const fused::Params& p)
     }
 }
 
+// The run-time-geometry kernel for layers with C a multiple of 32: fills the plan and the
+// dynamic shared memory it needs; false = the layer does not fit it.
+static bool plan_wide(fused::Params& p, const q4_conv_desc& d, const uint8_t* X, const uint8_t* Y, size_t* smem)
+{
+    if (d.C % 32 != 0 || d.OC % 32 != 0 || d.OC < 32) return false;
+    if ((uintptr_t)X % 16 != 0 || (uintptr_t)Y % 16 != 0) return false;
+    const int nsplit = (d.OC + 127) / 128;
+    const int N = d.OC / nsplit;
+    if (N * nsplit != d.OC || N % 32 != 0) return false;
+    const int64_t KS = (int64_t)d.KH * d.KW * d.C / 32;
+    if (KS < 1 || KS > 4096) return false;
+    const int64_t bufbytes = plan_staging(p, d, X, convtc::ROWS, false);
+    if (bufbytes <= 0 || !p.vec16) return false;
+    const int64_t fixed = convtc::wide_layout(N, (int)KS).off_buf + 1024;
+    const int64_t least = convtc::WPW + 2;             // the ring: more buffers than producer warps
+    int64_t nb = (64 * 1024 + bufbytes - 1) / bufbytes + 2;
+    const int64_t room = (convtc::SMEM_LIMIT_WIDE - fixed) / bufbytes;
+    if (nb > convtc::NBMAX) nb = convtc::NBMAX;
+    if (nb < least) nb = least;
+    if (nb > room) nb = room;
+    if (nb < least) return false;
+    p.nbuf = (int32_t)nb;
+    p.KS = (int32_t)KS;
+    p.tcN = N; p.tcSplit = nsplit; p.OCtot = d.OC;
+    *smem = (size_t)(fixed + nb * bufbytes);
+    return true;
+}
+
+static cudaError_t launch_wide(const fused::Params& p, size_t smem, cudaStream_t st)
+{
+    auto kernel = convtc::conv_tc_wide_kernel;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         convtc::SMEM_LIMIT_WIDE);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        sms = 148;
+    const int64_t ptiles = (p.M + convtc::ROWS - 1) / convtc::ROWS;
+    int64_t grid = ptiles * p.tcSplit < sms ? ptiles * p.tcSplit : sms / p.tcSplit * p.tcSplit;
+    if (grid < p.tcSplit) grid = p.tcSplit;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(convtc::WIDE_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    e = cudaLaunchKernelEx(&cfg, kernel, p);
+    count_launch();
+    return e;
+}
+
 bool conv_tc_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                        const uint8_t* Y)
 {
     (void)Wt; (void)ldw;
     const TcChoice c = choose_instance(d);
-    if (c.id < 0) return false;
+    if (c.id < 0) {
+        fused::Params pw;
+        size_t smem = 0;
+        return plan_wide(pw, d, X, Y, &smem);
+    }
     if ((uintptr_t)Y % 16 != 0) return false;
     const int OW = (d.W + 2 * d.pad_w - d.KW) / d.stride_w + 1;
     if (OW % c.P != 0) return false;
@@ -829,7 +1307,20 @@ cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, con
                            const RequantParams& rq, uint8_t* Y, cudaStream_t st)
 {
     const TcChoice c = choose_instance(d);
-    if (c.id < 0) return cudaErrorInvalidValue;
+    if (c.id < 0) {
+        fused::Params p{};
+        size_t smem = 0;
+        if (!plan_wide(p, d, X, Y, &smem)) return cudaErrorInvalidValue;
+        p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;
+        p.zb_ch = p.mult_ch = p.shift_ch = nullptr;
+        p.za = za; p.zb = zb; p.rq = rq;
+        p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
+        p.status = device_status_ptr();
+        if (!p.status) return cudaErrorUnknown;
+        if (p.M == 0) return cudaSuccess;
+        log_choice("q4_conv2d", "fused implicit GEMM on tcgen05, run-time geometry (C a multiple of 32)");
+        return launch_wide(p, smem, st);
+    }
     fused::Params p{};
     if (plan_staging(p, d, X, convtc::ROWS * c.P, c.nib) <= 0) return cudaErrorInvalidValue;
     p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;

@@ -84,6 +84,56 @@ def test_tensor_memory_conv_kernel_matches_oracle(q4, g, given_sums):
         q4.q4_set_variant(0)
 
 
+WIDE_LAYERS = [  # N, H, W, C, OC, KH, KW, sh, sw, ph, pw, shift
+    (2, 12, 12, 32, 32, 3, 3, 1, 1, 1, 1, 6),       # 32 -> 32
+    (3, 9, 11, 32, 64, 3, 3, 1, 1, 1, 1, 6),        # odd sizes
+    (2, 16, 16, 64, 64, 3, 3, 1, 1, 1, 1, 7),       # 64 -> 64
+    (2, 16, 16, 64, 128, 3, 3, 1, 1, 1, 1, 7),      # 64 -> 128: 128 columns
+    (2, 8, 8, 128, 256, 3, 3, 1, 1, 1, 1, 8),       # 128 -> 256: channels split over two CTAs
+    (3, 10, 14, 32, 96, 5, 5, 2, 1, 2, 2, 1),       # 5x5, mixed strides, padding 2, 64-bit rounding
+    (5, 7, 9, 64, 32, 1, 1, 1, 1, 0, 0, 5),         # 1x1
+    (2, 13, 10, 32, 64, 3, 2, 3, 2, 0, 1, 5),       # rectangular filter, stride 3 / 2
+    (40, 4, 4, 32, 64, 3, 3, 1, 1, 1, 1, 6),        # many images per tile
+    (1, 40, 36, 32, 160, 3, 3, 1, 1, 1, 1, 6),      # 160 channels: not two halves of whole 32-column chunks, explicit path
+    (1, 24, 20, 96, 192, 3, 3, 2, 2, 1, 1, 7),      # 192 channels: two CTAs of 96 where shared memory has the room
+]
+
+
+@pytest.mark.parametrize("g", WIDE_LAYERS)
+@pytest.mark.parametrize("given_sums", [False, True])
+def test_run_time_geometry_kernel_for_wide_layers(q4, g, given_sums):
+    """Layers with C a multiple of 32 through q4_conv2d: the tensor-memory kernel with
+    run-time geometry where it applies (one launch), the explicit path elsewhere; both
+    against the oracle."""
+    import torch
+    N, H, W, C, OC, KH, KW, sh, sw, ph, pw, shift = g
+    seed = 9500 + sum(g)
+    args = (N, H, W, C, OC, KH, KW, sh, sw, ph, pw)
+    dq, do = q4.ConvDesc(*args), oracle.ConvDesc(*args)
+    K = KH * KW * C
+    X = wl.rand_flat_nibbles(seed, 1, N * H * W * C)
+    Wt = wl.rand_packed(seed, 2, OC, K)
+    bias = wl.rand_ints(seed, 3, -300, 300, OC).astype(np.int32) if given_sums else None
+    za, zb = (int(v) for v in wl.rand_ints(seed, 4, 0, 15, 2))
+    rq = ((1 << 30) + 987654321 % (1 << 30), shift, 3, 1, 14)
+    want = oracle.conv2d(X, Wt, bias, do, za, zb, oracle.Requant(*rq))
+    ws = torch.empty(q4.q4_conv2d_workspace_bytes(dq), dtype=torch.uint8, device="cuda")
+    Y = torch.full((dq.M + 8, OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
+    colsum = None
+    if given_sums:
+        colsum = dev(oracle.unpack_rows(Wt, K).astype(np.int64).sum(axis=1).astype(np.int32))
+    n0 = q4.q4_launch_count()
+    q4.q4_conv2d(dev(X), dev(Wt), dq, za, zb, q4.Requant(*rq), Y[:dq.M], ws,
+                 None if bias is None else dev(bias), colsum)
+    launches = q4.q4_launch_count() - n0
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    out = Y.cpu().numpy()
+    assert (out[:dq.M] == want).all()
+    assert (out[dq.M:] == 0xA5).all()
+    if (C, OC) in ((32, 32), (32, 64), (64, 64), (64, 128), (128, 256), (64, 32), (32, 96)):
+        assert launches == 1             # the tensor-memory kernel took it: no unrolled matrix
+
+
 def test_which_layers_take_the_tensor_memory_kernel(q4, capfd):
     """The kernel's instances are chosen by layer class; everything else keeps its path."""
     import os

@@ -39,7 +39,7 @@ def layer(seed, N, H, W, C, OC, k, s, p):
 LAYERS = ((900, (6, 32, 32, 16, 72, 3, 1, 1)),
           (901, (3, 17, 13, 8, 6, 3, 2, 1)),
           (902, (2, 9, 11, 3, 6, 5, 1, 2)),
-          (903, (74, 16, 16, 32, 384, 1, 1, 0)))
+          (903, (74, 16, 16, 32, 400, 1, 1, 0)))
 
 
 def test_static_scratch_entry_point_matches_oracle_and_q4_conv2d_on_calls_in_a_row():
