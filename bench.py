@@ -43,7 +43,7 @@ FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel,
 # or None when no capture exists for the kernel as it stands (see profiles/).
-DOMINANT_KERNEL_TRAFFIC_BYTES = 335_000_000   # profiles/gemm_tc_pair_kernel.md, 8192^3 launch
+DOMINANT_KERNEL_TRAFFIC_BYTES = 337_080_000   # profiles/gemm_tc_pair_kernel.md, 8192^3 launch of the kernel as it stands
 
 
 def measured_peaks():
@@ -814,6 +814,16 @@ def run_case(args):
         else:
             call = lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, g.za, g.zb, rq, ws=wsg)
         units, unit = 2.0 * n ** 3 / 1e12, "TOPS"
+    elif args.case == "wide":
+        # a layer wider than the paper's: 3x3, stride 1, pad 1, 64 -> 128 channels on 32 x 32 images
+        d = q4.ConvDesc(n, 32, 32, 64, 128, 3, 3, 1, 1, 1, 1)
+        X = torch.randint(0, 256, (n * 32 * 32 * 32,), dtype=torch.uint8, device="cuda")
+        Wt = torch.randint(0, 256, (128, 9 * 32), dtype=torch.uint8, device="cuda")
+        Y = torch.empty((d.M, 64), dtype=torch.uint8, device="cuda")
+        ws = torch.empty(q4.q4_conv2d_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+        rq = q4.Requant((1 << 30) + 5, 8, 0, 0, 15)
+        call = lambda: q4.q4_conv2d(X, Wt, d, 7, 8, rq, Y, ws)
+        units, unit = 2.0 * d.M * d.K * 128 / 1e12, "TOPS"
     else:
         if args.case == "c4layer":
             # layer `--layer` of the c4 chain on random input of its shape
@@ -869,7 +879,7 @@ def main():
                     help="skip the per-layer timing of the c4 chain that follows the timed steps")
     ap.add_argument("--ref-seconds", type=float, default=None,
                     help="--impl reference: CPU seconds of oracle work per step (default: sized from --steps)")
-    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "gemm_u8", "quantize", "requant_channels", "conv", "im2col", "c4layer"],
+    ap.add_argument("--case", default=None, choices=["gemm", "gemm_requant", "gemm_u8", "quantize", "requant_channels", "conv", "im2col", "c4layer", "wide"],
                     help="profile one call in a loop instead of the benchmark step")
     ap.add_argument("--layer", type=int, default=0, help="--case c4layer: 0..4 = L1..L4, FC")
     ap.add_argument("--presums", action="store_true", help="--case gemm: pass precomputed depth sums")
