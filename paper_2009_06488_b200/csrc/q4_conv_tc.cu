@@ -54,7 +54,10 @@ constexpr int NBMAX = 8;           // staged input buffers: at most this many, a
 #ifndef Q4_CTC_SUSPEND
 #define Q4_CTC_SUSPEND 1
 #endif
-constexpr int PWN = 4;             // producer warps
+#ifndef Q4_CTC_PWN
+#define Q4_CTC_PWN 3
+#endif
+constexpr int PWN = Q4_CTC_PWN;     // producer warps
 constexpr int ROWS = 128;          // GEMM rows per tile (UMMA M)
 constexpr int SMEM_LIMIT = 200 * 1024;
 constexpr int SMEM_LIMIT_WIDE = 224 * 1024;
@@ -73,7 +76,13 @@ struct Shape {
     static constexpr int COLS = (P - 1) * SW + KW;            // input columns of a row's window
     static constexpr int WW = NIB ? (COLS + 7) / 8 : COLS * CW;   // packed words per window row
     static constexpr int NW = KH * WW;                        // packed words per GEMM row
-    static constexpr int KS = (NW + 3) / 4;                   // 32-byte depth steps
+    // 32-byte depth steps.  The words past NW carry the per-channel constants of Eq. 3 into
+    // the product (their A bytes are the same for every row: 1, then 255s; their B bytes the
+    // constant's digits d0 + 255 * (d1 + d2 + ...), signed bytes): a layer whose depth fills
+    // its last step gets one step more.
+    static constexpr int KS = NW / 4 + 1;
+    static constexpr int SPARE = KS * 4 - NW;                 // 1..4 words = 8 * SPARE bytes
+    static constexpr int QMAX = (8 * SPARE - 1) * 127;        // largest |d1 + d2 + ...|
     static constexpr int N = P * OC;
     static constexpr int ACCW = N < 32 ? 32 : N;
     static constexpr int ACOLS = KS * 8;                      // tensor-memory columns of one A tile
@@ -333,6 +342,7 @@ conv_tc_kernel(const Params p)
     auto bar_mma_done = [&](int g) { return bar0 + 8u * (uint32_t)(2 * NBMAX + GMAX + g); };
     const int NB = p.nbuf;
     const uint32_t tmem_slot = sbase + L::OFF_MISC, abort_flag = sbase + L::OFF_MISC + 4;
+    const uint32_t preload_flag = sbase + L::OFF_MISC + 8;
     uint8_t* buf0 = smem + L::OFF_BUF;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -348,6 +358,7 @@ conv_tc_kernel(const Params p)
             mbar_init(bar_mma_done(g), 1);
         }
         sts32(abort_flag, 0);
+        sts32(preload_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == PWN) {
@@ -372,6 +383,7 @@ conv_tc_kernel(const Params p)
     // The producers start copying the first tiles at once; meanwhile the other warps
     // prepare the weights (synchronising among themselves on a named barrier).
     uint32_t tmem_base = 0;
+    bool use_preload = false;              // a constant beyond the digits' range: preloaded accumulators instead
     if (warp >= PWN) {
         constexpr int NT = THREADS - PWN * 32;         // threads that prepare the weights
         constexpr int TASKS = N * KS * 4;              // eight-byte groups of B
@@ -427,13 +439,14 @@ conv_tc_kernel(const Params p)
                     }
                 }
             }
-            const int kbyte = 8 * wd;
-            uint8_t* dst = smem + L::OFF_B + (kbyte >> 7) * (N * 128) + n * 128 +
-                           ((((kbyte & 127) >> 4) ^ (n & 7)) << 4) + (kbyte & 15);
-            *reinterpret_cast<uint2*>(dst) = make_uint2(lo, hi);
+            if (wd < S::NW) {                          // (the words past the depth hold the constants' digits)
+                const int kbyte = 8 * wd;
+                uint8_t* dst = smem + L::OFF_B + (kbyte >> 7) * (N * 128) + n * 128 +
+                               ((((kbyte & 127) >> 4) ^ (n & 7)) << 4) + (kbyte & 15);
+                *reinterpret_cast<uint2*>(dst) = make_uint2(lo, hi);
+            }
             if (px == 0 && !p.colsum_w && raw) atomicAdd(&colterm[oc], raw);     // every tap once
         }
-        fence_async_smem();                // B, before the async proxy (the MMA) reads it
         sync_workers();
         // per-column constant: what is left of Eq. 3 (column n = px*OC + oc)
         int cterm = 0;
@@ -441,13 +454,53 @@ conv_tc_kernel(const Params p)
             const int cs = p.colsum_w ? p.colsum_w[wt] : colterm[wt];
             cterm = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
                           (uint32_t)(p.bias ? p.bias[wt] : 0));
+            int d0 = cterm % 255;
+            if (d0 > 127) d0 -= 255;
+            if (d0 < -127) d0 += 255;
+            const int qd = (cterm - d0) / 255;
+            if (qd > S::QMAX || qd < -S::QMAX) sts32(preload_flag, 1);
         }
-        sync_workers();                    // every weight sum has been read
+        sync_workers();                    // every weight sum has been read, the flag is final
+        use_preload = lds32(preload_flag) != 0;
         if (wt < OC) {
             // column position of channel wt within its group of eight: the inverse of ch8
             const int pos = (wt & ~7) + 2 * (wt & 3) + ((wt >> 2) & 1);
-            for (int px = 0; px < P; ++px) colterm[px * OC + pos] = cterm;
+            int d0 = cterm % 255;
+            if (d0 > 127) d0 -= 255;
+            if (d0 < -127) d0 += 255;
+            int qd = use_preload ? 0 : (cterm - d0) / 255;
+            if (use_preload) d0 = 0;
+            // the digits, eight per spare word (low four bytes, then high four)
+            uint32_t dw[2 * S::SPARE];
+#pragma unroll
+            for (int i = 0; i < 2 * S::SPARE; ++i) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    int dgt;
+                    if (i == 0 && b == 0) {
+                        dgt = d0;
+                    } else {
+                        dgt = qd > 127 ? 127 : qd < -127 ? -127 : qd;
+                        qd -= dgt;
+                    }
+                    word |= ((uint32_t)dgt & 0xFFu) << (8 * b);
+                }
+                dw[i] = word;
+            }
+            for (int px = 0; px < P; ++px) {
+                const int n = px * OC + pos;
+                colterm[n] = cterm;
+#pragma unroll
+                for (int i = 0; i < S::SPARE; ++i) {
+                    const int kbyte = 8 * (S::NW + i);
+                    uint8_t* dst = smem + L::OFF_B + (kbyte >> 7) * (N * 128) + n * 128 +
+                                   ((((kbyte & 127) >> 4) ^ (n & 7)) << 4) + (kbyte & 15);
+                    *reinterpret_cast<uint2*>(dst) = make_uint2(dw[2 * i], dw[2 * i + 1]);
+                }
+            }
         }
+        fence_async_smem();                // B, before the async proxy (the MMA) reads it
         tc_fence_before();
         sync_workers();
         tc_fence_after();
@@ -476,7 +529,8 @@ conv_tc_kernel(const Params p)
 #pragma unroll
                 for (int ks = 0; ks < KS; ++ks)
                     tc_mma_i8_ts(d_tmem, a_tmem + (uint32_t)(8 * ks),
-                                 bdesc0 + (uint64_t)((ks >> 2) * ((N * 128) >> 4) + 2 * (ks & 3)), idesc, 1u);
+                                 bdesc0 + (uint64_t)((ks >> 2) * ((N * 128) >> 4) + 2 * (ks & 3)), idesc,
+                                 (ks > 0 || use_preload) ? 1u : 0u);
                 tc_commit(bar_mma_done(g));
             }
             __syncwarp();
@@ -565,8 +619,7 @@ conv_tc_kernel(const Params p)
                     }
                 }
             }
-#pragma unroll
-            for (int i = S::NW; i < KS * 4; ++i) w[i] = 0;
+            // (the words past the depth are the constants' step: see below)
             // Everyone in my group finished the previous tile's epilogue before arriving
             // below, so the A slot and the accumulator are free: A, then the constants the
             // accumulator columns start from.
@@ -575,16 +628,25 @@ conv_tc_kernel(const Params p)
                 uint32_t r8[8];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    r8[2 * j] = w[4 * ks + j] & 0x0F0F0F0Fu;
-                    r8[2 * j + 1] = (w[4 * ks + j] >> 4) & 0x0F0F0F0Fu;
+                    const int wd = 4 * ks + j;
+                    if (wd < S::NW) {
+                        r8[2 * j] = w[wd] & 0x0F0F0F0Fu;
+                        r8[2 * j + 1] = (w[wd] >> 4) & 0x0F0F0F0Fu;
+                    } else {
+                        // the constants' bytes: 1, then 255s
+                        r8[2 * j] = wd == S::NW ? 0xFFFFFF01u : 0xFFFFFFFFu;
+                        r8[2 * j + 1] = 0xFFFFFFFFu;
+                    }
                 }
                 tc_st8(a_taddr + (uint32_t)(8 * ks), r8);
             }
+            if (use_preload) {
 #pragma unroll
-            for (int j = 0; j < N / 8; ++j) {
-                const uint4 x = lds128(colterm_s + 4 * (8 * j)), y = lds128(colterm_s + 4 * (8 * j + 4));
-                const uint32_t r8[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
-                tc_st8(acc_taddr + (uint32_t)(8 * j), r8);
+                for (int j = 0; j < N / 8; ++j) {
+                    const uint4 x = lds128(colterm_s + 4 * (8 * j)), y = lds128(colterm_s + 4 * (8 * j + 4));
+                    const uint32_t r8[8] = {x.x, x.y, x.z, x.w, y.x, y.y, y.z, y.w};
+                    tc_st8(acc_taddr + (uint32_t)(8 * j), r8);
+                }
             }
             if (tr) TR(2, k, 2);
             tc_wait_st();

@@ -134,6 +134,48 @@ def test_run_time_geometry_kernel_for_wide_layers(q4, g, given_sums):
         assert launches == 1             # the tensor-memory kernel took it: no unrolled matrix
 
 
+@pytest.mark.parametrize("g", [(3, 48, 48, 8, 16, 3, 3, 2, 2, 1, 1), (2, 8, 8, 1, 8, 3, 3, 1, 1, 1, 1),
+                               (3, 32, 32, 16, 32, 3, 3, 1, 1, 1, 1), (2, 16, 16, 64, 128, 3, 3, 1, 1, 1, 1)])
+@pytest.mark.parametrize("big", [200_000, 3_000_000, -40_000_000])
+def test_large_per_channel_constants(q4, g, big):
+    """The kernels carry Eq. 3's per-channel constant into the product as signed-byte digits
+    of an extra depth step; a bias that pushes it beyond the digits' range (about 226 000 with
+    one spare word, a million with a whole step) switches to preloaded accumulators.  Both
+    routes against the oracle.  Every channel's bias (a quarter of |big| up to |big|) is placed
+    so that its accumulators straddle a rounding boundary of the re-quantizer: an error in the
+    constant far smaller than one code step then flips output values."""
+    import torch
+    args = g
+    N, H, W, C, OC = g[:5]
+    dq, do = q4.ConvDesc(*args), oracle.ConvDesc(*args)
+    K = 9 * C
+    seed = 9900 + sum(g)
+    X = wl.rand_flat_nibbles(seed, 1, N * H * W * C)
+    Wt = wl.rand_packed(seed, 2, OC, K)
+    za, zb = 6, 9
+    shift = max(2, int(np.ceil(np.log2(abs(big) / 6.0))))
+    mult = (1 << 30) + 12345
+    real = mult / 2.0 ** (31 + shift)
+    acc0 = oracle.conv2d_direct(X, Wt, do, za, zb).reshape(-1, OC).astype(np.int64)
+    j = 1 + np.arange(OC) % 6
+    sign = 1 if big > 0 else -1
+    bias = (sign * np.round((j + 0.5) / real) - np.median(acc0, axis=0)).astype(np.int64)
+    assert np.abs(bias).max() < 2 ** 30 and np.abs(bias).min() > abs(big) / 8
+    bias = bias.astype(np.int32)
+    rq = (mult, shift, 7, 0, 15)
+    want = oracle.conv2d(X, Wt, bias, do, za, zb, oracle.Requant(*rq))
+    codes = oracle.unpack_rows(want, OC)
+    # most channels produce both codes next to their boundary
+    assert sum(len(np.unique(codes[:, n])) >= 2 for n in range(OC)) >= OC // 2
+    ws = torch.empty(q4.q4_conv2d_workspace_bytes(dq), dtype=torch.uint8, device="cuda")
+    Y = torch.full((dq.M, OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
+    n0 = q4.q4_launch_count()
+    q4.q4_conv2d(dev(X), dev(Wt), dq, za, zb, q4.Requant(*rq), Y, ws, dev(bias))
+    assert q4.q4_launch_count() - n0 == 1
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    assert (Y.cpu().numpy() == want).all()
+
+
 def test_which_layers_take_the_tensor_memory_kernel(q4, capfd):
     """The kernel's instances are chosen by layer class; everything else keeps its path."""
     import os
