@@ -138,6 +138,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    // Launched with programmatic stream serialization: everything above may overlap the end
+    // of the previous kernel of the stream; no operand is read and nothing is written before
+    // that kernel has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -485,19 +490,29 @@ static q4_status launch_bn(const GemmParams& g, bool rq, cudaStream_t st)
     const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     cudaError_t e;
     // the attribute is per kernel and per device: set on every call, it is cheap
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel waits before it touches memory
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = C::SMEM;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (rq) {
         e = cudaFuncSetAttribute(gemm_tc_kernel<BN, true>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
         if (e != cudaSuccess) return Q4_ERR_CUDA;
-        gemm_tc_kernel<BN, true><<<grid, NTHREADS, C::SMEM, st>>>(tmA, tmB, p);
+        e = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, true>, tmA, tmB, p);
     } else {
         e = cudaFuncSetAttribute(gemm_tc_kernel<BN, false>,
                                  cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM);
         if (e != cudaSuccess) return Q4_ERR_CUDA;
-        gemm_tc_kernel<BN, false><<<grid, NTHREADS, C::SMEM, st>>>(tmA, tmB, p);
+        e = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<BN, false>, tmA, tmB, p);
     }
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+    return e == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
 q4_status launch_gemm_tc(const GemmParams& g, bool rq, cudaStream_t st)
