@@ -359,10 +359,18 @@ q4_status q4_conv2d_static(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                            const q4_conv_desc* d, int32_t za, int32_t zb, const q4_requant* rq,
                            uint8_t* Y, void* stream)
 {
+    // the same argument checks, in the same order, as q4_conv2d
     q4_status s = check_conv(d, za);
     if (s != Q4_OK) return s;
+    if ((s = check_requant(rq)) != Q4_OK) return s;
+    if (zb < 0 || zb > 15) return Q4_ERR_RANGE;
+    if (d->OC < 0 || (d->OC & 1)) return Q4_ERR_INVALID_ARG;
+    const ConvShape cs = conv_shape(d);
+    if (ldw < ((int64_t)cs.K + 1) / 2) return Q4_ERR_INVALID_ARG;
+    if (cs.M == 0 || d->OC == 0) return Q4_OK;
+    if (!X || !Wt || !Y) return Q4_ERR_INVALID_ARG;
     // the layer must fit the built-in array; nothing is launched otherwise
-    if (conv_shape(d).bytes > (size_t)Q4_STATIC_SCRATCH_BYTES) return Q4_ERR_STATIC_SCRATCH;
+    if (cs.bytes > (size_t)Q4_STATIC_SCRATCH_BYTES) return Q4_ERR_STATIC_SCRATCH;
     void* scratch = static_scratch_ptr();
     if (!scratch) return Q4_ERR_CUDA;
     // q4_conv2d rewrites the whole unrolled matrix (pad nibbles included) and every row
@@ -539,12 +547,16 @@ q4_status q4_gemm_host(const uint8_t* hA, int64_t lda, const uint8_t* hBt, int64
     uint8_t* dA = static_cast<uint8_t*>(dev_staging);
     uint8_t* dB = dA + up((size_t)M * lda);
     int32_t* dC = reinterpret_cast<int32_t*>(dB + up((size_t)N * ldb));
-    if (cudaMemcpyAsync(dA, hA, (size_t)M * lda, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpyAsync(dB, hBt, (size_t)N * ldb, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // only the bytes the header promises to touch: ceil(K / 2) of every operand row, N
+    // elements of every output row (pitch padding is neither read nor written)
+    const size_t kbytes = ((size_t)K + 1) / 2;
+    if (cudaMemcpy2DAsync(dA, (size_t)lda, hA, (size_t)lda, kbytes, (size_t)M, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpy2DAsync(dB, (size_t)ldb, hBt, (size_t)ldb, kbytes, (size_t)N, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return Q4_ERR_CUDA;
     s = q4_gemm(dA, lda, dB, ldb, dC, ldc, M, N, K, za, zb, nullptr, nullptr, nullptr, 0, stream);
     if (s != Q4_OK) return s;
-    if (cudaMemcpyAsync(hC, dC, (size_t)M * ldc * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    if (cudaMemcpy2DAsync(hC, (size_t)ldc * 4, dC, (size_t)ldc * 4, (size_t)N * 4, (size_t)M,
+                          cudaMemcpyDeviceToHost, st) != cudaSuccess)
         return Q4_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }

@@ -20,8 +20,9 @@
 // order, so the product is unchanged.
 //
 // Every mbarrier wait is bounded by a clock limit.  A wait that expires raises the
-// kernel's abort flag and the device status word; all roles then fall through their
-// loops with short waits and leave through the common exit (TMEM is freed).
+// kernel's abort flag and the device status word; every role then finishes its current
+// tile with short waits, takes no further tile and leaves through the common exit (TMEM
+// is freed).
 #include <cuda.h>
 
 #include <mutex>
@@ -148,7 +149,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+            for (int tile = blockIdx.x; tile < ntiles && !lds32(abort_flag); tile += gridDim.x) {
                 const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
                 for (int s = 0; s < p.nslab; ++s, ++it) {
                     const int st = it % C::STAGES;
@@ -166,7 +167,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         if (lane == 0) {
             constexpr uint32_t idesc = make_idesc_u8(BN);
             uint32_t it = 0, lt = 0;
-            for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+            for (int tile = blockIdx.x; tile < ntiles && !lds32(abort_flag); tile += gridDim.x, ++lt) {
                 const int acc = lt & 1;
                 const uint32_t aph = (lt >> 1) & 1u;
                 mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
@@ -194,7 +195,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // ------------------------------------------------------------ unpack warps
         const int ut = threadIdx.x - 64;
         uint32_t it = 0, lt = 0;
-        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+        for (int tile = blockIdx.x; tile < ntiles && !lds32(abort_flag); tile += gridDim.x, ++lt) {
             int psum[C::NT];
 #pragma unroll
             for (int j = 0; j < C::NT; ++j) psum[j] = 0;
@@ -265,7 +266,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int row = lg * 32 + lane;          // row of the tile held by this thread
         const int et = threadIdx.x - (2 + UW) * 32;   // 0..127
         uint32_t lt = 0;
-        for (int tile = blockIdx.x; tile < ntiles; tile += gridDim.x, ++lt) {
+        for (int tile = blockIdx.x; tile < ntiles && !lds32(abort_flag); tile += gridDim.x, ++lt) {
             const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
             const int acc = lt & 1;
             const uint32_t aph = (lt >> 1) & 1u;

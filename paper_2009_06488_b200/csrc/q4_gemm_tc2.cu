@@ -29,7 +29,8 @@
 // The depth order inside each 32-value group (even nibbles, then odd) is the same for A
 // and Bt, so the product is unchanged.  Every mbarrier wait is bounded; the only
 // unbounded waits are the cluster barriers at entry and exit, which every thread
-// reaches unconditionally.
+// reaches unconditionally.  A wait that runs out raises the CTA's abort flag: every role
+// then finishes its current tile with short waits and takes no further tile.
 #include <cuda.h>
 
 #include "q4_common.cuh"
@@ -198,7 +199,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int tile = cluster_id; tile < ntiles; tile += nclusters) {
+            for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters) {
                 const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
                 const int arow = tm * 256 + (int)rank * TMC;
                 const int brow = tn * BNC + (int)rank * BH;
@@ -228,7 +229,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t a_tmem0 = tmem_base + (uint32_t)ACOL0;
             const uint64_t bdesc0 = make_kmajor_sw128_desc(sbase + OFF_B);
             uint32_t lt = 0;
-            for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
+            for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
                 const int acc = (int)(lt % NACC);
                 const uint32_t aph = (lt / NACC) & 1u;
                 mbar_wait_cl(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
@@ -281,7 +282,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         } else if (lane == 0) {
             // -------------------------------------------------------- peer relay (per tile)
             uint32_t lt = 0;
-            for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
+            for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
                 const int acc = (int)(lt % NACC);
                 const uint32_t aph = (lt / NACC) & 1u;
                 if (lt >= (uint32_t)NACC) {
@@ -314,7 +315,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             b_hi[j] = (uint32_t)(r * UROW + (((2 * c + 1) ^ sw) << 4));
         }
         uint32_t lt = 0;
-        for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
+        for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
             int psum_a = 0;
             int psum_b[NTB];
 #pragma unroll
@@ -425,7 +426,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int row = lg * 32 + lane;
         const int et = threadIdx.x - (2 + UW) * 32;
         uint32_t lt = 0;
-        for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
+        for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
             const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
             const int acc = (int)(lt % NACC);
             const uint32_t aph = (lt / NACC) & 1u;

@@ -105,6 +105,19 @@ def test_host_side_validation_needs_no_device(lib):
     assert c(CD(2, 2, 2, 16, 32, 3, 3, 1, 1, 0, 0), 0x10000, 1 << 20) == INVALID   # kernel larger than image
     assert c(CD(2, 8, 8, 16, 31, 3, 3, 1, 1, 1, 1), 0x10000, 1 << 20) == INVALID   # odd channel count out
 
+    # the entry point with built-in scratch checks its arguments like q4_conv2d, before its size
+    # test and before it looks up the array: none of these calls needs a device
+    lib.q4_conv2d_static.argtypes = [vp, vp, i64, vp, vp, ctypes.POINTER(CD), i32, i32, ctypes.POINTER(RQ), vp, vp]
+    st = lambda d, **kw: lib.q4_conv2d_static(kw.get("X", fake), fake, kw.get("ldw", 72), None, None, ctypes.byref(d),
+                                              kw.get("za", 0), kw.get("zb", 0),
+                                              ctypes.byref(kw.get("rq", rq)) if kw.get("rq", rq) else None, fake, None)
+    big = CD(256, 32, 32, 16, 32, 3, 3, 1, 1, 1, 1)                 # needs ~21 MB of scratch
+    assert st(big) == 8                                              # Q4_ERR_STATIC_SCRATCH
+    assert st(big, rq=None) == INVALID and st(big, zb=16) == RANGE and st(big, ldw=71) == INVALID
+    assert st(big, rq=RQ(1 << 29, 8, 0, 0, 15)) == RANGE and st(big, X=None) == INVALID
+    assert st(CD(256, 32, 32, 16, 31, 3, 3, 1, 1, 1, 1)) == INVALID
+    assert st(CD(0, 32, 32, 16, 32, 3, 3, 1, 1, 1, 1)) == 0         # empty: no-op, no lookup
+
 
 def test_compute_call_without_a_device_fails_loudly(lib):
     import torch
