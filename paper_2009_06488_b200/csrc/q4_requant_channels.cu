@@ -58,8 +58,9 @@ requant_channels_vec_kernel(const ChannelParams p)
         rnd[e] = (1 << (s - 1)) + (p.zo << s);
     }
     const int kza = p.K * p.za;
-    // four rows per step: their eight 16-byte loads are issued before any is used
-    constexpr int RB = 4;
+    // rows per step whose loads are issued before any is used: one (two and four were
+    // measured slower: the registers they take cost more occupancy than the loads gain)
+    constexpr int RB = 1;
     for (int r0 = blockIdx.y; r0 < p.M; r0 += RB * gridDim.y) {
         int4 c0[RB], c1[RB];
         int rowfac[RB];
