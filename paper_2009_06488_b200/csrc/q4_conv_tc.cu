@@ -724,6 +724,11 @@ constexpr int WNCH = 4;             // chunks in the ring
 constexpr int WSB = Q4_CTC_WSB, WSE = Q4_CTC_WSE;     // build / epilogue warps per lane quarter
 constexpr int WPW = 2;              // producer warps (a tile is one bulk copy per image; two keep up)
 constexpr int WNBAR = 2 * NBMAX + 2 * WNCH + 4;
+// A build set's consecutive chunks are at most 2 * WSB - 1 chunks apart (the last one of a tile
+// and the first one of the next).  A set that waits for a ring slot must not be more than one
+// use of that slot ahead of the MMA warp (mbarrier phases are told apart by one parity bit),
+// so the distance has to stay within the ring.
+static_assert(2 * WSB - 1 <= WNCH, "build sets may run at most one ring round ahead");
 
 struct WideLayout {
     int off_tab, off_ct, off_geo, off_bar, off_misc, off_buf;     // after B (at 0)
@@ -987,9 +992,10 @@ conv_tc_wide_kernel(const Params p)
                 const uint32_t cg = cg0 + (uint32_t)c;
                 const int slot = (int)(cg % WNCH);
                 // the MMAs that read this slot WNCH chunks ago are complete
-                if (warp == WPW + 1) TR(2, k, 2 + c);
+                if (warp == WPW + 1 && c == 0) TR(2, k, 2);
                 if (!wait_idle(bar_a_free(slot), ((cg / WNCH) & 1u) ^ 1u, abort_flag, p.status)) { ok = false; break; }
                 tc_fence_after();
+                if (warp == WPW + 1 && c == 0) TR(2, k, 3);
                 const int ks0 = c * WCK;
                 // a depth step is 16 bytes of one tap; taps left or right of the image read as
                 // the zero point.  All table entries, then all loads, then the unpacking: the
@@ -999,6 +1005,7 @@ conv_tc_wide_kernel(const Params p)
 #pragma unroll
                 for (int j = 0; j < WCK; ++j)
                     if (ks0 + j < KS) te[j] = lds64(tab_s + 8 * (ks0 + j));
+                if (warp == WPW + 1 && c == 0) TR(2, k, 4);
 #pragma unroll
                 for (int j = 0; j < WCK; ++j) {
                     v[j] = make_uint4(zfill, zfill, zfill, zfill);
@@ -1020,7 +1027,9 @@ conv_tc_wide_kernel(const Params p)
                         tc_st8(a_taddr + (uint32_t)(slot * (8 * WCK) + 8 * j), r8);
                     }
                 }
+                if (warp == WPW + 1 && c == 0) TR(2, k, 5);
                 tc_wait_st();
+                if (warp == WPW + 1 && c == 0) TR(2, k, 6);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(bar_a_ready(slot));
