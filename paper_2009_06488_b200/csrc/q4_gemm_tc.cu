@@ -102,18 +102,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const bool need_cb = (g.colsum_b == nullptr);
     const bool need_sums = need_ra || need_cb;
     const int ntiles = p.tiles_m * p.tiles_n;
-    // per-channel re-quantization: the 32-bit rounding form needs every shift in 2..27
-    const bool pc = REQUANT && g.mult_ch != nullptr;
-    int pc_fast = 1;
-    if (pc) {
-        int ok = 1;
-        for (int n = threadIdx.x; n < g.N; n += NTHREADS) {
-            const int sh = g.shift_ch[n];
-            ok = ok && sh >= 2 && sh <= 27;
-        }
-        pc_fast = __syncthreads_and(ok);
-    }
-
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(bar_full_p(s), 1);
@@ -144,6 +132,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // that kernel has completed.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // per-channel re-quantization: the 32-bit rounding form needs every shift in 2..27
+    const bool pc = REQUANT && g.mult_ch != nullptr;
+    int pc_fast = 1;
+    if (pc) {
+        int ok = 1;
+        for (int n = threadIdx.x; n < g.N; n += NTHREADS) {
+            const int sh = g.shift_ch[n];
+            ok = ok && sh >= 2 && sh <= 27;
+        }
+        pc_fast = __syncthreads_and(ok);
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer

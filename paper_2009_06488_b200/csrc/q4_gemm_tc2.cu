@@ -151,18 +151,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const bool need_cb = (g.colsum_b == nullptr);
     const bool need_sums = need_ra || need_cb;
     const int ntiles = p.tiles_m * p.tiles_n;
-    // per-channel re-quantization: the 32-bit rounding form needs every shift in 2..27
-    const bool pc = REQUANT && g.mult_ch != nullptr;
-    int pc_fast = 1;
-    if (pc) {
-        int ok = 1;
-        for (int n = threadIdx.x; n < g.N; n += NTHREADS) {
-            const int sh = g.shift_ch[n];
-            ok = ok && sh >= 2 && sh <= 27;
-        }
-        pc_fast = __syncthreads_and(ok);
-    }
-
     if (threadIdx.x == 0) {
         for (int s = 0; s < PS; ++s) {
             mbar_init(bar_full_p(s), 1);
@@ -194,6 +182,22 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     cluster_sync_all();              // barriers of both CTAs are initialised past this point
     tc_fence_after();
     const uint32_t tmem_base = (uint32_t)lds32(tmem_slot);
+    // Launched with programmatic stream serialization: everything above may overlap the end
+    // of the previous kernel of the stream; no operand is read and nothing is written before
+    // that kernel has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // per-channel re-quantization: the 32-bit rounding form needs every shift in 2..27
+    const bool pc = REQUANT && g.mult_ch != nullptr;
+    int pc_fast = 1;
+    if (pc) {
+        int ok = 1;
+        for (int n = threadIdx.x; n < g.N; n += NTHREADS) {
+            const int sh = g.shift_ch[n];
+            ok = ok && sh >= 2 && sh <= 27;
+        }
+        pc_fast = __syncthreads_and(ok);
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -604,14 +608,16 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     int& max_clusters = max_clusters_dev[dev];
     auto kernel = pair::gemm_tc_pair_kernel<RQ, BPRE>;
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel waits before it touches memory
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(pair::NTHREADS);
     cfg.dynamicSmemBytes = pair::SMEM;
     cfg.stream = st;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     if (!max_clusters) {
         if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM) !=
             cudaSuccess) return Q4_ERR_CUDA;
