@@ -30,7 +30,11 @@
 // and Bt, so the product is unchanged.  Every mbarrier wait is bounded; the only
 // unbounded waits are the cluster barriers at entry and exit, which every thread
 // reaches unconditionally.  A wait that runs out raises the CTA's abort flag: every role
-// then finishes its current tile with short waits and takes no further tile.
+// then finishes its current tile with short waits and takes no further tile.  The waits
+// acquire at CTA scope -- what they order is asynchronous-proxy traffic (TMA, tcgen05)
+// fenced explicitly -- except the wait on the depth-sum exchange, the one place where data
+// written by the peer CTA's threads with ordinary stores is read afterwards: a
+// cluster-scope acquire costs an L1 invalidate per try (8192^3: 367 -> 359 us without).
 #include <cuda.h>
 
 #include "q4_common.cuh"
@@ -83,6 +87,7 @@ constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
 constexpr int SMEM = OFF_MISC + 16 + 1024;
 
 static_assert(BH * 4 % GT == 0, "Bt tasks must divide evenly");
+static_assert(G <= PS, "a group's packed-ring slot advances by G per stage and wraps at most once");
 static_assert(NACC * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
 static_assert(BS % US == 0, "the MMA loop walks blocks of BS stages and derives the A slot from the position in the block");
 static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
@@ -210,7 +215,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 for (int s = 0; s < p.nslab; ++s, ++it) {
                     const int st = it % PS;
                     const uint32_t ph = (it / PS) & 1u;
-                    mbar_wait_cl(bar_empty_p(st), ph ^ 1u, abort_flag, g.status);
+                    mbar_wait(bar_empty_p(st), ph ^ 1u, abort_flag, g.status);
                     mbar_expect_tx(bar_full_p(st), (uint32_t)(BPRE ? PA : PSTAGE));
                     const uint32_t dst = sbase + OFF_P + st * PSTAGE;
                     tma_load_2d(dst, &tmA, s * PROW, arow, bar_full_p(st));
@@ -218,7 +223,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         tma_load_2d(dst + PA, &tmB, s * PROW, brow, bar_full_p(st));
                     } else {
                         const int bst = it % BS;
-                        mbar_wait_cl(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
+                        mbar_wait(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
                         mbar_expect_tx(bar_full_b(bst), (uint32_t)BSTAGE);
                         tma_load_2d(sbase + OFF_B + bst * BSTAGE, &tmB, s * UROW, brow, bar_full_b(bst));
                     }
@@ -236,8 +241,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
                 const int acc = (int)(lt % NACC);
                 const uint32_t aph = (lt / NACC) & 1u;
-                mbar_wait_cl(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
-                if (lt >= (uint32_t)NACC) mbar_wait_cl(bar_peer_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                if (lt >= (uint32_t)NACC) mbar_wait(bar_peer_tempty(acc), aph ^ 1u, abort_flag, g.status);
                 tc_fence_after();
                 // both epilogues are done with buffer `acc`: tell the unpack warps of both CTAs
                 if (elect_one()) tc_commit_pair(bar_tstart(acc), 3);
@@ -254,24 +259,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         const uint32_t it = blk + (uint32_t)j;
                         if (it < it_begin || it >= it_end) continue;        // warp-uniform
                         // A ring slot j % US: its phase is (it / US) & 1, blk being a multiple of US
-                        mbar_wait_cl(bar_full_u(j % US), (bph + (uint32_t)(j / US)) & 1u, abort_flag, g.status);
+                        mbar_wait(bar_full_u(j % US), (bph + (uint32_t)(j / US)) & 1u, abort_flag, g.status);
                         tc_fence_after();
                         const uint32_t a_tmem = a_tmem0 + (uint32_t)((j % US) * 32);
                         const uint64_t bdesc = bdesc0 + (uint64_t)(j * (BSTAGE >> 4));
-                        const int rem = g.K - (int)(it - it_begin) * SLAB;
                         if (elect_one()) {
-                            if (rem >= SLAB) {
-                                tc_mma_i8_pair_ts(d_tmem, a_tmem, bdesc, kIdesc, it > it_begin ? 1u : 0u);
-                                tc_mma_i8_pair_ts(d_tmem, a_tmem + 8u, bdesc + 2u, kIdesc, 1u);
-                                tc_mma_i8_pair_ts(d_tmem, a_tmem + 16u, bdesc + 4u, kIdesc, 1u);
-                                tc_mma_i8_pair_ts(d_tmem, a_tmem + 24u, bdesc + 6u, kIdesc, 1u);
-                            } else {
-                                const int ksteps = (rem + 31) / 32;
-                                for (int i = 0; i < ksteps; ++i)
-                                    tc_mma_i8_pair_ts(d_tmem, a_tmem + (uint32_t)(8 * i),
-                                                      bdesc + (uint64_t)(2 * i), kIdesc,
-                                                      (it > it_begin || i > 0) ? 1u : 0u);
-                            }
+                            // a ragged last stage is multiplied whole: its missing depth is zeros
+                            tc_mma_i8_pair_ts(d_tmem, a_tmem, bdesc, kIdesc, it > it_begin ? 1u : 0u);
+                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 8u, bdesc + 2u, kIdesc, 1u);
+                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 16u, bdesc + 4u, kIdesc, 1u);
+                            tc_mma_i8_pair_ts(d_tmem, a_tmem + 24u, bdesc + 6u, kIdesc, 1u);
                             // one commit frees this stage's Bt slot and, through the same
                             // barrier, its A slot (see the unpack warps' wait)
                             tc_commit_pair(bar_empty_b(j), 3);
@@ -290,7 +287,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const int acc = (int)(lt % NACC);
                 const uint32_t aph = (lt / NACC) & 1u;
                 if (lt >= (uint32_t)NACC) {
-                    mbar_wait_cl(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                    mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
                     mbar_arrive_cluster(map_to_cta(bar_peer_tempty(acc), 0));
                 }
             }
@@ -318,90 +315,87 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             b_lo[j] = (uint32_t)(r * UROW + (((2 * c) ^ sw) << 4));
             b_hi[j] = (uint32_t)(r * UROW + (((2 * c + 1) ^ sw) << 4));
         }
-        uint32_t lt = 0;
+        // Stages are numbered across tiles (every tile has nslab of them, so stage s of my
+        // lt-th tile is number lt * nslab + s); this group takes the numbers congruent to grp
+        // mod G, and carries its packed-ring slot and phase from one stage to the next.
+        int psum_a = 0;
+        int psum_b[NTB];
+        // One stage.  All four 32-deep steps are always expanded and multiplied: past the end
+        // of a ragged depth the TMA loads filled both operands with zeros, which add nothing
+        // to the products or to the depth sums.
+        auto unpack_stage = [&](uint32_t it, int pst, uint32_t pph) {
+            const int ust = (int)(it % US);
+            mbar_wait(bar_full_p(pst), pph, abort_flag, g.status);
+            const uint32_t ps = sbase + OFF_P + pst * PSTAGE;
+            // all shared-memory loads first, so their latencies overlap
+            uint4 wa[4], wb[NTB];
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                wa[c] = lds128(ps + a_ld[c]);
+#pragma unroll
+            for (int j = 0; j < NTB; ++j)
+                if (!BPRE) wb[j] = lds128(ps + b_ld[j]);
+            // Bt first: its shared-memory ring is twice as deep as the tensor-memory ring
+            // of A, so this wait is normally over and the work hides behind the MMAs
+            if (!BPRE) {
+                const int bst = (int)(it % BS);
+                mbar_wait(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
+                const uint32_t us = sbase + OFF_B + bst * BSTAGE;
+#pragma unroll
+                for (int j = 0; j < NTB; ++j) {
+                    uint4 lo, hi;
+                    unpack16(wb[j], lo, hi);
+                    if (need_cb) psum_b[j] = chunk_sum(lo, hi, psum_b[j]);
+                    sts128(us + b_lo[j], lo);
+                    sts128(us + b_hi[j], hi);
+                }
+            }
+            // A: expand my row in registers, then wait for its tensor-memory stage
+            uint4 alo[4], ahi[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                unpack16(wa[c], alo[c], ahi[c]);
+                if (need_ra) psum_a = chunk_sum(alo[c], ahi[c], psum_a);
+            }
+            // my A slot was last used by stage it - US, whose MMAs' commit arrived on the
+            // Bt ring's barrier of that stage
+            if (it >= (uint32_t)US)
+                mbar_wait(bar_empty_b((it - US) % BS), ((it - US) / BS) & 1u, abort_flag, g.status);
+            tc_fence_after();
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t r8[8] = {alo[c].x, alo[c].y, alo[c].z, alo[c].w,
+                                        ahi[c].x, ahi[c].y, ahi[c].z, ahi[c].w};
+                tc_st8(a_taddr + (uint32_t)(ust * 32 + 8 * c), r8);
+            }
+            // BPRE: my CTA's expanded Bt stage has landed (the leader learns it through my arrive)
+            if (BPRE) mbar_wait(bar_full_b(it % BS), (it / BS) & 1u, abort_flag, g.status);
+            tc_wait_st();                 // my tensor-memory stores are complete
+            fence_async_smem();           // my shared-memory stores are visible to the MMA
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive_cluster_relaxed(full_u_leader + 8u * (uint32_t)ust);
+                mbar_arrive_relaxed(bar_empty_p(pst));
+            }
+        };
+        uint32_t lt = 0, it = (uint32_t)grp, pph = 0;
+        int pst = grp % PS;
         for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
-            int psum_a = 0;
-            int psum_b[NTB];
+            psum_a = 0;
 #pragma unroll
             for (int j = 0; j < NTB; ++j) psum_b[j] = 0;
-            // every tile has nslab stages, so stage s of my lt-th tile is number
-            // lt * nslab + s overall; this group takes the numbers congruent to grp mod G
-            const uint32_t it0 = lt * (uint32_t)p.nslab;
-            for (int s = (int)((grp + G - it0 % G) % G); s < p.nslab; s += G) {
-                const uint32_t it = it0 + (uint32_t)s;
-                const int pst = it % PS, ust = it % US;
-                const uint32_t pph = (it / PS) & 1u;
-                const int rem = g.K - s * SLAB;
-                const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
-                mbar_wait_cl(bar_full_p(pst), pph, abort_flag, g.status);
-                const uint32_t ps = sbase + OFF_P + pst * PSTAGE;
-                // phase A: my row of A.  Loads first (their latencies overlap), expand in
-                // registers, then wait for the operand stage and store to tensor memory.
-                // all shared-memory loads first, so their latencies overlap
-                uint4 wa[4], wb[NTB];
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (c < ksteps) wa[c] = lds128(ps + a_ld[c]);
-#pragma unroll
-                for (int j = 0; j < NTB; ++j)
-                    if (!BPRE && ((gt + j * GT) & 3) < ksteps) wb[j] = lds128(ps + b_ld[j]);
-                // Bt first: its shared-memory ring is twice as deep as the tensor-memory ring
-                // of A, so this wait is normally over and the work hides behind the MMAs
-                if (!BPRE) {
-                    const int bst = it % BS;
-                    mbar_wait_cl(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
-                    const uint32_t us = sbase + OFF_B + bst * BSTAGE;
-#pragma unroll
-                    for (int j = 0; j < NTB; ++j) {
-                        if (((gt + j * GT) & 3) < ksteps) {
-                            uint4 lo, hi;
-                            unpack16(wb[j], lo, hi);
-                            if (need_cb) psum_b[j] = chunk_sum(lo, hi, psum_b[j]);
-                            sts128(us + b_lo[j], lo);
-                            sts128(us + b_hi[j], hi);
-                        }
-                    }
-                }
-                // A: expand my row in registers, then wait for its tensor-memory stage
-                {
-                    uint4 alo[4], ahi[4];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (c < ksteps) {
-                            unpack16(wa[c], alo[c], ahi[c]);
-                            if (need_ra) psum_a = chunk_sum(alo[c], ahi[c], psum_a);
-                        }
-                    }
-                    // my A slot was last used by stage it - US, whose MMAs' commit arrived on the
-                    // Bt ring's barrier of that stage
-                    if (it >= (uint32_t)US)
-                        mbar_wait_cl(bar_empty_b((it - US) % BS), ((it - US) / BS) & 1u, abort_flag, g.status);
-                    tc_fence_after();
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (c < ksteps) {
-                            const uint32_t r8[8] = {alo[c].x, alo[c].y, alo[c].z, alo[c].w,
-                                                    ahi[c].x, ahi[c].y, ahi[c].z, ahi[c].w};
-                            tc_st8(a_taddr + (uint32_t)(ust * 32 + 8 * c), r8);
-                        }
-                    }
-                }
-                // BPRE: my CTA's expanded Bt stage has landed (the leader learns it through my arrive)
-                if (BPRE) mbar_wait_cl(bar_full_b(it % BS), (it / BS) & 1u, abort_flag, g.status);
-                tc_wait_st();                 // my tensor-memory stores are complete
-                fence_async_smem();           // my shared-memory stores are visible to the MMA
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive_cluster_relaxed(full_u_leader + 8u * (uint32_t)ust);
-                    mbar_arrive_relaxed(bar_empty_p(pst));
-                }
+            const uint32_t it_end = (lt + 1) * (uint32_t)p.nslab;
+            for (; it < it_end; it += G) {
+                unpack_stage(it, pst, pph);
+                pst += G;
+                if (pst >= PS) { pst -= PS; pph ^= 1u; }
             }
             if (need_sums) {
                 const int acc = (int)(lt % NACC);
                 const uint32_t aph = (lt / NACC) & 1u;
                 // both CTAs' epilogues NACC tiles back are done with this sums buffer
-                mbar_wait_cl(bar_tstart(acc), aph, abort_flag, g.status);
+                mbar_wait(bar_tstart(acc), aph, abort_flag, g.status);
                 const uint32_t mine = sums_s + 4 * ((acc * G + grp) * SUMS_N);
                 sts32(mine + 4 * arow, psum_a);
 #pragma unroll
@@ -473,7 +467,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
             asm volatile("bar.sync 1, 128;" ::: "memory");
 
-            mbar_wait_cl(bar_tfull(acc), aph, abort_flag, g.status);
+            mbar_wait(bar_tfull(acc), aph, abort_flag, g.status);
             tc_fence_after();
             const uint32_t taddr0 = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(acc * BNC);
 #pragma unroll 1
