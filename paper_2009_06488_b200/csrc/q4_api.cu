@@ -88,11 +88,12 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
     p.status = status_ptr();
     if (!p.status) return Q4_ERR_CUDA;
     const int v = variant();
-    // The CTA-pair kernel pays off from about two waves of its 256 x 192 tiles (74 pairs);
-    // below that the single-CTA kernel, with narrower tiles and its sums taken in the
-    // kernel, finishes sooner.  Variant 2 always takes the pair kernel where it applies.
-    const long long pair_tiles = ((long long)p.M + 255) / 256 * (((long long)p.N + 191) / 192);
-    if (v != 1 && v != 3 && gemm_tc_pair_supported(p) && (v == 2 || pair_tiles >= 148)) {
+    // The CTA-pair kernel pays off from about 32 of its 256 x 256 tiles (2048^3 is one wave of
+    // 64: 12.7 us against 18.7 us); below that the single-CTA kernel, with narrower tiles and
+    // its sums taken in the kernel, finishes sooner (1024^3: 7.4 against 8.3 us).  Variant 2
+    // always takes the pair kernel where it applies.
+    const long long pair_tiles = ((long long)p.M + 255) / 256 * (((long long)p.N + 255) / 256);
+    if (v != 1 && v != 3 && gemm_tc_pair_supported(p) && (v == 2 || pair_tiles >= 32)) {
         // Large problems use the workspace, if given, for work that is better done once per
         // call than once per output tile: the depth sums, and -- with the full size -- the
         // expansion of Bt to bytes.  A smaller workspace still takes the sums; without one

@@ -1,6 +1,6 @@
 // Tensor-core 4-bit quantized GEMM for large problems (Eq. 2 of the paper, all four
-// terms): CTA pairs computing 256 x 192 output tiles with tcgen05.mma.cta_group::2, the
-// A operand fed from tensor memory.
+// terms): CTA pairs computing 256 x 192 or 256 x 256 output tiles with
+// tcgen05.mma.cta_group::2, the A operand fed from tensor memory.
 //
 // Why this shape.  The unpack (nibbles -> bytes) is bounded by the shared-memory
 // load/store pipe, 128 B/clk: every packed byte is read once and every unpacked byte
@@ -12,10 +12,11 @@
 // Per 128-deep stage a CTA then moves 8 KB (A, loads only) + 6 KB + 12 KB (Bt, loads and
 // stores) through the load/store pipe -- about half of what the MMA's 384 clocks allow.
 //
-// Tensor memory (512 columns): two accumulators of 192 columns (the epilogue of tile t
-// overlaps the main loop of t+1) and four A stages of 32 columns (128 depth bytes).
-// The unpacked Bt stages live in a deeper shared-memory ring (eight), so only the short
-// tensor-memory store of A sits between "stage free" and "operands ready".
+// Tensor memory (512 columns), 192-column tiles: two accumulators (the epilogue of tile t
+// overlaps the main loop of t+1) and four A stages of 32 columns (128 depth bytes); the
+// unpacked Bt stages live in a deeper shared-memory ring (eight), so only the short
+// tensor-memory store of A sits between "stage free" and "operands ready".  256-column
+// tiles: one accumulator, six A stages, six Bt stages (see Cfg).
 //
 // Roles per CTA (18 warps): warp 0 TMA producer (its own 128 rows of A, 64-byte-swizzled
 // so that row-per-lane reads are conflict-free, and its own 96 rows of Bt; no
@@ -43,58 +44,63 @@
 namespace q4 {
 namespace pair {
 
-#ifndef Q4_PAIR_BNC
-#define Q4_PAIR_BNC 192
-#endif
 constexpr int TMC = 128;             // rows of A per CTA
-constexpr int BNC = Q4_PAIR_BNC;     // columns of the pair tile (192 or 256)
-constexpr int BH = BNC / 2;          // rows of Bt staged per CTA
 constexpr int PROW = 64, UROW = 128, SLAB = 128;
-// Tensor memory holds NACC accumulators of BNC columns and US A stages of 32 columns.
-// 192 columns: two accumulators (the epilogue of a tile overlaps the next tile's main
-// loop) and four A stages.  256 columns (-DQ4_PAIR_BNC=256; bit-exact, measured 2 %
-// slower at 8192^3): one accumulator, six A stages, a third more work per MMA
-// instruction, but also a third more unpack work per CTA and stage, which is what
-// binds.
-constexpr int NACC = BNC == 256 ? 1 : 2;
 constexpr int PS = 6;                // packed stages (A 8 KB + Bt BH * 64 B)
-constexpr int US = BNC == 256 ? 6 : 4;   // A operand stages in tensor memory
-constexpr int BS = BNC == 256 ? 6 : 8;   // Bt operand stages in shared memory (BH * 128 B each)
 constexpr int PA = TMC * PROW;       // packed A bytes per stage
-constexpr int PSTAGE = PA + BH * PROW;
-constexpr int BSTAGE = BH * UROW;    // unpacked Bt bytes per stage
 #ifndef Q4_PAIR_GROUPS
 #define Q4_PAIR_GROUPS 3
 #endif
 constexpr int G = Q4_PAIR_GROUPS, WPG = 4, GT = WPG * 32;   // unpack groups, warps / threads per group
 constexpr int UW = G * WPG;
-constexpr int NTB = BH * 4 / GT;     // Bt tasks (16-byte packed chunks) per thread per stage
 constexpr int NTHREADS = (2 + UW + 4) * 32;
 constexpr int TMEM_COLS = 512;
-constexpr int ACOL0 = NACC * BNC;    // first TMEM column of the A stages
-constexpr int SUMS_N = TMC + BNC;    // per buffer and group: 128 row sums, BNC column sums
+constexpr int STG_BYTES = 4 * 32 * 128;    // int32 epilogue staging: 4 warps x 32 rows x 128 B
 
-constexpr int OFF_B = 0;
-constexpr int OFF_P = OFF_B + BS * BSTAGE;
-constexpr int OFF_STG = OFF_P + PS * PSTAGE;      // int32 epilogue staging: 4 warps x 32 rows x 128 B
-constexpr int STG_BYTES = 4 * 32 * 128;
-constexpr int OFF_SUMS = OFF_STG + STG_BYTES;
-constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
-constexpr int OFF_PC = OFF_COLTERM + BNC * 4;       // per-channel: int32 [4][BNC] zero point, multiplier, rounding, shift
-constexpr int OFF_BAR = OFF_PC + 4 * BNC * 4;
-constexpr int NBAR = 2 * PS + 2 * US + 2 * BS + 10;
-constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
-constexpr int SMEM = OFF_MISC + 16 + 1024;
+// Two tile widths, chosen per problem by the launcher.  Tensor memory holds NACC
+// accumulators of BNC columns and US A stages of 32 columns.
+// 192 columns: two accumulators (the epilogue of a tile overlaps the next tile's main
+// loop), four A stages, eight Bt stages.
+// 256 columns: one accumulator (its epilogue is exposed once per tile), six A and six Bt
+// stages; a third more work per MMA instruction and per unpacked row of A.  It wins where
+// its tile count fits the 74 CTA pairs better or the depth is long (8192^3: 313 against
+// 332 us; 2048^3 is one wave of 64 tiles: 12.7 against 15.8 us), and loses at 4096^3 (four
+// waves with four exposed epilogues against five overlapped ones).
+template <int BNC_>
+struct Cfg {
+    static constexpr int BNC = BNC_;             // columns of the pair tile
+    static constexpr int BH = BNC / 2;           // rows of Bt staged per CTA
+    static constexpr int NACC = BNC == 256 ? 1 : 2;
+    static constexpr int US = BNC == 256 ? 6 : 4;   // A operand stages in tensor memory
+    static constexpr int BS = BNC == 256 ? 6 : 8;   // Bt operand stages in shared memory (BH * 128 B each)
+    static constexpr int PSTAGE = PA + BH * PROW;
+    static constexpr int BSTAGE = BH * UROW;     // unpacked Bt bytes per stage
+    static constexpr int NTB = BH * 4 / GT;      // Bt tasks (16-byte packed chunks) per thread per stage
+    static constexpr int ACOL0 = NACC * BNC;     // first TMEM column of the A stages
+    static constexpr int SUMS_N = TMC + BNC;     // per buffer and group: 128 row sums, BNC column sums
 
-static_assert(BH * 4 % GT == 0, "Bt tasks must divide evenly");
+    static constexpr int OFF_B = 0;
+    static constexpr int OFF_P = OFF_B + BS * BSTAGE;
+    static constexpr int OFF_STG = OFF_P + PS * PSTAGE;
+    static constexpr int OFF_SUMS = OFF_STG + STG_BYTES;
+    static constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
+    static constexpr int OFF_PC = OFF_COLTERM + BNC * 4;       // per-channel: int32 [4][BNC] zero point, multiplier, rounding, shift
+    static constexpr int OFF_BAR = OFF_PC + 4 * BNC * 4;
+    static constexpr int NBAR = 2 * PS + 2 * US + 2 * BS + 10;
+    static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
+    static constexpr int SMEM = OFF_MISC + 16 + 1024;
+
+    static_assert(BH * 4 % GT == 0, "Bt tasks must divide evenly");
+    static_assert(NACC * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
+    static_assert(BS % US == 0, "the MMA loop walks blocks of BS stages and derives the A slot from the position in the block");
+    static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
+    static_assert(OFF_STG % 1024 == 0, "staging tile alignment (128-byte swizzle atoms)");
+    static_assert(SMEM <= 227 * 1024, "shared memory budget");
+
+    // D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC.
+    static constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)(BNC >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+};
 static_assert(G <= PS, "a group's packed-ring slot advances by G per stage and wraps at most once");
-static_assert(NACC * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
-static_assert(BS % US == 0, "the MMA loop walks blocks of BS stages and derives the A slot from the position in the block");
-static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
-static_assert(OFF_STG % 1024 == 0, "staging tile alignment (128-byte swizzle atoms)");
-
-// D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC.
-constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)(BNC >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 
 struct Params {
     GemmParams g;
@@ -120,11 +126,17 @@ __device__ __forceinline__ int chunk_sum(const uint4& lo, const uint4& hi, int a
 // BPRE: Bt arrives already expanded to one byte per value (by bt_expand_kernel, once per
 // call, in the same depth order the unpack gives A) and is loaded by TMA straight into
 // the swizzled operand ring; the unpack warps then handle A only.
-template <bool REQUANT, bool BPRE>
+template <int BNC, bool REQUANT, bool BPRE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const Params p)
 {
+    using C = Cfg<BNC>;
+    constexpr int BH = C::BH, NACC = C::NACC, US = C::US, BS = C::BS, PSTAGE = C::PSTAGE, BSTAGE = C::BSTAGE,
+                  NTB = C::NTB, ACOL0 = C::ACOL0, SUMS_N = C::SUMS_N, OFF_B = C::OFF_B, OFF_P = C::OFF_P,
+                  OFF_STG = C::OFF_STG, OFF_SUMS = C::OFF_SUMS, OFF_COLTERM = C::OFF_COLTERM, OFF_PC = C::OFF_PC,
+                  OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC;
+    constexpr uint32_t kIdesc = C::kIdesc;
     extern __shared__ uint8_t smem_raw[];
     // the same offset in both CTAs: dynamic shared memory starts at the same address
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -589,18 +601,19 @@ bool make_packed_map(CUtensorMap* tm, const uint8_t* base, int64_t ld, int rows,
 
 bool gemm_tc_pair_supported(const GemmParams& p)
 {
-    return gemm_tc_supported(p) && p.M >= 256 && p.N >= pair::BNC;
+    return gemm_tc_supported(p) && p.M >= 256 && p.N >= 192;
 }
 
-template <bool RQ, bool BPRE>
+template <int BNC, bool RQ, bool BPRE>
 static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                const CUtensorMap& tmC, long long tiles, cudaStream_t st)
 {
-    static int max_clusters_dev[64] = {};     // per device
+    static int max_clusters_dev[64] = {};     // per device (and per instance of this template)
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return Q4_ERR_CUDA;
     int& max_clusters = max_clusters_dev[dev];
-    auto kernel = pair::gemm_tc_pair_kernel<RQ, BPRE>;
+    auto kernel = pair::gemm_tc_pair_kernel<BNC, RQ, BPRE>;
+    constexpr int SMEM = pair::Cfg<BNC>::SMEM;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -608,12 +621,12 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;     // the kernel waits before it touches memory
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(pair::NTHREADS);
-    cfg.dynamicSmemBytes = pair::SMEM;
+    cfg.dynamicSmemBytes = SMEM;
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = 2;
     if (!max_clusters) {
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, pair::SMEM) !=
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM) !=
             cudaSuccess) return Q4_ERR_CUDA;
         int sms = 148, n = 0;
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -631,7 +644,7 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     return e == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
-// Expanded Bt [N x K8 bytes], pitch ld8: box = 128 bytes x 96 rows, written with the
+// Expanded Bt [N x K8 bytes], pitch ld8: box = 128 bytes x BNC/2 rows, written with the
 // 128-byte swizzle, i.e. directly in the layout the MMA's K-major descriptor reads.
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -665,13 +678,13 @@ static bool make_c_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, in
               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static bool make_b8_map(CUtensorMap* tm, const uint8_t* base, int64_t ld8, int rows, int k8)
+static bool make_b8_map(CUtensorMap* tm, const uint8_t* base, int64_t ld8, int rows, int k8, int box_rows)
 {
     EncodeFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {(cuuint64_t)k8, (cuuint64_t)rows};
     cuuint64_t strides[1] = {(cuuint64_t)ld8};
-    cuuint32_t box[2] = {(cuuint32_t)pair::UROW, (cuuint32_t)pair::BH};
+    cuuint32_t box[2] = {(cuuint32_t)pair::UROW, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box,
               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -684,13 +697,30 @@ bool make_c32_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, int col
     return make_c_map(tm, base, ldc, rows, cols);
 }
 
-q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8,
-                              int64_t ld8)
+// Tile width for a problem: estimated clocks of the busiest CTA pair with either width, from
+// measured stage and epilogue times (192 columns: 520 clk per 128-deep stage, epilogues
+// overlapped but the last; 256 columns: 565 clk per stage and 6200 clk of exposed epilogue
+// per tile).
+int gemm_tc_pair_width(const GemmParams& g)
 {
+    if (g.N < 256) return 192;
+    const long long nslab = ((g.K + 1) / 2 + pair::PROW - 1) / pair::PROW;
+    const long long tm = ((long long)g.M + 255) / 256;
+    const long long t192 = tm * (((long long)g.N + 191) / 192), t256 = tm * (((long long)g.N + 255) / 256);
+    const long long pairs = 74;
+    const long long c192 = (t192 + pairs - 1) / pairs * nslab * 520 + 5000;
+    const long long c256 = (t256 + pairs - 1) / pairs * (nslab * 565 + 6200);
+    return c256 < c192 ? 256 : 192;
+}
+
+template <int BNC>
+static q4_status launch_pair_w(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8, int64_t ld8)
+{
+    using C = pair::Cfg<BNC>;
     pair::Params p;
     p.g = g;
     p.tiles_m = (g.M + 255) / 256;
-    p.tiles_n = (g.N + pair::BNC - 1) / pair::BNC;
+    p.tiles_n = (g.N + BNC - 1) / BNC;
     const int kbytes = (g.K + 1) / 2;
     p.nslab = (kbytes + pair::PROW - 1) / pair::PROW;
     p.c_vec = (!rq && ((uintptr_t)g.C % 16 == 0) && (g.ldc % 4 == 0)) ? 1 : 0;
@@ -707,13 +737,20 @@ q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, con
     if (b8) {
         // expanded Bt: the kernel cannot take the column sums itself
         if (!g.colsum_b) return Q4_ERR_INVALID_ARG;
-        if (!make_b8_map(&tmB, b8, ld8, g.N, (g.K + 31) / 32 * 32)) return Q4_ERR_CUDA;
-        return rq ? launch_pair_t<true, true>(p, tmA, tmB, tmC, tiles, st)
-                  : launch_pair_t<false, true>(p, tmA, tmB, tmC, tiles, st);
+        if (!make_b8_map(&tmB, b8, ld8, g.N, (g.K + 31) / 32 * 32, C::BH)) return Q4_ERR_CUDA;
+        return rq ? launch_pair_t<BNC, true, true>(p, tmA, tmB, tmC, tiles, st)
+                  : launch_pair_t<BNC, false, true>(p, tmA, tmB, tmC, tiles, st);
     }
-    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, pair::BH, false)) return Q4_ERR_CUDA;
-    return rq ? launch_pair_t<true, false>(p, tmA, tmB, tmC, tiles, st)
-              : launch_pair_t<false, false>(p, tmA, tmB, tmC, tiles, st);
+    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, C::BH, false)) return Q4_ERR_CUDA;
+    return rq ? launch_pair_t<BNC, true, false>(p, tmA, tmB, tmC, tiles, st)
+              : launch_pair_t<BNC, false, false>(p, tmA, tmB, tmC, tiles, st);
+}
+
+q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8,
+                              int64_t ld8)
+{
+    return gemm_tc_pair_width(g) == 256 ? launch_pair_w<256>(g, rq, st, b8, ld8)
+                                        : launch_pair_w<192>(g, rq, st, b8, ld8);
 }
 
 }  // namespace q4

@@ -357,7 +357,7 @@ gemm_u8_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 for (int s = 0; s < p.nslab; ++s, ++it) {
                     const int st = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
-                    mbar_wait_cl(bar_empty(st), ph ^ 1u, abort_flag, g.status);
+                    mbar_wait(bar_empty(st), ph ^ 1u, abort_flag, g.status);
                     const uint32_t full = full_leader + 8u * (uint32_t)st;
                     mbar_expect_tx_cluster(full, (uint32_t)STAGE);
                     const uint32_t dst = sbase + st * STAGE;
@@ -373,13 +373,13 @@ gemm_u8_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int tile = cluster_id; tile < ntiles; tile += nclusters, ++lt) {
                 const int acc = lt & 1;
                 const uint32_t aph = (lt >> 1) & 1u;
-                mbar_wait_cl(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BNC);
                 for (int s = 0; s < p.nslab; ++s, ++it) {
                     const int st = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
-                    mbar_wait_cl(bar_full(st), ph, abort_flag, g.status);
+                    mbar_wait(bar_full(st), ph, abort_flag, g.status);
                     tc_fence_after();
                     const uint32_t ua = sbase + st * STAGE;
                     const uint64_t adesc = make_kmajor_sw128_desc(ua);
@@ -417,7 +417,7 @@ gemm_u8_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
             asm volatile("bar.sync 1, 128;" ::: "memory");
 
-            mbar_wait_cl(bar_tfull(acc), aph, abort_flag, g.status);
+            mbar_wait(bar_tfull(acc), aph, abort_flag, g.status);
             tc_fence_after();
             const uint32_t taddr0 = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(acc * BNC);
 #pragma unroll 1
