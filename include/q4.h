@@ -352,8 +352,10 @@ q4_status q4_selftest_wait_timeout(int* outcome_dev, void* stream);
  * kernels only, 2 = tensor-core kernels or an error where their alignment rules do
  * not hold, 3 = like 2 but never the CTA-pair kernel, 4 = automatic except that
  * convolution layers skip the tensor-memory (tcgen05) fused kernel and take the warp-level
- * fused kernels.  Returns the previous value.  Process-wide; also read once from the
- * environment variable Q4_FORCE_VARIANT ("simt" / "tc" / "tc1" / "fused1"). */
+ * fused kernels, 5 / 6 = like 2 with the CTA-pair GEMM kernel's tile width fixed at 192 / 256
+ * columns (it is otherwise chosen from the problem's shape).  Returns the previous value.
+ * Process-wide; also read once from the environment variable Q4_FORCE_VARIANT ("simt" / "tc" /
+ * "tc1" / "fused1" / "tc192" / "tc256"). */
 int q4_set_variant(int variant);
 /* With Q4_LOG=1 in the environment every GEMM / convolution call prints one line to stderr
  * naming the kernel it was given. */

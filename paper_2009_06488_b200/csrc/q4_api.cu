@@ -37,10 +37,16 @@ static int variant()
         if (e && !std::strcmp(e, "tc")) v = 2;
         if (e && !std::strcmp(e, "tc1")) v = 3;
         if (e && !std::strcmp(e, "fused1")) v = 4;
+        if (e && !std::strcmp(e, "tc192")) v = 5;
+        if (e && !std::strcmp(e, "tc256")) v = 6;
         g_variant.store(v, std::memory_order_relaxed);
     }
     return v;
 }
+
+// Variants 5 and 6 are variant 2 with the CTA-pair kernel's tile width fixed.
+static int variant_kind() { const int v = variant(); return v >= 5 ? 2 : v; }
+static int forced_pair_width() { const int v = variant(); return v == 5 ? 192 : v == 6 ? 256 : 0; }
 
 static unsigned* status_ptr()
 {
@@ -87,7 +93,7 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
 {
     p.status = status_ptr();
     if (!p.status) return Q4_ERR_CUDA;
-    const int v = variant();
+    const int v = variant_kind();
     // The CTA-pair kernel pays off from about 32 of its 256 x 256 tiles (2048^3 is one wave of
     // 64: 12.7 us against 18.7 us); below that the single-CTA kernel, with narrower tiles and
     // its sums taken in the kernel, finishes sooner (1024^3: 7.4 against 8.3 us).  Variant 2
@@ -117,7 +123,7 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
                 p.rowsum_a = wa;
             }
             log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "CTA-pair tcgen05 kernel, Bt expanded once per call");
-            return launch_gemm_tc_pair(p, rq, st, b8, ld8);
+            return launch_gemm_tc_pair(p, rq, st, b8, ld8, forced_pair_width());
         }
         if ((!p.rowsum_a || !p.colsum_b) && ws_ok && ws_bytes >= sums_bytes) {
             const bool do_a = !p.rowsum_a, do_b = !p.colsum_b;
@@ -127,7 +133,7 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
             if (do_b) p.colsum_b = wb;
         }
         log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "CTA-pair tcgen05 kernel");
-        return launch_gemm_tc_pair(p, rq, st);
+        return launch_gemm_tc_pair(p, rq, st, nullptr, 0, forced_pair_width());
     }
     if (v != 1 && gemm_tc_supported(p)) {
         log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "single-CTA tcgen05 kernel");
@@ -254,7 +260,7 @@ q4_status q4_gemm_requant_channels(const uint8_t* A, int64_t lda, const uint8_t*
     p.rq = RequantParams{1 << 30, 2, zo, clamp_lo, clamp_hi};      // multiplier and shift come per channel
     p.zb_ch = zb; p.mult_ch = mult; p.shift_ch = shift;
     // the per-channel epilogue lives in the tensor-core kernels
-    if (variant() == 1) return Q4_ERR_UNSUPPORTED;
+    if (variant_kind() == 1) return Q4_ERR_UNSUPPORTED;
     if (!gemm_tc_supported(p)) return Q4_ERR_ALIGNMENT;
     return run_gemm(p, true, static_cast<cudaStream_t>(stream), ws, ws_bytes);
 }
@@ -316,7 +322,7 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     // unrolled matrix (variants 1 and 3 keep the explicit unroll + GEMM path testable):
     // on the tensor-memory path where it has an instance for the layer (variant 4 skips
     // it), else on the warp-level kernels.
-    const int v = variant();
+    const int v = variant_kind();
     if ((v == 0 || v == 2) && conv_tc_supported(*d, X, Wt, ldw, Y)) {
         const RequantParams rqp{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
         return launch_conv_tc(X, Wt, ldw, colsum_w, bias, *d, za, zb, rqp, Y, st) == cudaSuccess
@@ -580,7 +586,7 @@ q4_status q4_last_device_status(void* stream)
 int q4_set_variant(int v)
 {
     const int prev = variant();
-    g_variant.store((v >= 1 && v <= 4) ? v : 0, std::memory_order_relaxed);
+    g_variant.store((v >= 1 && v <= 6) ? v : 0, std::memory_order_relaxed);
     return prev;
 }
 

@@ -16,7 +16,8 @@
 // overlaps the main loop of t+1) and four A stages of 32 columns (128 depth bytes); the
 // unpacked Bt stages live in a deeper shared-memory ring (eight), so only the short
 // tensor-memory store of A sits between "stage free" and "operands ready".  256-column
-// tiles: one accumulator, six A stages, six Bt stages (see Cfg).
+// tiles: three half accumulators of 128 columns in rotation, four A and four Bt stages
+// (see Cfg).
 //
 // Roles per CTA (18 warps): warp 0 TMA producer (its own 128 rows of A, 64-byte-swizzled
 // so that row-per-lane reads are conflict-free, and its own 96 rows of Bt; no
@@ -45,8 +46,7 @@ namespace q4 {
 namespace pair {
 
 constexpr int TMC = 128;             // rows of A per CTA
-constexpr int PROW = 64, UROW = 128, SLAB = 128;
-constexpr int PS = 6;                // packed stages (A 8 KB + Bt BH * 64 B)
+constexpr int PROW = 64, UROW = 128;
 constexpr int PA = TMC * PROW;       // packed A bytes per stage
 #ifndef Q4_PAIR_GROUPS
 #define Q4_PAIR_GROUPS 3
@@ -61,22 +61,37 @@ constexpr int STG_BYTES = 4 * 32 * 128;    // int32 epilogue staging: 4 warps x 
 // accumulators of BNC columns and US A stages of 32 columns.
 // 192 columns: two accumulators (the epilogue of a tile overlaps the next tile's main
 // loop), four A stages, eight Bt stages.
-// 256 columns: one accumulator (its epilogue is exposed once per tile), six A and six Bt
-// stages; a third more work per MMA instruction and per unpacked row of A.  It wins where
-// its tile count fits the 74 CTA pairs better or the depth is long (8192^3: 313 against
-// 332 us; 2048^3 is one wave of 64 tiles: 12.7 against 15.8 us), and loses at 4096^3 (four
-// waves with four exposed epilogues against five overlapped ones).
+// 256 columns: a third more work per unpacked row of A, but two whole accumulators would
+// leave no room for A.  The accumulator is therefore two halves of 128 columns out of three
+// half-buffers (ROT): every tile's upper half (columns 128..255) lives in the middle buffer,
+// the lower halves alternate between the outer two, and each depth step is two MMAs of 128
+// columns (the same tensor time as one of 256).  The epilogue drains the upper half first;
+// the next tile's lower-half MMAs start at once on the free outer buffer and only its
+// upper-half MMAs wait for that half drain, so about a third of the epilogue is exposed
+// instead of all of it.  Four A and four Bt stages.  It wins where its tile count fits the
+// 74 CTA pairs better or the depth is long, and loses e.g. at 4096^3 (four waves against
+// five of 192-column tiles with fully overlapped epilogues).
 template <int BNC_>
 struct Cfg {
     static constexpr int BNC = BNC_;             // columns of the pair tile
     static constexpr int BH = BNC / 2;           // rows of Bt staged per CTA
-    static constexpr int NACC = BNC == 256 ? 1 : 2;
-    static constexpr int US = BNC == 256 ? 6 : 4;   // A operand stages in tensor memory
-    static constexpr int BS = BNC == 256 ? 6 : 8;   // Bt operand stages in shared memory (BH * 128 B each)
+    static constexpr bool ROT = BNC == 256;      // rotating half accumulators
+    static constexpr int NACC = ROT ? 1 : 2;     // whole accumulators / depth-sum buffers in flight
+    static constexpr int US = 4;                 // A operand stages in tensor memory
+#ifndef Q4_PAIR_BS256
+#define Q4_PAIR_BS256 4
+#endif
+    static constexpr int BS = ROT ? Q4_PAIR_BS256 : 8;   // Bt operand stages in shared memory (BH * 128 B each)
+    static constexpr int WALK = BS % US == 0 ? BS : (BS % 2 == 0 ? BS * US / 2 : BS * US);   // a common multiple of both rings
+    static constexpr int BBOX = ROT ? BH / 2 : BH;   // rows per TMA box of Bt
+#ifndef Q4_PAIR_PS256
+#define Q4_PAIR_PS256 8
+#endif
+    static constexpr int PS = ROT ? Q4_PAIR_PS256 : 6;   // packed stages (A 8 KB + Bt BH * 64 B)
     static constexpr int PSTAGE = PA + BH * PROW;
     static constexpr int BSTAGE = BH * UROW;     // unpacked Bt bytes per stage
     static constexpr int NTB = BH * 4 / GT;      // Bt tasks (16-byte packed chunks) per thread per stage
-    static constexpr int ACOL0 = NACC * BNC;     // first TMEM column of the A stages
+    static constexpr int ACOL0 = ROT ? 384 : NACC * BNC;     // first TMEM column of the A stages
     static constexpr int SUMS_N = TMC + BNC;     // per buffer and group: 128 row sums, BNC column sums
 
     static constexpr int OFF_B = 0;
@@ -86,21 +101,21 @@ struct Cfg {
     static constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
     static constexpr int OFF_PC = OFF_COLTERM + BNC * 4;       // per-channel: int32 [4][BNC] zero point, multiplier, rounding, shift
     static constexpr int OFF_BAR = OFF_PC + 4 * BNC * 4;
-    static constexpr int NBAR = 2 * PS + 2 * US + 2 * BS + 10;
+    static constexpr int NBAR = 2 * PS + 2 * US + 2 * BS + 12;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM = OFF_MISC + 16 + 1024;
 
     static_assert(BH * 4 % GT == 0, "Bt tasks must divide evenly");
-    static_assert(NACC * BNC + US * 32 <= TMEM_COLS, "tensor memory budget");
-    static_assert(BS % US == 0, "the MMA loop walks blocks of BS stages and derives the A slot from the position in the block");
+    static_assert(ACOL0 + US * 32 <= TMEM_COLS, "tensor memory budget");
+    static_assert(WALK % BS == 0 && WALK % US == 0, "the MMA loop walks blocks of WALK stages and derives both ring slots from the position in the block");
     static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
     static_assert(OFF_STG % 1024 == 0, "staging tile alignment (128-byte swizzle atoms)");
     static_assert(SMEM <= 227 * 1024, "shared memory budget");
+    static_assert(G <= PS, "a group's packed-ring slot advances by G per stage and wraps at most once");
 
-    // D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC.
-    static constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)(BNC >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+    // D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC (ROT: BNC / 2 per MMA).
+    static constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)((ROT ? BNC / 2 : BNC) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
 };
-static_assert(G <= PS, "a group's packed-ring slot advances by G per stage and wraps at most once");
 
 struct Params {
     GemmParams g;
@@ -137,6 +152,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                   OFF_STG = C::OFF_STG, OFF_SUMS = C::OFF_SUMS, OFF_COLTERM = C::OFF_COLTERM, OFF_PC = C::OFF_PC,
                   OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC;
     constexpr uint32_t kIdesc = C::kIdesc;
+    constexpr bool ROT = C::ROT;
+    constexpr int PS = C::PS, WALK = C::WALK;
     extern __shared__ uint8_t smem_raw[];
     // the same offset in both CTAs: dynamic shared memory starts at the same address
     const uint32_t sbase = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -151,11 +168,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     auto bar_empty_b   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + s); };
     auto bar_full_b    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + BS + s); };
     const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US + 2 * BS);
+    // accumulator buffers: two whole ones, or (ROT) 0 / 1 = the outer half-buffers of even /
+    // odd tiles, 2 = the middle one
     auto bar_tfull       = [&](int a) { return barT + 8u * (uint32_t)a; };
     auto bar_tempty      = [&](int a) { return barT + 8u * (uint32_t)(2 + a); };
-    auto bar_peer_tempty = [&](int a) { return barT + 8u * (uint32_t)(4 + a); };
-    auto bar_sums        = [&](int a) { return barT + 8u * (uint32_t)(6 + a); };
-    auto bar_tstart      = [&](int a) { return barT + 8u * (uint32_t)(8 + a); };
+    auto bar_peer_tempty = [&](int a) { return barT + 8u * (uint32_t)(5 + a); };
+    auto bar_sums        = [&](int a) { return barT + 8u * (uint32_t)(8 + a); };
+    auto bar_tstart      = [&](int a) { return barT + 8u * (uint32_t)(10 + a); };
     const uint32_t tmem_slot = sbase + OFF_MISC;
     const uint32_t abort_flag = sbase + OFF_MISC + 4;
 
@@ -181,10 +200,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull(a), 1);
-            mbar_init(bar_tempty(a), 128);
-            mbar_init(bar_peer_tempty(a), 1);
             mbar_init(bar_sums(a), 2 * UW);      // one arrive per unpack warp of each CTA
             mbar_init(bar_tstart(a), 1);
+        }
+        for (int a = 0; a < 3; ++a) {
+            mbar_init(bar_tempty(a), 128);
+            mbar_init(bar_peer_tempty(a), 1);
         }
         sts32(abort_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -223,7 +244,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters) {
                 const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
                 const int arow = tm * 256 + (int)rank * TMC;
-                const int brow = tn * BNC + (int)rank * BH;
+                // ROT: my Bt rows are two runs of 64, one from each half of the tile's columns
+                const int brow = tn * BNC + (int)rank * C::BBOX;
                 for (int s = 0; s < p.nslab; ++s, ++it) {
                     const int st = it % PS;
                     const uint32_t ph = (it / PS) & 1u;
@@ -233,11 +255,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     tma_load_2d(dst, &tmA, s * PROW, arow, bar_full_p(st));
                     if (!BPRE) {
                         tma_load_2d(dst + PA, &tmB, s * PROW, brow, bar_full_p(st));
+                        if (ROT) tma_load_2d(dst + PA + C::BBOX * PROW, &tmB, s * PROW, brow + BH, bar_full_p(st));
                     } else {
                         const int bst = it % BS;
                         mbar_wait(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
                         mbar_expect_tx(bar_full_b(bst), (uint32_t)BSTAGE);
                         tma_load_2d(sbase + OFF_B + bst * BSTAGE, &tmB, s * UROW, brow, bar_full_b(bst));
+                        if (ROT) tma_load_2d(sbase + OFF_B + bst * BSTAGE + C::BBOX * UROW, &tmB, s * UROW, brow + BH,
+                                             bar_full_b(bst));
                     }
                 }
             }
@@ -249,41 +274,96 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // elected lane issues the MMAs and commits.
             const uint32_t a_tmem0 = tmem_base + (uint32_t)ACOL0;
             const uint64_t bdesc0 = make_kmajor_sw128_desc(sbase + OFF_B);
+            constexpr uint32_t kUpper = (uint32_t)(BH / 2 * UROW >> 4);   // ROT: descriptor offset of Bt rows 64..127
             uint32_t lt = 0;
             for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
                 const int acc = (int)(lt % NACC);
                 const uint32_t aph = (lt / NACC) & 1u;
-                mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
-                if (lt >= (uint32_t)NACC) mbar_wait(bar_peer_tempty(acc), aph ^ 1u, abort_flag, g.status);
-                tc_fence_after();
-                // both epilogues are done with buffer `acc`: tell the unpack warps of both CTAs
-                if (elect_one()) tc_commit_pair(bar_tstart(acc), 3);
-                __syncwarp();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BNC);
                 // Stages are numbered across tiles (stage s of my lt-th tile is lt*nslab + s).
-                // The loop walks them in aligned blocks of BS so that ring slots, tensor-memory
-                // columns, descriptors and barrier addresses are compile-time offsets.
                 const uint32_t it_begin = lt * (uint32_t)p.nslab, it_end = it_begin + (uint32_t)p.nslab;
-                for (uint32_t blk = it_begin - it_begin % BS; blk < it_end; blk += BS) {
+                uint32_t d_tmem, d_up = 0, it_main = it_begin;
+                if (!ROT) {
+                    mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                    if (lt >= (uint32_t)NACC) mbar_wait(bar_peer_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                    tc_fence_after();
+                    // both epilogues are done with buffer `acc`: tell the unpack warps of both CTAs
+                    if (elect_one()) tc_commit_pair(bar_tstart(acc), 3);
+                    __syncwarp();
+                    d_tmem = tmem_base + (uint32_t)(acc * BNC);
+                } else {
+                    // Lower half: the outer buffer of this tile's parity, drained two tiles ago.
+                    const int lo = (int)(lt & 1u);
+                    const uint32_t lph = ((lt >> 1) & 1u) ^ 1u, mph = (lt & 1u) ^ 1u;
+                    mbar_wait(bar_tempty(lo), lph, abort_flag, g.status);
+                    if (lt >= 2u) mbar_wait(bar_peer_tempty(lo), lph, abort_flag, g.status);
+                    tc_fence_after();
+                    d_tmem = tmem_base + (lo ? 256u : 0u);
+                    d_up = tmem_base + 128u;
+                    // The lower-half MMAs of the first stages run while the previous tile's upper
+                    // half is still being drained from the middle buffer ...
+                    const uint32_t la = (uint32_t)p.nslab < (uint32_t)US ? (uint32_t)p.nslab : (uint32_t)US;
+                    for (uint32_t k = 0; k < la; ++k) {
+                        const uint32_t it = it_begin + k;
+                        mbar_wait(bar_full_u((int)(it % US)), (it / US) & 1u, abort_flag, g.status);
+                        tc_fence_after();
+                        const uint32_t a_tmem = a_tmem0 + (it % US) * 32u;
+                        const uint64_t bdesc = bdesc0 + (uint64_t)((it % BS) * (uint32_t)(BSTAGE >> 4));
+                        if (elect_one()) {
+#pragma unroll
+                            for (uint32_t i = 0; i < 4; ++i)
+                                tc_mma_i8_pair_ts(d_tmem, a_tmem + 8u * i, bdesc + 2u * i, kIdesc, (k | i) ? 1u : 0u);
+                        }
+                        __syncwarp();
+                    }
+                    // ... then the upper halves of the same stages, once it is free
+                    mbar_wait(bar_tempty(2), mph, abort_flag, g.status);
+                    if (lt >= 1u) mbar_wait(bar_peer_tempty(2), mph, abort_flag, g.status);
+                    tc_fence_after();
+                    // both epilogues have also read the previous tile's depth sums by now
+                    if (elect_one()) tc_commit_pair(bar_tstart(acc), 3);
+                    __syncwarp();
+                    for (uint32_t k = 0; k < la; ++k) {
+                        const uint32_t it = it_begin + k;
+                        const uint32_t a_tmem = a_tmem0 + (it % US) * 32u;
+                        const uint64_t bdesc = bdesc0 + (uint64_t)((it % BS) * (uint32_t)(BSTAGE >> 4) + kUpper);
+                        if (elect_one()) {
+#pragma unroll
+                            for (uint32_t i = 0; i < 4; ++i)
+                                tc_mma_i8_pair_ts(d_up, a_tmem + 8u * i, bdesc + 2u * i, kIdesc, (k | i) ? 1u : 0u);
+                            tc_commit_pair(bar_empty_b((int)(it % BS)), 3);
+                        }
+                        __syncwarp();
+                    }
+                    it_main = it_begin + la;
+                }
+                // The loop walks the stages in aligned blocks of WALK (a multiple of both ring depths)
+                // so that ring slots, tensor-memory columns, descriptors and barrier addresses are
+                // compile-time offsets.
+                for (uint32_t blk = it_main - it_main % WALK; blk < it_end; blk += WALK) {
                     const uint32_t bph = (blk / US) & 1u;     // phase of A slot 0 in this block
 #pragma unroll
-                    for (int j = 0; j < BS; ++j) {
+                    for (int j = 0; j < WALK; ++j) {
                         const uint32_t it = blk + (uint32_t)j;
-                        if (it < it_begin || it >= it_end) continue;        // warp-uniform
+                        if (it < it_main || it >= it_end) continue;        // warp-uniform
                         // A ring slot j % US: its phase is (it / US) & 1, blk being a multiple of US
                         mbar_wait(bar_full_u(j % US), (bph + (uint32_t)(j / US)) & 1u, abort_flag, g.status);
                         tc_fence_after();
                         const uint32_t a_tmem = a_tmem0 + (uint32_t)((j % US) * 32);
-                        const uint64_t bdesc = bdesc0 + (uint64_t)(j * (BSTAGE >> 4));
+                        const uint64_t bdesc = bdesc0 + (uint64_t)((j % BS) * (BSTAGE >> 4));
                         if (elect_one()) {
                             // a ragged last stage is multiplied whole: its missing depth is zeros
                             tc_mma_i8_pair_ts(d_tmem, a_tmem, bdesc, kIdesc, it > it_begin ? 1u : 0u);
                             tc_mma_i8_pair_ts(d_tmem, a_tmem + 8u, bdesc + 2u, kIdesc, 1u);
                             tc_mma_i8_pair_ts(d_tmem, a_tmem + 16u, bdesc + 4u, kIdesc, 1u);
                             tc_mma_i8_pair_ts(d_tmem, a_tmem + 24u, bdesc + 6u, kIdesc, 1u);
+                            if (ROT) {
+#pragma unroll
+                                for (uint32_t i = 0; i < 4; ++i)
+                                    tc_mma_i8_pair_ts(d_up, a_tmem + 8u * i, bdesc + kUpper + 2u * i, kIdesc, 1u);
+                            }
                             // one commit frees this stage's Bt slot and, through the same
                             // barrier, its A slot (see the unpack warps' wait)
-                            tc_commit_pair(bar_empty_b(j), 3);
+                            tc_commit_pair(bar_empty_b(j % BS), 3);
                         }
                         __syncwarp();
                     }
@@ -294,13 +374,26 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
         } else if (lane == 0) {
             // -------------------------------------------------------- peer relay (per tile)
+            // forwards "my epilogue has drained the buffer" to the leader, which issues the MMAs
             uint32_t lt = 0;
             for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
-                const int acc = (int)(lt % NACC);
-                const uint32_t aph = (lt / NACC) & 1u;
-                if (lt >= (uint32_t)NACC) {
-                    mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
-                    mbar_arrive_cluster(map_to_cta(bar_peer_tempty(acc), 0));
+                if (!ROT) {
+                    const int acc = (int)(lt % NACC);
+                    const uint32_t aph = (lt / NACC) & 1u;
+                    if (lt >= (uint32_t)NACC) {
+                        mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
+                        mbar_arrive_cluster(map_to_cta(bar_peer_tempty(acc), 0));
+                    }
+                } else {
+                    const int lo = (int)(lt & 1u);
+                    if (lt >= 2u) {
+                        mbar_wait(bar_tempty(lo), ((lt >> 1) & 1u) ^ 1u, abort_flag, g.status);
+                        mbar_arrive_cluster(map_to_cta(bar_peer_tempty(lo), 0));
+                    }
+                    if (lt >= 1u) {
+                        mbar_wait(bar_tempty(2), (lt & 1u) ^ 1u, abort_flag, g.status);
+                        mbar_arrive_cluster(map_to_cta(bar_peer_tempty(2), 0));
+                    }
                 }
             }
         }
@@ -417,8 +510,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
                     const int id = gt + j * GT;
                     if ((id & 3) == 0) {
-                        // column sum of my half of Bt: both CTAs need it
-                        const uint32_t a = mine + 4 * (TMC + (int)rank * BH + (id >> 2));
+                        // column sum of one of my rows of Bt: both CTAs need it.  Tile column
+                        // of my row r: my run of BH rows, or (ROT) one of my two runs of 64
+                        const int r = id >> 2;
+                        const int col = !ROT ? (int)rank * BH + r
+                                             : (r < C::BBOX ? (int)rank * C::BBOX + r : BH + (int)rank * C::BBOX + r - C::BBOX);
+                        const uint32_t a = mine + 4 * (TMC + col);
                         sts32(a, t);
                         sts32_cluster(map_to_cta(a, peer), t);
                     }
@@ -481,13 +578,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
             mbar_wait(bar_tfull(acc), aph, abort_flag, g.status);
             tc_fence_after();
-            const uint32_t taddr0 = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(acc * BNC);
+            const uint32_t taddr0 = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(ROT ? 0 : acc * BNC);
 #pragma unroll 1
-            for (int ch = 0; ch < BNC / 32; ++ch) {
+            for (int ci = 0; ci < BNC / 32; ++ci) {
+                // ROT: the upper half (the middle buffer, which the next tile needs first), then
+                // the lower half in this tile's outer buffer
+                const int ch = ROT ? ((ci + BNC / 64) & (BNC / 32 - 1)) : ci;
                 const int nc = n0 + ch * 32;
-                if (nc >= g.N) break;
+                const uint32_t tcol = (ROT && ch < BNC / 64 && (lt & 1u)) ? 256u + (uint32_t)(ch * 32) : (uint32_t)(ch * 32);
+                if (nc < g.N) {            // warp-uniform
                 uint32_t r[32];
-                tc_ld32(taddr0 + (uint32_t)(ch * 32), r);
+                tc_ld32(taddr0 + tcol, r);
                 tc_wait_ld();
                 if (pc) {
                     // the column's own zero point in Eq. 2's row-sum term
@@ -576,9 +677,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         }
                     }
                 }
+                }
+                if (ROT && ci == BNC / 64 - 1) {
+                    // the middle buffer is drained: the next tile's upper-half MMAs may start
+                    tc_fence_before();
+                    mbar_arrive(bar_tempty(2));
+                }
             }
             tc_fence_before();
-            mbar_arrive(bar_tempty(acc));
+            mbar_arrive(bar_tempty(ROT ? (int)(lt & 1u) : acc));
             asm volatile("bar.sync 1, 128;" ::: "memory");
         }
         if (!REQUANT && p.c_tma && lane == 0) bulk_wait_all();   // my TMA stores are complete
@@ -644,7 +751,7 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     return e == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
-// Expanded Bt [N x K8 bytes], pitch ld8: box = 128 bytes x BNC/2 rows, written with the
+// Expanded Bt [N x K8 bytes], pitch ld8: box = 128 bytes x box_rows, written with the
 // 128-byte swizzle, i.e. directly in the layout the MMA's K-major descriptor reads.
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
@@ -699,17 +806,17 @@ bool make_c32_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, int col
 
 // Tile width for a problem: estimated clocks of the busiest CTA pair with either width, from
 // measured stage and epilogue times (192 columns: 520 clk per 128-deep stage, epilogues
-// overlapped but the last; 256 columns: 565 clk per stage and 6200 clk of exposed epilogue
-// per tile).
+// overlapped but the last; 256 columns: 540 clk per stage, 4200 clk per tile of exposed
+// half drain and pipeline restart, 2500 clk for the last half).  Checked against forced
+// widths at 1536^3, 2048^3, 3072^3, 4096^3, 4096 x 11008 x 4096, 6144^3, 8192^3.
 int gemm_tc_pair_width(const GemmParams& g)
 {
-    if (g.N < 256) return 192;
     const long long nslab = ((g.K + 1) / 2 + pair::PROW - 1) / pair::PROW;
     const long long tm = ((long long)g.M + 255) / 256;
     const long long t192 = tm * (((long long)g.N + 191) / 192), t256 = tm * (((long long)g.N + 255) / 256);
     const long long pairs = 74;
     const long long c192 = (t192 + pairs - 1) / pairs * nslab * 520 + 5000;
-    const long long c256 = (t256 + pairs - 1) / pairs * (nslab * 565 + 6200);
+    const long long c256 = (t256 + pairs - 1) / pairs * (nslab * 540 + 4200) + 2500;
     return c256 < c192 ? 256 : 192;
 }
 
@@ -737,20 +844,20 @@ static q4_status launch_pair_w(const GemmParams& g, bool rq, cudaStream_t st, co
     if (b8) {
         // expanded Bt: the kernel cannot take the column sums itself
         if (!g.colsum_b) return Q4_ERR_INVALID_ARG;
-        if (!make_b8_map(&tmB, b8, ld8, g.N, (g.K + 31) / 32 * 32, C::BH)) return Q4_ERR_CUDA;
+        if (!make_b8_map(&tmB, b8, ld8, g.N, (g.K + 31) / 32 * 32, C::BBOX)) return Q4_ERR_CUDA;
         return rq ? launch_pair_t<BNC, true, true>(p, tmA, tmB, tmC, tiles, st)
                   : launch_pair_t<BNC, false, true>(p, tmA, tmB, tmC, tiles, st);
     }
-    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, C::BH, false)) return Q4_ERR_CUDA;
+    if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, C::BBOX, false)) return Q4_ERR_CUDA;
     return rq ? launch_pair_t<BNC, true, false>(p, tmA, tmB, tmC, tiles, st)
               : launch_pair_t<BNC, false, false>(p, tmA, tmB, tmC, tiles, st);
 }
 
 q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8,
-                              int64_t ld8)
+                              int64_t ld8, int width)
 {
-    return gemm_tc_pair_width(g) == 256 ? launch_pair_w<256>(g, rq, st, b8, ld8)
-                                        : launch_pair_w<192>(g, rq, st, b8, ld8);
+    if (width != 192 && width != 256) width = gemm_tc_pair_width(g);
+    return width == 256 ? launch_pair_w<256>(g, rq, st, b8, ld8) : launch_pair_w<192>(g, rq, st, b8, ld8);
 }
 
 }  // namespace q4

@@ -9,6 +9,7 @@ from paper_2009_06488_b200 import workloads as wl
 pytestmark = pytest.mark.gpu
 
 SIMT, TC, TC1 = 1, 2, 3      # general kernel / tensor-core (auto) / single-CTA tensor-core only
+TC192, TC256 = 5, 6          # tensor-core with the CTA-pair kernel's tile width fixed
 
 
 @pytest.fixture(scope="module")
@@ -129,6 +130,34 @@ def test_pair_and_single_tensor_core_kernels_agree_with_oracle(q4, variant, shap
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=16) == wantq).all()
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=3) == wantq).all()   # byte stores
     assert (run_requant(q4, c, variant, rq, c.bias, use_ws=True) == wantq).all()
+    assert (run_requant(q4, c, variant, rq, c.bias, use_ws="expanded") == wantq).all()
+
+
+# Both tile widths of the CTA-pair kernel on the same problems: column tails that leave the
+# upper half of a 256-column tile empty or ragged, depths shorter than the operand rings, and
+# enough tiles per CTA pair (four and more) for the accumulator buffers to go round.
+WIDTH_SHAPES = [(256, 256, 128), (300, 320, 1000), (257, 200, 129), (512, 390, 64), (384, 512, 33),
+                (4096, 4352, 256), (5000, 4100, 130), (2304, 2048, 640)]
+
+
+@pytest.mark.parametrize("variant", [TC192, TC256])
+@pytest.mark.parametrize("shape", WIDTH_SHAPES)
+def test_pair_kernel_tile_widths_agree_with_oracle(q4, variant, shape):
+    M, N, K = shape
+    c = aligned_case(M, N, K, seed=M * 13 + N * 5 + K, with_bias=True)
+    want = oracle.gemm(c.A, c.Bt, M, N, K, c.za, c.zb)
+    got, _, _ = run_gemm(q4, c, variant, ldc_pad=4)           # depth sums taken inside the kernel
+    assert (got == want).all()
+    got, _, _ = run_gemm(q4, c, variant, sums=True)
+    assert (got == want).all()
+    got, _, _ = run_gemm(q4, c, variant, use_ws="expanded")   # Bt expanded once per call
+    assert (got == want).all()
+    got, _, _ = run_gemm(q4, c, variant, ldc_pad=1)           # unaligned int32 pitch: scalar stores
+    assert (got == want).all()
+    rq = oracle.Requant(c.mult, 6, 4, 4, 15)
+    wantq = oracle.requant_matrix(want, c.bias, rq)
+    assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=16) == wantq).all()
+    assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=3) == wantq).all()
     assert (run_requant(q4, c, variant, rq, c.bias, use_ws="expanded") == wantq).all()
 
 

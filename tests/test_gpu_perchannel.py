@@ -65,7 +65,7 @@ FUSED_SHAPES = [(64, 64, 256), (130, 72, 100), (300, 264, 1000), (257, 136, 33),
                 (256, 192, 128), (700, 200, 257), (512, 768, 64), (2048, 1024, 512)]
 
 
-@pytest.mark.parametrize("variant", [3, 2])          # single-CTA / CTA-pair tensor-core kernel
+@pytest.mark.parametrize("variant", [3, 5, 6])       # single-CTA / CTA-pair kernel with 192- and 256-column tiles
 @pytest.mark.parametrize("shape", FUSED_SHAPES)
 @pytest.mark.parametrize("shifts", [(0, 14), (2, 14), (20, 31)])
 def test_per_channel_parameters_in_the_gemm_epilogue(q4, variant, shape, shifts):
