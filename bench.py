@@ -43,7 +43,7 @@ FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel,
 # or None when no capture exists for the kernel as it stands (see profiles/).
-DOMINANT_KERNEL_TRAFFIC_BYTES = 337_080_000   # profiles/gemm_tc_pair_kernel.md, 8192^3 launch of the kernel as it stands
+DOMINANT_KERNEL_TRAFFIC_BYTES = 334_690_000   # profiles/gemm_tc_pair_kernel.md, 8192^3 launch of the kernel as it stands
 
 
 def measured_peaks():
@@ -438,6 +438,14 @@ def time_gemm_sweep(q4, wl, reps: int = 20):
         r = max(3, min(reps, int(2e10 / ops * 4) + 3))
         ms = graph_time_ms([lambda: q4.q4_gemm(A, Bt, C, c.M, c.N, c.K, c.za, c.zb, None, cb, ws)], r)
         out[name] = {"q4_gemm_ms": ms, "q4_gemm_tops": ops / (ms * 1e-3) / 1e12}
+        # context: the library's int8 GEMM (s8 x s8 -> s32, no zero points, no unpack) on the shape
+        try:
+            Ai = torch.randint(-128, 127, (c.M, c.K), dtype=torch.int8, device="cuda")
+            Bi = torch.randint(-128, 127, (c.N, c.K), dtype=torch.int8, device="cuda").t()
+            out[name]["library_int8_ms"] = graph_time_ms([lambda: torch._int_mm(Ai, Bi)], r)
+            del Ai, Bi
+        except Exception as e:      # not every build has it
+            out[name]["library_int8_ms"] = None
         if not name.startswith("c5"):
             Cq = torch.empty((c.M, c.N // 2), dtype=torch.uint8, device="cuda")
             rq = q4.Requant(c.mult, c.shift, 0, 0, 15)
@@ -685,7 +693,7 @@ def run_ours(args):
 
     roofline = {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
                 "frac": gemm_tops / int8_peak, "traffic": DOMINANT_KERNEL_TRAFFIC_BYTES,
-                "kernel": "gemm_tc_pair_kernel<false,false> (q4_gemm 8192^3, int32 output)",
+                "kernel": "gemm_tc_pair_kernel<256,false,false> (q4_gemm 8192^3, int32 output)",
                 "peak_source": f"2 x {peaks['source']} bf16 {'sustained' if sustained else 'burst'} "
                                f"({peaks['bf16_sustained'] if sustained else peaks['bf16']} TFLOP/s): the kernel is "
                                f"timed inside a region of {total_ms / 1e3:.2f} s; nominal int8:bf16 ratio 2",
