@@ -55,7 +55,7 @@ constexpr int G = Q4_PAIR_GROUPS, WPG = 4, GT = WPG * 32;   // unpack groups, wa
 constexpr int UW = G * WPG;
 constexpr int NTHREADS = (2 + UW + 4) * 32;
 constexpr int TMEM_COLS = 512;
-constexpr int STG_BYTES = 4 * 32 * 128;    // int32 epilogue staging: 4 warps x 32 rows x 128 B
+constexpr int STG_SET = 4 * 32 * 128;      // int32 epilogue staging: 4 warps x 32 rows x 128 B
 
 // Two tile widths, chosen per problem by the launcher.  Tensor memory holds NACC
 // accumulators of BNC columns and US A stages of 32 columns.
@@ -71,9 +71,15 @@ constexpr int STG_BYTES = 4 * 32 * 128;    // int32 epilogue staging: 4 warps x 
 // instead of all of it.  Four A and four Bt stages.  It wins where its tile count fits the
 // 74 CTA pairs better or the depth is long, and loses e.g. at 4096^3 (four waves against
 // five of 192-column tiles with fully overlapped epilogues).
-template <int BNC_>
+// NSTG: staging slices per epilogue warp.  With two, a TMA store reads one while the next is
+// filled, which shortens an exposed epilogue (2048^3, one wave: 13.4 -> 12.6 us); the 256-column
+// configuration pays for the second set with a packed stage, which long problems miss
+// (8192^3: 297 -> 302 us), so it exists in both forms and the launcher picks by wave count.
+template <int BNC_, int NSTG_>
 struct Cfg {
     static constexpr int BNC = BNC_;             // columns of the pair tile
+    static constexpr int NSTG = NSTG_;
+    static constexpr int STG_BYTES = NSTG * STG_SET;
     static constexpr int BH = BNC / 2;           // rows of Bt staged per CTA
     static constexpr bool ROT = BNC == 256;      // rotating half accumulators
     static constexpr int NACC = ROT ? 1 : 2;     // whole accumulators / depth-sum buffers in flight
@@ -84,10 +90,7 @@ struct Cfg {
     static constexpr int BS = ROT ? Q4_PAIR_BS256 : 8;   // Bt operand stages in shared memory (BH * 128 B each)
     static constexpr int WALK = BS % US == 0 ? BS : (BS % 2 == 0 ? BS * US / 2 : BS * US);   // a common multiple of both rings
     static constexpr int BBOX = ROT ? BH / 2 : BH;   // rows per TMA box of Bt
-#ifndef Q4_PAIR_PS256
-#define Q4_PAIR_PS256 8
-#endif
-    static constexpr int PS = ROT ? Q4_PAIR_PS256 : 6;   // packed stages (A 8 KB + Bt BH * 64 B)
+    static constexpr int PS = ROT ? (NSTG == 2 ? 7 : 8) : 6;   // packed stages (A 8 KB + Bt BH * 64 B)
     static constexpr int PSTAGE = PA + BH * PROW;
     static constexpr int BSTAGE = BH * UROW;     // unpacked Bt bytes per stage
     static constexpr int NTB = BH * 4 / GT;      // Bt tasks (16-byte packed chunks) per thread per stage
@@ -141,12 +144,12 @@ __device__ __forceinline__ int chunk_sum(const uint4& lo, const uint4& hi, int a
 // BPRE: Bt arrives already expanded to one byte per value (by bt_expand_kernel, once per
 // call, in the same depth order the unpack gives A) and is loaded by TMA straight into
 // the swizzled operand ring; the unpack warps then handle A only.
-template <int BNC, bool REQUANT, bool BPRE>
+template <int BNC, int NSTG, bool REQUANT, bool BPRE>
 __global__ void __launch_bounds__(NTHREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const Params p)
 {
-    using C = Cfg<BNC>;
+    using C = Cfg<BNC, NSTG>;
     constexpr int BH = C::BH, NACC = C::NACC, US = C::US, BS = C::BS, PSTAGE = C::PSTAGE, BSTAGE = C::BSTAGE,
                   NTB = C::NTB, ACOL0 = C::ACOL0, SUMS_N = C::SUMS_N, OFF_B = C::OFF_B, OFF_P = C::OFF_P,
                   OFF_STG = C::OFF_STG, OFF_SUMS = C::OFF_SUMS, OFF_COLTERM = C::OFF_COLTERM, OFF_PC = C::OFF_PC,
@@ -615,8 +618,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     // int32 tile out through shared memory and one TMA store per warp: my
                     // row's 128 bytes go to the swizzled staging slice of my warp; rows and
                     // columns past M / N are clipped by the tensor map
-                    const uint32_t slice = sbase + OFF_STG + (uint32_t)(lg * 4096);
-                    if (lane == 0) bulk_wait_read();       // the previous store has read the slice
+                    const uint32_t slice = sbase + OFF_STG + (uint32_t)(((NSTG > 1 ? (ci & 1) : 0) * 4 + lg) * 4096);
+                    if (lane == 0) {                       // the store that last used this slice has read it
+                        if (NSTG > 1) bulk_wait_read_but_one(); else bulk_wait_read();
+                    }
                     __syncwarp();
 #pragma unroll
                     for (int qd = 0; qd < 8; ++qd)
@@ -711,7 +716,7 @@ bool gemm_tc_pair_supported(const GemmParams& p)
     return gemm_tc_supported(p) && p.M >= 256 && p.N >= 192;
 }
 
-template <int BNC, bool RQ, bool BPRE>
+template <int BNC, int NSTG, bool RQ, bool BPRE>
 static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                const CUtensorMap& tmC, long long tiles, cudaStream_t st)
 {
@@ -719,8 +724,8 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return Q4_ERR_CUDA;
     int& max_clusters = max_clusters_dev[dev];
-    auto kernel = pair::gemm_tc_pair_kernel<BNC, RQ, BPRE>;
-    constexpr int SMEM = pair::Cfg<BNC>::SMEM;
+    auto kernel = pair::gemm_tc_pair_kernel<BNC, NSTG, RQ, BPRE>;
+    constexpr int SMEM = pair::Cfg<BNC, NSTG>::SMEM;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -820,10 +825,10 @@ int gemm_tc_pair_width(const GemmParams& g)
     return c256 < c192 ? 256 : 192;
 }
 
-template <int BNC>
+template <int BNC, int NSTG>
 static q4_status launch_pair_w(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8, int64_t ld8)
 {
-    using C = pair::Cfg<BNC>;
+    using C = pair::Cfg<BNC, NSTG>;
     pair::Params p;
     p.g = g;
     p.tiles_m = (g.M + 255) / 256;
@@ -845,19 +850,22 @@ static q4_status launch_pair_w(const GemmParams& g, bool rq, cudaStream_t st, co
         // expanded Bt: the kernel cannot take the column sums itself
         if (!g.colsum_b) return Q4_ERR_INVALID_ARG;
         if (!make_b8_map(&tmB, b8, ld8, g.N, (g.K + 31) / 32 * 32, C::BBOX)) return Q4_ERR_CUDA;
-        return rq ? launch_pair_t<BNC, true, true>(p, tmA, tmB, tmC, tiles, st)
-                  : launch_pair_t<BNC, false, true>(p, tmA, tmB, tmC, tiles, st);
+        return rq ? launch_pair_t<BNC, NSTG, true, true>(p, tmA, tmB, tmC, tiles, st)
+                  : launch_pair_t<BNC, NSTG, false, true>(p, tmA, tmB, tmC, tiles, st);
     }
     if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, C::BBOX, false)) return Q4_ERR_CUDA;
-    return rq ? launch_pair_t<BNC, true, false>(p, tmA, tmB, tmC, tiles, st)
-              : launch_pair_t<BNC, false, false>(p, tmA, tmB, tmC, tiles, st);
+    return rq ? launch_pair_t<BNC, NSTG, true, false>(p, tmA, tmB, tmC, tiles, st)
+              : launch_pair_t<BNC, NSTG, false, false>(p, tmA, tmB, tmC, tiles, st);
 }
 
 q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8,
                               int64_t ld8, int width)
 {
     if (width != 192 && width != 256) width = gemm_tc_pair_width(g);
-    return width == 256 ? launch_pair_w<256>(g, rq, st, b8, ld8) : launch_pair_w<192>(g, rq, st, b8, ld8);
+    if (width == 192) return launch_pair_w<192, 2>(g, rq, st, b8, ld8);
+    // few tiles per CTA pair: the last tile's exposed epilogue weighs more than ring depth
+    const long long t256 = (((long long)g.M + 255) / 256) * (((long long)g.N + 255) / 256);
+    return t256 <= 3 * 74 ? launch_pair_w<256, 2>(g, rq, st, b8, ld8) : launch_pair_w<256, 1>(g, rq, st, b8, ld8);
 }
 
 }  // namespace q4
