@@ -284,7 +284,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const uint32_t aph = (lt / NACC) & 1u;
                 // Stages are numbered across tiles (stage s of my lt-th tile is lt*nslab + s).
                 const uint32_t it_begin = lt * (uint32_t)p.nslab, it_end = it_begin + (uint32_t)p.nslab;
-                uint32_t d_tmem, d_up = 0, it_main = it_begin;
+                uint32_t d_tmem, d_up = 0, it_main = it_begin, it_tail = it_end;
                 if (!ROT) {
                     mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
                     if (lt >= (uint32_t)NACC) mbar_wait(bar_peer_tempty(acc), aph ^ 1u, abort_flag, g.status);
@@ -338,16 +338,21 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         __syncwarp();
                     }
                     it_main = it_begin + la;
+                    // the stages of the tail (see below): up to US of those left
+                    const uint32_t left = (uint32_t)p.nslab - la;
+                    it_tail = it_end - (left < (uint32_t)US ? left : (uint32_t)US);
+                    if (it_tail == it_end && elect_one()) tc_commit_pair(bar_tfull(1), 3);   // no tail: the upper half is complete
+                    __syncwarp();
                 }
                 // The loop walks the stages in aligned blocks of WALK (a multiple of both ring depths)
                 // so that ring slots, tensor-memory columns, descriptors and barrier addresses are
                 // compile-time offsets.
-                for (uint32_t blk = it_main - it_main % WALK; blk < it_end; blk += WALK) {
+                for (uint32_t blk = it_main - it_main % WALK; blk < it_tail; blk += WALK) {
                     const uint32_t bph = (blk / US) & 1u;     // phase of A slot 0 in this block
 #pragma unroll
                     for (int j = 0; j < WALK; ++j) {
                         const uint32_t it = blk + (uint32_t)j;
-                        if (it < it_main || it >= it_end) continue;        // warp-uniform
+                        if (it < it_main || it >= it_tail) continue;        // warp-uniform
                         // A ring slot j % US: its phase is (it / US) & 1, blk being a multiple of US
                         mbar_wait(bar_full_u(j % US), (bph + (uint32_t)(j / US)) & 1u, abort_flag, g.status);
                         tc_fence_after();
@@ -371,6 +376,36 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         __syncwarp();
                     }
                     (void)bph;
+                }
+                if (ROT && it_tail < it_end) {
+                    // Tail: the last stages' upper-half MMAs first, so that the epilogue can start on
+                    // the middle buffer -- which the next tile needs first -- while their lower-half
+                    // MMAs and the next tile's first lower-half MMAs still run.
+                    for (uint32_t it = it_tail; it < it_end; ++it) {
+                        mbar_wait(bar_full_u((int)(it % US)), (it / US) & 1u, abort_flag, g.status);
+                        tc_fence_after();
+                        const uint32_t a_tmem = a_tmem0 + (it % US) * 32u;
+                        const uint64_t bdesc = bdesc0 + (uint64_t)((it % BS) * (uint32_t)(BSTAGE >> 4) + kUpper);
+                        if (elect_one()) {
+#pragma unroll
+                            for (uint32_t i = 0; i < 4; ++i)
+                                tc_mma_i8_pair_ts(d_up, a_tmem + 8u * i, bdesc + 2u * i, kIdesc, 1u);
+                        }
+                        __syncwarp();
+                    }
+                    if (elect_one()) tc_commit_pair(bar_tfull(1), 3);      // the upper half is complete
+                    __syncwarp();
+                    for (uint32_t it = it_tail; it < it_end; ++it) {
+                        const uint32_t a_tmem = a_tmem0 + (it % US) * 32u;
+                        const uint64_t bdesc = bdesc0 + (uint64_t)((it % BS) * (uint32_t)(BSTAGE >> 4));
+                        if (elect_one()) {
+#pragma unroll
+                            for (uint32_t i = 0; i < 4; ++i)
+                                tc_mma_i8_pair_ts(d_tmem, a_tmem + 8u * i, bdesc + 2u * i, kIdesc, 1u);
+                            tc_commit_pair(bar_empty_b((int)(it % BS)), 3);
+                        }
+                        __syncwarp();
+                    }
                 }
                 if (elect_one()) tc_commit_pair(bar_tfull(acc), 3);
                 __syncwarp();
@@ -579,7 +614,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
             asm volatile("bar.sync 1, 128;" ::: "memory");
 
-            mbar_wait(bar_tfull(acc), aph, abort_flag, g.status);
+            // ROT: barrier 1 = this tile's upper half is complete, barrier 0 = all of it
+            mbar_wait(bar_tfull(ROT ? 1 : acc), aph, abort_flag, g.status);
             tc_fence_after();
             const uint32_t taddr0 = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(ROT ? 0 : acc * BNC);
 #pragma unroll 1
@@ -687,6 +723,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     // the middle buffer is drained: the next tile's upper-half MMAs may start
                     tc_fence_before();
                     mbar_arrive(bar_tempty(2));
+                    mbar_wait(bar_tfull(0), aph, abort_flag, g.status);
+                    tc_fence_after();
                 }
             }
             tc_fence_before();
