@@ -250,11 +250,14 @@ def graph_time_ms(calls, reps: int, rounds: int = 5) -> float:
     return statistics.median(ts)
 
 
-def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20, net=None, hbm_peak: float | None = None):
+def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20, net=None, hbm_peak: float | None = None,
+                  prepared: bool = False):
     """Device time of every layer of a layer chain (default: the c4 chain) and of the whole
     chain.  Each layer: `reps` launches replayed from a CUDA graph, and -- as a cross-check --
     launched eagerly back to back behind a busy GPU.  The chain: all layers in order, each
-    feeding the next, `reps // 2` times from one graph."""
+    feeding the next, `reps // 2` times from one graph.  prepared: the layers that have a
+    tensor-memory kernel run from a weight image prepared once (q4_conv2d_prepare_weights /
+    q4_conv2d_prepared) instead of preparing their weights inside every launch."""
     import torch
     if net is None:
         net = wl.c4(batch=batch, seed=4000, centred=True)
@@ -271,6 +274,12 @@ def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20, net=None, hbm_peak:
         rq = q4.Requant(L.mult, L.shift, L.zo, L.clamp_lo, L.clamp_hi)
         call = (lambda Xf=X.reshape(-1), Wt=Wt, d=d, L=L, rq=rq, Y=Y, ws=ws, b=b, cw=cw:
                 q4.q4_conv2d(Xf, Wt, d, L.za, L.zb, rq, Y, ws, b, cw))
+        nimg = q4.q4_conv2d_weights_bytes(d) if prepared else 0
+        if nimg:
+            img = torch.empty(nimg, dtype=torch.uint8, device="cuda")
+            q4.q4_conv2d_prepare_weights(Wt, d, L.za, L.zb, img, b, cw)
+            call = (lambda Xf=X.reshape(-1), img=img, d=d, L=L, rq=rq, Y=Y:
+                    q4.q4_conv2d_prepared(Xf, img, d, L.za, rq, Y))
         calls.append(call)
         for _ in range(3):
             call()
@@ -300,7 +309,8 @@ def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20, net=None, hbm_peak:
            "layers": layers,
            "timing": f"`ms`: the whole chain replayed {max(2, reps // 2)} times from one CUDA graph, median of 5; "
                      f"per layer: {reps} launches from a CUDA graph (`ms`) and eager back to back (`ms_eager`); "
-                     "weight sums prepared once"}
+                     + ("weights prepared once (q4_conv2d_prepare_weights) where the layer has a tensor-memory kernel"
+                        if prepared else "weight sums prepared once")}
     if hbm_peak:
         out["frac_of_hbm"] = out["compulsory_gbs"] / hbm_peak
     return out

@@ -161,6 +161,35 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                     uint8_t* Y, void* ws, size_t ws_bytes, void* stream);
 
 /*
+ * Convolution layers with the weight-side work done once (Section II-B: what depends only
+ * on the weights -- here their zero-point-corrected, tile-ordered copy and the per-channel
+ * constants of Eq. 3 -- "can be computed only once").  For the layer classes that run on
+ * the tensor-memory kernels, q4_conv2d_prepare_weights writes that copy (an opaque image,
+ * valid for this descriptor, za, zb, bias and this build of the library) into `prepared`,
+ * and q4_conv2d_prepared runs the layer from it: the same arithmetic and the same output
+ * bytes as q4_conv2d, without the per-launch weight preparation inside the kernel (3 to 5
+ * thousand clocks per CTA).
+ *
+ * q4_conv2d_weights_bytes: bytes of the image for the layer, 0 if the layer's geometry has no
+ * such kernel (then use q4_conv2d).  Host call, no device access.
+ * q4_conv2d_prepare_weights: Wt, ldw, colsum_w (optional), bias (optional), za, zb as in
+ * q4_conv2d; `prepared` a device buffer of at least q4_conv2d_weights_bytes(d) bytes, 16-byte
+ * aligned, owned by the caller, written by one small kernel on `stream`.
+ * q4_conv2d_prepared: X, Y, rq, za as in q4_conv2d (za must be the one the image was
+ * prepared with); needs no workspace.
+ * Errors: as q4_conv2d; Q4_ERR_UNSUPPORTED when the layer (or the alignment of X / Y: 16
+ * bytes) has no tensor-memory kernel, Q4_ERR_WORKSPACE when prepared_bytes is too small,
+ * Q4_ERR_ALIGNMENT when `prepared` is not 16-byte aligned.  Nothing is launched on error.
+ */
+size_t q4_conv2d_weights_bytes(const q4_conv_desc* d);
+q4_status q4_conv2d_prepare_weights(const uint8_t* Wt, int64_t ldw, const int32_t* colsum_w,
+                                    const int32_t* bias, const q4_conv_desc* d, int32_t za, int32_t zb,
+                                    void* prepared, size_t prepared_bytes, void* stream);
+q4_status q4_conv2d_prepared(const uint8_t* X, const void* prepared, size_t prepared_bytes,
+                             const q4_conv_desc* d, int32_t za, const q4_requant* rq, uint8_t* Y,
+                             void* stream);
+
+/*
  * q4_conv2d for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of q4_conv2d, same arithmetic, same
  * kernels, same results.)

@@ -37,7 +37,8 @@ EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_st
            "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak",
            "q4_quant_params", "q4_quantize", "q4_dequantize", "q4_gemm_u8",
            "q4_gemm_u8_workspace_bytes", "q4_selftest_wait_timeout", "q4_requant_channels", "q4_conv2d_channels",
-           "q4_gemm_requant_channels"]
+           "q4_gemm_requant_channels", "q4_conv2d_weights_bytes", "q4_conv2d_prepare_weights",
+           "q4_conv2d_prepared"]
 
 
 class Q4Error(RuntimeError):
@@ -112,6 +113,10 @@ _lib.q4_conv2d.argtypes = [_vp, _vp, _i64, _vp, _vp, ctypes.POINTER(_ConvDesc), 
                            ctypes.POINTER(_Requant), _vp, _vp, _sz, _vp]
 _lib.q4_conv2d_static.argtypes = [_vp, _vp, _i64, _vp, _vp, ctypes.POINTER(_ConvDesc), _i32, _i32,
                                   ctypes.POINTER(_Requant), _vp, _vp]
+_lib.q4_conv2d_weights_bytes.argtypes = [ctypes.POINTER(_ConvDesc)]
+_lib.q4_conv2d_weights_bytes.restype = _sz
+_lib.q4_conv2d_prepare_weights.argtypes = [_vp, _i64, _vp, _vp, ctypes.POINTER(_ConvDesc), _i32, _i32, _vp, _sz, _vp]
+_lib.q4_conv2d_prepared.argtypes = [_vp, _vp, _sz, ctypes.POINTER(_ConvDesc), _i32, ctypes.POINTER(_Requant), _vp, _vp]
 _lib.q4_gemm_workspace_bytes.argtypes = [_i32, _i32, _i32]
 _lib.q4_gemm_workspace_bytes.restype = _sz
 _lib.q4_gemm_workspace_bytes_expanded.argtypes = [_i32, _i32, _i32]
@@ -278,6 +283,33 @@ def q4_conv2d_static(X, Wt, d: ConvDesc, za: int, zb: int, rq: Requant, Y, bias=
     _check(_lib.q4_conv2d_static(_ptr(X), _ptr(Wt), _rows(Wt, "Wt"), _ptr(colsum_w), _ptr(bias),
                                  ctypes.byref(c), za, zb, ctypes.byref(r), _ptr(Y), _stream()),
            "q4_conv2d_static")
+    return Y
+
+
+def q4_conv2d_weights_bytes(d: ConvDesc) -> int:
+    """Bytes of the layer's prepared weight image, 0 if the layer has no tensor-memory kernel."""
+    c = d._c()
+    return int(_lib.q4_conv2d_weights_bytes(ctypes.byref(c)))
+
+
+def q4_conv2d_prepare_weights(Wt, d: ConvDesc, za: int, zb: int, prepared, bias=None, colsum_w=None):
+    """The layer's weight-side work, once: writes the opaque image q4_conv2d_prepared runs from
+    into ``prepared`` (uint8 CUDA tensor of q4_conv2d_weights_bytes(d) bytes); see include/q4.h."""
+    _dev(Wt, torch.uint8, "Wt"); _dev(prepared, torch.uint8, "prepared")
+    _dev(bias, torch.int32, "bias"); _dev(colsum_w, torch.int32, "colsum_w")
+    c = d._c()
+    _check(_lib.q4_conv2d_prepare_weights(_ptr(Wt), _rows(Wt, "Wt"), _ptr(colsum_w), _ptr(bias), ctypes.byref(c),
+                                          za, zb, _ptr(prepared), prepared.numel(), _stream()),
+           "q4_conv2d_prepare_weights")
+    return prepared
+
+
+def q4_conv2d_prepared(X, prepared, d: ConvDesc, za: int, rq: Requant, Y):
+    """q4_conv2d from a prepared weight image (same output bytes, no workspace); see include/q4.h."""
+    _dev(X, torch.uint8, "X"); _dev(prepared, torch.uint8, "prepared"); _dev(Y, torch.uint8, "Y")
+    c, r = d._c(), rq._c()
+    _check(_lib.q4_conv2d_prepared(_ptr(X), _ptr(prepared), prepared.numel(), ctypes.byref(c), za,
+                                   ctypes.byref(r), _ptr(Y), _stream()), "q4_conv2d_prepared")
     return Y
 
 

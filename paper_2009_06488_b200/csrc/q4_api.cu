@@ -365,6 +365,57 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     return run_gemm(p, true, st);
 }
 
+size_t q4_conv2d_weights_bytes(const q4_conv_desc* d)
+{
+    if (!d || check_conv(d, 0) != Q4_OK || d->OC <= 0 || (d->OC & 1)) return 0;
+    return conv_tc_image_bytes(*d);
+}
+
+q4_status q4_conv2d_prepare_weights(const uint8_t* Wt, int64_t ldw, const int32_t* colsum_w,
+                                    const int32_t* bias, const q4_conv_desc* d, int32_t za, int32_t zb,
+                                    void* prepared, size_t prepared_bytes, void* stream)
+{
+    q4_status s = check_conv(d, za);
+    if (s != Q4_OK) return s;
+    if (zb < 0 || zb > 15) return Q4_ERR_RANGE;
+    if (d->OC <= 0 || (d->OC & 1)) return Q4_ERR_INVALID_ARG;
+    const ConvShape cs = conv_shape(d);
+    if (ldw < ((int64_t)cs.K + 1) / 2) return Q4_ERR_INVALID_ARG;
+    if (!Wt || !prepared) return Q4_ERR_INVALID_ARG;
+    const size_t need = conv_tc_image_bytes(*d);
+    if (need == 0) return Q4_ERR_UNSUPPORTED;
+    if (prepared_bytes < need) return Q4_ERR_WORKSPACE;
+    if ((uintptr_t)prepared % 16 != 0) return Q4_ERR_ALIGNMENT;
+    const RequantParams rqp{1 << 30, 0, 0, 0, 15};       // not used by the preparation
+    return launch_conv_tc(nullptr, Wt, ldw, colsum_w, bias, *d, za, zb, rqp, nullptr,
+                          static_cast<cudaStream_t>(stream), nullptr, static_cast<uint8_t*>(prepared)) == cudaSuccess
+               ? Q4_OK : Q4_ERR_CUDA;
+}
+
+q4_status q4_conv2d_prepared(const uint8_t* X, const void* prepared, size_t prepared_bytes,
+                             const q4_conv_desc* d, int32_t za, const q4_requant* rq, uint8_t* Y,
+                             void* stream)
+{
+    q4_status s = check_conv(d, za);
+    if (s != Q4_OK) return s;
+    if ((s = check_requant(rq)) != Q4_OK) return s;
+    if (d->OC <= 0 || (d->OC & 1)) return Q4_ERR_INVALID_ARG;
+    if (!prepared) return Q4_ERR_INVALID_ARG;
+    const size_t need = conv_tc_image_bytes(*d);
+    if (need == 0) return Q4_ERR_UNSUPPORTED;
+    if (prepared_bytes < need) return Q4_ERR_WORKSPACE;
+    if ((uintptr_t)prepared % 16 != 0) return Q4_ERR_ALIGNMENT;
+    const ConvShape cs = conv_shape(d);
+    if (cs.M == 0) return Q4_OK;
+    if (!X || !Y) return Q4_ERR_INVALID_ARG;
+    const int v = variant_kind();
+    if ((v != 0 && v != 2) || !conv_tc_supported(*d, X, nullptr, 0, Y)) return Q4_ERR_UNSUPPORTED;
+    const RequantParams rqp{rq->mult, rq->shift, rq->zo, rq->clamp_lo, rq->clamp_hi};
+    return launch_conv_tc(X, nullptr, 0, nullptr, nullptr, *d, za, 0, rqp, Y, static_cast<cudaStream_t>(stream),
+                          static_cast<const uint8_t*>(prepared), nullptr) == cudaSuccess
+               ? Q4_OK : Q4_ERR_CUDA;
+}
+
 q4_status q4_conv2d_static(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                            const int32_t* colsum_w, const int32_t* bias,
                            const q4_conv_desc* d, int32_t za, int32_t zb, const q4_requant* rq,

@@ -22,6 +22,10 @@ struct Params {
     const int32_t* mult_ch;
     const int32_t* shift_ch;
     uint8_t* Y;
+    // the tensor-memory kernels' weight image (the B operand, the per-column constants, a flag):
+    // prep_out = build it and write it there, do nothing else; prep_in = take it from there
+    const uint8_t* prep_in;
+    uint8_t* prep_out;
     int64_t M;
     int32_t H, W, C, KH, KW, OH, OW, sh, sw, ph, pw;
     int32_t K, KS;             // depth, number of 32-byte MMA depth steps

@@ -94,7 +94,7 @@ struct Shape {
 };
 
 constexpr int GMAX = 6;             // worker groups
-constexpr int NBAR = 2 * NBMAX + 2 * GMAX;
+constexpr int NBAR = 2 * NBMAX + 2 * GMAX + 2;      // (an even count keeps what follows 16-byte aligned)
 template <class S> struct Layout {
     static constexpr int OFF_B = 0;
     static constexpr int OFF_CT = OFF_B + S::B_BYTES;         // int32 [N] per-column constants
@@ -340,6 +340,7 @@ conv_tc_kernel(const Params p)
     const uint32_t full0 = bar0, empty0 = bar0 + 8 * NBMAX;
     auto bar_a_ready  = [&](int g) { return bar0 + 8u * (uint32_t)(2 * NBMAX + g); };
     auto bar_mma_done = [&](int g) { return bar0 + 8u * (uint32_t)(2 * NBMAX + GMAX + g); };
+    const uint32_t bar_prep = bar0 + 8u * (uint32_t)(2 * NBMAX + 2 * GMAX);     // a prepared weight image has landed
     const int NB = p.nbuf;
     const uint32_t tmem_slot = sbase + L::OFF_MISC, abort_flag = sbase + L::OFF_MISC + 4;
     const uint32_t preload_flag = sbase + L::OFF_MISC + 8;
@@ -357,6 +358,7 @@ conv_tc_kernel(const Params p)
             mbar_init(bar_a_ready(g), 4);
             mbar_init(bar_mma_done(g), 1);
         }
+        mbar_init(bar_prep, 1);
         sts32(abort_flag, 0);
         sts32(preload_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -384,7 +386,17 @@ conv_tc_kernel(const Params p)
     // prepare the weights (synchronising among themselves on a named barrier).
     uint32_t tmem_base = 0;
     bool use_preload = false;              // a constant beyond the digits' range: preloaded accumulators instead
-    if (warp >= PWN) {
+    constexpr uint32_t IMAGE = (uint32_t)(S::B_BYTES + N * 4);     // B and the per-column constants, contiguous
+    if (warp >= PWN && p.prep_in != nullptr) {
+        // The weights were prepared ahead of time (the B operand, the constants, the flag):
+        // one bulk copy brings them in; only the MMA warp has to wait for it.
+        if (tid == PWN * 32) {
+            mbar_expect_tx(bar_prep, IMAGE);
+            fused::bulk_load_row(sbase + L::OFF_B, p.prep_in, IMAGE, bar_prep);
+        }
+        use_preload = __ldg(reinterpret_cast<const int*>(p.prep_in + IMAGE)) != 0;
+        tmem_base = (uint32_t)lds32(tmem_slot);
+    } else if (warp >= PWN) {
         constexpr int NT = THREADS - PWN * 32;         // threads that prepare the weights
         constexpr int TASKS = N * KS * 4;              // eight-byte groups of B
         const int wt = tid - PWN * 32;
@@ -396,17 +408,48 @@ conv_tc_kernel(const Params p)
         // j = nibble / C and channel c = nibble % C, which is tap kw = j - px*sw of pixel px
         // if that is a tap at all.  Even nibbles go to bytes 0..3, odd ones to bytes 4..7 of
         // the eight-byte group -- the order the workers give A.
-#pragma unroll 8
-        for (int it = 0; it < (TASKS + NT - 1) / NT; ++it) {
+        // Two passes: first every packed word this thread needs is requested (the loads'
+        // latencies overlap), then the words are expanded and stored.
+        constexpr int NIT = (TASKS + NT - 1) / NT;
+        // where task idx finds its packed word: row n, depth word wd -> (valid, channel, tap, word)
+        auto locate = [&](int idx, int& n, int& wd, int& px, int& oc, int& kh, int& i) {
+            n = idx / (KS * 4); wd = idx - n * (KS * 4);
+            px = n / OC;
+            const int ocp = n - px * OC;
+            oc = (ocp & ~7) + ch8(ocp & 7);            // the channel this column stands for
+            kh = wd / WW; i = wd - kh * WW;
+        };
+        uint32_t wv[NIT];
+        if constexpr (!S::NIB) {
+#pragma unroll
+            for (int it = 0; it < NIT; ++it) {
+                const int idx = wt + it * NT;
+                wv[it] = 0;
+                int n, wd, px, oc, kh, i;
+                locate(idx, n, wd, px, oc, kh, i);
+                // word i of the window row is word cw of input column j: one packed word
+                // of the weights where that column is a tap of pixel px
+                const int j = i / S::CW, cw = i - j * S::CW;
+                const int kw = j - px * S::SW;
+                if (idx < TASKS && wd < S::NW && kw >= 0 && kw < S::KW) {
+                    const uint8_t* src = p.Wt + (int64_t)oc * p.ldw + ((kh * S::KW + kw) * S::C) / 2 + 4 * cw;
+                    if (p.wt_words) {
+                        wv[it] = __ldg(reinterpret_cast<const uint32_t*>(src));
+                    } else {
+                        for (int q = 0; q < 4; ++q) wv[it] |= (uint32_t)__ldg(src + q) << (8 * q);
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < NIT; ++it) {
             const int idx = wt + it * NT;
             if (idx >= TASKS) break;
-            const int n = idx / (KS * 4), wd = idx - n * (KS * 4);
-            const int px = n / OC, ocp = n - px * OC;
-            const int oc = (ocp & ~7) + ch8(ocp & 7);  // the channel this column stands for
+            int n, wd, px, oc, kh, i;
+            locate(idx, n, wd, px, oc, kh, i);
             uint32_t lo = 0, hi = 0;
             int raw = 0;
             if (wd < S::NW) {
-                const int kh = wd / WW, i = wd - kh * WW;
                 if constexpr (S::NIB) {
 #pragma unroll
                     for (int e = 0; e < 8; ++e) {
@@ -420,22 +463,12 @@ conv_tc_kernel(const Params p)
                         }
                     }
                 } else {
-                    // word i of the window row is word cw of input column j: one packed word
-                    // of the weights where that column is a tap of pixel px
-                    const int j = i / S::CW, cw = i - j * S::CW;
+                    const int j = i / S::CW;
                     const int kw = j - px * S::SW;
                     if (kw >= 0 && kw < S::KW) {
-                        const uint8_t* src = p.Wt + (int64_t)oc * p.ldw + ((kh * S::KW + kw) * S::C) / 2 + 4 * cw;
-                        uint32_t wv;
-                        if (p.wt_words) {
-                            wv = *reinterpret_cast<const uint32_t*>(src);
-                        } else {
-                            wv = 0;
-                            for (int q = 0; q < 4; ++q) wv |= (uint32_t)src[q] << (8 * q);
-                        }
-                        raw = nibble_sum(wv);
-                        lo = fused::sub_zb(wv & 0x0F0F0F0Fu, (uint32_t)p.zb);
-                        hi = fused::sub_zb((wv >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                        raw = nibble_sum(wv[it]);
+                        lo = fused::sub_zb(wv[it] & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                        hi = fused::sub_zb((wv[it] >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
                     }
                 }
             }
@@ -505,6 +538,13 @@ conv_tc_kernel(const Params p)
         sync_workers();
         tc_fence_after();
         tmem_base = (uint32_t)lds32(tmem_slot);
+        if (p.prep_out != nullptr) {
+            // preparation only: the image goes to memory (this launch has no tiles)
+            const uint4* src = reinterpret_cast<const uint4*>(smem + L::OFF_B);
+            uint4* dst = reinterpret_cast<uint4*>(p.prep_out);
+            for (int i = wt; i < (int)(IMAGE / 16); i += NT) dst[i] = src[i];
+            if (wt == 0) dst[IMAGE / 16] = make_uint4(use_preload ? 1u : 0u, 0u, 0u, 0u);
+        }
     }
 
     if (warp < PWN) {
@@ -518,6 +558,7 @@ conv_tc_kernel(const Params p)
         const uint64_t bdesc0 = make_kmajor_sw128_desc(sbase + L::OFF_B);
         int g = 0;
         uint32_t t = 0;                                // tile k is group g's t-th tile
+        if (p.prep_in != nullptr && mytiles > 0) mbar_wait(bar_prep, 0, abort_flag, p.status);
         for (int k = 0; k < mytiles; ++k) {
             TR(1, k, 0);
             if (!wait_idle(bar_a_ready(g), t & 1u, abort_flag, p.status)) break;
@@ -641,6 +682,7 @@ conv_tc_kernel(const Params p)
                 tc_st8(a_taddr + (uint32_t)(8 * ks), r8);
             }
             if (use_preload) {
+                if (p.prep_in != nullptr) mbar_wait(bar_prep, 0, abort_flag, p.status);     // the constants are in the image
 #pragma unroll
                 for (int j = 0; j < N / 8; ++j) {
                     const uint4 x = lds128(colterm_s + 4 * (8 * j)), y = lds128(colterm_s + 4 * (8 * j + 4));
@@ -723,12 +765,11 @@ constexpr int WNCH = 4;             // chunks in the ring
 #endif
 constexpr int WSB = Q4_CTC_WSB, WSE = Q4_CTC_WSE;     // build / epilogue warps per lane quarter
 constexpr int WPW = 2;              // producer warps (a tile is one bulk copy per image; two keep up)
-constexpr int WNBAR = 2 * NBMAX + 2 * WNCH + 4;
-// A build set's consecutive chunks are at most 2 * WSB - 1 chunks apart (the last one of a tile
-// and the first one of the next).  A set that waits for a ring slot must not be more than one
-// use of that slot ahead of the MMA warp (mbarrier phases are told apart by one parity bit),
-// so the distance has to stay within the ring.
-static_assert(2 * WSB - 1 <= WNCH, "build sets may run at most one ring round ahead");
+constexpr int WNBAR = 2 * NBMAX + 2 * WNCH + 6;     // (even: what follows stays 16-byte aligned)
+// A build set's consecutive chunks are WSB chunks apart.  A set that waits for a ring slot must
+// not be more than one use of that slot ahead of the MMA warp (mbarrier phases are told apart
+// by one parity bit), so the distance has to stay within the ring.
+static_assert(WSB <= WNCH, "build sets may run at most one ring round ahead");
 
 struct WideLayout {
     int off_tab, off_ct, off_geo, off_bar, off_misc, off_buf;     // after B (at 0)
@@ -774,6 +815,7 @@ conv_tc_wide_kernel(const Params p)
     auto bar_a_free    = [&](int c) { return bar0 + 8u * (uint32_t)(2 * NBMAX + WNCH + c); };
     auto bar_acc_full  = [&](int a) { return bar0 + 8u * (uint32_t)(2 * NBMAX + 2 * WNCH + a); };
     auto bar_acc_empty = [&](int a) { return bar0 + 8u * (uint32_t)(2 * NBMAX + 2 * WNCH + 2 + a); };
+    const uint32_t bar_prep = bar0 + 8u * (uint32_t)(2 * NBMAX + 2 * WNCH + 4);      // a prepared weight image has landed
     const int NB = p.nbuf;
     const uint32_t tmem_slot = sbase + L.off_misc, abort_flag = sbase + L.off_misc + 4;
     const uint32_t preload_flag = sbase + L.off_misc + 8;
@@ -798,6 +840,7 @@ conv_tc_wide_kernel(const Params p)
             mbar_init(bar_acc_full(a), 1);
             mbar_init(bar_acc_empty(a), 4 * WSE);
         }
+        mbar_init(bar_prep, 1);
         sts32(abort_flag, 0);
         sts32(preload_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -822,7 +865,9 @@ conv_tc_wide_kernel(const Params p)
         constexpr int NT = WIDE_THREADS - WPW * 32;
         const int wt = tid - WPW * 32;
         auto sync_workers = [] { asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory"); };
-        for (int i = wt; i < N; i += NT) colterm[i] = 0;
+        const bool prepared = p.prep_in != nullptr;
+        if (!prepared)
+            for (int i = wt; i < N; i += NT) colterm[i] = 0;
         // depth step ks = (kh, kw, c4): where its 16 bytes sit relative to a pixel's window
         // start, and which window column it belongs to
         for (int ks = wt; ks < KS; ks += NT) {
@@ -831,38 +876,65 @@ conv_tc_wide_kernel(const Params p)
             tab[ks] = make_int2(kh * p.rowbytes + kw * p.unit + 16 * c4, kw);
         }
         sync_workers();
+        // a CTA's share of a prepared image: B, the per-column constants, 16 bytes with the flag
+        const uint32_t b_bytes = (uint32_t)L.off_tab, share_bytes = b_bytes + (uint32_t)N * 4u + 16u;
+        if (prepared) {
+            const uint8_t* img = p.prep_in + (size_t)(blockIdx.x % nsplit) * share_bytes;
+            if (wt == 0) {
+                mbar_expect_tx(bar_prep, b_bytes + (uint32_t)N * 4u);
+                fused::bulk_load_row(sbase, img, b_bytes, bar_prep);
+                fused::bulk_load_row(colterm_s, img + b_bytes, (uint32_t)N * 4u, bar_prep);
+            }
+            use_preload = __ldg(reinterpret_cast<const int*>(img + b_bytes + (uint32_t)N * 4u)) != 0;
+            tmem_base = (uint32_t)lds32(tmem_slot);
+        } else {
         // B: row n is output channel oc0 + (n with the ch8 order inside each group of eight);
         // depth step ks is bytes 16 ks .. 16 ks + 15 of the weight row
         const int tasks = N * KS;
-#pragma unroll 4
-        for (int idx = wt; idx < tasks; idx += NT) {
-            const int n = idx / KS, ks = idx - n * KS;
-            const int oc = oc0 + (n & ~7) + ch8(n & 7);
-            const uint8_t* src = p.Wt + (int64_t)oc * p.ldw + 16 * ks;
-            uint32_t wv[4];
-            if (p.wt_words) {
+        const bool wt_vec = (((uintptr_t)p.Wt | (uintptr_t)p.ldw) & 15) == 0;
+        // four tasks at a time: all their loads are requested before any is expanded
+        for (int base = wt; base < tasks; base += 4 * NT) {
+            uint4 wq[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) wv[j] = reinterpret_cast<const uint32_t*>(src)[j];
-            } else {
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    wv[j] = 0;
-                    for (int q = 0; q < 4; ++q) wv[j] |= (uint32_t)src[4 * j + q] << (8 * q);
+            for (int u = 0; u < 4; ++u) {
+                const int idx = base + u * NT;
+                wq[u] = make_uint4(0, 0, 0, 0);
+                if (idx < tasks) {
+                    const int n = idx / KS, ks = idx - n * KS;
+                    const int oc = oc0 + (n & ~7) + ch8(n & 7);
+                    const uint8_t* src = p.Wt + (int64_t)oc * p.ldw + 16 * ks;
+                    if (wt_vec) {
+                        wq[u] = __ldg(reinterpret_cast<const uint4*>(src));
+                    } else if (p.wt_words) {
+                        const uint32_t* s4 = reinterpret_cast<const uint32_t*>(src);
+                        wq[u] = make_uint4(__ldg(s4), __ldg(s4 + 1), __ldg(s4 + 2), __ldg(s4 + 3));
+                    } else {
+                        uint32_t t[4] = {0, 0, 0, 0};
+                        for (int b = 0; b < 16; ++b) t[b >> 2] |= (uint32_t)__ldg(src + b) << (8 * (b & 3));
+                        wq[u] = make_uint4(t[0], t[1], t[2], t[3]);
+                    }
                 }
             }
-            uint32_t o[8];
-            int raw = 0;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                raw += nibble_sum(wv[j]);
-                o[2 * j] = fused::sub_zb(wv[j] & 0x0F0F0F0Fu, (uint32_t)p.zb);
-                o[2 * j + 1] = fused::sub_zb((wv[j] >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
+            for (int u = 0; u < 4; ++u) {
+                const int idx = base + u * NT;
+                if (idx >= tasks) break;
+                const int n = idx / KS, ks = idx - n * KS;
+                const uint32_t wv[4] = {wq[u].x, wq[u].y, wq[u].z, wq[u].w};
+                uint32_t o[8];
+                int raw = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    raw += nibble_sum(wv[j]);
+                    o[2 * j] = fused::sub_zb(wv[j] & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                    o[2 * j + 1] = fused::sub_zb((wv[j] >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                }
+                uint8_t* row = smem + (ks >> 2) * (N * 128) + n * 128;
+                const int c = 2 * (ks & 3);
+                *reinterpret_cast<uint4*>(row + ((c ^ (n & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint4*>(row + (((c + 1) ^ (n & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
+                if (!p.colsum_w && raw) atomicAdd(&colterm[n], raw);          // by column position
             }
-            uint8_t* row = smem + (ks >> 2) * (N * 128) + n * 128;
-            const int c = 2 * (ks & 3);
-            *reinterpret_cast<uint4*>(row + ((c ^ (n & 7)) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-            *reinterpret_cast<uint4*>(row + (((c + 1) ^ (n & 7)) << 4)) = make_uint4(o[4], o[5], o[6], o[7]);
-            if (!p.colsum_w && raw) atomicAdd(&colterm[n], raw);          // by column position
         }
         sync_workers();
         int cterm = 0;
@@ -914,6 +986,17 @@ conv_tc_wide_kernel(const Params p)
         sync_workers();
         tc_fence_after();
         tmem_base = (uint32_t)lds32(tmem_slot);
+        if (p.prep_out != nullptr) {
+            // preparation only: my share of the image goes to memory (this launch has no tiles)
+            uint8_t* img = p.prep_out + (size_t)(blockIdx.x % nsplit) * share_bytes;
+            const uint4* src = reinterpret_cast<const uint4*>(smem);
+            uint4* dst = reinterpret_cast<uint4*>(img);
+            for (int i = wt; i < (int)(b_bytes / 16); i += NT) dst[i] = src[i];
+            const uint4* cs = reinterpret_cast<const uint4*>(smem + L.off_ct);
+            for (int i = wt; i < N / 4; i += NT) dst[b_bytes / 16 + i] = cs[i];
+            if (wt == 0) dst[b_bytes / 16 + N / 4] = make_uint4(use_preload ? 1u : 0u, 0u, 0u, 0u);
+        }
+        }
     }
 
     if (warp < WPW) {
@@ -926,6 +1009,7 @@ conv_tc_wide_kernel(const Params p)
         const uint32_t blk = (uint32_t)(N * 128) >> 4;          // descriptor units per 128-byte depth block of B
         uint32_t cg = 0;                               // chunks issued so far
         bool ok = true;
+        if (p.prep_in != nullptr && mytiles > 0) mbar_wait(bar_prep, 0, abort_flag, p.status);
         for (int k = 0; k < mytiles && ok; ++k) {
             const int acc = k & 1;
             TR(1, k, 0);
@@ -959,7 +1043,7 @@ conv_tc_wide_kernel(const Params p)
         }
     } else if (warp < WPW + 1 + 4 * WSB) {
         // ---------------------------------------------------------------- build warps
-        const int sb = (warp - (WPW + 1)) >> 2;        // my set: the tile's chunks sb, sb + WSB, ...
+        const int sb = (warp - (WPW + 1)) >> 2;        // my set: every WSB-th chunk, counted across tiles
         const int q = warp & 3;
         const int row = q * 32 + lane;
         const uint32_t a_taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)ARING0;
@@ -988,7 +1072,9 @@ conv_tc_wide_kernel(const Params p)
             const int col0 = ow * p.sw - p.pw;         // input column of my window's first column
             const uint32_t src = bufaddr + (uint32_t)(16 + slot0 * p.rowbytes + col0 * p.unit);
             const uint32_t cg0 = (uint32_t)k * (uint32_t)nchunks;
-            for (int c = sb; c < nchunks; c += WSB) {
+            // chunks are dealt to the sets round-robin over the whole run of tiles, so that a tile of
+            // three chunks does not leave one set with two of them every time
+            for (int c = (int)(((uint32_t)sb + (uint32_t)WSB - cg0 % (uint32_t)WSB) % (uint32_t)WSB); c < nchunks; c += WSB) {
                 const uint32_t cg = cg0 + (uint32_t)c;
                 const int slot = (int)(cg % WNCH);
                 // the MMAs that read this slot WNCH chunks ago are complete
@@ -1060,6 +1146,7 @@ conv_tc_wide_kernel(const Params p)
             }
         };
         if (use_preload) {
+            if (p.prep_in != nullptr) mbar_wait(bar_prep, 0, abort_flag, p.status);     // the constants are in the image
             preload(0);
             preload(1);
             tc_wait_st();
@@ -1239,7 +1326,7 @@ cudaError_t launch_instance(const fused::Params& p, cudaStream_t st)
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         sms = 148;
     const int64_t tiles = (p.M + S::TILE - 1) / S::TILE;
-    const int grid = (int)(tiles < sms ? tiles : sms);
+    const int grid = p.prep_out ? 1 : (int)(tiles < sms ? tiles : sms);      // preparation: one CTA, no tiles
     // Programmatic stream serialization: the grid may be scheduled while the previous
     // kernel of the stream drains; the kernel itself waits (griddepcontrol.wait) before it
     // touches memory.
@@ -1373,9 +1460,35 @@ bool conv_tc_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t* W
     return ring_for(c.id, p) > 0;
 }
 
+template <class S> static size_t image_bytes_of() { return (size_t)S::B_BYTES + (size_t)S::N * 4 + 16; }
+
+// Bytes of the prepared weight image of a layer (see launch_conv_tc), 0 if no tensor-memory
+// kernel serves the layer's geometry.
+size_t conv_tc_image_bytes(const q4_conv_desc& d)
+{
+    if (!conv_tc_supported(d, nullptr, nullptr, 0, nullptr)) return 0;
+    const TcChoice c = choose_instance(d);
+    switch (c.id) {
+        case 0: return image_bytes_of<S_gray>();
+        case 1: return image_bytes_of<S_8_16>();
+        case 2: return image_bytes_of<S_16_32>();
+        case 3: return image_bytes_of<S_32_64>();
+        case 4: return image_bytes_of<S_16_32s1>();
+        default: break;
+    }
+    fused::Params p{};
+    size_t smem = 0;
+    if (!plan_wide(p, d, nullptr, nullptr, &smem)) return 0;
+    return (size_t)p.tcSplit * ((size_t)convtc::wide_layout(p.tcN, p.KS).off_tab + (size_t)p.tcN * 4 + 16);
+}
+
+// prep_out: only prepare the weights (B operand, per-column constants, fallback flag) into
+// that buffer of conv_tc_image_bytes(d) bytes; X and Y are not touched.  prep_in: run the layer
+// from such an image; Wt, colsum_w, bias and zb are not read.
 cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, const int32_t* colsum_w,
                            const int32_t* bias, const q4_conv_desc& d, int32_t za, int32_t zb,
-                           const RequantParams& rq, uint8_t* Y, cudaStream_t st)
+                           const RequantParams& rq, uint8_t* Y, cudaStream_t st, const uint8_t* prep_in,
+                           uint8_t* prep_out)
 {
     const TcChoice c = choose_instance(d);
     if (c.id < 0) {
@@ -1386,10 +1499,13 @@ cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, con
         p.zb_ch = p.mult_ch = p.shift_ch = nullptr;
         p.za = za; p.zb = zb; p.rq = rq;
         p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
+        p.prep_in = prep_in; p.prep_out = prep_out;
         p.status = device_status_ptr();
         if (!p.status) return cudaErrorUnknown;
-        if (p.M == 0) return cudaSuccess;
-        log_choice("q4_conv2d", "fused implicit GEMM on tcgen05, run-time geometry (C a multiple of 32)");
+        if (prep_out) p.M = 0;                         // no tiles: the CTAs prepare their shares and leave
+        else if (p.M == 0) return cudaSuccess;
+        log_choice(prep_out ? "q4_conv2d_prepare_weights" : "q4_conv2d",
+                   "fused implicit GEMM on tcgen05, run-time geometry (C a multiple of 32)");
         return launch_wide(p, smem, st);
     }
     fused::Params p{};
@@ -1399,10 +1515,13 @@ cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, con
     p.za = za; p.zb = zb; p.rq = rq;
     p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
     p.nbuf = ring_for(c.id, p);
+    p.prep_in = prep_in; p.prep_out = prep_out;
     p.status = device_status_ptr();
     if (!p.status) return cudaErrorUnknown;
-    if (p.M == 0) return cudaSuccess;
-    log_choice("q4_conv2d", "fused implicit GEMM on tcgen05 (A built in tensor memory)");
+    if (prep_out) p.M = 0;                             // no tiles: one CTA prepares the image and leaves
+    else if (p.M == 0) return cudaSuccess;
+    log_choice(prep_out ? "q4_conv2d_prepare_weights" : "q4_conv2d",
+               "fused implicit GEMM on tcgen05 (A built in tensor memory)");
     switch (c.id) {
         case 0: return launch_instance<S_gray, Q4_CTC_G0>(p, st);
         case 1: return launch_instance<S_8_16, Q4_CTC_G1>(p, st);

@@ -191,3 +191,49 @@ def test_validation_of_the_per_channel_entry_points(lib):
     assert c(CD(2, 8, 8, 16, 72, 3, 3, 1, 1, 1, 1), ldw=72) == 5            # unsupported: 72 output channels
     assert c(d, Y=fake + 4) == 5                                            # unsupported: Y not 8-byte aligned
     assert c(CD(0, 8, 8, 16, 32, 3, 3, 1, 1, 1, 1)) == 0
+
+
+def test_prepared_weight_entry_points_validate_without_a_device(lib):
+    vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_size_t
+    INVALID, ALIGN, RANGE, WORKSPACE = 1, 2, 3, 4
+    lib.q4_conv2d_weights_bytes.argtypes = [ctypes.POINTER(CD)]
+    lib.q4_conv2d_weights_bytes.restype = sz
+    lib.q4_conv2d_prepare_weights.argtypes = [vp, i64, vp, vp, ctypes.POINTER(CD), i32, i32, vp, sz, vp]
+    lib.q4_conv2d_prepared.argtypes = [vp, vp, sz, ctypes.POINTER(CD), i32, ctypes.POINTER(RQ), vp, vp]
+    lib.q4_status_string.restype = ctypes.c_char_p
+    UNSUPPORTED = next(c for c in range(1, 16) if b"unsupported" in lib.q4_status_string(c).lower()
+                       or b"not supported" in lib.q4_status_string(c).lower())
+    fake = 0x1000       # never dereferenced
+    c3 = CD(2, 32, 32, 16, 32, 3, 3, 1, 1, 1, 1)          # a layer class of the tensor-memory kernels
+    wide = CD(2, 16, 16, 128, 256, 3, 3, 1, 1, 1, 1)       # two CTAs' shares
+    odd = CD(2, 9, 11, 3, 6, 5, 5, 1, 1, 2, 2)             # no tensor-memory kernel
+    nb = lib.q4_conv2d_weights_bytes(ctypes.byref(c3))
+    # B: 64 columns x 7 depth steps of 32 bytes in two 128-byte blocks, 64 constants, 16 bytes of flag
+    assert nb == 2 * 64 * 128 + 64 * 4 + 16
+    nw = lib.q4_conv2d_weights_bytes(ctypes.byref(wide))
+    assert nw == 2 * (10 * 128 * 128 + 128 * 4 + 16)       # 36 + 1 steps -> ten blocks of 128 columns
+    assert lib.q4_conv2d_weights_bytes(ctypes.byref(odd)) == 0
+    assert lib.q4_conv2d_weights_bytes(None) == 0
+    rq = RQ(1 << 30, 8, 0, 0, 15)
+    prep = lambda d, **kw: lib.q4_conv2d_prepare_weights(kw.get("Wt", fake), kw.get("ldw", 72), None, None, ctypes.byref(d),
+                                                         kw.get("za", 0), kw.get("zb", 0), kw.get("out", fake),
+                                                         kw.get("nbytes", nb), None)
+    assert prep(c3, Wt=None) == INVALID
+    assert prep(c3, out=None) == INVALID
+    assert prep(c3, ldw=71) == INVALID
+    assert prep(c3, zb=16) == RANGE
+    assert prep(c3, za=-1) == RANGE
+    assert prep(c3, nbytes=nb - 1) == WORKSPACE
+    assert prep(c3, out=fake + 8) == ALIGN
+    assert prep(odd, ldw=38) == UNSUPPORTED
+    run = lambda d, **kw: lib.q4_conv2d_prepared(kw.get("X", fake), kw.get("img", fake), kw.get("nbytes", nb), ctypes.byref(d),
+                                                 kw.get("za", 0), ctypes.byref(kw.get("rq", rq)), kw.get("Y", fake), None)
+    assert run(c3, img=None) == INVALID
+    assert run(c3, X=None) == INVALID
+    assert run(c3, Y=None) == INVALID
+    assert run(c3, nbytes=nb - 16) == WORKSPACE
+    assert run(c3, img=fake + 4) == ALIGN
+    assert run(c3, rq=RQ(1 << 29, 8, 0, 0, 15)) == RANGE
+    assert run(c3, Y=fake + 8) == UNSUPPORTED               # output rows not 16-byte aligned: use q4_conv2d
+    assert run(odd) == UNSUPPORTED
+    assert run(CD(0, 32, 32, 16, 32, 3, 3, 1, 1, 1, 1)) == 0    # empty batch: a no-op

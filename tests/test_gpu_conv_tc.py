@@ -24,6 +24,27 @@ def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
+def check_prepared_weights(q4, Xd, Wt, dq, za, zb, rq, bias, colsum, want):
+    """The same layer from a weight image prepared ahead of time: one launch, the same bytes,
+    nothing written past the image."""
+    import torch
+    nb = q4.q4_conv2d_weights_bytes(dq)
+    assert nb > 0 and nb % 16 == 0
+    img = torch.full((nb + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+    n0 = q4.q4_launch_count()
+    q4.q4_conv2d_prepare_weights(dev(Wt), dq, za, zb, img[:nb], None if bias is None else dev(bias), colsum)
+    assert q4.q4_launch_count() - n0 == 1
+    Y = torch.full((dq.M + 64, dq.OC // 2), 0x3C, dtype=torch.uint8, device="cuda")
+    n0 = q4.q4_launch_count()
+    q4.q4_conv2d_prepared(Xd, img[:nb], dq, za, q4.Requant(*rq), Y[:dq.M])
+    assert q4.q4_launch_count() - n0 == 1
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    out = Y.cpu().numpy()
+    assert (out[:dq.M] == want).all()
+    assert (out[dq.M:] == 0x3C).all()
+    assert (img[nb:].cpu().numpy() == 0xA5).all()
+
+
 TC_LAYERS = [  # N, H, W, C, OC, stride, pad_h, shift
     (2, 8, 8, 1, 8, 1, 1, 5),          # gray first layer, less than one tile
     (5, 48, 48, 1, 8, 1, 1, 5),        # ... tiles that end inside an image
@@ -82,6 +103,7 @@ def test_tensor_memory_conv_kernel_matches_oracle(q4, g, given_sums):
         assert (Y2.cpu().numpy() == want).all()
     finally:
         q4.q4_set_variant(0)
+    check_prepared_weights(q4, Xd[:X.size], Wt, dq, za, zb, rq, bias, colsum, want)
 
 
 WIDE_LAYERS = [  # N, H, W, C, OC, KH, KW, sh, sw, ph, pw, shift
@@ -132,6 +154,10 @@ def test_run_time_geometry_kernel_for_wide_layers(q4, g, given_sums):
     assert (out[dq.M:] == 0xA5).all()
     if (C, OC) in ((32, 32), (32, 64), (64, 64), (64, 128), (128, 256), (64, 32), (32, 96)):
         assert launches == 1             # the tensor-memory kernel took it: no unrolled matrix
+    if launches == 1:
+        check_prepared_weights(q4, dev(X), Wt, dq, za, zb, rq, bias, colsum, want)
+    else:
+        assert q4.q4_conv2d_weights_bytes(dq) == 0       # no tensor-memory kernel, no image
 
 
 @pytest.mark.parametrize("g", [(3, 48, 48, 8, 16, 3, 3, 2, 2, 1, 1), (2, 8, 8, 1, 8, 3, 3, 1, 1, 1, 1),
@@ -174,6 +200,7 @@ def test_large_per_channel_constants(q4, g, big):
     assert q4.q4_launch_count() - n0 == 1
     assert q4.q4_last_device_status() == q4.Q4_OK
     assert (Y.cpu().numpy() == want).all()
+    check_prepared_weights(q4, dev(X), Wt, dq, za, zb, rq, bias, None, want)     # both routes from an image too
 
 
 def test_which_layers_take_the_tensor_memory_kernel(q4, capfd):
