@@ -316,6 +316,34 @@ def time_c4_chain(q4, wl, batch: int = 4096, reps: int = 20, net=None, hbm_peak:
     return out
 
 
+def time_wide_layers(q4, reps: int = 10):
+    """Layers wider than the paper's (3x3, stride 1, padding 1, batch 256): one launch of the
+    run-time-geometry tensor-memory kernel, through q4_conv2d and from weights prepared once."""
+    import torch
+    out = {}
+    for (H, C, OC) in ((32, 64, 64), (32, 64, 128), (16, 128, 256)):
+        d = q4.ConvDesc(256, H, H, C, OC, 3, 3, 1, 1, 1, 1)
+        X = torch.randint(0, 256, (256 * H * H * C // 2,), dtype=torch.uint8, device="cuda")
+        Wt = torch.randint(0, 256, (OC, 9 * C // 2), dtype=torch.uint8, device="cuda")
+        Y = torch.empty((d.M, OC // 2), dtype=torch.uint8, device="cuda")
+        ws = torch.empty(q4.q4_conv2d_workspace_bytes(d), dtype=torch.uint8, device="cuda")
+        rq = q4.Requant((1 << 30) + 5, 8, 0, 0, 15)
+        ops = 2.0 * d.M * d.K * OC
+        n0 = q4.q4_launch_count()
+        q4.q4_conv2d(X, Wt, d, 7, 8, rq, Y, ws)
+        launches = q4.q4_launch_count() - n0
+        ms = graph_time_ms([lambda: q4.q4_conv2d(X, Wt, d, 7, 8, rq, Y, ws)], reps)
+        r = {"launches": launches, "ms": ms, "tops": ops / (ms * 1e-3) / 1e12}
+        nimg = q4.q4_conv2d_weights_bytes(d)
+        if nimg:
+            img = torch.empty(nimg, dtype=torch.uint8, device="cuda")
+            q4.q4_conv2d_prepare_weights(Wt, d, 7, 8, img)
+            ms = graph_time_ms([lambda: q4.q4_conv2d_prepared(X, img, d, 7, rq, Y)], reps)
+            r.update({"ms_weights_prepared": ms, "tops_weights_prepared": ops / (ms * 1e-3) / 1e12})
+        out[f"{C}to{OC}_{H}x{H}_batch256"] = r
+    return out
+
+
 def time_im2col(q4, wl, hbm_peak: float, batch: int = 4096, reps: int = 10):
     """Device time of q4_im2col (the explicit unrolling, with row sums) on the c3 layer shape at a
     batch whose matrix (about 0.34 GB at 4096) exceeds L2, so the stores go to HBM.  Algorithmic
@@ -675,6 +703,11 @@ def run_ours(args):
     c4_detail = time_c4_chain(q4, wl, hbm_peak=peaks["hbm"]) if extra else None
     c3_256 = time_c4_chain(q4, wl, net=wl.c3(), hbm_peak=peaks["hbm"]) if extra else None
     c3_4096 = time_c4_chain(q4, wl, net=wl.c3(batch=4096), hbm_peak=peaks["hbm"]) if extra else None
+    # the same with the weight-side work done once (q4_conv2d_prepare_weights / q4_conv2d_prepared)
+    c4_prep = time_c4_chain(q4, wl, hbm_peak=peaks["hbm"], prepared=True) if extra else None
+    wide_detail = time_wide_layers(q4) if extra else None
+    c3_256_prep = time_c4_chain(q4, wl, net=wl.c3(), hbm_peak=peaks["hbm"], prepared=True) if extra else None
+    c3_4096_prep = time_c4_chain(q4, wl, net=wl.c3(batch=4096), hbm_peak=peaks["hbm"], prepared=True) if extra else None
     t2_detail = None
     if extra:
         # the layer list of the paper's Table II (six convolutions on 25 x 33 gray images) with
@@ -749,6 +782,10 @@ def run_ours(args):
                          "matrix is never written)",
             "c3_batch256": conv_case(c3_256), "c3_batch4096": conv_case(c3_4096),
             "c4_chain_batch4096": conv_case(c4_detail),
+            "weights_prepared_once": {"c3_batch256": conv_case(c3_256_prep), "c3_batch4096": conv_case(c3_4096_prep),
+                                      "c4_chain_batch4096": conv_case(c4_prep),
+                                      "what": "q4_conv2d_prepared: the layers run from weight images prepared "
+                                              "once per layer (Section II-B), not rebuilt inside every launch"},
             "timing": "replayed from CUDA graphs, median of 5 (see detail for per-layer and eager figures)"},
         "cpu_baseline": cpu_baseline,
         "detail": {
@@ -762,6 +799,9 @@ def run_ours(args):
             "c2_sweep_and_c5": sweep,
             "c4_chain_batch4096": c4_detail,
             "c3_batch256": c3_256, "c3_batch4096": c3_4096,
+            "c4_chain_batch4096_weights_prepared": c4_prep,
+            "wide_layers": wide_detail,
+            "c3_batch256_weights_prepared": c3_256_prep, "c3_batch4096_weights_prepared": c3_4096_prep,
             "paper_table2_layers_batch4096": t2_detail,
             "q4_im2col": im2col_detail,
             "float_boundary": float_detail,
