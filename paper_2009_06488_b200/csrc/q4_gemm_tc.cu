@@ -35,7 +35,6 @@ namespace q4 {
 constexpr int TM = 128;            // rows of A per tile (UMMA M)
 constexpr int PROW = 64;           // packed bytes per row per stage
 constexpr int UROW = 128;          // unpacked bytes per row per stage (one swizzle row)
-constexpr int SLAB = 128;          // depth values per stage
 constexpr int UW = 8;              // unpack warps
 constexpr int UT = UW * 32;        // unpack threads
 constexpr int NTHREADS = (2 + UW + 4) * 32;
@@ -180,9 +179,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t ua = sbase + C::OFF_U + st * C::USTAGE;
                     const uint64_t adesc = make_kmajor_sw128_desc(ua);
                     const uint64_t bdesc = make_kmajor_sw128_desc(ua + TM * UROW);
-                    const int rem = g.K - s * SLAB;
-                    const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
-                    for (int i = 0; i < ksteps; ++i)
+                    // all four 32-deep steps, always: past the end of a ragged depth the TMA
+                    // loads filled both operands with zeros
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
                         tc_mma_i8(d_tmem, adesc + (uint64_t)(2 * i), bdesc + (uint64_t)(2 * i), idesc,
                                   (s > 0 || i > 0) ? 1u : 0u);
                     tc_commit(bar_empty_u(st));
@@ -201,19 +201,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             for (int s = 0; s < p.nslab; ++s, ++it) {
                 const int st = it % C::STAGES;
                 const uint32_t ph = (it / C::STAGES) & 1u;
-                const int rem = g.K - s * SLAB;
-                const int ksteps = rem >= SLAB ? 4 : (rem + 31) / 32;
                 mbar_wait(bar_full_p(st), ph, abort_flag, g.status);
-                mbar_wait(bar_empty_u(st), ph ^ 1u, abort_flag, g.status);
-                tc_fence_after();
                 const uint32_t ps = sbase + C::OFF_P + st * C::PSTAGE;
                 const uint32_t us = sbase + C::OFF_U + st * C::USTAGE;
+                // all loads first (their latencies overlap), then the wait for the unpacked slot
+                uint4 wv[C::NT];
+#pragma unroll
+                for (int j = 0; j < C::NT; ++j) {
+                    const int id = ut + j * UT;
+                    if (id < C::ROWS * 4) wv[j] = lds128(ps + (id >> 2) * PROW + (id & 3) * 16);
+                }
+                mbar_wait(bar_empty_u(st), ph ^ 1u, abort_flag, g.status);
+                tc_fence_after();
 #pragma unroll
                 for (int j = 0; j < C::NT; ++j) {
                     const int id = ut + j * UT;
                     const int r = id >> 2, c = id & 3;
-                    if (id < C::ROWS * 4 && c < ksteps) {
-                        const uint4 w = lds128(ps + r * PROW + c * 16);
+                    if (id < C::ROWS * 4) {
+                        const uint4 w = wv[j];
                         uint4 lo, hi;
                         lo.x = w.x & 0x0F0F0F0Fu; hi.x = (w.x >> 4) & 0x0F0F0F0Fu;
                         lo.y = w.y & 0x0F0F0F0Fu; hi.y = (w.y >> 4) & 0x0F0F0F0Fu;
