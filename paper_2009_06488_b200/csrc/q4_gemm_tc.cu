@@ -40,22 +40,30 @@ constexpr int UT = UW * 32;        // unpack threads
 constexpr int NTHREADS = (2 + UW + 4) * 32;
 
 template <int BN> struct Cfg {
+    // The unpack warps work as two groups of four that take the stages in turn, so that one
+    // group's loads, fences and hand-over hide behind the other's work (256 columns: one group,
+    // shared memory has no room for a second set of partial sums).
+    static constexpr int UG = BN == 256 ? 1 : 2;
+    static constexpr int GT = UT / UG;                         // threads per group
     static constexpr int ROWS = TM + BN;
     static constexpr int PSTAGE = ROWS * PROW;
     static constexpr int USTAGE = ROWS * UROW;
     static constexpr int STAGES = (BN == 256) ? 3 : 4;
-    static constexpr int NT = (ROWS * 4 + UT - 1) / UT;        // unpack tasks per thread
+    static constexpr int NT = (ROWS * 4 + GT - 1) / GT;        // unpack tasks (16-byte packed chunks) per thread and stage
+    static constexpr int NBATCH = (NT + 5) / 6;                // ... taken in batches of at most six (registers)
+    static constexpr int NTB = (NT + NBATCH - 1) / NBATCH;
     static constexpr int TMEM_COLS = (2 * BN < 32) ? 32 : 2 * BN;
     // layout: [U stages][P stages][sums 2*ROWS int32][colterm BN int32][barriers][misc]
     static constexpr int OFF_U = 0;
     static constexpr int OFF_P = OFF_U + STAGES * USTAGE;
     static constexpr int OFF_SUMS = OFF_P + STAGES * PSTAGE;
-    static constexpr int OFF_COLTERM = OFF_SUMS + 2 * ROWS * 4;
+    static constexpr int OFF_COLTERM = OFF_SUMS + 2 * UG * ROWS * 4;   // sums: int32 [2 accumulators][UG groups][ROWS]
     static constexpr int OFF_PC = OFF_COLTERM + BN * 4;        // per-channel: int32 [4][BN]
     static constexpr int OFF_BAR = OFF_PC + 4 * BN * 4;
     static constexpr int NBAR = 4 * STAGES + 6;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM = OFF_MISC + 16 + 1024;          // + slack to align the base
+    static_assert(SMEM <= 227 * 1024, "shared memory budget");
 };
 
 // Instruction descriptor: D = s32, A = B = unsigned 8-bit, both K-major, M = 128, N = BN.
@@ -81,7 +89,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const uint32_t sbase = smem_u32(smem);
 
-    const uint32_t sums_s = sbase + C::OFF_SUMS;          // int32 [2][ROWS]
+    const uint32_t sums_s = sbase + C::OFF_SUMS;          // int32 [2][UG][ROWS]
     const uint32_t colterm_s = sbase + C::OFF_COLTERM;    // int32 [BN]
     const uint32_t pc_s = sbase + C::OFF_PC;              // int32 [4][BN]: zero point, multiplier, rounding, shift
     const uint32_t bar0 = sbase + C::OFF_BAR;
@@ -104,8 +112,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (threadIdx.x == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(bar_full_p(s), 1);
-            mbar_init(bar_empty_p(s), UW);   // one arrive per unpack warp
-            mbar_init(bar_full_u(s), UW);
+            mbar_init(bar_empty_p(s), UW / C::UG);   // one arrive per warp of the group that took the stage
+            mbar_init(bar_full_u(s), UW / C::UG);
             mbar_init(bar_empty_u(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -192,54 +200,66 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
     } else if (warp < 2 + UW) {
         // ------------------------------------------------------------ unpack warps
-        const int ut = threadIdx.x - 64;
-        uint32_t it = 0, lt = 0;
+        constexpr int UG = C::UG, GT = C::GT;
+        const int grp = (warp - 2) / (UW / UG);          // takes the stages with it % UG == grp
+        const int gt = threadIdx.x - 64 - grp * GT;      // 0 .. GT-1 inside the group
+        uint32_t it = (uint32_t)grp, lt = 0;
         for (int tile = blockIdx.x; tile < ntiles && !lds32(abort_flag); tile += gridDim.x, ++lt) {
             int psum[C::NT];
 #pragma unroll
             for (int j = 0; j < C::NT; ++j) psum[j] = 0;
-            for (int s = 0; s < p.nslab; ++s, ++it) {
+            // stages are numbered across tiles: stage s of my lt-th tile is lt * nslab + s
+            const uint32_t it_end = (lt + 1) * (uint32_t)p.nslab;
+            for (; it < it_end; it += UG) {
                 const int st = it % C::STAGES;
                 const uint32_t ph = (it / C::STAGES) & 1u;
                 mbar_wait(bar_full_p(st), ph, abort_flag, g.status);
                 const uint32_t ps = sbase + C::OFF_P + st * C::PSTAGE;
                 const uint32_t us = sbase + C::OFF_U + st * C::USTAGE;
-                // all loads first (their latencies overlap), then the wait for the unpacked slot
-                uint4 wv[C::NT];
 #pragma unroll
-                for (int j = 0; j < C::NT; ++j) {
-                    const int id = ut + j * UT;
-                    if (id < C::ROWS * 4) wv[j] = lds128(ps + (id >> 2) * PROW + (id & 3) * 16);
-                }
-                mbar_wait(bar_empty_u(st), ph ^ 1u, abort_flag, g.status);
-                tc_fence_after();
+                for (int b = 0; b < C::NBATCH; ++b) {
+                    // a batch's loads first (their latencies overlap), then -- before the first
+                    // store -- the wait for the unpacked slot
+                    uint4 wv[C::NTB];
 #pragma unroll
-                for (int j = 0; j < C::NT; ++j) {
-                    const int id = ut + j * UT;
-                    const int r = id >> 2, c = id & 3;
-                    if (id < C::ROWS * 4) {
-                        const uint4 w = wv[j];
-                        uint4 lo, hi;
-                        lo.x = w.x & 0x0F0F0F0Fu; hi.x = (w.x >> 4) & 0x0F0F0F0Fu;
-                        lo.y = w.y & 0x0F0F0F0Fu; hi.y = (w.y >> 4) & 0x0F0F0F0Fu;
-                        lo.z = w.z & 0x0F0F0F0Fu; hi.z = (w.z >> 4) & 0x0F0F0F0Fu;
-                        lo.w = w.w & 0x0F0F0F0Fu; hi.w = (w.w >> 4) & 0x0F0F0F0Fu;
-                        const uint32_t row = us + r * UROW;
-                        const int sw = r & 7;
-                        sts128(row + (((2 * c) ^ sw) << 4), lo);
-                        sts128(row + (((2 * c + 1) ^ sw) << 4), hi);
-                        if (need_sums) {
-                            int t = psum[j];
-                            t = dp4a_u8(lo.x + hi.x, 0x01010101u, t);
-                            t = dp4a_u8(lo.y + hi.y, 0x01010101u, t);
-                            t = dp4a_u8(lo.z + hi.z, 0x01010101u, t);
-                            t = dp4a_u8(lo.w + hi.w, 0x01010101u, t);
-                            psum[j] = t;
+                    for (int jj = 0; jj < C::NTB; ++jj) {
+                        const int j = b * C::NTB + jj;
+                        const int id = gt + j * GT;
+                        if (j < C::NT && id < C::ROWS * 4) wv[jj] = lds128(ps + (id >> 2) * PROW + (id & 3) * 16);
+                    }
+                    if (b == 0) {
+                        mbar_wait(bar_empty_u(st), ph ^ 1u, abort_flag, g.status);
+                        tc_fence_after();
+                    }
+#pragma unroll
+                    for (int jj = 0; jj < C::NTB; ++jj) {
+                        const int j = b * C::NTB + jj;
+                        const int id = gt + j * GT;
+                        const int r = id >> 2, c = id & 3;
+                        if (j < C::NT && id < C::ROWS * 4) {
+                            const uint4 w = wv[jj];
+                            uint4 lo, hi;
+                            lo.x = w.x & 0x0F0F0F0Fu; hi.x = (w.x >> 4) & 0x0F0F0F0Fu;
+                            lo.y = w.y & 0x0F0F0F0Fu; hi.y = (w.y >> 4) & 0x0F0F0F0Fu;
+                            lo.z = w.z & 0x0F0F0F0Fu; hi.z = (w.z >> 4) & 0x0F0F0F0Fu;
+                            lo.w = w.w & 0x0F0F0F0Fu; hi.w = (w.w >> 4) & 0x0F0F0F0Fu;
+                            const uint32_t row = us + r * UROW;
+                            const int sw = r & 7;
+                            sts128(row + (((2 * c) ^ sw) << 4), lo);
+                            sts128(row + (((2 * c + 1) ^ sw) << 4), hi);
+                            if (need_sums) {
+                                int t = psum[j];
+                                t = dp4a_u8(lo.x + hi.x, 0x01010101u, t);
+                                t = dp4a_u8(lo.y + hi.y, 0x01010101u, t);
+                                t = dp4a_u8(lo.z + hi.z, 0x01010101u, t);
+                                t = dp4a_u8(lo.w + hi.w, 0x01010101u, t);
+                                psum[j] = t;
+                            }
                         }
                     }
                 }
                 // every lane publishes its own writes to the async proxy; one lane per warp
-                // then arrives (256 arrives on one barrier word serialise badly)
+                // then arrives (many arrives on one barrier word serialise badly)
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) {
@@ -257,9 +277,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     int t = psum[j];
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 1);
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
-                    const int id = ut + j * UT;
+                    const int id = gt + j * GT;
                     if (id < C::ROWS * 4 && (id & 3) == 0)
-                        sts32(sums_s + 4 * (acc * C::ROWS + (id >> 2)), t);
+                        sts32(sums_s + 4 * ((acc * UG + grp) * C::ROWS + (id >> 2)), t);
                 }
                 mbar_arrive(bar_sums(acc));
             }
@@ -282,7 +302,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const int n = n0 + j;
                 int cb = 0, bias = 0, zbn = pc ? 0 : g.zb;
                 if (n < g.N) {
-                    cb = need_cb ? lds32(sums_s + 4 * (acc * C::ROWS + TM + j)) : g.colsum_b[n];
+                    if (need_cb) {
+#pragma unroll
+                        for (int gi = 0; gi < C::UG; ++gi) cb += lds32(sums_s + 4 * ((acc * C::UG + gi) * C::ROWS + TM + j));
+                    } else {
+                        cb = g.colsum_b[n];
+                    }
                     if (REQUANT && g.bias) bias = g.bias[n];
                     if (pc && g.zb_ch) zbn = g.zb_ch[n];
                 }
@@ -299,7 +324,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 }
             }
             int ra = 0;
-            if (need_ra) ra = lds32(sums_s + 4 * (acc * C::ROWS + row));
+            if (need_ra) {
+#pragma unroll
+                for (int gi = 0; gi < C::UG; ++gi) ra += lds32(sums_s + 4 * ((acc * C::UG + gi) * C::ROWS + row));
+            }
             else if (m < g.M) ra = g.rowsum_a[m];
             const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
             asm volatile("bar.sync 1, 128;" ::: "memory");
