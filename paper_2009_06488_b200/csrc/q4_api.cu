@@ -536,8 +536,13 @@ q4_status q4_conv2d_channels(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
     const void* words[] = {colsum_w, bias, zb, mult, shift};
     for (const void* w : words)
         if ((uintptr_t)w % 4) return Q4_ERR_ALIGNMENT;
-    if (!conv_fused_supported(*d, X, Wt, ldw, Y, true)) return Q4_ERR_UNSUPPORTED;
     const RequantParams rqp{1 << 30, 2, zo, clamp_lo, clamp_hi};     // multiplier and shift come per channel
+    // the tensor-memory kernels where they have an instance for the layer (variant 4 skips them)
+    const int v = variant_kind();
+    if ((v == 0 || v == 2) && conv_tc_supported(*d, X, Wt, ldw, Y))
+        return launch_conv_tc(X, Wt, ldw, colsum_w, bias, *d, za, 0, rqp, Y, static_cast<cudaStream_t>(stream),
+                              nullptr, nullptr, zb, mult, shift) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+    if (!conv_fused_supported(*d, X, Wt, ldw, Y, true)) return Q4_ERR_UNSUPPORTED;
     return launch_conv_fused(X, Wt, ldw, colsum_w, bias, *d, za, 0, rqp, Y, static_cast<cudaStream_t>(stream),
                              zb, mult, shift) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }

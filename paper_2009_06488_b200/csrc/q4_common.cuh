@@ -163,7 +163,9 @@ bool        conv_tc_supported(const q4_conv_desc& d, const uint8_t* X, const uin
 cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, const int32_t* colsum_w,
                            const int32_t* bias, const q4_conv_desc& d, int32_t za, int32_t zb,
                            const RequantParams& rq, uint8_t* Y, cudaStream_t st,
-                           const uint8_t* prep_in = nullptr, uint8_t* prep_out = nullptr);
+                           const uint8_t* prep_in = nullptr, uint8_t* prep_out = nullptr,
+                           const int32_t* zb_ch = nullptr, const int32_t* mult_ch = nullptr,
+                           const int32_t* shift_ch = nullptr);
 size_t      conv_tc_image_bytes(const q4_conv_desc& d);
 cudaError_t launch_im2col(const uint8_t* X, const q4_conv_desc& d, int32_t za, uint8_t* A,
                           int64_t lda, int32_t* rowsum_a, cudaStream_t st);

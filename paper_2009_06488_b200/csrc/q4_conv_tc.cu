@@ -98,7 +98,8 @@ constexpr int NBAR = 2 * NBMAX + 2 * GMAX + 2;      // (an even count keeps what
 template <class S> struct Layout {
     static constexpr int OFF_B = 0;
     static constexpr int OFF_CT = OFF_B + S::B_BYTES;         // int32 [N] per-column constants
-    static constexpr int OFF_GEO = OFF_CT + S::N * 4;         // int4 [NBMAX]
+    static constexpr int OFF_PC = OFF_CT + S::N * 4;          // int32 [3][N] per-column multiplier, rounding, shift
+    static constexpr int OFF_GEO = OFF_PC + 3 * S::N * 4;     // int4 [NBMAX]
     static constexpr int OFF_BAR = OFF_GEO + NBMAX * 16;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;       // tensor-memory base, abort flag
     static constexpr int OFF_BUF = OFF_MISC + 16;
@@ -321,7 +322,41 @@ __device__ __forceinline__ uint32_t requant8(const uint32_t* r, const RequantPar
     return o;
 }
 
-template <class S, int G>
+// The same with every column's own multiplier, rounding constant and shift (per output
+// channel), read from shared memory at pc_s + 4 * (array * n_cols + column): columns
+// col0 .. col0 + 7.  fast: every shift allows the 32-bit form (the arrays then hold
+// rnd = 2^(s-1) + ((zo - lo) << s) and s = shift - 1), else they hold the shifts themselves.
+__device__ __forceinline__ uint32_t requant8_channels(const uint32_t* r, const RequantParams& rq, uint32_t pc_s,
+                                                      int n_cols, int col0, bool fast, uint32_t hml2)
+{
+    const uint4 m0 = lds128(pc_s + 4 * col0), m1 = lds128(pc_s + 4 * (col0 + 4));
+    const uint4 s0 = lds128(pc_s + 4 * (2 * n_cols + col0)), s1 = lds128(pc_s + 4 * (2 * n_cols + col0 + 4));
+    const int mu[8] = {(int)m0.x, (int)m0.y, (int)m0.z, (int)m0.w, (int)m1.x, (int)m1.y, (int)m1.z, (int)m1.w};
+    const int sh[8] = {(int)s0.x, (int)s0.y, (int)s0.z, (int)s0.w, (int)s1.x, (int)s1.y, (int)s1.z, (int)s1.w};
+    if (fast) {
+        const uint4 r0 = lds128(pc_s + 4 * (n_cols + col0)), r1 = lds128(pc_s + 4 * (n_cols + col0 + 4));
+        const int rn[8] = {(int)r0.x, (int)r0.y, (int)r0.z, (int)r0.w, (int)r1.x, (int)r1.y, (int)r1.z, (int)r1.w};
+        uint32_t c[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int q0 = fused::mulhi_add((int)r[2 * i], mu[2 * i], rn[2 * i]) >> sh[2 * i];
+            const int q1 = fused::mulhi_add((int)r[2 * i + 1], mu[2 * i + 1], rn[2 * i + 1]) >> sh[2 * i + 1];
+            c[i] = __vimin_s16x2_relu(pack_sat16(q1, q0), hml2);
+        }
+        return fused::mad_u32(c[3], 1u << 12, fused::mad_u32(c[2], 1u << 8, fused::mad_u32(c[1], 1u << 4, c[0])));
+    }
+    uint32_t o = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        const RequantParams one{mu[e], sh[e], rq.zo, rq.lo, rq.hi};
+        o |= (requant_wide((int)r[e], one) - (uint32_t)rq.lo) << (4 * ch8(e));
+    }
+    return o;
+}
+
+// PC: per-channel weight zero points, multipliers and shifts (an instance of its own, so that
+// the per-tensor form keeps its registers).
+template <class S, int G, bool PC>
 __global__ void __launch_bounds__((PWN + 1 + 4 * G) * 32, 1)
 conv_tc_kernel(const Params p)
 {
@@ -344,6 +379,10 @@ conv_tc_kernel(const Params p)
     const int NB = p.nbuf;
     const uint32_t tmem_slot = sbase + L::OFF_MISC, abort_flag = sbase + L::OFF_MISC + 4;
     const uint32_t preload_flag = sbase + L::OFF_MISC + 8;
+    const uint32_t pcslow_flag = sbase + L::OFF_MISC + 12;        // per-channel: some shift needs the 64-bit form
+    const uint32_t pc_s = sbase + L::OFF_PC;
+    int32_t* pcv = reinterpret_cast<int32_t*>(smem + L::OFF_PC);
+    constexpr bool pc = PC;
     uint8_t* buf0 = smem + L::OFF_BUF;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -361,6 +400,7 @@ conv_tc_kernel(const Params p)
         mbar_init(bar_prep, 1);
         sts32(abort_flag, 0);
         sts32(preload_flag, 0);
+        sts32(pcslow_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == PWN) {
@@ -449,6 +489,7 @@ conv_tc_kernel(const Params p)
             locate(idx, n, wd, px, oc, kh, i);
             uint32_t lo = 0, hi = 0;
             int raw = 0;
+            const int zbo = pc ? (p.zb_ch ? __ldg(p.zb_ch + oc) : 0) : p.zb;      // this channel's weight zero point
             if (wd < S::NW) {
                 if constexpr (S::NIB) {
 #pragma unroll
@@ -458,7 +499,7 @@ conv_tc_kernel(const Params p)
                         if (kw >= 0 && kw < S::KW && j < S::COLS) {
                             const int nib = (int)fused::weight_nibble(p, oc, kh * S::KW + kw);
                             raw += nib;
-                            const uint32_t byte = (uint32_t)(nib - p.zb) & 0xFFu;
+                            const uint32_t byte = (uint32_t)(nib - zbo) & 0xFFu;
                             if (e & 1) hi |= byte << (8 * (e >> 1)); else lo |= byte << (8 * (e >> 1));
                         }
                     }
@@ -467,8 +508,8 @@ conv_tc_kernel(const Params p)
                     const int kw = j - px * S::SW;
                     if (kw >= 0 && kw < S::KW) {
                         raw = nibble_sum(wv[it]);
-                        lo = fused::sub_zb(wv[it] & 0x0F0F0F0Fu, (uint32_t)p.zb);
-                        hi = fused::sub_zb((wv[it] >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                        lo = fused::sub_zb(wv[it] & 0x0F0F0F0Fu, (uint32_t)zbo);
+                        hi = fused::sub_zb((wv[it] >> 4) & 0x0F0F0F0Fu, (uint32_t)zbo);
                     }
                 }
             }
@@ -485,8 +526,13 @@ conv_tc_kernel(const Params p)
         int cterm = 0;
         if (wt < OC) {
             const int cs = p.colsum_w ? p.colsum_w[wt] : colterm[wt];
-            cterm = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
+            const int zbo = pc ? (p.zb_ch ? p.zb_ch[wt] : 0) : p.zb;
+            cterm = (int)((uint32_t)(p.K * p.za * zbo) - (uint32_t)(p.za * cs) +
                           (uint32_t)(p.bias ? p.bias[wt] : 0));
+            if (pc) {
+                const int sh = p.shift_ch[wt];
+                if (sh < 2 || sh > 27) sts32(pcslow_flag, 1);
+            }
             int d0 = cterm % 255;
             if (d0 > 127) d0 -= 255;
             if (d0 < -127) d0 += 255;
@@ -521,9 +567,23 @@ conv_tc_kernel(const Params p)
                 }
                 dw[i] = word;
             }
+            // per channel: multiplier, rounding constant, shift of every column of the channel
+            int pmul = 0, prnd = 0, psh = 0;
+            if (pc) {
+                const bool pfast = lds32(pcslow_flag) == 0;
+                const int sh = p.shift_ch[wt];
+                pmul = p.mult_ch[wt];
+                psh = pfast ? sh - 1 : sh;
+                prnd = pfast ? (1 << (psh - 1)) + (p.rq.zo - p.rq.lo) * (1 << psh) : 0;
+            }
             for (int px = 0; px < P; ++px) {
                 const int n = px * OC + pos;
                 colterm[n] = cterm;
+                if (pc) {
+                    pcv[n] = pmul;
+                    pcv[N + n] = prnd;
+                    pcv[2 * N + n] = psh;
+                }
 #pragma unroll
                 for (int i = 0; i < S::SPARE; ++i) {
                     const int kbyte = 8 * (S::NW + i);
@@ -594,6 +654,7 @@ conv_tc_kernel(const Params p)
         const int rnd = fast ? (1 << (sh1 - 1)) + (p.rq.zo - p.rq.lo) * (1 << sh1) : 0;
         const uint32_t hml2 = (uint32_t)(p.rq.hi - p.rq.lo) * 0x00010001u;
         const uint32_t lofill = (uint32_t)p.rq.lo * 0x11111111u;
+        const bool pc_fast = pc && lds32(pcslow_flag) == 0;
         const uint32_t mstep = gridDim.x * (uint32_t)(S::TILE * G);
         uint32_t mbase = (blockIdx.x + (uint32_t)g * gridDim.x) * (uint32_t)S::TILE;
         int kb = g;                                    // k % NB (G <= NB)
@@ -717,8 +778,9 @@ conv_tc_kernel(const Params p)
                     uint32_t o[4];
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        o[j] = (fast ? requant8<true>(r[c] + 8 * j, p.rq, sh1, rnd, hml2)
-                                     : requant8<false>(r[c] + 8 * j, p.rq, sh1, rnd, hml2)) + lofill;
+                        o[j] = (pc ? requant8_channels(r[c] + 8 * j, p.rq, pc_s, N, (cb + c) * 32 + 8 * j, pc_fast, hml2)
+                                : fast ? requant8<true>(r[c] + 8 * j, p.rq, sh1, rnd, hml2)
+                                       : requant8<false>(r[c] + 8 * j, p.rq, sh1, rnd, hml2)) + lofill;
                     if (mrow < M32)
                         *reinterpret_cast<uint4*>(dst + (cb + c) * 16) = make_uint4(o[0], o[1], o[2], o[3]);
                 }
@@ -772,7 +834,7 @@ constexpr int WNBAR = 2 * NBMAX + 2 * WNCH + 6;     // (even: what follows stays
 static_assert(WSB <= WNCH, "build sets may run at most one ring round ahead");
 
 struct WideLayout {
-    int off_tab, off_ct, off_geo, off_bar, off_misc, off_buf;     // after B (at 0)
+    int off_tab, off_ct, off_pc, off_geo, off_bar, off_misc, off_buf;     // after B (at 0)
 };
 __host__ __device__ inline WideLayout wide_layout(int N, int KS)
 {
@@ -780,7 +842,8 @@ __host__ __device__ inline WideLayout wide_layout(int N, int KS)
     l.off_tab = ((KS + 1 + 3) / 4) * N * 128;          // B holds KS + 1 steps; then int2 [KS]: offset of the
                                                        // step's 16 bytes, its window column
     l.off_ct = l.off_tab + (KS * 8 + 15) / 16 * 16;
-    l.off_geo = l.off_ct + N * 4;
+    l.off_pc = l.off_ct + N * 4;                      // int32 [3][N]: per-column multiplier, rounding, shift
+    l.off_geo = l.off_pc + 3 * N * 4;
     l.off_bar = l.off_geo + NBMAX * 16;
     l.off_misc = l.off_bar + WNBAR * 8;
     l.off_buf = l.off_misc + 16;
@@ -789,9 +852,12 @@ __host__ __device__ inline WideLayout wide_layout(int N, int KS)
 
 constexpr int WIDE_THREADS = (WPW + 1 + 4 * WSB + 4 * WSE) * 32;
 
+// PC: per-channel weight zero points, multipliers and shifts (see conv_tc_kernel).
+template <bool PC>
 __global__ void __launch_bounds__(WIDE_THREADS, 1)
 conv_tc_wide_kernel(const Params p)
 {
+    constexpr bool pc = PC;
     const int N = p.tcN, KS = p.KS, CW4 = p.C / 32;   // columns of my tile, depth steps, steps per tap
     // One more depth step carries the per-channel constants of Eq. 3 into the product: its A
     // bytes are the same for every row, 1 then thirty-one times 255, and its B bytes are the
@@ -819,6 +885,9 @@ conv_tc_wide_kernel(const Params p)
     const int NB = p.nbuf;
     const uint32_t tmem_slot = sbase + L.off_misc, abort_flag = sbase + L.off_misc + 4;
     const uint32_t preload_flag = sbase + L.off_misc + 8;
+    const uint32_t pcslow_flag = sbase + L.off_misc + 12;         // per-channel: some shift needs the 64-bit form
+    const uint32_t pc_s = sbase + L.off_pc;
+    int32_t* pcv = reinterpret_cast<int32_t*>(smem + L.off_pc);
     uint8_t* buf0 = smem + L.off_buf;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // my share of the output channels, and my pixel tiles
@@ -843,6 +912,7 @@ conv_tc_wide_kernel(const Params p)
         mbar_init(bar_prep, 1);
         sts32(abort_flag, 0);
         sts32(preload_flag, 0);
+        sts32(pcslow_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == WPW) {
@@ -920,14 +990,15 @@ conv_tc_wide_kernel(const Params p)
                 const int idx = base + u * NT;
                 if (idx >= tasks) break;
                 const int n = idx / KS, ks = idx - n * KS;
+                const int zbo = pc ? (p.zb_ch ? __ldg(p.zb_ch + oc0 + (n & ~7) + ch8(n & 7)) : 0) : p.zb;
                 const uint32_t wv[4] = {wq[u].x, wq[u].y, wq[u].z, wq[u].w};
                 uint32_t o[8];
                 int raw = 0;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
                     raw += nibble_sum(wv[j]);
-                    o[2 * j] = fused::sub_zb(wv[j] & 0x0F0F0F0Fu, (uint32_t)p.zb);
-                    o[2 * j + 1] = fused::sub_zb((wv[j] >> 4) & 0x0F0F0F0Fu, (uint32_t)p.zb);
+                    o[2 * j] = fused::sub_zb(wv[j] & 0x0F0F0F0Fu, (uint32_t)zbo);
+                    o[2 * j + 1] = fused::sub_zb((wv[j] >> 4) & 0x0F0F0F0Fu, (uint32_t)zbo);
                 }
                 uint8_t* row = smem + (ks >> 2) * (N * 128) + n * 128;
                 const int c = 2 * (ks & 3);
@@ -941,8 +1012,13 @@ conv_tc_wide_kernel(const Params p)
         if (wt < N) {
             const int oc = oc0 + (wt & ~7) + ch8(wt & 7);
             const int cs = p.colsum_w ? p.colsum_w[oc] : colterm[wt];
-            cterm = (int)((uint32_t)(p.K * p.za * p.zb) - (uint32_t)(p.za * cs) +
+            const int zbo = pc ? (p.zb_ch ? p.zb_ch[oc] : 0) : p.zb;
+            cterm = (int)((uint32_t)(p.K * p.za * zbo) - (uint32_t)(p.za * cs) +
                           (uint32_t)(p.bias ? p.bias[oc] : 0));
+            if (pc) {
+                const int sh = p.shift_ch[oc];
+                if (sh < 2 || sh > 27) sts32(pcslow_flag, 1);
+            }
             // digits: cterm = d0 + 255 * q, d0 in -127..127, q spread over thirty-one bytes
             int d0 = cterm % 255;
             if (d0 > 127) d0 -= 255;
@@ -954,6 +1030,16 @@ conv_tc_wide_kernel(const Params p)
         use_preload = lds32(preload_flag) != 0;
         if (wt < N) {
             colterm[wt] = cterm;
+            if (pc) {
+                // this column's multiplier, rounding constant and shift
+                const int oc = oc0 + (wt & ~7) + ch8(wt & 7);
+                const bool pfast = lds32(pcslow_flag) == 0;
+                const int sh = p.shift_ch[oc];
+                const int psh = pfast ? sh - 1 : sh;
+                pcv[wt] = p.mult_ch[oc];
+                pcv[N + wt] = pfast ? (1 << (psh - 1)) + (p.rq.zo - p.rq.lo) * (1 << psh) : 0;
+                pcv[2 * N + wt] = psh;
+            }
             int d0 = cterm % 255;
             if (d0 > 127) d0 -= 255;
             if (d0 < -127) d0 += 255;
@@ -1135,6 +1221,7 @@ conv_tc_wide_kernel(const Params p)
         const int rnd = fast ? (1 << (sh1 - 1)) + (p.rq.zo - p.rq.lo) * (1 << sh1) : 0;
         const uint32_t hml2 = (uint32_t)(p.rq.hi - p.rq.lo) * 0x00010001u;
         const uint32_t lofill = (uint32_t)p.rq.lo * 0x11111111u;
+        const bool pc_fast = pc && lds32(pcslow_flag) == 0;
         auto preload = [&](int acc) {                  // my chunks start from the channels' constants
             for (int ch = se; ch < N / 32; ch += WSE) {
 #pragma unroll
@@ -1181,8 +1268,9 @@ conv_tc_wide_kernel(const Params p)
                 uint32_t o[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    o[j] = (fast ? requant8<true>(r + 8 * j, p.rq, sh1, rnd, hml2)
-                                 : requant8<false>(r + 8 * j, p.rq, sh1, rnd, hml2)) + lofill;
+                    o[j] = (pc ? requant8_channels(r + 8 * j, p.rq, pc_s, N, ch * 32 + 8 * j, pc_fast, hml2)
+                            : fast ? requant8<true>(r + 8 * j, p.rq, sh1, rnd, hml2)
+                                   : requant8<false>(r + 8 * j, p.rq, sh1, rnd, hml2)) + lofill;
                 if (mrow < M32) *reinterpret_cast<uint4*>(dst + ch * 16) = make_uint4(o[0], o[1], o[2], o[3]);
             }
             if (warp == WPW + 1 + 4 * WSB) TR(3, k, 2);
@@ -1314,7 +1402,7 @@ template <class S, int G>
 cudaError_t launch_instance(const fused::Params& p, cudaStream_t st)
 {
     using L = convtc::Layout<S>;
-    auto kernel = convtc::conv_tc_kernel<S, G>;
+    auto kernel = p.mult_ch ? convtc::conv_tc_kernel<S, G, true> : convtc::conv_tc_kernel<S, G, false>;
     const size_t smem = (size_t)L::FIXED + (size_t)p.nbuf * (size_t)p.bufbytes;
     if (p.nbuf < G || p.nbuf <= convtc::PWN || smem > (size_t)convtc::SMEM_LIMIT) return cudaErrorInvalidValue;
     // the attribute is per kernel and per device: set on every call, it is cheap
@@ -1413,7 +1501,7 @@ static bool plan_wide(fused::Params& p, const q4_conv_desc& d, const uint8_t* X,
 
 static cudaError_t launch_wide(const fused::Params& p, size_t smem, cudaStream_t st)
 {
-    auto kernel = convtc::conv_tc_wide_kernel;
+    auto kernel = p.mult_ch ? convtc::conv_tc_wide_kernel<true> : convtc::conv_tc_wide_kernel<false>;
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          convtc::SMEM_LIMIT_WIDE);
     if (e != cudaSuccess) return e;
@@ -1484,19 +1572,22 @@ size_t conv_tc_image_bytes(const q4_conv_desc& d)
 
 // prep_out: only prepare the weights (B operand, per-column constants, fallback flag) into
 // that buffer of conv_tc_image_bytes(d) bytes; X and Y are not touched.  prep_in: run the layer
-// from such an image; Wt, colsum_w, bias and zb are not read.
+// from such an image; Wt, colsum_w, bias and zb are not read.  mult_ch / shift_ch (both or
+// neither) and zb_ch (optional): per output channel; zb, rq.mult and rq.shift are then unused.
 cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, const int32_t* colsum_w,
                            const int32_t* bias, const q4_conv_desc& d, int32_t za, int32_t zb,
                            const RequantParams& rq, uint8_t* Y, cudaStream_t st, const uint8_t* prep_in,
-                           uint8_t* prep_out)
+                           uint8_t* prep_out, const int32_t* zb_ch, const int32_t* mult_ch,
+                           const int32_t* shift_ch)
 {
+    if (mult_ch && (prep_in || prep_out)) return cudaErrorInvalidValue;    // images are per-tensor
     const TcChoice c = choose_instance(d);
     if (c.id < 0) {
         fused::Params p{};
         size_t smem = 0;
         if (!plan_wide(p, d, X, Y, &smem)) return cudaErrorInvalidValue;
         p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;
-        p.zb_ch = p.mult_ch = p.shift_ch = nullptr;
+        p.zb_ch = zb_ch; p.mult_ch = mult_ch; p.shift_ch = shift_ch;
         p.za = za; p.zb = zb; p.rq = rq;
         p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
         p.prep_in = prep_in; p.prep_out = prep_out;
@@ -1511,7 +1602,7 @@ cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, con
     fused::Params p{};
     if (plan_staging(p, d, X, convtc::ROWS * c.P, c.nib) <= 0) return cudaErrorInvalidValue;
     p.X = X; p.Wt = Wt; p.ldw = ldw; p.colsum_w = colsum_w; p.bias = bias; p.Y = Y;
-    p.zb_ch = p.mult_ch = p.shift_ch = nullptr;
+    p.zb_ch = zb_ch; p.mult_ch = mult_ch; p.shift_ch = shift_ch;
     p.za = za; p.zb = zb; p.rq = rq;
     p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
     p.nbuf = ring_for(c.id, p);

@@ -203,6 +203,14 @@ CONV_PC = [  # N, H, W, C, OC, KH, KW, sh, sw, ph, pw
     (5, 12, 20, 1, 8, 3, 3, 1, 1, 0, 0),        # output rows not groups of four: expanded copy, MMA kernel
     (2, 11, 9, 3, 24, 3, 3, 1, 1, 1, 1),        # odd channel count
     (40, 9, 10, 8, 40, 3, 3, 1, 1, 1, 1),       # many tiles
+    # layer classes of the tensor-memory kernels (the others above that match one take it too)
+    (3, 32, 32, 16, 32, 3, 3, 1, 1, 1, 1),      # 16 -> 32, stride 1, two pixels per GEMM row
+    (5, 24, 24, 16, 32, 3, 3, 2, 2, 1, 1),      # 16 -> 32, stride 2
+    (9, 12, 12, 32, 64, 3, 3, 2, 2, 1, 1),      # 32 -> 64, stride 2, one pixel per row
+    (37, 10, 16, 8, 16, 3, 3, 2, 2, 1, 1),      # 8 -> 16, stride 2, four pixels per row, several images per tile
+    (2, 16, 16, 64, 128, 3, 3, 1, 1, 1, 1),     # run-time-geometry kernel, 128 columns
+    (2, 8, 8, 128, 256, 3, 3, 1, 1, 1, 1),      # ... channels split over two CTAs
+    (3, 10, 14, 32, 96, 5, 5, 2, 1, 2, 2),      # ... 5x5, mixed strides
 ]
 
 
