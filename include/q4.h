@@ -286,9 +286,11 @@ q4_status q4_gemm_requant_channels(const uint8_t* A, int64_t lda, const uint8_t*
  * unrolled matrix is never written; no workspace): like q4_conv2d, but output channel n has
  * its own weight zero point zb[n] (0..15), multiplier mult[n] in [2^30, 2^31) and shift[n] in
  * 0..31 (DEVICE arrays of OC int32, not range-checked); colsum_w and bias may be NULL.
- * Layers the fused kernel does not take (OC not a multiple of 8 or above 64, Y not 8-byte
- * aligned, too large for shared memory) return Q4_ERR_UNSUPPORTED: run those as q4_im2col,
- * q4_gemm with zb = 0 and q4_requant_channels.  Extension of the paper's per-matrix scheme
+ * The layer runs on the tensor-memory kernels where they have an instance for it (the
+ * 3x3 layer classes of the workloads; any layer with C and OC multiples of 32), else on the
+ * warp-level fused kernels.  Layers neither takes (e.g. OC not a multiple of 8, or above 64
+ * with C not a multiple of 32; Y not 8-byte aligned; too large for shared memory) return
+ * Q4_ERR_UNSUPPORTED: run those as q4_im2col, q4_gemm with zb = 0 and q4_requant_channels.  Extension of the paper's per-matrix scheme
  * (Section II-A), see q4_requant_channels.
  */
 q4_status q4_conv2d_channels(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
