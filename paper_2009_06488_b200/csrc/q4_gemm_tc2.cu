@@ -2,15 +2,17 @@
 // terms): CTA pairs computing 256 x 192 or 256 x 256 output tiles with
 // tcgen05.mma.cta_group::2, the A operand fed from tensor memory.
 //
-// Why this shape.  The unpack (nibbles -> bytes) is bounded by the shared-memory
-// load/store pipe, 128 B/clk: every packed byte is read once and every unpacked byte
-// written once before the MMA can read it.  Two things cut that traffic:
+// Why this shape.  The unpack (nibbles -> bytes) costs shared-memory traffic -- every
+// packed byte is read once and every unpacked byte written once before the MMA can read
+// it, through a 128 B/clk pipe -- and instructions of the unpack warps, which is what
+// bound the kernel in the end.  Two things cut the traffic:
 //   * a CTA pair shares the Bt tile, so each CTA stages and unpacks only half of it;
 //   * the unpacked A rows never touch shared memory: each unpack thread owns one row,
 //     expands its 64 packed bytes in registers and writes them to tensor memory
 //     (tcgen05.st), from where the MMA reads A directly.
 // Per 128-deep stage a CTA then moves 8 KB (A, loads only) + 6 KB + 12 KB (Bt, loads and
-// stores) through the load/store pipe -- about half of what the MMA's 384 clocks allow.
+// stores; 8 + 16 KB with 256-column tiles) through the load/store pipe -- about half of
+// what the MMAs' 400 to 530 clocks allow.
 //
 // Tensor memory (512 columns), 192-column tiles: two accumulators (the epilogue of tile t
 // overlaps the main loop of t+1) and four A stages of 32 columns (128 depth bytes); the
@@ -20,13 +22,13 @@
 // (see Cfg).
 //
 // Roles per CTA (18 warps): warp 0 TMA producer (its own 128 rows of A, 64-byte-swizzled
-// so that row-per-lane reads are conflict-free, and its own 96 rows of Bt; no
-// multicast); warps 2..13 unpack, as three groups of four that take stages in turn so
+// so that row-per-lane reads are conflict-free, and its own half of the tile's rows of Bt;
+// no multicast); warps 2..13 unpack, as three groups of four that take stages in turn so
 // one group's waits and fences hide behind the others' work, and arrive -- from both
 // CTAs -- on the leader CTA's "operands ready" barrier; warp 1 of the leader CTA issues
 // the pair MMAs and commits to both CTAs' barriers; warp 1 of the peer CTA relays
-// "accumulator drained" once per tile; the last four warps are the epilogue.  Column sums of the two
-// Bt halves are exchanged through distributed shared memory.
+// "accumulator drained" to the leader; the last four warps are the epilogue.  Column sums
+// of the two CTAs' Bt rows are exchanged through distributed shared memory.
 //
 // The depth order inside each 32-value group (even nibbles, then odd) is the same for A
 // and Bt, so the product is unchanged.  Every mbarrier wait is bounded; the only
