@@ -59,7 +59,8 @@ typedef enum {
     Q4_ERR_UNSUPPORTED = 5,     /* valid, but this entry point has no kernel for it         */
     Q4_ERR_CUDA = 6,            /* a CUDA runtime / driver call failed                     */
     Q4_ERR_DEVICE_TIMEOUT = 7,  /* a bounded device-side wait expired                      */
-    Q4_ERR_STATIC_SCRATCH = 8   /* problem needs more scratch than q4_conv2d_static holds  */
+    Q4_ERR_STATIC_SCRATCH = 8,  /* problem needs more scratch than q4_conv2d_static holds  */
+    Q4_ERR_WEIGHT_IMAGE = 9     /* q4_conv2d_prepared was given another layer's weight image */
 } q4_status;
 
 /* Integer re-quantization of an int32 accumulator to the next layer's uint4 input.
@@ -177,6 +178,11 @@ q4_status q4_conv2d(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
  * aligned, owned by the caller, written by one small kernel on `stream`.
  * q4_conv2d_prepared: X, Y, rq, za as in q4_conv2d (za must be the one the image was
  * prepared with); needs no workspace.
+ * An image does not depend on the batch, the image size, the vertical stride or the
+ * paddings: one image serves every descriptor that differs in those only.  It carries a tag
+ * of what it does depend on besides the weights (kernel, filter, channel counts, horizontal
+ * stride, za, image format); q4_conv2d_prepared given an image with another tag writes
+ * nothing to Y, and the next q4_last_device_status on the device returns Q4_ERR_WEIGHT_IMAGE.
  * Errors: as q4_conv2d; Q4_ERR_UNSUPPORTED when the layer (or the alignment of X / Y: 16
  * bytes) has no tensor-memory kernel, Q4_ERR_WORKSPACE when prepared_bytes is too small,
  * Q4_ERR_ALIGNMENT when `prepared` is not 16-byte aligned.  Nothing is launched on error.
@@ -366,8 +372,9 @@ size_t q4_gemm_host_staging_bytes(int32_t M, int32_t N, int32_t K,
                                   int64_t lda, int64_t ldb, int64_t ldc);
 
 /* Synchronizes `stream`, then returns Q4_ERR_DEVICE_TIMEOUT if any kernel of this
- * library gave up a bounded wait on the current device since the last call (the
- * flag is cleared), Q4_ERR_CUDA if the stream reports an error, else Q4_OK. */
+ * library gave up a bounded wait on the current device since the last call,
+ * Q4_ERR_WEIGHT_IMAGE if q4_conv2d_prepared refused a weight image (the flags are cleared),
+ * Q4_ERR_CUDA if the stream reports an error, else Q4_OK. */
 q4_status q4_last_device_status(void* stream);
 
 /*

@@ -27,7 +27,7 @@ if not os.path.exists(LIB_PATH):
 _lib = ctypes.CDLL(LIB_PATH)
 
 (Q4_OK, Q4_ERR_INVALID_ARG, Q4_ERR_ALIGNMENT, Q4_ERR_RANGE, Q4_ERR_WORKSPACE,
- Q4_ERR_UNSUPPORTED, Q4_ERR_CUDA, Q4_ERR_DEVICE_TIMEOUT, Q4_ERR_STATIC_SCRATCH) = range(9)
+ Q4_ERR_UNSUPPORTED, Q4_ERR_CUDA, Q4_ERR_DEVICE_TIMEOUT, Q4_ERR_STATIC_SCRATCH, Q4_ERR_WEIGHT_IMAGE) = range(10)
 Q4_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_static",

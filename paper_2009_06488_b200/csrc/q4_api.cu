@@ -638,7 +638,7 @@ q4_status q4_last_device_status(void* stream)
     if (cudaMemcpy(&word, dptr, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return Q4_ERR_CUDA;
     if (word) {
         if (cudaMemset(dptr, 0, sizeof(word)) != cudaSuccess) return Q4_ERR_CUDA;
-        return Q4_ERR_DEVICE_TIMEOUT;
+        return (word & kStatusTimeout) ? Q4_ERR_DEVICE_TIMEOUT : Q4_ERR_WEIGHT_IMAGE;
     }
     return Q4_OK;
 }
@@ -661,6 +661,7 @@ const char* q4_status_string(q4_status s)
         case Q4_ERR_RANGE: return "value out of range";
         case Q4_ERR_WORKSPACE: return "workspace missing or too small";
         case Q4_ERR_UNSUPPORTED: return "unsupported";
+        case Q4_ERR_WEIGHT_IMAGE: return "weight image prepared for another layer";
         case Q4_ERR_CUDA: return "CUDA error";
         case Q4_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
         case Q4_ERR_STATIC_SCRATCH:

@@ -11,6 +11,7 @@ namespace q4 {
 
 // Bits of the device status word (reported by q4_last_device_status).
 constexpr unsigned kStatusTimeout = 1u;
+constexpr unsigned kStatusWeightImage = 2u;     // a prepared weight image with another layer's tag
 
 struct RequantParams {
     int32_t mult, shift, zo, lo, hi;

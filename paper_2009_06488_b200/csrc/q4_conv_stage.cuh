@@ -26,6 +26,7 @@ struct Params {
     // prep_out = build it and write it there, do nothing else; prep_in = take it from there
     const uint8_t* prep_in;
     uint8_t* prep_out;
+    uint32_t prep_tag;         // what the image is for (layer class, filter, channels, za, build): written / checked
     int64_t M;
     int32_t H, W, C, KH, KW, OH, OW, sh, sw, ph, pw;
     int32_t K, KS;             // depth, number of 32-byte MMA depth steps

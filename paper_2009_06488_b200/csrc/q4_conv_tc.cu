@@ -419,22 +419,31 @@ conv_tc_kernel(const Params p)
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t ntiles = (p.M + S::TILE - 1) / S::TILE;
-    const int mytiles = (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+    int mytiles = (int)((ntiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
     const uint32_t M32 = (uint32_t)p.M;
+    constexpr uint32_t IMAGE = (uint32_t)(S::B_BYTES + N * 4);     // B and the per-column constants, contiguous
+    // A prepared weight image ends in {fallback flag, tag}.  An image with another tag (another
+    // layer class, filter, channel counts, za or build) is not used: the launch does nothing and
+    // the status word says why.
+    uint2 trailer = make_uint2(0u, p.prep_tag);
+    if (p.prep_in != nullptr) trailer = __ldg(reinterpret_cast<const uint2*>(p.prep_in + IMAGE));
+    if (trailer.y != p.prep_tag) {
+        mytiles = 0;
+        if (tid == 0) atomicOr(p.status, kStatusWeightImage);
+    }
 
     // The producers start copying the first tiles at once; meanwhile the other warps
     // prepare the weights (synchronising among themselves on a named barrier).
     uint32_t tmem_base = 0;
     bool use_preload = false;              // a constant beyond the digits' range: preloaded accumulators instead
-    constexpr uint32_t IMAGE = (uint32_t)(S::B_BYTES + N * 4);     // B and the per-column constants, contiguous
     if (warp >= PWN && p.prep_in != nullptr) {
         // The weights were prepared ahead of time (the B operand, the constants, the flag):
         // one bulk copy brings them in; only the MMA warp has to wait for it.
-        if (tid == PWN * 32) {
+        if (tid == PWN * 32 && mytiles > 0) {
             mbar_expect_tx(bar_prep, IMAGE);
             fused::bulk_load_row(sbase + L::OFF_B, p.prep_in, IMAGE, bar_prep);
         }
-        use_preload = __ldg(reinterpret_cast<const int*>(p.prep_in + IMAGE)) != 0;
+        use_preload = trailer.x != 0;
         tmem_base = (uint32_t)lds32(tmem_slot);
     } else if (warp >= PWN) {
         constexpr int NT = THREADS - PWN * 32;         // threads that prepare the weights
@@ -603,7 +612,7 @@ conv_tc_kernel(const Params p)
             const uint4* src = reinterpret_cast<const uint4*>(smem + L::OFF_B);
             uint4* dst = reinterpret_cast<uint4*>(p.prep_out);
             for (int i = wt; i < (int)(IMAGE / 16); i += NT) dst[i] = src[i];
-            if (wt == 0) dst[IMAGE / 16] = make_uint4(use_preload ? 1u : 0u, 0u, 0u, 0u);
+            if (wt == 0) dst[IMAGE / 16] = make_uint4(use_preload ? 1u : 0u, p.prep_tag, 0u, 0u);
         }
     }
 
@@ -926,8 +935,18 @@ conv_tc_wide_kernel(const Params p)
     asm volatile("griddepcontrol.wait;" ::: "memory");             // see conv_tc_kernel
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int64_t ntiles = (p.M + ROWS - 1) / ROWS;
-    const int mytiles = (int)((ntiles - tile0 + tstride - 1) / tstride);
+    int mytiles = (int)((ntiles - tile0 + tstride - 1) / tstride);
     const uint32_t M32 = (uint32_t)p.M;
+    // a CTA's share of a prepared image: B, the per-column constants, {fallback flag, tag} (see conv_tc_kernel)
+    const uint32_t b_bytes = (uint32_t)L.off_tab, share_bytes = b_bytes + (uint32_t)N * 4u + 16u;
+    uint2 trailer = make_uint2(0u, p.prep_tag);
+    if (p.prep_in != nullptr)
+        trailer = __ldg(reinterpret_cast<const uint2*>(p.prep_in + (size_t)(blockIdx.x % nsplit) * share_bytes + b_bytes +
+                                                       (uint32_t)N * 4u));
+    if (trailer.y != p.prep_tag) {
+        mytiles = 0;
+        if (tid == 0) atomicOr(p.status, kStatusWeightImage);
+    }
 
     uint32_t tmem_base = 0;
     bool use_preload = false;
@@ -946,16 +965,14 @@ conv_tc_wide_kernel(const Params p)
             tab[ks] = make_int2(kh * p.rowbytes + kw * p.unit + 16 * c4, kw);
         }
         sync_workers();
-        // a CTA's share of a prepared image: B, the per-column constants, 16 bytes with the flag
-        const uint32_t b_bytes = (uint32_t)L.off_tab, share_bytes = b_bytes + (uint32_t)N * 4u + 16u;
         if (prepared) {
             const uint8_t* img = p.prep_in + (size_t)(blockIdx.x % nsplit) * share_bytes;
-            if (wt == 0) {
+            if (wt == 0 && mytiles > 0) {
                 mbar_expect_tx(bar_prep, b_bytes + (uint32_t)N * 4u);
                 fused::bulk_load_row(sbase, img, b_bytes, bar_prep);
                 fused::bulk_load_row(colterm_s, img + b_bytes, (uint32_t)N * 4u, bar_prep);
             }
-            use_preload = __ldg(reinterpret_cast<const int*>(img + b_bytes + (uint32_t)N * 4u)) != 0;
+            use_preload = trailer.x != 0;
             tmem_base = (uint32_t)lds32(tmem_slot);
         } else {
         // B: row n is output channel oc0 + (n with the ch8 order inside each group of eight);
@@ -1080,7 +1097,7 @@ conv_tc_wide_kernel(const Params p)
             for (int i = wt; i < (int)(b_bytes / 16); i += NT) dst[i] = src[i];
             const uint4* cs = reinterpret_cast<const uint4*>(smem + L.off_ct);
             for (int i = wt; i < N / 4; i += NT) dst[b_bytes / 16 + i] = cs[i];
-            if (wt == 0) dst[b_bytes / 16 + N / 4] = make_uint4(use_preload ? 1u : 0u, 0u, 0u, 0u);
+            if (wt == 0) dst[b_bytes / 16 + N / 4] = make_uint4(use_preload ? 1u : 0u, p.prep_tag, 0u, 0u);
         }
         }
     }
@@ -1548,6 +1565,20 @@ bool conv_tc_supported(const q4_conv_desc& d, const uint8_t* X, const uint8_t* W
     return ring_for(c.id, p) > 0;
 }
 
+// What a weight image is for: everything its contents depend on besides the weights, their zero
+// point and the bias -- the kernel (instance or run-time geometry, with its pixels per row), the
+// filter, the channel counts, the horizontal stride, za, and this build's image format.  Batch,
+// image size, vertical stride and paddings do not enter: one image serves them all.
+static uint32_t image_tag(const q4_conv_desc& d, int32_t za, int instance, int P)
+{
+    const uint32_t f[] = {0x51345747u /* format 1 */, (uint32_t)instance, (uint32_t)P, (uint32_t)d.C, (uint32_t)d.OC,
+                          (uint32_t)d.KH, (uint32_t)d.KW, (uint32_t)d.stride_w, (uint32_t)za};
+    uint32_t h = 2166136261u;                          // FNV-1a over the words' bytes
+    for (uint32_t w : f)
+        for (int b = 0; b < 4; ++b) { h ^= (w >> (8 * b)) & 0xFFu; h *= 16777619u; }
+    return h ? h : 1u;
+}
+
 template <class S> static size_t image_bytes_of() { return (size_t)S::B_BYTES + (size_t)S::N * 4 + 16; }
 
 // Bytes of the prepared weight image of a layer (see launch_conv_tc), 0 if no tensor-memory
@@ -1590,7 +1621,7 @@ cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, con
         p.zb_ch = zb_ch; p.mult_ch = mult_ch; p.shift_ch = shift_ch;
         p.za = za; p.zb = zb; p.rq = rq;
         p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
-        p.prep_in = prep_in; p.prep_out = prep_out;
+        p.prep_in = prep_in; p.prep_out = prep_out; p.prep_tag = image_tag(d, za, 100, 1);
         p.status = device_status_ptr();
         if (!p.status) return cudaErrorUnknown;
         if (prep_out) p.M = 0;                         // no tiles: the CTAs prepare their shares and leave
@@ -1606,7 +1637,7 @@ cudaError_t launch_conv_tc(const uint8_t* X, const uint8_t* Wt, int64_t ldw, con
     p.za = za; p.zb = zb; p.rq = rq;
     p.wt_words = (uintptr_t)Wt % 4 == 0 && ldw % 4 == 0;
     p.nbuf = ring_for(c.id, p);
-    p.prep_in = prep_in; p.prep_out = prep_out;
+    p.prep_in = prep_in; p.prep_out = prep_out; p.prep_tag = image_tag(d, za, c.id, c.P);
     p.status = device_status_ptr();
     if (!p.status) return cudaErrorUnknown;
     if (prep_out) p.M = 0;                             // no tiles: one CTA prepares the image and leaves

@@ -45,6 +45,45 @@ def check_prepared_weights(q4, Xd, Wt, dq, za, zb, rq, bias, colsum, want):
     assert (img[nb:].cpu().numpy() == 0xA5).all()
 
 
+def test_weight_image_serves_other_batches_and_sizes_but_not_other_layers(q4):
+    """An image depends on the layer class, the filter, the channel counts and za, not on the
+    batch or the image size; given to another layer it is refused: nothing is written and
+    the device status says so."""
+    import torch
+    rq = ((1 << 30) + 77, 5, 3, 1, 14)
+    za, zb = 6, 9
+    base = (3, 32, 32, 16, 32, 3, 3, 1, 1, 1, 1)
+    seed = 9700
+    Wt = wl.rand_packed(seed, 2, 32, 144)
+    bias = wl.rand_ints(seed, 3, -300, 300, 32).astype(np.int32)
+    d0 = q4.ConvDesc(*base)
+    nb = q4.q4_conv2d_weights_bytes(d0)
+    img = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    q4.q4_conv2d_prepare_weights(dev(Wt), d0, za, zb, img, dev(bias))
+    for g in ((7, 20, 24, 16, 32, 3, 3, 1, 1, 1, 1), (1, 64, 40, 16, 32, 3, 3, 1, 1, 0, 1)):   # other batch / size / padding
+        dq, do = q4.ConvDesc(*g), oracle.ConvDesc(*g)
+        assert q4.q4_conv2d_weights_bytes(dq) == nb
+        X = wl.rand_flat_nibbles(seed + g[0], 1, g[0] * g[1] * g[2] * g[3])
+        want = oracle.conv2d(X, Wt, bias, do, za, zb, oracle.Requant(*rq))
+        Y = torch.full((dq.M, 16), 0x3C, dtype=torch.uint8, device="cuda")
+        q4.q4_conv2d_prepared(dev(X), img, dq, za, q4.Requant(*rq), Y)
+        assert q4.q4_last_device_status() == q4.Q4_OK
+        assert (Y.cpu().numpy() == want).all()
+    # the stride-2 layer class of the same channel counts has an image of the same size, but another tag
+    other = q4.ConvDesc(3, 32, 32, 16, 32, 3, 3, 2, 2, 1, 1)
+    assert q4.q4_conv2d_weights_bytes(other) == nb
+    X = dev(wl.rand_flat_nibbles(seed, 9, 3 * 32 * 32 * 16))
+    Y = torch.full((other.M, 16), 0x3C, dtype=torch.uint8, device="cuda")
+    q4.q4_conv2d_prepared(X, img, other, za, q4.Requant(*rq), Y)
+    assert q4.q4_last_device_status() == q4.Q4_ERR_WEIGHT_IMAGE
+    assert (Y.cpu().numpy() == 0x3C).all()                  # nothing written
+    Y0 = torch.full((d0.M, 16), 0x3C, dtype=torch.uint8, device="cuda")
+    q4.q4_conv2d_prepared(X, img, d0, za + 1, q4.Requant(*rq), Y0)                # another za
+    assert (Y0.cpu().numpy() == 0x3C).all()
+    assert q4.q4_last_device_status() == q4.Q4_ERR_WEIGHT_IMAGE
+    assert q4.q4_last_device_status() == q4.Q4_OK            # reported once
+
+
 TC_LAYERS = [  # N, H, W, C, OC, stride, pad_h, shift
     (2, 8, 8, 1, 8, 1, 1, 5),          # gray first layer, less than one tile
     (5, 48, 48, 1, 8, 1, 1, 5),        # ... tiles that end inside an image
