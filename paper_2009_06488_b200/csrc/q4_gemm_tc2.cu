@@ -69,8 +69,9 @@ constexpr int STG_SET = 4 * 32 * 128;      // int32 epilogue staging: 4 warps x 
 // the lower halves alternate between the outer two, and each depth step is two MMAs of 128
 // columns (the same tensor time as one of 256).  The epilogue drains the upper half first;
 // the next tile's lower-half MMAs start at once on the free outer buffer and only its
-// upper-half MMAs wait for that half drain, so about a third of the epilogue is exposed
-// instead of all of it.  Four A and four Bt stages.  It wins where its tile count fits the
+// upper-half MMAs wait for that half drain; a tile's last upper-half MMAs are issued before
+// its last lower-half ones, so that the drain starts early.  About a third of the epilogue is
+// exposed instead of all of it.  Four A and four Bt stages.  It wins where its tile count fits the
 // 74 CTA pairs better or the depth is long, and loses e.g. at 4096^3 (four waves against
 // five of 192-column tiles with fully overlapped epilogues).
 // NSTG: staging slices per epilogue warp.  With two, a TMA store reads one while the next is
@@ -86,11 +87,8 @@ struct Cfg {
     static constexpr bool ROT = BNC == 256;      // rotating half accumulators
     static constexpr int NACC = ROT ? 1 : 2;     // whole accumulators / depth-sum buffers in flight
     static constexpr int US = 4;                 // A operand stages in tensor memory
-#ifndef Q4_PAIR_BS256
-#define Q4_PAIR_BS256 4
-#endif
-    static constexpr int BS = ROT ? Q4_PAIR_BS256 : 8;   // Bt operand stages in shared memory (BH * 128 B each)
-    static constexpr int WALK = BS % US == 0 ? BS : (BS % 2 == 0 ? BS * US / 2 : BS * US);   // a common multiple of both rings
+    static constexpr int BS = ROT ? 4 : 8;       // Bt operand stages in shared memory (BH * 128 B each)
+    static constexpr int WALK = BS;              // stages per block of the MMA loop: a multiple of both ring depths
     static constexpr int BBOX = ROT ? BH / 2 : BH;   // rows per TMA box of Bt
     static constexpr int PS = ROT ? (NSTG == 2 ? 7 : 8) : 6;   // packed stages (A 8 KB + Bt BH * 64 B)
     static constexpr int PSTAGE = PA + BH * PROW;
