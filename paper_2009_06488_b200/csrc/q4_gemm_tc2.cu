@@ -157,11 +157,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                   OFF_BAR = C::OFF_BAR, OFF_MISC = C::OFF_MISC;
     constexpr uint32_t kIdesc = C::kIdesc;
     constexpr bool ROT = C::ROT;
-    // Per-channel launches that unpack Bt themselves store its rows in the order ch8() within
-    // every group of eight, so that an accumulator register pair holds channels i and i + 4: the
-    // epilogue then re-quantizes eight values at a time (requant8_channels: 8192^3 358 -> 327 us).
-    // (The per-tensor epilogue gains nothing from it: measured 310 against 297 us.)
-    constexpr bool CAN_PERM = REQUANT && !BPRE;
     constexpr int PS = C::PS, WALK = C::WALK;
     extern __shared__ uint8_t smem_raw[];
     // the same offset in both CTAs: dynamic shared memory starts at the same address
@@ -236,7 +231,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // per-channel re-quantization: the 32-bit rounding form needs every shift in 2..27
     const bool pc = REQUANT && g.mult_ch != nullptr;
-    const bool PERM = CAN_PERM && pc;            // (uniform over the launch)
     int pc_fast = 1;
     if (pc) {
         int ok = 1;
@@ -454,27 +448,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t full_u_leader = map_to_cta(bar_full_u(0), 0);  // barrier in the leader CTA
         // per-thread, stage-independent offsets: my four packed chunks of A (swizzled), my
         // packed chunks of Bt and where their two unpacked halves go
-        // Bt row of task id (four tasks per row).  With permuted rows, the eight lanes of a
-        // quarter warp -- which a 16-byte shared-memory access serves together -- take two rows
-        // whose source rows AND destination rows differ in parity (0 and 5, 1 and 4, 2 and 7,
-        // 3 and 6 of each group of eight), so that neither their loads nor their stores collide.
-        auto bt_row = [PERM](int id) {
-            const int r = id >> 2;
-            return PERM ? (r & ~7) + (int)((0x63724150u >> (4 * (r & 7))) & 7u) : r;
-        };
         uint32_t a_ld[4], b_ld[NTB], b_lo[NTB], b_hi[NTB];
 #pragma unroll
         for (int c = 0; c < 4; ++c) a_ld[c] = a_off + (((uint32_t)c ^ a_sw) << 4);
 #pragma unroll
         for (int j = 0; j < NTB; ++j) {
             const int id = gt + j * GT;
-            const int r = bt_row(id), c = id & 3;
-            // where row r goes: its place among its group of eight (the inverse of ch8)
-            const int rd = PERM ? (r & ~7) + 2 * (r & 3) + ((r >> 2) & 1) : r;
-            const int sw = rd & 7;
+            const int r = id >> 2, c = id & 3, sw = r & 7;
             b_ld[j] = (uint32_t)(PA + r * PROW + c * 16);
-            b_lo[j] = (uint32_t)(rd * UROW + (((2 * c) ^ sw) << 4));
-            b_hi[j] = (uint32_t)(rd * UROW + (((2 * c + 1) ^ sw) << 4));
+            b_lo[j] = (uint32_t)(r * UROW + (((2 * c) ^ sw) << 4));
+            b_hi[j] = (uint32_t)(r * UROW + (((2 * c + 1) ^ sw) << 4));
         }
         // Stages are numbered across tiles (every tile has nslab of them, so stage s of my
         // lt-th tile is number lt * nslab + s); this group takes the numbers congruent to grp
@@ -568,7 +551,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if ((id & 3) == 0) {
                         // column sum of one of my rows of Bt: both CTAs need it.  Tile column
                         // of my row r: my run of BH rows, or (ROT) one of my two runs of 64
-                        const int r = bt_row(id);
+                        const int r = id >> 2;
                         const int col = !ROT ? (int)rank * BH + r
                                              : (r < C::BBOX ? (int)rank * C::BBOX + r : BH + (int)rank * C::BBOX + r - C::BBOX);
                         const uint32_t a = mine + 4 * (TMC + col);
@@ -598,14 +581,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (need_sums) mbar_wait_cl(bar_sums(acc), aph, abort_flag, g.status);
             const uint32_t s0 = sums_s + 4 * (acc * G * SUMS_N);
             for (int j = et; j < BNC; j += 128) {
-                // accumulator column j holds this channel of the tile
-                const int jc = PERM ? (j & ~7) + ch8(j & 7) : j;
-                const int n = n0 + jc;
+                const int n = n0 + j;
                 int cb = 0, bias = 0, zbn = pc ? 0 : g.zb;
                 if (n < g.N) {
                     if (need_cb) {
 #pragma unroll
-                        for (int gi = 0; gi < G; ++gi) cb += lds32(s0 + 4 * (gi * SUMS_N + TMC + jc));
+                        for (int gi = 0; gi < G; ++gi) cb += lds32(s0 + 4 * (gi * SUMS_N + TMC + j));
                     } else {
                         cb = g.colsum_b[n];
                     }
@@ -620,7 +601,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const int s = pc_fast ? sh - 1 : sh;
                     sts32(pc_s + 4 * j, zbn);
                     sts32(pc_s + 4 * (BNC + j), mult);
-                    sts32(pc_s + 4 * (2 * BNC + j), pc_fast ? (1 << (s - 1)) + (g.rq.zo - (PERM ? g.rq.lo : 0)) * (1 << s) : 0);
+                    sts32(pc_s + 4 * (2 * BNC + j), pc_fast ? (1 << (s - 1)) + (g.rq.zo - g.rq.lo) * (1 << s) : 0);
                     sts32(pc_s + 4 * (3 * BNC + j), s);
                 }
             }
@@ -705,27 +686,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         }
                     } else {
                         uint32_t o[4];
-                        if (PERM) {
-                            // eight values at a time; each word holds value - lo per nibble
+                        if (pc) {
+                            // eight values at a time (channels i and i + 4 share a packed pair); each
+                            // word holds value - lo per nibble
                             const uint32_t hml2 = (uint32_t)(g.rq.hi - g.rq.lo) * 0x00010001u;
                             const uint32_t lofill = (uint32_t)g.rq.lo * 0x11111111u;
 #pragma unroll
                             for (int qd = 0; qd < 4; ++qd)
-                                o[qd] = requant8_channels(r + 8 * qd, g.rq, pc_s + 4 * BNC, BNC, ch * 32 + 8 * qd,
-                                                          pc_fast != 0, hml2) + lofill;
-                        } else if (pc) {
-#pragma unroll
-                            for (int qd = 0; qd < 8; ++qd) {
-                                const uint4 mu = lds128(pc_s + 4 * (BNC + ch * 32 + 4 * qd));
-                                const uint4 rn = lds128(pc_s + 4 * (2 * BNC + ch * 32 + 4 * qd));
-                                const uint4 sf = lds128(pc_s + 4 * (3 * BNC + ch * 32 + 4 * qd));
-                                const uint32_t h =
-                                    requant_channel((int32_t)r[4 * qd + 0], (int)mu.x, (int)rn.x, (int)sf.x, pc_fast, g.rq) |
-                                    requant_channel((int32_t)r[4 * qd + 1], (int)mu.y, (int)rn.y, (int)sf.y, pc_fast, g.rq) << 4 |
-                                    requant_channel((int32_t)r[4 * qd + 2], (int)mu.z, (int)rn.z, (int)sf.z, pc_fast, g.rq) << 8 |
-                                    requant_channel((int32_t)r[4 * qd + 3], (int)mu.w, (int)rn.w, (int)sf.w, pc_fast, g.rq) << 12;
-                                if (qd & 1) o[qd >> 1] |= h << 16; else o[qd >> 1] = h;
-                            }
+                                o[qd] = requant8_channels<true>(r + 8 * qd, g.rq, pc_s + 4 * BNC, BNC, ch * 32 + 8 * qd,
+                                                                pc_fast != 0, hml2) + lofill;
                         } else {
 #pragma unroll
                             for (int qd = 0; qd < 4; ++qd) {

@@ -69,6 +69,10 @@ __device__ __forceinline__ uint32_t requant8(const uint32_t* r, const RequantPar
 // channel), read from shared memory at pc_s + 4 * (array * n_cols + column): columns
 // col0 .. col0 + 7.  fast: every shift allows the 32-bit form (the arrays then hold
 // rnd = 2^(s-1) + ((zo - lo) << s) and s = shift - 1), else they hold the shifts themselves.
+// NATURAL: the eight accumulators (and their parameters) are channels 0..7 in order -- the
+// halves of a packed pair may be any two registers, so channels i and i + 4 are paired directly;
+// otherwise they come in the ch8 order of the convolution kernels' B operand.
+template <bool NATURAL = false>
 __device__ __forceinline__ uint32_t requant8_channels(const uint32_t* r, const RequantParams& rq, uint32_t pc_s,
                                                       int n_cols, int col0, bool fast, uint32_t hml2)
 {
@@ -82,8 +86,9 @@ __device__ __forceinline__ uint32_t requant8_channels(const uint32_t* r, const R
         uint32_t c[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-            const int q0 = mulhi_add((int)r[2 * i], mu[2 * i], rn[2 * i]) >> sh[2 * i];
-            const int q1 = mulhi_add((int)r[2 * i + 1], mu[2 * i + 1], rn[2 * i + 1]) >> sh[2 * i + 1];
+            const int a = NATURAL ? i : 2 * i, b = NATURAL ? i + 4 : 2 * i + 1;     // channels i and i + 4
+            const int q0 = mulhi_add((int)r[a], mu[a], rn[a]) >> sh[a];
+            const int q1 = mulhi_add((int)r[b], mu[b], rn[b]) >> sh[b];
             c[i] = __vimin_s16x2_relu(pack_sat16(q1, q0), hml2);
         }
         return mad_u32(c[3], 1u << 12, mad_u32(c[2], 1u << 8, mad_u32(c[1], 1u << 4, c[0])));
@@ -92,7 +97,7 @@ __device__ __forceinline__ uint32_t requant8_channels(const uint32_t* r, const R
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         const RequantParams one{mu[e], sh[e], rq.zo, rq.lo, rq.hi};
-        o |= (requant_wide((int)r[e], one) - (uint32_t)rq.lo) << (4 * ch8(e));
+        o |= (requant_wide((int)r[e], one) - (uint32_t)rq.lo) << (4 * (NATURAL ? e : ch8(e)));
     }
     return o;
 }
