@@ -78,23 +78,6 @@ __device__ __forceinline__ uint32_t requant(int32_t acc, const RequantParams& rq
     return (uint32_t)q;
 }
 
-// Per-channel form of requant(): the column's multiplier, and for the fast form (every
-// shift of the call in 2..27) the rounding constant 2^(s-1) + zo * 2^s with s = shift - 1,
-// so that (mulhi + rnd) >> s is already q + zo; otherwise `s` holds the shift itself and the
-// 64-bit form is used.
-__device__ __forceinline__ uint32_t requant_channel(int32_t acc, int32_t mult, int32_t rnd, int32_t s,
-                                                    bool fast, const RequantParams& rq)
-{
-    if (fast) {
-        int q = (__mulhi(acc, mult) + rnd) >> s;
-        q = max(q, rq.lo);
-        q = min(q, rq.hi);
-        return (uint32_t)q;
-    }
-    const RequantParams one{mult, s, rq.zo, rq.lo, rq.hi};
-    return requant_wide(acc, one);
-}
-
 // Unsigned 4 x 8-bit dot product accumulated into a (wrapping) 32-bit value.
 __device__ __forceinline__ int dp4a_u8(uint32_t a, uint32_t b, int c)
 {

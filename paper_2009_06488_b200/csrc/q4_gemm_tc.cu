@@ -28,6 +28,7 @@
 #include <mutex>
 
 #include "q4_common.cuh"
+#include "q4_requant8.cuh"
 #include "q4_tc_ptx.cuh"
 
 namespace q4 {
@@ -319,7 +320,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const int s = pc_fast ? sh - 1 : sh;
                     sts32(pc_s + 4 * j, zbn);
                     sts32(pc_s + 4 * (BN + j), mult);
-                    sts32(pc_s + 4 * (2 * BN + j), pc_fast ? (1 << (s - 1)) + g.rq.zo * (1 << s) : 0);
+                    sts32(pc_s + 4 * (2 * BN + j), pc_fast ? (1 << (s - 1)) + (g.rq.zo - g.rq.lo) * (1 << s) : 0);
                     sts32(pc_s + 4 * (3 * BN + j), s);
                 }
             }
@@ -380,18 +381,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     } else {
                         uint32_t o[4];
                         if (pc) {
+                            // eight values at a time (channels i and i + 4 share a packed pair); each
+                            // word holds value - lo per nibble
+                            const uint32_t hml2 = (uint32_t)(g.rq.hi - g.rq.lo) * 0x00010001u;
+                            const uint32_t lofill = (uint32_t)g.rq.lo * 0x11111111u;
 #pragma unroll
-                            for (int q = 0; q < 8; ++q) {
-                                const uint4 mu = lds128(pc_s + 4 * (BN + ch * 32 + 4 * q));
-                                const uint4 rn = lds128(pc_s + 4 * (2 * BN + ch * 32 + 4 * q));
-                                const uint4 sf = lds128(pc_s + 4 * (3 * BN + ch * 32 + 4 * q));
-                                const uint32_t h =
-                                    requant_channel((int32_t)r[4 * q + 0], (int)mu.x, (int)rn.x, (int)sf.x, pc_fast, g.rq) |
-                                    requant_channel((int32_t)r[4 * q + 1], (int)mu.y, (int)rn.y, (int)sf.y, pc_fast, g.rq) << 4 |
-                                    requant_channel((int32_t)r[4 * q + 2], (int)mu.z, (int)rn.z, (int)sf.z, pc_fast, g.rq) << 8 |
-                                    requant_channel((int32_t)r[4 * q + 3], (int)mu.w, (int)rn.w, (int)sf.w, pc_fast, g.rq) << 12;
-                                if (q & 1) o[q >> 1] |= h << 16; else o[q >> 1] = h;
-                            }
+                            for (int q = 0; q < 4; ++q)
+                                o[q] = requant8_channels<true>(r + 8 * q, g.rq, pc_s + 4 * BN, BN, ch * 32 + 8 * q,
+                                                               pc_fast != 0, hml2) + lofill;
                         } else {
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {

@@ -9,6 +9,7 @@
 // packed two per byte.  One pass over the int32 matrix: bound by HBM (4 bytes read and half
 // a byte written per value).
 #include "q4_common.cuh"
+#include "q4_requant8.cuh"
 
 namespace q4 {
 
@@ -42,9 +43,11 @@ requant_channels_vec_kernel(const ChannelParams p)
     const int j = blockIdx.x * blockDim.x + threadIdx.x;      // output word within a row
     if (j >= p.N / 8) return;
     int zb[8], bias[8], mult[8], sh[8], rnd[8];
-    // 32-bit form of the rounding shift (see requant() in q4_common.cuh) with the output zero
-    // point folded into the rounding constant: ((hi + 2^(s-1) + zo * 2^s) >> s), s = shift - 1;
-    // it needs 2 <= shift <= 27 so that the sum stays inside 32 bits
+    // 32-bit form of the rounding shift (see requant() in q4_common.cuh) with zo - lo folded
+    // into the rounding constant: ((hi + 2^(s-1) + (zo - lo) * 2^s) >> s), s = shift - 1, is
+    // already value - lo before the clamp; it needs 2 <= shift <= 27 so that the sum stays inside
+    // 32 bits.  Channels i and i + 4 are then packed with saturation into the halves of one
+    // register, clamped together, and three multiply-adds gather the four pairs (requant8()).
     bool fast = true;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
@@ -55,9 +58,10 @@ requant_channels_vec_kernel(const ChannelParams p)
         sh[e] = p.shift[n];
         fast = fast && sh[e] >= 2 && sh[e] <= 27;
         const int s = fast ? sh[e] - 1 : 1;
-        rnd[e] = (1 << (s - 1)) + (p.zo << s);
+        rnd[e] = (1 << (s - 1)) + (p.zo - p.lo) * (1 << s);
     }
     const int kza = p.K * p.za;
+    const uint32_t hml2 = (uint32_t)(p.hi - p.lo) * 0x00010001u, lofill = (uint32_t)p.lo * 0x11111111u;
     // rows per step whose loads are issued before any is used: one (two and four were
     // measured slower: the registers they take cost more occupancy than the loads gain)
     constexpr int RB = 1;
@@ -81,13 +85,16 @@ requant_channels_vec_kernel(const ChannelParams p)
             const int c[8] = {c0[u].x, c0[u].y, c0[u].z, c0[u].w, c1[u].x, c1[u].y, c1[u].z, c1[u].w};
             uint32_t word = 0;
             if (fast) {
+                int q[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac[u]) + (uint32_t)bias[e]);
-                    int q = (__mulhi(acc, mult[e]) + rnd[e]) >> (sh[e] - 1);
-                    q = min(max(q, p.lo), p.hi);
-                    word |= (uint32_t)q << (4 * e);
+                    q[e] = mulhi_add(acc, mult[e], rnd[e]) >> (sh[e] - 1);
                 }
+                uint32_t pr[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) pr[i] = __vimin_s16x2_relu(pack_sat16(q[i + 4], q[i]), hml2);
+                word = mad_u32(pr[3], 1u << 12, mad_u32(pr[2], 1u << 8, mad_u32(pr[1], 1u << 4, pr[0]))) + lofill;
             } else {
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
