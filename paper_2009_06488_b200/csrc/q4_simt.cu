@@ -191,6 +191,11 @@ __global__ void __launch_bounds__(256) operand_sums_kernel(const uint8_t* __rest
                                                            int rows_b, int32_t* __restrict__ sums_b,
                                                            int K, int vec)
 {
+    // Launched with programmatic stream serialization (its launch overlaps the previous kernel's
+    // tail): nothing is read before that kernel has completed; the kernel after this one -- the
+    // GEMM, which waits in the same way -- may begin its prologue at once.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x % 32;
     const int kbytes = (K + 1) / 2;
     const int total = rows_a + rows_b;
@@ -238,9 +243,19 @@ cudaError_t launch_operand_sums(const uint8_t* A, int64_t lda, int32_t rows_a, i
     const int vec = ((rows_a == 0 || ((uintptr_t)A % 16 == 0 && lda % 16 == 0)) &&
                      (rows_b == 0 || ((uintptr_t)B % 16 == 0 && ldb % 16 == 0))) ? 1 : 0;
     int blocks = (total + 7) / 8 < 148 * 16 ? (total + 7) / 8 : 148 * 16;
-    operand_sums_kernel<<<blocks, 256, 0, st>>>(A, lda, rows_a, sums_a, B, ldb, rows_b, sums_b, K, vec);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)blocks);
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, operand_sums_kernel, A, (int64_t)lda, (int)rows_a, sums_a, B,
+                                             (int64_t)ldb, (int)rows_b, sums_b, (int)K, vec);
     count_launch();
-    return cudaGetLastError();
+    return e;
 }
 
 // Weight-side preparation for the large-GEMM kernel, once per call ("its quantized
