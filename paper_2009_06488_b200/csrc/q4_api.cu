@@ -125,10 +125,12 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
             log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "CTA-pair tcgen05 kernel, Bt expanded once per call");
             return launch_gemm_tc_pair(p, rq, st, b8, ld8, forced_pair_width());
         }
-        // The sums pre-pass is a launch of its own (about 3 us); below about 1e11 operations the
-        // kernel takes the sums itself sooner (2048^3: 13.6 against 16.1 us), above it the
-        // pre-pass wins (4096^3: 58.5 against 62.2 us, 8192^3: 306 against 323 us).
-        const bool prepass_pays = 2.0 * p.M * p.N * p.K >= 1e11;
+        // The sums pre-pass is a launch of its own (about 3 us plus its pass over the operands).
+        // Row sums alone the kernel takes as cheaply itself (they stay inside a CTA: 4096^3 51.7
+        // against 54.4 us with the pre-pass, 8192^3 306 against 305 us); column sums need an
+        // exchange between the CTAs of a pair, and from about 1e11 operations the pre-pass is
+        // cheaper than that (8192^3: 305 against 320 us); below, the kernel takes both.
+        const bool prepass_pays = !p.colsum_b && 2.0 * p.M * p.N * p.K >= 1e11;
         if ((!p.rowsum_a || !p.colsum_b) && ws_ok && ws_bytes >= sums_bytes && prepass_pays) {
             const bool do_a = !p.rowsum_a, do_b = !p.colsum_b;
             if (launch_operand_sums(p.A, p.lda, do_a ? p.M : 0, wa, p.Bt, p.ldb, do_b ? p.N : 0, wb,

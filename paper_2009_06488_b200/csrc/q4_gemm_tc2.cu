@@ -204,7 +204,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull(a), 1);
-            mbar_init(bar_sums(a), 2 * UW);      // one arrive per unpack warp of each CTA
+            // one arrive per unpack warp: of both CTAs where column sums are exchanged, else of this one
+            mbar_init(bar_sums(a), need_cb ? 2 * UW : UW);
             mbar_init(bar_tstart(a), 1);
         }
         for (int a = 0; a < 3; ++a) {
@@ -561,8 +562,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive_cluster(map_to_cta(bar_sums(acc), rank));
-                    mbar_arrive_cluster(map_to_cta(bar_sums(acc), peer));
+                    if (need_cb) {
+                        mbar_arrive_cluster(map_to_cta(bar_sums(acc), rank));
+                        mbar_arrive_cluster(map_to_cta(bar_sums(acc), peer));
+                    } else {
+                        mbar_arrive(bar_sums(acc));       // row sums stay in this CTA
+                    }
                 }
             }
         }
@@ -578,7 +583,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t aph = (lt / NACC) & 1u;
             const int m = tm * 256 + (int)rank * TMC + row;
             const int n0 = tn * BNC;
-            if (need_sums) mbar_wait_cl(bar_sums(acc), aph, abort_flag, g.status);
+            if (need_cb) mbar_wait_cl(bar_sums(acc), aph, abort_flag, g.status);      // the peer's stores are read below
+            else if (need_ra) mbar_wait(bar_sums(acc), aph, abort_flag, g.status);
             const uint32_t s0 = sums_s + 4 * (acc * G * SUMS_N);
             for (int j = et; j < BNC; j += 128) {
                 const int n = n0 + j;
@@ -626,10 +632,27 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const int ch = ROT ? ((ci + BNC / 64) & (BNC / 32 - 1)) : ci;
                 const int nc = n0 + ch * 32;
                 const uint32_t tcol = (ROT && ch < BNC / 64 && (lt & 1u)) ? 256u + (uint32_t)(ch * 32) : (uint32_t)(ch * 32);
+                if (ROT && ci == BNC / 64 - 1) {
+                    // Last chunk of the upper half.  The whole tile must be seen complete before
+                    // the middle buffer is handed back: once it is, the next tile may complete too
+                    // (a short depth), and a wait for this tile's parity would then miss it.  The
+                    // tile's last MMAs ended long ago (they ran while the first chunks were drained).
+                    mbar_wait(bar_tfull(0), aph, abort_flag, g.status);
+                    tc_fence_after();
+                    if (nc >= g.N) {       // a chunk past the last column: nothing to read
+                        tc_fence_before();
+                        mbar_arrive(bar_tempty(2));
+                    }
+                }
                 if (nc < g.N) {            // warp-uniform
                 uint32_t r[32];
                 tc_ld32(taddr0 + tcol, r);
                 tc_wait_ld();
+                if (ROT && ci == BNC / 64 - 1) {
+                    // the middle buffer is in registers: the next tile's upper-half MMAs may start
+                    tc_fence_before();
+                    mbar_arrive(bar_tempty(2));
+                }
                 if (pc) {
                     // the column's own zero point in Eq. 2's row-sum term
 #pragma unroll
@@ -715,13 +738,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         }
                     }
                 }
-                }
-                if (ROT && ci == BNC / 64 - 1) {
-                    // the middle buffer is drained: the next tile's upper-half MMAs may start
-                    tc_fence_before();
-                    mbar_arrive(bar_tempty(2));
-                    mbar_wait(bar_tfull(0), aph, abort_flag, g.status);
-                    tc_fence_after();
                 }
             }
             tc_fence_before();
