@@ -736,7 +736,7 @@ def run_ours(args):
 
     roofline = {"bound": "tensor", "achieved": gemm_tops, "peak": int8_peak, "unit": "TOP/s",
                 "frac": gemm_tops / int8_peak, "traffic": DOMINANT_KERNEL_TRAFFIC_BYTES,
-                "kernel": "gemm_tc_pair_kernel<256,1,false,false> (q4_gemm 8192^3, int32 output)",
+                "kernel": "gemm_tc_pair_kernel<256,1,false> (q4_gemm 8192^3, int32 output)",
                 "peak_source": f"2 x {peaks['source']} bf16 {'sustained' if sustained else 'burst'} "
                                f"({peaks['bf16_sustained'] if sustained else peaks['bf16']} TFLOP/s): the kernel is "
                                f"timed inside a region of {total_ms / 1e3:.2f} s; nominal int8:bf16 ratio 2",

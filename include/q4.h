@@ -105,10 +105,6 @@ typedef struct {
  * 16-byte aligned.  With it, large problems take the sums that were not supplied in
  * one bandwidth-bound pass over the operands instead of inside the GEMM kernel, which
  * is faster; without it (NULL) the result is the same.  Its contents are scratch.
- * A workspace of q4_gemm_workspace_bytes_expanded(M, N, K) bytes additionally lets a
- * large problem prepare the weights once per call (Bt expanded to one byte per value,
- * loaded by TMA straight into the MMA's operand ring; Section II-B: what depends only on
- * the weights is computed once).  Same results; at present not faster than the default.
  */
 q4_status q4_gemm(const uint8_t* A, int64_t lda, const uint8_t* Bt, int64_t ldb,
                   int32_t* C, int64_t ldc, int32_t M, int32_t N, int32_t K,
@@ -231,7 +227,6 @@ q4_status q4_conv2d_static(const uint8_t* X, const uint8_t* Wt, int64_t ldw,
                            uint8_t* Y, void* stream);
 
 size_t q4_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K);
-size_t q4_gemm_workspace_bytes_expanded(int32_t M, int32_t N, int32_t K);
 size_t q4_conv2d_workspace_bytes(const q4_conv_desc* d);
 
 /*

@@ -31,7 +31,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 Q4_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = ["q4_gemm", "q4_gemm_requant", "q4_im2col", "q4_conv2d", "q4_conv2d_static",
-           "q4_gemm_workspace_bytes", "q4_gemm_workspace_bytes_expanded",
+           "q4_gemm_workspace_bytes",
            "q4_conv2d_workspace_bytes", "q4_pack_bt", "q4_row_sums", "q4_gemm_host",
            "q4_gemm_host_staging_bytes", "q4_last_device_status", "q4_set_variant",
            "q4_launch_count", "q4_status_string", "q4_version", "q4_measure_mma_peak",
@@ -119,8 +119,6 @@ _lib.q4_conv2d_prepare_weights.argtypes = [_vp, _i64, _vp, _vp, ctypes.POINTER(_
 _lib.q4_conv2d_prepared.argtypes = [_vp, _vp, _sz, ctypes.POINTER(_ConvDesc), _i32, ctypes.POINTER(_Requant), _vp, _vp]
 _lib.q4_gemm_workspace_bytes.argtypes = [_i32, _i32, _i32]
 _lib.q4_gemm_workspace_bytes.restype = _sz
-_lib.q4_gemm_workspace_bytes_expanded.argtypes = [_i32, _i32, _i32]
-_lib.q4_gemm_workspace_bytes_expanded.restype = _sz
 _lib.q4_conv2d_workspace_bytes.argtypes = [ctypes.POINTER(_ConvDesc)]
 _lib.q4_conv2d_workspace_bytes.restype = _sz
 _lib.q4_pack_bt.argtypes = [_vp, _i64, _vp, _i64, _i32, _i32, _vp]
@@ -220,8 +218,6 @@ def q4_gemm_workspace_bytes(M: int, N: int, K: int) -> int:
     return int(_lib.q4_gemm_workspace_bytes(M, N, K))
 
 
-def q4_gemm_workspace_bytes_expanded(M: int, N: int, K: int) -> int:
-    return int(_lib.q4_gemm_workspace_bytes_expanded(M, N, K))
 
 
 def q4_conv2d_workspace_bytes(d: ConvDesc) -> int:

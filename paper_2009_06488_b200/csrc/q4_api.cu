@@ -100,31 +100,15 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
     // always takes the pair kernel where it applies.
     const long long pair_tiles = ((long long)p.M + 255) / 256 * (((long long)p.N + 255) / 256);
     if (v != 1 && v != 3 && gemm_tc_pair_supported(p) && (v == 2 || pair_tiles >= 32)) {
-        // Large problems use the workspace, if given, for work that is better done once per
-        // call than once per output tile: the depth sums, and -- with the full size -- the
-        // expansion of Bt to bytes.  A smaller workspace still takes the sums; without one
-        // the kernel does everything itself.  The results are identical.
-        // Layout of the workspace: [row sums of A][column sums of Bt][Bt expanded to bytes].
+        // Large problems use the workspace, if given, for the depth sums where one pass over
+        // an operand is cheaper than every output tile taking them again; without one the
+        // kernel does everything itself.  The results are identical.
+        // Layout of the workspace: [row sums of A][column sums of Bt].
         const size_t sums_bytes = round256(4 * (size_t)p.M) + round256(4 * (size_t)p.N);
-        const int64_t ld8 = ((int64_t)p.K + 127) / 128 * 128;
-        const size_t full_bytes = sums_bytes + (size_t)p.N * (size_t)ld8;
         const bool ws_ok = ws && (uintptr_t)ws % 16 == 0;
         int32_t* wa = static_cast<int32_t*>(ws);
         int32_t* wb = ws ? reinterpret_cast<int32_t*>(static_cast<uint8_t*>(ws) + round256(4 * (size_t)p.M))
                          : nullptr;
-        if (ws_ok && ws_bytes >= full_bytes) {
-            // weights prepared once per call: expanded Bt + its column sums; row sums of A
-            uint8_t* b8 = static_cast<uint8_t*>(ws) + sums_bytes;
-            if (launch_bt_expand(p.Bt, p.ldb, p.N, p.K, b8, ld8, wb, st) != cudaSuccess) return Q4_ERR_CUDA;
-            if (!p.colsum_b) p.colsum_b = wb;
-            if (!p.rowsum_a) {
-                if (launch_operand_sums(p.A, p.lda, p.M, wa, p.Bt, p.ldb, 0, wb, p.K, st) != cudaSuccess)
-                    return Q4_ERR_CUDA;
-                p.rowsum_a = wa;
-            }
-            log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "CTA-pair tcgen05 kernel, Bt expanded once per call");
-            return launch_gemm_tc_pair(p, rq, st, b8, ld8, forced_pair_width());
-        }
         // The sums pre-pass is a launch of its own (about 3 us plus its pass over the operands).
         // Row sums alone the kernel takes as cheaply itself (they stay inside a CTA: 4096^3 51.7
         // against 54.4 us with the pre-pass, 8192^3 306 against 305 us); column sums need an
@@ -139,7 +123,7 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
             if (do_b) p.colsum_b = wb;
         }
         log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "CTA-pair tcgen05 kernel");
-        return launch_gemm_tc_pair(p, rq, st, nullptr, 0, forced_pair_width());
+        return launch_gemm_tc_pair(p, rq, st, forced_pair_width());
     }
     if (v != 1 && gemm_tc_supported(p)) {
         log_choice(rq ? "q4_gemm_requant" : "q4_gemm", "single-CTA tcgen05 kernel");
@@ -290,14 +274,6 @@ size_t q4_gemm_workspace_bytes(int32_t M, int32_t N, int32_t K)
     (void)K;
     if (M < 0 || N < 0) return 0;
     return round256(4 * (size_t)M) + round256(4 * (size_t)N);   // depth sums of both operands
-}
-
-size_t q4_gemm_workspace_bytes_expanded(int32_t M, int32_t N, int32_t K)
-{
-    if (M < 0 || N < 0 || K < 1) return 0;
-    // depth sums of both operands + Bt expanded to one byte per value
-    return round256(4 * (size_t)M) + round256(4 * (size_t)N) +
-           (size_t)N * (size_t)(((int64_t)K + 127) / 128 * 128);
 }
 
 size_t q4_conv2d_workspace_bytes(const q4_conv_desc* d)

@@ -118,10 +118,7 @@ bool        gemm_tc_supported(const GemmParams& p);
 q4_status   launch_gemm_tc(const GemmParams& p, bool requant, cudaStream_t st);
 bool        gemm_tc_pair_supported(const GemmParams& p);
 // width: 192 or 256 columns per tile, 0 = chosen from the problem's shape
-q4_status   launch_gemm_tc_pair(const GemmParams& p, bool requant, cudaStream_t st,
-                                const uint8_t* b8 = nullptr, int64_t ld8 = 0, int width = 0);
-cudaError_t launch_bt_expand(const uint8_t* Bt, int64_t ldb, int32_t N, int32_t K, uint8_t* b8,
-                             int64_t ld8, int32_t* colsum, cudaStream_t st);
+q4_status   launch_gemm_tc_pair(const GemmParams& p, bool requant, cudaStream_t st, int width = 0);
 cudaError_t launch_pack_bt(const uint8_t* B_kn, int64_t ldb_kn, uint8_t* Bt, int64_t ldb,
                            int32_t K, int32_t N, cudaStream_t st);
 cudaError_t launch_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,

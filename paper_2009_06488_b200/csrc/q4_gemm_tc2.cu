@@ -105,7 +105,7 @@ struct Cfg {
     static constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
     static constexpr int OFF_PC = OFF_COLTERM + BNC * 4;       // per-channel: int32 [4][BNC] zero point, multiplier, rounding, shift
     static constexpr int OFF_BAR = OFF_PC + 4 * BNC * 4;
-    static constexpr int NBAR = 2 * PS + 2 * US + 2 * BS + 12;
+    static constexpr int NBAR = 2 * PS + 2 * US + BS + 12;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM = OFF_MISC + 16 + 1024;
 
@@ -142,10 +142,7 @@ __device__ __forceinline__ int chunk_sum(const uint4& lo, const uint4& hi, int a
     return dp4a_u8(t, 0x01010101u, acc);
 }
 
-// BPRE: Bt arrives already expanded to one byte per value (by bt_expand_kernel, once per
-// call, in the same depth order the unpack gives A) and is loaded by TMA straight into
-// the swizzled operand ring; the unpack warps then handle A only.
-template <int BNC, int NSTG, bool REQUANT, bool BPRE>
+template <int BNC, int NSTG, bool REQUANT>
 __global__ void __launch_bounds__(NTHREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmC, const Params p)
@@ -170,8 +167,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     auto bar_empty_p   = [&](int s) { return bar0 + 8u * (uint32_t)(PS + s); };
     auto bar_full_u    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + s); };
     auto bar_empty_b   = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + s); };
-    auto bar_full_b    = [&](int s) { return bar0 + 8u * (uint32_t)(2 * PS + 2 * US + BS + s); };
-    const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US + 2 * BS);
+    const uint32_t barT = bar0 + 8u * (uint32_t)(2 * PS + 2 * US + BS);
     // accumulator buffers: two whole ones, or (ROT) 0 / 1 = the outer half-buffers of even /
     // odd tiles, 2 = the middle one
     auto bar_tfull       = [&](int a) { return barT + 8u * (uint32_t)a; };
@@ -198,10 +194,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         for (int s = 0; s < US; ++s)
             mbar_init(bar_full_u(s), 2 * WPG);   // used in the leader: a group's warps of both CTAs
-        for (int s = 0; s < BS; ++s) {
+        for (int s = 0; s < BS; ++s)
             mbar_init(bar_empty_b(s), 1);
-            mbar_init(bar_full_b(s), 1);         // BPRE: the TMA load of an expanded Bt stage
-        }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull(a), 1);
             // one arrive per unpack warp: of both CTAs where column sums are exchanged, else of this one
@@ -255,20 +249,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const int st = it % PS;
                     const uint32_t ph = (it / PS) & 1u;
                     mbar_wait(bar_empty_p(st), ph ^ 1u, abort_flag, g.status);
-                    mbar_expect_tx(bar_full_p(st), (uint32_t)(BPRE ? PA : PSTAGE));
+                    mbar_expect_tx(bar_full_p(st), (uint32_t)PSTAGE);
                     const uint32_t dst = sbase + OFF_P + st * PSTAGE;
                     tma_load_2d(dst, &tmA, s * PROW, arow, bar_full_p(st));
-                    if (!BPRE) {
-                        tma_load_2d(dst + PA, &tmB, s * PROW, brow, bar_full_p(st));
-                        if (ROT) tma_load_2d(dst + PA + C::BBOX * PROW, &tmB, s * PROW, brow + BH, bar_full_p(st));
-                    } else {
-                        const int bst = it % BS;
-                        mbar_wait(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
-                        mbar_expect_tx(bar_full_b(bst), (uint32_t)BSTAGE);
-                        tma_load_2d(sbase + OFF_B + bst * BSTAGE, &tmB, s * UROW, brow, bar_full_b(bst));
-                        if (ROT) tma_load_2d(sbase + OFF_B + bst * BSTAGE + C::BBOX * UROW, &tmB, s * UROW, brow + BH,
-                                             bar_full_b(bst));
-                    }
+                    tma_load_2d(dst + PA, &tmB, s * PROW, brow, bar_full_p(st));
+                    if (ROT) tma_load_2d(dst + PA + C::BBOX * PROW, &tmB, s * PROW, brow + BH, bar_full_p(st));
                 }
             }
         }
@@ -479,10 +464,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 wa[c] = lds128(ps + a_ld[c]);
 #pragma unroll
             for (int j = 0; j < NTB; ++j)
-                if (!BPRE) wb[j] = lds128(ps + b_ld[j]);
-            // Bt first: its shared-memory ring is twice as deep as the tensor-memory ring
-            // of A, so this wait is normally over and the work hides behind the MMAs
-            if (!BPRE) {
+                wb[j] = lds128(ps + b_ld[j]);
+            // Bt first: with 192 columns its shared-memory ring is twice as deep as the
+            // tensor-memory ring of A, so this wait is normally over and the work hides behind
+            // the MMAs
+            {
                 const int bst = (int)(it % BS);
                 mbar_wait(bar_empty_b(bst), ((it / BS) & 1u) ^ 1u, abort_flag, g.status);
                 const uint32_t us = sbase + OFF_B + bst * BSTAGE;
@@ -513,8 +499,6 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                         ahi[c].x, ahi[c].y, ahi[c].z, ahi[c].w};
                 tc_st8(a_taddr + (uint32_t)(ust * 32 + 8 * c), r8);
             }
-            // BPRE: my CTA's expanded Bt stage has landed (the leader learns it through my arrive)
-            if (BPRE) mbar_wait(bar_full_b(it % BS), (it / BS) & 1u, abort_flag, g.status);
             tc_wait_st();                 // my tensor-memory stores are complete
             fence_async_smem();           // my shared-memory stores are visible to the MMA
             tc_fence_before();
@@ -544,7 +528,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const uint32_t mine = sums_s + 4 * ((acc * G + grp) * SUMS_N);
                 sts32(mine + 4 * arow, psum_a);
 #pragma unroll
-                for (int j = 0; j < (BPRE ? 0 : NTB); ++j) {
+                for (int j = 0; j < NTB; ++j) {
                     int t = psum_b[j];
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 1);
                     t += __shfl_xor_sync(0xFFFFFFFFu, t, 2);
@@ -767,7 +751,7 @@ bool gemm_tc_pair_supported(const GemmParams& p)
     return gemm_tc_supported(p) && p.M >= 256 && p.N >= 192;
 }
 
-template <int BNC, int NSTG, bool RQ, bool BPRE>
+template <int BNC, int NSTG, bool RQ>
 static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, const CUtensorMap& tmB,
                                const CUtensorMap& tmC, long long tiles, cudaStream_t st)
 {
@@ -775,7 +759,7 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return Q4_ERR_CUDA;
     int& max_clusters = max_clusters_dev[dev];
-    auto kernel = pair::gemm_tc_pair_kernel<BNC, NSTG, RQ, BPRE>;
+    auto kernel = pair::gemm_tc_pair_kernel<BNC, NSTG, RQ>;
     constexpr int SMEM = pair::Cfg<BNC, NSTG>::SMEM;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
@@ -807,8 +791,6 @@ static q4_status launch_pair_t(const pair::Params& p, const CUtensorMap& tmA, co
     return e == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
 }
 
-// Expanded Bt [N x K8 bytes], pitch ld8: box = 128 bytes x box_rows, written with the
-// 128-byte swizzle, i.e. directly in the layout the MMA's K-major descriptor reads.
 typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                              const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                              CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -841,19 +823,6 @@ static bool make_c_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, in
               CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-static bool make_b8_map(CUtensorMap* tm, const uint8_t* base, int64_t ld8, int rows, int k8, int box_rows)
-{
-    EncodeFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)k8, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld8};
-    cuuint32_t box[2] = {(cuuint32_t)pair::UROW, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides, box,
-              estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 // The same map for other translation units.
 bool make_c32_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, int cols)
 {
@@ -877,7 +846,7 @@ int gemm_tc_pair_width(const GemmParams& g)
 }
 
 template <int BNC, int NSTG>
-static q4_status launch_pair_w(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8, int64_t ld8)
+static q4_status launch_pair_w(const GemmParams& g, bool rq, cudaStream_t st)
 {
     using C = pair::Cfg<BNC, NSTG>;
     pair::Params p;
@@ -897,26 +866,18 @@ static q4_status launch_pair_w(const GemmParams& g, bool rq, cudaStream_t st, co
         p.c_tma = 1;
     }
     const long long tiles = (long long)p.tiles_m * p.tiles_n;
-    if (b8) {
-        // expanded Bt: the kernel cannot take the column sums itself
-        if (!g.colsum_b) return Q4_ERR_INVALID_ARG;
-        if (!make_b8_map(&tmB, b8, ld8, g.N, (g.K + 31) / 32 * 32, C::BBOX)) return Q4_ERR_CUDA;
-        return rq ? launch_pair_t<BNC, NSTG, true, true>(p, tmA, tmB, tmC, tiles, st)
-                  : launch_pair_t<BNC, NSTG, false, true>(p, tmA, tmB, tmC, tiles, st);
-    }
     if (!make_packed_map(&tmB, g.Bt, g.ldb, g.N, kbytes, C::BBOX, false)) return Q4_ERR_CUDA;
-    return rq ? launch_pair_t<BNC, NSTG, true, false>(p, tmA, tmB, tmC, tiles, st)
-              : launch_pair_t<BNC, NSTG, false, false>(p, tmA, tmB, tmC, tiles, st);
+    return rq ? launch_pair_t<BNC, NSTG, true>(p, tmA, tmB, tmC, tiles, st)
+              : launch_pair_t<BNC, NSTG, false>(p, tmA, tmB, tmC, tiles, st);
 }
 
-q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, const uint8_t* b8,
-                              int64_t ld8, int width)
+q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, int width)
 {
     if (width != 192 && width != 256) width = gemm_tc_pair_width(g);
-    if (width == 192) return launch_pair_w<192, 2>(g, rq, st, b8, ld8);
+    if (width == 192) return launch_pair_w<192, 2>(g, rq, st);
     // few tiles per CTA pair: the last tile's exposed epilogue weighs more than ring depth
     const long long t256 = (((long long)g.M + 255) / 256) * (((long long)g.N + 255) / 256);
-    return t256 <= 3 * 74 ? launch_pair_w<256, 2>(g, rq, st, b8, ld8) : launch_pair_w<256, 1>(g, rq, st, b8, ld8);
+    return t256 <= 3 * 74 ? launch_pair_w<256, 2>(g, rq, st) : launch_pair_w<256, 1>(g, rq, st);
 }
 
 }  // namespace q4

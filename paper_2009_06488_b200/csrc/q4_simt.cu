@@ -258,59 +258,6 @@ cudaError_t launch_operand_sums(const uint8_t* A, int64_t lda, int32_t rows_a, i
     return e;
 }
 
-// Weight-side preparation for the large-GEMM kernel, once per call ("its quantized
-// approximation ... and sums over columns can be computed only once", Section II-B):
-// Bt is expanded to one byte per value, each 16-byte packed chunk becoming its 16 even
-// nibbles followed by its 16 odd nibbles -- the depth order the kernel's unpack gives A --
-// and the column sums of Eq. 2's third term are taken on the way.  One warp per row.
-__global__ void __launch_bounds__(256) bt_expand_kernel(const uint8_t* __restrict__ Bt, int64_t ldb,
-                                                        int N, int K, uint8_t* __restrict__ b8,
-                                                        int64_t ld8, int32_t* __restrict__ colsum,
-                                                        int vec)
-{
-    const int lane = threadIdx.x % 32;
-    const int kbytes = (K + 1) / 2;
-    const int nchunks = (K + 31) / 32;
-    for (int n = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32; n < N;
-         n += gridDim.x * (blockDim.x / 32)) {
-        const uint8_t* row = Bt + (int64_t)n * ldb;
-        uint8_t* out = b8 + (int64_t)n * ld8;
-        int s = 0;
-        for (int c = lane; c < nchunks; c += 32) {
-            uint4 w;
-            if (vec && 16 * c + 16 <= kbytes) {
-                w = *reinterpret_cast<const uint4*>(row + 16 * c);
-            } else {
-                uint32_t t[4] = {0, 0, 0, 0};
-                for (int b = 0; b < 16; ++b)
-                    if (16 * c + b < kbytes) t[b >> 2] |= (uint32_t)row[16 * c + b] << (8 * (b & 3));
-                w = make_uint4(t[0], t[1], t[2], t[3]);
-            }
-            const uint4 lo = make_uint4(w.x & 0x0F0F0F0Fu, w.y & 0x0F0F0F0Fu, w.z & 0x0F0F0F0Fu,
-                                        w.w & 0x0F0F0F0Fu);
-            const uint4 hi = make_uint4((w.x >> 4) & 0x0F0F0F0Fu, (w.y >> 4) & 0x0F0F0F0Fu,
-                                        (w.z >> 4) & 0x0F0F0F0Fu, (w.w >> 4) & 0x0F0F0F0Fu);
-            *reinterpret_cast<uint4*>(out + 32 * c) = lo;
-            *reinterpret_cast<uint4*>(out + 32 * c + 16) = hi;
-            s += nibble_sum(w.x) + nibble_sum(w.y) + nibble_sum(w.z) + nibble_sum(w.w);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
-        if (lane == 0) colsum[n] = s;
-    }
-}
-
-cudaError_t launch_bt_expand(const uint8_t* Bt, int64_t ldb, int32_t N, int32_t K, uint8_t* b8,
-                             int64_t ld8, int32_t* colsum, cudaStream_t st)
-{
-    if (N <= 0) return cudaSuccess;
-    const int vec = ((uintptr_t)Bt % 16 == 0 && ldb % 16 == 0) ? 1 : 0;
-    int blocks = (N + 7) / 8 < 148 * 16 ? (N + 7) / 8 : 148 * 16;
-    bt_expand_kernel<<<blocks, 256, 0, st>>>(Bt, ldb, N, K, b8, ld8, colsum, vec);
-    count_launch();
-    return cudaGetLastError();
-}
-
 cudaError_t launch_row_sums(const uint8_t* P, int64_t ld, int32_t rows, int32_t K,
                             int32_t* sums, cudaStream_t st)
 {

@@ -35,12 +35,13 @@ def run_gemm(q4, c, variant, ldc_pad=0, sums=False, use_ws=False):
         cb = torch.empty(c.N, dtype=torch.int32, device="cuda")
         q4.q4_row_sums(A, c.M, c.K, ra)
         q4.q4_row_sums(Bt, c.N, c.K, cb)
+        if sums == "cols":      # the weights' sums only: the kernel takes the row sums of A
+            ra = None
+        if sums == "rows":
+            cb = None
     ws = None
-    if use_ws:     # scratch (poisoned): the depth sums; "expanded" = sums + Bt expanded to bytes
-        nbytes = q4.q4_gemm_workspace_bytes(c.M, c.N, c.K)
-        if use_ws == "expanded":
-            nbytes = q4.q4_gemm_workspace_bytes_expanded(c.M, c.N, c.K)
-        ws = torch.full((nbytes,), 0xA5, dtype=torch.uint8, device="cuda")
+    if use_ws:     # scratch (poisoned): the depth sums
+        ws = torch.full((q4.q4_gemm_workspace_bytes(c.M, c.N, c.K),), 0xA5, dtype=torch.uint8, device="cuda")
     q4.q4_gemm(A, Bt, C, c.M, c.N, c.K, c.za, c.zb, ra, cb, ws)
     assert q4.q4_last_device_status() == q4.Q4_OK
     out = C.cpu().numpy()
@@ -56,8 +57,7 @@ def run_requant(q4, c, variant, rq, bias=None, ld_pad=0, use_ws=False):
     Cq = torch.full((c.M, c.N // 2 + ld_pad), 0xA5, dtype=torch.uint8, device="cuda")
     ws = None
     if use_ws:
-        ws = torch.full((q4.q4_gemm_workspace_bytes_expanded(c.M, c.N, c.K) if use_ws == "expanded" else
-                         q4.q4_gemm_workspace_bytes(c.M, c.N, c.K),), 0xA5, dtype=torch.uint8, device="cuda")
+        ws = torch.full((q4.q4_gemm_workspace_bytes(c.M, c.N, c.K),), 0xA5, dtype=torch.uint8, device="cuda")
     q4.q4_gemm_requant(A, Bt, Cq, c.M, c.N, c.K, c.za, c.zb,
                        q4.Requant(rq.mult, rq.shift, rq.zo, rq.clamp_lo, rq.clamp_hi),
                        None if bias is None else dev(bias), ws=ws)
@@ -121,16 +121,15 @@ def test_pair_and_single_tensor_core_kernels_agree_with_oracle(q4, variant, shap
     assert (got == want).all()
     got, _, _ = run_gemm(q4, c, variant, use_ws=True)     # sums taken by the pre-pass
     assert (got == want).all()
-    got, _, _ = run_gemm(q4, c, variant, use_ws="expanded")   # Bt expanded once per call as well
+    got, _, _ = run_gemm(q4, c, variant, sums="cols", use_ws=True)    # row sums of A inside the kernel
     assert (got == want).all()
-    got, _, _ = run_gemm(q4, c, variant, sums=True, use_ws="expanded")
+    got, _, _ = run_gemm(q4, c, variant, sums="rows")                 # column sums of Bt inside the kernel
     assert (got == want).all()
     rq = oracle.Requant(c.mult, 6, 4, 4, 15)
     wantq = oracle.requant_matrix(want, c.bias, rq)
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=16) == wantq).all()
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=3) == wantq).all()   # byte stores
     assert (run_requant(q4, c, variant, rq, c.bias, use_ws=True) == wantq).all()
-    assert (run_requant(q4, c, variant, rq, c.bias, use_ws="expanded") == wantq).all()
 
 
 # Both tile widths of the CTA-pair kernel on the same problems: column tails that leave the
@@ -150,7 +149,9 @@ def test_pair_kernel_tile_widths_agree_with_oracle(q4, variant, shape):
     assert (got == want).all()
     got, _, _ = run_gemm(q4, c, variant, sums=True)
     assert (got == want).all()
-    got, _, _ = run_gemm(q4, c, variant, use_ws="expanded")   # Bt expanded once per call
+    got, _, _ = run_gemm(q4, c, variant, sums="cols")         # row sums alone: they stay inside a CTA
+    assert (got == want).all()
+    got, _, _ = run_gemm(q4, c, variant, sums="rows", use_ws=True)
     assert (got == want).all()
     got, _, _ = run_gemm(q4, c, variant, ldc_pad=1)           # unaligned int32 pitch: scalar stores
     assert (got == want).all()
@@ -158,7 +159,7 @@ def test_pair_kernel_tile_widths_agree_with_oracle(q4, variant, shape):
     wantq = oracle.requant_matrix(want, c.bias, rq)
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=16) == wantq).all()
     assert (run_requant(q4, c, variant, rq, c.bias, ld_pad=3) == wantq).all()
-    assert (run_requant(q4, c, variant, rq, c.bias, use_ws="expanded") == wantq).all()
+    assert (run_requant(q4, c, variant, rq, c.bias, use_ws=True) == wantq).all()
 
 
 @pytest.mark.parametrize("variant", [SIMT, TC])
