@@ -35,23 +35,27 @@ __device__ __forceinline__ uint32_t requant_one(int32_t acc, int32_t mult, int32
     return (uint32_t)min(max(q, lo), hi);
 }
 
-// Eight consecutive channels (one 32-bit word of output) per thread; a thread keeps its
-// channels' parameters in registers and walks rows blockIdx.y, blockIdx.y + gridDim.y, ...
-__global__ void __launch_bounds__(256)
+// Four consecutive channels and two rows per thread.  A thread keeps its channels' parameters
+// in registers (40 registers in all: 1536 threads are resident per SM, each with two 16-byte
+// loads in flight; eight channels per thread took 64 registers and reached 0.69 of the copy
+// bandwidth where this form reaches 0.80) and walks the row pairs blockIdx.y,
+// blockIdx.y + gridDim.y, ...  The two rows' values of a channel share a packed pair, so the
+// gathered word holds row r's four nibbles in its low half and row r + 1's in its high half.
+__global__ void __launch_bounds__(256, 6)
 requant_channels_vec_kernel(const ChannelParams p)
 {
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;      // output word within a row
-    if (j >= p.N / 8) return;
-    int zb[8], bias[8], mult[8], sh[8], rnd[8];
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;      // group of four channels
+    if (j >= p.N / 4) return;
+    int zb[4], bias[4], mult[4], sh[4], rnd[4];
     // 32-bit form of the rounding shift (see requant() in q4_common.cuh) with zo - lo folded
     // into the rounding constant: ((hi + 2^(s-1) + (zo - lo) * 2^s) >> s), s = shift - 1, is
     // already value - lo before the clamp; it needs 2 <= shift <= 27 so that the sum stays inside
-    // 32 bits.  Channels i and i + 4 are then packed with saturation into the halves of one
-    // register, clamped together, and three multiply-adds gather the four pairs (requant8()).
+    // 32 bits.  Two values are then packed with saturation into the halves of one register,
+    // clamped together, and three multiply-adds gather the four pairs.
     bool fast = true;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) {
-        const int n = 8 * j + e;
+    for (int e = 0; e < 4; ++e) {
+        const int n = 4 * j + e;
         zb[e] = p.zb ? p.zb[n] : 0;
         bias[e] = p.bias ? p.bias[n] : 0;
         mult[e] = p.mult[n];
@@ -62,48 +66,36 @@ requant_channels_vec_kernel(const ChannelParams p)
     }
     const int kza = p.K * p.za;
     const uint32_t hml2 = (uint32_t)(p.hi - p.lo) * 0x00010001u, lofill = (uint32_t)p.lo * 0x11111111u;
-    // rows per step whose loads are issued before any is used: one (two and four were
-    // measured slower: the registers they take cost more occupancy than the loads gain)
-    constexpr int RB = 1;
-    for (int r0 = blockIdx.y; r0 < p.M; r0 += RB * gridDim.y) {
-        int4 c0[RB], c1[RB];
-        int rowfac[RB];
+    for (int r = 2 * blockIdx.y; r < p.M; r += 2 * gridDim.y) {
+        const bool two = r + 1 < p.M;
+        const int r1 = two ? r + 1 : r;
+        const int4 c0 = __ldcs(reinterpret_cast<const int4*>(p.C0 + (int64_t)r * p.ldc + 4 * j));
+        const int4 c1 = __ldcs(reinterpret_cast<const int4*>(p.C0 + (int64_t)r1 * p.ldc + 4 * j));
+        const int f0 = p.rowsum_a[r] - kza, f1 = p.rowsum_a[r1] - kza;       // sum_k (a - za)
+        const int a[4] = {c0.x, c0.y, c0.z, c0.w}, b[4] = {c1.x, c1.y, c1.z, c1.w};
+        uint32_t word = 0;
+        if (fast) {
+            uint32_t pr[4];
 #pragma unroll
-        for (int u = 0; u < RB; ++u) {
-            const int r = r0 + u * gridDim.y;
-            if (r < p.M) {
-                const int4* src = reinterpret_cast<const int4*>(p.C0 + (int64_t)r * p.ldc + 8 * j);
-                c0[u] = __ldcs(src);
-                c1[u] = __ldcs(src + 1);
-                rowfac[u] = p.rowsum_a[r] - kza;              // sum_k (a - za)
+            for (int e = 0; e < 4; ++e) {
+                const int acc0 = (int)((uint32_t)a[e] - (uint32_t)(zb[e] * f0) + (uint32_t)bias[e]);
+                const int acc1 = (int)((uint32_t)b[e] - (uint32_t)(zb[e] * f1) + (uint32_t)bias[e]);
+                const int q0 = mulhi_add(acc0, mult[e], rnd[e]) >> (sh[e] - 1);
+                const int q1 = mulhi_add(acc1, mult[e], rnd[e]) >> (sh[e] - 1);
+                pr[e] = __vimin_s16x2_relu(pack_sat16(q1, q0), hml2);
+            }
+            word = mad_u32(pr[3], 1u << 12, mad_u32(pr[2], 1u << 8, mad_u32(pr[1], 1u << 4, pr[0]))) + lofill;
+        } else {
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int acc0 = (int)((uint32_t)a[e] - (uint32_t)(zb[e] * f0) + (uint32_t)bias[e]);
+                const int acc1 = (int)((uint32_t)b[e] - (uint32_t)(zb[e] * f1) + (uint32_t)bias[e]);
+                word |= requant_one(acc0, mult[e], sh[e], p.zo, p.lo, p.hi) << (4 * e);
+                word |= requant_one(acc1, mult[e], sh[e], p.zo, p.lo, p.hi) << (16 + 4 * e);
             }
         }
-#pragma unroll
-        for (int u = 0; u < RB; ++u) {
-            const int r = r0 + u * gridDim.y;
-            if (r >= p.M) break;
-            const int c[8] = {c0[u].x, c0[u].y, c0[u].z, c0[u].w, c1[u].x, c1[u].y, c1[u].z, c1[u].w};
-            uint32_t word = 0;
-            if (fast) {
-                int q[8];
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac[u]) + (uint32_t)bias[e]);
-                    q[e] = mulhi_add(acc, mult[e], rnd[e]) >> (sh[e] - 1);
-                }
-                uint32_t pr[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) pr[i] = __vimin_s16x2_relu(pack_sat16(q[i + 4], q[i]), hml2);
-                word = mad_u32(pr[3], 1u << 12, mad_u32(pr[2], 1u << 8, mad_u32(pr[1], 1u << 4, pr[0]))) + lofill;
-            } else {
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const int acc = (int)((uint32_t)c[e] - (uint32_t)(zb[e] * rowfac[u]) + (uint32_t)bias[e]);
-                    word |= requant_one(acc, mult[e], sh[e], p.zo, p.lo, p.hi) << (4 * e);
-                }
-            }
-            *reinterpret_cast<uint32_t*>(p.Cq + (int64_t)r * p.ldcq + 4 * j) = word;
-        }
+        *reinterpret_cast<uint16_t*>(p.Cq + (int64_t)r * p.ldcq + 2 * j) = (uint16_t)word;
+        if (two) *reinterpret_cast<uint16_t*>(p.Cq + (int64_t)r1 * p.ldcq + 2 * j) = (uint16_t)(word >> 16);
     }
 }
 
@@ -138,15 +130,17 @@ cudaError_t launch_requant_channels(const int32_t* C0, int64_t ldc, int32_t M, i
                                     cudaStream_t st)
 {
     ChannelParams p{C0, ldc, M, N, K, za, rowsum_a, zb, bias, mult, shift, zo, lo, hi, Cq, ldcq};
-    const bool vec = N % 8 == 0 && ldc % 4 == 0 && (uintptr_t)C0 % 16 == 0 && ldcq % 4 == 0 &&
-                     (uintptr_t)Cq % 4 == 0;
+    const bool vec = N % 4 == 0 && ldc % 4 == 0 && (uintptr_t)C0 % 16 == 0 && ldcq % 2 == 0 &&
+                     (uintptr_t)Cq % 2 == 0;
     if (vec) {
-        const int words = N / 8;
-        const int bx = words < 256 ? (words + 31) / 32 * 32 : 256;
-        const unsigned gx = (unsigned)((words + bx - 1) / bx);
-        int64_t gy = (int64_t)148 * 16 / gx;
+        // one resident wave: six blocks of 256 threads per SM (more blocks than are resident
+        // at once measured slower: 148 x 8 blocks 71 us against 57 us at 8192 x 8192)
+        const int groups = N / 4;
+        const int bx = groups < 256 ? (groups + 31) / 32 * 32 : 256;
+        const unsigned gx = (unsigned)((groups + bx - 1) / bx);
+        int64_t gy = (int64_t)148 * 6 / gx;
         if (gy < 1) gy = 1;
-        if (gy > M) gy = M;
+        if (gy > ((int64_t)M + 1) / 2) gy = ((int64_t)M + 1) / 2;
         if (gy > 65535) gy = 65535;
         requant_channels_vec_kernel<<<dim3(gx, (unsigned)gy), bx, 0, st>>>(p);
     } else {

@@ -45,7 +45,7 @@ def run(q4, A, Bt, M, N, K, za, zb, bias, mult, shift, zo, lo, hi, ldc_pad=0, ld
 
 
 SHAPES = [(1, 2, 1), (64, 64, 256), (130, 70, 100), (300, 264, 1000), (257, 136, 33), (1000, 520, 777),
-          (2048, 1024, 512)]
+          (259, 132, 65), (3, 4, 9), (2048, 1024, 512)]     # 132, 4: whole groups of four channels, not of eight
 
 
 @pytest.mark.parametrize("shape", SHAPES)
