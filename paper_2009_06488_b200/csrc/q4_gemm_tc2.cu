@@ -76,9 +76,9 @@ constexpr int STG_SET = 4 * 32 * 128;      // int32 epilogue staging: 4 warps x 
 // 74 CTA pairs better or the depth is long, and loses e.g. at 4096^3 (four waves against
 // five of 192-column tiles with fully overlapped epilogues).
 // NSTG: staging slices per epilogue warp.  With two, a TMA store reads one while the next is
-// filled, which shortens an exposed epilogue (2048^3, one wave: 13.4 -> 12.6 us); the 256-column
-// configuration pays for the second set with a packed stage, which long problems miss
-// (8192^3: 297 -> 302 us), so it exists in both forms and the launcher picks by wave count.
+// filled.  The 192-column form has room for two; in the 256-column form a second set would
+// cost a packed stage, which long problems miss (8192^3: 297 -> 302 us), and short ones no
+// longer need it since the unpack warps help to drain a CTA pair's last tile.
 template <int BNC_, int NSTG_>
 struct Cfg {
     static constexpr int BNC = BNC_;             // columns of the pair tile
@@ -91,7 +91,7 @@ struct Cfg {
     static constexpr int BS = ROT ? 4 : 8;       // Bt operand stages in shared memory (BH * 128 B each)
     static constexpr int WALK = BS;              // stages per block of the MMA loop: a multiple of both ring depths
     static constexpr int BBOX = ROT ? BH / 2 : BH;   // rows per TMA box of Bt
-    static constexpr int PS = ROT ? (NSTG == 2 ? 7 : 8) : 6;   // packed stages (A 8 KB + Bt BH * 64 B)
+    static constexpr int PS = ROT ? 8 : 6;       // packed stages (A 8 KB + Bt BH * 64 B)
     static constexpr int PSTAGE = PA + BH * PROW;
     static constexpr int BSTAGE = BH * UROW;     // unpacked Bt bytes per stage
     static constexpr int NTB = BH * 4 / GT;      // Bt tasks (16-byte packed chunks) per thread per stage
@@ -105,7 +105,7 @@ struct Cfg {
     static constexpr int OFF_COLTERM = OFF_SUMS + 2 * G * SUMS_N * 4;
     static constexpr int OFF_PC = OFF_COLTERM + BNC * 4;       // per-channel: int32 [4][BNC] zero point, multiplier, rounding, shift
     static constexpr int OFF_BAR = OFF_PC + 4 * BNC * 4;
-    static constexpr int NBAR = 2 * PS + 2 * US + BS + 12;
+    static constexpr int NBAR = 2 * PS + 2 * US + BS + 13;
     static constexpr int OFF_MISC = OFF_BAR + NBAR * 8;
     static constexpr int SMEM = OFF_MISC + 16 + 1024;
 
@@ -115,7 +115,10 @@ struct Cfg {
     static_assert(BSTAGE % 1024 == 0 && PSTAGE % 1024 == 0, "stage alignment");
     static_assert(OFF_STG % 1024 == 0, "staging tile alignment (128-byte swizzle atoms)");
     static_assert(SMEM <= 227 * 1024, "shared memory budget");
+    static_assert(!ROT || NSTG == 1, "the 256-column form has room for one set of staging slices");
     static_assert(G <= PS, "a group's packed-ring slot advances by G per stage and wraps at most once");
+    static_assert(((BNC / 32 - 1) / 2) * WPG * 2 * 4096 <= PS * PSTAGE && G + 1 >= (BNC / 32 + 1) / 2,
+                  "last tile: the helping unpack warps stage two chunks each in the packed ring, and with the epilogue warps they cover every chunk");
 
     // D = s32, A = B = unsigned 8-bit, K-major, M = 256 (pair), N = BNC (ROT: BNC / 2 per MMA).
     static constexpr uint32_t kIdesc = (2u << 4) | ((uint32_t)((ROT ? BNC / 2 : BNC) >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
@@ -175,6 +178,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     auto bar_peer_tempty = [&](int a) { return barT + 8u * (uint32_t)(5 + a); };
     auto bar_sums        = [&](int a) { return barT + 8u * (uint32_t)(8 + a); };
     auto bar_tstart      = [&](int a) { return barT + 8u * (uint32_t)(10 + a); };
+    const uint32_t bar_final = barT + 8u * 12u;      // the last tile's column terms are in shared memory
     const uint32_t tmem_slot = sbase + OFF_MISC;
     const uint32_t abort_flag = sbase + OFF_MISC + 4;
 
@@ -206,6 +210,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_init(bar_tempty(a), 128);
             mbar_init(bar_peer_tempty(a), 1);
         }
+        mbar_init(bar_final, 128);
         sts32(abort_flag, 0);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
@@ -235,6 +240,109 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         pc_fast = __syncthreads_and(ok);
     }
+
+    // One 32-column chunk of an accumulator: tensor memory -> Eq. 2's remaining terms -> the
+    // output (int32 through a staging slice and a TMA store, or re-quantized and packed).
+    // taddr: the chunk in tensor memory (my lane quarter lg); ch, nc: its first column in the
+    // tile / in C; m, ra, rowterm: my row, its depth sum and Eq. 2's row term; slice: my
+    // 4 KB staging slice and how to wait for it (0: it is free, 1: my stores have all read
+    // their slices, 2: all but the latest); release_mid: hand the middle half-buffer back
+    // once the chunk is in registers.
+    auto drain_chunk = [&](uint32_t taddr, int ch, int nc, int lg, int tm, int m, int ra, uint32_t rowterm,
+                           uint32_t slice, int slice_wait, bool release_mid) {
+        uint32_t r[32];
+        tc_ld32(taddr, r);
+        tc_wait_ld();
+        if (ROT && release_mid) {
+            // the middle buffer is in registers: the next tile's upper-half MMAs may start
+            tc_fence_before();
+            mbar_arrive(bar_tempty(2));
+        }
+        if (pc) {
+            // the column's own zero point in Eq. 2's row-sum term
+#pragma unroll
+            for (int qd = 0; qd < 8; ++qd) {
+                const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
+                const uint4 zz = lds128(pc_s + 4 * (ch * 32 + 4 * qd));
+                r[4 * qd + 0] += ct.x - (uint32_t)ra * zz.x;
+                r[4 * qd + 1] += ct.y - (uint32_t)ra * zz.y;
+                r[4 * qd + 2] += ct.z - (uint32_t)ra * zz.z;
+                r[4 * qd + 3] += ct.w - (uint32_t)ra * zz.w;
+            }
+        } else {
+#pragma unroll
+            for (int qd = 0; qd < 8; ++qd) {
+                const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
+                r[4 * qd + 0] += rowterm + ct.x;
+                r[4 * qd + 1] += rowterm + ct.y;
+                r[4 * qd + 2] += rowterm + ct.z;
+                r[4 * qd + 3] += rowterm + ct.w;
+            }
+        }
+        if (!REQUANT && p.c_tma) {
+            // int32 tile out through shared memory and one TMA store per warp: my
+            // row's 128 bytes go to the swizzled staging slice of my warp; rows and
+            // columns past M / N are clipped by the tensor map
+            if (lane == 0) {                       // the store that last used this slice has read it
+                if (slice_wait == 2) bulk_wait_read_but_one(); else if (slice_wait == 1) bulk_wait_read();
+            }
+            __syncwarp();
+#pragma unroll
+            for (int qd = 0; qd < 8; ++qd)
+                sts128(slice + (uint32_t)(lane * 128 + ((qd ^ (lane & 7)) << 4)),
+                       make_uint4(r[4 * qd], r[4 * qd + 1], r[4 * qd + 2], r[4 * qd + 3]));
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                tma_store_2d(&tmC, slice, nc, tm * 256 + (int)rank * TMC + lg * 32);
+                bulk_commit();
+            }
+        } else if (m < g.M) {
+            const bool full = (nc + 32 <= g.N);
+            if (!REQUANT) {
+                int32_t* dst = g.C + (int64_t)m * g.ldc + nc;
+                if (full && p.c_vec) {
+#pragma unroll
+                    for (int qd = 0; qd < 8; ++qd)
+                        *reinterpret_cast<uint4*>(dst + 4 * qd) =
+                            make_uint4(r[4 * qd], r[4 * qd + 1], r[4 * qd + 2], r[4 * qd + 3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (nc + j < g.N) dst[j] = (int32_t)r[j];
+                }
+            } else {
+                uint32_t o[4];
+                if (pc) {
+                    // eight values at a time (channels i and i + 4 share a packed pair); each
+                    // word holds value - lo per nibble
+                    const uint32_t hml2 = (uint32_t)(g.rq.hi - g.rq.lo) * 0x00010001u;
+                    const uint32_t lofill = (uint32_t)g.rq.lo * 0x11111111u;
+#pragma unroll
+                    for (int qd = 0; qd < 4; ++qd)
+                        o[qd] = requant8_channels<true>(r + 8 * qd, g.rq, pc_s + 4 * BNC, BNC, ch * 32 + 8 * qd,
+                                                        pc_fast != 0, hml2) + lofill;
+                } else {
+#pragma unroll
+                    for (int qd = 0; qd < 4; ++qd) {
+                        uint32_t wv = 0;
+#pragma unroll
+                        for (int e = 0; e < 8; ++e)
+                            wv |= requant((int32_t)r[8 * qd + e], g.rq) << (4 * e);
+                        o[qd] = wv;
+                    }
+                }
+                uint8_t* dst = g.Cq + (int64_t)m * g.ldcq + (nc >> 1);
+                if (full && p.cq_vec) {
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                } else {
+#pragma unroll
+                    for (int b = 0; b < 16; ++b)
+                        if (nc + 2 * b < g.N) dst[b] = (uint8_t)(o[b >> 2] >> (8 * (b & 3)));
+                }
+            }
+        }
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -555,6 +663,46 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
             }
         }
+        // The last tile of this CTA pair has no next tile to hide its epilogue behind, and the
+        // unpack warps are idle from its last stages on: each of them drains two of the tile's
+        // chunks in its own lane quarter (the epilogue warp of the quarter takes the first
+        // two).  Staging slices: the packed ring, which nothing reads or fills any more once an
+        // accumulator (half) is complete -- every stage of the tile has been expanded by then.
+        if (lt > 0 && !lds32(abort_flag)) {
+            const uint32_t ltf = lt - 1;
+            const int tile = cluster_id + (int)ltf * nclusters;
+            const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+            const int acc = (int)(ltf % NACC);
+            const uint32_t aph = (ltf / NACC) & 1u;
+            const int m = tm * 256 + (int)rank * TMC + arow;
+            const int n0 = tn * BNC;
+            mbar_wait(bar_final, 0, abort_flag, g.status);
+            int ra = 0;
+            if (need_ra) {
+                const uint32_t s0 = sums_s + 4 * (acc * G * SUMS_N);
+#pragma unroll
+                for (int gi = 0; gi < G; ++gi) ra += lds32(s0 + 4 * (gi * SUMS_N + arow));
+            } else if (m < g.M) {
+                ra = g.rowsum_a[m];
+            }
+            const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
+            const uint32_t taddr0 = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(ROT ? 0 : acc * BNC);
+#pragma unroll 1
+            for (int k = 0; k < 2; ++k) {
+                const int ci = 2 * (grp + 1) + k;              // in the epilogue's drain order
+                if (ci >= BNC / 32) break;
+                const int ch = ROT ? ((ci + BNC / 64) & (BNC / 32 - 1)) : ci;
+                const int nc = n0 + ch * 32;
+                const uint32_t tcol = (ROT && ch < BNC / 64 && (ltf & 1u)) ? 256u + (uint32_t)(ch * 32) : (uint32_t)(ch * 32);
+                mbar_wait(bar_tfull(ROT ? (ci < BNC / 64 ? 1 : 0) : acc), aph, abort_flag, g.status);
+                tc_fence_after();
+                if (nc < g.N)              // warp-uniform
+                    drain_chunk(taddr0 + tcol, ch, nc, q, tm, m, ra, rowterm,
+                                sbase + OFF_P + (uint32_t)((2 * (warp - 2) + k) * 4096), 0, false);
+            }
+            tc_fence_before();
+            if (!REQUANT && p.c_tma && lane == 0) bulk_wait_all();   // my TMA stores are complete
+        }
     } else {
         // ------------------------------------------------------------ epilogue warps
         const int lg = warp & 3;
@@ -604,13 +752,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
             const uint32_t rowterm = (uint32_t)0 - (uint32_t)(g.zb * ra);
             asm volatile("bar.sync 1, 128;" ::: "memory");
+            // My CTA pair's last tile: the unpack warps have nothing left to expand and drain
+            // all chunks but the first two of every lane quarter (see the end of their branch).
+            const bool last_tile = tile + nclusters >= ntiles;
+            if (last_tile) mbar_arrive(bar_final);
 
             // ROT: barrier 1 = this tile's upper half is complete, barrier 0 = all of it
             mbar_wait(bar_tfull(ROT ? 1 : acc), aph, abort_flag, g.status);
             tc_fence_after();
             const uint32_t taddr0 = tmem_base + ((uint32_t)(lg * 32) << 16) + (uint32_t)(ROT ? 0 : acc * BNC);
 #pragma unroll 1
-            for (int ci = 0; ci < BNC / 32; ++ci) {
+            for (int ci = 0; ci < (last_tile ? 2 : BNC / 32); ++ci) {
                 // ROT: the upper half (the middle buffer, which the next tile needs first), then
                 // the lower half in this tile's outer buffer
                 const int ch = ROT ? ((ci + BNC / 64) & (BNC / 32 - 1)) : ci;
@@ -628,101 +780,10 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         mbar_arrive(bar_tempty(2));
                     }
                 }
-                if (nc < g.N) {            // warp-uniform
-                uint32_t r[32];
-                tc_ld32(taddr0 + tcol, r);
-                tc_wait_ld();
-                if (ROT && ci == BNC / 64 - 1) {
-                    // the middle buffer is in registers: the next tile's upper-half MMAs may start
-                    tc_fence_before();
-                    mbar_arrive(bar_tempty(2));
-                }
-                if (pc) {
-                    // the column's own zero point in Eq. 2's row-sum term
-#pragma unroll
-                    for (int qd = 0; qd < 8; ++qd) {
-                        const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
-                        const uint4 zz = lds128(pc_s + 4 * (ch * 32 + 4 * qd));
-                        r[4 * qd + 0] += ct.x - (uint32_t)ra * zz.x;
-                        r[4 * qd + 1] += ct.y - (uint32_t)ra * zz.y;
-                        r[4 * qd + 2] += ct.z - (uint32_t)ra * zz.z;
-                        r[4 * qd + 3] += ct.w - (uint32_t)ra * zz.w;
-                    }
-                } else {
-#pragma unroll
-                    for (int qd = 0; qd < 8; ++qd) {
-                        const uint4 ct = lds128(colterm_s + 4 * (ch * 32 + 4 * qd));
-                        r[4 * qd + 0] += rowterm + ct.x;
-                        r[4 * qd + 1] += rowterm + ct.y;
-                        r[4 * qd + 2] += rowterm + ct.z;
-                        r[4 * qd + 3] += rowterm + ct.w;
-                    }
-                }
-                if (!REQUANT && p.c_tma) {
-                    // int32 tile out through shared memory and one TMA store per warp: my
-                    // row's 128 bytes go to the swizzled staging slice of my warp; rows and
-                    // columns past M / N are clipped by the tensor map
-                    const uint32_t slice = sbase + OFF_STG + (uint32_t)(((NSTG > 1 ? (ci & 1) : 0) * 4 + lg) * 4096);
-                    if (lane == 0) {                       // the store that last used this slice has read it
-                        if (NSTG > 1) bulk_wait_read_but_one(); else bulk_wait_read();
-                    }
-                    __syncwarp();
-#pragma unroll
-                    for (int qd = 0; qd < 8; ++qd)
-                        sts128(slice + (uint32_t)(lane * 128 + ((qd ^ (lane & 7)) << 4)),
-                               make_uint4(r[4 * qd], r[4 * qd + 1], r[4 * qd + 2], r[4 * qd + 3]));
-                    fence_async_smem();
-                    __syncwarp();
-                    if (lane == 0) {
-                        tma_store_2d(&tmC, slice, nc, tm * 256 + (int)rank * TMC + lg * 32);
-                        bulk_commit();
-                    }
-                } else if (m < g.M) {
-                    const bool full = (nc + 32 <= g.N);
-                    if (!REQUANT) {
-                        int32_t* dst = g.C + (int64_t)m * g.ldc + nc;
-                        if (full && p.c_vec) {
-#pragma unroll
-                            for (int qd = 0; qd < 8; ++qd)
-                                *reinterpret_cast<uint4*>(dst + 4 * qd) =
-                                    make_uint4(r[4 * qd], r[4 * qd + 1], r[4 * qd + 2], r[4 * qd + 3]);
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (nc + j < g.N) dst[j] = (int32_t)r[j];
-                        }
-                    } else {
-                        uint32_t o[4];
-                        if (pc) {
-                            // eight values at a time (channels i and i + 4 share a packed pair); each
-                            // word holds value - lo per nibble
-                            const uint32_t hml2 = (uint32_t)(g.rq.hi - g.rq.lo) * 0x00010001u;
-                            const uint32_t lofill = (uint32_t)g.rq.lo * 0x11111111u;
-#pragma unroll
-                            for (int qd = 0; qd < 4; ++qd)
-                                o[qd] = requant8_channels<true>(r + 8 * qd, g.rq, pc_s + 4 * BNC, BNC, ch * 32 + 8 * qd,
-                                                                pc_fast != 0, hml2) + lofill;
-                        } else {
-#pragma unroll
-                            for (int qd = 0; qd < 4; ++qd) {
-                                uint32_t wv = 0;
-#pragma unroll
-                                for (int e = 0; e < 8; ++e)
-                                    wv |= requant((int32_t)r[8 * qd + e], g.rq) << (4 * e);
-                                o[qd] = wv;
-                            }
-                        }
-                        uint8_t* dst = g.Cq + (int64_t)m * g.ldcq + (nc >> 1);
-                        if (full && p.cq_vec) {
-                            *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
-                        } else {
-#pragma unroll
-                            for (int b = 0; b < 16; ++b)
-                                if (nc + 2 * b < g.N) dst[b] = (uint8_t)(o[b >> 2] >> (8 * (b & 3)));
-                        }
-                    }
-                }
-                }
+                if (nc < g.N)              // warp-uniform
+                    drain_chunk(taddr0 + tcol, ch, nc, lg, tm, m, ra, rowterm,
+                                sbase + OFF_STG + (uint32_t)(((NSTG > 1 ? (ci & 1) : 0) * 4 + lg) * 4096),
+                                NSTG > 1 ? 2 : 1, ci == BNC / 64 - 1);
             }
             tc_fence_before();
             mbar_arrive(bar_tempty(ROT ? (int)(lt & 1u) : acc));
@@ -832,7 +893,7 @@ bool make_c32_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, int col
 // Tile width for a problem: estimated clocks of the busiest CTA pair with either width, from
 // measured stage and epilogue times (192 columns: 520 clk per 128-deep stage, epilogues
 // overlapped but the last; 256 columns: 540 clk per stage, 4200 clk per tile of exposed
-// half drain and pipeline restart, 2500 clk for the last half).  Checked against forced
+// half drain and pipeline restart, 1000 clk for the last tile's shared drain).  Checked against forced
 // widths at 1536^3, 2048^3, 3072^3, 4096^3, 4096 x 11008 x 4096, 6144^3, 8192^3.
 int gemm_tc_pair_width(const GemmParams& g)
 {
@@ -841,7 +902,7 @@ int gemm_tc_pair_width(const GemmParams& g)
     const long long t192 = tm * (((long long)g.N + 191) / 192), t256 = tm * (((long long)g.N + 255) / 256);
     const long long pairs = 74;
     const long long c192 = (t192 + pairs - 1) / pairs * nslab * 520 + 5000;
-    const long long c256 = (t256 + pairs - 1) / pairs * (nslab * 540 + 4200) + 2500;
+    const long long c256 = (t256 + pairs - 1) / pairs * (nslab * 540 + 4200) + 1000;
     return c256 < c192 ? 256 : 192;
 }
 
@@ -875,9 +936,7 @@ q4_status launch_gemm_tc_pair(const GemmParams& g, bool rq, cudaStream_t st, int
 {
     if (width != 192 && width != 256) width = gemm_tc_pair_width(g);
     if (width == 192) return launch_pair_w<192, 2>(g, rq, st);
-    // few tiles per CTA pair: the last tile's exposed epilogue weighs more than ring depth
-    const long long t256 = (((long long)g.M + 255) / 256) * (((long long)g.N + 255) / 256);
-    return t256 <= 3 * 74 ? launch_pair_w<256, 2>(g, rq, st) : launch_pair_w<256, 1>(g, rq, st);
+    return launch_pair_w<256, 1>(g, rq, st);
 }
 
 }  // namespace q4

@@ -34,8 +34,8 @@ def layer(seed, N, H, W, C, OC, k, s, p):
 
 # N, H, W, C, OC, k, stride, pad -- a large layer first, then smaller ones with other
 # pitches and row counts; the last is a 1x1 layer large enough for the big-GEMM kernel: its
-# unrolled matrix is the input itself and the array holds only the depth sums that a
-# pre-pass writes and the GEMM reads
+# unrolled matrix is the input itself, and at this size the kernel takes the depth sums
+# itself, so the call is a single launch that must leave the array alone and still agree
 LAYERS = ((900, (6, 32, 32, 16, 72, 3, 1, 1)),
           (901, (3, 17, 13, 8, 6, 3, 2, 1)),
           (902, (2, 9, 11, 3, 6, 5, 1, 2)),
@@ -59,8 +59,9 @@ def test_static_scratch_entry_point_matches_oracle_and_q4_conv2d_on_calls_in_a_r
         got = torch.full((d.M, L.OC // 2), 0x5A, dtype=torch.uint8, device="cuda")
         n0 = q4.q4_launch_count()
         q4.q4_conv2d_static(Xd, Wd, d, L.za, L.zb, rq, got, bd)
-        # more than one kernel: the scratch array was written (unroll or sums) and read back
-        assert q4.q4_launch_count() - n0 >= 2
+        # more than one kernel: the scratch array was written (the unrolled matrix and its row
+        # sums) and read back; a 1x1 layer has nothing to unroll
+        assert q4.q4_launch_count() - n0 >= (1 if L.KH == 1 else 2)
         torch.cuda.synchronize()
         assert q4.q4_last_device_status() == q4.Q4_OK
         want = oracle.conv2d(X, L.Wt, L.bias, oracle.ConvDesc(*args), L.za, L.zb,
