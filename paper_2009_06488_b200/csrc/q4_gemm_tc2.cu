@@ -893,7 +893,7 @@ bool make_c32_map(CUtensorMap* tm, int32_t* base, int64_t ldc, int rows, int col
 // Tile width for a problem: estimated clocks of the busiest CTA pair with either width, from
 // measured stage and epilogue times (192 columns: 520 clk per 128-deep stage, epilogues
 // overlapped but the last; 256 columns: 540 clk per stage, 4200 clk per tile of exposed
-// half drain and pipeline restart, 1000 clk for the last tile's shared drain).  Checked against forced
+// half drain and pipeline restart, 2500 clk for the last tile's drain).  Checked against forced
 // widths at 1536^3, 2048^3, 3072^3, 4096^3, 4096 x 11008 x 4096, 6144^3, 8192^3.
 int gemm_tc_pair_width(const GemmParams& g)
 {
@@ -902,7 +902,7 @@ int gemm_tc_pair_width(const GemmParams& g)
     const long long t192 = tm * (((long long)g.N + 191) / 192), t256 = tm * (((long long)g.N + 255) / 256);
     const long long pairs = 74;
     const long long c192 = (t192 + pairs - 1) / pairs * nslab * 520 + 5000;
-    const long long c256 = (t256 + pairs - 1) / pairs * (nslab * 540 + 4200) + 1000;
+    const long long c256 = (t256 + pairs - 1) / pairs * (nslab * 540 + 4200) + 2500;
     return c256 < c192 ? 256 : 192;
 }
 
