@@ -473,7 +473,9 @@ def time_gemm_sweep(q4, wl, reps: int = 20):
         ws = torch.empty(q4.q4_gemm_workspace_bytes(c.M, c.N, c.K), dtype=torch.uint8, device="cuda")
         cb = q4.q4_row_sums(Bt, c.N, c.K, torch.empty(c.N, dtype=torch.int32, device="cuda"))
         ops = 2.0 * c.M * c.N * c.K
-        r = max(3, min(reps, int(2e10 / ops * 4) + 3))
+        # launches per graph replay: enough that the replay's own launch cost (several us) is
+        # spread thin -- 20 up to 4096^3, 4 for the 600 us calls of c5
+        r = max(3, min(reps, int(4e12 / ops) + 3))
         ms = graph_time_ms([lambda: q4.q4_gemm(A, Bt, C, c.M, c.N, c.K, c.za, c.zb, None, cb, ws)], r)
         out[name] = {"q4_gemm_ms": ms, "q4_gemm_tops": ops / (ms * 1e-3) / 1e12}
         # context: the library's int8 GEMM (s8 x s8 -> s32, no zero points, no unpack) on the shape
@@ -501,9 +503,9 @@ def time_gemm_sweep(q4, wl, reps: int = 20):
     chan = lambda lo, hi: torch.randint(lo, hi, (n,), dtype=torch.int32, device="cuda")
     zb_c, bias_c, mult_c, shift_c = chan(0, 16), chan(-512, 513), chan(1 << 30, (1 << 31) - 1), chan(8, 17)
     rq = q4.Requant(c.mult, c.shift, 0, 0, 15)
-    t_pt = graph_time_ms([lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, c.za, c.zb, rq, colsum_b=cb, ws=ws)], 5)
+    t_pt = graph_time_ms([lambda: q4.q4_gemm_requant(A, Bt, Cq, n, n, n, c.za, c.zb, rq, colsum_b=cb, ws=ws)], 6)
     t_pc = graph_time_ms([lambda: q4.q4_gemm_requant_channels(A, Bt, Cq, n, n, n, c.za, zb_c, mult_c, shift_c,
-                                                              0, 0, 15, bias_c, None, cb, ws)], 5)
+                                                              0, 0, 15, bias_c, None, cb, ws)], 6)
     out["per_channel_epilogue_8192"] = {"q4_gemm_requant_ms": t_pt, "q4_gemm_requant_channels_ms": t_pc,
                                         "ratio": t_pc / t_pt}
     return out

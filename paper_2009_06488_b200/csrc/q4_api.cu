@@ -94,12 +94,15 @@ static q4_status run_gemm(GemmParams& p, bool rq, cudaStream_t st, void* ws = nu
     p.status = status_ptr();
     if (!p.status) return Q4_ERR_CUDA;
     const int v = variant_kind();
-    // The CTA-pair kernel pays off from about 32 of its 256 x 256 tiles (2048^3 is one wave of
-    // 64: 12.7 us against 18.7 us); below that the single-CTA kernel, with narrower tiles and
-    // its sums taken in the kernel, finishes sooner (1024^3: 7.4 against 8.3 us).  Variant 2
-    // always takes the pair kernel where it applies.
+    // The CTA-pair kernel pays off from about 64 of its 256 x 256 tiles (2048^3 is one wave of
+    // 64: 12.1 us against 18.7 us), or from 32 where the depth is long enough to carry its
+    // fixed costs -- prologue, pipeline fill, a last tile of 256 x 256 to drain; below that the
+    // single-CTA kernel, with narrower tiles and its sums taken in the kernel, finishes sooner
+    // (1024^3: 6.5 against 8.7 us; 1536^3, 36 tiles: 9.4 against 10.5 us; 8192 x 256 x 1024, 32
+    // tiles: 7.8 against 9.3 us).  Variant 2 always takes the pair kernel where it applies.
     const long long pair_tiles = ((long long)p.M + 255) / 256 * (((long long)p.N + 255) / 256);
-    if (v != 1 && v != 3 && gemm_tc_pair_supported(p) && (v == 2 || pair_tiles >= 32)) {
+    const bool pair_pays = pair_tiles >= 64 || (pair_tiles >= 32 && p.K >= 2048);
+    if (v != 1 && v != 3 && gemm_tc_pair_supported(p) && (v == 2 || pair_pays)) {
         // Large problems use the workspace, if given, for the depth sums where one pass over
         // an operand is cheaper than every output tile taking them again; without one the
         // kernel does everything itself.  The results are identical.
