@@ -353,11 +353,15 @@ q4_status q4_dequantize(const int32_t* C, int64_t ldc, int32_t rows, int32_t col
 
 /*
  * q4_gemm with HOST operands: copies A and Bt to the device, runs q4_gemm and
- * copies C back, all on `stream`, then synchronizes it.  hA / hBt / hC are host
- * pointers with the same pitches as above (pinned memory makes the copies
- * asynchronous).  dev_staging is a DEVICE buffer owned by the caller of at least
- * q4_gemm_host_staging_bytes(...) bytes, 256-byte aligned; it holds the device
- * copies, so this entry point allocates nothing either.
+ * copies C back, then synchronizes `stream`.  The work is ordered behind `stream`
+ * and goes in row slices over `stream` and one stream of the library's own (created
+ * on first use, one per device), so that a slice's copy back overlaps the next
+ * slice's upload and product; when the call returns all of it is complete.  hA /
+ * hBt / hC are host pointers with the same pitches as above (pinned memory makes
+ * the copies asynchronous, and only then do they overlap).  dev_staging is a DEVICE
+ * buffer owned by the caller of at least q4_gemm_host_staging_bytes(...) bytes,
+ * 256-byte aligned; it holds the device copies and the column sums of Bt, so this
+ * entry point allocates no device memory either.
  */
 q4_status q4_gemm_host(const uint8_t* hA, int64_t lda, const uint8_t* hBt, int64_t ldb,
                        int32_t* hC, int64_t ldc, int32_t M, int32_t N, int32_t K,

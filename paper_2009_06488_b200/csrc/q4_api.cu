@@ -1,5 +1,6 @@
 // C ABI of the q4 library (declared in q4.h): argument validation, kernel selection,
 // launch.  No allocation, no synchronization except where the header says so.
+#include <mutex>
 #include <atomic>
 #include <cstdio>
 #include <cstdlib>
@@ -575,7 +576,28 @@ size_t q4_gemm_host_staging_bytes(int32_t M, int32_t N, int32_t K,
     (void)K;
     if (M < 0 || N < 0 || lda < 0 || ldb < 0 || ldc < 0) return 0;
     auto up = [](size_t b) { return (b + 255) / 256 * 256; };
-    return up((size_t)M * (size_t)lda) + up((size_t)N * (size_t)ldb) + up((size_t)M * (size_t)ldc * 4);
+    return up((size_t)M * (size_t)lda) + up((size_t)N * (size_t)ldb) + up((size_t)M * (size_t)ldc * 4) +
+           up((size_t)N * 4);      // the column sums of Bt, taken once for all row slices
+}
+
+// A second stream and two events per device for q4_gemm_host, created on first use and
+// kept for the life of the process.
+struct HostPipe { cudaStream_t side = nullptr; cudaEvent_t weights = nullptr, done = nullptr; bool ok = false; };
+static HostPipe* host_pipe()
+{
+    static HostPipe pipes[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    HostPipe& h = pipes[dev];
+    if (!h.ok) {
+        if (cudaStreamCreateWithFlags(&h.side, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h.weights, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&h.done, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        h.ok = true;
+    }
+    return &h;
 }
 
 q4_status q4_gemm_host(const uint8_t* hA, int64_t lda, const uint8_t* hBt, int64_t ldb,
@@ -595,18 +617,43 @@ q4_status q4_gemm_host(const uint8_t* hA, int64_t lda, const uint8_t* hBt, int64
     uint8_t* dA = static_cast<uint8_t*>(dev_staging);
     uint8_t* dB = dA + up((size_t)M * lda);
     int32_t* dC = reinterpret_cast<int32_t*>(dB + up((size_t)N * ldb));
+    int32_t* dcb = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(dC) + up((size_t)M * ldc * 4));
     // only the bytes the header promises to touch: ceil(K / 2) of every operand row, N
     // elements of every output row (pitch padding is neither read nor written)
     const size_t kbytes = ((size_t)K + 1) / 2;
-    if (cudaMemcpy2DAsync(dA, (size_t)lda, hA, (size_t)lda, kbytes, (size_t)M, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-        cudaMemcpy2DAsync(dB, (size_t)ldb, hBt, (size_t)ldb, kbytes, (size_t)N, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    // The int32 result is eight times the bytes of a packed operand, so the call is bound by
+    // the copy back.  Rows go in slices that alternate between two streams: a slice's
+    // download overlaps the next slice's upload and product (the two directions have their
+    // own copy engines).  Bt and its column sums are needed by every slice and go first.
+    HostPipe* hp = host_pipe();
+    if (!hp) return Q4_ERR_CUDA;
+    if (cudaMemcpy2DAsync(dB, (size_t)ldb, hBt, (size_t)ldb, kbytes, (size_t)N, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return Q4_ERR_CUDA;
-    s = q4_gemm(dA, lda, dB, ldb, dC, ldc, M, N, K, za, zb, nullptr, nullptr, nullptr, 0, stream);
-    if (s != Q4_OK) return s;
-    if (cudaMemcpy2DAsync(hC, (size_t)ldc * 4, dC, (size_t)ldc * 4, (size_t)N * 4, (size_t)M,
-                          cudaMemcpyDeviceToHost, st) != cudaSuccess)
-        return Q4_ERR_CUDA;
-    return cudaStreamSynchronize(st) == cudaSuccess ? Q4_OK : Q4_ERR_CUDA;
+    if (launch_row_sums(dB, ldb, N, K, dcb, st) != cudaSuccess) return Q4_ERR_CUDA;
+    if (cudaEventRecord(hp->weights, st) != cudaSuccess ||
+        cudaStreamWaitEvent(hp->side, hp->weights, 0) != cudaSuccess) return Q4_ERR_CUDA;
+    int32_t slice = (M / 8 + 255) / 256 * 256;        // about eight slices, whole tiles of 256 rows
+    if (slice < 1024) slice = 1024;
+    int k = 0;
+    for (int32_t m0 = 0; m0 < M; m0 += slice, ++k) {
+        const int32_t rows = M - m0 < slice ? M - m0 : slice;
+        cudaStream_t sk = (k & 1) ? hp->side : st;
+        if (cudaMemcpy2DAsync(dA + (size_t)m0 * lda, (size_t)lda, hA + (size_t)m0 * lda, (size_t)lda, kbytes,
+                              (size_t)rows, cudaMemcpyHostToDevice, sk) != cudaSuccess) return Q4_ERR_CUDA;
+        s = q4_gemm(dA + (size_t)m0 * lda, lda, dB, ldb, dC + (size_t)m0 * ldc, ldc, rows, N, K, za, zb, nullptr,
+                    dcb, nullptr, 0, sk);
+        if (s != Q4_OK) break;
+        if (cudaMemcpy2DAsync(hC + (size_t)m0 * ldc, (size_t)ldc * 4, dC + (size_t)m0 * ldc, (size_t)ldc * 4,
+                              (size_t)N * 4, (size_t)rows, cudaMemcpyDeviceToHost, sk) != cudaSuccess) {
+            s = Q4_ERR_CUDA;
+            break;
+        }
+    }
+    // the caller's stream ends behind the side stream, whatever happened above
+    if (cudaEventRecord(hp->done, hp->side) != cudaSuccess ||
+        cudaStreamWaitEvent(st, hp->done, 0) != cudaSuccess) return Q4_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return Q4_ERR_CUDA;
+    return s;
 }
 
 q4_status q4_last_device_status(void* stream)

@@ -338,3 +338,15 @@ def test_host_entry_point(q4):
     q4.q4_set_variant(0)
     q4.q4_gemm_host(hA, hBt, hC, c.M, c.N, c.K, c.za, c.zb, staging)
     assert (hC.numpy() == oracle.gemm(c.A, c.Bt, c.M, c.N, c.K, c.za, c.zb)).all()
+    # several row slices over the two streams (slices of 1024 rows, a ragged last one), int32
+    # pitch wider than a row: the padding on the host stays as it was
+    c = aligned_case(2500, 264, 200, seed=13)
+    hA, hBt = torch.from_numpy(c.A).pin_memory(), torch.from_numpy(c.Bt).pin_memory()
+    hC = torch.full((c.M, c.N + 4), -7, dtype=torch.int32).pin_memory()
+    staging = torch.full((q4.q4_gemm_host_staging_bytes(c.M, c.N, c.K, c.lda, c.ldb, c.N + 4),), 0xA5,
+                         dtype=torch.uint8, device="cuda")
+    for _ in range(2):          # the second call finds the first call's leftovers in the staging buffer
+        q4.q4_gemm_host(hA, hBt, hC, c.M, c.N, c.K, c.za, c.zb, staging)
+        assert q4.q4_last_device_status() == q4.Q4_OK
+        assert (hC.numpy()[:, :c.N] == oracle.gemm(c.A, c.Bt, c.M, c.N, c.K, c.za, c.zb)).all()
+        assert (hC.numpy()[:, c.N:] == -7).all()
