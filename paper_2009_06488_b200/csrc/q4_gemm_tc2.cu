@@ -507,7 +507,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
         } else if (lane == 0) {
             // -------------------------------------------------------- peer relay (per tile)
-            // forwards "my epilogue has drained the buffer" to the leader, which issues the MMAs
+            // forwards "my epilogue has drained the buffer" to the leader, which issues the MMAs.
+            // The arrives carry no release: what they order is the epilogue's tensor-memory
+            // loads, which were complete (tcgen05.wait::ld) and fenced before the epilogue
+            // threads arrived on the barrier this thread has just seen complete; the releasing
+            // form took the relay 1100 clk per arrive, on the path of the next tile's MMAs.
             uint32_t lt = 0;
             for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
                 if (!ROT) {
@@ -515,17 +519,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t aph = (lt / NACC) & 1u;
                     if (lt >= (uint32_t)NACC) {
                         mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, g.status);
-                        mbar_arrive_cluster(map_to_cta(bar_peer_tempty(acc), 0));
+                        mbar_arrive_cluster_relaxed(map_to_cta(bar_peer_tempty(acc), 0));
                     }
                 } else {
                     const int lo = (int)(lt & 1u);
                     if (lt >= 2u) {
                         mbar_wait(bar_tempty(lo), ((lt >> 1) & 1u) ^ 1u, abort_flag, g.status);
-                        mbar_arrive_cluster(map_to_cta(bar_peer_tempty(lo), 0));
+                        mbar_arrive_cluster_relaxed(map_to_cta(bar_peer_tempty(lo), 0));
                     }
                     if (lt >= 1u) {
                         mbar_wait(bar_tempty(2), (lt & 1u) ^ 1u, abort_flag, g.status);
-                        mbar_arrive_cluster(map_to_cta(bar_peer_tempty(2), 0));
+                        mbar_arrive_cluster_relaxed(map_to_cta(bar_peer_tempty(2), 0));
                     }
                 }
             }
