@@ -712,7 +712,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int lg = warp & 3;
         const int row = lg * 32 + lane;
         const int et = threadIdx.x - (2 + UW) * 32;
-        uint32_t lt = 0;
+        uint32_t lt = 0, nstore = 0;            // tiles taken, chunks drained by my warp
         for (int tile = cluster_id; tile < ntiles && !lds32(abort_flag); tile += nclusters, ++lt) {
             const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
             const int acc = (int)(lt % NACC);
@@ -784,10 +784,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         mbar_arrive(bar_tempty(2));
                     }
                 }
-                if (nc < g.N)              // warp-uniform
+                if (nc < g.N) {            // warp-uniform
+                    // Two staging slices alternate by the count of chunks drained, not by the
+                    // chunk's position: a tile whose last columns lie past N drains an odd number
+                    // of chunks, and "all but the latest store have read their slice" protects a
+                    // slice only if the latest store used the other one.
                     drain_chunk(taddr0 + tcol, ch, nc, lg, tm, m, ra, rowterm,
-                                sbase + OFF_STG + (uint32_t)(((NSTG > 1 ? (ci & 1) : 0) * 4 + lg) * 4096),
+                                sbase + OFF_STG + (uint32_t)(((NSTG > 1 ? (nstore & 1u) : 0u) * 4 + (uint32_t)lg) * 4096),
                                 NSTG > 1 ? 2 : 1, ci == BNC / 64 - 1);
+                    ++nstore;
+                }
             }
             tc_fence_before();
             mbar_arrive(bar_tempty(ROT ? (int)(lt & 1u) : acc));

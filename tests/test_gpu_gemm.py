@@ -162,6 +162,28 @@ def test_pair_kernel_tile_widths_agree_with_oracle(q4, variant, shape):
     assert (run_requant(q4, c, variant, rq, c.bias, use_ws=True) == wantq).all()
 
 
+def test_odd_number_of_chunks_per_tile_with_short_depth(q4):
+    """192-column tiles whose last column tile drains five of its six 32-column chunks
+    (N = 1116), one depth stage per tile, depth sums taken in the kernel: the int32 staging
+    slices of an epilogue warp alternate from store to store, and the next tile's first
+    store follows the last one of this tile within a few hundred clocks.  Repeated, because
+    what this guards against is a race (a slice refilled while its store still reads it)."""
+    import torch
+    M, N, K = 5415, 1116, 28
+    c = aligned_case(M, N, K, seed=4242)
+    want = torch.from_numpy(oracle.gemm(c.A, c.Bt, M, N, K, c.za, c.zb)).cuda()
+    A, Bt = dev(c.A), dev(c.Bt)
+    q4.q4_set_variant(TC192)
+    try:
+        for _ in range(60):
+            C = torch.full((M, N), -1515870811, dtype=torch.int32, device="cuda")
+            q4.q4_gemm(A, Bt, C, M, N, K, c.za, c.zb)
+            assert torch.equal(C, want)
+        assert q4.q4_last_device_status() == q4.Q4_OK
+    finally:
+        q4.q4_set_variant(0)
+
+
 @pytest.mark.parametrize("variant", [SIMT, TC])
 def test_precomputed_sums_give_the_same_result(q4, variant):
     c = aligned_case(200, 72, 300, seed=77)
