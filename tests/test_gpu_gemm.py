@@ -162,6 +162,45 @@ def test_pair_kernel_tile_widths_agree_with_oracle(q4, variant, shape):
     assert (run_requant(q4, c, variant, rq, c.bias, use_ws=True) == wantq).all()
 
 
+def _random_shapes(count, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for _ in range(count):
+        M = int(rng.integers(1, 2600)) if rng.random() < 0.75 else int(rng.integers(3000, 7000))
+        N = 2 * int(rng.integers(1, 700))
+        K = int(rng.integers(1, 600)) if rng.random() < 0.6 else int(rng.integers(1, 48))   # many one-stage tiles
+        out.append((M, N, K))
+    return out
+
+
+@pytest.mark.parametrize("shape", _random_shapes(36, 20260101))
+def test_random_shapes_every_kernel_and_sums_combination(q4, shape):
+    """Seeded random shapes (ragged in every dimension, a third of them with one or two
+    depth stages per tile so that a CTA's tiles follow each other within a few thousand
+    clocks) through the automatic choice and each forced kernel, with the depth sums given,
+    given for the weights only, and taken through a workspace: int32 and re-quantized output
+    against the oracle."""
+    import torch
+    M, N, K = shape
+    c = aligned_case(M, N, K, seed=M * 131 + N * 17 + K, with_bias=True)
+    want = oracle.gemm(c.A, c.Bt, M, N, K, c.za, c.zb)
+    rq = oracle.Requant(c.mult, 7, 3, 1, 14)
+    wantq = oracle.requant_matrix(want, c.bias, rq)
+    for variant in (0, TC1, TC192, TC256):
+        for kw in ({}, {"sums": True}, {"sums": "cols"}, {"use_ws": True}):
+            try:
+                got, _, _ = run_gemm(q4, c, variant, **kw)
+            except q4.Q4Error as e:          # a forced kernel that does not take the shape
+                assert e.status in (q4.Q4_ERR_ALIGNMENT, q4.Q4_ERR_UNSUPPORTED)
+                continue
+            assert (got == want).all(), (variant, kw)
+        try:
+            assert (run_requant(q4, c, variant, rq, c.bias) == wantq).all(), variant
+        except q4.Q4Error as e:
+            assert e.status in (q4.Q4_ERR_ALIGNMENT, q4.Q4_ERR_UNSUPPORTED)
+    q4.q4_set_variant(0)
+
+
 def test_odd_number_of_chunks_per_tile_with_short_depth(q4):
     """192-column tiles whose last column tile drains five of its six 32-column chunks
     (N = 1116), one depth stage per tile, depth sums taken in the kernel: the int32 staging
