@@ -705,7 +705,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                                 sbase + OFF_P + (uint32_t)((2 * (warp - 2) + k) * 4096), 0, false);
             }
             tc_fence_before();
-            if (!REQUANT && p.c_tma && lane == 0) bulk_wait_all();   // my TMA stores are complete
+            if (!REQUANT && p.c_tma && lane == 0) bulk_wait_read();  // my TMA stores have read their slices; their writes complete with the grid
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
@@ -799,7 +799,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             mbar_arrive(bar_tempty(ROT ? (int)(lt & 1u) : acc));
             asm volatile("bar.sync 1, 128;" ::: "memory");
         }
-        if (!REQUANT && p.c_tma && lane == 0) bulk_wait_all();   // my TMA stores are complete
+        if (!REQUANT && p.c_tma && lane == 0) bulk_wait_read();  // my TMA stores have read their slices; their writes complete with the grid
     }
 
     tc_fence_before();

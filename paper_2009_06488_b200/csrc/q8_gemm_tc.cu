@@ -463,7 +463,7 @@ gemm_u8_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (lane == 0) mbar_arrive_cluster(tempty_leader + 8u * (uint32_t)acc);
             asm volatile("bar.sync 1, 128;" ::: "memory");   // colterm_s is rewritten next tile
         }
-        if (p.c_tma && lane == 0) bulk_wait_all();   // my TMA stores are complete
+        if (p.c_tma && lane == 0) bulk_wait_read();  // my TMA stores have read their slices; their writes complete with the grid
     }
 
     tc_fence_before();
