@@ -43,7 +43,7 @@ FALLBACK_BF16_TFLOPS = 1590.0
 FALLBACK_HBM_GBS = 6650.0
 # ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel,
 # or None when no capture exists for the kernel as it stands (see profiles/).
-DOMINANT_KERNEL_TRAFFIC_BYTES = 342_500_000   # profiles/gemm_tc_pair_kernel.md, 8192^3 launch of the kernel as it stands
+DOMINANT_KERNEL_TRAFFIC_BYTES = 340_000_000   # profiles/gemm_tc_pair_kernel.md, 8192^3 launch of the kernel as it stands
 
 
 def measured_peaks():
