@@ -269,3 +269,72 @@ def test_which_layers_take_the_tensor_memory_kernel(q4, capfd):
     assert len(lines) == 3
     assert "tcgen05" in lines[0]
     assert "tcgen05" not in lines[1] and "tcgen05" not in lines[2]
+
+
+def _random_layers(count, seed):
+    """Seeded layer geometries: half of them from the tensor-memory kernels' layer classes with
+    enough rows for several tiles per CTA, half anything the entry points accept."""
+    rng = np.random.default_rng(seed)
+    out = []
+    while len(out) < count:
+        if len(out) % 2 == 0:
+            C = int(rng.choice([1, 8, 16, 32, 64])); OC = int(rng.choice([8, 16, 32, 64, 128]))
+            KH = KW = 3; s = int(rng.choice([1, 2])); p = 1
+            H = int(rng.choice([8, 12, 16, 24, 32])); W = H if rng.random() < 0.7 else int(rng.integers(6, 40))
+            Nb = int(rng.integers(1, 60)) if C * OC <= 512 else int(rng.integers(1, 8))
+        else:
+            C = int(rng.choice([1, 2, 3, 4, 8, 16, 24])); OC = int(rng.choice([2, 6, 8, 16, 24, 32, 72]))
+            KH = int(rng.choice([1, 2, 3, 5])); KW = KH if rng.random() < 0.7 else int(rng.choice([1, 2, 3]))
+            s = int(rng.choice([1, 1, 2])); p = int(rng.integers(0, (min(KH, KW) + 1) // 2 + 1))
+            H = int(rng.integers(max(KH, 4), 30)); W = int(rng.integers(max(KW, 4), 30))
+            Nb = int(rng.integers(1, 12))
+        if (Nb * H * W * C) % 2:
+            Nb += 1
+        if (Nb * H * W * C) % 2 == 0:
+            out.append((Nb, H, W, C, OC, KH, KW, s, s, p, p))
+    return out
+
+
+@pytest.mark.parametrize("g", _random_layers(28, 20260102))
+def test_random_layers_through_every_convolution_entry_point(q4, g):
+    """q4_conv2d (automatic choice and the explicit unroll + GEMM route), q4_conv2d_channels and,
+    where the layer has one, the prepared weight image: the oracle's bytes from each."""
+    import torch
+    Nb, H, W, C, OC, KH, KW, s, _, p, _ = g
+    dq, do = q4.ConvDesc(*g), oracle.ConvDesc(*g)
+    K = KH * KW * C
+    seed = 7000 + sum(g)
+    X = wl.rand_flat_nibbles(seed, 1, Nb * H * W * C)
+    Wt = wl.rand_packed(seed, 2, OC, K)
+    bias = wl.rand_ints(seed, 3, -400, 400, OC).astype(np.int32)
+    za, zb = 5, 11
+    rq = ((1 << 30) + 12345 * (seed % 97), 4 + seed % 5, 3, 1, 14)
+    want = oracle.conv2d(X, Wt, bias, do, za, zb, oracle.Requant(*rq))
+    Xd = torch.zeros((X.size + 31) // 16 * 16, dtype=torch.uint8, device="cuda")
+    Xd[:X.size] = dev(X)
+    ws = torch.full((max(q4.q4_conv2d_workspace_bytes(dq), 16),), 0xA5, dtype=torch.uint8, device="cuda")
+    try:
+        for variant in (0, 4):
+            q4.q4_set_variant(variant)
+            Y = torch.full((dq.M, OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
+            q4.q4_conv2d(Xd, dev(Wt), dq, za, zb, q4.Requant(*rq), Y, ws, dev(bias))
+            assert q4.q4_last_device_status() == q4.Q4_OK
+            assert (Y.cpu().numpy() == want).all(), variant
+    finally:
+        q4.q4_set_variant(0)
+    if q4.q4_conv2d_weights_bytes(dq):
+        check_prepared_weights(q4, Xd, Wt, dq, za, zb, rq, bias, None, want)
+    # per-channel weights: zero points, multipliers and shifts of their own
+    zbc = wl.rand_ints(seed, 4, 0, 15, OC).astype(np.int32)
+    mult = wl.rand_ints(seed, 5, 1 << 30, (1 << 31) - 1, OC).astype(np.int32)
+    shift = wl.rand_ints(seed, 6, 0 if seed % 3 == 0 else 2, 12, OC).astype(np.int32)
+    Ao, _ = oracle.im2col(X, do, za, (K + 1) // 2)
+    wantc = oracle.requant_channels(oracle.gemm_channels(Ao, Wt, dq.M, OC, K, za, zbc, bias), mult, shift, 2, 1, 14)
+    Y = torch.full((dq.M, OC // 2), 0xA5, dtype=torch.uint8, device="cuda")
+    try:
+        q4.q4_conv2d_channels(Xd, dev(Wt), dq, za, dev(zbc), dev(mult), dev(shift), 2, 1, 14, Y, dev(bias))
+    except q4.Q4Error as e:
+        assert e.status == q4.Q4_ERR_UNSUPPORTED      # layers the fused kernels do not take
+        return
+    assert q4.q4_last_device_status() == q4.Q4_OK
+    assert (Y.cpu().numpy() == wantc).all()
